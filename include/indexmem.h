@@ -1,0 +1,203 @@
+/*
+ * indexmem.h — C ABI of the IndexMem per-layer decode / chunked-prefill hot path for NVIDIA B200.
+ *
+ * The library keeps, for every (layer, sequence) pair, a budgeted KV cache, the indexer key cache,
+ * the pooled importance scores and the latent memory state (M, b), and advances them with two hot
+ * calls: im_prefill_chunk and im_decode_step.  Symbols follow the paper: H query heads, H_kv KV
+ * heads, d = d_head, D = d_model = H*d, D_kv = H_kv*d, G_q = H/H_kv, H_I = H_index, d_I = d_index,
+ * d_M = d_mem, B = KV budget B_max, tau = compression interval.
+ *
+ * Conventions for every entry point
+ *   - "dev" pointers are device (HBM) addresses owned by the caller; "host" pointers are ordinary
+ *     host memory.  Tensors are dense, row-major, innermost dimension last, 16-byte aligned.
+ *   - bf16 means the 16-bit brain-float bit pattern (upper half of an IEEE float32).
+ *   - The two hot calls only enqueue kernels on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream) and return without synchronising; they allocate nothing.  All calls
+ *     on one context must be issued in stream order on one stream at a time.
+ *   - Return value: IM_OK (0) or a negative im_error.  No exception, abort or device trap crosses the
+ *     boundary.  im_last_error() describes the most recent failure on the calling thread.  Problems
+ *     that only the device can see (for example a non-finite score) set a sticky device status word
+ *     that im_status() reads back.
+ *   - There is no CPU fallback: without a CUDA device every call that needs one fails with
+ *     IM_ERR_CUDA.
+ */
+#ifndef INDEXMEM_H_
+#define INDEXMEM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct im_ctx im_ctx; /* opaque host object; device state lives in the caller's workspace */
+
+typedef enum im_error {
+  IM_OK = 0,
+  IM_ERR_ARG = -1,      /* invalid argument or configuration                                  */
+  IM_ERR_CAPACITY = -2, /* a sequence would exceed its slot capacity, or workspace too small  */
+  IM_ERR_STATE = -3,    /* device status word is set (non-finite score, inconsistent count)   */
+  IM_ERR_CUDA = -4,     /* a CUDA runtime/driver call failed                                   */
+  IM_ERR_TIMEOUT = -5   /* a bounded device-side wait gave up                                  */
+} im_error;
+
+/* Hyper-parameters of the method.  Zero in a field marked "0 =>" selects the paper's value. */
+typedef struct im_config {
+  int32_t n_layers;          /* independent layers held by the context                              */
+  int32_t max_seqs;          /* sequence states per layer                                           */
+  int32_t n_q_heads;         /* H                                              (App. Notation)      */
+  int32_t n_kv_heads;        /* H_kv, divides H                                (App. Notation)      */
+  int32_t head_dim;          /* d, a multiple of 16, <= 256                    (App. Notation)      */
+  int32_t n_index_heads;     /* H_I ; 0 => max(1, H/4)                         (Sec. 4, hyperparameters) */
+  int32_t index_dim;         /* d_I ; 0 => max(1, d/8); <= 64                  (Sec. 4, hyperparameters) */
+  int32_t mem_dim;           /* d_M ; 0 => max(1, D/8)                         (Sec. 4, hyperparameters) */
+  int32_t budget;            /* B: entries kept by a compression, sinks included (Sec. 4, schedule) */
+  int32_t compress_interval; /* tau >= 1: decode tokens between compressions   (Sec. 4, schedule)   */
+  int32_t max_chunk;         /* longest prefill chunk; slot capacity is B + max(tau, max_chunk)     */
+  int32_t n_sink;            /* first tokens that are never evicted; < B       (Sec. 4, setup)      */
+  int32_t act;               /* indexer activation: 0 ReLU, 1 identity         (Sec. 3.1, z = act(q.k)) */
+  int32_t enable_memory;     /* 0: no memory write and no readout term         (Eq. 4 with g = 0)   */
+  int32_t out_f32;           /* 0: `out` of im_decode_step is bf16; 1: float32                       */
+  int32_t pending_slots;     /* rank-one writes folded lazily into M (0 => 16); see im_decode_step  */
+  float softmax_scale;       /* 0 => 1/sqrt(d)                                 (Sec. 2.1)           */
+  float lambda;              /* decay of Eq. 6-7, (0,1]; 0 => 1                                      */
+  float eta;                 /* write strength of Eq. 6-7, > 0; 0 => 1                               */
+  float eps;                 /* epsilon of Eq. 5; 0 => 1e-6                                          */
+  float norm_eps;            /* epsilon of the indexer RMSNorm; 0 => 1e-6     (Sec. 3.1)            */
+  float init_std;            /* std of the seeded weight init; 0 => 0.02                             */
+  uint64_t seed;             /* seed of the weight init done by im_create                            */
+} im_config;
+
+/* Weight tensors of one layer (Sec. 3.1 and 3.2), all bf16 except IM_W_BG (one float32). */
+typedef enum im_weight {
+  IM_W_UQ = 0,    /* U_q      [H_I*d_I, D]   indexer query down-projection           */
+  IM_W_UK = 1,    /* U_k      [d_I, D]       indexer key projection                  */
+  IM_W_G = 2,     /* G        [H_I, D]       head gate                               */
+  IM_W_THETA = 3, /* Linear_theta [d_M, D]   memory feature map phi                  */
+  IM_W_WG = 4,    /* w_g      [D]            weight of the scalar readout gate g(q)  */
+  IM_W_BG = 5     /* b_g      [1] float32    bias of g(q)                            */
+} im_weight;
+
+/* Per-(layer, sequence) state pieces for im_state_export / im_state_import. */
+typedef enum im_state {
+  IM_S_COUNTS = 0, /* int32[8]: n entries, tokens seen T, since, evict steps, n evicted by last compression, pending writes, 0, n_sel */
+  IM_S_POS = 1,    /* int32[n]          original position of the entry in each slot                   */
+  IM_S_IMP = 2,    /* float32[n]        pooled importance since the last compression (-inf = unscored) */
+  IM_S_KIDX = 3,   /* bf16[n, d_I]      cached indexer keys                                            */
+  IM_S_K = 4,      /* bf16[n, H_kv, d]  cached keys                                                    */
+  IM_S_V = 5,      /* bf16[n, H_kv, d]  cached values                                                  */
+  IM_S_M = 6,      /* float32[d_M, D_kv] latent state in KV space (export folds pending writes and decay in) */
+  IM_S_B = 7,      /* float32[d_M]      stabiliser vector b                                            */
+  IM_S_EVICTED = 8, /* int32[n_evicted] positions evicted by the last compression, ascending (export only) */
+  IM_S_SEL_POS = 9, /* int32[n_sel]     positions of the entries the last compression chose among (export only) */
+  IM_S_SEL_IMP = 10 /* float32[n_sel]   their pooled importance at that moment, same order (export only)        */
+} im_state;
+
+/* Bytes of device workspace im_create needs for `cfg`; 0 if the configuration is invalid. */
+size_t im_workspace_bytes(const im_config* cfg);
+
+/*
+ * Creates a context over `dev_workspace` (device memory of at least im_workspace_bytes(cfg) bytes,
+ * 256-byte aligned, owned by the caller, must outlive the context and the current CUDA device must
+ * be the one that owns it).  Zeroes the state, draws seeded N(0, init_std^2) bf16 weights for every
+ * layer (b_g = 0) and synchronises the device once.  On success *out receives the context.
+ */
+int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes, im_ctx** out);
+
+/* Releases the host object.  The workspace stays with the caller.  Synchronises the device. */
+int im_destroy(im_ctx* ctx);
+
+/* Clears the state of one sequence in one layer (layer = -1: all layers; seq = -1: all sequences). Enqueued on the stream. */
+int im_reset(im_ctx* ctx, int layer, int seq, void* cuda_stream);
+
+/*
+ * Chunked prefill of one layer for n_seq sequences (Sec. 4 schedule: ingest, score with every query
+ * of the chunk, compress to the budget, write the evicted pairs to memory; Sec. 3.1; Eq. 6-7).
+ *   seq_ids  host int32[n_seq], distinct, each in [0, max_seqs)
+ *   chunk_len C, 1 <= C <= max_chunk; the same for all sequences of the call
+ *   x        dev bf16 [n_seq, C, D]       hidden states X
+ *   q_pre    dev bf16 [n_seq, C, H, d]    pre-RoPE queries Q (indexer input)
+ *   k, v     dev bf16 [n_seq, C, H_kv, d] keys / values to cache
+ * Appends the C tokens, pools A_{s,t} (Sec. 3.1) over the chunk's queries under the causal mask into
+ * the importance of every cached entry, then compresses: if more than B entries are cached the B
+ * best (importance descending, position ascending, sinks first) stay, the rest are written to the
+ * latent memory (Eq. 6-7, one evict step) and the cache is compacted.  Attention outputs for the
+ * chunk's own queries are not produced.
+ * Errors: IM_ERR_ARG (bad ids, sizes, null pointers), IM_ERR_CAPACITY (n + C > capacity).
+ */
+int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, int chunk_len,
+                     const void* x, const void* q_pre, const void* k, const void* v, void* cuda_stream);
+
+/*
+ * One decode token per sequence for one layer (Sec. 4 schedule, decode side; Eq. 4-7).
+ *   x      dev bf16 [n_seq, D]        hidden state of the new token
+ *   q_pre  dev bf16 [n_seq, H, d]     pre-RoPE query (indexer input); may alias q
+ *   q      dev bf16 [n_seq, H, d]     attention query; also the input of Linear_theta and g
+ *   k_new, v_new dev bf16 [n_seq, H_kv, d]
+ *   out    dev [n_seq, H, d] bf16 (float32 when out_f32 = 1): o = o_attn + g(q) m(q)   (Eq. 4)
+ * Steps: append the token; score every cached entry with the new query and pool by max into its
+ * importance; every tau-th token of a sequence compress to the budget as in im_prefill_chunk; then
+ * attention over the retained entries plus the gated memory readout (Eq. 5).  The evict step happens
+ * before the attention of the same call.
+ * A compression that evicts at most `pending_slots` entries keeps them as rank-one terms next to M
+ * and the readout adds them exactly; they are folded into M when the list fills.  This is Eq. 6-7
+ * re-associated, not an approximation.
+ * Errors: IM_ERR_ARG, IM_ERR_CAPACITY (a sequence has no free slot).
+ */
+int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, const void* x,
+                   const void* q_pre, const void* q, const void* k_new, const void* v_new, void* out,
+                   void* cuda_stream);
+
+/* Copies one weight tensor of a layer from / to host memory (bytes must equal the tensor size). Synchronous. */
+int im_set_weights(im_ctx* ctx, int layer, int which, const void* host_buf, size_t bytes);
+int im_get_weights(im_ctx* ctx, int layer, int which, void* host_buf, size_t bytes);
+
+/*
+ * Copies one piece of a sequence's state to / from host memory.  Synchronous (device-wide).
+ * Export: `bytes` is the buffer capacity; the piece is sized by the current entry count n.
+ * Import: IM_S_COUNTS first fixes n, then the other pieces must have exactly the matching size;
+ * importing IM_S_M replaces the latent state (pending writes are dropped, decay scale reset).
+ * Slot order is free: entries are identified by their position.
+ */
+int im_state_export(im_ctx* ctx, int layer, int seq, int which, void* host_buf, size_t bytes);
+int im_state_import(im_ctx* ctx, int layer, int seq, int which, const void* host_buf, size_t bytes);
+
+/*
+ * Row-generic budgeted selection (Sec. 2.2: I = TopK(S, L')), usable without a context.
+ *   scores dev float32 [rows, n], pos dev int32 [rows, n] (distinct within a row)
+ *   keep   dev uint8  [rows, n]  receives 1 for the min(B, n) retained entries of each row
+ *   n_evict dev int32 [rows]     receives n - min(B, n)
+ * Order: key descending, position ascending, where key = +inf for pos < n_sink and -0.0 == +0.0.
+ * Bit-exact and deterministic.  Scores must not be NaN.
+ */
+int im_topb_select(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,
+                   uint8_t* keep, int32_t* n_evict, void* cuda_stream);
+
+/* Synchronises the stream and returns the sticky device status word (0 = clean) in *device_status. */
+int im_status(im_ctx* ctx, void* cuda_stream, int32_t* device_status);
+
+/*
+ * Measurement hook (no counterpart in the paper): between im_profile_begin and im_profile_end every
+ * im_decode_step records a pair of CUDA events on its stream around the attention + readout kernel
+ * (the kernel that streams the retained K/V and M).  im_profile_end synchronises, returns the summed
+ * device time of the recorded launches in *total_ms and their number in *n_records, and releases the
+ * events.  At most max_records launches are recorded.  Must not be used while the stream is being
+ * captured into a CUDA graph.
+ */
+int im_profile_begin(im_ctx* ctx, int max_records);
+int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
+
+/* Number of kernels this library has launched on behalf of `ctx` since im_create. */
+int64_t im_launch_count(im_ctx* ctx);
+
+/* Resolved configuration (defaults filled in) and slot capacity per sequence. */
+int im_get_config(im_ctx* ctx, im_config* out, int32_t* capacity);
+
+/* Thread-local description of the last error returned on this thread ("" if none). */
+const char* im_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* INDEXMEM_H_ */

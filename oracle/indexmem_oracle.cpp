@@ -83,6 +83,8 @@ struct Seq {
   int64_t T = 0;               // tokens appended so far (next position)
   int32_t since = 0;           // decode tokens since the last compression
   std::vector<int32_t> last_evicted;   // positions evicted by the latest COMPRESS, ascending
+  std::vector<int32_t> sel_pos;        // what the latest COMPRESS chose among: positions ...
+  std::vector<float> sel_acc;          // ... and pooled importance (cache order)
   int64_t n_evict_steps = 0;
 };
 
@@ -258,6 +260,9 @@ void compress(const Layer& L, Seq& S) {
   S.since = 0;
   S.last_evicted.clear();
   const int n = (int)S.R.size();
+  S.sel_pos.resize(n);
+  S.sel_acc.resize(n);
+  for (int i = 0; i < n; ++i) { S.sel_pos[i] = S.R[i].pos; S.sel_acc[i] = S.R[i].acc; }
   if (n > L.c.B) {
     std::vector<float> sc(n);
     std::vector<int32_t> ps(n);
@@ -446,6 +451,13 @@ int orc_last_evicted(void* h, int seq, int32_t* pos, int cap) {
   Seq& S = static_cast<Layer*>(h)->seqs[seq];
   int n = (int)S.last_evicted.size();
   for (int i = 0; i < n && i < cap; ++i) pos[i] = S.last_evicted[i];
+  return n;
+}
+
+int orc_last_selection(void* h, int seq, int32_t* pos, float* acc, int cap) {
+  Seq& S = static_cast<Layer*>(h)->seqs[seq];
+  int n = (int)S.sel_pos.size();
+  for (int i = 0; i < n && i < cap; ++i) { pos[i] = S.sel_pos[i]; acc[i] = S.sel_acc[i]; }
   return n;
 }
 

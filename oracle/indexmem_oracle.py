@@ -101,6 +101,7 @@ def _load():
     L.orc_export_entries.argtypes = [vp, C.c_int, vp, vp, vp, vp, vp]
     L.orc_export_memory.argtypes = [vp, C.c_int, vp, vp]
     L.orc_last_evicted.argtypes = [vp, C.c_int, vp, C.c_int]
+    L.orc_last_selection.argtypes = [vp, C.c_int, vp, vp, C.c_int]
     L.orc_index_key.argtypes = [vp, vp, vp]
     L.orc_index_query.argtypes = [vp, vp, vp, vp, vp]
     L.orc_index_scores.argtypes = [vp, vp, vp, vp, C.c_int, vp]
@@ -242,6 +243,14 @@ class OracleLayer:
         buf = np.empty(cap, np.int32)
         n = self.lib.orc_last_evicted(self.h, seq, _p(buf), cap)
         return buf[:n]
+
+    def last_selection(self, seq=0):
+        """(pos int32[n], acc float32[n]) of the entries the latest compression chose among."""
+        n = self.lib.orc_last_selection(self.h, seq, None, None, 0)
+        pos = np.empty(max(n, 1), np.int32)
+        acc = np.empty(max(n, 1), np.float32)
+        self.lib.orc_last_selection(self.h, seq, _p(pos), _p(acc), n)
+        return pos[:n], acc[:n]
 
     # ---- stage functions
     def index_key(self, x) -> np.ndarray:

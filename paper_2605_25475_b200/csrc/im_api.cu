@@ -1,0 +1,695 @@
+// Host side of libindexmem: configuration, workspace layout, the C ABI and the order of the
+// kernels inside the two hot calls.  Every step of the path runs in the kernels of the other
+// translation units; nothing here computes on the CPU except argument checks, host mirrors of the
+// per-sequence counters (they are deterministic functions of the call history) and the
+// non-hot-path state export/import.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "im_internal.cuh"
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+#define CK(call)                                                                              \
+  do {                                                                                        \
+    cudaError_t e_ = (call);                                                                  \
+    if (e_ != cudaSuccess) return fail(IM_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  ImState st;
+  ImScratch sc;
+  std::vector<ImWeights> w;
+  size_t state_begin, state_end;  // byte range holding per-unit state (zeroed at create)
+  size_t total;
+};
+
+bool resolve(const im_config* in, im_config* c, ImDims* p) {
+  if (!in) return false;
+  *c = *in;
+  if (c->n_layers < 1 || c->max_seqs < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  if (c->head_dim < 16 || c->head_dim % 16 || c->head_dim > 256) return false;
+  if (c->n_index_heads == 0) c->n_index_heads = std::max(1, c->n_q_heads / 4);
+  if (c->index_dim == 0) c->index_dim = std::max(1, c->head_dim / 8);
+  if (c->mem_dim == 0) c->mem_dim = std::max(1, c->n_q_heads * c->head_dim / 8);
+  if (c->n_index_heads < 1 || c->n_index_heads > 64 || c->index_dim < 1 || c->index_dim > 64) return false;
+  if (c->mem_dim < 1) return false;
+  if (c->compress_interval < 1) return false;
+  if (c->max_chunk < 0) return false;
+  if (c->n_sink < 0 || c->budget <= c->n_sink || c->budget < 1) return false;
+  if (c->act != 0 && c->act != 1) return false;
+  if (c->pending_slots == 0) c->pending_slots = 16;
+  if (c->pending_slots < 1 || c->pending_slots > 64) return false;
+  if (c->softmax_scale == 0.f) c->softmax_scale = 1.0f / sqrtf((float)c->head_dim);
+  if (c->lambda == 0.f) c->lambda = 1.f;
+  if (c->eta == 0.f) c->eta = 1.f;
+  if (c->eps == 0.f) c->eps = 1e-6f;
+  if (c->norm_eps == 0.f) c->norm_eps = 1e-6f;
+  if (c->init_std == 0.f) c->init_std = 0.02f;
+  if (!(c->lambda > 0.f && c->lambda <= 1.f) || !(c->eta > 0.f) || !(c->eps > 0.f)) return false;
+  long long cap = (long long)c->budget + std::max(c->compress_interval, std::max(c->max_chunk, 1));
+  cap = (cap + IM_SLOT_ALIGN - 1) / IM_SLOT_ALIGN * IM_SLOT_ALIGN;
+  if (cap > (1ll << 30)) return false;
+  ImDims& q = *p;
+  q.L = c->n_layers; q.S = c->max_seqs;
+  q.H = c->n_q_heads; q.Hkv = c->n_kv_heads; q.d = c->head_dim;
+  q.D = q.H * q.d; q.Dkv = q.Hkv * q.d; q.Gq = q.H / q.Hkv;
+  q.HI = c->n_index_heads; q.dI = c->index_dim; q.dM = c->mem_dim;
+  q.B = c->budget; q.tau = c->compress_interval; q.cap = (int)cap; q.tail = q.cap - q.B;
+  q.n_sink = c->n_sink; q.act = c->act; q.mem = c->enable_memory ? 1 : 0; q.F = c->pending_slots;
+  q.out_f32 = c->out_f32 ? 1 : 0; q.max_chunk = std::max(c->max_chunk, 1);
+  q.R3 = q.HI * q.dI + q.dI + q.HI;
+  q.R5 = q.R3 + q.dM + 1;
+  q.max_splits = (q.cap + 255) / 256;
+  q.scale = c->softmax_scale; q.lambda = c->lambda; q.eta = c->eta; q.eps = c->eps; q.norm_eps = c->norm_eps;
+  if (q.Gq > 16) return false;
+  return true;
+}
+
+// Carves the workspace.  base == nullptr: only sizes are computed.
+void carve(const ImDims& p, char* base, Layout* lo) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> char* {
+    off = align_up(off, 256);
+    char* ptr = base ? base + off : nullptr;
+    off += bytes;
+    return ptr;
+  };
+  const size_t U = (size_t)p.L * p.S;
+  lo->state_begin = 0;
+  lo->st.Kc = (bf16*)take(U * p.Hkv * p.cap * p.d * 2);
+  lo->st.Vc = (bf16*)take(U * p.Hkv * p.cap * p.d * 2);
+  lo->st.kidx = (bf16*)take(U * p.cap * p.dI * 2);
+  lo->st.pos = (int32_t*)take(U * p.cap * 4);
+  lo->st.imp = (float*)take(U * p.cap * 4);
+  lo->st.keep = (uint8_t*)take(U * p.cap);
+  lo->st.sel_pos = (int32_t*)take(U * p.cap * 4);
+  lo->st.sel_imp = (float*)take(U * p.cap * 4);
+  lo->st.ev_slot = (int32_t*)take(U * p.tail * 4);
+  lo->st.ev_pos = (int32_t*)take(U * p.tail * 4);
+  lo->st.Mhat = (float*)take(U * p.dM * p.Dkv * 4);
+  lo->st.bvec = (float*)take(U * p.dM * 4);
+  lo->st.cscale = (float*)take(U * 4);
+  lo->st.pend_phi = (float*)take(U * p.F * p.dM * 4);
+  lo->st.pend_v = (bf16*)take(U * p.F * p.Dkv * 2);
+  lo->st.pend_w = (float*)take(U * p.F * 4);
+  lo->st.ctr = (int32_t*)take(U * CTR_STRIDE * 4);
+  lo->st.status = (int32_t*)take(256);
+  lo->state_end = off;
+  lo->w.resize(p.L);
+  for (int l = 0; l < p.L; ++l) {
+    ImWeights& w = lo->w[l];
+    w.Uq = (bf16*)take((size_t)p.HI * p.dI * p.D * 2);
+    w.Uk = (bf16*)take((size_t)p.dI * p.D * 2);
+    w.G = (bf16*)take((size_t)p.HI * p.D * 2);
+    w.Wt = (bf16*)take((size_t)p.dM * p.D * 2);
+    w.wg = (bf16*)take((size_t)p.D * 2);
+    w.bg = (float*)take(256);
+    w.Wfold = (float*)take((size_t)p.dM * p.Dkv * 4);
+  }
+  lo->sc.raw = (float*)take((size_t)p.S * p.max_chunk * p.R5 * 4);
+  lo->sc.kidx_new = (bf16*)take((size_t)p.S * p.max_chunk * p.dI * 2);
+  lo->sc.phi = (float*)take((size_t)p.S * p.tail * p.dM * 4);
+  lo->sc.moves = (int32_t*)take((size_t)p.S * 2 * p.tail * 4);
+  lo->sc.part = (float*)take((size_t)p.S * p.H * p.max_splits * (p.d + 2) * 4);
+  lo->total = align_up(off, 256);
+}
+
+struct HostUnit {
+  int n = 0;       // cached entries
+  long long T = 0; // tokens seen
+  int since = 0;   // decode tokens since the last compression
+  int npend = 0;   // pending rank-one writes
+};
+
+}  // namespace
+
+struct im_ctx {
+  im_config cfg;
+  ImDims p;
+  Layout lo;
+  std::vector<HostUnit> hu;
+  int64_t launches = 0;
+  int device = 0;
+  std::vector<cudaEvent_t> prof_ev;  // pairs (start, stop)
+  size_t prof_used = 0;              // events recorded so far
+};
+
+namespace {
+
+ImLaunch make_launch(im_ctx* ctx, int layer, cudaStream_t s) {
+  ImLaunch L;
+  L.p = ctx->p;
+  L.st = ctx->lo.st;
+  L.w = ctx->lo.w[layer];
+  L.sc = ctx->lo.sc;
+  L.stream = s;
+  L.launches = &ctx->launches;
+  return L;
+}
+
+int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall* call) {
+  if (!ctx) return fail(IM_ERR_ARG, "null context");
+  if (layer < 0 || layer >= ctx->p.L) return fail(IM_ERR_ARG, "layer %d out of range [0,%d)", layer, ctx->p.L);
+  if (n_seq < 1 || n_seq > ctx->p.S || n_seq > IM_MAX_CALL_SEQS)
+    return fail(IM_ERR_ARG, "n_seq %d out of range [1,%d]", n_seq, std::min(ctx->p.S, IM_MAX_CALL_SEQS));
+  if (!seq_ids) return fail(IM_ERR_ARG, "null seq_ids");
+  std::vector<char> seen(ctx->p.S, 0);
+  for (int i = 0; i < n_seq; ++i) {
+    int s = seq_ids[i];
+    if (s < 0 || s >= ctx->p.S) return fail(IM_ERR_ARG, "seq id %d out of range [0,%d)", s, ctx->p.S);
+    if (seen[s]) return fail(IM_ERR_ARG, "seq id %d repeated in one call", s);
+    seen[s] = 1;
+    call->seq[i] = s;
+  }
+  call->layer = layer;
+  call->n_seq = n_seq;
+  call->C = 1;
+  return IM_OK;
+}
+
+#define CKL(call)                                                                                 \
+  do {                                                                                            \
+    cudaError_t e_ = (call);                                                                      \
+    if (e_ != cudaSuccess) return fail(IM_ERR_CUDA, "launch %s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+// The evict step shared by both hot calls: select -> memory write -> compaction, for the sequences
+// of `call` whose host mirror says they are over budget (others are skipped on the device).
+int run_compress(im_ctx* ctx, const ImLaunch& L, const ImCall& call) {
+  const ImDims& p = ctx->p;
+  int ne_max = 0;
+  // The fold kernel is always enqueued (its blocks leave at once unless the device flags the step
+  // as a fold), so that a captured sequence of launches stays valid for every later step.
+  const bool direct = true;
+  for (int i = 0; i < call.n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)call.layer * p.S + call.seq[i]];
+    ne_max = std::max(ne_max, std::max(0, u.n - p.B));
+  }
+  CKL(im_launch_select(L, call));  // also restarts the pooling of every sequence in the call
+  if (ne_max > 0) {
+    if (p.mem) CKL(im_launch_memory_write(L, call, ne_max, direct));
+    CKL(im_launch_compact(L, call));
+  }
+  for (int i = 0; i < call.n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)call.layer * p.S + call.seq[i]];
+    int ne = std::max(0, u.n - p.B);
+    if (ne > 0) {
+      if (p.mem) {
+        // the device takes the same decision per sequence: fold everything when the list overflows
+        if (u.npend + ne > p.F) u.npend = 0; else u.npend += ne;
+      }
+      u.n = p.B;
+    }
+    u.since = 0;
+  }
+  return IM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* im_last_error(void) { return g_err; }
+
+size_t im_workspace_bytes(const im_config* cfg) {
+  im_config c;
+  ImDims p;
+  if (!resolve(cfg, &c, &p)) return 0;
+  Layout lo;
+  carve(p, nullptr, &lo);
+  return lo.total;
+}
+
+int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes, im_ctx** out) {
+  if (!out) return fail(IM_ERR_ARG, "null out");
+  *out = nullptr;
+  im_config c;
+  ImDims p;
+  if (!resolve(cfg, &c, &p)) return fail(IM_ERR_ARG, "invalid configuration");
+  if (!dev_workspace || ((uintptr_t)dev_workspace & 255)) return fail(IM_ERR_ARG, "workspace null or not 256-byte aligned");
+  im_ctx* ctx = new (std::nothrow) im_ctx();
+  if (!ctx) return fail(IM_ERR_ARG, "out of host memory");
+  ctx->cfg = c;
+  ctx->p = p;
+  carve(p, (char*)dev_workspace, &ctx->lo);
+  if (ctx->lo.total > workspace_bytes) {
+    size_t need = ctx->lo.total;
+    delete ctx;
+    return fail(IM_ERR_CAPACITY, "workspace too small: need %zu bytes, got %zu", need, workspace_bytes);
+  }
+  ctx->hu.assign((size_t)p.L * p.S, HostUnit());
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e == cudaSuccess)
+    e = cudaMemsetAsync((char*)dev_workspace + ctx->lo.state_begin, 0, ctx->lo.state_end - ctx->lo.state_begin, 0);
+  // cscale = 1 for every unit
+  if (e == cudaSuccess) {
+    std::vector<float> ones((size_t)p.L * p.S, 1.0f);
+    e = cudaMemcpy(ctx->lo.st.cscale, ones.data(), ones.size() * 4, cudaMemcpyHostToDevice);
+  }
+  for (int l = 0; l < p.L && e == cudaSuccess; ++l) {
+    e = im_launch_init_weights(p, ctx->lo.w[l], l, c.seed, c.init_std, 0);
+    if (e == cudaSuccess) e = im_launch_fold_theta(p, ctx->lo.w[l], 0);
+  }
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    delete ctx;
+    return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
+  }
+  *out = ctx;
+  return IM_OK;
+}
+
+int im_destroy(im_ctx* ctx) {
+  if (!ctx) return fail(IM_ERR_ARG, "null context");
+  cudaError_t e = cudaDeviceSynchronize();
+  delete ctx;
+  if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
+  return IM_OK;
+}
+
+int im_get_config(im_ctx* ctx, im_config* out, int32_t* capacity) {
+  if (!ctx) return fail(IM_ERR_ARG, "null context");
+  if (out) *out = ctx->cfg;
+  if (capacity) *capacity = ctx->p.cap;
+  return IM_OK;
+}
+
+int64_t im_launch_count(im_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int im_reset(im_ctx* ctx, int layer, int seq, void* cuda_stream) {
+  if (!ctx) return fail(IM_ERR_ARG, "null context");
+  const ImDims& p = ctx->p;
+  if (layer < -1 || layer >= p.L || seq < -1 || seq >= p.S) return fail(IM_ERR_ARG, "layer/seq out of range");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  for (int l = 0; l < p.L; ++l) {
+    if (layer >= 0 && l != layer) continue;
+    for (int q = 0; q < p.S; ++q) {
+      if (seq >= 0 && q != seq) continue;
+      size_t u = (size_t)l * p.S + q;
+      ImState& st = ctx->lo.st;
+      CK(cudaMemsetAsync(st.ctr + u * CTR_STRIDE, 0, CTR_STRIDE * 4, s));
+      CK(cudaMemsetAsync(st.Mhat + u * p.dM * p.Dkv, 0, (size_t)p.dM * p.Dkv * 4, s));
+      CK(cudaMemsetAsync(st.bvec + u * p.dM, 0, (size_t)p.dM * 4, s));
+      // 1.0f as a byte pattern cannot be produced by memset: use a 4-byte copy from a static
+      static const float one = 1.0f;
+      CK(cudaMemcpyAsync(st.cscale + u, &one, 4, cudaMemcpyHostToDevice, s));
+      ctx->hu[u] = HostUnit();
+    }
+  }
+  return IM_OK;
+}
+
+int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, int chunk_len, const void* x,
+                     const void* q_pre, const void* k, const void* v, void* cuda_stream) {
+  ImCall call;
+  int rc = check_call(ctx, layer, n_seq, seq_ids, &call);
+  if (rc) return rc;
+  const ImDims& p = ctx->p;
+  if (chunk_len < 1 || chunk_len > p.max_chunk)
+    return fail(IM_ERR_ARG, "chunk_len %d out of range [1,%d]", chunk_len, p.max_chunk);
+  if (!x || !q_pre || !k || !v) return fail(IM_ERR_ARG, "null tensor");
+  int n_max = 0;
+  for (int i = 0; i < n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    if (u.n + chunk_len > p.cap)
+      return fail(IM_ERR_CAPACITY, "sequence %d: %d cached + chunk %d exceeds capacity %d", call.seq[i], u.n, chunk_len, p.cap);
+    n_max = std::max(n_max, u.n + chunk_len);
+  }
+  call.C = chunk_len;
+  ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
+  // a0: indexer projections of every chunk token (Sec. 3.1)
+  ImProjJobs jobs;
+  memset(&jobs, 0, sizeof(jobs));
+  ImRows r = im_rows(p);
+  jobs.job[0] = {L.w.Uq, (const bf16*)q_pre, p.HI * p.dI, r.uq};
+  jobs.job[1] = {L.w.G, (const bf16*)x, p.HI, r.g};
+  jobs.n_jobs = 2;
+  jobs.Dn = p.D;
+  jobs.NV = n_seq * chunk_len;
+  jobs.out_stride = p.R3;
+  jobs.total_rows = 0;
+  for (int j = 0; j < jobs.n_jobs; ++j) jobs.total_rows += jobs.job[j].rows;
+  CKL(im_launch_proj(L, jobs, L.sc.raw));
+  CKL(im_launch_proj_key(L, x, n_seq * chunk_len));
+  CKL(im_launch_prefill_append(L, call, k, v));
+  // a1: pooled importance under the causal mask
+  CKL(im_launch_prefill_score(L, call, n_max));
+  for (int i = 0; i < n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    u.n += chunk_len;
+    u.T += chunk_len;
+  }
+  // a2-a4
+  return run_compress(ctx, L, call);
+}
+
+int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, const void* x, const void* q_pre,
+                   const void* q, const void* k_new, const void* v_new, void* out, void* cuda_stream) {
+  ImCall call;
+  int rc = check_call(ctx, layer, n_seq, seq_ids, &call);
+  if (rc) return rc;
+  const ImDims& p = ctx->p;
+  if (!x || !q_pre || !q || !k_new || !v_new || !out) return fail(IM_ERR_ARG, "null tensor");
+  bool due_any = false, due_all = true;
+  for (int i = 0; i < n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    if (u.n + 1 > p.cap) return fail(IM_ERR_CAPACITY, "sequence %d has no free slot (capacity %d)", call.seq[i], p.cap);
+    bool due = (u.since + 1 == p.tau);
+    due_any |= due;
+    due_all &= due;
+  }
+  if (due_any != due_all)
+    return fail(IM_ERR_ARG, "sequences of one decode call must be at the same phase of the compression interval");
+  ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
+  // a0: projections (Sec. 3.1 features, phi(q) of Eq. 5, gate of Eq. 4)
+  ImProjJobs jobs;
+  memset(&jobs, 0, sizeof(jobs));
+  ImRows r = im_rows(p);
+  jobs.job[0] = {L.w.Uq, (const bf16*)q_pre, p.HI * p.dI, r.uq};
+  jobs.job[1] = {L.w.G, (const bf16*)x, p.HI, r.g};
+  jobs.job[2] = {L.w.Wt, (const bf16*)q, p.dM, r.theta};
+  jobs.job[3] = {L.w.wg, (const bf16*)q, 1, r.wg};
+  jobs.n_jobs = p.mem ? 4 : 2;
+  jobs.Dn = p.D;
+  jobs.NV = n_seq;
+  jobs.out_stride = p.R5;
+  jobs.total_rows = 0;
+  for (int j = 0; j < jobs.n_jobs; ++j) jobs.total_rows += jobs.job[j].rows;
+  CKL(im_launch_proj(L, jobs, L.sc.raw));
+  CKL(im_launch_proj_key(L, x, n_seq));
+  // append + a1: score every cached entry with the new query
+  CKL(im_launch_decode_index(L, call, k_new, v_new));
+  int n_max = 0;
+  for (int i = 0; i < n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    u.n += 1;
+    u.T += 1;
+    u.since += 1;
+  }
+  // a2-a4 every tau-th token
+  if (due_all) {
+    rc = run_compress(ctx, L, call);
+    if (rc) return rc;
+  }
+  for (int i = 0; i < n_seq; ++i) n_max = std::max(n_max, ctx->hu[(size_t)layer * p.S + call.seq[i]].n);
+  // a5-a6: attention over the retained entries + gated readout
+  const bool prof = ctx->prof_used + 2 <= ctx->prof_ev.size();
+  if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], L.stream));
+  CKL(im_launch_attention(L, call, q, out, n_max));
+  if (prof) {
+    CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], L.stream));
+    ctx->prof_used += 2;
+  }
+  return IM_OK;
+}
+
+int im_profile_begin(im_ctx* ctx, int max_records) {
+  if (!ctx || max_records < 1 || max_records > (1 << 20)) return fail(IM_ERR_ARG, "bad profile request");
+  if (!ctx->prof_ev.empty()) return fail(IM_ERR_STATE, "profiling already active");
+  ctx->prof_ev.resize((size_t)max_records * 2);
+  ctx->prof_used = 0;
+  for (auto& e : ctx->prof_ev) {
+    cudaError_t rc = cudaEventCreate(&e);
+    if (rc != cudaSuccess) {
+      ctx->prof_ev.clear();
+      return fail(IM_ERR_CUDA, "cudaEventCreate: %s", cudaGetErrorString(rc));
+    }
+  }
+  return IM_OK;
+}
+
+int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records) {
+  if (!ctx || !total_ms || !n_records) return fail(IM_ERR_ARG, "null argument");
+  *total_ms = 0.0;
+  *n_records = 0;
+  if (ctx->prof_ev.empty()) return fail(IM_ERR_STATE, "profiling not active");
+  cudaError_t rc = cudaDeviceSynchronize();
+  for (size_t i = 0; i + 1 < ctx->prof_used && rc == cudaSuccess; i += 2) {
+    float ms = 0.f;
+    rc = cudaEventElapsedTime(&ms, ctx->prof_ev[i], ctx->prof_ev[i + 1]);
+    *total_ms += ms;
+    *n_records += 1;
+  }
+  for (auto& e : ctx->prof_ev) cudaEventDestroy(e);
+  ctx->prof_ev.clear();
+  ctx->prof_used = 0;
+  if (rc != cudaSuccess) return fail(IM_ERR_CUDA, "im_profile_end: %s", cudaGetErrorString(rc));
+  return IM_OK;
+}
+
+static size_t weight_bytes(const ImDims& p, int which) {
+  switch (which) {
+    case IM_W_UQ: return (size_t)p.HI * p.dI * p.D * 2;
+    case IM_W_UK: return (size_t)p.dI * p.D * 2;
+    case IM_W_G: return (size_t)p.HI * p.D * 2;
+    case IM_W_THETA: return (size_t)p.dM * p.D * 2;
+    case IM_W_WG: return (size_t)p.D * 2;
+    case IM_W_BG: return 4;
+    default: return 0;
+  }
+}
+static void* weight_ptr(const ImWeights& w, int which) {
+  switch (which) {
+    case IM_W_UQ: return w.Uq;
+    case IM_W_UK: return w.Uk;
+    case IM_W_G: return w.G;
+    case IM_W_THETA: return w.Wt;
+    case IM_W_WG: return w.wg;
+    case IM_W_BG: return w.bg;
+    default: return nullptr;
+  }
+}
+
+int im_set_weights(im_ctx* ctx, int layer, int which, const void* host_buf, size_t bytes) {
+  if (!ctx || !host_buf) return fail(IM_ERR_ARG, "null argument");
+  if (layer < 0 || layer >= ctx->p.L) return fail(IM_ERR_ARG, "layer out of range");
+  size_t want = weight_bytes(ctx->p, which);
+  if (want == 0 || want != bytes) return fail(IM_ERR_ARG, "weight %d: expected %zu bytes, got %zu", which, want, bytes);
+  CK(cudaDeviceSynchronize());
+  CK(cudaMemcpy(weight_ptr(ctx->lo.w[layer], which), host_buf, bytes, cudaMemcpyHostToDevice));
+  if (which == IM_W_THETA) {
+    CKL(im_launch_fold_theta(ctx->p, ctx->lo.w[layer], 0));
+    CK(cudaDeviceSynchronize());
+  }
+  return IM_OK;
+}
+
+int im_get_weights(im_ctx* ctx, int layer, int which, void* host_buf, size_t bytes) {
+  if (!ctx || !host_buf) return fail(IM_ERR_ARG, "null argument");
+  if (layer < 0 || layer >= ctx->p.L) return fail(IM_ERR_ARG, "layer out of range");
+  size_t want = weight_bytes(ctx->p, which);
+  if (want == 0 || want != bytes) return fail(IM_ERR_ARG, "weight %d: expected %zu bytes, got %zu", which, want, bytes);
+  CK(cudaDeviceSynchronize());
+  CK(cudaMemcpy(host_buf, weight_ptr(ctx->lo.w[layer], which), bytes, cudaMemcpyDeviceToHost));
+  return IM_OK;
+}
+
+int im_state_export(im_ctx* ctx, int layer, int seq, int which, void* host_buf, size_t bytes) {
+  if (!ctx || !host_buf) return fail(IM_ERR_ARG, "null argument");
+  const ImDims& p = ctx->p;
+  if (layer < 0 || layer >= p.L || seq < 0 || seq >= p.S) return fail(IM_ERR_ARG, "layer/seq out of range");
+  CK(cudaDeviceSynchronize());
+  const size_t u = (size_t)layer * p.S + seq;
+  const ImState& st = ctx->lo.st;
+  int32_t ctr[CTR_STRIDE];
+  CK(cudaMemcpy(ctr, st.ctr + u * CTR_STRIDE, sizeof(ctr), cudaMemcpyDeviceToHost));
+  const int n = ctr[CTR_N];
+  if (n < 0 || n > p.cap) return fail(IM_ERR_STATE, "device entry count %d outside [0,%d]", n, p.cap);
+  auto need = [&](size_t want) -> int {
+    if (bytes < want) return fail(IM_ERR_ARG, "state %d: buffer of %zu bytes, need %zu", which, bytes, want);
+    return IM_OK;
+  };
+  int rc;
+  switch (which) {
+    case IM_S_COUNTS:
+      if ((rc = need(sizeof(ctr)))) return rc;
+      memcpy(host_buf, ctr, sizeof(ctr));
+      return IM_OK;
+    case IM_S_POS:
+      if ((rc = need((size_t)n * 4))) return rc;
+      CK(cudaMemcpy(host_buf, st.pos + u * p.cap, (size_t)n * 4, cudaMemcpyDeviceToHost));
+      return IM_OK;
+    case IM_S_IMP:
+      if ((rc = need((size_t)n * 4))) return rc;
+      CK(cudaMemcpy(host_buf, st.imp + u * p.cap, (size_t)n * 4, cudaMemcpyDeviceToHost));
+      return IM_OK;
+    case IM_S_KIDX:
+      if ((rc = need((size_t)n * p.dI * 2))) return rc;
+      CK(cudaMemcpy(host_buf, st.kidx + u * p.cap * p.dI, (size_t)n * p.dI * 2, cudaMemcpyDeviceToHost));
+      return IM_OK;
+    case IM_S_K:
+    case IM_S_V: {
+      if ((rc = need((size_t)n * p.Dkv * 2))) return rc;
+      const bf16* src = (which == IM_S_K ? st.Kc : st.Vc) + u * p.Hkv * p.cap * p.d;
+      // device layout [Hkv][cap][d] -> host layout [n][Hkv][d]
+      for (int h = 0; h < p.Hkv; ++h)
+        CK(cudaMemcpy2D((char*)host_buf + (size_t)h * p.d * 2, (size_t)p.Dkv * 2, src + (size_t)h * p.cap * p.d,
+                        (size_t)p.d * 2, (size_t)p.d * 2, n, cudaMemcpyDeviceToHost));
+      return IM_OK;
+    }
+    case IM_S_M: {
+      const size_t cnt = (size_t)p.dM * p.Dkv;
+      if ((rc = need(cnt * 4))) return rc;
+      std::vector<float> M(cnt), phi((size_t)p.F * p.dM), w(p.F);
+      std::vector<uint16_t> pv((size_t)p.F * p.Dkv);
+      float c = 1.f;
+      CK(cudaMemcpy(M.data(), st.Mhat + u * cnt, cnt * 4, cudaMemcpyDeviceToHost));
+      CK(cudaMemcpy(phi.data(), st.pend_phi + u * p.F * p.dM, phi.size() * 4, cudaMemcpyDeviceToHost));
+      CK(cudaMemcpy(pv.data(), st.pend_v + u * p.F * p.Dkv, pv.size() * 2, cudaMemcpyDeviceToHost));
+      CK(cudaMemcpy(w.data(), st.pend_w + u * p.F, w.size() * 4, cudaMemcpyDeviceToHost));
+      CK(cudaMemcpy(&c, st.cscale + u, 4, cudaMemcpyDeviceToHost));
+      const int np = ctr[CTR_NPEND];
+      float* outp = (float*)host_buf;
+      for (int m = 0; m < p.dM; ++m)
+        for (int col = 0; col < p.Dkv; ++col) {
+          double acc = M[(size_t)m * p.Dkv + col];
+          for (int q = 0; q < np; ++q) {
+            uint32_t bits = ((uint32_t)pv[(size_t)q * p.Dkv + col]) << 16;
+            float vv;
+            memcpy(&vv, &bits, 4);
+            acc += (double)w[q] * (double)phi[(size_t)q * p.dM + m] * (double)vv;
+          }
+          outp[(size_t)m * p.Dkv + col] = (float)((double)c * acc);
+        }
+      return IM_OK;
+    }
+    case IM_S_B:
+      if ((rc = need((size_t)p.dM * 4))) return rc;
+      CK(cudaMemcpy(host_buf, st.bvec + u * p.dM, (size_t)p.dM * 4, cudaMemcpyDeviceToHost));
+      return IM_OK;
+    case IM_S_EVICTED: {
+      const int ne = ctr[CTR_NEVICT];
+      if (ne < 0 || ne > p.tail) return fail(IM_ERR_STATE, "device evicted count %d outside [0,%d]", ne, p.tail);
+      if ((rc = need((size_t)ne * 4))) return rc;
+      CK(cudaMemcpy(host_buf, st.ev_pos + u * p.tail, (size_t)ne * 4, cudaMemcpyDeviceToHost));
+      std::sort((int32_t*)host_buf, (int32_t*)host_buf + ne);
+      return IM_OK;
+    }
+    case IM_S_SEL_POS:
+    case IM_S_SEL_IMP: {
+      const int ns = ctr[CTR_NSEL];
+      if (ns < 0 || ns > p.cap) return fail(IM_ERR_STATE, "device selection count %d outside [0,%d]", ns, p.cap);
+      if ((rc = need((size_t)ns * 4))) return rc;
+      const void* src = which == IM_S_SEL_POS ? (const void*)(st.sel_pos + u * p.cap) : (const void*)(st.sel_imp + u * p.cap);
+      CK(cudaMemcpy(host_buf, src, (size_t)ns * 4, cudaMemcpyDeviceToHost));
+      return IM_OK;
+    }
+    default:
+      return fail(IM_ERR_ARG, "unknown state piece %d", which);
+  }
+}
+
+int im_state_import(im_ctx* ctx, int layer, int seq, int which, const void* host_buf, size_t bytes) {
+  if (!ctx || !host_buf) return fail(IM_ERR_ARG, "null argument");
+  const ImDims& p = ctx->p;
+  if (layer < 0 || layer >= p.L || seq < 0 || seq >= p.S) return fail(IM_ERR_ARG, "layer/seq out of range");
+  CK(cudaDeviceSynchronize());
+  const size_t u = (size_t)layer * p.S + seq;
+  const ImState& st = ctx->lo.st;
+  HostUnit& hu = ctx->hu[u];
+  auto exact = [&](size_t want) -> int {
+    if (bytes != want) return fail(IM_ERR_ARG, "state %d: got %zu bytes, expected %zu", which, bytes, want);
+    return IM_OK;
+  };
+  int rc;
+  const int n = hu.n;
+  switch (which) {
+    case IM_S_COUNTS: {
+      if ((rc = exact(CTR_STRIDE * 4))) return rc;
+      int32_t ctr[CTR_STRIDE];
+      memcpy(ctr, host_buf, sizeof(ctr));
+      if (ctr[CTR_N] < 0 || ctr[CTR_N] > p.cap || ctr[CTR_SINCE] < 0 || ctr[CTR_SINCE] >= p.tau || ctr[CTR_T] < ctr[CTR_N])
+        return fail(IM_ERR_ARG, "inconsistent counters");
+      ctr[CTR_NPEND] = 0;  // pending writes cannot be imported; IM_S_M carries the folded state
+      ctr[CTR_NEVICT] = 0;
+      ctr[CTR_DIRECT] = 0;
+      ctr[CTR_NSEL] = 0;
+      int32_t old[CTR_STRIDE];
+      CK(cudaMemcpy(old, st.ctr + u * CTR_STRIDE, sizeof(old), cudaMemcpyDeviceToHost));
+      if (old[CTR_NPEND] != 0) return fail(IM_ERR_STATE, "import IM_S_M before IM_S_COUNTS when writes are pending");
+      CK(cudaMemcpy(st.ctr + u * CTR_STRIDE, ctr, sizeof(ctr), cudaMemcpyHostToDevice));
+      hu.n = ctr[CTR_N];
+      hu.T = ctr[CTR_T];
+      hu.since = ctr[CTR_SINCE];
+      hu.npend = 0;
+      return IM_OK;
+    }
+    case IM_S_POS:
+      if ((rc = exact((size_t)n * 4))) return rc;
+      CK(cudaMemcpy(st.pos + u * p.cap, host_buf, bytes, cudaMemcpyHostToDevice));
+      return IM_OK;
+    case IM_S_IMP:
+      if ((rc = exact((size_t)n * 4))) return rc;
+      CK(cudaMemcpy(st.imp + u * p.cap, host_buf, bytes, cudaMemcpyHostToDevice));
+      return IM_OK;
+    case IM_S_KIDX:
+      if ((rc = exact((size_t)n * p.dI * 2))) return rc;
+      CK(cudaMemcpy(st.kidx + u * p.cap * p.dI, host_buf, bytes, cudaMemcpyHostToDevice));
+      return IM_OK;
+    case IM_S_K:
+    case IM_S_V: {
+      if ((rc = exact((size_t)n * p.Dkv * 2))) return rc;
+      bf16* dst = (which == IM_S_K ? st.Kc : st.Vc) + u * p.Hkv * p.cap * p.d;
+      for (int h = 0; h < p.Hkv; ++h)
+        CK(cudaMemcpy2D(dst + (size_t)h * p.cap * p.d, (size_t)p.d * 2, (const char*)host_buf + (size_t)h * p.d * 2,
+                        (size_t)p.Dkv * 2, (size_t)p.d * 2, n, cudaMemcpyHostToDevice));
+      return IM_OK;
+    }
+    case IM_S_M: {
+      if ((rc = exact((size_t)p.dM * p.Dkv * 4))) return rc;
+      CK(cudaMemcpy(st.Mhat + u * p.dM * p.Dkv, host_buf, bytes, cudaMemcpyHostToDevice));
+      const float one = 1.f;
+      const int32_t zero = 0;
+      CK(cudaMemcpy(st.cscale + u, &one, 4, cudaMemcpyHostToDevice));
+      CK(cudaMemcpy(st.ctr + u * CTR_STRIDE + CTR_NPEND, &zero, 4, cudaMemcpyHostToDevice));
+      hu.npend = 0;
+      return IM_OK;
+    }
+    case IM_S_B:
+      if ((rc = exact((size_t)p.dM * 4))) return rc;
+      CK(cudaMemcpy(st.bvec + u * p.dM, host_buf, bytes, cudaMemcpyHostToDevice));
+      return IM_OK;
+    default:
+      return fail(IM_ERR_ARG, "state piece %d cannot be imported", which);
+  }
+}
+
+int im_topb_select(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink, uint8_t* keep,
+                   int32_t* n_evict, void* cuda_stream) {
+  if (!scores || !pos || !keep || !n_evict) return fail(IM_ERR_ARG, "null tensor");
+  if (rows < 0 || n < 0 || budget < 0 || n_sink < 0) return fail(IM_ERR_ARG, "negative size");
+  if (rows == 0) return IM_OK;
+  CKL(im_launch_topb(scores, pos, rows, n, budget, n_sink, keep, n_evict, (cudaStream_t)cuda_stream));
+  return IM_OK;
+}
+
+int im_status(im_ctx* ctx, void* cuda_stream, int32_t* device_status) {
+  if (!ctx || !device_status) return fail(IM_ERR_ARG, "null argument");
+  CK(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+  CK(cudaMemcpy(device_status, ctx->lo.st.status, 4, cudaMemcpyDeviceToHost));
+  if (*device_status & ST_TIMEOUT) return fail(IM_ERR_TIMEOUT, "a bounded device wait gave up (status %d)", *device_status);
+  if (*device_status) return fail(IM_ERR_STATE, "device status %d (1: non-finite score, 2: count mismatch)", *device_status);
+  return IM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,556 @@
+// Indexer side of the path: projections (a0), append, indexer scores pooled by max (a1), budgeted
+// selection (a2), plus weight initialisation.  Symbols follow Sec. 3.1 of the paper.
+#include "im_internal.cuh"
+
+namespace {
+
+constexpr float NEG_INF = -__builtin_huge_valf();
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// a0: out[v][row0 + r] = sum_i W[r][i] * in[v][i]   (bf16 inputs, float32 accumulation)
+// One warp per (row, vector).  grid = (total_rows, ceil(NV / 8)), block = 256 (8 warps = 8 vectors).
+__global__ void k_proj(ImProjJobs jobs, float* __restrict__ out) {
+  int r = blockIdx.x, j = 0;  // blockIdx.x enumerates the rows of all jobs back to back
+  while (j + 1 < jobs.n_jobs && r >= jobs.job[j].rows) {
+    r -= jobs.job[j].rows;
+    ++j;
+  }
+  const ImProjJob job = jobs.job[j];
+  const int row = job.row0 + r;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int v = blockIdx.y * 8 + warp;
+  if (v >= jobs.NV) return;
+  const int Dn = jobs.Dn;
+  const uint4* w4 = reinterpret_cast<const uint4*>(job.W + (size_t)r * Dn);
+  const uint4* x4 = reinterpret_cast<const uint4*>(job.in + (size_t)v * Dn);
+  float acc = 0.f;
+  for (int c = lane; c < Dn / 8; c += 32) {
+    uint4 a = w4[c], b = x4[c];
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      acc = fmaf(__uint_as_float(aw[k] << 16), __uint_as_float(bw[k] << 16), acc);
+      acc = fmaf(__uint_as_float(aw[k] & 0xffff0000u), __uint_as_float(bw[k] & 0xffff0000u), acc);
+    }
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) out[(size_t)v * jobs.out_stride + row] = acc;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Indexer key of one token: k = bf16( RMSNorm(U_k x) )  (Sec. 3.1).  The cached key is a quantised
+// code, so the value that gets rounded is computed in float64: the bf16 bits then do not depend on
+// the summation order and agree with any other float64 evaluation.
+// One warp per token.  grid = ceil(NV / 4), block = 128.
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__global__ void k_proj_key(ImDims p, const bf16* __restrict__ Uk, const bf16* __restrict__ x, int NV,
+                           bf16* __restrict__ kidx_new) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int v = blockIdx.x * 4 + warp;
+  if (v >= NV) return;
+  const uint4* x4 = reinterpret_cast<const uint4*>(x + (size_t)v * p.D);
+  double ms = 0.0;
+  double mine = 0.0;  // lane r keeps u[r] (d_I <= 64: two rounds)
+  double mine2 = 0.0;
+  for (int r = 0; r < p.dI; ++r) {
+    const uint4* w4 = reinterpret_cast<const uint4*>(Uk + (size_t)r * p.D);
+    double acc = 0.0;
+    for (int c = lane; c < p.D / 8; c += 32) {
+      const uint4 a = w4[c], b = x4[c];
+      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        // the product of two bf16 values is exact in float32
+        acc += (double)(__uint_as_float(aw[k] << 16) * __uint_as_float(bw[k] << 16));
+        acc += (double)(__uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u));
+      }
+    }
+    acc = warp_sum_d(acc);
+    ms += acc * acc;
+    if (lane == (r & 31)) {
+      if (r < 32) mine = acc; else mine2 = acc;
+    }
+  }
+  const double inv = 1.0 / sqrt(ms / (double)p.dI + (double)p.norm_eps);
+  if (lane < p.dI) kidx_new[(size_t)v * p.dI + lane] = __double2bfloat16(mine * inv);
+  if (lane + 32 < p.dI) kidx_new[(size_t)v * p.dI + lane + 32] = __double2bfloat16(mine2 * inv);
+}
+
+// ------------------------------------------------------------------------------------------------
+// RMSNorm pieces shared by decode and prefill: finalise one token's raw projections in place.
+//   raw[uq ..]  -> q features, RMS-normalised per indexer head
+//   raw[g ..]   -> alpha = G x / sqrt(H_I d_I)
+// Executed by one warp; lanes stride over heads / elements.
+__device__ void finalize_features(const ImDims& p, float* raw, int lane) {
+  const ImRows r = im_rows(p);
+  for (int h = lane; h < p.HI; h += 32) {
+    float* y = raw + r.uq + h * p.dI;
+    float ms = 0.f;
+    for (int i = 0; i < p.dI; ++i) ms = fmaf(y[i], y[i], ms);
+    const float inv = 1.0f / sqrtf(ms / (float)p.dI + p.norm_eps);
+    for (int i = 0; i < p.dI; ++i) y[i] *= inv;
+  }
+  const float gs = 1.0f / sqrtf((float)p.HI * (float)p.dI);
+  for (int h = lane; h < p.HI; h += 32) raw[r.g + h] *= gs;
+}
+
+// A_{s,t} = sum_h alpha_h * act(q_h . k_t)   (Sec. 3.1), q/alpha in shared memory, k in registers
+__device__ __forceinline__ float index_score(const ImDims& p, const float* __restrict__ qf,
+                                             const float* __restrict__ alpha, const float* __restrict__ k) {
+  float A = 0.f;
+  for (int h = 0; h < p.HI; ++h) {
+    float z = 0.f;
+    for (int i = 0; i < p.dI; ++i) z = fmaf(qf[h * p.dI + i], k[i], z);
+    if (p.act == 0) z = fmaxf(z, 0.f);
+    A = fmaf(alpha[h], z, A);
+  }
+  return A;
+}
+
+// ------------------------------------------------------------------------------------------------
+// decode: append the token and pool the new query's scores into every cached entry.
+// grid = n_seq, block = 256.
+__global__ void k_decode_index(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __restrict__ k_new,
+                               const bf16* __restrict__ v_new) {
+  extern __shared__ float smem[];
+  float* s_raw = smem;  // [R3]
+  const int i = blockIdx.x;
+  const int seq = call.seq[i];
+  const size_t u = (size_t)call.layer * p.S + seq;
+  int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  const int n = ctr[CTR_N];
+  const int T = ctr[CTR_T];
+  const ImRows r = im_rows(p);
+  const int tid = threadIdx.x;
+  if (n < 0 || n >= p.cap) {  // never write out of bounds: flag and leave
+    if (tid == 0) atomicOr(st.status, ST_COUNT);
+    return;
+  }
+  float* raw = sc.raw + (size_t)i * p.R5;
+  for (int k = tid; k < p.R3; k += blockDim.x) s_raw[k] = raw[k];
+  __syncthreads();
+  if (tid < 32) finalize_features(p, s_raw, tid);
+  __syncthreads();
+  // cache the new entry in slot n
+  bf16* kid = st.kidx + (u * p.cap + n) * p.dI;
+  for (int k = tid; k < p.dI; k += blockDim.x) {
+    const bf16 b = sc.kidx_new[(size_t)i * p.dI + k];
+    kid[k] = b;
+    s_raw[r.uk + k] = __bfloat162float(b);  // the new slot is scored with the cached (rounded) key
+  }
+  const int dv = p.d / 8;  // 16-byte vectors per head row
+  for (int k = tid; k < p.Hkv * dv; k += blockDim.x) {
+    const int h = k / dv, c = k % dv;
+    const uint4* ks = reinterpret_cast<const uint4*>(k_new + (size_t)i * p.Dkv + h * p.d) + c;
+    const uint4* vs = reinterpret_cast<const uint4*>(v_new + (size_t)i * p.Dkv + h * p.d) + c;
+    const size_t row = ((u * p.Hkv + h) * p.cap + n) * p.d;
+    reinterpret_cast<uint4*>(st.Kc + row)[c] = *ks;
+    reinterpret_cast<uint4*>(st.Vc + row)[c] = *vs;
+  }
+  if (tid == 0) st.pos[u * p.cap + n] = T;
+  __syncthreads();
+  const float* qf = s_raw + r.uq;
+  const float* alpha = s_raw + r.g;
+  const int n1 = n + 1;
+  bool bad = false;
+  for (int t = tid; t < n1; t += blockDim.x) {
+    float kk[64];
+    if (t == n) {
+      for (int k = 0; k < p.dI; ++k) kk[k] = s_raw[r.uk + k];
+    } else {
+      const bf16* row = st.kidx + (u * p.cap + t) * p.dI;
+      for (int k = 0; k < p.dI; ++k) kk[k] = __bfloat162float(row[k]);
+    }
+    const float A = index_score(p, qf, alpha, kk);
+    bad |= !isfinite(A);
+    const float old = (t == n) ? NEG_INF : st.imp[u * p.cap + t];
+    st.imp[u * p.cap + t] = fmaxf(old, A);
+  }
+  if (bad) atomicOr(st.status, ST_NONFINITE);
+  if (tid == 0) {
+    ctr[CTR_N] = n1;
+    ctr[CTR_T] = T + 1;
+    ctr[CTR_SINCE] = ctr[CTR_SINCE] + 1;
+    ctr[CTR_NEVICT] = 0;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// prefill: finalise the features of every chunk token, append K/V/kidx/pos.
+// grid = (C, n_seq), block = 128.  The counters are advanced by the scoring kernel.
+__global__ void k_prefill_append(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __restrict__ K,
+                                 const bf16* __restrict__ V) {
+  const int c = blockIdx.x, i = blockIdx.y;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  const int n = ctr[CTR_N], T = ctr[CTR_T];
+  const int tid = threadIdx.x;
+  if (n < 0 || n + call.C > p.cap) {
+    if (tid == 0 && c == 0) atomicOr(st.status, ST_COUNT);
+    return;
+  }
+  const ImRows r = im_rows(p);
+  float* raw = sc.raw + ((size_t)i * call.C + c) * p.R3;
+  if (tid < 32) finalize_features(p, raw, tid);
+  __syncthreads();
+  const int slot = n + c;
+  bf16* kid = st.kidx + (u * p.cap + slot) * p.dI;
+  for (int k = tid; k < p.dI; k += blockDim.x) kid[k] = sc.kidx_new[((size_t)i * call.C + c) * p.dI + k];
+  const int dv = p.d / 8;
+  for (int k = tid; k < p.Hkv * dv; k += blockDim.x) {
+    const int h = k / dv, cc = k % dv;
+    const size_t src = ((size_t)i * call.C + c) * p.Dkv + h * p.d;
+    const size_t row = ((u * p.Hkv + h) * p.cap + slot) * p.d;
+    reinterpret_cast<uint4*>(st.Kc + row)[cc] = reinterpret_cast<const uint4*>(K + src)[cc];
+    reinterpret_cast<uint4*>(st.Vc + row)[cc] = reinterpret_cast<const uint4*>(V + src)[cc];
+  }
+  if (tid == 0) {
+    st.pos[u * p.cap + slot] = T + c;
+    st.imp[u * p.cap + slot] = NEG_INF;
+  }
+}
+
+// prefill a1: imp_t = max(imp_t, max over chunk queries s with pos_s >= pos_t of A_{s,t}).
+// grid = (ceil(n_max / 32), n_seq), block = 256 = 32 entries x 8 query lanes.
+constexpr int PS_QT = 32;  // queries staged per tile
+__global__ void k_prefill_score(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  extern __shared__ float smem[];
+  const int nq = p.HI * p.dI;
+  float* s_q = smem;                       // [PS_QT][nq]
+  float* s_a = s_q + PS_QT * nq;           // [PS_QT][HI]
+  float* s_max = s_a + PS_QT * p.HI;       // [8][32]
+  const int i = blockIdx.y;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  const int n0 = ctr[CTR_N], T = ctr[CTR_T];
+  const int n1 = n0 + call.C;
+  if (n0 < 0 || n1 > p.cap) return;  // flagged by the append kernel
+  const int e0 = blockIdx.x * 32;
+  if (e0 >= n1) return;
+  const int el = threadIdx.x & 31, ql = threadIdx.x >> 5;
+  const int e = e0 + el;
+  const bool live = e < n1;
+  const ImRows r = im_rows(p);
+  float kk[64];
+  int epos = 0x7fffffff;
+  if (live) {
+    const bf16* row = st.kidx + (u * p.cap + e) * p.dI;
+    for (int k = 0; k < p.dI; ++k) kk[k] = __bfloat162float(row[k]);
+    epos = st.pos[u * p.cap + e];
+  } else {
+    for (int k = 0; k < p.dI; ++k) kk[k] = 0.f;
+  }
+  float best = NEG_INF;
+  bool bad = false;
+  // queries before the oldest entry of this block cannot see it: skip whole tiles
+  int min_pos = epos;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) min_pos = min(min_pos, __shfl_xor_sync(0xffffffffu, min_pos, o));
+  int c_first = max(0, min_pos - T);
+  c_first = (c_first / PS_QT) * PS_QT;
+  for (int c0 = c_first; c0 < call.C; c0 += PS_QT) {
+    const int cn = min(PS_QT, call.C - c0);
+    __syncthreads();
+    for (int k = threadIdx.x; k < cn * nq; k += blockDim.x) {
+      const int cc = k / nq, j = k % nq;
+      s_q[cc * nq + j] = sc.raw[((size_t)i * call.C + c0 + cc) * p.R3 + r.uq + j];
+    }
+    for (int k = threadIdx.x; k < cn * p.HI; k += blockDim.x) {
+      const int cc = k / p.HI, j = k % p.HI;
+      s_a[cc * p.HI + j] = sc.raw[((size_t)i * call.C + c0 + cc) * p.R3 + r.g + j];
+    }
+    __syncthreads();
+    if (live) {
+      for (int cc = ql; cc < cn; cc += 8) {
+        if (T + c0 + cc < epos) continue;  // causal mask
+        const float A = index_score(p, s_q + cc * nq, s_a + cc * p.HI, kk);
+        bad |= !isfinite(A);
+        best = fmaxf(best, A);
+      }
+    }
+  }
+  __syncthreads();
+  s_max[ql * 32 + el] = best;
+  __syncthreads();
+  if (ql == 0 && live) {
+    for (int k = 1; k < 8; ++k) best = fmaxf(best, s_max[k * 32 + el]);
+    st.imp[u * p.cap + e] = fmaxf(st.imp[u * p.cap + e], best);
+  }
+  if (bad) atomicOr(st.status, ST_NONFINITE);
+}
+
+// advance the counters after the chunk has been appended and scored.  grid = n_seq, block = 32.
+__global__ void k_prefill_commit(ImDims p, ImState st, ImCall call) {
+  const size_t u = (size_t)call.layer * p.S + call.seq[blockIdx.x];
+  int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  if (threadIdx.x == 0) {
+    const int n0 = ctr[CTR_N];
+    if (n0 < 0 || n0 + call.C > p.cap) return;
+    ctr[CTR_N] = n0 + call.C;
+    ctr[CTR_T] = ctr[CTR_T] + call.C;
+    ctr[CTR_NEVICT] = 0;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// a2: budgeted selection of one row (one thread block).  Radix select of the k-th largest 64-bit
+// key (score image, ~position), eight passes of eight bits; keys are distinct, so exactly k entries
+// compare >= the threshold.
+struct SelectShared {
+  uint32_t hist[256];
+  uint32_t digit, remaining;
+};
+
+__device__ uint64_t block_kth_largest_key(const float* __restrict__ score, const int32_t* __restrict__ pos, int n,
+                                          int k, int n_sink, SelectShared* sh) {
+  uint64_t prefix = 0, mask = 0;
+  if (threadIdx.x == 0) sh->remaining = (uint32_t)k;
+  for (int shift = 56; shift >= 0; shift -= 8) {
+    for (int b = threadIdx.x; b < 256; b += blockDim.x) sh->hist[b] = 0;
+    __syncthreads();
+    for (int t = threadIdx.x; t < n; t += blockDim.x) {
+      const uint64_t key = im_select_key(score[t], pos[t], n_sink);
+      if ((key & mask) == prefix) atomicAdd(&sh->hist[(uint32_t)(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t rem = sh->remaining, cum = 0;
+      int b = 255;
+      for (; b > 0; --b) {
+        const uint32_t c = sh->hist[b];
+        if (cum + c >= rem) break;
+        cum += c;
+      }
+      sh->digit = (uint32_t)b;
+      sh->remaining = rem - cum;
+    }
+    __syncthreads();
+    prefix |= (uint64_t)sh->digit << shift;
+    mask |= 0xFFull << shift;
+    __syncthreads();
+  }
+  return prefix;
+}
+
+// exclusive prefix sum of one int per thread over the block (blockDim.x <= 1024); returns the total
+__device__ int block_exclusive_scan(int v, int* out_excl, int* s_tmp /*[33]*/) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) s_tmp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const int nw = (blockDim.x + 31) >> 5;
+    int w = lane < nw ? s_tmp[lane] : 0;
+    int wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += t;
+    }
+    if (lane < nw) s_tmp[lane] = wi - w;
+    if (lane == nw - 1) s_tmp[32] = wi;
+  }
+  __syncthreads();
+  *out_excl = incl - v + s_tmp[warp];
+  const int total = s_tmp[32];
+  __syncthreads();
+  return total;
+}
+
+// Compression of every sequence in the call (Sec. 4 schedule): restart pooling; if over budget,
+// flag the retained entries and list the evicted slots in ascending slot order.
+// grid = n_seq, block = 256.
+__global__ void k_select(ImDims p, ImState st, ImCall call) {
+  __shared__ SelectShared sh;
+  __shared__ int s_tmp[33];
+  const size_t u = (size_t)call.layer * p.S + call.seq[blockIdx.x];
+  int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  const int n = ctr[CTR_N];
+  float* imp = st.imp + u * p.cap;
+  const int32_t* pos = st.pos + u * p.cap;
+  uint8_t* keep = st.keep + u * p.cap;
+  if (n < 0 || n > p.cap) {
+    if (threadIdx.x == 0) atomicOr(st.status, ST_COUNT);
+    return;
+  }
+  int ne = 0;
+  // keep what the selection saw (debug/parity export)
+  for (int t = threadIdx.x; t < n; t += blockDim.x) {
+    st.sel_pos[u * p.cap + t] = pos[t];
+    st.sel_imp[u * p.cap + t] = imp[t];
+  }
+  if (n > p.B) {
+    ne = n - p.B;
+    const uint64_t thr = block_kth_largest_key(imp, pos, n, p.B, p.n_sink, &sh);
+    // ordered list of the evicted slots: each thread owns a contiguous run of slots
+    const int per = (n + blockDim.x - 1) / blockDim.x;
+    const int t0 = min(n, (int)threadIdx.x * per), t1 = min(n, t0 + per);
+    int cnt = 0;
+    for (int t = t0; t < t1; ++t) {
+      const bool k = im_select_key(imp[t], pos[t], p.n_sink) >= thr;
+      keep[t] = k ? 1 : 0;
+      cnt += k ? 0 : 1;
+    }
+    int off;
+    const int total = block_exclusive_scan(cnt, &off, s_tmp);
+    if (total != ne && threadIdx.x == 0) atomicOr(st.status, ST_COUNT);
+    int32_t* evs = st.ev_slot + u * p.tail;
+    int32_t* evp = st.ev_pos + u * p.tail;
+    for (int t = t0; t < t1; ++t)
+      if (!keep[t] && off < p.tail) {
+        evs[off] = t;
+        evp[off] = pos[t];
+        ++off;
+      }
+    __syncthreads();
+  }
+  for (int t = threadIdx.x; t < n; t += blockDim.x) imp[t] = NEG_INF;
+  if (threadIdx.x == 0) {
+    ctr[CTR_SINCE] = 0;
+    ctr[CTR_NSEL] = n;
+    ctr[CTR_NEVICT] = ne;
+    // fold everything into M in this evict step if the pending list cannot take the evicted set
+    ctr[CTR_DIRECT] = (p.mem && ne > 0 && ctr[CTR_NPEND] + ne > p.F) ? 1 : 0;
+    if (ne > 0) ctr[CTR_EVSTEPS] = ctr[CTR_EVSTEPS] + 1;
+  }
+}
+
+// Row-generic selection without a context.  grid = rows, block = 256.
+__global__ void k_topb(const float* __restrict__ scores, const int32_t* __restrict__ pos, int n, int B, int n_sink,
+                       uint8_t* __restrict__ keep, int32_t* __restrict__ n_evict) {
+  __shared__ SelectShared sh;
+  const size_t row = blockIdx.x;
+  const float* s = scores + row * n;
+  const int32_t* ps = pos + row * n;
+  uint8_t* k = keep + row * n;
+  if (n <= B) {
+    for (int t = threadIdx.x; t < n; t += blockDim.x) k[t] = 1;
+    if (threadIdx.x == 0) n_evict[row] = 0;
+    return;
+  }
+  if (B == 0) {
+    for (int t = threadIdx.x; t < n; t += blockDim.x) k[t] = 0;
+    if (threadIdx.x == 0) n_evict[row] = n;
+    return;
+  }
+  const uint64_t thr = block_kth_largest_key(s, ps, n, B, n_sink, &sh);
+  for (int t = threadIdx.x; t < n; t += blockDim.x) k[t] = im_select_key(s[t], ps[t], n_sink) >= thr ? 1 : 0;
+  if (threadIdx.x == 0) n_evict[row] = n - B;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Seeded N(0, std^2) bf16 init: counter-based (splitmix64 of (seed, layer, tensor, index)) + Box-Muller.
+__device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+__global__ void k_init_normal(bf16* __restrict__ dst, size_t n, uint64_t key, float std) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint64_t r = splitmix64(key ^ splitmix64(i));
+  const float u1 = ((float)((r >> 40) + 1)) * (1.0f / 16777216.0f);   // (0, 1]
+  const float u2 = ((float)((r >> 8) & 0xFFFFFFu)) * (1.0f / 16777216.0f);
+  const float z = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+  dst[i] = __float2bfloat16_rn(z * std);
+}
+
+// Wfold[m][g*d + c] = sum over the query heads j of group g of Wt[m][j*d + c]   (float32)
+__global__ void k_fold_theta(ImDims p, const bf16* __restrict__ Wt, float* __restrict__ Wfold) {
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (size_t)p.dM * p.Dkv) return;
+  const int m = (int)(idx / p.Dkv), col = (int)(idx % p.Dkv);
+  const int g = col / p.d, c = col % p.d;
+  float s = 0.f;
+  for (int j = g * p.Gq; j < (g + 1) * p.Gq; ++j) s += __bfloat162float(Wt[(size_t)m * p.D + j * p.d + c]);
+  Wfold[idx] = s;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------ launchers
+cudaError_t im_launch_proj(const ImLaunch& L, const ImProjJobs& jobs, float* out) {
+  dim3 grid(jobs.total_rows, (jobs.NV + 7) / 8);
+  k_proj<<<grid, 256, 0, L.stream>>>(jobs, out);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_proj_key(const ImLaunch& L, const void* x, int NV) {
+  k_proj_key<<<(NV + 3) / 4, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, L.sc.kidx_new);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_decode_index(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new) {
+  const size_t smem = (size_t)L.p.R3 * 4;
+  k_decode_index<<<call.n_seq, 256, smem, L.stream>>>(L.p, L.st, L.sc, call, (const bf16*)k_new, (const bf16*)v_new);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_prefill_append(const ImLaunch& L, const ImCall& call, const void* k, const void* v) {
+  dim3 grid(call.C, call.n_seq);
+  k_prefill_append<<<grid, 128, 0, L.stream>>>(L.p, L.st, L.sc, call, (const bf16*)k, (const bf16*)v);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_prefill_score(const ImLaunch& L, const ImCall& call, int n_max) {
+  dim3 grid((n_max + 31) / 32, call.n_seq);
+  const size_t smem = ((size_t)PS_QT * (L.p.HI * L.p.dI + L.p.HI) + 256) * 4;
+  k_prefill_score<<<grid, 256, smem, L.stream>>>(L.p, L.st, L.sc, call);
+  ++*L.launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  k_prefill_commit<<<call.n_seq, 32, 0, L.stream>>>(L.p, L.st, call);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call) {
+  k_select<<<call.n_seq, 256, 0, L.stream>>>(L.p, L.st, call);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,
+                           uint8_t* keep, int32_t* n_evict, cudaStream_t stream) {
+  k_topb<<<rows, 256, 0, stream>>>(scores, pos, n, budget, n_sink, keep, n_evict);
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_init_weights(const ImDims& p, const ImWeights& w, int layer, uint64_t seed, float std,
+                                   cudaStream_t stream) {
+  struct T { bf16* ptr; size_t n; } ts[5] = {{w.Uq, (size_t)p.HI * p.dI * p.D}, {w.Uk, (size_t)p.dI * p.D},
+                                             {w.G, (size_t)p.HI * p.D}, {w.Wt, (size_t)p.dM * p.D}, {w.wg, (size_t)p.D}};
+  for (int t = 0; t < 5; ++t) {
+    const uint64_t key = seed * 0x9E3779B97F4A7C15ull + ((uint64_t)layer << 8) + (uint64_t)t;
+    k_init_normal<<<(unsigned)((ts[t].n + 255) / 256), 256, 0, stream>>>(ts[t].ptr, ts[t].n, key, std);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaMemsetAsync(w.bg, 0, 4, stream);
+}
+
+cudaError_t im_launch_fold_theta(const ImDims& p, const ImWeights& w, cudaStream_t stream) {
+  const size_t n = (size_t)p.dM * p.Dkv;
+  k_fold_theta<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(p, w.Wt, w.Wfold);
+  return cudaGetLastError();
+}

@@ -1,0 +1,217 @@
+"""GPU-vs-oracle parity of the hot path, through the C ABI (``-m gpu``).
+
+Every test drives the CUDA library and the CPU oracle with the same seeded inputs (tests/parity.py)
+at sizes the oracle finishes in seconds, spanning several tiles and ragged tails, plus the edge
+cases of the method (ties, sinks, empty eviction, decay, interval pooling, disabled memory,
+non-power-of-two head shapes).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import indexmem_oracle as orc
+from paper_2605_25475_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def im():
+    from paper_2605_25475_b200 import binding
+    return binding
+
+
+def _pair(*a, **k):
+    from tests.parity import Pair
+    return Pair(*a, **k)
+
+
+TINY = synth.CONFIGS["tiny"]
+
+
+# ------------------------------------------------------------------ K2 alone: bit-exact selection
+@pytest.mark.parametrize("n,B,n_sink", [(1, 1, 0), (7, 3, 2), (300, 300, 4), (300, 400, 4), (2049, 2048, 4),
+                                         (4096, 2048, 4), (5000, 1, 0), (16384, 1024, 4), (777, 0, 0)])
+def test_topb_select_bit_exact(im, n, B, n_sink):
+    rng = np.random.default_rng(n * 131 + B)
+    rows = 5
+    # heavy ties: half of the ReLU scores are exactly zero, both signs of zero, unscored (-inf) entries
+    sc = rng.standard_normal((rows, n)).astype(np.float32)
+    sc[rng.random((rows, n)) < 0.4] = 0.0
+    sc[rng.random((rows, n)) < 0.1] = -0.0
+    sc[rng.random((rows, n)) < 0.05] = -np.inf
+    sc[1] = 0.0                                           # one row of pure ties
+    sc[2] = np.round(sc[2] * 2) / 2                       # few distinct values
+    pos = np.stack([rng.permutation(n * 3)[:n] for _ in range(rows)]).astype(np.int32)
+    keep, nev = im.im_topb_select(torch.tensor(sc).cuda(), torch.tensor(pos).cuda(), B, n_sink)
+    torch.cuda.synchronize()
+    keep, nev = keep.cpu().numpy(), nev.cpu().numpy()
+    for r in range(rows):
+        want = orc.select_top_b(sc[r], pos[r], B, n_sink)
+        assert np.array_equal(keep[r], want), f"row {r}"
+        assert nev[r] == n - min(n, B)
+
+
+# ------------------------------------------------------------------ the small benchmark configuration
+def test_tiny_config_end_to_end():
+    """1 layer, 4 q heads / 1 KV head, d 64, 1024-token context in one chunk -> B 256, 64 decode steps."""
+    p = _pair(TINY)
+    p.prefill(0)
+    for s in range(TINY.steps):
+        p.decode(s)
+    st = p.stats
+    assert st["kidx_flips"] == 0
+    assert st["cut_divergences"] <= 2
+    assert st["max_out_err"] <= 2e-3 and st["max_M_err"] <= 2e-3 and st["max_score_err"] <= 1e-5
+
+
+def test_tiny_config_float32_output():
+    wl = TINY.replace(name="tiny_f32", ctx=512, chunk=512, B=128, steps=12)
+    p = _pair(wl, out_f32=1)
+    p.prefill(0)
+    for s in range(wl.steps):
+        out, ob, od = p.decode(s)
+        assert out.dtype == torch.float32
+    assert p.stats["max_out_err"] <= 1e-4
+
+
+# ------------------------------------------------------------------ reduced copies of the larger configurations
+def test_llama_shape_reduced():
+    """32 q / 8 KV heads, d 128 (widths 8 x 16, d_M 512), lognormal key norms; ragged sizes."""
+    wl = synth.CONFIGS["llama8b_b1"].replace(name="llama_red", ctx=700, chunk=700, B=300, steps=20)
+    p = _pair(wl)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
+
+
+def test_qwen_shape_reduced_batch():
+    """28 q / 4 KV heads (G_q 7, H_I 7, d_M 448): nothing is a power of two; 3 sequences, needles."""
+    wl = synth.CONFIGS["qwen7b_b8"].replace(name="qwen_red", n_seq=3, ctx=600, chunk=600, B=200, steps=10, n_needles=8)
+    p = _pair(wl)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
+
+
+def test_chunked_prefill_reduced():
+    """Mistral-shaped chunked prefill: several chunks, eviction to the budget after each."""
+    wl = synth.CONFIGS["mistral7b_prefill"].replace(name="mistral_red", ctx=4 * 160, chunk=160, B=192, steps=4)
+    p = _pair(wl)
+    for c in range(4):
+        p.prefill(c)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.o.evict_steps(0) == 3 + wl.steps
+    assert p.stats["max_M_err"] <= 2e-3
+
+
+# ------------------------------------------------------------------ edge cases of the method
+def test_budget_never_reached_is_exact_attention(im):
+    wl = TINY.replace(name="nobudget", ctx=100, chunk=100, B=4096, steps=5, n_needles=2)
+    p = _pair(wl, max_chunk=100)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.o.evict_steps(0) == 0 and p.g.counts(0, 0)["n"] == 105
+    assert not p.g.export(0, 0, im.IM_S_M).any()
+
+
+def test_memory_disabled():
+    wl = TINY.replace(name="nomem", ctx=300, chunk=300, B=64, steps=8, n_needles=2)
+    p = _pair(wl, enable_memory=0)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3
+
+
+def test_decay_and_write_strength():
+    wl = TINY.replace(name="decay", ctx=300, chunk=300, B=64, steps=40, n_needles=2)
+    p = _pair(wl, lambda_=0.9, eta=0.5, pending_slots=4)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_M_err"] <= 2e-3
+
+
+def test_interval_pooling_tau():
+    """tau = 8: scores pooled by max over the interval's queries, 8 entries evicted at once."""
+    wl = TINY.replace(name="tau8", ctx=200, chunk=200, B=96, steps=24, tau=8, n_needles=2)
+    p = _pair(wl, pending_slots=16)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+        assert p.g.counts(0, 0)["n"] == 96 + (s + 1) % 8
+    assert p.o.evict_steps(0) == 1 + 3
+
+
+def test_identity_activation_and_all_ties():
+    wl = TINY.replace(name="ident", ctx=150, chunk=150, B=40, steps=4, n_needles=0)
+    p = _pair(wl, act=1)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    # G = 0: alpha = 0, every score ties at zero, the lowest positions stay
+    p2 = _pair(wl.replace(name="ties"))
+    w = dict(p2.weights)
+    w["G"] = torch.zeros_like(w["G"])
+    p2.o.set_weights({k: synth.f32(v) for k, v in w.items()})
+    p2.g.set_weights(0, w)
+    p2.prefill(0)
+    assert p2.o.positions(0).tolist() == list(range(40))
+    for s in range(3):
+        p2.decode(s)
+
+
+def test_single_token_chunks_and_subset_of_sequences(im):
+    """Chunks of one token; calls that address a subset of the sequences in arbitrary order."""
+    wl = TINY.replace(name="subset", n_seq=3, ctx=24, chunk=1, B=10, steps=0, n_needles=0)
+    p = _pair(wl, max_chunk=8)
+    for c in range(12):
+        p.prefill(c)
+    dev = p.device
+    # sequences 2 and 0 only, in that order
+    x, q, k, v = synth.decode_inputs(wl, 0, 0)
+    ids = [2, 0]
+    ob, od = p.o.decode_batch(ids, synth.f32(x[ids]), synth.f32(q[ids]), synth.f32(q[ids]), synth.f32(k[ids]), synth.f32(v[ids]))
+    out = p.g.decode_step(0, ids, x[ids].to(dev).contiguous(), q[ids].to(dev).contiguous(), q[ids].to(dev).contiguous(),
+                          k[ids].to(dev).contiguous(), v[ids].to(dev).contiguous())
+    assert p.g.status() == 0
+    p.check_out(out, ob, od)
+    assert p.g.counts(0, 1)["T"] == 12 and p.g.counts(0, 0)["T"] == 13
+
+
+def test_errors_are_reported_not_fatal(im):
+    wl = TINY.replace(name="errs", ctx=32, chunk=32, B=16, steps=0, n_needles=0)
+    p = _pair(wl)
+    dev = p.device
+    X, Q, K, V = [t.to(dev) for t in synth.prefill_inputs(wl, 0, 0)]
+    with pytest.raises(im.IndexMemError) as e:
+        im.im_prefill_chunk(p.g.ctx, 0, [5], 32, X, Q, K, V)
+    assert e.value.code == im.IM_ERR_ARG
+    with pytest.raises(im.IndexMemError) as e:
+        im.im_prefill_chunk(p.g.ctx, 0, [0], 33, X, Q, K, V)
+    assert e.value.code == im.IM_ERR_ARG
+    with pytest.raises(im.IndexMemError) as e:
+        im.im_prefill_chunk(p.g.ctx, 1, [0], 32, X, Q, K, V)
+    assert e.value.code == im.IM_ERR_ARG
+    # the context is still usable
+    p.prefill(0)
+    assert p.g.status() == 0
+
+
+def test_seeded_weight_init_statistics(im):
+    g = im.IndexMem(im.Config(n_layers=2, max_seqs=1, n_q_heads=8, n_kv_heads=2, head_dim=64, budget=32, seed=7))
+    g2 = im.IndexMem(im.Config(n_layers=2, max_seqs=1, n_q_heads=8, n_kv_heads=2, head_dim=64, budget=32, seed=7))
+    w0, w1, v0 = g.get_weights(0), g.get_weights(1), g2.get_weights(0)
+    for name in ("U_q", "U_k", "G", "W_theta", "w_g"):
+        a = w0[name].float()
+        assert torch.equal(w0[name], v0[name])               # same seed, same weights
+        assert not torch.equal(w0[name], w1[name])           # layers differ
+        if a.numel() > 2000:
+            assert abs(a.mean().item()) < 3 * 0.02 / a.numel() ** 0.5 + 1e-4
+            assert abs(a.std().item() - 0.02) < 0.002
+    assert w0["b_g"].item() == 0.0
