@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the IndexMem decode hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+Workload (N = 1): the 32-layer Llama-3-8B-shaped KV stack, batch 32, 16K-token context ingested in
+eight 2048-token chunks with eviction to the budget B = 2048 after each, then decode steps with a
+compression every token (tau = 1).  One "step" is one decode token for all 32 sequences through all
+32 layers: projections, indexer scores, top-B selection, memory write, compaction, attention over
+the retained entries and the gated memory readout.  Inputs and weights are seeded synthetic draws
+(paper_2605_25475_b200/synth.py).
+
+With N > 1 (torchrun) every rank runs its own replica on its own 32 sequences (the path has no
+exchange step, so this is weak scaling without a data-path collective); time is the max over ranks.
+
+One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2605_25475_b200 import synth
+
+METRIC = "decode_step_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------------------------
+# algorithmic bytes: what one decode step has to touch in HBM at tau = 1, n = B + 1
+def algorithmic_bytes(wl: synth.Workload):
+    n = wl.B + 1
+    weights = 2 * (wl.HI * wl.dI * wl.D + wl.dI * wl.D + wl.HI * wl.D + wl.dM * wl.D + wl.D) + 4 * wl.dM * wl.Dkv
+    kv = n * 2 * wl.Dkv * 2
+    state = 4 * wl.dM * wl.Dkv + 4 * wl.dM
+    kidx = n * wl.dI * 2
+    io = (5 * wl.D + 4 * wl.Dkv) * 2
+    evict = 4 * wl.dM + 2 * wl.Dkv + 4 * wl.Dkv
+    per_seq = kv + state + kidx + io + evict
+    per_layer = weights + wl.n_seq * per_seq
+    return {"step": wl.n_layers * per_layer, "attn_launch": wl.n_seq * (kv + state), "per_seq": per_seq,
+            "weights": weights}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx, self.proc, self.path = gpu_index, None, f"/tmp/indexmem_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.idx), "-lms", "200"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------------------------
+def build_context(wl: synth.Workload, device, ingest=True, log=lambda *a: None):
+    from paper_2605_25475_b200 import binding as im
+    g = im.IndexMem(im.Config(n_layers=wl.n_layers, max_seqs=wl.n_seq, n_q_heads=wl.H, n_kv_heads=wl.Hkv,
+                              head_dim=wl.d, budget=wl.B, compress_interval=wl.tau, max_chunk=wl.chunk,
+                              n_sink=wl.n_sink), device)
+    ids = list(range(wl.n_seq))
+    for layer in range(wl.n_layers):
+        g.set_weights(layer, {k: v.cpu() for k, v in synth.make_weights(wl, layer, device).items()})
+    if ingest:
+        t0 = time.time()
+        for c in range(wl.ctx // wl.chunk):
+            for layer in range(wl.n_layers):
+                X, Q, K, V = synth.prefill_inputs(wl, layer, c, device)
+                g.prefill_chunk(layer, ids, X, Q, K, V)
+            torch.cuda.synchronize()
+            log(f"ingested chunk {c + 1}/{wl.ctx // wl.chunk} ({time.time() - t0:.1f}s)")
+        assert g.status() == 0
+    return g, ids
+
+
+def decode_inputs_all(wl, n_steps, device):
+    """[n_steps][4] tensors stacked over layers: x [L, n, D], q [L, n, H, d], k, v [L, n, Hkv, d]."""
+    steps = []
+    for s in range(n_steps):
+        parts = [synth.decode_inputs(wl, layer, s, device) for layer in range(wl.n_layers)]
+        steps.append(tuple(torch.stack([p[i] for p in parts]).contiguous() for i in range(4)))
+    return steps
+
+
+def run_ours(args, rank, world, device):
+    from paper_2605_25475_b200 import binding as im
+    wl = synth.CONFIGS[args.workload]
+    log = (lambda *a: print("[bench]", *a, file=sys.stderr, flush=True)) if rank == 0 else (lambda *a: None)
+    g, ids = build_context(wl, device, log=log)
+    L = wl.n_layers
+    n_in = min(8, args.steps + args.warmup)                      # distinct input sets, cycled
+    inputs = decode_inputs_all(wl, n_in, device)
+    sx, sq, sk, sv = [torch.empty_like(t) for t in inputs[0]]    # static buffers the graph reads
+    out = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=device)
+
+    def one_step():
+        for layer in range(L):
+            g.decode_step(layer, ids, sx[layer], sq[layer], sq[layer], sk[layer], sv[layer], out[layer])
+
+    def load(step):
+        x, q, k, v = inputs[step % n_in]
+        sx.copy_(x); sq.copy_(q); sk.copy_(k); sv.copy_(v)
+
+    stream = torch.cuda.Stream(device)
+    graph = None
+    launches_per_step = None
+    with torch.cuda.stream(stream):
+        load(0)
+        c0 = g.launch_count()
+        one_step()                                               # reaches the steady state n = B
+        launches_per_step = g.launch_count() - c0
+        stream.synchronize()
+        if args.graph:
+            graph = torch.cuda.CUDAGraph()
+            load(1)
+            with torch.cuda.graph(graph, stream=stream):
+                one_step()
+        step_fn = graph.replay if graph is not None else one_step
+        for w in range(args.warmup):
+            load(w + 2)
+            step_fn()
+        stream.synchronize()
+        barrier(world)
+        sampler = ClockSampler(torch.cuda.current_device() if device.index is None else device.index)
+        if rank == 0:
+            sampler.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for s in range(args.steps):
+            load(args.warmup + 2 + s)
+            step_fn()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        barrier(world)
+        ms = ev0.elapsed_time(ev1)
+        clocks = sampler.stop() if rank == 0 else None
+        assert g.status() == 0
+        ms = max_over_ranks(ms, world, device)
+
+        # per-launch time of the dominant kernel: the same steps again, un-graphed, with the
+        # library recording CUDA events around the attention + readout launch on this stream
+        im.im_profile_begin(g.ctx, args.steps * L)
+        for s in range(args.steps):
+            load(s)
+            one_step()
+        attn_ms, attn_n = im.im_profile_end(g.ctx)
+
+        # end to end: host buffers in, host buffer out, copies inside the timed region
+        e2e = run_e2e(args, wl, g, ids, inputs, stream, world, device)
+
+    tokens = wl.n_seq * args.steps * world
+    ab = algorithmic_bytes(wl)
+    peaks = measured_peaks()
+    attn_launch_s = attn_ms / max(attn_n, 1) * 1e-3
+    achieved = ab["attn_launch"] / attn_launch_s / 1e9
+    res = {
+        "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H,
+                   "kv_heads": wl.Hkv, "head_dim": wl.d, "context": wl.ctx, "budget": wl.B, "tau": wl.tau,
+                   "cuda_graph": bool(args.graph),
+                   "l2": "inputs larger than L2 (each step streams %.1f GB)" % (ab["step"] / 1e9)},
+        "hbm_gbs_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9,
+        "hbm_frac_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "roofline": {"bound": "hbm", "kernel": "attention+readout", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                     "traffic": args.traffic, "bytes_per_launch": ab["attn_launch"],
+                     "us_per_launch": attn_launch_s * 1e6},
+        "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+    }
+    return res, wl
+
+
+def run_e2e(args, wl, g, ids, inputs, stream, world, device):
+    L = wl.n_layers
+    n_in = len(inputs)
+    host = [tuple(t.cpu().pin_memory() for t in inp) for inp in inputs]
+    dx, dq, dk, dv = [torch.empty_like(t) for t in inputs[0]]
+    dout = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=device)
+    hout = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host[0])
+    d2h = hout.numel() * hout.element_size()
+
+    def step(s):
+        hx, hq, hk, hv = host[s % n_in]
+        for layer in range(L):
+            dx[layer].copy_(hx[layer], non_blocking=True)
+            dq[layer].copy_(hq[layer], non_blocking=True)
+            dk[layer].copy_(hk[layer], non_blocking=True)
+            dv[layer].copy_(hv[layer], non_blocking=True)
+            g.decode_step(layer, ids, dx[layer], dq[layer], dq[layer], dk[layer], dv[layer], dout[layer])
+            hout[layer].copy_(dout[layer], non_blocking=True)
+        stream.synchronize()                                     # the caller has the step's result on the host
+
+    for s in range(min(3, args.warmup)):
+        step(s)
+    barrier(world)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for s in range(args.steps):
+        step(s)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    ms = max_over_ranks(ev0.elapsed_time(ev1), world, device)
+    return {"value": wl.n_seq * args.steps * world / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms / args.steps}
+
+
+# ----------------------------------------------------------------------------------------------
+def oracle_sample(wl, n_units, n_steps, log=lambda *a: None):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: n_units sequences of
+    layer 0, cache brought to the budget by ingesting two chunks (a decode step's cost depends on
+    B and the widths, not on how much context was ingested before), n_steps decode steps timed."""
+    from oracle import indexmem_oracle as orc
+    sub = wl.replace(n_seq=n_units)
+    o = orc.OracleLayer(orc.OracleConfig(H=wl.H, Hkv=wl.Hkv, d=wl.d, B=wl.B, tau=wl.tau, n_sink=wl.n_sink), n_units)
+    o.set_weights({k: synth.f32(v) for k, v in synth.make_weights(wl, 0).items()})
+    ids = list(range(n_units))
+    t0 = time.time()
+    for c in range(2 if wl.ctx // wl.chunk >= 2 else 1):
+        X, Q, K, V = synth.prefill_inputs(sub, 0, c)
+        o.prefill_batch(ids, synth.f32(X), synth.f32(Q), synth.f32(K), synth.f32(V))
+    log(f"oracle sample set up in {time.time() - t0:.1f}s")
+    ins = [tuple(synth.f32(t) for t in synth.decode_inputs(sub, 0, s)) for s in range(n_steps)]
+    t0 = time.time()
+    for s in range(n_steps):
+        x, q, k, v = ins[s]
+        o.decode_batch(ids, x, q, q, k, v)
+    dt = time.time() - t0
+    cores = min(n_units, len(os.sched_getaffinity(0)))
+    unit_steps = n_units * n_steps
+    # one unit-step = one token of one sequence through one layer; a full token crosses n_layers layers
+    tok_s = unit_steps / wl.n_layers / dt
+    return {"value": tok_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n_units} sequences x 1 layer x {n_steps} decode steps at n=B={wl.B} "
+                      f"(cache filled by two {wl.chunk}-token chunks), scaled by 1/{wl.n_layers} layers to whole tokens; "
+                      f"{dt:.1f}s of CPU time on {cores} threads"}, dt
+
+
+def run_reference(args, rank, world):
+    wl = synth.CONFIGS[args.workload]
+    if rank != 0:
+        return None
+    from oracle import indexmem_oracle as orc
+    orc.build()
+    n_units = min(len(os.sched_getaffinity(0)), wl.n_seq, 8)
+    # each "step" of this arm is one decode step of the sample; keep the whole run to a few minutes
+    steps = max(1, min(args.steps, 64))
+    base, dt = oracle_sample(wl, n_units, steps,
+                             log=lambda *a: print("[bench]", *a, file=sys.stderr, flush=True))
+    return {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wl.n_seq / base["value"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "budget": wl.B,
+                       "tau": wl.tau},
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+# ----------------------------------------------------------------------------------------------
+_dist = None
+
+
+def barrier(world):
+    if world > 1:
+        _dist.barrier()
+
+
+def max_over_ranks(ms, world, device):
+    if world == 1:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    _dist.all_reduce(t, op=_dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def main():
+    global _dist
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=32)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b_stack", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--graph", type=int, default=1, help="replay the step from a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as is)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        res = run_reference(args, rank, world)
+        if res is not None:
+            print(json.dumps(res), flush=True)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        import torch.distributed as dist
+        _dist = dist
+        dist.init_process_group("nccl", device_id=device)
+    res, wl = run_ours(args, rank, world, device)
+    if rank == 0:
+        if not args.no_cpu_baseline and world == 1:
+            from oracle import indexmem_oracle as orc
+            orc.build()
+            n_units = min(len(os.sched_getaffinity(0)), wl.n_seq, 8)
+            res["cpu_baseline"], _ = oracle_sample(wl, n_units, 384,
+                                                   log=lambda *a: print("[bench]", *a, file=sys.stderr, flush=True))
+        else:
+            res["cpu_baseline"] = None
+        print(json.dumps(res), flush=True)
+    if world > 1:
+        _dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
