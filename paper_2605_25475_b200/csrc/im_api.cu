@@ -130,7 +130,12 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->sc.kidx_new = (bf16*)take((size_t)p.S * p.max_chunk * p.dI * 2);
   lo->sc.phi = (float*)take((size_t)p.S * p.tail * p.dM * 4);
   lo->sc.moves = (int32_t*)take((size_t)p.S * 2 * p.tail * 4);
-  lo->sc.part = (float*)take((size_t)p.S * p.H * p.max_splits * (p.d + 2) * 4);
+  {
+    const size_t generic = (size_t)p.S * p.H * p.max_splits * (p.d + 2);
+    const size_t stream = ((size_t)IM_ATTN_MAX_CTAS * IM_ATTN_WARPS + (size_t)p.S * p.Hkv) * p.Gq * (p.d + 2);
+    lo->sc.part = (float*)take(std::max(generic, stream) * 4);
+  }
+  lo->sc.rpart = (float*)take((size_t)p.S * ((p.dM + IM_READOUT_ROWS - 1) / IM_READOUT_ROWS) * p.Dkv * 4);
   lo->total = align_up(off, 256);
 }
 
@@ -150,6 +155,10 @@ struct im_ctx {
   std::vector<HostUnit> hu;
   int64_t launches = 0;
   int device = 0;
+  alignas(64) unsigned char mapK[128];  // TMA descriptors of the K / V caches
+  alignas(64) unsigned char mapV[128];
+  bool fast_attn = false;
+  int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
   std::vector<cudaEvent_t> prof_ev;  // pairs (start, stop)
   size_t prof_used = 0;              // events recorded so far
 };
@@ -269,6 +278,14 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
   for (int l = 0; l < p.L && e == cudaSuccess; ++l) {
     e = im_launch_init_weights(p, ctx->lo.w[l], l, c.seed, c.init_std, 0);
     if (e == cudaSuccess) e = im_launch_fold_theta(p, ctx->lo.w[l], 0);
+  }
+  if (e == cudaSuccess && im_attn_fast_supported(p)) {
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
+    if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK, ctx->mapV);
+    if (e == cudaSuccess) e = im_attn_prepare(p);
+    ctx->n_ctas = std::max(1, std::min(sms, IM_ATTN_MAX_CTAS));
+    ctx->fast_attn = (e == cudaSuccess);
   }
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
@@ -415,7 +432,12 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   // a5-a6: attention over the retained entries + gated readout
   const bool prof = ctx->prof_used + 2 <= ctx->prof_ev.size();
   if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], L.stream));
-  CKL(im_launch_attention(L, call, q, out, n_max));
+  if (ctx->fast_attn) {
+    if (p.mem) CKL(im_launch_readout(L, call));
+    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, out, ctx->n_ctas));
+  } else {
+    CKL(im_launch_attention(L, call, q, out, n_max));
+  }
   if (prof) {
     CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], L.stream));
     ctx->prof_used += 2;

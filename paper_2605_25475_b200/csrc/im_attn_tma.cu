@@ -1,0 +1,526 @@
+// a5-a6, B200 path: attention over the retained entries as a persistent, TMA-fed flash-decode
+// kernel; the memory readout (Eq. 5) as a streaming GEMV; one merge kernel that fuses both (Eq. 4).
+//
+// Attention kernel.  HBM-bound (every retained K/V byte is read once per step), so the design is
+// about keeping loads in flight, not about FLOPs:
+//   * the retained entries of a (sequence, KV head) row form tiles of 32 keys; all tiles of all rows
+//     are cut into equal contiguous runs, one run per warp (stream-K style: perfect balance for any
+//     mix of lengths, at most one partial result per row boundary inside a run);
+//   * every warp owns a private ring of 16 KB stages (K tile + V tile), filled by TMA tensor copies
+//     (128-byte swizzle) that its lane 0 issues, completion on one mbarrier per stage.  No CTA-wide
+//     barrier exists in the main loop;
+//   * the math runs on mma.sync m16n8k16 with the KEYS on the M axis and the G_q query heads of the
+//     KV head (padded to 8) on N: S^T = K Q^T, then O^T += V^T P^T.  P^T is moved from the
+//     accumulator layout to the B-operand layout with movmatrix.  P is split into two bf16 terms so
+//     that the product is accurate to 2^-17, not 2^-9.
+#include <cuda.h>
+
+#include "im_internal.cuh"
+
+namespace {
+
+constexpr float NEG_INF = -__builtin_huge_valf();
+constexpr int TILE = IM_ATTN_TILE;       // keys per tile
+constexpr int STAGES = 3;                // ring depth per warp
+constexpr int WARPS = IM_ATTN_WARPS;     // consumer warps per CTA (each also issues its own TMA)
+constexpr uint32_t WAIT_LIMIT = 1u << 22;  // try_wait attempts before a warp gives up and flags ST_TIMEOUT
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// bounded wait: returns false if the phase did not complete within the limit
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movm_t(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// two floats -> packed bf16x2 (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+struct RowMap {        // tile bookkeeping shared by the attention and merge kernels
+  long long q;         // tiles per warp run
+  long long total;     // total tiles
+};
+
+// tiles of sequence i (all KV heads have the same count)
+__device__ __forceinline__ int tiles_of(int n) { return (n + TILE - 1) / TILE; }
+
+// ------------------------------------------------------------------------------------------------
+// Persistent attention kernel.  grid = #SMs (or fewer), block = WARPS * 32.
+// Shared memory: per warp STAGES x 16 KB (1024-byte aligned), then barriers and the per-sequence
+// prefix of tile counts.
+template <int DH>
+__global__ void __launch_bounds__(WARPS * 32, 1)
+k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, ImDims p, ImState st,
+              ImScratch sc, ImCall call, const bf16* __restrict__ q) {
+  static_assert(DH == 64 || DH == 128, "head dims with a fast path");
+  constexpr int KSTEPS = DH / 16;            // k-steps of the S = K Q^T product
+  constexpr int DT = DH / 16;                // 16-row tiles of O^T
+  constexpr int BOXES = DH / 64;             // 128-byte column boxes per row
+  constexpr int TILE_BYTES = TILE * DH * 2;  // one K (or V) tile
+  constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  unsigned char* ring = smem + (size_t)warp * STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)WARPS * STAGES * STAGE_BYTES);
+  long long* s_pref = reinterpret_cast<long long*>(bars + WARPS * STAGES);  // [n_seq + 1]
+  int* s_n = reinterpret_cast<int*>(s_pref + IM_MAX_CALL_SEQS + 1);         // [n_seq]
+
+  // ---- tile prefix over the sequences of the call (every CTA computes the same table)
+  for (int i = threadIdx.x; i < call.n_seq; i += blockDim.x) {
+    const size_t u = (size_t)call.layer * p.S + call.seq[i];
+    s_n[i] = max(0, min(st.ctr[u * CTR_STRIDE + CTR_N], p.cap));
+  }
+  if (lane == 0) {
+    for (int s = 0; s < STAGES; ++s) mbar_init(smem_u32(&bars[warp * STAGES + s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    long long acc = 0;
+    for (int i = 0; i < call.n_seq; ++i) {
+      s_pref[i] = acc;
+      acc += (long long)tiles_of(s_n[i]) * p.Hkv;
+    }
+    s_pref[call.n_seq] = acc;
+  }
+  __syncthreads();
+  const long long total = s_pref[call.n_seq];
+  const long long WT = (long long)gridDim.x * WARPS;
+  const long long qrun = (total + WT - 1) / WT;
+  const long long wglob = (long long)blockIdx.x * WARPS + warp;
+  const long long run0 = min(total, wglob * qrun), run1 = min(total, run0 + qrun);
+  if (run0 >= run1) return;
+
+  // ---- position of the first tile of the run: sequence i, KV head h, tile tt
+  int i = 0;
+  {
+    int lo = 0, hi = call.n_seq;  // last i with s_pref[i] <= run0
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_pref[mid] <= run0) lo = mid; else hi = mid;
+    }
+    i = lo;
+    while (i < call.n_seq - 1 && tiles_of(s_n[i]) == 0) ++i;  // empty sequences own no tiles
+  }
+  int nt = tiles_of(s_n[i]);
+  int h = (int)((run0 - s_pref[i]) / nt), tt = (int)((run0 - s_pref[i]) % nt);
+
+  // iterator used by the producer side (runs STAGES tiles ahead of the consumer side)
+  int pi = i, ph = h, ptt = tt, pnt = nt;
+  long long issued = run0;
+  auto issue = [&](long long j) {  // lane 0 only: load global tile j (== issued) into stage j % STAGES
+    const int s = (int)((j - run0) % STAGES);
+    const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
+    const uint32_t dst = smem_u32(ring + (size_t)s * STAGE_BYTES);
+    const size_t u = (size_t)call.layer * p.S + call.seq[pi];
+    const int row = (int)((u * p.Hkv + ph) * (size_t)p.cap) + ptt * TILE;
+    mbar_expect_tx(bar, STAGE_BYTES);
+#pragma unroll
+    for (int b = 0; b < BOXES; ++b) {
+      tma_load_2d(dst + b * (TILE * 128), &tmK, b * 64, row, bar);
+      tma_load_2d(dst + TILE_BYTES + b * (TILE * 128), &tmV, b * 64, row, bar);
+    }
+    // advance the producer iterator
+    if (++ptt == pnt) {
+      ptt = 0;
+      if (++ph == p.Hkv) {
+        ph = 0;
+        do { ++pi; } while (pi < call.n_seq && tiles_of(s_n[pi]) == 0);
+        pnt = pi < call.n_seq ? tiles_of(s_n[pi]) : 1;
+      }
+    }
+  };
+  if (lane == 0) {
+    for (int k = 0; k < STAGES && issued < run1; ++k) issue(issued++);
+  }
+
+  const float sl2 = p.scale * 1.4426950408889634f;  // softmax in base 2
+  bool ok = true;
+  long long j = run0;
+  while (j < run1 && ok) {
+    // ---- one (sequence, KV head) segment of the run
+    const size_t u = (size_t)call.layer * p.S + call.seq[i];
+    const int n = s_n[i];
+    const long long row_id = (long long)i * p.Hkv + h;
+    // Q^T as B fragments: head g of the group (zero for the padding heads)
+    uint32_t qf[KSTEPS][2];
+    {
+      const bf16* qrow = q + ((size_t)i * p.H + (size_t)h * p.Gq + g) * DH;
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        qf[ks][0] = g < p.Gq ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t) : 0u;
+        qf[ks][1] = g < p.Gq ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t + 8) : 0u;
+      }
+    }
+    float o[DT][4];
+#pragma unroll
+    for (int dt = 0; dt < DT; ++dt) o[dt][0] = o[dt][1] = o[dt][2] = o[dt][3] = 0.f;
+    float m0 = NEG_INF, m1 = NEG_INF, l0 = 0.f, l1 = 0.f;  // heads 2t, 2t+1 (l: this thread's share)
+
+    for (; tt < nt && j < run1; ++tt, ++j) {
+      const int s = (int)((j - run0) % STAGES);
+      const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
+      if (!mbar_wait(bar, (uint32_t)(((j - run0) / STAGES) & 1))) { ok = false; break; }
+      const uint32_t Ks = smem_u32(ring + (size_t)s * STAGE_BYTES), Vs = Ks + TILE_BYTES;
+      // ---- S^T = K Q^T : [32 keys] x [8 heads]
+      float sacc[TILE / 16][4];
+#pragma unroll
+      for (int mt = 0; mt < TILE / 16; ++mt) {
+        sacc[mt][0] = sacc[mt][1] = sacc[mt][2] = sacc[mt][3] = 0.f;
+        const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+          const int c = ks * 2 + (lane >> 4);
+          const uint32_t addr = Ks + (c >> 3) * (TILE * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+          uint32_t a0, a1, a2, a3;
+          ldsm_x4(addr, a0, a1, a2, a3);
+          mma_bf16(sacc[mt], a0, a1, a2, a3, qf[ks][0], qf[ks][1]);
+        }
+      }
+      // ---- online softmax (base 2); keys beyond n are masked
+      const int key0 = tt * TILE;
+      float tmax0 = NEG_INF, tmax1 = NEG_INF;
+#pragma unroll
+      for (int mt = 0; mt < TILE / 16; ++mt) {
+        const bool v0 = key0 + mt * 16 + g < n, v1 = key0 + mt * 16 + g + 8 < n;
+        sacc[mt][0] = v0 ? sacc[mt][0] * sl2 : NEG_INF;
+        sacc[mt][1] = v0 ? sacc[mt][1] * sl2 : NEG_INF;
+        sacc[mt][2] = v1 ? sacc[mt][2] * sl2 : NEG_INF;
+        sacc[mt][3] = v1 ? sacc[mt][3] * sl2 : NEG_INF;
+        tmax0 = fmaxf(tmax0, fmaxf(sacc[mt][0], sacc[mt][2]));
+        tmax1 = fmaxf(tmax1, fmaxf(sacc[mt][1], sacc[mt][3]));
+      }
+#pragma unroll
+      for (int off = 4; off < 32; off <<= 1) {
+        tmax0 = fmaxf(tmax0, __shfl_xor_sync(0xffffffffu, tmax0, off));
+        tmax1 = fmaxf(tmax1, __shfl_xor_sync(0xffffffffu, tmax1, off));
+      }
+      const float mn0 = fmaxf(m0, tmax0), mn1 = fmaxf(m1, tmax1);
+      // every tile holds at least one valid key, so mn0/mn1 are finite
+      const float c0 = exp2f(m0 - mn0), c1 = exp2f(m1 - mn1);
+      m0 = mn0; m1 = mn1;
+      l0 *= c0; l1 *= c1;
+#pragma unroll
+      for (int dt = 0; dt < DT; ++dt) {
+        o[dt][0] *= c0; o[dt][1] *= c1; o[dt][2] *= c0; o[dt][3] *= c1;
+      }
+      uint32_t ph_[TILE / 16][2], pl_[TILE / 16][2];  // P^T as B fragments, high and low bf16 terms
+#pragma unroll
+      for (int mt = 0; mt < TILE / 16; ++mt) {
+        const float p0 = exp2f(sacc[mt][0] - mn0), p1 = exp2f(sacc[mt][1] - mn1);
+        const float p2 = exp2f(sacc[mt][2] - mn0), p3 = exp2f(sacc[mt][3] - mn1);
+        l0 += p0 + p2;
+        l1 += p1 + p3;
+        const uint32_t hi01 = pack_bf16(p0, p1), hi23 = pack_bf16(p2, p3);
+        const uint32_t lo01 = pack_bf16(p0 - __uint_as_float(hi01 << 16), p1 - __uint_as_float(hi01 & 0xffff0000u));
+        const uint32_t lo23 = pack_bf16(p2 - __uint_as_float(hi23 << 16), p3 - __uint_as_float(hi23 & 0xffff0000u));
+        ph_[mt][0] = movm_t(hi01); ph_[mt][1] = movm_t(hi23);
+        pl_[mt][0] = movm_t(lo01); pl_[mt][1] = movm_t(lo23);
+      }
+      // ---- O^T += V^T P^T : [DH] x [8 heads]
+#pragma unroll
+      for (int dt = 0; dt < DT; ++dt) {
+#pragma unroll
+        for (int kt = 0; kt < TILE / 16; ++kt) {
+          const int r = kt * 16 + (lane & 7) + (lane >> 4) * 8;
+          const int c = dt * 2 + ((lane >> 3) & 1);
+          const uint32_t addr = Vs + (c >> 3) * (TILE * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+          uint32_t a0, a1, a2, a3;
+          ldsm_x4_t(addr, a0, a1, a2, a3);
+          mma_bf16(o[dt], a0, a1, a2, a3, ph_[kt][0], ph_[kt][1]);
+          mma_bf16(o[dt], a0, a1, a2, a3, pl_[kt][0], pl_[kt][1]);
+        }
+      }
+      // ---- the stage is free again: refill it
+      __syncwarp();
+      if (lane == 0 && issued < run1) issue(issued++);
+    }
+    if (!ok) break;
+    // ---- segment finished: write the partial (unnormalised O, max, sum) of this row
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+      l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+    }
+    {
+      // Rows are served by consecutive warps and consecutive rows share at most one warp, so
+      // (warp index + row index) is a collision-free slot id below WT + rows.
+      const long long slot = wglob + row_id;
+      float* dst = sc.part + (size_t)slot * p.Gq * (DH + 2);
+      const int hh0 = 2 * t, hh1 = 2 * t + 1;
+#pragma unroll
+      for (int dt = 0; dt < DT; ++dt) {
+        if (hh0 < p.Gq) {
+          dst[(size_t)hh0 * (DH + 2) + dt * 16 + g] = o[dt][0];
+          dst[(size_t)hh0 * (DH + 2) + dt * 16 + g + 8] = o[dt][2];
+        }
+        if (hh1 < p.Gq) {
+          dst[(size_t)hh1 * (DH + 2) + dt * 16 + g] = o[dt][1];
+          dst[(size_t)hh1 * (DH + 2) + dt * 16 + g + 8] = o[dt][3];
+        }
+      }
+      if (g == 0) {
+        if (hh0 < p.Gq) { dst[(size_t)hh0 * (DH + 2) + DH] = m0; dst[(size_t)hh0 * (DH + 2) + DH + 1] = l0; }
+        if (hh1 < p.Gq) { dst[(size_t)hh1 * (DH + 2) + DH] = m1; dst[(size_t)hh1 * (DH + 2) + DH + 1] = l1; }
+      }
+    }
+    // ---- next row
+    if (tt == nt) {
+      tt = 0;
+      if (++h == p.Hkv) {
+        h = 0;
+        do { ++i; } while (i < call.n_seq && tiles_of(s_n[i]) == 0);
+        if (i >= call.n_seq) break;
+        nt = tiles_of(s_n[i]);
+      }
+    }
+  }
+  if (!ok && lane == 0) atomicOr(st.status, ST_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Readout partials: rpart[i][rc][col] = sum over the 32 rows m of chunk rc of phi_q[m] * Mhat[m][col].
+// grid = (ceil(dM / 32), n_seq), block = 256; each thread owns 4 consecutive columns.
+constexpr int R_ROWS = IM_READOUT_ROWS;
+__global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  __shared__ float s_phi[R_ROWS];
+  const int rc = blockIdx.x, i = blockIdx.y;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const ImRows r = im_rows(p);
+  const int m0 = rc * R_ROWS, mcnt = min(R_ROWS, p.dM - m0);
+  if (threadIdx.x < R_ROWS) s_phi[threadIdx.x] = threadIdx.x < mcnt ? sc.raw[(size_t)i * p.R5 + r.theta + m0 + threadIdx.x] : 0.f;
+  __syncthreads();
+  const float* Mh = st.Mhat + (u * p.dM + m0) * (size_t)p.Dkv;
+  const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
+  float* dst = sc.rpart + ((size_t)i * nchunk + rc) * p.Dkv;
+  for (int c4 = threadIdx.x; c4 < p.Dkv / 4; c4 += blockDim.x) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    int m = 0;
+    for (; m + 8 <= mcnt; m += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = __ldg(reinterpret_cast<const float4*>(Mh + (size_t)(m + k) * p.Dkv) + c4);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const float f = s_phi[m + k];
+        acc.x = fmaf(f, v[k].x, acc.x); acc.y = fmaf(f, v[k].y, acc.y);
+        acc.z = fmaf(f, v[k].z, acc.z); acc.w = fmaf(f, v[k].w, acc.w);
+      }
+    }
+    for (; m < mcnt; ++m) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(Mh + (size_t)m * p.Dkv) + c4);
+      const float f = s_phi[m];
+      acc.x = fmaf(f, v.x, acc.x); acc.y = fmaf(f, v.y, acc.y);
+      acc.z = fmaf(f, v.z, acc.z); acc.w = fmaf(f, v.w, acc.w);
+    }
+    reinterpret_cast<float4*>(dst)[c4] = acc;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Merge: softmax-merge of the attention partials of one (sequence, KV head) row, readout (Eq. 5)
+// from the row-chunk partials and the pending rank-one terms, gate, fuse (Eq. 4), store.
+// grid = (Hkv, n_seq), block = DH.
+template <int DH, typename OutT>
+__global__ void __launch_bounds__(DH) k_attn_merge_rows(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call,
+                                                         int n_ctas, OutT* __restrict__ out) {
+  __shared__ float s_dot[64];
+  __shared__ float s_red[DH / 32];
+  __shared__ float s_den;
+  const int h = blockIdx.x, i = blockIdx.y, c = threadIdx.x;
+  const int warp = c >> 5, lane = c & 31;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  // ---- rebuild the tile bookkeeping of the attention kernel
+  long long pref = 0, total = 0;
+  int nt_i = 0;
+  for (int k = 0; k < call.n_seq; ++k) {
+    const size_t uk = (size_t)call.layer * p.S + call.seq[k];
+    const int nk = tiles_of(max(0, min(st.ctr[uk * CTR_STRIDE + CTR_N], p.cap)));
+    if (k == i) { pref = total; nt_i = nk; }
+    total += (long long)nk * p.Hkv;
+  }
+  const long long WT = (long long)n_ctas * WARPS;
+  const long long qrun = (total + WT - 1) / WT;
+  const long long row_first = pref + (long long)h * nt_i, row_last = row_first + nt_i - 1;
+  const long long row_id = (long long)i * p.Hkv + h;
+  float mkv = 0.f, gate = 0.f;
+  if (p.mem) {
+    const ImRows r = im_rows(p);
+    const float* raw = sc.raw + (size_t)i * p.R5;
+    const float* phiq = raw + r.theta;
+    const int np = min(ctr[CTR_NPEND], p.F);
+    float part_den = 0.f;
+    for (int m = c; m < p.dM; m += DH) part_den = fmaf(phiq[m] * phiq[m], st.bvec[u * p.dM + m], part_den);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) part_den += __shfl_xor_sync(0xffffffffu, part_den, off);
+    if (lane == 0) s_red[warp] = part_den;
+    for (int pp = warp; pp < np; pp += DH / 32) {
+      const float* ph = st.pend_phi + (u * p.F + pp) * p.dM;
+      float v = 0.f;
+      for (int m = lane; m < p.dM; m += 32) v = fmaf(phiq[m], ph[m], v);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+      if (lane == 0) s_dot[pp] = v * st.pend_w[u * p.F + pp];
+    }
+    __syncthreads();
+    if (c == 0) {
+      float d = p.eps;
+      for (int k = 0; k < DH / 32; ++k) d += s_red[k];
+      s_den = d;
+    }
+    __syncthreads();
+    const int col = h * DH + c;
+    const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
+    const float* rp = sc.rpart + (size_t)i * nchunk * p.Dkv + col;
+    for (int k = 0; k < nchunk; ++k) mkv += rp[(size_t)k * p.Dkv];
+    for (int pp = 0; pp < np; ++pp) mkv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mkv);
+    mkv = st.cscale[u] * mkv / s_den;
+    gate = 1.0f / (1.0f + expf(-(raw[r.wg] + w.bg[0])));
+  }
+  for (int hh = 0; hh < p.Gq; ++hh) {
+    float res = 0.f;
+    if (nt_i > 0) {
+      const long long w0 = row_first / qrun, w1 = row_last / qrun;
+      float M = NEG_INF;
+      for (long long wv = w0; wv <= w1; ++wv)
+        M = fmaxf(M, sc.part[((size_t)(wv + row_id) * p.Gq + hh) * (DH + 2) + DH]);
+      float L = 0.f, acc = 0.f;
+      for (long long wv = w0; wv <= w1; ++wv) {
+        const float* ps = sc.part + ((size_t)(wv + row_id) * p.Gq + hh) * (DH + 2);
+        const float e = exp2f(ps[DH] - M);
+        L = fmaf(ps[DH + 1], e, L);
+        acc = fmaf(ps[c], e, acc);
+      }
+      res = acc / L;
+    }
+    res = fmaf(gate, mkv, res);
+    const size_t idx = ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH + c;
+    if constexpr (sizeof(OutT) == 2) out[idx] = __float2bfloat16_rn(res);
+    else out[idx] = res;
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+// Encodes the tensor maps of the K and V caches: 2-D [rows = units * Hkv * cap, cols = d] bf16,
+// box = 64 columns x TILE rows, 128-byte swizzle.  Returns false if the fast path is unavailable.
+bool im_attn_fast_supported(const ImDims& p) { return (p.d == 64 || p.d == 128) && p.Gq <= 8 && p.Dkv % 4 == 0; }
+
+cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV) {
+  static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+  EncodeTiledFn enc = (EncodeTiledFn)fn;
+  const cuuint64_t rows = (cuuint64_t)p.L * p.S * p.Hkv * p.cap;
+  const cuuint64_t dims[2] = {(cuuint64_t)p.d, rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)p.d * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)TILE};
+  const cuuint32_t estr[2] = {1, 1};
+  void* bases[2] = {st.Kc, st.Vc};
+  void* maps[2] = {mapK, mapV};
+  for (int k = 0; k < 2; ++k) {
+    CUresult r = enc((CUtensorMap*)maps[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bases[k], dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
+  return cudaSuccess;
+}
+
+size_t im_attn_smem_bytes(const ImDims& p) {
+  const size_t stage = (size_t)2 * TILE * p.d * 2;
+  return (size_t)WARPS * STAGES * stage + (size_t)WARPS * STAGES * 8 + (IM_MAX_CALL_SEQS + 1) * 8 + IM_MAX_CALL_SEQS * 4 + 64;
+}
+
+cudaError_t im_attn_prepare(const ImDims& p) {
+  const int smem = (int)im_attn_smem_bytes(p);
+  cudaError_t e = cudaFuncSetAttribute(k_attn_stream<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_attn_stream<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+}
+
+cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call) {
+  const ImDims& p = L.p;
+  dim3 grid((p.dM + R_ROWS - 1) / R_ROWS, call.n_seq);
+  k_readout<<<grid, 256, 0, L.stream>>>(p, L.st, L.sc, call);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
+                                     const void* q, void* out, int n_ctas) {
+  const ImDims& p = L.p;
+  const size_t smem = im_attn_smem_bytes(p);
+  const CUtensorMap& mk = *(const CUtensorMap*)mapK;
+  const CUtensorMap& mv = *(const CUtensorMap*)mapV;
+  if (p.d == 64) k_attn_stream<64><<<n_ctas, WARPS * 32, smem, L.stream>>>(mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+  else k_attn_stream<128><<<n_ctas, WARPS * 32, smem, L.stream>>>(mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+  ++*L.launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  dim3 grid(p.Hkv, call.n_seq);
+  if (p.d == 64) {
+    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, 64, 0, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
+    else k_attn_merge_rows<64, bf16><<<grid, 64, 0, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
+  } else {
+    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, 128, 0, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
+    else k_attn_merge_rows<128, bf16><<<grid, 128, 0, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
+  }
+  ++*L.launches;
+  return cudaGetLastError();
+}

@@ -10,6 +10,10 @@ typedef __nv_bfloat16 bf16;
 
 #define IM_MAX_CALL_SEQS 256 /* sequences per hot call (the id list travels as a kernel parameter) */
 #define IM_SLOT_ALIGN 64     /* slot capacity is a multiple of the attention tile */
+#define IM_ATTN_TILE 32      /* keys per attention tile (one TMA box is 32 rows x 128 bytes) */
+#define IM_ATTN_WARPS 4      /* warps per CTA of the streaming attention kernel */
+#define IM_ATTN_MAX_CTAS 512 /* upper bound of its grid (one CTA per SM) */
+#define IM_READOUT_ROWS 32   /* rows of M per readout partial */
 
 // per-(layer, sequence) device counters
 enum { CTR_N = 0, CTR_T = 1, CTR_SINCE = 2, CTR_EVSTEPS = 3, CTR_NEVICT = 4, CTR_NPEND = 5, CTR_DIRECT = 6, CTR_NSEL = 7, CTR_STRIDE = 8 };
@@ -79,7 +83,9 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
   bf16* kidx_new;    // [max_seqs * max(1,max_chunk)][dI] indexer keys of the call's tokens
   float* phi;        // [max_seqs][tail][dM]   phi of the evicted keys
   int32_t* moves;    // [max_seqs][2][tail]    compaction: hole slots, survivor slots
-  float* part;       // [max_seqs][H][max_splits][d + 2] attention partials (acc, max, sum)
+  float* part;       // attention partials (acc[d], max, sum): generic kernel [max_seqs][H][max_splits][d + 2];
+                     // streaming kernel [warps + rows][Gq][d + 2]
+  float* rpart;      // [max_seqs][ceil(dM / IM_READOUT_ROWS)][Dkv] readout partials
 };
 
 struct ImCall {
@@ -116,6 +122,12 @@ cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_memory_write(const ImLaunch& L, const ImCall& call, int ne_max, bool direct);
 cudaError_t im_launch_compact(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const void* q, void* out, int n_max);
+bool im_attn_fast_supported(const ImDims& p);
+cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV);
+cudaError_t im_attn_prepare(const ImDims& p);
+cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call);
+cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
+                                     const void* q, void* out, int n_ctas);
 cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,
                            uint8_t* keep, int32_t* n_evict, cudaStream_t stream);
 cudaError_t im_launch_init_weights(const ImDims& p, const ImWeights& w, int layer, uint64_t seed, float std,
