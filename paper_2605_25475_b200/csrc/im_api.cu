@@ -124,12 +124,17 @@ void carve(const ImDims& p, char* base, Layout* lo) {
     w.Wt = (bf16*)take((size_t)p.dM * p.D * 2);
     w.wg = (bf16*)take((size_t)p.D * 2);
     w.bg = (float*)take(256);
-    w.Wfold = (float*)take((size_t)p.dM * p.Dkv * 4);
+    w.Wfh = (bf16*)take((size_t)p.dM * p.Dkv * 2);
+    w.Wfl = (bf16*)take((size_t)p.dM * p.Dkv * 2);
   }
-  lo->sc.raw = (float*)take((size_t)p.S * p.max_chunk * p.R5 * 4);
-  lo->sc.kidx_new = (bf16*)take((size_t)p.S * p.max_chunk * p.dI * 2);
+  lo->sc.raw = (float*)take((size_t)p.S * std::max(p.max_chunk, IM_KSPLIT) * p.R5 * 4);
+  lo->sc.keyp = (double*)take((size_t)p.S * std::max(p.max_chunk, IM_KSPLIT_KEY) * p.dI * 8);
+  lo->sc.evK = (bf16*)take((size_t)p.S * p.tail * p.Dkv * 2);
+  lo->sc.evV = (bf16*)take((size_t)p.S * p.tail * p.Dkv * 2);
   lo->sc.phi = (float*)take((size_t)p.S * p.tail * p.dM * 4);
-  lo->sc.moves = (int32_t*)take((size_t)p.S * 2 * p.tail * 4);
+  lo->sc.phip = (float*)take((size_t)IM_KSPLIT * p.S * p.F * p.dM * 4);
+  lo->sc.surv = (int32_t*)take((size_t)p.S * p.tail * 4);
+  lo->sc.nhole = (int32_t*)take((size_t)p.S * 4);
   {
     const size_t generic = (size_t)p.S * p.H * p.max_splits * (p.d + 2);
     const size_t stream = ((size_t)IM_ATTN_MAX_CTAS * IM_ATTN_WARPS + (size_t)p.S * p.Hkv) * p.Gq * (p.d + 2);
@@ -202,35 +207,50 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
     if (e_ != cudaSuccess) return fail(IM_ERR_CUDA, "launch %s: %s", #call, cudaGetErrorString(e_)); \
   } while (0)
 
-// The evict step shared by both hot calls: select -> memory write -> compaction, for the sequences
-// of `call` whose host mirror says they are over budget (others are skipped on the device).
-int run_compress(im_ctx* ctx, const ImLaunch& L, const ImCall& call) {
+int pick_ksplit(int K, int want) {
+  for (int s = want; s > 1; --s)
+    if (K % (16 * s) == 0) return s;
+  return 1;
+}
+
+// Host mirror of the pending-list bookkeeping the memory kernels do on the device.
+void mirror_memory(const ImDims& p, HostUnit& u, int ne) {
+  if (!p.mem || ne <= 0) return;
+  if (ne > p.F) { u.npend = 0; return; }
+  if (u.npend + ne > p.F) u.npend = 0;
+  u.npend += ne;
+}
+
+// phi of the gathered evicted keys (skinny GEMM against the folded Linear_theta), then Eq. 6-7.
+int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max) {
   const ImDims& p = ctx->p;
-  int ne_max = 0;
-  // The fold kernel is always enqueued (its blocks leave at once unless the device flags the step
-  // as a fold), so that a captured sequence of launches stays valid for every later step.
-  const bool direct = true;
-  for (int i = 0; i < call.n_seq; ++i) {
-    HostUnit& u = ctx->hu[(size_t)call.layer * p.S + call.seq[i]];
-    ne_max = std::max(ne_max, std::max(0, u.n - p.B));
+  ImGemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.job[0] = {L.w.Wfh, L.w.Wfl, p.dM, 0, 0};
+  g.n_jobs = 1;
+  g.in[0] = L.sc.evK;
+  g.in_cnt[0] = ne_max;
+  g.in_outer[0] = (long long)p.tail * p.Dkv;
+  g.in_inner[0] = p.Dkv;
+  g.NV = call.n_seq * ne_max;
+  g.K = p.Dkv;
+  g.out_cnt = ne_max;
+  g.out_inner = p.dM;
+  if (ne_max > p.F) {
+    call.phi_large = 1;
+    g.out = L.sc.phi;
+    g.out_outer = (long long)p.tail * p.dM;
+    g.ksplit = 1;
+    g.ks_stride = 0;
+  } else {
+    call.phi_large = 0;
+    g.out = L.sc.phip;
+    g.out_outer = (long long)p.F * p.dM;
+    g.ksplit = call.ksplit_phi;
+    g.ks_stride = (long long)call.n_seq * p.F * p.dM;
   }
-  CKL(im_launch_select(L, call));  // also restarts the pooling of every sequence in the call
-  if (ne_max > 0) {
-    if (p.mem) CKL(im_launch_memory_write(L, call, ne_max, direct));
-    CKL(im_launch_compact(L, call));
-  }
-  for (int i = 0; i < call.n_seq; ++i) {
-    HostUnit& u = ctx->hu[(size_t)call.layer * p.S + call.seq[i]];
-    int ne = std::max(0, u.n - p.B);
-    if (ne > 0) {
-      if (p.mem) {
-        // the device takes the same decision per sequence: fold everything when the list overflows
-        if (u.npend + ne > p.F) u.npend = 0; else u.npend += ne;
-      }
-      u.n = p.B;
-    }
-    u.since = 0;
-  }
+  CKL(im_launch_gemm(L, g));
+  CKL(im_launch_mem_update(L, call, ne_max));
   return IM_OK;
 }
 
@@ -345,39 +365,60 @@ int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, 
   if (chunk_len < 1 || chunk_len > p.max_chunk)
     return fail(IM_ERR_ARG, "chunk_len %d out of range [1,%d]", chunk_len, p.max_chunk);
   if (!x || !q_pre || !k || !v) return fail(IM_ERR_ARG, "null tensor");
-  int n_max = 0;
+  int n_max = 0, ne_max = 0;
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
     if (u.n + chunk_len > p.cap)
       return fail(IM_ERR_CAPACITY, "sequence %d: %d cached + chunk %d exceeds capacity %d", call.seq[i], u.n, chunk_len, p.cap);
     n_max = std::max(n_max, u.n + chunk_len);
+    ne_max = std::max(ne_max, u.n + chunk_len - p.B);
   }
   call.C = chunk_len;
+  call.prefill = 1;
+  call.ksplit = 1;
+  call.ksplit_key = 1;
+  call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
   ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
+  const int NV = n_seq * chunk_len;
+  // pending rank-one terms are folded into M before a compression that cannot append to the list
+  if (p.mem && ne_max > 0) CKL(im_launch_mem_fold(L, call));
   // a0: indexer projections of every chunk token (Sec. 3.1)
-  ImProjJobs jobs;
-  memset(&jobs, 0, sizeof(jobs));
   ImRows r = im_rows(p);
-  jobs.job[0] = {L.w.Uq, (const bf16*)q_pre, p.HI * p.dI, r.uq};
-  jobs.job[1] = {L.w.G, (const bf16*)x, p.HI, r.g};
-  jobs.n_jobs = 2;
-  jobs.Dn = p.D;
-  jobs.NV = n_seq * chunk_len;
-  jobs.out_stride = p.R3;
-  jobs.total_rows = 0;
-  for (int j = 0; j < jobs.n_jobs; ++j) jobs.total_rows += jobs.job[j].rows;
-  CKL(im_launch_proj(L, jobs, L.sc.raw));
-  CKL(im_launch_proj_key(L, x, n_seq * chunk_len));
+  ImGemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
+  g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
+  g.n_jobs = 2;
+  g.in[0] = (const bf16*)q_pre;
+  g.in[1] = (const bf16*)x;
+  for (int k = 0; k < 2; ++k) { g.in_cnt[k] = 1; g.in_outer[k] = p.D; g.in_inner[k] = 0; }
+  g.out = L.sc.raw;
+  g.out_cnt = 1;
+  g.out_outer = p.R3;
+  g.NV = NV;
+  g.K = p.D;
+  g.ksplit = 1;
+  CKL(im_launch_gemm(L, g));
+  CKL(im_launch_proj_key_split(L, x, NV, 1));
   CKL(im_launch_prefill_append(L, call, k, v));
   // a1: pooled importance under the causal mask
   CKL(im_launch_prefill_score(L, call, n_max));
+  // a2: selection (also restarts the pooling); a4: gather the evicted pairs, fill the holes
+  CKL(im_launch_select(L, call));
+  if (ne_max > 0) {
+    CKL(im_launch_gather_move(L, call, ne_max));
+    // a3: memory write
+    if (p.mem && (rc = run_memory_write(ctx, L, call, ne_max))) return rc;
+  }
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
-    u.n += chunk_len;
+    const int ne = std::max(0, u.n + chunk_len - p.B);
+    mirror_memory(p, u, ne);
+    u.n = u.n + chunk_len - ne;
     u.T += chunk_len;
+    u.since = 0;
   }
-  // a2-a4
-  return run_compress(ctx, L, call);
+  return IM_OK;
 }
 
 int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, const void* x, const void* q_pre,
@@ -388,47 +429,68 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   const ImDims& p = ctx->p;
   if (!x || !q_pre || !q || !k_new || !v_new || !out) return fail(IM_ERR_ARG, "null tensor");
   bool due_any = false, due_all = true;
+  int n_max = 0, ne_max = 0;
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
     if (u.n + 1 > p.cap) return fail(IM_ERR_CAPACITY, "sequence %d has no free slot (capacity %d)", call.seq[i], p.cap);
     bool due = (u.since + 1 == p.tau);
     due_any |= due;
     due_all &= due;
+    n_max = std::max(n_max, u.n + 1);
+    ne_max = std::max(ne_max, u.n + 1 - p.B);
   }
   if (due_any != due_all)
     return fail(IM_ERR_ARG, "sequences of one decode call must be at the same phase of the compression interval");
+  const bool due = due_all;
+  if (!due) ne_max = 0;
+  call.C = 1;
+  call.prefill = 0;
+  call.ksplit = pick_ksplit(p.D, IM_KSPLIT);
+  call.ksplit_key = (p.D % (8 * IM_KSPLIT_KEY) == 0) ? IM_KSPLIT_KEY : 1;
+  call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
   ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
-  // a0: projections (Sec. 3.1 features, phi(q) of Eq. 5, gate of Eq. 4)
-  ImProjJobs jobs;
-  memset(&jobs, 0, sizeof(jobs));
+  if (p.mem && ne_max > 0) CKL(im_launch_mem_fold(L, call));
+  // a0: projections (Sec. 3.1 features, phi(q) of Eq. 5, gate of Eq. 4) as K-split partial sums
   ImRows r = im_rows(p);
-  jobs.job[0] = {L.w.Uq, (const bf16*)q_pre, p.HI * p.dI, r.uq};
-  jobs.job[1] = {L.w.G, (const bf16*)x, p.HI, r.g};
-  jobs.job[2] = {L.w.Wt, (const bf16*)q, p.dM, r.theta};
-  jobs.job[3] = {L.w.wg, (const bf16*)q, 1, r.wg};
-  jobs.n_jobs = p.mem ? 4 : 2;
-  jobs.Dn = p.D;
-  jobs.NV = n_seq;
-  jobs.out_stride = p.R5;
-  jobs.total_rows = 0;
-  for (int j = 0; j < jobs.n_jobs; ++j) jobs.total_rows += jobs.job[j].rows;
-  CKL(im_launch_proj(L, jobs, L.sc.raw));
-  CKL(im_launch_proj_key(L, x, n_seq));
-  // append + a1: score every cached entry with the new query
-  CKL(im_launch_decode_index(L, call, k_new, v_new));
-  int n_max = 0;
+  ImGemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
+  g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
+  g.job[2] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
+  g.job[3] = {L.w.wg, nullptr, 1, r.wg, 2};
+  g.n_jobs = p.mem ? 4 : 2;
+  g.in[0] = (const bf16*)q_pre;
+  g.in[1] = (const bf16*)x;
+  g.in[2] = (const bf16*)q;
+  for (int k = 0; k < 3; ++k) { g.in_cnt[k] = 1; g.in_outer[k] = p.D; g.in_inner[k] = 0; }
+  g.out = L.sc.raw;
+  g.out_cnt = 1;
+  g.out_outer = p.R5;
+  g.ks_stride = (long long)n_seq * p.R5;
+  g.NV = n_seq;
+  g.K = p.D;
+  g.ksplit = call.ksplit;
+  CKL(im_launch_gemm(L, g));
+  CKL(im_launch_proj_key_split(L, x, n_seq, call.ksplit_key));
+  // append + a1 (+ a2, gather, a4 when the evicted set is small enough for one block per sequence)
+  const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
+  CKL(im_launch_decode_front(L, call, k_new, v_new, fused ? 1 : 0, n_max));
+  if (due && !fused) {
+    CKL(im_launch_select(L, call));
+    if (ne_max > 0) CKL(im_launch_gather_move(L, call, ne_max));
+  }
+  // a3: memory write
+  if (due && ne_max > 0 && p.mem && (rc = run_memory_write(ctx, L, call, ne_max))) return rc;
+  int n_att = 0;
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
-    u.n += 1;
+    const int ne = due ? std::max(0, u.n + 1 - p.B) : 0;
+    mirror_memory(p, u, ne);
+    u.n = u.n + 1 - ne;
     u.T += 1;
-    u.since += 1;
+    u.since = due ? 0 : u.since + 1;
+    n_att = std::max(n_att, u.n);
   }
-  // a2-a4 every tau-th token
-  if (due_all) {
-    rc = run_compress(ctx, L, call);
-    if (rc) return rc;
-  }
-  for (int i = 0; i < n_seq; ++i) n_max = std::max(n_max, ctx->hu[(size_t)layer * p.S + call.seq[i]].n);
   // a5-a6: attention over the retained entries + gated readout
   const bool prof = ctx->prof_used + 2 <= ctx->prof_ev.size();
   if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], L.stream));
@@ -436,7 +498,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     if (p.mem) CKL(im_launch_readout(L, call));
     CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, out, ctx->n_ctas));
   } else {
-    CKL(im_launch_attention(L, call, q, out, n_max));
+    CKL(im_launch_attention(L, call, q, out, n_att));
   }
   if (prof) {
     CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], L.stream));

@@ -114,8 +114,9 @@ __global__ void k_attn_merge(ImDims p, ImState st, ImWeights w, ImScratch sc, Im
   float res = o;
   if (p.mem) {
     const ImRows r = im_rows(p);
-    const float* raw = sc.raw + (size_t)i * p.R5;
-    const float* phiq = raw + r.theta;
+    extern __shared__ float phiq[];  // [dM] phi(q), summed over the K-split partials
+    for (int m = tid; m < p.dM; m += blockDim.x) phiq[m] = im_raw_sum(p, sc, call, i, r.theta + m);
+    __syncthreads();
     const int np = min(ctr[CTR_NPEND], p.F);
     // den = sum_m phi_q[m]^2 b[m] + eps
     float part_den = 0.f;
@@ -146,7 +147,7 @@ __global__ void k_attn_merge(ImDims p, ImState st, ImWeights w, ImScratch sc, Im
       for (int m = 0; m < p.dM; ++m) mv = fmaf(phiq[m], Mh[(size_t)m * p.Dkv + col], mv);
       for (int pp = 0; pp < np; ++pp) mv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mv);
       mv = st.cscale[u] * mv / s_scalar[0];
-      const float gate = 1.0f / (1.0f + expf(-(raw[r.wg] + w.bg[0])));
+      const float gate = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
       res = fmaf(gate, mv, o);
     }
   }
@@ -167,8 +168,8 @@ cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const voi
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   dim3 grid2(p.H, call.n_seq);
-  if (p.out_f32) k_attn_merge<float><<<grid2, 256, 0, L.stream>>>(p, L.st, L.w, L.sc, call, (float*)out);
-  else k_attn_merge<bf16><<<grid2, 256, 0, L.stream>>>(p, L.st, L.w, L.sc, call, (bf16*)out);
+  if (p.out_f32) k_attn_merge<float><<<grid2, 256, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, (float*)out);
+  else k_attn_merge<bf16><<<grid2, 256, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, (bf16*)out);
   ++*L.launches;
   return cudaGetLastError();
 }

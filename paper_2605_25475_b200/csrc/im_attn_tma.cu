@@ -335,7 +335,7 @@ __global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const ImRows r = im_rows(p);
   const int m0 = rc * R_ROWS, mcnt = min(R_ROWS, p.dM - m0);
-  if (threadIdx.x < R_ROWS) s_phi[threadIdx.x] = threadIdx.x < mcnt ? sc.raw[(size_t)i * p.R5 + r.theta + m0 + threadIdx.x] : 0.f;
+  if (threadIdx.x < R_ROWS) s_phi[threadIdx.x] = threadIdx.x < mcnt ? im_raw_sum(p, sc, call, i, r.theta + m0 + threadIdx.x) : 0.f;
   __syncthreads();
   const float* Mh = st.Mhat + (u * p.dM + m0) * (size_t)p.Dkv;
   const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
@@ -394,8 +394,9 @@ __global__ void __launch_bounds__(DH) k_attn_merge_rows(ImDims p, ImState st, Im
   float mkv = 0.f, gate = 0.f;
   if (p.mem) {
     const ImRows r = im_rows(p);
-    const float* raw = sc.raw + (size_t)i * p.R5;
-    const float* phiq = raw + r.theta;
+    extern __shared__ float phiq[];  // [dM] phi(q), summed over the K-split partials
+    for (int m = c; m < p.dM; m += DH) phiq[m] = im_raw_sum(p, sc, call, i, r.theta + m);
+    __syncthreads();
     const int np = min(ctr[CTR_NPEND], p.F);
     float part_den = 0.f;
     for (int m = c; m < p.dM; m += DH) part_den = fmaf(phiq[m] * phiq[m], st.bvec[u * p.dM + m], part_den);
@@ -423,7 +424,7 @@ __global__ void __launch_bounds__(DH) k_attn_merge_rows(ImDims p, ImState st, Im
     for (int k = 0; k < nchunk; ++k) mkv += rp[(size_t)k * p.Dkv];
     for (int pp = 0; pp < np; ++pp) mkv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mkv);
     mkv = st.cscale[u] * mkv / s_den;
-    gate = 1.0f / (1.0f + expf(-(raw[r.wg] + w.bg[0])));
+    gate = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
   }
   for (int hh = 0; hh < p.Gq; ++hh) {
     float res = 0.f;
@@ -515,11 +516,11 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   if (e != cudaSuccess) return e;
   dim3 grid(p.Hkv, call.n_seq);
   if (p.d == 64) {
-    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, 64, 0, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
-    else k_attn_merge_rows<64, bf16><<<grid, 64, 0, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
+    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, 64, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
+    else k_attn_merge_rows<64, bf16><<<grid, 64, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
   } else {
-    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, 128, 0, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
-    else k_attn_merge_rows<128, bf16><<<grid, 128, 0, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
+    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, 128, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
+    else k_attn_merge_rows<128, bf16><<<grid, 128, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
   }
   ++*L.launches;
   return cudaGetLastError();

@@ -1,0 +1,299 @@
+// Decode front end of one layer call, one thread block per sequence: finish the indexer features
+// from the K-split projection partials, append the token, score every cached entry with the new
+// query (a1), and - when the compression is due and small - select (a2), gather the evicted pairs
+// for the memory write and compact the cache (a4) in the same kernel.  Also the stand-alone gather
+// and move kernels used after k_select when the evicted set is large (prefill).
+#include "im_internal.cuh"
+
+namespace {
+
+constexpr float NEG_INF = -__builtin_huge_valf();
+constexpr int FRONT_THREADS = 512;
+
+struct FrontShared {
+  double kd[64];             // indexer key before normalisation (float64)
+  float q[64 * 64];          // q features [HI][dI] (only HI*dI used)
+  float alpha[64];
+  float knew[64];            // the new token's cached (rounded) indexer key
+  unsigned long long wmin[FRONT_THREADS / 32];
+  int wslot[FRONT_THREADS / 32];
+  int ev[IM_FRONT_MAX_NE];   // evicted slots, ascending after the sort
+  int surv[IM_FRONT_MAX_NE]; // retained entries found at or above the budget, ascending
+  int nh;
+};
+
+// grid = n_seq, block = FRONT_THREADS, dynamic smem = keys of the selection (8 bytes per entry) when
+// do_select, else 0.
+__global__ void __launch_bounds__(FRONT_THREADS)
+k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __restrict__ k_new,
+               const bf16* __restrict__ v_new, int do_select) {
+  extern __shared__ __align__(16) unsigned long long s_key[];
+  __shared__ FrontShared sh;
+  const int i = blockIdx.x, tid = threadIdx.x;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  const int n = ctr[CTR_N], T = ctr[CTR_T], since = ctr[CTR_SINCE];
+  if (n < 0 || n >= p.cap) {  // never write out of bounds: flag and leave
+    if (tid == 0) atomicOr(st.status, ST_COUNT);
+    return;
+  }
+  const ImRows r = im_rows(p);
+  const int nq = p.HI * p.dI;
+  // ---- finish the projections: sum the K-split partials in a fixed order
+  for (int k = tid; k < nq; k += FRONT_THREADS) {
+    sh.q[k] = im_raw_sum(p, sc, call, i, r.uq + k);
+  }
+  for (int k = tid; k < p.HI; k += FRONT_THREADS) {
+    sh.alpha[k] = im_raw_sum(p, sc, call, i, r.g + k) * (1.0f / sqrtf((float)p.HI * (float)p.dI));
+  }
+  for (int k = tid; k < p.dI; k += FRONT_THREADS) {
+    double s = 0.0;
+    for (int ks = 0; ks < call.ksplit_key; ++ks) s += sc.keyp[((size_t)ks * call.n_seq + i) * p.dI + k];
+    sh.kd[k] = s;
+  }
+  __syncthreads();
+  // RMSNorm of the q features per indexer head (float32) and of the key (float64, then bf16)
+  for (int h = tid; h < p.HI; h += FRONT_THREADS) {
+    float* y = sh.q + h * p.dI;
+    float ms = 0.f;
+    for (int k = 0; k < p.dI; ++k) ms = fmaf(y[k], y[k], ms);
+    const float inv = 1.0f / sqrtf(ms / (float)p.dI + p.norm_eps);
+    for (int k = 0; k < p.dI; ++k) y[k] *= inv;
+  }
+  if (tid >= 64 && tid < 64 + p.dI) {
+    const int k = tid - 64;
+    double ms = 0.0;
+    for (int j = 0; j < p.dI; ++j) ms += sh.kd[j] * sh.kd[j];
+    const double inv = 1.0 / sqrt(ms / (double)p.dI + (double)p.norm_eps);
+    const bf16 b = __double2bfloat16(sh.kd[k] * inv);
+    st.kidx[(u * p.cap + n) * p.dI + k] = b;
+    sh.knew[k] = __bfloat162float(b);
+  }
+  // ---- append K / V / position in slot n
+  const int dv = p.d / 8;
+  for (int k = tid; k < p.Hkv * dv; k += FRONT_THREADS) {
+    const int h = k / dv, c = k % dv;
+    const size_t row = ((u * p.Hkv + h) * p.cap + n) * p.d;
+    reinterpret_cast<uint4*>(st.Kc + row)[c] = reinterpret_cast<const uint4*>(k_new + (size_t)i * p.Dkv + h * p.d)[c];
+    reinterpret_cast<uint4*>(st.Vc + row)[c] = reinterpret_cast<const uint4*>(v_new + (size_t)i * p.Dkv + h * p.d)[c];
+  }
+  if (tid == 0) st.pos[u * p.cap + n] = T;
+  __syncthreads();
+  // ---- a1: A_t = sum_h alpha_h act(q_h . k_t), pooled by max into the importance
+  const int n1 = n + 1;
+  const bool due = (since + 1 == p.tau);
+  const bool select_here = do_select && due;
+  float* imp = st.imp + u * p.cap;
+  int32_t* pos = st.pos + u * p.cap;
+  bool bad = false;
+  for (int t = tid; t < n1; t += FRONT_THREADS) {
+    float kk[64];
+    if (t == n) {
+      for (int k = 0; k < p.dI; ++k) kk[k] = sh.knew[k];
+    } else if ((p.dI & 7) == 0) {
+      const uint4* row = reinterpret_cast<const uint4*>(st.kidx + (u * p.cap + t) * p.dI);
+      for (int c = 0; c < p.dI / 8; ++c) {
+        const uint4 w = row[c];
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          kk[c * 8 + 2 * k] = __uint_as_float(ww[k] << 16);
+          kk[c * 8 + 2 * k + 1] = __uint_as_float(ww[k] & 0xffff0000u);
+        }
+      }
+    } else {
+      const bf16* row = st.kidx + (u * p.cap + t) * p.dI;
+      for (int k = 0; k < p.dI; ++k) kk[k] = __bfloat162float(row[k]);
+    }
+    float A = 0.f;
+    for (int h = 0; h < p.HI; ++h) {
+      float z = 0.f;
+      for (int k = 0; k < p.dI; ++k) z = fmaf(sh.q[h * p.dI + k], kk[k], z);
+      if (p.act == 0) z = fmaxf(z, 0.f);
+      A = fmaf(sh.alpha[h], z, A);
+    }
+    bad |= !isfinite(A);
+    const float old = (t == n) ? NEG_INF : imp[t];
+    const float pooled = fmaxf(old, A);
+    const int ps = (t == n) ? T : pos[t];
+    if (due) {  // what the selection sees (parity export), then the pooling restarts
+      st.sel_pos[u * p.cap + t] = ps;
+      st.sel_imp[u * p.cap + t] = pooled;
+    }
+    if (select_here) {
+      s_key[t] = im_select_key(pooled, ps, p.n_sink);
+      imp[t] = NEG_INF;
+    } else {
+      imp[t] = pooled;
+    }
+  }
+  if (bad) atomicOr(st.status, ST_NONFINITE);
+  if (!select_here) {
+    // either not due, or the selection runs in the kernels that follow (they read imp / pos)
+    if (tid == 0) {
+      ctr[CTR_N] = n1;
+      ctr[CTR_T] = T + 1;
+      ctr[CTR_SINCE] = since + 1;
+      ctr[CTR_NEVICT] = 0;
+    }
+    return;
+  }
+  __syncthreads();
+  // ---- a2: the ne entries with the smallest keys leave (keys are distinct)
+  const int ne = n1 > p.B ? n1 - p.B : 0;
+  if (ne > IM_FRONT_MAX_NE) {  // the host never asks for this
+    if (tid == 0) atomicOr(st.status, ST_COUNT);
+    return;
+  }
+  for (int e = 0; e < ne; ++e) {
+    unsigned long long best = ~0ull;
+    int slot = -1;
+    for (int t = tid; t < n1; t += FRONT_THREADS) {
+      const unsigned long long k = s_key[t];
+      if (k < best) { best = k; slot = t; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int os = __shfl_xor_sync(0xffffffffu, slot, o);
+      if (ob < best) { best = ob; slot = os; }
+    }
+    if ((tid & 31) == 0) { sh.wmin[tid >> 5] = best; sh.wslot[tid >> 5] = slot; }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < FRONT_THREADS / 32; ++w)
+        if (sh.wmin[w] < best) { best = sh.wmin[w]; slot = sh.wslot[w]; }
+      sh.ev[e] = slot;
+      s_key[slot] = ~0ull;  // a real key never has this value: its low word is ~position with position >= 0
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    // ascending slot order; holes below the budget pair with the retained entries above it
+    for (int a = 1; a < ne; ++a) {
+      const int v = sh.ev[a];
+      int b = a - 1;
+      while (b >= 0 && sh.ev[b] > v) { sh.ev[b + 1] = sh.ev[b]; --b; }
+      sh.ev[b + 1] = v;
+    }
+    int nh = 0, ns = 0;
+    for (int a = 0; a < ne; ++a) nh += sh.ev[a] < p.B ? 1 : 0;
+    for (int t = p.B; t < n1; ++t) {
+      bool gone = false;
+      for (int a = 0; a < ne; ++a) gone |= sh.ev[a] == t;
+      if (!gone) sh.surv[ns++] = t;
+    }
+    if (ns != nh) atomicOr(st.status, ST_COUNT);
+    sh.nh = min(nh, ns);
+    for (int a = 0; a < ne; ++a) {
+      st.ev_slot[u * p.tail + a] = sh.ev[a];
+      st.ev_pos[u * p.tail + a] = (sh.ev[a] == n) ? T : pos[sh.ev[a]];
+    }
+  }
+  __syncthreads();
+  // ---- gather the evicted pairs for the memory write (a3 reads them from here)
+  for (int k = tid; k < ne * p.Hkv * dv; k += FRONT_THREADS) {
+    const int e = k / (p.Hkv * dv), rem = k % (p.Hkv * dv), h = rem / dv, c = rem % dv;
+    const size_t row = ((u * p.Hkv + h) * p.cap + sh.ev[e]) * p.d;
+    const size_t dst = ((size_t)i * p.tail + e) * p.Dkv + h * p.d;
+    reinterpret_cast<uint4*>(sc.evK + dst)[c] = reinterpret_cast<const uint4*>(st.Kc + row)[c];
+    reinterpret_cast<uint4*>(sc.evV + dst)[c] = reinterpret_cast<const uint4*>(st.Vc + row)[c];
+  }
+  __syncthreads();
+  // ---- a4: fill the holes below the budget with the retained entries from above it
+  const int nh = sh.nh;
+  for (int k = tid; k < nh * p.Hkv * dv; k += FRONT_THREADS) {
+    const int j = k / (p.Hkv * dv), rem = k % (p.Hkv * dv), h = rem / dv, c = rem % dv;
+    const size_t base = (u * p.Hkv + h) * p.cap;
+    reinterpret_cast<uint4*>(st.Kc + (base + sh.ev[j]) * p.d)[c] = reinterpret_cast<const uint4*>(st.Kc + (base + sh.surv[j]) * p.d)[c];
+    reinterpret_cast<uint4*>(st.Vc + (base + sh.ev[j]) * p.d)[c] = reinterpret_cast<const uint4*>(st.Vc + (base + sh.surv[j]) * p.d)[c];
+  }
+  for (int k = tid; k < nh * p.dI; k += FRONT_THREADS) {
+    const int j = k / p.dI, c = k % p.dI;
+    st.kidx[(u * p.cap + sh.ev[j]) * p.dI + c] = st.kidx[(u * p.cap + sh.surv[j]) * p.dI + c];
+  }
+  __syncthreads();  // ev_pos above read pos[] of the evicted slots before they are overwritten here
+  for (int j = tid; j < nh; j += FRONT_THREADS) pos[sh.ev[j]] = (sh.surv[j] == n) ? T : pos[sh.surv[j]];
+  if (tid == 0) {
+    ctr[CTR_N] = n1 - ne;
+    ctr[CTR_T] = T + 1;
+    ctr[CTR_SINCE] = 0;
+    ctr[CTR_NSEL] = n1;
+    ctr[CTR_NEVICT] = ne;
+    if (ne > 0) ctr[CTR_EVSTEPS] = ctr[CTR_EVSTEPS] + 1;
+  }
+}
+
+// Stand-alone versions for large evicted sets (after k_select): gather the evicted pairs, then move
+// the retained entries from above the budget into the holes.  Two kernels: every gather must be done
+// before a move overwrites an evicted slot.
+// grid = (ceil(ne_max / 4), n_seq), block = 256.
+__global__ void __launch_bounds__(256) k_gather_evicted(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  const int i = blockIdx.y;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
+  const int e0 = blockIdx.x * 4;
+  if (e0 >= ne) return;
+  const int cnt = min(4, ne - e0);
+  const int dv = p.d / 8;
+  for (int k = threadIdx.x; k < cnt * p.Hkv * dv; k += blockDim.x) {
+    const int e = e0 + k / (p.Hkv * dv), rem = k % (p.Hkv * dv), h = rem / dv, c = rem % dv;
+    const int slot = st.ev_slot[u * p.tail + e];
+    const size_t row = ((u * p.Hkv + h) * p.cap + slot) * p.d;
+    const size_t dst = ((size_t)i * p.tail + e) * p.Dkv + h * p.d;
+    reinterpret_cast<uint4*>(sc.evK + dst)[c] = reinterpret_cast<const uint4*>(st.Kc + row)[c];
+    reinterpret_cast<uint4*>(sc.evV + dst)[c] = reinterpret_cast<const uint4*>(st.Vc + row)[c];
+  }
+}
+
+__global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  const int i = blockIdx.y;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
+  const int nh = min(sc.nhole[i], ne);
+  const int j0 = blockIdx.x * 4;
+  if (ne <= 0 || j0 >= nh) return;
+  const int cnt = min(4, nh - j0);
+  const int dv = p.d / 8;
+  const int32_t* evs = st.ev_slot + u * p.tail;
+  const int32_t* surv = sc.surv + (size_t)i * p.tail;
+  for (int k = threadIdx.x; k < cnt * p.Hkv * dv; k += blockDim.x) {
+    const int j = j0 + k / (p.Hkv * dv), rem = k % (p.Hkv * dv), h = rem / dv, c = rem % dv;
+    const size_t base = (u * p.Hkv + h) * p.cap;
+    reinterpret_cast<uint4*>(st.Kc + (base + evs[j]) * p.d)[c] = reinterpret_cast<const uint4*>(st.Kc + (base + surv[j]) * p.d)[c];
+    reinterpret_cast<uint4*>(st.Vc + (base + evs[j]) * p.d)[c] = reinterpret_cast<const uint4*>(st.Vc + (base + surv[j]) * p.d)[c];
+  }
+  for (int k = threadIdx.x; k < cnt * p.dI; k += blockDim.x) {
+    const int j = j0 + k / p.dI, c = k % p.dI;
+    st.kidx[(u * p.cap + evs[j]) * p.dI + c] = st.kidx[(u * p.cap + surv[j]) * p.dI + c];
+  }
+  for (int j = j0 + threadIdx.x; j < j0 + cnt; j += blockDim.x) st.pos[u * p.cap + evs[j]] = st.pos[u * p.cap + surv[j]];
+}
+
+}  // namespace
+
+cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
+                                   int do_select, int n_max) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(k_decode_front, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const size_t smem = do_select ? (size_t)n_max * 8 : 0;
+  k_decode_front<<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, (const bf16*)k_new,
+                                                                (const bf16*)v_new, do_select);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max) {
+  dim3 grid((ne_max + 3) / 4, call.n_seq);
+  k_gather_evicted<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
+  ++*L.launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  k_move_survivors<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
+  ++*L.launches;
+  return cudaGetLastError();
+}

@@ -1,0 +1,173 @@
+// Skinny GEMMs of the path (a0 projections, phi of evicted keys): out[v][r] = sum_k W[r][k] * in[v][k]
+// with a handful to a few thousand weight rows and 1 .. 65536 input vectors, bf16 operands, float32
+// accumulation on mma.sync m16n8k16.  Weight-streaming bound in decode (every weight byte is read
+// once per call), so the grid is (16-row tiles) x (K splits) to spread the stream over the SMs; the
+// K-split partial sums are added by the consumer in a fixed order (deterministic).
+// Also here: the float64 indexer-key projection, split over K the same way.
+#include "im_internal.cuh"
+
+namespace {
+
+constexpr int KC = 512;                 // K elements staged per round
+constexpr int ROW_BYTES = KC * 2 + 16;  // padded smem row: consecutive rows shift by one 16-byte bank group
+constexpr int VB = 32;                  // vectors per CTA (4 warps x 8)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;  // src-size 0: the 16 bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x2(uint32_t addr, uint32_t& r0, uint32_t& r1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ const bf16* vec_ptr(const ImGemmArgs& a, int sel, long long v) {
+  return a.in[sel] + (v / a.in_cnt[sel]) * a.in_outer[sel] + (v % a.in_cnt[sel]) * a.in_inner[sel];
+}
+
+// grid = (row tiles over all jobs, ksplit, ceil(NV / 32)), block = 128, dynamic smem = 64 * ROW_BYTES
+__global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  unsigned char* sA = smem;                    // [16][ROW_BYTES]
+  unsigned char* sA2 = smem + 16 * ROW_BYTES;  // [16][ROW_BYTES] second weight term
+  unsigned char* sB = smem + 32 * ROW_BYTES;   // [32][ROW_BYTES]
+  int tile = blockIdx.x, j = 0;
+  while (j + 1 < a.n_jobs && tile >= (a.job[j].rows + 15) / 16) {
+    tile -= (a.job[j].rows + 15) / 16;
+    ++j;
+  }
+  const ImGemmJob job = a.job[j];
+  const int r0 = tile * 16;
+  const int ks = blockIdx.y;
+  const int kspan = a.K / a.ksplit;
+  const int kbeg = ks * kspan;
+  const long long v0 = (long long)blockIdx.z * VB;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int k0 = 0; k0 < kspan; k0 += KC) {
+    const int kc = min(KC, kspan - k0);     // multiple of 16
+    const int chunks = kc / 8;              // 16-byte chunks per row
+    __syncthreads();                        // previous round's reads are done
+    for (int idx = threadIdx.x; idx < 16 * chunks; idx += blockDim.x) {
+      const int r = idx / chunks, c = idx % chunks;
+      const bool valid = r0 + r < job.rows;
+      const bf16* src = job.W + (size_t)(valid ? r0 + r : 0) * a.K + kbeg + k0 + c * 8;
+      cp_async16(smem_u32(sA + r * ROW_BYTES + c * 16), src, valid);
+      if (job.W2) {
+        const bf16* src2 = job.W2 + (size_t)(valid ? r0 + r : 0) * a.K + kbeg + k0 + c * 8;
+        cp_async16(smem_u32(sA2 + r * ROW_BYTES + c * 16), src2, valid);
+      }
+    }
+    for (int idx = threadIdx.x; idx < VB * chunks; idx += blockDim.x) {
+      const int r = idx / chunks, c = idx % chunks;
+      const bool valid = v0 + r < a.NV;
+      const bf16* src = vec_ptr(a, job.in_sel, valid ? v0 + r : 0) + kbeg + k0 + c * 8;
+      cp_async16(smem_u32(sB + r * ROW_BYTES + c * 16), src, valid);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    // A fragment rows: lanes 0-7 rows 0-7 (k 0-7), 8-15 rows 8-15 (k 0-7), 16-23 rows 0-7 (k 8-15), 24-31 rows 8-15 (k 8-15)
+    const uint32_t aBase = smem_u32(sA) + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROW_BYTES + (lane >> 4) * 16;
+    // B fragment rows (= vectors): lanes 0-7 k 0-7, lanes 8-15 k 8-15 (lanes 16-31 ignored by .x2 but must be valid)
+    const uint32_t bBase = smem_u32(sB) + (warp * 8 + (lane & 7)) * ROW_BYTES + ((lane >> 3) & 1) * 16;
+    for (int kk = 0; kk < kc; kk += 16) {
+      uint32_t a0, a1, a2, a3, b0, b1;
+      ldsm_x4(aBase + kk * 2, a0, a1, a2, a3);
+      ldsm_x2(bBase + kk * 2, b0, b1);
+      mma_bf16(acc, a0, a1, a2, a3, b0, b1);
+      if (job.W2) {
+        ldsm_x4(aBase + 16 * ROW_BYTES + kk * 2, a0, a1, a2, a3);
+        mma_bf16(acc, a0, a1, a2, a3, b0, b1);
+      }
+    }
+  }
+  // C fragment: rows g / g+8 (weight rows), columns 2t / 2t+1 (vectors of this warp)
+  const long long vA = v0 + warp * 8 + 2 * t, vB = vA + 1;
+  float* outk = a.out + (size_t)ks * a.ks_stride;
+  const int rA = r0 + g, rB = r0 + g + 8;
+  if (vA < a.NV) {
+    float* o = outk + (vA / a.out_cnt) * a.out_outer + (vA % a.out_cnt) * a.out_inner + job.row0;
+    if (rA < job.rows) o[rA] = acc[0];
+    if (rB < job.rows) o[rB] = acc[2];
+  }
+  if (vB < a.NV) {
+    float* o = outk + (vB / a.out_cnt) * a.out_outer + (vB % a.out_cnt) * a.out_inner + job.row0;
+    if (rA < job.rows) o[rA] = acc[1];
+    if (rB < job.rows) o[rB] = acc[3];
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Indexer key projection U_k x in float64 (the cached key is a quantised code: the value that gets
+// rounded to bf16 must not depend on the summation order).  K is split over blockIdx.x; one warp
+// per vector.  keyp[ks][v][r] receives the partial sums.
+// grid = (ksplit, ceil(NV / 8)), block = 256.
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __restrict__ Uk, const bf16* __restrict__ x,
+                                                         int NV, int ksplit, double* __restrict__ keyp) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ks = blockIdx.x;
+  const long long v = (long long)blockIdx.y * 8 + warp;
+  if (v >= NV) return;
+  const int kspan = p.D / ksplit, kbeg = ks * kspan;  // kspan is a multiple of 8
+  const uint4* x4 = reinterpret_cast<const uint4*>(x + (size_t)v * p.D + kbeg);
+  double* dst = keyp + ((size_t)ks * NV + v) * p.dI;
+  for (int r = 0; r < p.dI; ++r) {
+    const uint4* w4 = reinterpret_cast<const uint4*>(Uk + (size_t)r * p.D + kbeg);
+    double acc = 0.0;
+    for (int c = lane; c < kspan / 8; c += 32) {
+      const uint4 a = w4[c], b = x4[c];
+      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        // a product of two bf16 values is exact in float32
+        acc += (double)(__uint_as_float(aw[k] << 16) * __uint_as_float(bw[k] << 16));
+        acc += (double)(__uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u));
+      }
+    }
+    acc = warp_sum_d(acc);
+    if (lane == 0) dst[r] = acc;
+  }
+}
+
+}  // namespace
+
+cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a) {
+  static bool attr_done = false;
+  const int smem = 64 * ROW_BYTES;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(k_skinny_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  int tiles = 0;
+  for (int j = 0; j < a.n_jobs; ++j) tiles += (a.job[j].rows + 15) / 16;
+  dim3 grid(tiles, a.ksplit, (unsigned)((a.NV + VB - 1) / VB));
+  k_skinny_gemm<<<grid, 128, smem, L.stream>>>(a);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, int ksplit) {
+  dim3 grid(ksplit, (NV + 7) / 8);
+  k_proj_key_split<<<grid, 256, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
+  ++*L.launches;
+  return cudaGetLastError();
+}

@@ -12,85 +12,8 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// ------------------------------------------------------------------------------------------------
-// a0: out[v][row0 + r] = sum_i W[r][i] * in[v][i]   (bf16 inputs, float32 accumulation)
-// One warp per (row, vector).  grid = (total_rows, ceil(NV / 8)), block = 256 (8 warps = 8 vectors).
-__global__ void k_proj(ImProjJobs jobs, float* __restrict__ out) {
-  int r = blockIdx.x, j = 0;  // blockIdx.x enumerates the rows of all jobs back to back
-  while (j + 1 < jobs.n_jobs && r >= jobs.job[j].rows) {
-    r -= jobs.job[j].rows;
-    ++j;
-  }
-  const ImProjJob job = jobs.job[j];
-  const int row = job.row0 + r;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int v = blockIdx.y * 8 + warp;
-  if (v >= jobs.NV) return;
-  const int Dn = jobs.Dn;
-  const uint4* w4 = reinterpret_cast<const uint4*>(job.W + (size_t)r * Dn);
-  const uint4* x4 = reinterpret_cast<const uint4*>(job.in + (size_t)v * Dn);
-  float acc = 0.f;
-  for (int c = lane; c < Dn / 8; c += 32) {
-    uint4 a = w4[c], b = x4[c];
-    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      acc = fmaf(__uint_as_float(aw[k] << 16), __uint_as_float(bw[k] << 16), acc);
-      acc = fmaf(__uint_as_float(aw[k] & 0xffff0000u), __uint_as_float(bw[k] & 0xffff0000u), acc);
-    }
-  }
-  acc = warp_sum(acc);
-  if (lane == 0) out[(size_t)v * jobs.out_stride + row] = acc;
-}
-
-// ------------------------------------------------------------------------------------------------
-// Indexer key of one token: k = bf16( RMSNorm(U_k x) )  (Sec. 3.1).  The cached key is a quantised
-// code, so the value that gets rounded is computed in float64: the bf16 bits then do not depend on
-// the summation order and agree with any other float64 evaluation.
-// One warp per token.  grid = ceil(NV / 4), block = 128.
-__device__ __forceinline__ double warp_sum_d(double v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-__global__ void k_proj_key(ImDims p, const bf16* __restrict__ Uk, const bf16* __restrict__ x, int NV,
-                           bf16* __restrict__ kidx_new) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int v = blockIdx.x * 4 + warp;
-  if (v >= NV) return;
-  const uint4* x4 = reinterpret_cast<const uint4*>(x + (size_t)v * p.D);
-  double ms = 0.0;
-  double mine = 0.0;  // lane r keeps u[r] (d_I <= 64: two rounds)
-  double mine2 = 0.0;
-  for (int r = 0; r < p.dI; ++r) {
-    const uint4* w4 = reinterpret_cast<const uint4*>(Uk + (size_t)r * p.D);
-    double acc = 0.0;
-    for (int c = lane; c < p.D / 8; c += 32) {
-      const uint4 a = w4[c], b = x4[c];
-      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        // the product of two bf16 values is exact in float32
-        acc += (double)(__uint_as_float(aw[k] << 16) * __uint_as_float(bw[k] << 16));
-        acc += (double)(__uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u));
-      }
-    }
-    acc = warp_sum_d(acc);
-    ms += acc * acc;
-    if (lane == (r & 31)) {
-      if (r < 32) mine = acc; else mine2 = acc;
-    }
-  }
-  const double inv = 1.0 / sqrt(ms / (double)p.dI + (double)p.norm_eps);
-  if (lane < p.dI) kidx_new[(size_t)v * p.dI + lane] = __double2bfloat16(mine * inv);
-  if (lane + 32 < p.dI) kidx_new[(size_t)v * p.dI + lane + 32] = __double2bfloat16(mine2 * inv);
-}
-
-// ------------------------------------------------------------------------------------------------
-// RMSNorm pieces shared by decode and prefill: finalise one token's raw projections in place.
-//   raw[uq ..]  -> q features, RMS-normalised per indexer head
-//   raw[g ..]   -> alpha = G x / sqrt(H_I d_I)
-// Executed by one warp; lanes stride over heads / elements.
+// RMSNorm of one token's raw q features per indexer head, in place, and alpha = G x / sqrt(H_I d_I)
+// (Sec. 3.1).  Executed by one warp; lanes stride over heads.
 __device__ void finalize_features(const ImDims& p, float* raw, int lane) {
   const ImRows r = im_rows(p);
   for (int h = lane; h < p.HI; h += 32) {
@@ -117,77 +40,8 @@ __device__ __forceinline__ float index_score(const ImDims& p, const float* __res
   return A;
 }
 
-// ------------------------------------------------------------------------------------------------
-// decode: append the token and pool the new query's scores into every cached entry.
-// grid = n_seq, block = 256.
-__global__ void k_decode_index(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __restrict__ k_new,
-                               const bf16* __restrict__ v_new) {
-  extern __shared__ float smem[];
-  float* s_raw = smem;  // [R3]
-  const int i = blockIdx.x;
-  const int seq = call.seq[i];
-  const size_t u = (size_t)call.layer * p.S + seq;
-  int32_t* ctr = st.ctr + u * CTR_STRIDE;
-  const int n = ctr[CTR_N];
-  const int T = ctr[CTR_T];
-  const ImRows r = im_rows(p);
-  const int tid = threadIdx.x;
-  if (n < 0 || n >= p.cap) {  // never write out of bounds: flag and leave
-    if (tid == 0) atomicOr(st.status, ST_COUNT);
-    return;
-  }
-  float* raw = sc.raw + (size_t)i * p.R5;
-  for (int k = tid; k < p.R3; k += blockDim.x) s_raw[k] = raw[k];
-  __syncthreads();
-  if (tid < 32) finalize_features(p, s_raw, tid);
-  __syncthreads();
-  // cache the new entry in slot n
-  bf16* kid = st.kidx + (u * p.cap + n) * p.dI;
-  for (int k = tid; k < p.dI; k += blockDim.x) {
-    const bf16 b = sc.kidx_new[(size_t)i * p.dI + k];
-    kid[k] = b;
-    s_raw[r.uk + k] = __bfloat162float(b);  // the new slot is scored with the cached (rounded) key
-  }
-  const int dv = p.d / 8;  // 16-byte vectors per head row
-  for (int k = tid; k < p.Hkv * dv; k += blockDim.x) {
-    const int h = k / dv, c = k % dv;
-    const uint4* ks = reinterpret_cast<const uint4*>(k_new + (size_t)i * p.Dkv + h * p.d) + c;
-    const uint4* vs = reinterpret_cast<const uint4*>(v_new + (size_t)i * p.Dkv + h * p.d) + c;
-    const size_t row = ((u * p.Hkv + h) * p.cap + n) * p.d;
-    reinterpret_cast<uint4*>(st.Kc + row)[c] = *ks;
-    reinterpret_cast<uint4*>(st.Vc + row)[c] = *vs;
-  }
-  if (tid == 0) st.pos[u * p.cap + n] = T;
-  __syncthreads();
-  const float* qf = s_raw + r.uq;
-  const float* alpha = s_raw + r.g;
-  const int n1 = n + 1;
-  bool bad = false;
-  for (int t = tid; t < n1; t += blockDim.x) {
-    float kk[64];
-    if (t == n) {
-      for (int k = 0; k < p.dI; ++k) kk[k] = s_raw[r.uk + k];
-    } else {
-      const bf16* row = st.kidx + (u * p.cap + t) * p.dI;
-      for (int k = 0; k < p.dI; ++k) kk[k] = __bfloat162float(row[k]);
-    }
-    const float A = index_score(p, qf, alpha, kk);
-    bad |= !isfinite(A);
-    const float old = (t == n) ? NEG_INF : st.imp[u * p.cap + t];
-    st.imp[u * p.cap + t] = fmaxf(old, A);
-  }
-  if (bad) atomicOr(st.status, ST_NONFINITE);
-  if (tid == 0) {
-    ctr[CTR_N] = n1;
-    ctr[CTR_T] = T + 1;
-    ctr[CTR_SINCE] = ctr[CTR_SINCE] + 1;
-    ctr[CTR_NEVICT] = 0;
-  }
-}
-
-// ------------------------------------------------------------------------------------------------
 // prefill: finalise the features of every chunk token, append K/V/kidx/pos.
-// grid = (C, n_seq), block = 128.  The counters are advanced by the scoring kernel.
+// grid = (C, n_seq), block = 128.  The counters are advanced by k_prefill_commit.
 __global__ void k_prefill_append(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __restrict__ K,
                                  const bf16* __restrict__ V) {
   const int c = blockIdx.x, i = blockIdx.y;
@@ -205,7 +59,14 @@ __global__ void k_prefill_append(ImDims p, ImState st, ImScratch sc, ImCall call
   __syncthreads();
   const int slot = n + c;
   bf16* kid = st.kidx + (u * p.cap + slot) * p.dI;
-  for (int k = tid; k < p.dI; k += blockDim.x) kid[k] = sc.kidx_new[((size_t)i * call.C + c) * p.dI + k];
+  // k = bf16(RMSNorm(U_k x)) from the float64 projection (one K split in prefill)
+  if (tid >= 32 && tid < 32 + p.dI) {
+    const double* ud = sc.keyp + ((size_t)i * call.C + c) * p.dI;
+    double ms = 0.0;
+    for (int j = 0; j < p.dI; ++j) ms += ud[j] * ud[j];
+    const double inv = 1.0 / sqrt(ms / (double)p.dI + (double)p.norm_eps);
+    kid[tid - 32] = __double2bfloat16(ud[tid - 32] * inv);
+  }
   const int dv = p.d / 8;
   for (int k = tid; k < p.Hkv * dv; k += blockDim.x) {
     const int h = k / dv, cc = k % dv;
@@ -375,7 +236,7 @@ __device__ int block_exclusive_scan(int v, int* out_excl, int* s_tmp /*[33]*/) {
 // Compression of every sequence in the call (Sec. 4 schedule): restart pooling; if over budget,
 // flag the retained entries and list the evicted slots in ascending slot order.
 // grid = n_seq, block = 256.
-__global__ void k_select(ImDims p, ImState st, ImCall call) {
+__global__ void k_select(ImDims p, ImState st, ImScratch sc, ImCall call) {
   __shared__ SelectShared sh;
   __shared__ int s_tmp[33];
   const size_t u = (size_t)call.layer * p.S + call.seq[blockIdx.x];
@@ -389,6 +250,7 @@ __global__ void k_select(ImDims p, ImState st, ImCall call) {
     return;
   }
   int ne = 0;
+  if (threadIdx.x == 0) sc.nhole[blockIdx.x] = 0;
   // keep what the selection saw (debug/parity export)
   for (int t = threadIdx.x; t < n; t += blockDim.x) {
     st.sel_pos[u * p.cap + t] = pos[t];
@@ -418,14 +280,26 @@ __global__ void k_select(ImDims p, ImState st, ImCall call) {
         ++off;
       }
     __syncthreads();
+    // retained entries at or above the budget, ascending: they fill the evicted slots below it
+    const int tl = n - p.B;  // == ne slots in [B, n)
+    const int per2 = (tl + blockDim.x - 1) / blockDim.x;
+    const int a0 = min(tl, (int)threadIdx.x * per2), a1 = min(tl, a0 + per2);
+    int cnt2 = 0;
+    for (int t = a0; t < a1; ++t) cnt2 += keep[p.B + t] ? 1 : 0;
+    int off2;
+    const int nh = block_exclusive_scan(cnt2, &off2, s_tmp);
+    int32_t* surv = sc.surv + (size_t)blockIdx.x * p.tail;
+    for (int t = a0; t < a1; ++t)
+      if (keep[p.B + t]) surv[off2++] = p.B + t;
+    if (threadIdx.x == 0) sc.nhole[blockIdx.x] = nh;
+    __syncthreads();
   }
   for (int t = threadIdx.x; t < n; t += blockDim.x) imp[t] = NEG_INF;
   if (threadIdx.x == 0) {
     ctr[CTR_SINCE] = 0;
     ctr[CTR_NSEL] = n;
     ctr[CTR_NEVICT] = ne;
-    // fold everything into M in this evict step if the pending list cannot take the evicted set
-    ctr[CTR_DIRECT] = (p.mem && ne > 0 && ctr[CTR_NPEND] + ne > p.F) ? 1 : 0;
+    ctr[CTR_N] = n - ne;  // the gather / move kernels that follow work from the lists, not from the count
     if (ne > 0) ctr[CTR_EVSTEPS] = ctr[CTR_EVSTEPS] + 1;
   }
 }
@@ -472,39 +346,21 @@ __global__ void k_init_normal(bf16* __restrict__ dst, size_t n, uint64_t key, fl
 }
 
 // Wfold[m][g*d + c] = sum over the query heads j of group g of Wt[m][j*d + c]   (float32)
-__global__ void k_fold_theta(ImDims p, const bf16* __restrict__ Wt, float* __restrict__ Wfold) {
+__global__ void k_fold_theta(ImDims p, const bf16* __restrict__ Wt, bf16* __restrict__ Wfh, bf16* __restrict__ Wfl) {
   const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (size_t)p.dM * p.Dkv) return;
   const int m = (int)(idx / p.Dkv), col = (int)(idx % p.Dkv);
   const int g = col / p.d, c = col % p.d;
   float s = 0.f;
   for (int j = g * p.Gq; j < (g + 1) * p.Gq; ++j) s += __bfloat162float(Wt[(size_t)m * p.D + j * p.d + c]);
-  Wfold[idx] = s;
+  const bf16 hi = __float2bfloat16_rn(s);
+  Wfh[idx] = hi;
+  Wfl[idx] = __float2bfloat16_rn(s - __bfloat162float(hi));
 }
 
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------ launchers
-cudaError_t im_launch_proj(const ImLaunch& L, const ImProjJobs& jobs, float* out) {
-  dim3 grid(jobs.total_rows, (jobs.NV + 7) / 8);
-  k_proj<<<grid, 256, 0, L.stream>>>(jobs, out);
-  ++*L.launches;
-  return cudaGetLastError();
-}
-
-cudaError_t im_launch_proj_key(const ImLaunch& L, const void* x, int NV) {
-  k_proj_key<<<(NV + 3) / 4, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, L.sc.kidx_new);
-  ++*L.launches;
-  return cudaGetLastError();
-}
-
-cudaError_t im_launch_decode_index(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new) {
-  const size_t smem = (size_t)L.p.R3 * 4;
-  k_decode_index<<<call.n_seq, 256, smem, L.stream>>>(L.p, L.st, L.sc, call, (const bf16*)k_new, (const bf16*)v_new);
-  ++*L.launches;
-  return cudaGetLastError();
-}
-
 cudaError_t im_launch_prefill_append(const ImLaunch& L, const ImCall& call, const void* k, const void* v) {
   dim3 grid(call.C, call.n_seq);
   k_prefill_append<<<grid, 128, 0, L.stream>>>(L.p, L.st, L.sc, call, (const bf16*)k, (const bf16*)v);
@@ -525,7 +381,7 @@ cudaError_t im_launch_prefill_score(const ImLaunch& L, const ImCall& call, int n
 }
 
 cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call) {
-  k_select<<<call.n_seq, 256, 0, L.stream>>>(L.p, L.st, call);
+  k_select<<<call.n_seq, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
 }
@@ -551,6 +407,6 @@ cudaError_t im_launch_init_weights(const ImDims& p, const ImWeights& w, int laye
 
 cudaError_t im_launch_fold_theta(const ImDims& p, const ImWeights& w, cudaStream_t stream) {
   const size_t n = (size_t)p.dM * p.Dkv;
-  k_fold_theta<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(p, w.Wt, w.Wfold);
+  k_fold_theta<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(p, w.Wt, w.Wfh, w.Wfl);
   return cudaGetLastError();
 }

@@ -75,14 +75,21 @@ struct ImWeights {  // one layer
   bf16* Wt;
   bf16* wg;
   float* bg;
-  float* Wfold;  // [dM][Dkv] float32: Linear_theta folded over each query-head group
+  // Linear_theta folded over each query-head group, [dM][Dkv]: Wfold[m][g*d+c] = sum_{j in group g} Wt[m][j*d+c],
+  // kept as two bf16 terms (Wfh + Wfl reproduces the float32 sum to 2^-17) so that it can feed the tensor cores
+  bf16* Wfh;
+  bf16* Wfl;
 };
 
 struct ImScratch {   // per call, shared by all layers, stream ordered
-  float* raw;        // [max_seqs * max(1,max_chunk)][R5 or R3] projection outputs (qf / alpha are finalised in place)
-  bf16* kidx_new;    // [max_seqs * max(1,max_chunk)][dI] indexer keys of the call's tokens
-  float* phi;        // [max_seqs][tail][dM]   phi of the evicted keys
-  int32_t* moves;    // [max_seqs][2][tail]    compaction: hole slots, survivor slots
+  float* raw;        // projection outputs: prefill [n_seq * C][R3]; decode K-split partials [IM_KSPLIT][n_seq][R5]
+  double* keyp;      // indexer-key projection in float64: prefill [n_seq * C][dI]; decode partials [IM_KSPLIT_KEY][n_seq][dI]
+  bf16* evK;         // [max_seqs][tail][Dkv]  evicted keys of the last compression, gathered
+  bf16* evV;         // [max_seqs][tail][Dkv]  evicted values
+  float* phi;        // [max_seqs][tail][dM]   phi of the evicted keys (evict steps with more than F entries)
+  float* phip;       // [IM_KSPLIT][max_seqs][F][dM] K-split partials of phi for evict steps with at most F entries
+  int32_t* surv;     // [max_seqs][tail]       compaction: retained entries found above the budget, ascending
+  int32_t* nhole;    // [max_seqs]             compaction: number of evicted slots below the budget
   float* part;       // attention partials (acc[d], max, sum): generic kernel [max_seqs][H][max_splits][d + 2];
                      // streaming kernel [warps + rows][Gq][d + 2]
   float* rpart;      // [max_seqs][ceil(dM / IM_READOUT_ROWS)][Dkv] readout partials
@@ -90,8 +97,36 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
 
 struct ImCall {
   int layer, n_seq, C;
+  int prefill;    // 1: im_prefill_chunk (always compresses), 0: im_decode_step (compresses every tau-th token)
+  int phi_large;  // 1: phi of the evicted keys lives in ImScratch::phi, 0: in the K-split partials phip
+  int ksplit, ksplit_key, ksplit_phi;  // K splits of the projections / key projection / phi partials of this call
   int seq[IM_MAX_CALL_SEQS];
 };
+
+// Skinny GEMM arguments: out[v][row0 + r] (+)= sum_k (W[r][k] + W2[r][k]) * in[v][k].
+// Vector v of input set s starts at in[s] + (v / in_cnt[s]) * in_outer[s] + (v % in_cnt[s]) * in_inner[s]
+// (elements); its outputs at out + (v / out_cnt) * out_outer + (v % out_cnt) * out_inner + ks * ks_stride.
+struct ImGemmJob {
+  const bf16* W;   // [rows][K]
+  const bf16* W2;  // optional second term of the weights (nullptr: none)
+  int rows, row0, in_sel;
+};
+struct ImGemmArgs {
+  ImGemmJob job[4];
+  int n_jobs;
+  const bf16* in[3];
+  long long in_outer[3], in_inner[3];
+  int in_cnt[3];
+  float* out;
+  long long out_outer, out_inner, ks_stride;
+  int out_cnt;
+  int NV, K, ksplit;
+};
+
+#define IM_KSPLIT 4       /* K splits of the decode projections (partials summed by the consumer) */
+#define IM_KSPLIT_KEY 16  /* K splits of the float64 indexer-key projection in decode */
+#define IM_FRONT_MAX_N 6144 /* entries the fused decode front kernel can select among (keys in shared memory) */
+#define IM_FRONT_MAX_NE 16  /* evicted entries per sequence the fused decode front kernel handles */
 
 struct ImProjJob {
   const bf16* W;   // [rows][Dn]
@@ -113,14 +148,16 @@ struct ImLaunch {
 };
 
 // ---- kernels' host launchers (each returns the cudaError of the launch)
-cudaError_t im_launch_proj(const ImLaunch& L, const ImProjJobs& jobs, float* out);
-cudaError_t im_launch_proj_key(const ImLaunch& L, const void* x, int NV);
-cudaError_t im_launch_decode_index(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new);
+cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a);
+cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, int ksplit);
+cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
+                                   int do_select, int n_max);
+cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
+cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call);
+cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_prefill_append(const ImLaunch& L, const ImCall& call, const void* k, const void* v);
 cudaError_t im_launch_prefill_score(const ImLaunch& L, const ImCall& call, int n_max);
 cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call);
-cudaError_t im_launch_memory_write(const ImLaunch& L, const ImCall& call, int ne_max, bool direct);
-cudaError_t im_launch_compact(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const void* q, void* out, int n_max);
 bool im_attn_fast_supported(const ImDims& p);
 cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV);
@@ -133,6 +170,21 @@ cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, in
 cudaError_t im_launch_init_weights(const ImDims& p, const ImWeights& w, int layer, uint64_t seed, float std,
                                    cudaStream_t stream);
 cudaError_t im_launch_fold_theta(const ImDims& p, const ImWeights& w, cudaStream_t stream);
+
+// Evict-step bookkeeping shared by the memory kernels: number of entries the compression of this
+// call will evict for a sequence whose counters are still those from before the call.
+__host__ __device__ inline int im_upcoming_evictions(const ImDims& p, int prefill, int C, int n, int since) {
+  const bool due = prefill || (since + 1 == p.tau);
+  const int over = n + C - p.B;
+  return (due && over > 0) ? over : 0;
+}
+
+// decode: projection row `row` of call sequence i, summed over the K-split partials in a fixed order
+__device__ __forceinline__ float im_raw_sum(const ImDims& p, const ImScratch& sc, const ImCall& call, int i, int row) {
+  float s = 0.f;
+  for (int ks = 0; ks < call.ksplit; ++ks) s += sc.raw[((size_t)ks * call.n_seq + i) * p.R5 + row];
+  return s;
+}
 
 // ---- small device helpers
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }

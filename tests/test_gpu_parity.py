@@ -215,3 +215,25 @@ def test_seeded_weight_init_statistics(im):
             assert abs(a.mean().item()) < 3 * 0.02 / a.numel() ** 0.5 + 1e-4
             assert abs(a.std().item() - 0.02) < 0.002
     assert w0["b_g"].item() == 0.0
+
+
+def test_generic_attention_path_small_head_dim():
+    """d = 32 has no TMA/mma fast path: the generic split kernels serve it."""
+    wl = synth.Workload("d32", 1, 2, 4, 2, 32, 200, 200, 72, 6, n_needles=2)
+    p = _pair(wl, dI=8, dM=24)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
+
+
+def test_long_interval_unfused_select_and_large_evicted_set():
+    """tau = 24: more evicted entries per compression than the fused decode kernel or the pending
+    list take, so the stand-alone select / gather / move kernels and the direct accumulation run."""
+    wl = TINY.replace(name="tau24", ctx=180, chunk=180, B=100, steps=48, tau=24, n_needles=2)
+    p = _pair(wl, lambda_=0.95)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.o.evict_steps(0) == 1 + 2
+    assert p.stats["max_M_err"] <= 2e-3
