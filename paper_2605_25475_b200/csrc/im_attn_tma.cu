@@ -15,6 +15,8 @@
 //     that the product is accurate to 2^-17, not 2^-9.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "im_internal.cuh"
 
 namespace {
@@ -367,43 +369,62 @@ __global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch
 // ------------------------------------------------------------------------------------------------
 // Merge: softmax-merge of the attention partials of one (sequence, KV head) row, readout (Eq. 5)
 // from the row-chunk partials and the pending rank-one terms, gate, fuse (Eq. 4), store.
-// grid = (Hkv, n_seq), block = DH.
+// grid = (Hkv, n_seq), block = 32 * max(Gq, DH / 32): warp hh merges query head hh of the group
+// (each lane DH/32 output columns), all heads in parallel; the readout vector of the KV head is
+// computed once by the whole block into shared memory.
 template <int DH, typename OutT>
-__global__ void __launch_bounds__(DH) k_attn_merge_rows(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call,
-                                                         int n_ctas, OutT* __restrict__ out) {
+__global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call,
+                                                          int n_ctas, OutT* __restrict__ out) {
+  constexpr int CPL = DH / 32;  // columns per lane
+  extern __shared__ float phiq[];  // [dM] phi(q), summed over the K-split partials
   __shared__ float s_dot[64];
-  __shared__ float s_red[DH / 32];
-  __shared__ float s_den;
-  const int h = blockIdx.x, i = blockIdx.y, c = threadIdx.x;
-  const int warp = c >> 5, lane = c & 31;
+  __shared__ float s_red[8];
+  __shared__ float s_mkv[DH];
+  __shared__ float s_gate;
+  const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int32_t* ctr = st.ctr + u * CTR_STRIDE;
-  // ---- rebuild the tile bookkeeping of the attention kernel
+  // ---- rebuild the tile bookkeeping of the attention kernel (lanes stride over the sequences)
   long long pref = 0, total = 0;
   int nt_i = 0;
-  for (int k = 0; k < call.n_seq; ++k) {
-    const size_t uk = (size_t)call.layer * p.S + call.seq[k];
-    const int nk = tiles_of(max(0, min(st.ctr[uk * CTR_STRIDE + CTR_N], p.cap)));
-    if (k == i) { pref = total; nt_i = nk; }
-    total += (long long)nk * p.Hkv;
+  for (int k0 = 0; k0 < call.n_seq; k0 += 32) {
+    const int k = k0 + lane;
+    int nk = 0;
+    if (k < call.n_seq) {
+      const size_t uk = (size_t)call.layer * p.S + call.seq[k];
+      nk = tiles_of(max(0, min(st.ctr[uk * CTR_STRIDE + CTR_N], p.cap)));
+    }
+    // inclusive prefix over the 32 lanes
+    long long incl = (long long)nk * p.Hkv;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const long long v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (i >= k0 && i < k0 + 32) {
+      pref = total + __shfl_sync(0xffffffffu, incl, i - k0) - (long long)__shfl_sync(0xffffffffu, nk, i - k0) * p.Hkv;
+      nt_i = __shfl_sync(0xffffffffu, nk, i - k0);
+    }
+    total += __shfl_sync(0xffffffffu, incl, 31);
   }
   const long long WT = (long long)n_ctas * WARPS;
   const long long qrun = (total + WT - 1) / WT;
   const long long row_first = pref + (long long)h * nt_i, row_last = row_first + nt_i - 1;
   const long long row_id = (long long)i * p.Hkv + h;
-  float mkv = 0.f, gate = 0.f;
+  // ---- readout of this KV head's columns: m(q)[col] (Eq. 5) and the gate (Eq. 4)
   if (p.mem) {
     const ImRows r = im_rows(p);
-    extern __shared__ float phiq[];  // [dM] phi(q), summed over the K-split partials
-    for (int m = c; m < p.dM; m += DH) phiq[m] = im_raw_sum(p, sc, call, i, r.theta + m);
+    for (int m = tid; m < p.dM; m += blockDim.x) phiq[m] = im_raw_sum(p, sc, call, i, r.theta + m);
+    if (tid == 0) s_gate = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
     __syncthreads();
     const int np = min(ctr[CTR_NPEND], p.F);
     float part_den = 0.f;
-    for (int m = c; m < p.dM; m += DH) part_den = fmaf(phiq[m] * phiq[m], st.bvec[u * p.dM + m], part_den);
+    for (int m = tid; m < p.dM; m += blockDim.x) part_den = fmaf(phiq[m] * phiq[m], st.bvec[u * p.dM + m], part_den);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) part_den += __shfl_xor_sync(0xffffffffu, part_den, off);
     if (lane == 0) s_red[warp] = part_den;
-    for (int pp = warp; pp < np; pp += DH / 32) {
+    for (int pp = warp; pp < np; pp += nwarps) {
       const float* ph = st.pend_phi + (u * p.F + pp) * p.dM;
       float v = 0.f;
       for (int m = lane; m < p.dM; m += 32) v = fmaf(phiq[m], ph[m], v);
@@ -412,40 +433,53 @@ __global__ void __launch_bounds__(DH) k_attn_merge_rows(ImDims p, ImState st, Im
       if (lane == 0) s_dot[pp] = v * st.pend_w[u * p.F + pp];
     }
     __syncthreads();
-    if (c == 0) {
-      float d = p.eps;
-      for (int k = 0; k < DH / 32; ++k) d += s_red[k];
-      s_den = d;
+    float den = p.eps;
+    for (int k = 0; k < nwarps; ++k) den += s_red[k];
+    const float cs = st.cscale[u];
+    const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
+    for (int c = tid; c < DH; c += blockDim.x) {
+      const int col = h * DH + c;
+      const float* rp = sc.rpart + (size_t)i * nchunk * p.Dkv + col;
+      float mv = 0.f;
+      for (int k = 0; k < nchunk; ++k) mv += rp[(size_t)k * p.Dkv];
+      for (int pp = 0; pp < np; ++pp) mv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mv);
+      s_mkv[c] = cs * mv / den;
     }
     __syncthreads();
-    const int col = h * DH + c;
-    const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
-    const float* rp = sc.rpart + (size_t)i * nchunk * p.Dkv + col;
-    for (int k = 0; k < nchunk; ++k) mkv += rp[(size_t)k * p.Dkv];
-    for (int pp = 0; pp < np; ++pp) mkv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mkv);
-    mkv = st.cscale[u] * mkv / s_den;
-    gate = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
   }
-  for (int hh = 0; hh < p.Gq; ++hh) {
-    float res = 0.f;
+  // ---- one warp per query head of the group
+  for (int hh = warp; hh < p.Gq; hh += nwarps) {
+    float res[CPL];
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) res[k] = 0.f;
     if (nt_i > 0) {
       const long long w0 = row_first / qrun, w1 = row_last / qrun;
-      float M = NEG_INF;
-      for (long long wv = w0; wv <= w1; ++wv)
-        M = fmaxf(M, sc.part[((size_t)(wv + row_id) * p.Gq + hh) * (DH + 2) + DH]);
-      float L = 0.f, acc = 0.f;
+      float M = NEG_INF, L = 0.f;
       for (long long wv = w0; wv <= w1; ++wv) {
         const float* ps = sc.part + ((size_t)(wv + row_id) * p.Gq + hh) * (DH + 2);
-        const float e = exp2f(ps[DH] - M);
-        L = fmaf(ps[DH + 1], e, L);
-        acc = fmaf(ps[c], e, acc);
+        const float mw = ps[DH], lw = ps[DH + 1];
+        float a[CPL];
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) a[k] = ps[lane + 32 * k];
+        const float Mn = fmaxf(M, mw);
+        const float eo = exp2f(M - Mn), en = exp2f(mw - Mn);  // exp2(-inf) = 0 for the first contributor
+        L = L * eo + lw * en;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[k] * en;
+        M = Mn;
       }
-      res = acc / L;
+      const float inv = 1.0f / L;
+#pragma unroll
+      for (int k = 0; k < CPL; ++k) res[k] *= inv;
     }
-    res = fmaf(gate, mkv, res);
-    const size_t idx = ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH + c;
-    if constexpr (sizeof(OutT) == 2) out[idx] = __float2bfloat16_rn(res);
-    else out[idx] = res;
+    const size_t base = ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH;
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) {
+      float v = res[k];
+      if (p.mem) v = fmaf(s_gate, s_mkv[lane + 32 * k], v);
+      if constexpr (sizeof(OutT) == 2) out[base + lane + 32 * k] = __float2bfloat16_rn(v);
+      else out[base + lane + 32 * k] = v;
+    }
   }
 }
 
@@ -515,12 +549,13 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   dim3 grid(p.Hkv, call.n_seq);
+  const int mthreads = 32 * std::max(p.Gq, p.d / 32);
   if (p.d == 64) {
-    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, 64, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
-    else k_attn_merge_rows<64, bf16><<<grid, 64, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
+    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, mthreads, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
+    else k_attn_merge_rows<64, bf16><<<grid, mthreads, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
   } else {
-    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, 128, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
-    else k_attn_merge_rows<128, bf16><<<grid, 128, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
+    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, mthreads, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
+    else k_attn_merge_rows<128, bf16><<<grid, mthreads, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
   }
   ++*L.launches;
   return cudaGetLastError();

@@ -24,6 +24,7 @@ struct FrontShared {
 
 // grid = n_seq, block = FRONT_THREADS, dynamic smem = keys of the selection (8 bytes per entry) when
 // do_select, else 0.
+template <int DI>  // d_I known at compile time (8, 16) keeps the key and the dot products in registers; 0: generic
 __global__ void __launch_bounds__(FRONT_THREADS)
 k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __restrict__ k_new,
                const bf16* __restrict__ v_new, int do_select) {
@@ -86,13 +87,16 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   float* imp = st.imp + u * p.cap;
   int32_t* pos = st.pos + u * p.cap;
   bool bad = false;
+  const int dI = DI > 0 ? DI : p.dI;
   for (int t = tid; t < n1; t += FRONT_THREADS) {
-    float kk[64];
+    float kk[DI > 0 ? DI : 64];
     if (t == n) {
-      for (int k = 0; k < p.dI; ++k) kk[k] = sh.knew[k];
-    } else if ((p.dI & 7) == 0) {
-      const uint4* row = reinterpret_cast<const uint4*>(st.kidx + (u * p.cap + t) * p.dI);
-      for (int c = 0; c < p.dI / 8; ++c) {
+#pragma unroll
+      for (int k = 0; k < dI; ++k) kk[k] = sh.knew[k];
+    } else if ((dI & 7) == 0) {
+      const uint4* row = reinterpret_cast<const uint4*>(st.kidx + (u * p.cap + t) * dI);
+#pragma unroll
+      for (int c = 0; c < dI / 8; ++c) {
         const uint4 w = row[c];
         const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
@@ -102,13 +106,14 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
         }
       }
     } else {
-      const bf16* row = st.kidx + (u * p.cap + t) * p.dI;
-      for (int k = 0; k < p.dI; ++k) kk[k] = __bfloat162float(row[k]);
+      const bf16* row = st.kidx + (u * p.cap + t) * dI;
+      for (int k = 0; k < dI; ++k) kk[k] = __bfloat162float(row[k]);
     }
     float A = 0.f;
     for (int h = 0; h < p.HI; ++h) {
       float z = 0.f;
-      for (int k = 0; k < p.dI; ++k) z = fmaf(sh.q[h * p.dI + k], kk[k], z);
+#pragma unroll
+      for (int k = 0; k < dI; ++k) z = fmaf(sh.q[h * dI + k], kk[k], z);
       if (p.act == 0) z = fmaxf(z, 0.f);
       A = fmaf(sh.alpha[h], z, A);
     }
@@ -276,13 +281,18 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
                                    int do_select, int n_max) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_decode_front, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8);
+    cudaError_t e = cudaFuncSetAttribute(k_decode_front<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
   const size_t smem = do_select ? (size_t)n_max * 8 : 0;
-  k_decode_front<<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, (const bf16*)k_new,
-                                                                (const bf16*)v_new, do_select);
+  const bf16* kn = (const bf16*)k_new;
+  const bf16* vn = (const bf16*)v_new;
+  if (L.p.dI == 16) k_decode_front<16><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select);
+  else if (L.p.dI == 8) k_decode_front<8><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select);
+  else k_decode_front<0><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select);
   ++*L.launches;
   return cudaGetLastError();
 }

@@ -60,21 +60,19 @@ __global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
     const int kc = min(KC, kspan - k0);     // multiple of 16
     const int chunks = kc / 8;              // 16-byte chunks per row
     __syncthreads();                        // previous round's reads are done
-    for (int idx = threadIdx.x; idx < 16 * chunks; idx += blockDim.x) {
-      const int r = idx / chunks, c = idx % chunks;
+    // warp w stages rows w, w+4, ...; one row pointer per row, lanes stride over its 16-byte chunks
+    for (int r = warp; r < 16; r += 4) {
       const bool valid = r0 + r < job.rows;
-      const bf16* src = job.W + (size_t)(valid ? r0 + r : 0) * a.K + kbeg + k0 + c * 8;
-      cp_async16(smem_u32(sA + r * ROW_BYTES + c * 16), src, valid);
-      if (job.W2) {
-        const bf16* src2 = job.W2 + (size_t)(valid ? r0 + r : 0) * a.K + kbeg + k0 + c * 8;
-        cp_async16(smem_u32(sA2 + r * ROW_BYTES + c * 16), src2, valid);
+      const size_t off = (size_t)(valid ? r0 + r : 0) * a.K + kbeg + k0;
+      for (int c = lane; c < chunks; c += 32) {
+        cp_async16(smem_u32(sA + r * ROW_BYTES + c * 16), job.W + off + c * 8, valid);
+        if (job.W2) cp_async16(smem_u32(sA2 + r * ROW_BYTES + c * 16), job.W2 + off + c * 8, valid);
       }
     }
-    for (int idx = threadIdx.x; idx < VB * chunks; idx += blockDim.x) {
-      const int r = idx / chunks, c = idx % chunks;
+    for (int r = warp; r < VB; r += 4) {
       const bool valid = v0 + r < a.NV;
-      const bf16* src = vec_ptr(a, job.in_sel, valid ? v0 + r : 0) + kbeg + k0 + c * 8;
-      cp_async16(smem_u32(sB + r * ROW_BYTES + c * 16), src, valid);
+      const bf16* src = vec_ptr(a, job.in_sel, valid ? v0 + r : 0) + kbeg + k0;
+      for (int c = lane; c < chunks; c += 32) cp_async16(smem_u32(sB + r * ROW_BYTES + c * 16), src + c * 8, valid);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -129,21 +127,33 @@ __global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __
   const int kspan = p.D / ksplit, kbeg = ks * kspan;  // kspan is a multiple of 8
   const uint4* x4 = reinterpret_cast<const uint4*>(x + (size_t)v * p.D + kbeg);
   double* dst = keyp + ((size_t)ks * NV + v) * p.dI;
-  for (int r = 0; r < p.dI; ++r) {
-    const uint4* w4 = reinterpret_cast<const uint4*>(Uk + (size_t)r * p.D + kbeg);
-    double acc = 0.0;
-    for (int c = lane; c < kspan / 8; c += 32) {
-      const uint4 a = w4[c], b = x4[c];
-      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+  for (int rb = 0; rb < p.dI; rb += 8) {  // 8 rows at a time: their loads are in flight together
+    double acc[8];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        // a product of two bf16 values is exact in float32
-        acc += (double)(__uint_as_float(aw[k] << 16) * __uint_as_float(bw[k] << 16));
-        acc += (double)(__uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u));
+    for (int j = 0; j < 8; ++j) acc[j] = 0.0;
+    for (int c = lane; c < kspan / 8; c += 32) {
+      const uint4 b = x4[c];
+      uint4 a[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        a[j] = rb + j < p.dI ? reinterpret_cast<const uint4*>(Uk + (size_t)(rb + j) * p.D + kbeg)[c] : make_uint4(0, 0, 0, 0);
+      const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t aw[4] = {a[j].x, a[j].y, a[j].z, a[j].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          // a product of two bf16 values is exact in float32
+          acc[j] += (double)(__uint_as_float(aw[k] << 16) * __uint_as_float(bw[k] << 16));
+          acc[j] += (double)(__uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u));
+        }
       }
     }
-    acc = warp_sum_d(acc);
-    if (lane == 0) dst[r] = acc;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const double s = warp_sum_d(acc[j]);
+      if (lane == 0 && rb + j < p.dI) dst[rb + j] = s;
+    }
   }
 }
 

@@ -27,21 +27,25 @@ __device__ __forceinline__ bool fold_needed(const ImDims& p, const ImCall& call,
   return np + ne > p.F;
 }
 
-// Mhat <- cscale * (Mhat + sum_p w_p phi_p v_p^T).  grid = (ceil(Dkv/64), ceil(dM/64), n_seq), block = 256,
-// each thread a 4x4 micro tile.  Blocks of sequences that need no fold leave at once.
+// Mhat <- cscale * (Mhat + sum_p w_p phi_p v_p^T).  grid = (FOLD_BLOCKS, n_seq), block = 256; a block
+// walks 64x64 tiles of Mhat, each thread a 4x4 micro tile.  Blocks of sequences that need no fold
+// leave at once (the kernel is part of every decode step so that a captured launch sequence stays valid).
+constexpr int FOLD_BLOCKS = 16;
 __global__ void __launch_bounds__(256) k_mem_fold(ImDims p, ImState st, ImCall call) {
   __shared__ float s_a[16][64 + 4];  // [entry][m]   w_p * phi_p
   __shared__ float s_b[16][64 + 4];  // [entry][col] v_p
-  const int i = blockIdx.z;
+  const int i = blockIdx.y;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int32_t* ctr = st.ctr + u * CTR_STRIDE;
   const float c = st.cscale[u];
   if (!fold_needed(p, call, ctr, c)) return;
   const int np = min(ctr[CTR_NPEND], p.F);
-  const int m0 = blockIdx.y * 64, col0 = blockIdx.x * 64;
+  const int tiles_x = (p.Dkv + 63) / 64, tiles_y = (p.dM + 63) / 64;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  float acc[4][4];
   float* Mh = st.Mhat + u * p.dM * p.Dkv;
+  for (int tile = blockIdx.x; tile < tiles_x * tiles_y; tile += gridDim.x) {
+  const int m0 = (tile / tiles_x) * 64, col0 = (tile % tiles_x) * 64;
+  float acc[4][4];
 #pragma unroll
   for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -83,6 +87,7 @@ __global__ void __launch_bounds__(256) k_mem_fold(ImDims p, ImState st, ImCall c
       const int m = m0 + ty * 4 + a, col = col0 + tx * 4 + b;
       if (m < p.dM && col < p.Dkv) Mh[(size_t)m * p.Dkv + col] = c * acc[a][b];
     }
+  }
 }
 
 // after every block of k_mem_fold has read cscale / the list: cscale <- 1, list emptied.
@@ -201,7 +206,7 @@ __global__ void __launch_bounds__(256) k_mem_accumulate(ImDims p, ImState st, Im
 
 cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call) {
   const ImDims& p = L.p;
-  dim3 grid((p.Dkv + 63) / 64, (p.dM + 63) / 64, call.n_seq);
+  dim3 grid(FOLD_BLOCKS, call.n_seq);
   k_mem_fold<<<grid, 256, 0, L.stream>>>(p, L.st, call);
   ++*L.launches;
   cudaError_t e = cudaGetLastError();
