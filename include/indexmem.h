@@ -188,6 +188,16 @@ int im_status(im_ctx* ctx, void* cuda_stream, int32_t* device_status);
 int im_profile_begin(im_ctx* ctx, int max_records);
 int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
 
+/*
+ * Execution option (no counterpart in the paper): with enable != 0 (the default where the streaming
+ * attention kernel is available) im_decode_step runs the pieces of a call that do not depend on each
+ * other - key projection, fold of the pending memory writes, readout, memory write - on two internal
+ * side streams that fork from and join back into `cuda_stream` inside the call; with 0 everything is
+ * enqueued on `cuda_stream` in order.  Results are identical.  The fork/join uses events only and can
+ * be captured into a CUDA graph.
+ */
+int im_set_concurrency(im_ctx* ctx, int enable);
+
 /* Number of kernels this library has launched on behalf of `ctx` since im_create. */
 int64_t im_launch_count(im_ctx* ctx);
 

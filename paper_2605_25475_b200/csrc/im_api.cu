@@ -163,6 +163,11 @@ struct im_ctx {
   alignas(64) unsigned char mapK[128];  // TMA descriptors of the K / V caches
   alignas(64) unsigned char mapV[128];
   bool fast_attn = false;
+  // Independent pieces of one decode call run on two side streams that fork from and join back into
+  // the caller's stream (plain event dependencies, so the pattern can be captured into a CUDA graph).
+  cudaStream_t side[2] = {nullptr, nullptr};
+  cudaEvent_t ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  bool concurrent = false;
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
   std::vector<cudaEvent_t> prof_ev;  // pairs (start, stop)
   size_t prof_used = 0;              // events recorded so far
@@ -307,8 +312,13 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     ctx->n_ctas = std::max(1, std::min(sms, IM_ATTN_MAX_CTAS));
     ctx->fast_attn = (e == cudaSuccess);
   }
+  for (int k = 0; k < 2 && e == cudaSuccess; ++k) e = cudaStreamCreateWithFlags(&ctx->side[k], cudaStreamNonBlocking);
+  for (int k = 0; k < 8 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
+  ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
+    for (int k = 0; k < 2; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
+    for (int k = 0; k < 8; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
     delete ctx;
     return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
   }
@@ -319,6 +329,8 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
 int im_destroy(im_ctx* ctx) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   cudaError_t e = cudaDeviceSynchronize();
+  for (int k = 0; k < 2; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
+  for (int k = 0; k < 8; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   delete ctx;
   if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
   return IM_OK;
@@ -448,8 +460,28 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   call.ksplit = pick_ksplit(p.D, IM_KSPLIT);
   call.ksplit_key = (p.D % (8 * IM_KSPLIT_KEY) == 0) ? IM_KSPLIT_KEY : 1;
   call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
-  ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
-  if (p.mem && ne_max > 0) CKL(im_launch_mem_fold(L, call));
+  // Streams: s0 is the caller's; s1 / s2 carry the pieces that do not depend on each other:
+  //   s0: projections -> front (append, score, select, compact) -> attention -> merge
+  //   s1: float64 key projection (needed by front); later phi of the evicted keys + memory write
+  //   s2: fold of the pending list (needs nothing from this call) -> readout (needs phi(q) only)
+  cudaStream_t s0 = (cudaStream_t)cuda_stream;
+  // An evicted set larger than the pending list is accumulated into Mhat itself, which the readout
+  // reads: that case keeps everything in order on one stream.
+  const bool conc = ctx->concurrent && ctx->fast_attn && ne_max <= p.F;
+  ImLaunch L = make_launch(ctx, layer, s0);
+  ImLaunch L1 = L, L2 = L;
+  if (conc) {
+    L1.stream = ctx->side[0];
+    L2.stream = ctx->side[1];
+    CK(cudaEventRecord(ctx->ev[0], s0));
+    CK(cudaStreamWaitEvent(L1.stream, ctx->ev[0], 0));
+    CK(cudaStreamWaitEvent(L2.stream, ctx->ev[0], 0));
+  }
+  const bool mem_write = due && ne_max > 0 && p.mem;
+  if (mem_write) {
+    CKL(im_launch_mem_fold(L2, call));
+    if (conc) CK(cudaEventRecord(ctx->ev[7], L2.stream));  // fold done: it read the counters of before the call
+  }
   // a0: projections (Sec. 3.1 features, phi(q) of Eq. 5, gate of Eq. 4) as K-split partial sums
   ImRows r = im_rows(p);
   ImGemmArgs g;
@@ -471,7 +503,18 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   g.K = p.D;
   g.ksplit = call.ksplit;
   CKL(im_launch_gemm(L, g));
-  CKL(im_launch_proj_key_split(L, x, n_seq, call.ksplit_key));
+  CKL(im_launch_proj_key_split(L1, x, n_seq, call.ksplit_key));
+  if (conc) {
+    CK(cudaEventRecord(ctx->ev[1], s0));                 // projections done
+    CK(cudaStreamWaitEvent(L2.stream, ctx->ev[1], 0));
+    CK(cudaEventRecord(ctx->ev[2], L1.stream));          // key projection done
+    CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
+    if (mem_write) CK(cudaStreamWaitEvent(s0, ctx->ev[7], 0));  // the front kernel changes the counters
+  }
+  // a6 (first half): phi(q)^T Mhat partial sums; needs the fold and phi(q) only
+  // (an evicted set larger than the pending list changes Mhat in this call: then the readout follows the write)
+  const bool readout_early = !(mem_write && ne_max > p.F);
+  if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call));
   // append + a1 (+ a2, gather, a4 when the evicted set is small enough for one block per sequence)
   const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
   CKL(im_launch_decode_front(L, call, k_new, v_new, fused ? 1 : 0, n_max));
@@ -479,8 +522,16 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CKL(im_launch_select(L, call));
     if (ne_max > 0) CKL(im_launch_gather_move(L, call, ne_max));
   }
-  // a3: memory write
-  if (due && ne_max > 0 && p.mem && (rc = run_memory_write(ctx, L, call, ne_max))) return rc;
+  // a3: memory write (needs the gathered evicted pairs and the fold)
+  if (mem_write) {
+    if (conc) {
+      CK(cudaEventRecord(ctx->ev[3], s0));               // evicted pairs gathered, cache compacted
+      CK(cudaStreamWaitEvent(L1.stream, ctx->ev[3], 0));
+      CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0)); // the fold emptied the list the write appends to
+    }
+    if ((rc = run_memory_write(ctx, L1, call, ne_max))) return rc;
+    if (ctx->fast_attn && !readout_early) CKL(im_launch_readout(L1, call));
+  }
   int n_att = 0;
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
@@ -491,19 +542,30 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     u.since = due ? 0 : u.since + 1;
     n_att = std::max(n_att, u.n);
   }
-  // a5-a6: attention over the retained entries + gated readout
+  // a5: attention over the retained entries; a6: merge with the readout, gate, fuse
   const bool prof = ctx->prof_used + 2 <= ctx->prof_ev.size();
-  if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], L.stream));
+  if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
   if (ctx->fast_attn) {
-    if (p.mem) CKL(im_launch_readout(L, call));
-    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, out, ctx->n_ctas));
+    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
+    if (conc) {
+      CK(cudaEventRecord(ctx->ev[5], L1.stream));
+      CK(cudaEventRecord(ctx->ev[6], L2.stream));
+      CK(cudaStreamWaitEvent(s0, ctx->ev[5], 0));
+      CK(cudaStreamWaitEvent(s0, ctx->ev[6], 0));
+    }
+    CKL(im_launch_attention_merge(L, call, out, ctx->n_ctas));
   } else {
     CKL(im_launch_attention(L, call, q, out, n_att));
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
   }
-  if (prof) {
-    CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], L.stream));
-    ctx->prof_used += 2;
-  }
+  if (prof) ctx->prof_used += 2;
+  return IM_OK;
+}
+
+int im_set_concurrency(im_ctx* ctx, int enable) {
+  if (!ctx) return fail(IM_ERR_ARG, "null context");
+  ctx->concurrent = enable != 0;
   return IM_OK;
 }
 

@@ -538,7 +538,7 @@ cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call) {
 }
 
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
-                                     const void* q, void* out, int n_ctas) {
+                                     const void* q, int n_ctas) {
   const ImDims& p = L.p;
   const size_t smem = im_attn_smem_bytes(p);
   const CUtensorMap& mk = *(const CUtensorMap*)mapK;
@@ -546,8 +546,11 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   if (p.d == 64) k_attn_stream<64><<<n_ctas, WARPS * 32, smem, L.stream>>>(mk, mv, p, L.st, L.sc, call, (const bf16*)q);
   else k_attn_stream<128><<<n_ctas, WARPS * 32, smem, L.stream>>>(mk, mv, p, L.st, L.sc, call, (const bf16*)q);
   ++*L.launches;
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas) {
+  const ImDims& p = L.p;
   dim3 grid(p.Hkv, call.n_seq);
   const int mthreads = 32 * std::max(p.Gq, p.d / 32);
   if (p.d == 64) {

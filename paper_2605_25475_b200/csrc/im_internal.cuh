@@ -164,7 +164,8 @@ cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, vo
 cudaError_t im_attn_prepare(const ImDims& p);
 cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
-                                     const void* q, void* out, int n_ctas);
+                                     const void* q, int n_ctas);
+cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas);
 cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,
                            uint8_t* keep, int32_t* n_evict, cudaStream_t stream);
 cudaError_t im_launch_init_weights(const ImDims& p, const ImWeights& w, int layer, uint64_t seed, float std,
