@@ -18,6 +18,7 @@ struct FrontShared {
   unsigned long long wmin[FRONT_THREADS / 32];
   int wslot[FRONT_THREADS / 32];
   int ev[IM_FRONT_MAX_NE];   // evicted slots, ascending after the sort
+  int evpos[IM_FRONT_MAX_NE];// their positions
   int surv[IM_FRONT_MAX_NE]; // retained entries found at or above the budget, ascending
   int nh;
 };
@@ -40,6 +41,32 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   }
   const ImRows r = im_rows(p);
   const int nq = p.HI * p.dI;
+  const int dI = DI > 0 ? DI : p.dI;
+  float* imp = st.imp + u * p.cap;
+  int32_t* pos = st.pos + u * p.cap;
+  // ---- issue the loads of the first batch of cached entries (they depend on nothing of this call)
+  constexpr int EPT = 4;
+  uint4 kraw[EPT][DI > 0 ? DI / 8 : 1];
+  float imp_old[EPT];
+  int pos_old[EPT];
+  auto load_batch = [&](int b0) {
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int t = b0 + e * FRONT_THREADS + tid;
+      imp_old[e] = NEG_INF;
+      pos_old[e] = 0;
+      if (t < n) {  // slot n is the token being appended
+        if (DI > 0) {
+          const uint4* row = reinterpret_cast<const uint4*>(st.kidx + (u * p.cap + t) * dI);
+#pragma unroll
+          for (int c = 0; c < (DI > 0 ? DI / 8 : 1); ++c) kraw[e][c] = row[c];
+        }
+        imp_old[e] = imp[t];
+        pos_old[e] = pos[t];
+      }
+    }
+  };
+  load_batch(0);
   // ---- finish the projections: sum the K-split partials in a fixed order
   for (int k = tid; k < nq; k += FRONT_THREADS) {
     sh.q[k] = im_raw_sum(p, sc, call, i, r.uq + k);
@@ -80,56 +107,58 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   }
   if (tid == 0) st.pos[u * p.cap + n] = T;
   __syncthreads();
-  // ---- a1: A_t = sum_h alpha_h act(q_h . k_t), pooled by max into the importance
+  // ---- a1: A_t = sum_h alpha_h act(q_h . k_t), pooled by max into the importance.
+  // Entries are handled in batches of EPT per thread; the loads of a batch are all issued before its
+  // arithmetic (the first batch was issued before the feature finalisation above).
   const int n1 = n + 1;
   const bool due = (since + 1 == p.tau);
   const bool select_here = do_select && due;
-  float* imp = st.imp + u * p.cap;
-  int32_t* pos = st.pos + u * p.cap;
   bool bad = false;
-  const int dI = DI > 0 ? DI : p.dI;
-  for (int t = tid; t < n1; t += FRONT_THREADS) {
-    float kk[DI > 0 ? DI : 64];
-    if (t == n) {
+  for (int b0 = 0; b0 < n1; b0 += EPT * FRONT_THREADS) {
+    if (b0 > 0) load_batch(b0);
 #pragma unroll
-      for (int k = 0; k < dI; ++k) kk[k] = sh.knew[k];
-    } else if ((dI & 7) == 0) {
-      const uint4* row = reinterpret_cast<const uint4*>(st.kidx + (u * p.cap + t) * dI);
+    for (int e = 0; e < EPT; ++e) {
+      const int t = b0 + e * FRONT_THREADS + tid;
+      if (t >= n1) continue;
+      float kk[DI > 0 ? DI : 64];
+      if (t == n) {
 #pragma unroll
-      for (int c = 0; c < dI / 8; ++c) {
-        const uint4 w = row[c];
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        for (int k = 0; k < dI; ++k) kk[k] = sh.knew[k];
+      } else if (DI > 0) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          kk[c * 8 + 2 * k] = __uint_as_float(ww[k] << 16);
-          kk[c * 8 + 2 * k + 1] = __uint_as_float(ww[k] & 0xffff0000u);
+        for (int c = 0; c < (DI > 0 ? DI / 8 : 1); ++c) {
+          const uint32_t ww[4] = {kraw[e][c].x, kraw[e][c].y, kraw[e][c].z, kraw[e][c].w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            kk[c * 8 + 2 * k] = __uint_as_float(ww[k] << 16);
+            kk[c * 8 + 2 * k + 1] = __uint_as_float(ww[k] & 0xffff0000u);
+          }
         }
+      } else {
+        const bf16* row = st.kidx + (u * p.cap + t) * dI;
+        for (int k = 0; k < dI; ++k) kk[k] = __bfloat162float(row[k]);
       }
-    } else {
-      const bf16* row = st.kidx + (u * p.cap + t) * dI;
-      for (int k = 0; k < dI; ++k) kk[k] = __bfloat162float(row[k]);
-    }
-    float A = 0.f;
-    for (int h = 0; h < p.HI; ++h) {
-      float z = 0.f;
+      float A = 0.f;
+      for (int h = 0; h < p.HI; ++h) {
+        float z = 0.f;
 #pragma unroll
-      for (int k = 0; k < dI; ++k) z = fmaf(sh.q[h * dI + k], kk[k], z);
-      if (p.act == 0) z = fmaxf(z, 0.f);
-      A = fmaf(sh.alpha[h], z, A);
-    }
-    bad |= !isfinite(A);
-    const float old = (t == n) ? NEG_INF : imp[t];
-    const float pooled = fmaxf(old, A);
-    const int ps = (t == n) ? T : pos[t];
-    if (due) {  // what the selection sees (parity export), then the pooling restarts
-      st.sel_pos[u * p.cap + t] = ps;
-      st.sel_imp[u * p.cap + t] = pooled;
-    }
-    if (select_here) {
-      s_key[t] = im_select_key(pooled, ps, p.n_sink);
-      imp[t] = NEG_INF;
-    } else {
-      imp[t] = pooled;
+        for (int k = 0; k < dI; ++k) z = fmaf(sh.q[h * dI + k], kk[k], z);
+        if (p.act == 0) z = fmaxf(z, 0.f);
+        A = fmaf(sh.alpha[h], z, A);
+      }
+      bad |= !isfinite(A);
+      const float pooled = fmaxf((t == n) ? NEG_INF : imp_old[e], A);
+      const int ps = (t == n) ? T : pos_old[e];
+      if (due) {  // what the selection sees (parity export), then the pooling restarts
+        st.sel_pos[u * p.cap + t] = ps;
+        st.sel_imp[u * p.cap + t] = pooled;
+      }
+      if (select_here) {
+        s_key[t] = im_select_key(pooled, ps, p.n_sink);
+        imp[t] = NEG_INF;
+      } else {
+        imp[t] = pooled;
+      }
     }
   }
   if (bad) atomicOr(st.status, ST_NONFINITE);
@@ -169,17 +198,19 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
       for (int w = 1; w < FRONT_THREADS / 32; ++w)
         if (sh.wmin[w] < best) { best = sh.wmin[w]; slot = sh.wslot[w]; }
       sh.ev[e] = slot;
-      s_key[slot] = ~0ull;  // a real key never has this value: its low word is ~position with position >= 0
+      sh.evpos[e] = (int)(0xFFFFFFFFu - (uint32_t)best);  // the key's low word is ~position
+      s_key[slot] = ~0ull;                                 // taken: the largest possible value
     }
     __syncthreads();
   }
   if (tid == 0) {
     // ascending slot order; holes below the budget pair with the retained entries above it
     for (int a = 1; a < ne; ++a) {
-      const int v = sh.ev[a];
+      const int v = sh.ev[a], vp = sh.evpos[a];
       int b = a - 1;
-      while (b >= 0 && sh.ev[b] > v) { sh.ev[b + 1] = sh.ev[b]; --b; }
+      while (b >= 0 && sh.ev[b] > v) { sh.ev[b + 1] = sh.ev[b]; sh.evpos[b + 1] = sh.evpos[b]; --b; }
       sh.ev[b + 1] = v;
+      sh.evpos[b + 1] = vp;
     }
     int nh = 0, ns = 0;
     for (int a = 0; a < ne; ++a) nh += sh.ev[a] < p.B ? 1 : 0;
@@ -192,32 +223,34 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     sh.nh = min(nh, ns);
     for (int a = 0; a < ne; ++a) {
       st.ev_slot[u * p.tail + a] = sh.ev[a];
-      st.ev_pos[u * p.tail + a] = (sh.ev[a] == n) ? T : pos[sh.ev[a]];
+      st.ev_pos[u * p.tail + a] = sh.evpos[a];
     }
   }
   __syncthreads();
-  // ---- gather the evicted pairs for the memory write (a3 reads them from here)
+  // ---- gather the evicted pairs for the memory write (a3) and, in the same pass, a4: a hole below
+  // the budget (the first nh evicted slots) receives the retained entry found above it.  A thread
+  // reads the evicted chunk before it overwrites it; the sources of the moves are never written.
+  const int nh = sh.nh;
   for (int k = tid; k < ne * p.Hkv * dv; k += FRONT_THREADS) {
     const int e = k / (p.Hkv * dv), rem = k % (p.Hkv * dv), h = rem / dv, c = rem % dv;
-    const size_t row = ((u * p.Hkv + h) * p.cap + sh.ev[e]) * p.d;
-    const size_t dst = ((size_t)i * p.tail + e) * p.Dkv + h * p.d;
-    reinterpret_cast<uint4*>(sc.evK + dst)[c] = reinterpret_cast<const uint4*>(st.Kc + row)[c];
-    reinterpret_cast<uint4*>(sc.evV + dst)[c] = reinterpret_cast<const uint4*>(st.Vc + row)[c];
-  }
-  __syncthreads();
-  // ---- a4: fill the holes below the budget with the retained entries from above it
-  const int nh = sh.nh;
-  for (int k = tid; k < nh * p.Hkv * dv; k += FRONT_THREADS) {
-    const int j = k / (p.Hkv * dv), rem = k % (p.Hkv * dv), h = rem / dv, c = rem % dv;
     const size_t base = (u * p.Hkv + h) * p.cap;
-    reinterpret_cast<uint4*>(st.Kc + (base + sh.ev[j]) * p.d)[c] = reinterpret_cast<const uint4*>(st.Kc + (base + sh.surv[j]) * p.d)[c];
-    reinterpret_cast<uint4*>(st.Vc + (base + sh.ev[j]) * p.d)[c] = reinterpret_cast<const uint4*>(st.Vc + (base + sh.surv[j]) * p.d)[c];
+    uint4* krow = reinterpret_cast<uint4*>(st.Kc + (base + sh.ev[e]) * p.d) + c;
+    uint4* vrow = reinterpret_cast<uint4*>(st.Vc + (base + sh.ev[e]) * p.d) + c;
+    const uint4 ke = *krow, ve = *vrow;
+    uint4 ks = ke, vs = ve;
+    if (e < nh) {
+      ks = reinterpret_cast<const uint4*>(st.Kc + (base + sh.surv[e]) * p.d)[c];
+      vs = reinterpret_cast<const uint4*>(st.Vc + (base + sh.surv[e]) * p.d)[c];
+    }
+    const size_t dst = ((size_t)i * p.tail + e) * p.Dkv + h * p.d;
+    reinterpret_cast<uint4*>(sc.evK + dst)[c] = ke;
+    reinterpret_cast<uint4*>(sc.evV + dst)[c] = ve;
+    if (e < nh) { *krow = ks; *vrow = vs; }
   }
   for (int k = tid; k < nh * p.dI; k += FRONT_THREADS) {
     const int j = k / p.dI, c = k % p.dI;
     st.kidx[(u * p.cap + sh.ev[j]) * p.dI + c] = st.kidx[(u * p.cap + sh.surv[j]) * p.dI + c];
   }
-  __syncthreads();  // ev_pos above read pos[] of the evicted slots before they are overwritten here
   for (int j = tid; j < nh; j += FRONT_THREADS) pos[sh.ev[j]] = (sh.surv[j] == n) ? T : pos[sh.surv[j]];
   if (tid == 0) {
     ctr[CTR_N] = n1 - ne;

@@ -36,12 +36,13 @@ __device__ __forceinline__ const bf16* vec_ptr(const ImGemmArgs& a, int sel, lon
   return a.in[sel] + (v / a.in_cnt[sel]) * a.in_outer[sel] + (v % a.in_cnt[sel]) * a.in_inner[sel];
 }
 
-// grid = (row tiles over all jobs, ksplit, ceil(NV / 32)), block = 128, dynamic smem = 64 * ROW_BYTES
+// grid = (row tiles over all jobs, ksplit, ceil(NV / 32)), block = 128.
+// Dynamic smem: two stages of (16 weight rows [+ 16 rows of the second term] + 32 vector rows) x ROW_BYTES;
+// the cp.async copies of round r+1 are in flight while round r is multiplied.
 __global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
-  unsigned char* sA = smem;                    // [16][ROW_BYTES]
-  unsigned char* sA2 = smem + 16 * ROW_BYTES;  // [16][ROW_BYTES] second weight term
-  unsigned char* sB = smem + 32 * ROW_BYTES;   // [32][ROW_BYTES]
+  const int stage_rows = a.any_w2 ? 64 : 48;
+  const int offB = a.any_w2 ? 32 : 16;  // row offset of the vector tile inside a stage
   int tile = blockIdx.x, j = 0;
   while (j + 1 < a.n_jobs && tile >= (a.job[j].rows + 15) / 16) {
     tile -= (a.job[j].rows + 15) / 16;
@@ -55,32 +56,40 @@ __global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
   const long long v0 = (long long)blockIdx.z * VB;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int k0 = 0; k0 < kspan; k0 += KC) {
-    const int kc = min(KC, kspan - k0);     // multiple of 16
-    const int chunks = kc / 8;              // 16-byte chunks per row
-    __syncthreads();                        // previous round's reads are done
-    // warp w stages rows w, w+4, ...; one row pointer per row, lanes stride over its 16-byte chunks
+  const int rounds = (kspan + KC - 1) / KC;
+  // warp w stages rows w, w+4, ...; one row pointer per row, lanes stride over its 16-byte chunks
+  auto issue = [&](int rd) {
+    unsigned char* st = smem + (size_t)(rd & 1) * stage_rows * ROW_BYTES;
+    const int k0 = rd * KC;
+    const int chunks = min(KC, kspan - k0) / 8;
     for (int r = warp; r < 16; r += 4) {
       const bool valid = r0 + r < job.rows;
       const size_t off = (size_t)(valid ? r0 + r : 0) * a.K + kbeg + k0;
       for (int c = lane; c < chunks; c += 32) {
-        cp_async16(smem_u32(sA + r * ROW_BYTES + c * 16), job.W + off + c * 8, valid);
-        if (job.W2) cp_async16(smem_u32(sA2 + r * ROW_BYTES + c * 16), job.W2 + off + c * 8, valid);
+        cp_async16(smem_u32(st + r * ROW_BYTES + c * 16), job.W + off + c * 8, valid);
+        if (job.W2) cp_async16(smem_u32(st + (16 + r) * ROW_BYTES + c * 16), job.W2 + off + c * 8, valid);
       }
     }
     for (int r = warp; r < VB; r += 4) {
       const bool valid = v0 + r < a.NV;
       const bf16* src = vec_ptr(a, job.in_sel, valid ? v0 + r : 0) + kbeg + k0;
-      for (int c = lane; c < chunks; c += 32) cp_async16(smem_u32(sB + r * ROW_BYTES + c * 16), src + c * 8, valid);
+      for (int c = lane; c < chunks; c += 32) cp_async16(smem_u32(st + (offB + r) * ROW_BYTES + c * 16), src + c * 8, valid);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  };
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  issue(0);
+  if (rounds > 1) issue(1);
+  for (int rd = 0; rd < rounds; ++rd) {
+    if (rd + 1 < rounds) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
+    const uint32_t stg = smem_u32(smem + (size_t)(rd & 1) * stage_rows * ROW_BYTES);
+    const int kc = min(KC, kspan - rd * KC);  // multiple of 16
     // A fragment rows: lanes 0-7 rows 0-7 (k 0-7), 8-15 rows 8-15 (k 0-7), 16-23 rows 0-7 (k 8-15), 24-31 rows 8-15 (k 8-15)
-    const uint32_t aBase = smem_u32(sA) + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROW_BYTES + (lane >> 4) * 16;
-    // B fragment rows (= vectors): lanes 0-7 k 0-7, lanes 8-15 k 8-15 (lanes 16-31 ignored by .x2 but must be valid)
-    const uint32_t bBase = smem_u32(sB) + (warp * 8 + (lane & 7)) * ROW_BYTES + ((lane >> 3) & 1) * 16;
+    const uint32_t aBase = stg + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROW_BYTES + (lane >> 4) * 16;
+    // B fragment rows (= vectors): lanes 0-7 k 0-7, lanes 8-15 k 8-15 (the other lanes' addresses are ignored by .x2)
+    const uint32_t bBase = stg + (offB + warp * 8 + (lane & 7)) * ROW_BYTES + ((lane >> 3) & 1) * 16;
     for (int kk = 0; kk < kc; kk += 16) {
       uint32_t a0, a1, a2, a3, b0, b1;
       ldsm_x4(aBase + kk * 2, a0, a1, a2, a3);
@@ -91,6 +100,8 @@ __global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
         mma_bf16(acc, a0, a1, a2, a3, b0, b1);
       }
     }
+    __syncthreads();  // everyone is done with this stage before it is refilled
+    if (rd + 2 < rounds) issue(rd + 2);
   }
   // C fragment: rows g / g+8 (weight rows), columns 2t / 2t+1 (vectors of this warp)
   const long long vA = v0 + warp * 8 + 2 * t, vB = vA + 1;
@@ -159,14 +170,17 @@ __global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __
 
 }  // namespace
 
-cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a) {
+cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
   static bool attr_done = false;
-  const int smem = 64 * ROW_BYTES;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_skinny_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(k_skinny_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 64 * ROW_BYTES);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
+  ImGemmArgs a = a_in;
+  a.any_w2 = 0;
+  for (int j = 0; j < a.n_jobs; ++j) a.any_w2 |= a.job[j].W2 != nullptr;
+  const int smem = 2 * (a.any_w2 ? 64 : 48) * ROW_BYTES;
   int tiles = 0;
   for (int j = 0; j < a.n_jobs; ++j) tiles += (a.job[j].rows + 15) / 16;
   dim3 grid(tiles, a.ksplit, (unsigned)((a.NV + VB - 1) / VB));

@@ -121,6 +121,7 @@ struct ImGemmArgs {
   long long out_outer, out_inner, ks_stride;
   int out_cnt;
   int NV, K, ksplit;
+  int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
 };
 
 #define IM_KSPLIT 4       /* K splits of the decode projections (partials summed by the consumer) */
