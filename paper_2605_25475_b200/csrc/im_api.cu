@@ -140,6 +140,7 @@ void carve(const ImDims& p, char* base, Layout* lo) {
     const size_t stream = ((size_t)IM_ATTN_MAX_CTAS * IM_ATTN_WARPS + (size_t)p.S * p.Hkv) * p.Gq * (p.d + 2);
     lo->sc.part = (float*)take(std::max(generic, stream) * 4);
   }
+  lo->sc.mres = (float*)take((size_t)p.S * (p.Dkv + 1) * 4);
   lo->sc.rpart = (float*)take((size_t)p.S * ((p.dM + IM_READOUT_ROWS - 1) / IM_READOUT_ROWS) * p.Dkv * 4);
   lo->total = align_up(off, 256);
 }
@@ -253,6 +254,7 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max) {
     g.out_outer = (long long)p.F * p.dM;
     g.ksplit = call.ksplit_phi;
     g.ks_stride = (long long)call.n_seq * p.F * p.dM;
+    g.kc = 64;  // 18 KB of shared memory: fits next to the resident attention blocks
   }
   CKL(im_launch_gemm(L, g));
   CKL(im_launch_mem_update(L, call, ne_max));
@@ -312,7 +314,13 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     ctx->n_ctas = std::max(1, std::min(sms, IM_ATTN_MAX_CTAS));
     ctx->fast_attn = (e == cudaSuccess);
   }
-  for (int k = 0; k < 2 && e == cudaSuccess; ++k) e = cudaStreamCreateWithFlags(&ctx->side[k], cudaStreamNonBlocking);
+  {
+    // the short side kernels should be dispatched ahead of the long attention grid when both are ready
+    int prio_lo = 0, prio_hi = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+    for (int k = 0; k < 2 && e == cudaSuccess; ++k)
+      e = cudaStreamCreateWithPriority(&ctx->side[k], cudaStreamNonBlocking, prio_hi);
+  }
   for (int k = 0; k < 8 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -461,12 +469,12 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   call.ksplit_key = (p.D % (8 * IM_KSPLIT_KEY) == 0) ? IM_KSPLIT_KEY : 1;
   call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
   // Streams: s0 is the caller's; s1 / s2 carry the pieces that do not depend on each other:
-  //   s0: projections -> front (append, score, select, compact) -> attention -> merge
-  //   s1: float64 key projection (needed by front); later phi of the evicted keys + memory write
-  //   s2: fold of the pending list (needs nothing from this call) -> readout (needs phi(q) only)
-  cudaStream_t s0 = (cudaStream_t)cuda_stream;
+  //   s0: indexer projections -> front (append, score, select, gather, compact) -> attention -> merge
+  //   s1: float64 key projection (needed by front); later phi of the evicted keys, memory write, readout finish
+  //   s2: fold of the pending list (needs nothing from this call) -> phi(q) / gate projections -> readout partials
   // An evicted set larger than the pending list is accumulated into Mhat itself, which the readout
-  // reads: that case keeps everything in order on one stream.
+  // reads: that case, and contexts without the streaming attention kernel, run in order on s0.
+  cudaStream_t s0 = (cudaStream_t)cuda_stream;
   const bool conc = ctx->concurrent && ctx->fast_attn && ne_max <= p.F;
   ImLaunch L = make_launch(ctx, layer, s0);
   ImLaunch L1 = L, L2 = L;
@@ -482,15 +490,10 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CKL(im_launch_mem_fold(L2, call));
     if (conc) CK(cudaEventRecord(ctx->ev[7], L2.stream));  // fold done: it read the counters of before the call
   }
-  // a0: projections (Sec. 3.1 features, phi(q) of Eq. 5, gate of Eq. 4) as K-split partial sums
+  // a0: projections as K-split partial sums.  Indexer part (Sec. 3.1 features) on s0 ...
   ImRows r = im_rows(p);
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
-  g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
-  g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
-  g.job[2] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
-  g.job[3] = {L.w.wg, nullptr, 1, r.wg, 2};
-  g.n_jobs = p.mem ? 4 : 2;
   g.in[0] = (const bf16*)q_pre;
   g.in[1] = (const bf16*)x;
   g.in[2] = (const bf16*)q;
@@ -502,19 +505,24 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   g.NV = n_seq;
   g.K = p.D;
   g.ksplit = call.ksplit;
+  g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
+  g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
+  g.n_jobs = 2;
   CKL(im_launch_gemm(L, g));
   CKL(im_launch_proj_key_split(L1, x, n_seq, call.ksplit_key));
+  // ... memory part (phi(q) of Eq. 5, gate logit of Eq. 4) on s2, followed by the readout partials
+  if (p.mem) {
+    g.job[0] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
+    g.job[1] = {L.w.wg, nullptr, 1, r.wg, 2};
+    CKL(im_launch_gemm(L2, g));
+  }
+  const bool readout_early = !(mem_write && ne_max > p.F);
+  if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call));
   if (conc) {
-    CK(cudaEventRecord(ctx->ev[1], s0));                 // projections done
-    CK(cudaStreamWaitEvent(L2.stream, ctx->ev[1], 0));
     CK(cudaEventRecord(ctx->ev[2], L1.stream));          // key projection done
     CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
     if (mem_write) CK(cudaStreamWaitEvent(s0, ctx->ev[7], 0));  // the front kernel changes the counters
   }
-  // a6 (first half): phi(q)^T Mhat partial sums; needs the fold and phi(q) only
-  // (an evicted set larger than the pending list changes Mhat in this call: then the readout follows the write)
-  const bool readout_early = !(mem_write && ne_max > p.F);
-  if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call));
   // append + a1 (+ a2, gather, a4 when the evicted set is small enough for one block per sequence)
   const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
   CKL(im_launch_decode_front(L, call, k_new, v_new, fused ? 1 : 0, n_max));
@@ -522,13 +530,13 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CKL(im_launch_select(L, call));
     if (ne_max > 0) CKL(im_launch_gather_move(L, call, ne_max));
   }
+  if (conc) {
+    CK(cudaEventRecord(ctx->ev[3], s0));                 // evicted pairs gathered, cache compacted
+    CK(cudaStreamWaitEvent(L1.stream, ctx->ev[3], 0));
+  }
   // a3: memory write (needs the gathered evicted pairs and the fold)
   if (mem_write) {
-    if (conc) {
-      CK(cudaEventRecord(ctx->ev[3], s0));               // evicted pairs gathered, cache compacted
-      CK(cudaStreamWaitEvent(L1.stream, ctx->ev[3], 0));
-      CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0)); // the fold emptied the list the write appends to
-    }
+    if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0));  // the fold emptied the list the write appends to
     if ((rc = run_memory_write(ctx, L1, call, ne_max))) return rc;
     if (ctx->fast_attn && !readout_early) CKL(im_launch_readout(L1, call));
   }
@@ -542,17 +550,26 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     u.since = due ? 0 : u.since + 1;
     n_att = std::max(n_att, u.n);
   }
-  // a5: attention over the retained entries; a6: merge with the readout, gate, fuse
+  // a5: attention over the retained entries; a6: readout finish (Eq. 5), merge, gate, fuse (Eq. 4)
   const bool prof = ctx->prof_used + 2 <= ctx->prof_ev.size();
   if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
   if (ctx->fast_attn) {
     CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
+    if (p.mem) {
+      if (conc) {
+        CK(cudaEventRecord(ctx->ev[6], L2.stream));      // readout partials done
+        CK(cudaStreamWaitEvent(L1.stream, ctx->ev[6], 0));
+      }
+      CKL(im_launch_readout_finish(L1, call));
+    }
     if (conc) {
       CK(cudaEventRecord(ctx->ev[5], L1.stream));
-      CK(cudaEventRecord(ctx->ev[6], L2.stream));
       CK(cudaStreamWaitEvent(s0, ctx->ev[5], 0));
-      CK(cudaStreamWaitEvent(s0, ctx->ev[6], 0));
+      if (!p.mem) {  // s2 did nothing but must still join before the call returns
+        CK(cudaEventRecord(ctx->ev[6], L2.stream));
+        CK(cudaStreamWaitEvent(s0, ctx->ev[6], 0));
+      }
     }
     CKL(im_launch_attention_merge(L, call, out, ctx->n_ctas));
   } else {

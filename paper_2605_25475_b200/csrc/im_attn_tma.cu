@@ -367,24 +367,73 @@ __global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch
 }
 
 // ------------------------------------------------------------------------------------------------
-// Merge: softmax-merge of the attention partials of one (sequence, KV head) row, readout (Eq. 5)
-// from the row-chunk partials and the pending rank-one terms, gate, fuse (Eq. 4), store.
-// grid = (Hkv, n_seq), block = 32 * max(Gq, DH / 32): warp hh merges query head hh of the group
-// (each lane DH/32 output columns), all heads in parallel; the readout vector of the KV head is
-// computed once by the whole block into shared memory.
-template <int DH, typename OutT>
-__global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call,
-                                                          int n_ctas, OutT* __restrict__ out) {
-  constexpr int CPL = DH / 32;  // columns per lane
+// Readout, second half (Eq. 5 and the gate of Eq. 4), once per sequence:
+//   mres[i][col] = cscale * ( sum_chunks rpart[col] + sum_p w_p (phi_q . phi_p) v_p[col] ) / ( sum_m phi_q[m]^2 b[m] + eps )
+//   mres[i][Dkv] = g(q)
+// Runs after the memory write of the call (it reads the pending list, b and cscale) and the readout
+// partials, off the critical path of the attention kernel.  grid = n_seq, block = 256, smem = dM floats.
+__global__ void __launch_bounds__(256) k_readout_finish(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call) {
   extern __shared__ float phiq[];  // [dM] phi(q), summed over the K-split partials
   __shared__ float s_dot[64];
   __shared__ float s_red[8];
-  __shared__ float s_mkv[DH];
-  __shared__ float s_gate;
+  const int i = blockIdx.x, tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const ImRows r = im_rows(p);
+  for (int m = tid; m < p.dM; m += 256) phiq[m] = im_raw_sum(p, sc, call, i, r.theta + m);
+  __syncthreads();
+  const int np = min(st.ctr[u * CTR_STRIDE + CTR_NPEND], p.F);
+  float part_den = 0.f;
+  for (int m = tid; m < p.dM; m += 256) part_den = fmaf(phiq[m] * phiq[m], st.bvec[u * p.dM + m], part_den);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) part_den += __shfl_xor_sync(0xffffffffu, part_den, off);
+  if (lane == 0) s_red[warp] = part_den;
+  // phi_q . phi_p, two pending entries per warp at a time so that their loads overlap
+  for (int pp = warp; pp < np; pp += 16) {
+    const float* ph0 = st.pend_phi + (u * p.F + pp) * p.dM;
+    const bool two = pp + 8 < np;
+    const float* ph1 = st.pend_phi + (u * p.F + (two ? pp + 8 : pp)) * p.dM;
+    float v0 = 0.f, v1 = 0.f;
+    for (int m = lane; m < p.dM; m += 32) {
+      v0 = fmaf(phiq[m], ph0[m], v0);
+      v1 = fmaf(phiq[m], ph1[m], v1);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      v0 += __shfl_xor_sync(0xffffffffu, v0, off);
+      v1 += __shfl_xor_sync(0xffffffffu, v1, off);
+    }
+    if (lane == 0) {
+      s_dot[pp] = v0 * st.pend_w[u * p.F + pp];
+      if (two) s_dot[pp + 8] = v1 * st.pend_w[u * p.F + pp + 8];
+    }
+  }
+  __syncthreads();
+  float den = p.eps;
+  for (int k = 0; k < 8; ++k) den += s_red[k];
+  const float scale = st.cscale[u] / den;
+  const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
+  float* dst = sc.mres + (size_t)i * (p.Dkv + 1);
+  for (int col = tid; col < p.Dkv; col += 256) {
+    const float* rp = sc.rpart + (size_t)i * nchunk * p.Dkv + col;
+    float mv = 0.f;
+    for (int k = 0; k < nchunk; ++k) mv += rp[(size_t)k * p.Dkv];
+    for (int pp = 0; pp < np; ++pp) mv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mv);
+    dst[col] = scale * mv;
+  }
+  if (tid == 0) dst[p.Dkv] = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
+}
+
+// Merge: softmax-merge of the attention partials of one (sequence, KV head) row, add the gated
+// memory readout (Eq. 4), store.
+// grid = (Hkv, n_seq), block = 32 * max(Gq, DH / 32): warp hh merges query head hh of the group
+// (each lane DH/32 output columns), all heads in parallel.
+template <int DH, typename OutT>
+__global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, ImScratch sc, ImCall call, int n_ctas,
+                                                          OutT* __restrict__ out) {
+  constexpr int CPL = DH / 32;  // columns per lane
   const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
-  const size_t u = (size_t)call.layer * p.S + call.seq[i];
-  const int32_t* ctr = st.ctr + u * CTR_STRIDE;
   // ---- rebuild the tile bookkeeping of the attention kernel (lanes stride over the sequences)
   long long pref = 0, total = 0;
   int nt_i = 0;
@@ -412,40 +461,15 @@ __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, I
   const long long qrun = (total + WT - 1) / WT;
   const long long row_first = pref + (long long)h * nt_i, row_last = row_first + nt_i - 1;
   const long long row_id = (long long)i * p.Hkv + h;
-  // ---- readout of this KV head's columns: m(q)[col] (Eq. 5) and the gate (Eq. 4)
+  // gated readout of this KV head's columns (computed by k_readout_finish)
+  float gm[CPL];
+#pragma unroll
+  for (int k = 0; k < CPL; ++k) gm[k] = 0.f;
   if (p.mem) {
-    const ImRows r = im_rows(p);
-    for (int m = tid; m < p.dM; m += blockDim.x) phiq[m] = im_raw_sum(p, sc, call, i, r.theta + m);
-    if (tid == 0) s_gate = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
-    __syncthreads();
-    const int np = min(ctr[CTR_NPEND], p.F);
-    float part_den = 0.f;
-    for (int m = tid; m < p.dM; m += blockDim.x) part_den = fmaf(phiq[m] * phiq[m], st.bvec[u * p.dM + m], part_den);
+    const float* mr = sc.mres + (size_t)i * (p.Dkv + 1);
+    const float gate = mr[p.Dkv];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) part_den += __shfl_xor_sync(0xffffffffu, part_den, off);
-    if (lane == 0) s_red[warp] = part_den;
-    for (int pp = warp; pp < np; pp += nwarps) {
-      const float* ph = st.pend_phi + (u * p.F + pp) * p.dM;
-      float v = 0.f;
-      for (int m = lane; m < p.dM; m += 32) v = fmaf(phiq[m], ph[m], v);
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-      if (lane == 0) s_dot[pp] = v * st.pend_w[u * p.F + pp];
-    }
-    __syncthreads();
-    float den = p.eps;
-    for (int k = 0; k < nwarps; ++k) den += s_red[k];
-    const float cs = st.cscale[u];
-    const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
-    for (int c = tid; c < DH; c += blockDim.x) {
-      const int col = h * DH + c;
-      const float* rp = sc.rpart + (size_t)i * nchunk * p.Dkv + col;
-      float mv = 0.f;
-      for (int k = 0; k < nchunk; ++k) mv += rp[(size_t)k * p.Dkv];
-      for (int pp = 0; pp < np; ++pp) mv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mv);
-      s_mkv[c] = cs * mv / den;
-    }
-    __syncthreads();
+    for (int k = 0; k < CPL; ++k) gm[k] = gate * mr[h * DH + lane + 32 * k];
   }
   // ---- one warp per query head of the group
   for (int hh = warp; hh < p.Gq; hh += nwarps) {
@@ -475,8 +499,7 @@ __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, I
     const size_t base = ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH;
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
-      float v = res[k];
-      if (p.mem) v = fmaf(s_gate, s_mkv[lane + 32 * k], v);
+      const float v = res[k] + gm[k];
       if constexpr (sizeof(OutT) == 2) out[base + lane + 32 * k] = __float2bfloat16_rn(v);
       else out[base + lane + 32 * k] = v;
     }
@@ -537,6 +560,12 @@ cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call) {
   return cudaGetLastError();
 }
 
+cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call) {
+  k_readout_finish<<<call.n_seq, 256, (size_t)L.p.dM * 4, L.stream>>>(L.p, L.st, L.w, L.sc, call);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
                                      const void* q, int n_ctas) {
   const ImDims& p = L.p;
@@ -554,11 +583,11 @@ cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, voi
   dim3 grid(p.Hkv, call.n_seq);
   const int mthreads = 32 * std::max(p.Gq, p.d / 32);
   if (p.d == 64) {
-    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, mthreads, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
-    else k_attn_merge_rows<64, bf16><<<grid, mthreads, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
+    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (float*)out);
+    else k_attn_merge_rows<64, bf16><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (bf16*)out);
   } else {
-    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, mthreads, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (float*)out);
-    else k_attn_merge_rows<128, bf16><<<grid, mthreads, (size_t)p.dM * 4, L.stream>>>(p, L.st, L.w, L.sc, call, n_ctas, (bf16*)out);
+    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (float*)out);
+    else k_attn_merge_rows<128, bf16><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (bf16*)out);
   }
   ++*L.launches;
   return cudaGetLastError();

@@ -8,8 +8,8 @@
 
 namespace {
 
-constexpr int KC = 512;                 // K elements staged per round
-constexpr int ROW_BYTES = KC * 2 + 16;  // padded smem row: consecutive rows shift by one 16-byte bank group
+constexpr int KC_MAX = 512;  // K elements staged per round (ImGemmArgs::kc, a multiple of 16, at most this)
+// A staged row takes kc * 2 + 16 bytes: consecutive rows shift by one 16-byte bank group (conflict-free ldmatrix).
 constexpr int VB = 32;                  // vectors per CTA (4 warps x 8)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -41,6 +41,7 @@ __device__ __forceinline__ const bf16* vec_ptr(const ImGemmArgs& a, int sel, lon
 // the cp.async copies of round r+1 are in flight while round r is multiplied.
 __global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
+  const int KC = a.kc, ROW_BYTES = a.kc * 2 + 16;
   const int stage_rows = a.any_w2 ? 64 : 48;
   const int offB = a.any_w2 ? 32 : 16;  // row offset of the vector tile inside a stage
   int tile = blockIdx.x, j = 0;
@@ -173,14 +174,15 @@ __global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __
 cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_skinny_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 64 * ROW_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(k_skinny_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 64 * (KC_MAX * 2 + 16));
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
   ImGemmArgs a = a_in;
   a.any_w2 = 0;
   for (int j = 0; j < a.n_jobs; ++j) a.any_w2 |= a.job[j].W2 != nullptr;
-  const int smem = 2 * (a.any_w2 ? 64 : 48) * ROW_BYTES;
+  if (a.kc <= 0 || a.kc > KC_MAX || a.kc % 16) a.kc = KC_MAX;
+  const int smem = 2 * (a.any_w2 ? 64 : 48) * (a.kc * 2 + 16);
   int tiles = 0;
   for (int j = 0; j < a.n_jobs; ++j) tiles += (a.job[j].rows + 15) / 16;
   dim3 grid(tiles, a.ksplit, (unsigned)((a.NV + VB - 1) / VB));

@@ -93,6 +93,7 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
   float* part;       // attention partials (acc[d], max, sum): generic kernel [max_seqs][H][max_splits][d + 2];
                      // streaming kernel [warps + rows][Gq][d + 2]
   float* rpart;      // [max_seqs][ceil(dM / IM_READOUT_ROWS)][Dkv] readout partials
+  float* mres;       // [max_seqs][Dkv + 1] memory readout m(q) in KV space, then the gate g(q)
 };
 
 struct ImCall {
@@ -121,6 +122,7 @@ struct ImGemmArgs {
   long long out_outer, out_inner, ks_stride;
   int out_cnt;
   int NV, K, ksplit;
+  int kc;      // K elements staged per round (0: the maximum, 512); small values keep the shared-memory footprint low
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
 };
 
@@ -164,6 +166,7 @@ bool im_attn_fast_supported(const ImDims& p);
 cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV);
 cudaError_t im_attn_prepare(const ImDims& p);
 cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call);
+cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
                                      const void* q, int n_ctas);
 cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas);
