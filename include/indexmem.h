@@ -189,14 +189,20 @@ int im_profile_begin(im_ctx* ctx, int max_records);
 int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
 
 /*
- * Execution option (no counterpart in the paper): with enable != 0 (the default where the streaming
- * attention kernel is available) im_decode_step runs the pieces of a call that do not depend on each
- * other - key projection, fold of the pending memory writes, readout, memory write - on two internal
- * side streams that fork from and join back into `cuda_stream` inside the call; with 0 everything is
- * enqueued on `cuda_stream` in order.  Results are identical.  The fork/join uses events only and can
- * be captured into a CUDA graph.
+ * Execution options (no counterpart in the paper).  Results are identical for every setting.
+ *   IM_OPT_CONCURRENCY   1 (default where the streaming attention kernel is available): im_decode_step
+ *                        runs the pieces of a call that do not depend on each other - fold of the pending
+ *                        memory writes, phi(q) projection and readout, memory write - on two internal side
+ *                        streams that fork from and join back into `cuda_stream` inside the call (events
+ *                        only, so the pattern can be captured into a CUDA graph); 0: everything is
+ *                        enqueued on `cuda_stream` in order.
+ *   IM_OPT_PREFETCH_NEXT 1 (default): while the attention kernel of layer l streams the K/V cache,
+ *                        im_decode_step prefetches into L2 what the small latency-bound kernels of layer
+ *                        (l + 1) mod n_layers will read for the same sequences (weights, indexer key cache,
+ *                        counters, pending memory terms); none of it depends on the output of layer l.
  */
-int im_set_concurrency(im_ctx* ctx, int enable);
+typedef enum im_option { IM_OPT_CONCURRENCY = 0, IM_OPT_PREFETCH_NEXT = 1 } im_option;
+int im_set_option(im_ctx* ctx, int option, int value);
 
 /* Number of kernels this library has launched on behalf of `ctx` since im_create. */
 int64_t im_launch_count(im_ctx* ctx);

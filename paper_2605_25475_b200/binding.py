@@ -64,12 +64,12 @@ _lib.im_launch_count.restype = C.c_int64
 _lib.im_get_config.argtypes = [_vp, C.POINTER(im_config), C.POINTER(C.c_int32)]
 _lib.im_profile_begin.argtypes = [_vp, _i32]
 _lib.im_profile_end.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
-_lib.im_set_concurrency.argtypes = [_vp, _i32]
+_lib.im_set_option.argtypes = [_vp, _i32, _i32]
 _lib.im_last_error.restype = C.c_char_p
 
 EXPORTED = ("im_workspace_bytes", "im_create", "im_destroy", "im_reset", "im_prefill_chunk", "im_decode_step",
             "im_set_weights", "im_get_weights", "im_state_export", "im_state_import", "im_topb_select",
-            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_concurrency")
+            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option")
 
 
 def _check(rc: int):
@@ -171,8 +171,11 @@ def im_profile_end(ctx):
     return ms.value, n.value
 
 
-def im_set_concurrency(ctx, enable: bool):
-    _check(_lib.im_set_concurrency(ctx, 1 if enable else 0))
+IM_OPT_CONCURRENCY, IM_OPT_PREFETCH_NEXT = 0, 1
+
+
+def im_set_option(ctx, option: int, value: int):
+    _check(_lib.im_set_option(ctx, option, value))
 
 
 def im_launch_count(ctx) -> int:

@@ -169,6 +169,7 @@ struct im_ctx {
   cudaStream_t side[2] = {nullptr, nullptr};
   cudaEvent_t ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   bool concurrent = false;
+  bool prefetch_next = true;         // warm L2 with the next layer's weights / index state during attention
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
   std::vector<cudaEvent_t> prof_ev;  // pairs (start, stop)
   size_t prof_used = 0;              // events recorded so far
@@ -505,6 +506,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   g.NV = n_seq;
   g.K = p.D;
   g.ksplit = call.ksplit;
+  const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
   g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
   g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
   g.n_jobs = 2;
@@ -518,13 +520,20 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   }
   const bool readout_early = !(mem_write && ne_max > p.F);
   if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call));
+  if (ctx->prefetch_next && ctx->fast_attn) {
+    // warm L2 for the next layer's small kernels while this layer's attention streams K/V
+    ImLaunch Lp = L2;
+    ImCall nxt = call;
+    nxt.layer = (layer + 1) % p.L;
+    Lp.w = ctx->lo.w[nxt.layer];
+    CKL(im_launch_prefetch_layer(Lp, nxt));
+  }
   if (conc) {
     CK(cudaEventRecord(ctx->ev[2], L1.stream));          // key projection done
     CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
     if (mem_write) CK(cudaStreamWaitEvent(s0, ctx->ev[7], 0));  // the front kernel changes the counters
   }
-  // append + a1 (+ a2, gather, a4 when the evicted set is small enough for one block per sequence)
-  const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
+  // append + a1 (+ a2, gather, a4 when the evicted set is small enough for one block / cluster per sequence)
   CKL(im_launch_decode_front(L, call, k_new, v_new, fused ? 1 : 0, n_max));
   if (due && !fused) {
     CKL(im_launch_select(L, call));
@@ -580,10 +589,13 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   return IM_OK;
 }
 
-int im_set_concurrency(im_ctx* ctx, int enable) {
+int im_set_option(im_ctx* ctx, int option, int value) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
-  ctx->concurrent = enable != 0;
-  return IM_OK;
+  switch (option) {
+    case IM_OPT_CONCURRENCY: ctx->concurrent = value != 0; return IM_OK;
+    case IM_OPT_PREFETCH_NEXT: ctx->prefetch_next = value != 0; return IM_OK;
+    default: return fail(IM_ERR_ARG, "unknown option %d", option);
+  }
 }
 
 int im_profile_begin(im_ctx* ctx, int max_records) {

@@ -50,11 +50,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   }
   return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+// L2 policy for data that is read once per step (the K/V stream, Mhat): evict first, so that the
+// small working set prefetched for the next layer's latency-bound kernels stays resident.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(pol)
       : "memory");
+}
+__device__ __forceinline__ float4 ldg_stream(const float4* ptr, uint64_t pol) {
+  float4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr), "l"(pol));
+  return v;
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -154,6 +167,7 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   int nt = tiles_of(s_n[i]);
   int h = (int)((run0 - s_pref[i]) / nt), tt = (int)((run0 - s_pref[i]) % nt);
 
+  const uint64_t pol = policy_evict_first();
   // iterator used by the producer side (runs STAGES tiles ahead of the consumer side)
   int pi = i, ph = h, ptt = tt, pnt = nt;
   long long issued = run0;
@@ -166,8 +180,8 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     mbar_expect_tx(bar, STAGE_BYTES);
 #pragma unroll
     for (int b = 0; b < BOXES; ++b) {
-      tma_load_2d(dst + b * (TILE * 128), &tmK, b * 64, row, bar);
-      tma_load_2d(dst + TILE_BYTES + b * (TILE * 128), &tmV, b * 64, row, bar);
+      tma_load_2d(dst + b * (TILE * 128), &tmK, b * 64, row, bar, pol);
+      tma_load_2d(dst + TILE_BYTES + b * (TILE * 128), &tmV, b * 64, row, bar, pol);
     }
     // advance the producer iterator
     if (++ptt == pnt) {
@@ -339,6 +353,7 @@ __global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch
   const int m0 = rc * R_ROWS, mcnt = min(R_ROWS, p.dM - m0);
   if (threadIdx.x < R_ROWS) s_phi[threadIdx.x] = threadIdx.x < mcnt ? im_raw_sum(p, sc, call, i, r.theta + m0 + threadIdx.x) : 0.f;
   __syncthreads();
+  const uint64_t pol = policy_evict_first();
   const float* Mh = st.Mhat + (u * p.dM + m0) * (size_t)p.Dkv;
   const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
   float* dst = sc.rpart + ((size_t)i * nchunk + rc) * p.Dkv;
@@ -348,7 +363,7 @@ __global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch
     for (; m + 8 <= mcnt; m += 8) {
       float4 v[8];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = __ldg(reinterpret_cast<const float4*>(Mh + (size_t)(m + k) * p.Dkv) + c4);
+      for (int k = 0; k < 8; ++k) v[k] = ldg_stream(reinterpret_cast<const float4*>(Mh + (size_t)(m + k) * p.Dkv) + c4, pol);
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         const float f = s_phi[m + k];
@@ -357,7 +372,7 @@ __global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch
       }
     }
     for (; m < mcnt; ++m) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(Mh + (size_t)m * p.Dkv) + c4);
+      const float4 v = ldg_stream(reinterpret_cast<const float4*>(Mh + (size_t)m * p.Dkv) + c4, pol);
       const float f = s_phi[m];
       acc.x = fmaf(f, v.x, acc.x); acc.y = fmaf(f, v.y, acc.y);
       acc.z = fmaf(f, v.z, acc.z); acc.w = fmaf(f, v.w, acc.w);

@@ -1,0 +1,63 @@
+// L2 warm-up for the latency-bound kernels of the next layer call.
+//
+// A decode step visits the layers in order and streams ~350 MB per layer through the 126 MB L2, so
+// by the time a layer comes round again (one step later) none of its weights, indexer keys, counters
+// or pending memory terms are cached, and its small kernels pay a DRAM (and page-walk) round trip for
+// every dependent load.  None of that data depends on the output of the previous layer, so while the
+// attention kernel of layer l streams K/V (with an evict-first policy), this kernel prefetches what
+// layer (l + 1) mod n_layers will read for the same sequences, with an evict-last policy.
+#include "im_internal.cuh"
+
+namespace {
+
+__device__ __forceinline__ void prefetch_range(const void* base, size_t bytes, size_t tid, size_t nthreads) {
+  const char* p = static_cast<const char*>(base);
+  for (size_t off = tid * 128; off < bytes; off += nthreads * 128)
+    asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(p + off));
+}
+
+// grid = (PF_BLOCKS, 1 + n_seq): y == 0 prefetches the weights of `w`, y == 1 + i the index state of
+// call sequence i in layer `call.layer` (the caller passes the NEXT layer in both).  block = 256.
+constexpr int PF_BLOCKS = 8;
+__global__ void __launch_bounds__(256) k_prefetch_layer(ImDims p, ImState st, ImWeights w, ImCall call) {
+  const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t nth = (size_t)gridDim.x * blockDim.x;
+  if (blockIdx.y == 0) {
+    prefetch_range(w.Uq, (size_t)p.HI * p.dI * p.D * 2, tid, nth);
+    prefetch_range(w.Uk, (size_t)p.dI * p.D * 2, tid, nth);
+    prefetch_range(w.G, (size_t)p.HI * p.D * 2, tid, nth);
+    if (p.mem) {
+      prefetch_range(w.Wt, (size_t)p.dM * p.D * 2, tid, nth);
+      prefetch_range(w.wg, (size_t)p.D * 2, tid, nth);
+      prefetch_range(w.Wfh, (size_t)p.dM * p.Dkv * 2, tid, nth);
+      prefetch_range(w.Wfl, (size_t)p.dM * p.Dkv * 2, tid, nth);
+      prefetch_range(w.bg, 4, tid, nth);
+    }
+    return;
+  }
+  const int i = blockIdx.y - 1;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  const int n = max(0, min(ctr[CTR_N], p.cap));
+  prefetch_range(st.kidx + u * p.cap * p.dI, (size_t)n * p.dI * 2, tid, nth);
+  prefetch_range(st.imp + u * p.cap, (size_t)n * 4, tid, nth);
+  prefetch_range(st.pos + u * p.cap, (size_t)n * 4, tid, nth);
+  if (p.mem) {
+    const int np = max(0, min(ctr[CTR_NPEND], p.F));
+    prefetch_range(st.bvec + u * p.dM, (size_t)p.dM * 4, tid, nth);
+    prefetch_range(st.pend_phi + u * p.F * p.dM, (size_t)np * p.dM * 4, tid, nth);
+    prefetch_range(st.pend_v + u * p.F * p.Dkv, (size_t)np * p.Dkv * 2, tid, nth);
+    prefetch_range(st.pend_w + u * p.F, (size_t)np * 4, tid, nth);
+    prefetch_range(st.cscale + u, 4, tid, nth);
+  }
+}
+
+}  // namespace
+
+// `L.w` and `call.layer` must describe the layer to warm up (not the one being computed).
+cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call) {
+  dim3 grid(PF_BLOCKS, 1 + call.n_seq);
+  k_prefetch_layer<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.w, call);
+  ++*L.launches;
+  return cudaGetLastError();
+}
