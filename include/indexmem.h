@@ -210,6 +210,32 @@ int64_t im_launch_count(im_ctx* ctx);
 /* Resolved configuration (defaults filled in) and slot capacity per sequence. */
 int im_get_config(im_ctx* ctx, im_config* out, int32_t* capacity);
 
+/*
+ * Softmax attention of one query token over a given K/V set, for callers that cannot allocate.
+ * (The paper has no counterpart: this is a service entry point, not a step of the method.)
+ *
+ * Some hosts of this library may not call cudaMalloc while they run: code inside a captured or
+ * latency-critical serving loop, plug-ins that are handed a fixed memory arena, processes whose
+ * device memory is fully committed to a KV pool.  Every other attention path here needs scratch
+ * (the per-split partial results) carved out of a caller-provided workspace.  This variant keeps that
+ * scratch in a fixed array inside the library image instead: 4 MiB of device memory that every GPU
+ * loading the library holds until the process exits.  The call makes no allocation of any kind.
+ *
+ *   q    dev bf16 [n_q_heads, head_dim]
+ *   k, v dev bf16 [n_kv_heads, n, head_dim]   (one contiguous slab per KV head)
+ *   out  dev bf16 [n_q_heads, head_dim]       out_j = sum_t softmax_t(scale * q_j . k_t) v_t, KV head j / G_q
+ *   softmax_scale 0 => 1/sqrt(head_dim);  head_dim <= 256;  n_q_heads a multiple of n_kv_heads
+ * Limit: n_q_heads * ceil(n / 256) * (head_dim + 2) <= 1,048,576 (the array's float count); larger
+ * problems are rejected with IM_ERR_CAPACITY and a message naming both numbers.
+ * The first call on a device looks up the array's device address (a host-side set-up step); make
+ * that first call before any stream capture.  All calls share the one array and nothing in it
+ * needs to start at zero (every partial that is read was written by the same call), but two calls
+ * that overlap on the GPU - different streams, or different host threads - race on it: serialise
+ * them.  Kernels are enqueued on `cuda_stream`; the call does not synchronise.
+ */
+int im_attention_noalloc(const void* q, const void* k, const void* v, int n_q_heads, int n_kv_heads, int head_dim,
+                         int n, float softmax_scale, void* out, void* cuda_stream);
+
 /* Thread-local description of the last error returned on this thread ("" if none). */
 const char* im_last_error(void);
 

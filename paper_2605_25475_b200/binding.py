@@ -65,11 +65,12 @@ _lib.im_get_config.argtypes = [_vp, C.POINTER(im_config), C.POINTER(C.c_int32)]
 _lib.im_profile_begin.argtypes = [_vp, _i32]
 _lib.im_profile_end.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
 _lib.im_set_option.argtypes = [_vp, _i32, _i32]
+_lib.im_attention_noalloc.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _i32, C.c_float, _vp, _vp]
 _lib.im_last_error.restype = C.c_char_p
 
 EXPORTED = ("im_workspace_bytes", "im_create", "im_destroy", "im_reset", "im_prefill_chunk", "im_decode_step",
             "im_set_weights", "im_get_weights", "im_state_export", "im_state_import", "im_topb_select",
-            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option")
+            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc")
 
 
 def _check(rc: int):
@@ -176,6 +177,28 @@ IM_OPT_CONCURRENCY, IM_OPT_PREFETCH_NEXT = 0, 1
 
 def im_set_option(ctx, option: int, value: int):
     _check(_lib.im_set_option(ctx, option, value))
+
+
+def im_attention_noalloc(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, softmax_scale: float = 0.0,
+                         out: torch.Tensor | None = None) -> torch.Tensor:
+    """Attention of one query token over k / v without any allocation inside the library.
+
+    q bf16 [H, d], k and v bf16 [Hkv, n, d] (CUDA, contiguous).  The scratch is a fixed 4 MiB array
+    inside the library, so H * ceil(n / 256) * (d + 2) must not exceed 1,048,576; calls must not
+    overlap on the GPU.  Pass `out` (bf16 [H, d]) to keep this wrapper from allocating the result.
+    """
+    H, d = q.shape
+    Hkv, n, d2 = k.shape
+    bf = torch.bfloat16
+    _dev(q, bf, H * d, "q"); _dev(k, bf, Hkv * n * d, "k"); _dev(v, bf, Hkv * n * d, "v")
+    if d2 != d:
+        raise ValueError("head_dim mismatch")
+    if out is None:
+        out = torch.empty((H, d), dtype=bf, device=q.device)
+    _dev(out, bf, H * d, "out")
+    _check(_lib.im_attention_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), H, Hkv, d, n, softmax_scale,
+                                     out.data_ptr(), _stream()))
+    return out
 
 
 def im_launch_count(ctx) -> int:

@@ -34,6 +34,12 @@ int fail(int code, const char* fmt, ...) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+}  // namespace
+
+int im_fail_message(int code, const char* msg) { return fail(code, "%s", msg); }
+
+namespace {
+
 struct Layout {
   ImState st;
   ImScratch sc;

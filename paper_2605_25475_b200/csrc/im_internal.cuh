@@ -126,6 +126,7 @@ struct ImGemmArgs {
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
 };
 
+#define IM_NOALLOC_MAX_FLOATS (1u << 20) /* floats in the built-in scratch array of im_attention_noalloc (4 MiB) */
 #define IM_KSPLIT 4       /* K splits of the decode projections (partials summed by the consumer) */
 #define IM_KSPLIT_KEY 16  /* K splits of the float64 indexer-key projection in decode */
 #define IM_FRONT_MAX_N 6144 /* entries the fused decode front kernel can select among (keys in shared memory) */
@@ -149,6 +150,9 @@ struct ImLaunch {
   cudaStream_t stream;
   int64_t* launches;
 };
+
+// records `msg` as the calling thread's last error and returns `code` (defined next to im_last_error)
+int im_fail_message(int code, const char* msg);
 
 // ---- kernels' host launchers (each returns the cudaError of the launch)
 cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a);
