@@ -1,0 +1,106 @@
+"""Parity at the benchmark's full layer shape and launch configuration (``-m gpu``).
+
+32 query / 8 KV heads, d = 128, B = 2048, batch 32, several layers in one context, decode steps
+replayed from a CUDA graph with the side streams on - exactly how bench.py drives the library.  The
+CPU oracle follows two sampled (layer, sequence) units through the same inputs (it cannot afford all
+64); for the other units properties that hold at any size are checked: entry count, sinks, distinct
+positions, evicted count, finite outputs.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import indexmem_oracle as orc
+from paper_2605_25475_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def test_stack_shape_sampled_units_under_graph_replay():
+    from paper_2605_25475_b200 import binding as im
+    from tests.parity import bf16_ulp
+    wl = synth.CONFIGS["llama8b_stack"].replace(name="stack_sampled", n_layers=2, ctx=4096)
+    dev = torch.device("cuda:0")
+    g = im.IndexMem(im.Config(n_layers=wl.n_layers, max_seqs=wl.n_seq, n_q_heads=wl.H, n_kv_heads=wl.Hkv,
+                              head_dim=wl.d, budget=wl.B, max_chunk=wl.chunk, n_sink=wl.n_sink), dev)
+    ids = list(range(wl.n_seq))
+    sampled = [(0, 5), (1, 29)]
+    oracles = {}
+    for layer in range(wl.n_layers):
+        w = synth.make_weights(wl, layer)
+        g.set_weights(layer, w)
+        for (l, s) in sampled:
+            if l == layer:
+                o = orc.OracleLayer(orc.OracleConfig(H=wl.H, Hkv=wl.Hkv, d=wl.d, B=wl.B, n_sink=wl.n_sink), 1)
+                o.set_weights({k: synth.f32(v) for k, v in w.items()})
+                oracles[(l, s)] = o
+    for c in range(wl.ctx // wl.chunk):
+        for layer in range(wl.n_layers):
+            X, Q, K, V = synth.prefill_inputs(wl, layer, c)
+            g.prefill_chunk(layer, ids, X.to(dev), Q.to(dev), K.to(dev), V.to(dev))
+            for (l, s), o in oracles.items():
+                if l == layer:
+                    o.prefill_chunk(0, synth.f32(X[s]), synth.f32(Q[s]), synth.f32(K[s]), synth.f32(V[s]))
+    assert g.status() == 0
+    for (l, s), o in oracles.items():
+        assert sorted(g.export(l, s, im.IM_S_POS).tolist()) == o.positions(0).tolist()
+
+    # decode: static input buffers, one captured step, replayed (bench.py's launch configuration)
+    n_steps = 4
+    ins = [[synth.decode_inputs(wl, layer, st) for layer in range(wl.n_layers)] for st in range(n_steps)]
+    sx = torch.empty((wl.n_layers, wl.n_seq, wl.D), dtype=torch.bfloat16, device=dev)
+    sq = torch.empty((wl.n_layers, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=dev)
+    sk = torch.empty((wl.n_layers, wl.n_seq, wl.Hkv, wl.d), dtype=torch.bfloat16, device=dev)
+    sv = torch.empty_like(sk)
+    out = torch.empty((wl.n_layers, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=dev)
+
+    def load(st):
+        for layer in range(wl.n_layers):
+            x, q, k, v = ins[st][layer]
+            sx[layer].copy_(x); sq[layer].copy_(q); sk[layer].copy_(k); sv[layer].copy_(v)
+
+    def one_step():
+        for layer in range(wl.n_layers):
+            g.decode_step(layer, ids, sx[layer], sq[layer], sq[layer], sk[layer], sv[layer], out[layer])
+
+    stream = torch.cuda.Stream(dev)
+    with torch.cuda.stream(stream):
+        load(0)
+        one_step()                      # eager first step: reaches n = B
+        stream.synchronize()
+        results = [out.float().cpu().numpy().copy()]
+        graph = torch.cuda.CUDAGraph()
+        load(1)
+        with torch.cuda.graph(graph, stream=stream):
+            one_step()
+        for st in range(1, n_steps):
+            load(st)
+            graph.replay()
+            stream.synchronize()
+            results.append(out.float().cpu().numpy().copy())
+    assert g.status() == 0
+
+    # oracle on the sampled units
+    for (l, s), o in oracles.items():
+        for st in range(n_steps):
+            x, q, k, v = ins[st][l]
+            ob, od = o.decode_step(0, synth.f32(x[s]), synth.f32(q[s]), synth.f32(q[s]), synth.f32(k[s]), synth.f32(v[s]))
+            got = results[st][l, s].astype(np.float64)
+            scale = np.abs(od).max()
+            half_ulp = 0.5 * bf16_ulp(np.maximum(np.abs(od), np.abs(got)))
+            assert np.all(np.abs(got - od) <= 2e-3 * scale + half_ulp), f"unit {(l, s)} step {st}"
+        assert sorted(g.export(l, s, im.IM_S_POS).tolist()) == o.positions(0).tolist()
+        Mo, bo = o.memory_kv(0)
+        Mg = g.export(l, s, im.IM_S_M).astype(np.float64)
+        assert np.abs(Mg - Mo).max() <= 2e-3 * np.abs(Mo).max()
+        assert np.abs(g.export(l, s, im.IM_S_B) - bo).max() <= 2e-3 * np.abs(bo).max()
+
+    # properties for every unit
+    for layer in range(wl.n_layers):
+        for s in range(0, wl.n_seq, 7):
+            cnt = g.counts(layer, s)
+            assert cnt["n"] == wl.B and cnt["T"] == wl.ctx + n_steps and cnt["n_evicted"] == 1
+            pos = g.export(layer, s, im.IM_S_POS)
+            assert len(set(pos.tolist())) == wl.B and set(range(wl.n_sink)) <= set(pos.tolist())
+            assert pos.max() < wl.ctx + n_steps
+    assert np.isfinite(results[-1]).all()
