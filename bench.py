@@ -240,11 +240,17 @@ def run_ours(args, rank, world, device):
         "hbm_frac_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"],
         "roofline": {"bound": "hbm", "kernel": "k_attn_stream", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     "traffic": args.traffic, "bytes_per_launch": ab["attn_launch"],
+                     "traffic": args.traffic if wl.name == "llama8b_stack" else None, "bytes_per_launch": ab["attn_launch"],
                      "us_per_launch": attn_launch_s * 1e6},
         "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
     }
     return res, wl
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_attn_stream launch (32 sequences, n = 2049 keys,
+# 8 KV heads of 128), from the ncu capture summarised under profiles/; a launch has this size whatever
+# the number of layers or the ingested context, so the figure needs no scaling.
+ATTN_TRAFFIC_NCU = 272.0e6
 
 
 def run_e2e(args, wl, g, ids, inputs, stream, world, device):
@@ -364,7 +370,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: run only this many layers (not the headline workload)")
     ap.add_argument("--context", type=int, default=0, help="profiling aid: ingest only this many context tokens")
-    ap.add_argument("--traffic", type=float, default=None,
+    ap.add_argument("--traffic", type=float, default=ATTN_TRAFFIC_NCU,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as is)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
