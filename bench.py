@@ -247,6 +247,60 @@ def run_ours(args, rank, world, device):
     return res, wl
 
 
+def run_prefill(args, device):
+    """Profiling aid, not the headline metric: chunked prefill of the Mistral-shaped configuration
+    (one layer, chunks of 2048 tokens into a budget of 2048), with the scoring kernel timed by the
+    library's own CUDA events for both of its implementations (tensor cores / CUDA cores)."""
+    from paper_2605_25475_b200 import binding as im
+    wl = synth.CONFIGS["mistral7b_prefill"]
+    if args.context:
+        wl = wl.replace(ctx=args.context)
+    g, ids = build_context(wl, device, ingest=False)
+    n_chunks = wl.ctx // wl.chunk
+    chunks = [synth.prefill_inputs(wl, 0, c, device) for c in range(min(n_chunks, 4))]
+    stream = torch.cuda.Stream(device)
+    HI, dI = max(1, wl.H // 4), wl.d // 8
+    res = {"mode": "prefill", "metric": "prefill_tokens_per_s", "unit": "tokens/s", "n_gpus": 1,
+           "steps": args.steps, "warmup": args.warmup, "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": wl.name, "prompt": wl.ctx, "chunk": wl.chunk, "budget": wl.B, "layers": 1,
+                      "n_seq": wl.n_seq}, "scoring": {}}
+    with torch.cuda.stream(stream):
+        for name, tensor in (("tensor_cores", 1), ("cuda_cores", 0)):
+            im.im_set_option(g.ctx, im.IM_OPT_PREFILL_TENSOR, tensor)
+            im.im_set_option(g.ctx, im.IM_OPT_PROFILE_TARGET, 1)
+
+            def one_pass():
+                g.reset()
+                for c in range(n_chunks):
+                    X, Q, K, V = chunks[c % len(chunks)]
+                    g.prefill_chunk(0, ids, X, Q, K, V)
+
+            for _ in range(args.warmup):
+                one_pass()
+            stream.synchronize()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(stream)
+            for _ in range(args.steps):
+                one_pass()
+            ev1.record(stream)
+            stream.synchronize()
+            ms = ev0.elapsed_time(ev1) / args.steps
+            im.im_profile_begin(g.ctx, n_chunks)
+            one_pass()
+            k_ms, k_n = im.im_profile_end(g.ctx)
+            assert g.status() == 0
+            # steady-state chunk: B old keys that every query sees + the chunk's own keys under the causal mask
+            pairs = wl.n_seq * (wl.B * wl.chunk + wl.chunk * (wl.chunk + 1) // 2)
+            flops = 2.0 * pairs * HI * dI
+            res["scoring"][name] = {"us_per_launch": k_ms / max(k_n, 1) * 1e3, "launches": k_n,
+                                    "algorithmic_gflop_per_steady_launch": flops / 1e9,
+                                    "ms_per_prompt": ms, "tokens_per_s": wl.n_seq * wl.ctx / (ms * 1e-3)}
+        im.im_set_option(g.ctx, im.IM_OPT_PROFILE_TARGET, 0)
+    res["value"] = res["scoring"]["tensor_cores"]["tokens_per_s"]
+    res["ms_per_step"] = res["scoring"]["tensor_cores"]["ms_per_prompt"]
+    return res
+
+
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_attn_stream launch (32 sequences, n = 2049 keys,
 # 8 KV heads of 128), from the ncu capture summarised under profiles/; a launch has this size whatever
 # the number of layers or the ingested context, so the figure needs no scaling.
@@ -366,6 +420,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_stack", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--mode", default="decode", choices=["decode", "prefill"],
+                    help="prefill: profiling aid that times the chunked prefill and its scoring kernel (1 GPU)")
     ap.add_argument("--graph", type=int, default=1, help="replay the step from a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: run only this many layers (not the headline workload)")
@@ -392,6 +448,10 @@ def main():
         import torch.distributed as dist
         _dist = dist
         dist.init_process_group("nccl", device_id=device)
+    if args.mode == "prefill":
+        if rank == 0:
+            print(json.dumps(run_prefill(args, device)), flush=True)
+        return
     res, wl = run_ours(args, rank, world, device)
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:

@@ -189,7 +189,7 @@ int im_profile_begin(im_ctx* ctx, int max_records);
 int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
 
 /*
- * Execution options (no counterpart in the paper).  Results are identical for every setting.
+ * Execution options (no counterpart in the paper).  Results are identical for every setting unless stated.
  *   IM_OPT_CONCURRENCY   1 (default where the streaming attention kernel is available): im_decode_step
  *                        runs the pieces of a call that do not depend on each other - fold of the pending
  *                        memory writes, phi(q) projection and readout, memory write - on two internal side
@@ -200,8 +200,22 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        im_decode_step prefetches into L2 what the small latency-bound kernels of layer
  *                        (l + 1) mod n_layers will read for the same sequences (weights, indexer key cache,
  *                        counters, pending memory terms); none of it depends on the output of layer l.
+ *   IM_OPT_PREFILL_TENSOR 1 (default where n_index_heads <= 8 and index_dim is 8 or 16): im_prefill_chunk
+ *                        evaluates the indexer scores of the chunk (Sec. 3.1, a dense [keys x d_I] x
+ *                        [d_I x queries * heads] contraction) on the tensor cores, float32 features split
+ *                        into three bf16 terms; 0: the CUDA-core kernel.  Both are within 1e-5 of a float32
+ *                        evaluation; they need not agree to the last bit.  Setting 1 on an unsupported
+ *                        shape returns IM_ERR_ARG.
+ *   IM_OPT_PROFILE_TARGET which kernel im_profile_begin / im_profile_end time: 0 (default) the attention
+ *                        kernel of im_decode_step, 1 the scoring kernel of im_prefill_chunk.  Cannot be
+ *                        changed while profiling is active (IM_ERR_STATE).
  */
-typedef enum im_option { IM_OPT_CONCURRENCY = 0, IM_OPT_PREFETCH_NEXT = 1 } im_option;
+typedef enum im_option {
+  IM_OPT_CONCURRENCY = 0,
+  IM_OPT_PREFETCH_NEXT = 1,
+  IM_OPT_PREFILL_TENSOR = 2,
+  IM_OPT_PROFILE_TARGET = 3
+} im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 
 /* Number of kernels this library has launched on behalf of `ctx` since im_create. */

@@ -148,6 +148,9 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   }
   lo->sc.mres = (float*)take((size_t)p.S * (p.Dkv + 1) * 4);
   lo->sc.rpart = (float*)take((size_t)p.S * ((p.dM + IM_READOUT_ROWS - 1) / IM_READOUT_ROWS) * p.Dkv * 4);
+  lo->sc.qpack = nullptr;
+  if (im_score_tc_supported(p))
+    lo->sc.qpack = (uint8_t*)take((size_t)p.S * ((p.max_chunk + IM_TC_QT - 1) / IM_TC_QT) * IM_TC_TILE_BYTES);
   lo->total = align_up(off, 256);
 }
 
@@ -177,6 +180,9 @@ struct im_ctx {
   bool concurrent = false;
   bool prefetch_next = true;         // warm L2 with the next layer's weights / index state during attention
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
+  int n_sm = 1;                      // SMs of the device
+  bool score_tc = false;             // prefill scoring runs on the tensor cores (tcgen05)
+  int prof_target = 0;               // kernel timed by im_profile_*: 0 attention (decode), 1 prefill scoring
   std::vector<cudaEvent_t> prof_ev;  // pairs (start, stop)
   size_t prof_used = 0;              // events recorded so far
 };
@@ -211,6 +217,7 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
   call->layer = layer;
   call->n_seq = n_seq;
   call->C = 1;
+  call->pack = 0;
   return IM_OK;
 }
 
@@ -321,6 +328,11 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     ctx->n_ctas = std::max(1, std::min(sms, IM_ATTN_MAX_CTAS));
     ctx->fast_attn = (e == cudaSuccess);
   }
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, ctx->device);
+  if (e == cudaSuccess && im_score_tc_supported(p)) {
+    e = im_score_tc_prepare();
+    ctx->score_tc = (e == cudaSuccess);
+  }
   {
     // the short side kernels should be dispatched ahead of the long attention grid when both are ready
     int prio_lo = 0, prio_hi = 0;
@@ -405,6 +417,7 @@ int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, 
   call.ksplit = 1;
   call.ksplit_key = 1;
   call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
+  call.pack = ctx->score_tc ? 1 : 0;
   ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
   const int NV = n_seq * chunk_len;
   // pending rank-one terms are folded into M before a compression that cannot append to the list
@@ -429,7 +442,17 @@ int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, 
   CKL(im_launch_proj_key_split(L, x, NV, 1));
   CKL(im_launch_prefill_append(L, call, k, v));
   // a1: pooled importance under the causal mask
-  CKL(im_launch_prefill_score(L, call, n_max));
+  {
+    const bool prof = ctx->prof_target == 1 && ctx->prof_used + 2 <= ctx->prof_ev.size();
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], L.stream));
+    if (call.pack) CKL(im_launch_prefill_score_tc(L, call, n_max, ctx->n_sm));
+    else CKL(im_launch_prefill_score(L, call, n_max));
+    if (prof) {
+      CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], L.stream));
+      ctx->prof_used += 2;
+    }
+  }
+  CKL(im_launch_prefill_commit(L, call));
   // a2: selection (also restarts the pooling); a4: gather the evicted pairs, fill the holes
   CKL(im_launch_select(L, call));
   if (ne_max > 0) {
@@ -566,7 +589,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     n_att = std::max(n_att, u.n);
   }
   // a5: attention over the retained entries; a6: readout finish (Eq. 5), merge, gate, fuse (Eq. 4)
-  const bool prof = ctx->prof_used + 2 <= ctx->prof_ev.size();
+  const bool prof = ctx->prof_target == 0 && ctx->prof_used + 2 <= ctx->prof_ev.size();
   if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
   if (ctx->fast_attn) {
     CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
@@ -600,6 +623,16 @@ int im_set_option(im_ctx* ctx, int option, int value) {
   switch (option) {
     case IM_OPT_CONCURRENCY: ctx->concurrent = value != 0; return IM_OK;
     case IM_OPT_PREFETCH_NEXT: ctx->prefetch_next = value != 0; return IM_OK;
+    case IM_OPT_PREFILL_TENSOR:
+      if (value && !im_score_tc_supported(ctx->p))
+        return fail(IM_ERR_ARG, "the tensor-core prefill scoring needs at most %d indexer heads of width 8 or 16", IM_TC_HP);
+      ctx->score_tc = value != 0;
+      return IM_OK;
+    case IM_OPT_PROFILE_TARGET:
+      if (value != 0 && value != 1) return fail(IM_ERR_ARG, "profile target %d: 0 = attention, 1 = prefill scoring", value);
+      if (!ctx->prof_ev.empty()) return fail(IM_ERR_STATE, "profiling is active");
+      ctx->prof_target = value;
+      return IM_OK;
     default: return fail(IM_ERR_ARG, "unknown option %d", option);
   }
 }

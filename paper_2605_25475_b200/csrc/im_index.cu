@@ -57,6 +57,36 @@ __global__ void k_prefill_append(ImDims p, ImState st, ImScratch sc, ImCall call
   float* raw = sc.raw + ((size_t)i * call.C + c) * p.R3;
   if (tid < 32) finalize_features(p, raw, tid);
   __syncthreads();
+  if (call.pack) {
+    // operand record of the tensor-core scoring: the token's features as three bf16 terms (their sum is the
+    // float32 value to 2^-24), each 16-byte row (8 features of one head slot) at its place in the
+    // shared-memory layout of a K-major operand without swizzle; alpha follows the three terms
+    const int n_qt = (call.C + IM_TC_QT - 1) / IM_TC_QT;
+    uint8_t* rec = sc.qpack + ((size_t)i * n_qt + c / IM_TC_QT) * IM_TC_TILE_BYTES;
+    const int sq = c % IM_TC_QT;
+    if (tid < 48) {
+      const int term = tid >> 4, kg = (tid >> 3) & 1, h = tid & 7;
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      if (h < p.HI && kg * 8 < p.dI) {
+        const float* y = raw + r.uq + h * p.dI + kg * 8;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float x0 = y[j];
+          const bf16 t0 = __float2bfloat16_rn(x0);
+          const float x1 = x0 - __bfloat162float(t0);
+          const bf16 t1 = __float2bfloat16_rn(x1);
+          const bf16 t2 = __float2bfloat16_rn(x1 - __bfloat162float(t1));
+          const bf16 t = term == 0 ? t0 : (term == 1 ? t1 : t2);
+          w[j >> 1] |= (uint32_t)__bfloat16_as_ushort(t) << (16 * (j & 1));
+        }
+      }
+      *reinterpret_cast<uint4*>(rec + term * (IM_TC_QT * IM_TC_HP * 32) + sq * 256 + kg * 128 + h * 16) =
+          make_uint4(w[0], w[1], w[2], w[3]);
+    } else if (tid >= 64 && tid < 64 + IM_TC_HP) {
+      const int h = tid - 64;
+      reinterpret_cast<float*>(rec + 3 * (IM_TC_QT * IM_TC_HP * 32))[sq * IM_TC_HP + h] = h < p.HI ? raw[r.g + h] : 0.f;
+    }
+  }
   const int slot = n + c;
   bf16* kid = st.kidx + (u * p.cap + slot) * p.dI;
   // k = bf16(RMSNorm(U_k x)) from the float64 projection (one K split in prefill)
@@ -373,8 +403,10 @@ cudaError_t im_launch_prefill_score(const ImLaunch& L, const ImCall& call, int n
   const size_t smem = ((size_t)PS_QT * (L.p.HI * L.p.dI + L.p.HI) + 256) * 4;
   k_prefill_score<<<grid, 256, smem, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_prefill_commit(const ImLaunch& L, const ImCall& call) {
   k_prefill_commit<<<call.n_seq, 32, 0, L.stream>>>(L.p, L.st, call);
   ++*L.launches;
   return cudaGetLastError();

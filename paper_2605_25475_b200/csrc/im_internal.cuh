@@ -14,6 +14,9 @@ typedef __nv_bfloat16 bf16;
 #define IM_ATTN_WARPS 4      /* warps per CTA of the streaming attention kernel */
 #define IM_ATTN_MAX_CTAS 512 /* upper bound of its grid (one CTA per SM) */
 #define IM_READOUT_ROWS 32   /* rows of M per readout partial */
+#define IM_TC_QT 32          /* queries per tile of the tensor-core prefill scoring */
+#define IM_TC_HP 8           /* head slots per query in its operand (indexer heads, zero padded) */
+#define IM_TC_TILE_BYTES 25600 /* one tile record: 3 bf16 terms x (256 rows x 32 bytes) + 256 alpha floats */
 
 // per-(layer, sequence) device counters
 enum { CTR_N = 0, CTR_T = 1, CTR_SINCE = 2, CTR_EVSTEPS = 3, CTR_NEVICT = 4, CTR_NPEND = 5, CTR_DIRECT = 6, CTR_NSEL = 7, CTR_STRIDE = 8 };
@@ -94,11 +97,13 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
                      // streaming kernel [warps + rows][Gq][d + 2]
   float* rpart;      // [max_seqs][ceil(dM / IM_READOUT_ROWS)][Dkv] readout partials
   float* mres;       // [max_seqs][Dkv + 1] memory readout m(q) in KV space, then the gate g(q)
+  uint8_t* qpack;    // [n_seq][ceil(C / IM_TC_QT)][IM_TC_TILE_BYTES] query operand of the tensor-core prefill scoring
 };
 
 struct ImCall {
   int layer, n_seq, C;
   int prefill;    // 1: im_prefill_chunk (always compresses), 0: im_decode_step (compresses every tau-th token)
+  int pack;       // prefill: 1 = the append kernel also writes the operand records of the tensor-core scoring
   int phi_large;  // 1: phi of the evicted keys lives in ImScratch::phi, 0: in the K-split partials phip
   int ksplit, ksplit_key, ksplit_phi;  // K splits of the projections / key projection / phi partials of this call
   int seq[IM_MAX_CALL_SEQS];
@@ -132,16 +137,6 @@ struct ImGemmArgs {
 #define IM_FRONT_MAX_N 6144 /* entries the fused decode front kernel can select among (keys in shared memory) */
 #define IM_FRONT_MAX_NE 16  /* evicted entries per sequence the fused decode front kernel handles */
 
-struct ImProjJob {
-  const bf16* W;   // [rows][Dn]
-  const bf16* in;  // [NV][Dn]
-  int rows, row0;  // rows of this job, first output row
-};
-struct ImProjJobs {
-  ImProjJob job[5];
-  int n_jobs, total_rows, Dn, NV, out_stride;
-};
-
 struct ImLaunch {
   ImDims p;
   ImState st;
@@ -165,6 +160,11 @@ cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_prefill_append(const ImLaunch& L, const ImCall& call, const void* k, const void* v);
 cudaError_t im_launch_prefill_score(const ImLaunch& L, const ImCall& call, int n_max);
+// tensor-core (tcgen05) version of the prefill scoring; needs ImCall::pack set for the append kernel
+bool im_score_tc_supported(const ImDims& p);
+cudaError_t im_score_tc_prepare();
+cudaError_t im_launch_prefill_score_tc(const ImLaunch& L, const ImCall& call, int n_max, int n_sm);
+cudaError_t im_launch_prefill_commit(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const void* q, void* out, int n_max);
 bool im_attn_fast_supported(const ImDims& p);

@@ -237,3 +237,42 @@ def test_long_interval_unfused_select_and_large_evicted_set():
         p.decode(s)
     assert p.o.evict_steps(0) == 1 + 2
     assert p.stats["max_M_err"] <= 2e-3
+
+
+# ------------------------------------------------------------------ prefill scoring: tensor-core and CUDA-core kernels
+@pytest.mark.parametrize("tensor", [1, 0])
+def test_prefill_scoring_both_kernels_several_key_tiles_ragged_chunks(im, tensor):
+    """Llama-shaped widths (8 x 16); 5 chunks of 333 tokens (not a multiple of the 32-query tile) into a
+    budget of 700, so that a call scores 1033 keys = 8 full key tiles and a ragged ninth, old keys that every
+    query sees next to chunk keys under the causal mask, for three sequences at once."""
+    wl = synth.CONFIGS["mistral7b_prefill"].replace(name="score_both", n_seq=3, ctx=5 * 333, chunk=333, B=700, steps=2)
+    p = _pair(wl)
+    im.im_set_option(p.g.ctx, im.IM_OPT_PREFILL_TENSOR, tensor)
+    for c in range(5):
+        p.prefill(c)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_score_err"] <= 1e-5 and p.stats["max_M_err"] <= 2e-3
+    assert p.stats["cut_divergences"] <= 2
+
+
+def test_prefill_scoring_tensor_identity_activation_and_narrow_widths(im):
+    """act = identity (scores of both signs: the pooled maximum goes through negative values) at the tiny
+    widths (one indexer head of 8 features: zero-padded head slots and K group), two chunks."""
+    wl = TINY.replace(name="score_ident", ctx=2 * 190, chunk=190, B=120, steps=2, n_needles=0)
+    p = _pair(wl, act=1)
+    for c in range(2):
+        p.prefill(c)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_score_err"] <= 1e-5
+
+
+def test_prefill_scoring_tensor_unsupported_shape_is_refused(im):
+    """More than eight indexer heads: the tensor-core kernel is not used, asking for it is an error."""
+    wl = TINY.replace(name="score_wide", H=48, Hkv=4, ctx=100, chunk=100, B=60, steps=1, n_needles=0)
+    p = _pair(wl)                                   # H_I = 12
+    with pytest.raises(im.IndexMemError):
+        im.im_set_option(p.g.ctx, im.IM_OPT_PREFILL_TENSOR, 1)
+    p.prefill(0)
+    p.decode(0)
