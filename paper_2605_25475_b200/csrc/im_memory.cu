@@ -118,18 +118,17 @@ __global__ void __launch_bounds__(256) k_mem_small(ImDims p, ImState st, ImScrat
   const int ne = min(ctr[CTR_NEVICT], p.tail);
   if (ne <= 0) return;
   const int np = min(ctr[CTR_NPEND], p.F);
-  const bool large = ne > p.F;
+  if (ne > p.F) return;  // large sets: b and Mhat are updated by k_mem_accumulate; cscale stays 1
   const float c_new = p.lambda * st.cscale[u];
   for (int m = threadIdx.x; m < p.dM; m += blockDim.x) {
     float s = 0.f;
     for (int e = 0; e < ne; ++e) {
       const float f = phi_at(p, sc, call, i, e, m);
       s = fmaf(f, f, s);
-      if (!large && np + e < p.F) st.pend_phi[(u * p.F + np + e) * p.dM + m] = f;
+      if (np + e < p.F) st.pend_phi[(u * p.F + np + e) * p.dM + m] = f;
     }
     st.bvec[u * p.dM + m] = p.lambda * st.bvec[u * p.dM + m] + p.eta * s;
   }
-  if (large) return;  // Mhat <- lambda Mhat + eta Phi^T V is done by k_mem_accumulate; cscale stays 1
   if (np + ne > p.F) {
     if (threadIdx.x == 0) atomicOr(st.status, ST_COUNT);  // the fold kernel should have made room
     return;
@@ -149,7 +148,8 @@ __global__ void __launch_bounds__(256) k_mem_small(ImDims p, ImState st, ImScrat
 }
 
 // Evicted sets larger than F: Mhat <- lambda * Mhat + eta * sum_e phi_e v_e^T (the list is empty and
-// cscale is 1 after the fold).  grid = (ceil(Dkv/64), ceil(dM/64), n_seq), block = 256.
+// cscale is 1 after the fold), and b <- lambda b + eta sum_e phi_e^2 by the blocks of the first tile column
+// (they stage every phi row of their 64 memory rows anyway).  grid = (ceil(Dkv/64), ceil(dM/64), n_seq), block = 256.
 __global__ void __launch_bounds__(256) k_mem_accumulate(ImDims p, ImState st, ImScratch sc, ImCall call) {
   __shared__ float s_a[16][64 + 4];
   __shared__ float s_b[16][64 + 4];
@@ -164,6 +164,7 @@ __global__ void __launch_bounds__(256) k_mem_accumulate(ImDims p, ImState st, Im
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+  float bsum = 0.f;
   const float* phi = sc.phi + (size_t)i * p.tail * p.dM;
   const bf16* V = sc.evV + (size_t)i * p.tail * p.Dkv;
   for (int k0 = 0; k0 < ne; k0 += 16) {
@@ -180,6 +181,8 @@ __global__ void __launch_bounds__(256) k_mem_accumulate(ImDims p, ImState st, Im
     }
     __syncthreads();
     const int lim = min(16, ne - k0);
+    if (blockIdx.x == 0 && threadIdx.x < 64)
+      for (int e = 0; e < lim; ++e) bsum = fmaf(s_a[e][threadIdx.x], s_a[e][threadIdx.x], bsum);
     for (int e = 0; e < lim; ++e) {
       float av[4], bv[4];
 #pragma unroll
@@ -191,6 +194,10 @@ __global__ void __launch_bounds__(256) k_mem_accumulate(ImDims p, ImState st, Im
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
     }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < 64 && m0 + threadIdx.x < p.dM) {
+    float* bp = st.bvec + u * p.dM + m0 + threadIdx.x;
+    *bp = p.lambda * *bp + p.eta * bsum;
   }
   float* Mh = st.Mhat + u * p.dM * p.Dkv;
 #pragma unroll
