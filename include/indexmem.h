@@ -191,11 +191,13 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
 /*
  * Execution options (no counterpart in the paper).  Results are identical for every setting unless stated.
  *   IM_OPT_CONCURRENCY   1 (default where the streaming attention kernel is available): im_decode_step
- *                        runs the pieces of a call that do not depend on each other - fold of the pending
- *                        memory writes, phi(q) projection and readout, memory write - on two internal side
- *                        streams that fork from and join back into `cuda_stream` inside the call (events
- *                        only, so the pattern can be captured into a CUDA graph); 0: everything is
- *                        enqueued on `cuda_stream` in order.
+ *                        starts the attention kernel at once over the entries cached before the call and
+ *                        runs the rest of the call (projections, append / score / select, memory write,
+ *                        readout) next to it on three internal side streams that fork from and join back
+ *                        into `cuda_stream` inside the call (events only, so the pattern can be captured
+ *                        into a CUDA graph); the merge adds the new token and removes the evicted entries
+ *                        from the softmax sums again, so the result is the attention over the retained set.
+ *                        0: everything is enqueued on `cuda_stream` in order.
  *   IM_OPT_PREFETCH_NEXT 1 (default): while the attention kernel of layer l streams the K/V cache,
  *                        im_decode_step prefetches into L2 what the small latency-bound kernels of layer
  *                        (l + 1) mod n_layers will read for the same sequences (weights, indexer key cache,
@@ -217,6 +219,15 @@ typedef enum im_option {
   IM_OPT_PROFILE_TARGET = 3
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
+
+/*
+ * Event counters kept on the device (no counterpart in the paper).  Synchronises the device.
+ *   IM_COUNT_MERGE_RECOMPUTE  query heads for which the merge of a decode call with concurrency found more
+ *                             than 90 % of the softmax mass on entries evicted in the same call and recomputed
+ *                             the head over the retained entries instead of removing those terms from the sums.
+ */
+typedef enum im_counter { IM_COUNT_MERGE_RECOMPUTE = 0 } im_counter;
+int im_event_count(im_ctx* ctx, int counter, int64_t* value);
 
 /* Number of kernels this library has launched on behalf of `ctx` since im_create. */
 int64_t im_launch_count(im_ctx* ctx);

@@ -65,12 +65,13 @@ _lib.im_get_config.argtypes = [_vp, C.POINTER(im_config), C.POINTER(C.c_int32)]
 _lib.im_profile_begin.argtypes = [_vp, _i32]
 _lib.im_profile_end.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
 _lib.im_set_option.argtypes = [_vp, _i32, _i32]
+_lib.im_event_count.argtypes = [_vp, _i32, C.POINTER(C.c_int64)]
 _lib.im_attention_noalloc.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _i32, C.c_float, _vp, _vp]
 _lib.im_last_error.restype = C.c_char_p
 
 EXPORTED = ("im_workspace_bytes", "im_create", "im_destroy", "im_reset", "im_prefill_chunk", "im_decode_step",
             "im_set_weights", "im_get_weights", "im_state_export", "im_state_import", "im_topb_select",
-            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc")
+            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc", "im_event_count")
 
 
 def _check(rc: int):
@@ -199,6 +200,15 @@ def im_attention_noalloc(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, soft
     _check(_lib.im_attention_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), H, Hkv, d, n, softmax_scale,
                                      out.data_ptr(), _stream()))
     return out
+
+
+IM_COUNT_MERGE_RECOMPUTE = 0
+
+
+def im_event_count(ctx, counter: int) -> int:
+    v = C.c_int64(0)
+    _check(_lib.im_event_count(ctx, counter, C.byref(v)))
+    return int(v.value)
 
 
 def im_launch_count(ctx) -> int:

@@ -173,9 +173,9 @@ struct im_ctx {
   alignas(64) unsigned char mapK[128];  // TMA descriptors of the K / V caches
   alignas(64) unsigned char mapV[128];
   bool fast_attn = false;
-  // Independent pieces of one decode call run on two side streams that fork from and join back into
+  // Independent pieces of one decode call run on three side streams that fork from and join back into
   // the caller's stream (plain event dependencies, so the pattern can be captured into a CUDA graph).
-  cudaStream_t side[2] = {nullptr, nullptr};
+  cudaStream_t side[3] = {nullptr, nullptr, nullptr};
   cudaEvent_t ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   bool concurrent = false;
   bool prefetch_next = true;         // warm L2 with the next layer's weights / index state during attention
@@ -218,6 +218,7 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
   call->n_seq = n_seq;
   call->C = 1;
   call->pack = 0;
+  call->defer = 0;
   return IM_OK;
 }
 
@@ -337,14 +338,14 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     // the short side kernels should be dispatched ahead of the long attention grid when both are ready
     int prio_lo = 0, prio_hi = 0;
     if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
-    for (int k = 0; k < 2 && e == cudaSuccess; ++k)
+    for (int k = 0; k < 3 && e == cudaSuccess; ++k)
       e = cudaStreamCreateWithPriority(&ctx->side[k], cudaStreamNonBlocking, prio_hi);
   }
   for (int k = 0; k < 8 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
-    for (int k = 0; k < 2; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
+    for (int k = 0; k < 3; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
     for (int k = 0; k < 8; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
     delete ctx;
     return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
@@ -356,7 +357,7 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
 int im_destroy(im_ctx* ctx) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   cudaError_t e = cudaDeviceSynchronize();
-  for (int k = 0; k < 2; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
+  for (int k = 0; k < 3; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
   for (int k = 0; k < 8; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   delete ctx;
   if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
@@ -498,29 +499,47 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   call.ksplit = pick_ksplit(p.D, IM_KSPLIT);
   call.ksplit_key = (p.D % (8 * IM_KSPLIT_KEY) == 0) ? IM_KSPLIT_KEY : 1;
   call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
-  // Streams: s0 is the caller's; s1 / s2 carry the pieces that do not depend on each other:
-  //   s0: indexer projections -> front (append, score, select, gather, compact) -> attention -> merge
-  //   s1: float64 key projection (needed by front); later phi of the evicted keys, memory write, readout finish
-  //   s2: fold of the pending list (needs nothing from this call) -> phi(q) / gate projections -> readout partials
-  // An evicted set larger than the pending list is accumulated into Mhat itself, which the readout
-  // reads: that case, and contexts without the streaming attention kernel, run in order on s0.
+  // Two schedules.
+  //  (A) deferred compaction - the streaming attention kernel is available and the selection, if one is
+  //      due, fits the fused front kernel: attention needs nothing of this call but q, so it starts at
+  //      once over the entries cached before the call.  The merge adds the new token, removes the evicted
+  //      entries again (exactly, see k_attn_merge_rows), and the holes are filled afterwards.
+  //        s0: attention ------------------------------------------------> merge -> fill holes, publish count
+  //        s1: indexer projections -> front (append, score, select, gather) -> phi of the evicted keys ->
+  //            memory write -> readout finish
+  //        s2: fold of the pending list -> phi(q) / gate projections -> readout partials -> L2 prefetch
+  //        s3: float64 key projection (needed by front)
+  //      With IM_OPT_CONCURRENCY off the same kernels run on s0 in an order that respects these arrows.
+  //  (B) in order on s0, attention after the compaction: everything else (large evicted sets, budgets
+  //      beyond the fused front kernel, head shapes without the streaming attention kernel).
   cudaStream_t s0 = (cudaStream_t)cuda_stream;
-  const bool conc = ctx->concurrent && ctx->fast_attn && ne_max <= p.F;
+  const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
+  const bool defer = ctx->fast_attn && (!due || fused) && ne_max <= p.F;
+  const bool conc = defer && ctx->concurrent;
+  call.defer = defer ? 1 : 0;
   ImLaunch L = make_launch(ctx, layer, s0);
-  ImLaunch L1 = L, L2 = L;
+  ImLaunch L1 = L, L2 = L, L3 = L;
   if (conc) {
     L1.stream = ctx->side[0];
     L2.stream = ctx->side[1];
+    L3.stream = ctx->side[2];
     CK(cudaEventRecord(ctx->ev[0], s0));
     CK(cudaStreamWaitEvent(L1.stream, ctx->ev[0], 0));
     CK(cudaStreamWaitEvent(L2.stream, ctx->ev[0], 0));
+    CK(cudaStreamWaitEvent(L3.stream, ctx->ev[0], 0));
+  }
+  const bool prof = ctx->prof_target == 0 && ctx->prof_used + 2 <= ctx->prof_ev.size();
+  if (defer && conc) {  // a5 first: it overlaps with everything below
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
+    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
   }
   const bool mem_write = due && ne_max > 0 && p.mem;
   if (mem_write) {
     CKL(im_launch_mem_fold(L2, call));
     if (conc) CK(cudaEventRecord(ctx->ev[7], L2.stream));  // fold done: it read the counters of before the call
   }
-  // a0: projections as K-split partial sums.  Indexer part (Sec. 3.1 features) on s0 ...
+  // a0: projections as K-split partial sums: indexer part (Sec. 3.1 features) ...
   ImRows r = im_rows(p);
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
@@ -535,20 +554,23 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   g.NV = n_seq;
   g.K = p.D;
   g.ksplit = call.ksplit;
-  const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
+  g.kc = conc ? 64 : 0;  // next to the attention CTAs only a small staging buffer fits into an SM's shared memory
   g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
   g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
   g.n_jobs = 2;
-  CKL(im_launch_gemm(L, g));
-  CKL(im_launch_proj_key_split(L1, x, n_seq, call.ksplit_key));
-  // ... memory part (phi(q) of Eq. 5, gate logit of Eq. 4) on s2, followed by the readout partials
+  CKL(im_launch_gemm(L1, g));
+  CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
+  if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // key projection done
+  // ... memory part (phi(q) of Eq. 5, gate logit of Eq. 4), followed by the readout partials
   if (p.mem) {
     g.job[0] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
     g.job[1] = {L.w.wg, nullptr, 1, r.wg, 2};
     CKL(im_launch_gemm(L2, g));
   }
+  // an evicted set larger than the pending list is accumulated into Mhat itself, which the readout reads
   const bool readout_early = !(mem_write && ne_max > p.F);
   if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call));
+  if (conc && p.mem) CK(cudaEventRecord(ctx->ev[6], L2.stream));  // readout partials done
   if (ctx->prefetch_next && ctx->fast_attn) {
     // warm L2 for the next layer's small kernels while this layer's attention streams K/V
     ImLaunch Lp = L2;
@@ -558,23 +580,19 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CKL(im_launch_prefetch_layer(Lp, nxt));
   }
   if (conc) {
-    CK(cudaEventRecord(ctx->ev[2], L1.stream));          // key projection done
-    CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
-    if (mem_write) CK(cudaStreamWaitEvent(s0, ctx->ev[7], 0));  // the front kernel changes the counters
+    CK(cudaEventRecord(ctx->ev[4], L2.stream));  // s2 finished
+    CK(cudaStreamWaitEvent(L1.stream, ctx->ev[2], 0));
+    if (mem_write) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0));  // the front kernel changes the counters
   }
-  // append + a1 (+ a2, gather, a4 when the evicted set is small enough for one block / cluster per sequence)
-  CKL(im_launch_decode_front(L, call, k_new, v_new, fused ? 1 : 0, n_max));
+  // append + a1 (+ a2 and the gather of the evicted pairs when the evicted set is small enough for one
+  // block per sequence; a4 in the same kernel unless the compaction is deferred)
+  CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max));
   if (due && !fused) {
-    CKL(im_launch_select(L, call));
-    if (ne_max > 0) CKL(im_launch_gather_move(L, call, ne_max));
-  }
-  if (conc) {
-    CK(cudaEventRecord(ctx->ev[3], s0));                 // evicted pairs gathered, cache compacted
-    CK(cudaStreamWaitEvent(L1.stream, ctx->ev[3], 0));
+    CKL(im_launch_select(L1, call));
+    if (ne_max > 0) CKL(im_launch_gather_move(L1, call, ne_max));
   }
   // a3: memory write (needs the gathered evicted pairs and the fold)
   if (mem_write) {
-    if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0));  // the fold emptied the list the write appends to
     if ((rc = run_memory_write(ctx, L1, call, ne_max))) return rc;
     if (ctx->fast_attn && !readout_early) CKL(im_launch_readout(L1, call));
   }
@@ -588,29 +606,26 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     u.since = due ? 0 : u.since + 1;
     n_att = std::max(n_att, u.n);
   }
-  // a5: attention over the retained entries; a6: readout finish (Eq. 5), merge, gate, fuse (Eq. 4)
-  const bool prof = ctx->prof_target == 0 && ctx->prof_used + 2 <= ctx->prof_ev.size();
-  if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
+  // a5: attention; a6: readout finish (Eq. 5), merge, gate, fuse (Eq. 4)
   if (ctx->fast_attn) {
-    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
-    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
+    if (!(defer && conc)) {
+      if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
+      CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
+      if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
+    }
     if (p.mem) {
-      if (conc) {
-        CK(cudaEventRecord(ctx->ev[6], L2.stream));      // readout partials done
-        CK(cudaStreamWaitEvent(L1.stream, ctx->ev[6], 0));
-      }
+      if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[6], 0));
       CKL(im_launch_readout_finish(L1, call));
     }
-    if (conc) {
+    if (conc) {  // every side stream joins the caller's stream (s3 joined s1 through the key projection event)
       CK(cudaEventRecord(ctx->ev[5], L1.stream));
       CK(cudaStreamWaitEvent(s0, ctx->ev[5], 0));
-      if (!p.mem) {  // s2 did nothing but must still join before the call returns
-        CK(cudaEventRecord(ctx->ev[6], L2.stream));
-        CK(cudaStreamWaitEvent(s0, ctx->ev[6], 0));
-      }
+      CK(cudaStreamWaitEvent(s0, ctx->ev[4], 0));
     }
-    CKL(im_launch_attention_merge(L, call, out, ctx->n_ctas));
+    CKL(im_launch_attention_merge(L, call, out, ctx->n_ctas, q, k_new, v_new));
+    if (defer) CKL(im_launch_decode_commit(L, call));
   } else {
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
     CKL(im_launch_attention(L, call, q, out, n_att));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
   }
@@ -836,7 +851,7 @@ int im_state_import(im_ctx* ctx, int layer, int seq, int which, const void* host
         return fail(IM_ERR_ARG, "inconsistent counters");
       ctr[CTR_NPEND] = 0;  // pending writes cannot be imported; IM_S_M carries the folded state
       ctr[CTR_NEVICT] = 0;
-      ctr[CTR_DIRECT] = 0;
+      ctr[CTR_NNEXT] = ctr[CTR_N];
       ctr[CTR_NSEL] = 0;
       int32_t old[CTR_STRIDE];
       CK(cudaMemcpy(old, st.ctr + u * CTR_STRIDE, sizeof(old), cudaMemcpyDeviceToHost));
@@ -894,6 +909,16 @@ int im_topb_select(const float* scores, const int32_t* pos, int rows, int n, int
   if (rows < 0 || n < 0 || budget < 0 || n_sink < 0) return fail(IM_ERR_ARG, "negative size");
   if (rows == 0) return IM_OK;
   CKL(im_launch_topb(scores, pos, rows, n, budget, n_sink, keep, n_evict, (cudaStream_t)cuda_stream));
+  return IM_OK;
+}
+
+int im_event_count(im_ctx* ctx, int counter, int64_t* value) {
+  if (!ctx || !value) return fail(IM_ERR_ARG, "null argument");
+  if (counter != IM_COUNT_MERGE_RECOMPUTE) return fail(IM_ERR_ARG, "unknown counter %d", counter);
+  CK(cudaDeviceSynchronize());
+  int32_t v = 0;
+  CK(cudaMemcpy(&v, ctx->lo.st.status + 1, 4, cudaMemcpyDeviceToHost));
+  *value = v;
   return IM_OK;
 }
 

@@ -439,13 +439,38 @@ __global__ void __launch_bounds__(256) k_readout_finish(ImDims p, ImState st, Im
   if (tid == 0) dst[p.Dkv] = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
 }
 
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// one more key for a running (base 2) softmax state of one query head spread over a warp
+template <int CPL>
+__device__ __forceinline__ void softmax_push(float s, const float (&v)[CPL], float& M, float& L, float (&res)[CPL]) {
+  const float Mn = fmaxf(M, s);
+  const float eo = exp2f(M - Mn), en = exp2f(s - Mn);
+  L = L * eo + en;
+#pragma unroll
+  for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + en * v[k];
+  M = Mn;
+}
+
 // Merge: softmax-merge of the attention partials of one (sequence, KV head) row, add the gated
 // memory readout (Eq. 4), store.
 // grid = (Hkv, n_seq), block = 32 * max(Gq, DH / 32): warp hh merges query head hh of the group
 // (each lane DH/32 output columns), all heads in parallel.
+//
+// Deferred compaction (call.defer): the partials cover the entries cached before the call, i.e. without the
+// new token and with the entries the selection has evicted meanwhile.  The attention over the retained set
+// (Eq. 4) is recovered exactly: the new token's term is added, the evicted entries' terms
+// exp(s_e) (1, v_e) are taken out of the sums again.  Taking out is safe in float32 while the evicted
+// entries hold at most 90 % of the softmax mass (the error of the remainder grows by at most 10); beyond
+// that the warp recomputes its head over the retained entries from the cache, which is still uncompacted.
 template <int DH, typename OutT>
 __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, ImScratch sc, ImCall call, int n_ctas,
-                                                          OutT* __restrict__ out) {
+                                                          OutT* __restrict__ out, const bf16* __restrict__ q,
+                                                          const bf16* __restrict__ k_new, const bf16* __restrict__ v_new) {
   constexpr int CPL = DH / 32;  // columns per lane
   const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
@@ -491,9 +516,9 @@ __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, I
     float res[CPL];
 #pragma unroll
     for (int k = 0; k < CPL; ++k) res[k] = 0.f;
+    float M = NEG_INF, L = 0.f;
     if (nt_i > 0) {
       const long long w0 = row_first / qrun, w1 = row_last / qrun;
-      float M = NEG_INF, L = 0.f;
       for (long long wv = w0; wv <= w1; ++wv) {
         const float* ps = sc.part + ((size_t)(wv + row_id) * p.Gq + hh) * (DH + 2);
         const float mw = ps[DH], lw = ps[DH + 1];
@@ -507,6 +532,84 @@ __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, I
         for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[k] * en;
         M = Mn;
       }
+    }
+    if (call.defer) {
+      const size_t u = (size_t)call.layer * p.S + call.seq[i];
+      const int n_old = max(0, min(st.ctr[u * CTR_STRIDE + CTR_N], p.cap - 1));  // = slot of the new token
+      const int ne = max(0, min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], IM_FRONT_MAX_NE));
+      const int32_t* evs = st.ev_slot + u * p.tail;
+      const float sl2 = p.scale * 1.4426950408889634f;
+      float qv[CPL], vv[CPL];
+      const bf16* qrow = q + ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH;
+#pragma unroll
+      for (int k = 0; k < CPL; ++k) qv[k] = __bfloat162float(qrow[lane + 32 * k]);
+      bool new_kept = true;
+      for (int a = 0; a < ne; ++a) new_kept &= evs[a] != n_old;
+      if (new_kept) {
+        const bf16* kr = k_new + (size_t)i * p.Dkv + h * DH;
+        const bf16* vr = v_new + (size_t)i * p.Dkv + h * DH;
+        float dot = 0.f;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) {
+          dot = fmaf(qv[k], __bfloat162float(kr[lane + 32 * k]), dot);
+          vv[k] = __bfloat162float(vr[lane + 32 * k]);
+        }
+        softmax_push<CPL>(warp_sum_f(dot) * sl2, vv, M, L, res);
+      }
+      float Lsub = 0.f, sub[CPL];
+#pragma unroll
+      for (int k = 0; k < CPL; ++k) sub[k] = 0.f;
+      for (int a = 0; a < ne; ++a) {
+        if (evs[a] >= n_old) continue;  // the new token itself: it was never added
+        const bf16* kr = sc.evK + ((size_t)i * p.tail + a) * p.Dkv + h * DH;
+        const bf16* vr = sc.evV + ((size_t)i * p.tail + a) * p.Dkv + h * DH;
+        float dot = 0.f;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) dot = fmaf(qv[k], __bfloat162float(kr[lane + 32 * k]), dot);
+        const float w = exp2f(warp_sum_f(dot) * sl2 - M);
+        Lsub += w;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) sub[k] = fmaf(w, __bfloat162float(vr[lane + 32 * k]), sub[k]);
+      }
+      if (Lsub <= 0.9f * L) {
+        L -= Lsub;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) res[k] -= sub[k];
+      } else {
+        // the evicted entries dominate this head's softmax: recompute it over the retained entries
+        if (lane == 0) atomicAdd(st.status + 1, 1);
+        M = NEG_INF;
+        L = 0.f;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) res[k] = 0.f;
+        const bf16* Kb = st.Kc + (u * p.Hkv + h) * (size_t)p.cap * DH;
+        const bf16* Vb = st.Vc + (u * p.Hkv + h) * (size_t)p.cap * DH;
+        for (int t = 0; t < n_old; ++t) {
+          bool gone = false;
+          for (int a = 0; a < ne; ++a) gone |= evs[a] == t;
+          if (gone) continue;
+          float dot = 0.f;
+#pragma unroll
+          for (int k = 0; k < CPL; ++k) {
+            dot = fmaf(qv[k], __bfloat162float(Kb[(size_t)t * DH + lane + 32 * k]), dot);
+            vv[k] = __bfloat162float(Vb[(size_t)t * DH + lane + 32 * k]);
+          }
+          softmax_push<CPL>(warp_sum_f(dot) * sl2, vv, M, L, res);
+        }
+        if (new_kept) {
+          const bf16* kr = k_new + (size_t)i * p.Dkv + h * DH;
+          const bf16* vr = v_new + (size_t)i * p.Dkv + h * DH;
+          float dot = 0.f;
+#pragma unroll
+          for (int k = 0; k < CPL; ++k) {
+            dot = fmaf(qv[k], __bfloat162float(kr[lane + 32 * k]), dot);
+            vv[k] = __bfloat162float(vr[lane + 32 * k]);
+          }
+          softmax_push<CPL>(warp_sum_f(dot) * sl2, vv, M, L, res);
+        }
+      }
+    }
+    if (L > 0.f) {
       const float inv = 1.0f / L;
 #pragma unroll
       for (int k = 0; k < CPL; ++k) res[k] *= inv;
@@ -593,16 +696,20 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   return cudaGetLastError();
 }
 
-cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas) {
+cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas, const void* q,
+                                      const void* k_new, const void* v_new) {
+  const bf16* qp = (const bf16*)q;
+  const bf16* kp = (const bf16*)k_new;
+  const bf16* vp = (const bf16*)v_new;
   const ImDims& p = L.p;
   dim3 grid(p.Hkv, call.n_seq);
   const int mthreads = 32 * std::max(p.Gq, p.d / 32);
   if (p.d == 64) {
-    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (float*)out);
-    else k_attn_merge_rows<64, bf16><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (bf16*)out);
+    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (float*)out, qp, kp, vp);
+    else k_attn_merge_rows<64, bf16><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (bf16*)out, qp, kp, vp);
   } else {
-    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (float*)out);
-    else k_attn_merge_rows<128, bf16><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (bf16*)out);
+    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (float*)out, qp, kp, vp);
+    else k_attn_merge_rows<128, bf16><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (bf16*)out, qp, kp, vp);
   }
   ++*L.launches;
   return cudaGetLastError();

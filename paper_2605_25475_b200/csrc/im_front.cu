@@ -12,7 +12,6 @@ constexpr int FRONT_THREADS = 512;
 
 struct FrontShared {
   double kd[64];             // indexer key before normalisation (float64)
-  float q[64 * 64];          // q features [HI][dI] (only HI*dI used)
   float alpha[64];
   float knew[64];            // the new token's cached (rounded) indexer key
   unsigned long long wmin[FRONT_THREADS / 32];
@@ -24,13 +23,14 @@ struct FrontShared {
 };
 
 // grid = n_seq, block = FRONT_THREADS, dynamic smem = keys of the selection (8 bytes per entry) when
-// do_select, else 0.
+// do_select (`key_slots` of them), followed by the q features [HI][dI] (float32).
 template <int DI>  // d_I known at compile time (8, 16) keeps the key and the dot products in registers; 0: generic
-__global__ void __launch_bounds__(FRONT_THREADS)
+__global__ void __maxnreg__(80)
 k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __restrict__ k_new,
-               const bf16* __restrict__ v_new, int do_select) {
+               const bf16* __restrict__ v_new, int do_select, int key_slots) {
   extern __shared__ __align__(16) unsigned long long s_key[];
   __shared__ FrontShared sh;
+  float* s_q = reinterpret_cast<float*>(s_key + key_slots);
   const int i = blockIdx.x, tid = threadIdx.x;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   int32_t* ctr = st.ctr + u * CTR_STRIDE;
@@ -69,7 +69,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   load_batch(0);
   // ---- finish the projections: sum the K-split partials in a fixed order
   for (int k = tid; k < nq; k += FRONT_THREADS) {
-    sh.q[k] = im_raw_sum(p, sc, call, i, r.uq + k);
+    s_q[k] = im_raw_sum(p, sc, call, i, r.uq + k);
   }
   for (int k = tid; k < p.HI; k += FRONT_THREADS) {
     sh.alpha[k] = im_raw_sum(p, sc, call, i, r.g + k) * (1.0f / sqrtf((float)p.HI * (float)p.dI));
@@ -82,7 +82,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   __syncthreads();
   // RMSNorm of the q features per indexer head (float32) and of the key (float64, then bf16)
   for (int h = tid; h < p.HI; h += FRONT_THREADS) {
-    float* y = sh.q + h * p.dI;
+    float* y = s_q + h * p.dI;
     float ms = 0.f;
     for (int k = 0; k < p.dI; ++k) ms = fmaf(y[k], y[k], ms);
     const float inv = 1.0f / sqrtf(ms / (float)p.dI + p.norm_eps);
@@ -142,7 +142,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
       for (int h = 0; h < p.HI; ++h) {
         float z = 0.f;
 #pragma unroll
-        for (int k = 0; k < dI; ++k) z = fmaf(sh.q[h * dI + k], kk[k], z);
+        for (int k = 0; k < dI; ++k) z = fmaf(s_q[h * dI + k], kk[k], z);
         if (p.act == 0) z = fmaxf(z, 0.f);
         A = fmaf(sh.alpha[h], z, A);
       }
@@ -165,7 +165,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   if (!select_here) {
     // either not due, or the selection runs in the kernels that follow (they read imp / pos)
     if (tid == 0) {
-      ctr[CTR_N] = n1;
+      ctr[call.defer ? CTR_NNEXT : CTR_N] = n1;
       ctr[CTR_T] = T + 1;
       ctr[CTR_SINCE] = since + 1;
       ctr[CTR_NEVICT] = 0;
@@ -225,12 +225,16 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
       st.ev_slot[u * p.tail + a] = sh.ev[a];
       st.ev_pos[u * p.tail + a] = sh.evpos[a];
     }
+    if (call.defer) {  // the moves are made by k_move_survivors once the attention kernel has read the cache
+      sc.nhole[i] = sh.nh;
+      for (int a = 0; a < sh.nh; ++a) sc.surv[(size_t)i * p.tail + a] = sh.surv[a];
+    }
   }
   __syncthreads();
   // ---- gather the evicted pairs for the memory write (a3) and, in the same pass, a4: a hole below
   // the budget (the first nh evicted slots) receives the retained entry found above it.  A thread
   // reads the evicted chunk before it overwrites it; the sources of the moves are never written.
-  const int nh = sh.nh;
+  const int nh = call.defer ? 0 : sh.nh;
   for (int k = tid; k < ne * p.Hkv * dv; k += FRONT_THREADS) {
     const int e = k / (p.Hkv * dv), rem = k % (p.Hkv * dv), h = rem / dv, c = rem % dv;
     const size_t base = (u * p.Hkv + h) * p.cap;
@@ -253,7 +257,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   }
   for (int j = tid; j < nh; j += FRONT_THREADS) pos[sh.ev[j]] = (sh.surv[j] == n) ? T : pos[sh.surv[j]];
   if (tid == 0) {
-    ctr[CTR_N] = n1 - ne;
+    ctr[call.defer ? CTR_NNEXT : CTR_N] = n1 - ne;
     ctr[CTR_T] = T + 1;
     ctr[CTR_SINCE] = 0;
     ctr[CTR_NSEL] = n1;
@@ -288,9 +292,12 @@ __global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, Im
   const int i = blockIdx.y;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
+  // deferred compaction: this is the call's last kernel, it publishes the new entry count
+  if (call.defer && blockIdx.x == 0 && threadIdx.x == 0) st.ctr[u * CTR_STRIDE + CTR_N] = st.ctr[u * CTR_STRIDE + CTR_NNEXT];
+  if (ne <= 0) return;
   const int nh = min(sc.nhole[i], ne);
   const int j0 = blockIdx.x * 4;
-  if (ne <= 0 || j0 >= nh) return;
+  if (j0 >= nh) return;
   const int cnt = min(4, nh - j0);
   const int dv = p.d / 8;
   const int32_t* evs = st.ev_slot + u * p.tail;
@@ -314,18 +321,27 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
                                    int do_select, int n_max) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_decode_front<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8);
+    cudaError_t e = cudaFuncSetAttribute(k_decode_front<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  const size_t smem = do_select ? (size_t)n_max * 8 : 0;
+  const int key_slots = do_select ? n_max : 0;
+  const size_t smem = (size_t)key_slots * 8 + (size_t)L.p.HI * L.p.dI * 4;
   const bf16* kn = (const bf16*)k_new;
   const bf16* vn = (const bf16*)v_new;
-  if (L.p.dI == 16) k_decode_front<16><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select);
-  else if (L.p.dI == 8) k_decode_front<8><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select);
-  else k_decode_front<0><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select);
+  if (L.p.dI == 16) k_decode_front<16><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
+  else if (L.p.dI == 8) k_decode_front<8><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
+  else k_decode_front<0><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+// last kernel of a decode call with deferred compaction: fills the holes, advances the entry count
+cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call) {
+  dim3 grid((IM_FRONT_MAX_NE + 3) / 4, call.n_seq);
+  k_move_survivors<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
 }

@@ -19,7 +19,10 @@ typedef __nv_bfloat16 bf16;
 #define IM_TC_TILE_BYTES 25600 /* one tile record: 3 bf16 terms x (256 rows x 32 bytes) + 256 alpha floats */
 
 // per-(layer, sequence) device counters
-enum { CTR_N = 0, CTR_T = 1, CTR_SINCE = 2, CTR_EVSTEPS = 3, CTR_NEVICT = 4, CTR_NPEND = 5, CTR_DIRECT = 6, CTR_NSEL = 7, CTR_STRIDE = 8 };
+enum { CTR_N = 0, CTR_T = 1, CTR_SINCE = 2, CTR_EVSTEPS = 3, CTR_NEVICT = 4, CTR_NPEND = 5, CTR_NNEXT = 6, CTR_NSEL = 7, CTR_STRIDE = 8 };
+
+// CTR_NNEXT: in a decode call with deferred compaction, the entry count the call will leave; CTR_N keeps the
+// count from before the call until the call's last kernel (the attention and merge kernels read it).
 
 // device status bits (sticky)
 enum { ST_NONFINITE = 1, ST_COUNT = 2, ST_TIMEOUT = 4 };
@@ -103,6 +106,9 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
 struct ImCall {
   int layer, n_seq, C;
   int prefill;    // 1: im_prefill_chunk (always compresses), 0: im_decode_step (compresses every tau-th token)
+  int defer;      // decode: 1 = the attention kernel runs over the entries cached before the call while the front
+                  // kernel appends / scores / selects; the merge adds the new token and takes the evicted entries
+                  // out again, and the holes are filled (and CTR_N advanced) by the call's last kernel
   int pack;       // prefill: 1 = the append kernel also writes the operand records of the tensor-core scoring
   int phi_large;  // 1: phi of the evicted keys lives in ImScratch::phi, 0: in the K-split partials phip
   int ksplit, ksplit_key, ksplit_phi;  // K splits of the projections / key projection / phi partials of this call
@@ -174,7 +180,9 @@ cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
                                      const void* q, int n_ctas);
-cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas);
+cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas, const void* q,
+                                      const void* k_new, const void* v_new);
+cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,
                            uint8_t* keep, int32_t* n_evict, cudaStream_t stream);
 cudaError_t im_launch_init_weights(const ImDims& p, const ImWeights& w, int layer, uint64_t seed, float std,

@@ -276,3 +276,47 @@ def test_prefill_scoring_tensor_unsupported_shape_is_refused(im):
         im.im_set_option(p.g.ctx, im.IM_OPT_PREFILL_TENSOR, 1)
     p.prefill(0)
     p.decode(0)
+
+
+# ------------------------------------------------------------------ decode with the attention kernel started before the selection
+def test_peaked_attention_evicted_entry_dominates_softmax(im):
+    """softmax_scale = 6: every head's attention is close to one-hot, so the entry evicted in a step often
+    carries nearly all of a head's softmax mass.  The merge must then recompute the head over the retained
+    entries (removing the term from the sums would cancel catastrophically); the counter shows that it did."""
+    wl = TINY.replace(name="peaked", ctx=64, chunk=64, B=32, steps=60, n_needles=0)
+    p = _pair(wl, scale=6.0)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3
+    assert im.im_event_count(p.g.ctx, im.IM_COUNT_MERGE_RECOMPUTE) > 0
+
+
+@pytest.mark.parametrize("conc", [0, 1])
+def test_decode_schedules_agree_with_the_oracle(im, conc):
+    """The in-order schedule and the concurrent one (attention first, evicted terms removed in the merge)
+    against the oracle on the same inputs: several sequences, evictions every step, needles, then steps on a
+    cache that is not full yet (nothing evicted, the new token only added)."""
+    wl = synth.CONFIGS["llama8b_b1"].replace(name="sched", n_seq=3, ctx=333, chunk=333, B=300, steps=12, n_needles=4)
+    p = _pair(wl)
+    im.im_set_option(p.g.ctx, im.IM_OPT_CONCURRENCY, conc)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
+    wl2 = wl.replace(name="sched_notfull", ctx=40, chunk=40, B=64, steps=30)   # fills up at step 24
+    p2 = _pair(wl2)
+    im.im_set_option(p2.g.ctx, im.IM_OPT_CONCURRENCY, conc)
+    p2.prefill(0)
+    for s in range(wl2.steps):
+        p2.decode(s)
+    assert p2.stats["max_out_err"] <= 2e-3
+
+
+def test_decode_from_an_empty_cache(im):
+    """No prefill at all: the first decode step attends to the new token alone."""
+    wl = TINY.replace(name="empty_start", ctx=0, chunk=8, B=16, steps=24, n_needles=0)
+    p = _pair(wl)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3
