@@ -196,6 +196,7 @@ def run_ours(args, rank, world, device):
             sampler.start()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
+        rec0 = im.im_event_count(g.ctx, im.IM_COUNT_MERGE_RECOMPUTE)
         ev0.record(stream)
         for s in range(args.steps):
             load(args.warmup + 2 + s)
@@ -204,6 +205,7 @@ def run_ours(args, rank, world, device):
         torch.cuda.synchronize()
         barrier(world)
         ms = ev0.elapsed_time(ev1)
+        recomputes = im.im_event_count(g.ctx, im.IM_COUNT_MERGE_RECOMPUTE) - rec0
         clocks = sampler.stop() if rank == 0 else None
         assert g.status() == 0
         ms = max_over_ranks(ms, world, device)
@@ -242,6 +244,7 @@ def run_ours(args, rank, world, device):
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "traffic": args.traffic if wl.name == "llama8b_stack" else None, "bytes_per_launch": ab["attn_launch"],
                      "us_per_launch": attn_launch_s * 1e6},
+        "merge_recomputes_per_step": recomputes / args.steps,
         "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
     }
     return res, wl

@@ -146,7 +146,9 @@ void carve(const ImDims& p, char* base, Layout* lo) {
     const size_t stream = ((size_t)IM_ATTN_MAX_CTAS * IM_ATTN_WARPS + (size_t)p.S * p.Hkv) * p.Gq * (p.d + 2);
     lo->sc.part = (float*)take(std::max(generic, stream) * 4);
   }
-  lo->sc.mres = (float*)take((size_t)p.S * (p.Dkv + 1) * 4);
+  lo->sc.mres = (float*)take((size_t)p.S * (p.Dkv + 2) * 4);
+  lo->sc.phiq = (float*)take((size_t)p.S * p.dM * 4);
+  lo->sc.n_att = (int32_t*)take((size_t)p.S * 4);
   lo->sc.rpart = (float*)take((size_t)p.S * ((p.dM + IM_READOUT_ROWS - 1) / IM_READOUT_ROWS) * p.Dkv * 4);
   lo->sc.qpack = nullptr;
   if (im_score_tc_supported(p))
@@ -176,7 +178,7 @@ struct im_ctx {
   // Independent pieces of one decode call run on three side streams that fork from and join back into
   // the caller's stream (plain event dependencies, so the pattern can be captured into a CUDA graph).
   cudaStream_t side[3] = {nullptr, nullptr, nullptr};
-  cudaEvent_t ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t ev[10] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   bool concurrent = false;
   bool prefetch_next = true;         // warm L2 with the next layer's weights / index state during attention
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
@@ -243,7 +245,8 @@ void mirror_memory(const ImDims& p, HostUnit& u, int ne) {
 }
 
 // phi of the gathered evicted keys (skinny GEMM against the folded Linear_theta), then Eq. 6-7.
-int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max) {
+// With `update` = false only the GEMM is launched (the caller launches im_launch_mem_update later).
+int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, bool update = true) {
   const ImDims& p = ctx->p;
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
@@ -270,9 +273,10 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max) {
     g.ksplit = call.ksplit_phi;
     g.ks_stride = (long long)call.n_seq * p.F * p.dM;
     g.kc = 64;  // 18 KB of shared memory: fits next to the resident attention blocks
+    g.direct = call.prefill ? 0 : 1;
   }
   CKL(im_launch_gemm(L, g));
-  CKL(im_launch_mem_update(L, call, ne_max));
+  if (update) CKL(im_launch_mem_update(L, call, ne_max));
   return IM_OK;
 }
 
@@ -341,12 +345,12 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     for (int k = 0; k < 3 && e == cudaSuccess; ++k)
       e = cudaStreamCreateWithPriority(&ctx->side[k], cudaStreamNonBlocking, prio_hi);
   }
-  for (int k = 0; k < 8 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
+  for (int k = 0; k < 10 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     for (int k = 0; k < 3; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
-    for (int k = 0; k < 8; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+    for (int k = 0; k < 10; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
     delete ctx;
     return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
   }
@@ -358,7 +362,7 @@ int im_destroy(im_ctx* ctx) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   cudaError_t e = cudaDeviceSynchronize();
   for (int k = 0; k < 3; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
-  for (int k = 0; k < 8; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+  for (int k = 0; k < 10; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   delete ctx;
   if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
   return IM_OK;
@@ -503,12 +507,16 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   //  (A) deferred compaction - the streaming attention kernel is available and the selection, if one is
   //      due, fits the fused front kernel: attention needs nothing of this call but q, so it starts at
   //      once over the entries cached before the call.  The merge adds the new token, removes the evicted
-  //      entries again (exactly, see k_attn_merge_rows), and the holes are filled afterwards.
-  //        s0: attention ------------------------------------------------> merge -> fill holes, publish count
+  //      entries again (exactly, see k_attn_merge_rows), adds the terms of this call's memory write to the
+  //      readout, and fills the holes.
+  //        s0: attention ----------------------------------------------------------> merge
   //        s1: indexer projections -> front (append, score, select, gather) -> phi of the evicted keys ->
-  //            memory write -> readout finish
-  //        s2: fold of the pending list -> phi(q) / gate projections -> readout partials -> L2 prefetch
-  //        s3: float64 key projection (needed by front)
+  //            readout over the memory after the write (k_readout_apply)
+  //            [-> memory write: not needed by the merge, it only has to end with the call]
+  //        s2: phi(q) / gate projections -> readout partials -> readout over the memory as it is before
+  //            the write
+  //        s3: fold of the pending list -> float64 key projection (needed by front) -> L2 prefetch for the
+  //            next layer
   //      With IM_OPT_CONCURRENCY off the same kernels run on s0 in an order that respects these arrows.
   //  (B) in order on s0, attention after the compaction: everything else (large evicted sets, budgets
   //      beyond the fused front kernel, head shapes without the streaming attention kernel).
@@ -529,17 +537,29 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CK(cudaStreamWaitEvent(L3.stream, ctx->ev[0], 0));
   }
   const bool prof = ctx->prof_target == 0 && ctx->prof_used + 2 <= ctx->prof_ev.size();
-  if (defer && conc) {  // a5 first: it overlaps with everything below
+  if (conc) {  // a5 first: it overlaps with everything below
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
     CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
   }
   const bool mem_write = due && ne_max > 0 && p.mem;
+  // s3: fold (reads the counters of before the call; the readout reads the folded state), key projection
   if (mem_write) {
-    CKL(im_launch_mem_fold(L2, call));
-    if (conc) CK(cudaEventRecord(ctx->ev[7], L2.stream));  // fold done: it read the counters of before the call
+    CKL(im_launch_mem_fold(L3, call));
+    if (conc) CK(cudaEventRecord(ctx->ev[7], L3.stream));
   }
-  // a0: projections as K-split partial sums: indexer part (Sec. 3.1 features) ...
+  CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
+  if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // fold and key projection done
+  if (ctx->prefetch_next && ctx->fast_attn) {
+    // warm L2 for the next layer's small kernels while this layer's attention streams K/V
+    ImLaunch Lp = L3;
+    ImCall nxt = call;
+    nxt.layer = (layer + 1) % p.L;
+    Lp.w = ctx->lo.w[nxt.layer];
+    CKL(im_launch_prefetch_layer(Lp, nxt));
+  }
+  if (conc) CK(cudaEventRecord(ctx->ev[8], L3.stream));  // s3 finished
+  // a0: projections as K-split partial sums: indexer part (Sec. 3.1 features) on s1 ...
   ImRows r = im_rows(p);
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
@@ -555,13 +575,12 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   g.K = p.D;
   g.ksplit = call.ksplit;
   g.kc = conc ? 64 : 0;  // next to the attention CTAs only a small staging buffer fits into an SM's shared memory
+  g.direct = 1;          // (used only where the direct variant cannot be: K splits that are not multiples of 32)
   g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
   g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
   g.n_jobs = 2;
   CKL(im_launch_gemm(L1, g));
-  CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
-  if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // key projection done
-  // ... memory part (phi(q) of Eq. 5, gate logit of Eq. 4), followed by the readout partials
+  // ... memory part (phi(q) of Eq. 5, gate logit of Eq. 4) on s2, followed by the readout
   if (p.mem) {
     g.job[0] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
     g.job[1] = {L.w.wg, nullptr, 1, r.wg, 2};
@@ -569,20 +588,12 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   }
   // an evicted set larger than the pending list is accumulated into Mhat itself, which the readout reads
   const bool readout_early = !(mem_write && ne_max > p.F);
+  if (conc && mem_write) CK(cudaStreamWaitEvent(L2.stream, ctx->ev[7], 0));
   if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call));
-  if (conc && p.mem) CK(cudaEventRecord(ctx->ev[6], L2.stream));  // readout partials done
-  if (ctx->prefetch_next && ctx->fast_attn) {
-    // warm L2 for the next layer's small kernels while this layer's attention streams K/V
-    ImLaunch Lp = L2;
-    ImCall nxt = call;
-    nxt.layer = (layer + 1) % p.L;
-    Lp.w = ctx->lo.w[nxt.layer];
-    CKL(im_launch_prefetch_layer(Lp, nxt));
-  }
+  if (defer && p.mem) CKL(im_launch_readout_finish(L2, call));  // over the memory as it is before this call's write
   if (conc) {
     CK(cudaEventRecord(ctx->ev[4], L2.stream));  // s2 finished
-    CK(cudaStreamWaitEvent(L1.stream, ctx->ev[2], 0));
-    if (mem_write) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0));  // the front kernel changes the counters
+    CK(cudaStreamWaitEvent(L1.stream, ctx->ev[2], 0));  // the front kernel changes the counters the fold reads
   }
   // append + a1 (+ a2 and the gather of the evicted pairs when the evicted set is small enough for one
   // block per sequence; a4 in the same kernel unless the compaction is deferred)
@@ -591,11 +602,15 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CKL(im_launch_select(L1, call));
     if (ne_max > 0) CKL(im_launch_gather_move(L1, call, ne_max));
   }
-  // a3: memory write (needs the gathered evicted pairs and the fold)
-  if (mem_write) {
-    if ((rc = run_memory_write(ctx, L1, call, ne_max))) return rc;
-    if (ctx->fast_attn && !readout_early) CKL(im_launch_readout(L1, call));
-  }
+  // a3: memory write (needs the gathered evicted pairs and the fold).  With deferred compaction the readout
+  // of the state after the write is formed from phi of the evicted keys (k_readout_apply), and the state
+  // update itself follows off the critical path, after the readout that wants the state from before it.
+  if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, !defer))) return rc;
+  if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[4], 0));  // s2 joins here
+  if (defer && p.mem) CKL(im_launch_readout_apply(L1, call));
+  if (conc) CK(cudaEventRecord(ctx->ev[3], L1.stream));  // everything the merge needs from s1
+  if (defer && mem_write) CKL(im_launch_mem_update(L1, call, ne_max));
+  if (mem_write && ctx->fast_attn && !readout_early) CKL(im_launch_readout(L1, call));
   int n_att = 0;
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
@@ -606,24 +621,23 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     u.since = due ? 0 : u.since + 1;
     n_att = std::max(n_att, u.n);
   }
-  // a5: attention; a6: readout finish (Eq. 5), merge, gate, fuse (Eq. 4)
+  // a5: attention; a6: merge, gate, fuse (Eq. 4)
   if (ctx->fast_attn) {
-    if (!(defer && conc)) {
+    if (!conc) {
       if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
       CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
       if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
     }
-    if (p.mem) {
-      if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[6], 0));
-      CKL(im_launch_readout_finish(L1, call));
-    }
-    if (conc) {  // every side stream joins the caller's stream (s3 joined s1 through the key projection event)
-      CK(cudaEventRecord(ctx->ev[5], L1.stream));
-      CK(cudaStreamWaitEvent(s0, ctx->ev[5], 0));
-      CK(cudaStreamWaitEvent(s0, ctx->ev[4], 0));
+    if (!defer && p.mem) CKL(im_launch_readout_finish(L, call));  // after the memory write
+    if (conc) {
+      CK(cudaStreamWaitEvent(s0, ctx->ev[3], 0));  // s1 (which waited for s2)
+      CK(cudaStreamWaitEvent(s0, ctx->ev[8], 0));  // s3
     }
     CKL(im_launch_attention_merge(L, call, out, ctx->n_ctas, q, k_new, v_new));
-    if (defer) CKL(im_launch_decode_commit(L, call));
+    if (conc) {  // the memory write only has to end with the call
+      CK(cudaEventRecord(ctx->ev[5], L1.stream));
+      CK(cudaStreamWaitEvent(s0, ctx->ev[5], 0));
+    }
   } else {
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
     CKL(im_launch_attention(L, call, q, out, n_att));

@@ -130,6 +130,7 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   for (int i = threadIdx.x; i < call.n_seq; i += blockDim.x) {
     const size_t u = (size_t)call.layer * p.S + call.seq[i];
     s_n[i] = max(0, min(st.ctr[u * CTR_STRIDE + CTR_N], p.cap));
+    if (blockIdx.x == 0) sc.n_att[i] = s_n[i];  // what the merge kernel rebuilds the tile bookkeeping from
   }
   if (lane == 0) {
     for (int s = 0; s < STAGES; ++s) mbar_init(smem_u32(&bars[warp * STAGES + s]), 1);
@@ -202,7 +203,6 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   long long j = run0;
   while (j < run1 && ok) {
     // ---- one (sequence, KV head) segment of the run
-    const size_t u = (size_t)call.layer * p.S + call.seq[i];
     const int n = s_n[i];
     const long long row_id = (long long)i * p.Hkv + h;
     // Q^T as B fragments: head g of the group (zero for the padding heads)
@@ -385,8 +385,10 @@ __global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch
 // Readout, second half (Eq. 5 and the gate of Eq. 4), once per sequence:
 //   mres[i][col] = cscale * ( sum_chunks rpart[col] + sum_p w_p (phi_q . phi_p) v_p[col] ) / ( sum_m phi_q[m]^2 b[m] + eps )
 //   mres[i][Dkv] = g(q)
-// Runs after the memory write of the call (it reads the pending list, b and cscale) and the readout
-// partials, off the critical path of the attention kernel.  grid = n_seq, block = 256, smem = dM floats.
+// Without deferred compaction it runs after the memory write of the call (it reads the pending list, b and
+// cscale).  With it (call.defer) it runs BEFORE the write and leaves numerator cscale * (...) and the
+// denominator sum apart; the merge kernel adds the terms of the entries written in this call, so that the
+// readout does not wait for the selection.  grid = n_seq, block = 256, smem = dM floats.
 __global__ void __launch_bounds__(256) k_readout_finish(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call) {
   extern __shared__ float phiq[];  // [dM] phi(q), summed over the K-split partials
   __shared__ float s_dot[64];
@@ -426,9 +428,11 @@ __global__ void __launch_bounds__(256) k_readout_finish(ImDims p, ImState st, Im
   __syncthreads();
   float den = p.eps;
   for (int k = 0; k < 8; ++k) den += s_red[k];
-  const float scale = st.cscale[u] / den;
+  // deferred compaction: numerator and denominator sum over the state from before the call's memory write
+  const float scale = call.defer ? st.cscale[u] : st.cscale[u] / den;
   const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
-  float* dst = sc.mres + (size_t)i * (p.Dkv + 1);
+  float* dst = sc.mres + (size_t)i * (p.Dkv + 2);
+  for (int m = tid; m < p.dM; m += 256) sc.phiq[(size_t)i * p.dM + m] = phiq[m];
   for (int col = tid; col < p.Dkv; col += 256) {
     const float* rp = sc.rpart + (size_t)i * nchunk * p.Dkv + col;
     float mv = 0.f;
@@ -436,7 +440,59 @@ __global__ void __launch_bounds__(256) k_readout_finish(ImDims p, ImState st, Im
     for (int pp = 0; pp < np; ++pp) mv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mv);
     dst[col] = scale * mv;
   }
-  if (tid == 0) dst[p.Dkv] = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
+  if (tid == 0) {
+    dst[p.Dkv] = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
+    dst[p.Dkv + 1] = den - p.eps;
+  }
+}
+
+// Deferred compaction, between the readout over the memory of before the call (k_readout_finish) and the
+// merge: Eq. 5 over the memory after this call's write (Eq. 6-7), M' = lambda M + eta sum_e phi_e v_e^T,
+// b' = lambda b + eta sum_e phi_e^2 (applied only if something was evicted):
+//   m[col] = (decay P[col] + eta sum_e (phi_q . phi_e) v_e[col]) / (eps + decay D + eta sum_e sum_m phi_q[m]^2 phi_e[m]^2)
+// in place over P.  Needs phi of the evicted keys (K-split partials) but not the state update itself.
+// grid = n_seq, block = 256.
+__global__ void __launch_bounds__(256) k_readout_apply(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  __shared__ float s_dot[IM_FRONT_MAX_NE][8], s_sq[IM_FRONT_MAX_NE][8];
+  const int i = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int ne = max(0, min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], min(IM_FRONT_MAX_NE, p.F)));
+  float* mr = sc.mres + (size_t)i * (p.Dkv + 2);
+  const float D = mr[p.Dkv + 1];
+  const float* pq = sc.phiq + (size_t)i * p.dM;
+  for (int e = 0; e < ne; ++e) {
+    float dot = 0.f, sq = 0.f;
+    for (int m = tid; m < p.dM; m += 256) {
+      float f = 0.f;
+      for (int ks = 0; ks < call.ksplit_phi; ++ks) f += sc.phip[(((size_t)ks * call.n_seq + i) * p.F + e) * p.dM + m];
+      const float qf = pq[m];
+      dot = fmaf(qf, f, dot);
+      sq = fmaf(qf * qf, f * f, sq);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    }
+    if (lane == 0) { s_dot[e][warp] = dot; s_sq[e][warp] = sq; }
+  }
+  __syncthreads();
+  const float decay = ne > 0 ? p.lambda : 1.0f;
+  float den = p.eps + decay * D;
+  for (int e = 0; e < ne; ++e) {
+    float sq = 0.f;
+    for (int w = 0; w < 8; ++w) sq += s_sq[e][w];
+    den = fmaf(p.eta, sq, den);
+  }
+  for (int col = tid; col < p.Dkv; col += 256) {
+    float num = decay * mr[col];
+    for (int e = 0; e < ne; ++e) {
+      float dot = 0.f;
+      for (int w = 0; w < 8; ++w) dot += s_dot[e][w];
+      num = fmaf(p.eta * dot, __bfloat162float(sc.evV[((size_t)i * p.tail + e) * p.Dkv + col]), num);
+    }
+    mr[col] = num / den;
+  }
 }
 
 __device__ __forceinline__ float warp_sum_f(float v) {
@@ -472,18 +528,48 @@ __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, I
                                                           OutT* __restrict__ out, const bf16* __restrict__ q,
                                                           const bf16* __restrict__ k_new, const bf16* __restrict__ v_new) {
   constexpr int CPL = DH / 32;  // columns per lane
+  __shared__ int s_ev[IM_FRONT_MAX_NE], s_sv[IM_FRONT_MAX_NE];
   const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int hh0 = min(warp, p.Gq - 1);  // the head this warp merges first (usually its only one)
+  // ---- every load whose address depends on no other load is issued here, ahead of its use: this kernel is
+  // on the critical path of the call and a dependent chain of loads costs a memory round trip per link
+  const int na_lane = lane < call.n_seq ? sc.n_att[lane] : 0;
+  const int ne_raw = st.ctr[u * CTR_STRIDE + CTR_NEVICT];
+  const int nh_raw = sc.nhole[i];
+  const int n_next = st.ctr[u * CTR_STRIDE + CTR_NNEXT];
+  const int ev_l = lane < IM_FRONT_MAX_NE ? st.ev_slot[u * p.tail + min(lane, p.tail - 1)] : -1;
+  const int sv_l = lane < IM_FRONT_MAX_NE ? sc.surv[(size_t)i * p.tail + min(lane, p.tail - 1)] : -1;
+  const float* mr = sc.mres + (size_t)i * (p.Dkv + 2);
+  float gate = 0.f, mcol[CPL], qv[CPL], kn[CPL], vn[CPL], ek0[CPL], ev0[CPL];
+  {
+    const bf16* qrow = q + ((size_t)i * p.H + (size_t)h * p.Gq + hh0) * DH;
+    const bf16* kr = k_new + (size_t)i * p.Dkv + h * DH;
+    const bf16* vr = v_new + (size_t)i * p.Dkv + h * DH;
+    const bf16* ekr = sc.evK + (size_t)i * p.tail * p.Dkv + h * DH;
+    const bf16* evr = sc.evV + (size_t)i * p.tail * p.Dkv + h * DH;
+    if (p.mem) gate = mr[p.Dkv];
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) {
+      const int c = lane + 32 * k;
+      mcol[k] = p.mem ? mr[h * DH + c] : 0.f;
+      qv[k] = __bfloat162float(qrow[c]);
+      kn[k] = __bfloat162float(kr[c]);
+      vn[k] = __bfloat162float(vr[c]);
+      ek0[k] = call.defer ? __bfloat162float(ekr[c]) : 0.f;
+      ev0[k] = call.defer ? __bfloat162float(evr[c]) : 0.f;
+    }
+  }
   // ---- rebuild the tile bookkeeping of the attention kernel (lanes stride over the sequences)
   long long pref = 0, total = 0;
-  int nt_i = 0;
+  int nt_i = 0, n_old = 0;
   for (int k0 = 0; k0 < call.n_seq; k0 += 32) {
     const int k = k0 + lane;
-    int nk = 0;
-    if (k < call.n_seq) {
-      const size_t uk = (size_t)call.layer * p.S + call.seq[k];
-      nk = tiles_of(max(0, min(st.ctr[uk * CTR_STRIDE + CTR_N], p.cap)));
-    }
+    int na = 0;
+    if (k0 == 0) na = na_lane;
+    else if (k < call.n_seq) na = sc.n_att[k];
+    const int nk = tiles_of(na);
     // inclusive prefix over the 32 lanes
     long long incl = (long long)nk * p.Hkv;
 #pragma unroll
@@ -494,120 +580,134 @@ __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, I
     if (i >= k0 && i < k0 + 32) {
       pref = total + __shfl_sync(0xffffffffu, incl, i - k0) - (long long)__shfl_sync(0xffffffffu, nk, i - k0) * p.Hkv;
       nt_i = __shfl_sync(0xffffffffu, nk, i - k0);
+      n_old = __shfl_sync(0xffffffffu, na, i - k0);
     }
     total += __shfl_sync(0xffffffffu, incl, 31);
   }
+  n_old = max(0, min(n_old, p.cap - 1));  // with deferred compaction: the slot of the new token
   const long long WT = (long long)n_ctas * WARPS;
   const long long qrun = (total + WT - 1) / WT;
   const long long row_first = pref + (long long)h * nt_i, row_last = row_first + nt_i - 1;
   const long long row_id = (long long)i * p.Hkv + h;
-  // gated readout of this KV head's columns (computed by k_readout_finish)
-  float gm[CPL];
-#pragma unroll
-  for (int k = 0; k < CPL; ++k) gm[k] = 0.f;
-  if (p.mem) {
-    const float* mr = sc.mres + (size_t)i * (p.Dkv + 1);
-    const float gate = mr[p.Dkv];
-#pragma unroll
-    for (int k = 0; k < CPL; ++k) gm[k] = gate * mr[h * DH + lane + 32 * k];
-  }
+  const int ne = call.defer ? max(0, min(ne_raw, IM_FRONT_MAX_NE)) : 0;
+  if (warp == 0 && lane < IM_FRONT_MAX_NE) { s_ev[lane] = ev_l; s_sv[lane] = sv_l; }
+  const float sl2 = p.scale * 1.4426950408889634f;
   // ---- one warp per query head of the group
   for (int hh = warp; hh < p.Gq; hh += nwarps) {
     float res[CPL];
 #pragma unroll
     for (int k = 0; k < CPL; ++k) res[k] = 0.f;
     float M = NEG_INF, L = 0.f;
-    if (nt_i > 0) {
-      const long long w0 = row_first / qrun, w1 = row_last / qrun;
-      for (long long wv = w0; wv <= w1; ++wv) {
-        const float* ps = sc.part + ((size_t)(wv + row_id) * p.Gq + hh) * (DH + 2);
-        const float mw = ps[DH], lw = ps[DH + 1];
-        float a[CPL];
-#pragma unroll
-        for (int k = 0; k < CPL; ++k) a[k] = ps[lane + 32 * k];
-        const float Mn = fmaxf(M, mw);
-        const float eo = exp2f(M - Mn), en = exp2f(mw - Mn);  // exp2(-inf) = 0 for the first contributor
-        L = L * eo + lw * en;
-#pragma unroll
-        for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[k] * en;
-        M = Mn;
-      }
-    }
-    if (call.defer) {
-      const size_t u = (size_t)call.layer * p.S + call.seq[i];
-      const int n_old = max(0, min(st.ctr[u * CTR_STRIDE + CTR_N], p.cap - 1));  // = slot of the new token
-      const int ne = max(0, min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], IM_FRONT_MAX_NE));
-      const int32_t* evs = st.ev_slot + u * p.tail;
-      const float sl2 = p.scale * 1.4426950408889634f;
-      float qv[CPL], vv[CPL];
+    if (call.defer && hh != hh0) {  // a warp with a second head (blocks with fewer warps than heads): its query row
       const bf16* qrow = q + ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH;
 #pragma unroll
       for (int k = 0; k < CPL; ++k) qv[k] = __bfloat162float(qrow[lane + 32 * k]);
+    }
+    const bf16* Kb = st.Kc + (u * p.Hkv + h) * (size_t)p.cap * DH;
+    const bf16* Vb = st.Vc + (u * p.Hkv + h) * (size_t)p.cap * DH;
+    // Pass 0 merges the stored partials; with deferred compaction it then takes the evicted entries' terms
+    // out of the sums.  If those hold more than 90 % of the mass, pass 1 starts over and recomputes, from the
+    // cache, the partials whose key range holds an evicted entry (without it); the others are exact already.
+    for (int pass = 0; pass < 2; ++pass) {
+      M = NEG_INF;
+      L = 0.f;
+#pragma unroll
+      for (int k = 0; k < CPL; ++k) res[k] = 0.f;
+      if (nt_i > 0) {
+        const long long w0 = row_first / qrun, w1 = row_last / qrun;
+        for (long long wv = w0; wv <= w1; ++wv) {
+          // keys of this partial: the tiles of the row that fall into run wv
+          const int lt0 = (int)(max(wv * qrun, row_first) - row_first);
+          const int lt1 = (int)(min((wv + 1) * qrun - 1, row_last) - row_first);
+          const int key0 = lt0 * TILE, key1 = min((lt1 + 1) * TILE, n_old);
+          bool dirty = false;
+          if (pass == 1)
+            for (int a = 0; a < ne; ++a) {
+              const int sl = __shfl_sync(0xffffffffu, ev_l, a);
+              dirty |= sl >= key0 && sl < key1;
+            }
+          if (!dirty) {
+            const float* ps = sc.part + ((size_t)(wv + row_id) * p.Gq + hh) * (DH + 2);
+            const float mw = ps[DH], lw = ps[DH + 1];
+            float a[CPL];
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) a[k] = ps[lane + 32 * k];
+            const float Mn = fmaxf(M, mw);
+            const float eo = exp2f(M - Mn), en = exp2f(mw - Mn);  // exp2(-inf) = 0 for the first contributor
+            L = L * eo + lw * en;
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[k] * en;
+            M = Mn;
+          } else {
+            // four keys per round so that their loads overlap; an evicted key gets the score -inf
+            for (int t0 = key0; t0 < key1; t0 += 4) {
+              float kk[4][CPL], vk[4][CPL], sc4[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int t = min(t0 + j, key1 - 1);
+#pragma unroll
+                for (int k = 0; k < CPL; ++k) {
+                  kk[j][k] = __bfloat162float(Kb[(size_t)t * DH + lane + 32 * k]);
+                  vk[j][k] = __bfloat162float(Vb[(size_t)t * DH + lane + 32 * k]);
+                }
+              }
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                float dot = 0.f;
+#pragma unroll
+                for (int k = 0; k < CPL; ++k) dot = fmaf(qv[k], kk[j][k], dot);
+                sc4[j] = warp_sum_f(dot) * sl2;
+                bool gone = t0 + j >= key1;
+                for (int a = 0; a < ne; ++a) gone |= __shfl_sync(0xffffffffu, ev_l, a) == t0 + j;
+                if (gone) sc4[j] = NEG_INF;
+              }
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                if (sc4[j] > NEG_INF) softmax_push<CPL>(sc4[j], vk[j], M, L, res);
+            }
+          }
+        }
+      }
+      if (!call.defer) break;
       bool new_kept = true;
-      for (int a = 0; a < ne; ++a) new_kept &= evs[a] != n_old;
+      for (int a = 0; a < ne; ++a) new_kept &= __shfl_sync(0xffffffffu, ev_l, a) != n_old;
       if (new_kept) {
-        const bf16* kr = k_new + (size_t)i * p.Dkv + h * DH;
-        const bf16* vr = v_new + (size_t)i * p.Dkv + h * DH;
         float dot = 0.f;
 #pragma unroll
-        for (int k = 0; k < CPL; ++k) {
-          dot = fmaf(qv[k], __bfloat162float(kr[lane + 32 * k]), dot);
-          vv[k] = __bfloat162float(vr[lane + 32 * k]);
-        }
-        softmax_push<CPL>(warp_sum_f(dot) * sl2, vv, M, L, res);
+        for (int k = 0; k < CPL; ++k) dot = fmaf(qv[k], kn[k], dot);
+        softmax_push<CPL>(warp_sum_f(dot) * sl2, vn, M, L, res);
       }
+      if (pass == 1) break;
       float Lsub = 0.f, sub[CPL];
 #pragma unroll
       for (int k = 0; k < CPL; ++k) sub[k] = 0.f;
       for (int a = 0; a < ne; ++a) {
-        if (evs[a] >= n_old) continue;  // the new token itself: it was never added
-        const bf16* kr = sc.evK + ((size_t)i * p.tail + a) * p.Dkv + h * DH;
-        const bf16* vr = sc.evV + ((size_t)i * p.tail + a) * p.Dkv + h * DH;
+        if (__shfl_sync(0xffffffffu, ev_l, a) >= n_old) continue;  // the new token itself: it was never added
+        float ke[CPL], ve[CPL];
+        if (a == 0) {
+#pragma unroll
+          for (int k = 0; k < CPL; ++k) { ke[k] = ek0[k]; ve[k] = ev0[k]; }
+        } else {
+          const bf16* kr = sc.evK + ((size_t)i * p.tail + a) * p.Dkv + h * DH;
+          const bf16* vr = sc.evV + ((size_t)i * p.tail + a) * p.Dkv + h * DH;
+#pragma unroll
+          for (int k = 0; k < CPL; ++k) { ke[k] = __bfloat162float(kr[lane + 32 * k]); ve[k] = __bfloat162float(vr[lane + 32 * k]); }
+        }
         float dot = 0.f;
 #pragma unroll
-        for (int k = 0; k < CPL; ++k) dot = fmaf(qv[k], __bfloat162float(kr[lane + 32 * k]), dot);
+        for (int k = 0; k < CPL; ++k) dot = fmaf(qv[k], ke[k], dot);
         const float w = exp2f(warp_sum_f(dot) * sl2 - M);
         Lsub += w;
 #pragma unroll
-        for (int k = 0; k < CPL; ++k) sub[k] = fmaf(w, __bfloat162float(vr[lane + 32 * k]), sub[k]);
+        for (int k = 0; k < CPL; ++k) sub[k] = fmaf(w, ve[k], sub[k]);
       }
       if (Lsub <= 0.9f * L) {
         L -= Lsub;
 #pragma unroll
         for (int k = 0; k < CPL; ++k) res[k] -= sub[k];
-      } else {
-        // the evicted entries dominate this head's softmax: recompute it over the retained entries
-        if (lane == 0) atomicAdd(st.status + 1, 1);
-        M = NEG_INF;
-        L = 0.f;
-#pragma unroll
-        for (int k = 0; k < CPL; ++k) res[k] = 0.f;
-        const bf16* Kb = st.Kc + (u * p.Hkv + h) * (size_t)p.cap * DH;
-        const bf16* Vb = st.Vc + (u * p.Hkv + h) * (size_t)p.cap * DH;
-        for (int t = 0; t < n_old; ++t) {
-          bool gone = false;
-          for (int a = 0; a < ne; ++a) gone |= evs[a] == t;
-          if (gone) continue;
-          float dot = 0.f;
-#pragma unroll
-          for (int k = 0; k < CPL; ++k) {
-            dot = fmaf(qv[k], __bfloat162float(Kb[(size_t)t * DH + lane + 32 * k]), dot);
-            vv[k] = __bfloat162float(Vb[(size_t)t * DH + lane + 32 * k]);
-          }
-          softmax_push<CPL>(warp_sum_f(dot) * sl2, vv, M, L, res);
-        }
-        if (new_kept) {
-          const bf16* kr = k_new + (size_t)i * p.Dkv + h * DH;
-          const bf16* vr = v_new + (size_t)i * p.Dkv + h * DH;
-          float dot = 0.f;
-#pragma unroll
-          for (int k = 0; k < CPL; ++k) {
-            dot = fmaf(qv[k], __bfloat162float(kr[lane + 32 * k]), dot);
-            vv[k] = __bfloat162float(vr[lane + 32 * k]);
-          }
-          softmax_push<CPL>(warp_sum_f(dot) * sl2, vv, M, L, res);
-        }
+        break;
       }
+      if (lane == 0) atomicAdd(st.status + 1, 1);  // the evicted entries dominate this head's softmax
     }
     if (L > 0.f) {
       const float inv = 1.0f / L;
@@ -617,9 +717,33 @@ __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, I
     const size_t base = ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH;
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
-      const float v = res[k] + gm[k];
+      const float v = res[k] + gate * mcol[k];  // Eq. 4: attention over the retained set + gated memory readout
       if constexpr (sizeof(OutT) == 2) out[base + lane + 32 * k] = __float2bfloat16_rn(v);
       else out[base + lane + 32 * k] = v;
+    }
+  }
+  if (call.defer) {
+    // a4, deferred: the attention kernel has read the cache and every warp of this block is done with the
+    // rows of this KV head, so the holes below the budget can take the retained entries found above it
+    // (block h moves the K / V rows of its head; block 0 also the indexer keys and positions, and publishes
+    // the entry count, which no other block of this kernel reads)
+    __syncthreads();
+    const int nh = min(max(nh_raw, 0), ne);
+    constexpr int CH = DH / 8;  // 16-byte chunks per row
+    const size_t base = (u * p.Hkv + h) * (size_t)p.cap;
+    for (int k = tid; k < nh * CH; k += blockDim.x) {
+      const int j = k / CH, c = k % CH;
+      const int dst = s_ev[j], src = s_sv[j];
+      reinterpret_cast<uint4*>(st.Kc + (base + dst) * DH)[c] = reinterpret_cast<const uint4*>(st.Kc + (base + src) * DH)[c];
+      reinterpret_cast<uint4*>(st.Vc + (base + dst) * DH)[c] = reinterpret_cast<const uint4*>(st.Vc + (base + src) * DH)[c];
+    }
+    if (h == 0) {
+      for (int k = tid; k < nh * p.dI; k += blockDim.x) {
+        const int j = k / p.dI, c = k % p.dI;
+        st.kidx[(u * p.cap + s_ev[j]) * p.dI + c] = st.kidx[(u * p.cap + s_sv[j]) * p.dI + c];
+      }
+      for (int j = tid; j < nh; j += blockDim.x) st.pos[u * p.cap + s_ev[j]] = st.pos[u * p.cap + s_sv[j]];
+      if (tid == 0) st.ctr[u * CTR_STRIDE + CTR_N] = n_next;
     }
   }
 }
@@ -680,6 +804,12 @@ cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call) {
 
 cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call) {
   k_readout_finish<<<call.n_seq, 256, (size_t)L.p.dM * 4, L.stream>>>(L.p, L.st, L.w, L.sc, call);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_readout_apply(const ImLaunch& L, const ImCall& call) {
+  k_readout_apply<<<call.n_seq, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
 }

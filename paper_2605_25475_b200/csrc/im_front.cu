@@ -225,7 +225,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
       st.ev_slot[u * p.tail + a] = sh.ev[a];
       st.ev_pos[u * p.tail + a] = sh.evpos[a];
     }
-    if (call.defer) {  // the moves are made by k_move_survivors once the attention kernel has read the cache
+    if (call.defer) {  // the moves are made by the merge kernel, after the attention kernel has read the cache
       sc.nhole[i] = sh.nh;
       for (int a = 0; a < sh.nh; ++a) sc.surv[(size_t)i * p.tail + a] = sh.surv[a];
     }
@@ -292,8 +292,6 @@ __global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, Im
   const int i = blockIdx.y;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
-  // deferred compaction: this is the call's last kernel, it publishes the new entry count
-  if (call.defer && blockIdx.x == 0 && threadIdx.x == 0) st.ctr[u * CTR_STRIDE + CTR_N] = st.ctr[u * CTR_STRIDE + CTR_NNEXT];
   if (ne <= 0) return;
   const int nh = min(sc.nhole[i], ne);
   const int j0 = blockIdx.x * 4;
@@ -334,14 +332,6 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
   if (L.p.dI == 16) k_decode_front<16><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
   else if (L.p.dI == 8) k_decode_front<8><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
   else k_decode_front<0><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
-  ++*L.launches;
-  return cudaGetLastError();
-}
-
-// last kernel of a decode call with deferred compaction: fills the holes, advances the entry count
-cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call) {
-  dim3 grid((IM_FRONT_MAX_NE + 3) / 4, call.n_seq);
-  k_move_survivors<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
 }

@@ -121,6 +121,95 @@ __global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// Decode variant for at most a few dozen vectors: the same product with the MMA fragments loaded straight
+// from global memory, no shared-memory staging.  It has to run next to the attention kernel, whose CTAs
+// leave about 30 KB of shared memory per SM, and it is latency bound: what counts is how many weight bytes
+// a warp has in flight.  The contraction index may be permuted as long as both operands use the same
+// permutation, so a thread takes 8 consecutive k (one 16-byte load) of its fragment row and feeds them to
+// two k-steps: k-step s of a 32-wide chunk uses elements 4s .. 4s+3 of every thread's vector.  A warp
+// issues all loads of up to 4 chunks before the first MMA.
+// grid = (row tiles over all jobs, ksplit, ceil(NV / 32)), block = 256: the warps take the 32-wide chunks of
+// the K split round-robin and their accumulators are added through shared memory in warp order.
+constexpr int DG_DEPTH = 4;   // 32-wide chunks whose loads (weights and vectors) a warp has in flight
+constexpr int DG_WARPS = 8;
+__global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
+  __shared__ float red[DG_WARPS][16][33];
+  int tile = blockIdx.x, j = 0;
+  while (j + 1 < a.n_jobs && tile >= (a.job[j].rows + 15) / 16) {
+    tile -= (a.job[j].rows + 15) / 16;
+    ++j;
+  }
+  const ImGemmJob job = a.job[j];
+  const int r0 = tile * 16;
+  const int ks = blockIdx.y;
+  const int kspan = a.K / a.ksplit;  // a multiple of 32 (checked by the launcher)
+  const int kbeg = ks * kspan;
+  const long long v0 = (long long)blockIdx.z * VB;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int n_chunks = kspan / 32;
+  // fragment rows of this thread (clamped: results of rows / vectors out of range are not stored)
+  const int rowA = min(r0 + g, job.rows - 1), rowB = min(r0 + g + 8, job.rows - 1);
+  const bf16* xb[4];
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) xb[nt] = vec_ptr(a, job.in_sel, min(v0 + nt * 8 + g, (long long)a.NV - 1)) + kbeg + 8 * t;
+  float acc[4][4];
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+  const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+  for (int c0 = warp; c0 < n_chunks; c0 += DG_WARPS * DG_DEPTH) {
+    // every load of the batch is issued before the first MMA: one memory round trip per batch
+    uint4 fx[DG_DEPTH][4];
+#pragma unroll
+    for (int d = 0; d < DG_DEPTH; ++d) {
+      const int c = c0 + DG_WARPS * d;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) fx[d][nt] = c < n_chunks ? *reinterpret_cast<const uint4*>(xb[nt] + c * 32) : zero4;
+    }
+    for (int term = 0; term < (job.W2 ? 2 : 1); ++term) {
+      const bf16* W = term ? job.W2 : job.W;
+      const bf16* wa = W + (size_t)rowA * a.K + kbeg + 8 * t;
+      const bf16* wb = W + (size_t)rowB * a.K + kbeg + 8 * t;
+      uint4 fa[DG_DEPTH], fb[DG_DEPTH];
+#pragma unroll
+      for (int d = 0; d < DG_DEPTH; ++d) {
+        const int c = c0 + DG_WARPS * d;
+        fa[d] = c < n_chunks ? *reinterpret_cast<const uint4*>(wa + c * 32) : zero4;
+        fb[d] = c < n_chunks ? *reinterpret_cast<const uint4*>(wb + c * 32) : zero4;
+      }
+#pragma unroll
+      for (int d = 0; d < DG_DEPTH; ++d) {
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          mma_bf16(acc[nt], fa[d].x, fb[d].x, fa[d].y, fb[d].y, fx[d][nt].x, fx[d][nt].y);
+          mma_bf16(acc[nt], fa[d].z, fb[d].z, fa[d].w, fb[d].w, fx[d][nt].z, fx[d][nt].w);
+        }
+      }
+    }
+  }
+  // C fragment: rows g / g+8, columns 8 nt + 2t / + 1
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) {
+    red[warp][g][nt * 8 + 2 * t] = acc[nt][0];
+    red[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1];
+    red[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2];
+    red[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3];
+  }
+  __syncthreads();
+  float* outk = a.out + (size_t)ks * a.ks_stride;
+  for (int idx = threadIdx.x; idx < 16 * VB; idx += DG_WARPS * 32) {
+    const int r = idx & 15, vl = idx >> 4;
+    const long long v = v0 + vl;
+    if (v < a.NV && r0 + r < job.rows) {
+      float sum = 0.f;
+#pragma unroll
+      for (int w = 0; w < DG_WARPS; ++w) sum += red[w][r][vl];  // warp order: deterministic
+      outk[(v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0 + r] = sum;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Indexer key projection U_k x in float64 (the cached key is a quantised code: the value that gets
 // rounded to bf16 must not depend on the summation order).  K is split over blockIdx.x; one warp
 // per vector.  keyp[ks][v][r] receives the partial sums.
@@ -179,6 +268,14 @@ cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
     attr_done = true;
   }
   ImGemmArgs a = a_in;
+  if (a.direct && a.ksplit > 0 && a.K % a.ksplit == 0 && (a.K / a.ksplit) % 32 == 0 && a.NV > 0) {
+    int tiles = 0;
+    for (int j = 0; j < a.n_jobs; ++j) tiles += (a.job[j].rows + 15) / 16;
+    dim3 grid(tiles, a.ksplit, (unsigned)((a.NV + VB - 1) / VB));
+    k_direct_gemm<<<grid, DG_WARPS * 32, 0, L.stream>>>(a);
+    ++*L.launches;
+    return cudaGetLastError();
+  }
   a.any_w2 = 0;
   for (int j = 0; j < a.n_jobs; ++j) a.any_w2 |= a.job[j].W2 != nullptr;
   if (a.kc <= 0 || a.kc > KC_MAX || a.kc % 16) a.kc = KC_MAX;

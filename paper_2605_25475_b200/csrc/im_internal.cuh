@@ -99,7 +99,11 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
   float* part;       // attention partials (acc[d], max, sum): generic kernel [max_seqs][H][max_splits][d + 2];
                      // streaming kernel [warps + rows][Gq][d + 2]
   float* rpart;      // [max_seqs][ceil(dM / IM_READOUT_ROWS)][Dkv] readout partials
-  float* mres;       // [max_seqs][Dkv + 1] memory readout m(q) in KV space, then the gate g(q)
+  float* mres;       // [max_seqs][Dkv + 2] memory readout in KV space, the gate g(q), the denominator sum.  In a call
+                     // with deferred compaction: numerator and denominator sum of Eq. 5 over the state from before
+                     // the call's memory write (the merge adds the write's terms); otherwise the final m(q), gate, -
+  float* phiq;       // [max_seqs][dM] phi(q) of the call (K-split partials summed)
+  int32_t* n_att;    // [max_seqs] entries per sequence the streaming attention kernel of the call ran over
   uint8_t* qpack;    // [n_seq][ceil(C / IM_TC_QT)][IM_TC_TILE_BYTES] query operand of the tensor-core prefill scoring
 };
 
@@ -134,6 +138,7 @@ struct ImGemmArgs {
   int out_cnt;
   int NV, K, ksplit;
   int kc;      // K elements staged per round (0: the maximum, 512); small values keep the shared-memory footprint low
+  int direct;  // 1: few vectors (decode) - the variant without shared-memory staging, if the K split is a multiple of 32
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
 };
 
@@ -178,11 +183,12 @@ cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, vo
 cudaError_t im_attn_prepare(const ImDims& p);
 cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call);
+cudaError_t im_launch_readout_apply(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
                                      const void* q, int n_ctas);
 cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas, const void* q,
                                       const void* k_new, const void* v_new);
-cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call);
+
 cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,
                            uint8_t* keep, int32_t* n_evict, cudaStream_t stream);
 cudaError_t im_launch_init_weights(const ImDims& p, const ImWeights& w, int layer, uint64_t seed, float std,
