@@ -177,7 +177,7 @@ struct im_ctx {
   bool fast_attn = false;
   // Independent pieces of one decode call run on three side streams that fork from and join back into
   // the caller's stream (plain event dependencies, so the pattern can be captured into a CUDA graph).
-  cudaStream_t side[3] = {nullptr, nullptr, nullptr};
+  cudaStream_t side[4] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t ev[10] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   bool concurrent = false;
   bool prefetch_next = true;         // warm L2 with the next layer's weights / index state during attention
@@ -342,14 +342,14 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     // the short side kernels should be dispatched ahead of the long attention grid when both are ready
     int prio_lo = 0, prio_hi = 0;
     if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
-    for (int k = 0; k < 3 && e == cudaSuccess; ++k)
+    for (int k = 0; k < 4 && e == cudaSuccess; ++k)
       e = cudaStreamCreateWithPriority(&ctx->side[k], cudaStreamNonBlocking, prio_hi);
   }
   for (int k = 0; k < 10 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
-    for (int k = 0; k < 3; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
+    for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
     for (int k = 0; k < 10; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
     delete ctx;
     return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
@@ -361,7 +361,7 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
 int im_destroy(im_ctx* ctx) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   cudaError_t e = cudaDeviceSynchronize();
-  for (int k = 0; k < 3; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
+  for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
   for (int k = 0; k < 10; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   delete ctx;
   if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
@@ -509,14 +509,14 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   //      once over the entries cached before the call.  The merge adds the new token, removes the evicted
   //      entries again (exactly, see k_attn_merge_rows), adds the terms of this call's memory write to the
   //      readout, and fills the holes.
-  //        s0: attention ----------------------------------------------------------> merge
+  //        s0: (waits for the three projections) attention ------------------------> merge
   //        s1: indexer projections -> front (append, score, select, gather) -> phi of the evicted keys ->
   //            readout over the memory after the write (k_readout_apply)
   //            [-> memory write: not needed by the merge, it only has to end with the call]
   //        s2: phi(q) / gate projections -> readout partials -> readout over the memory as it is before
   //            the write
-  //        s3: fold of the pending list -> float64 key projection (needed by front) -> L2 prefetch for the
-  //            next layer
+  //        s3: float64 key projection (needed by front) -> L2 prefetch for the next layer
+  //        s4: fold of the pending list (before front, which changes the counters, and before the readout)
   //      With IM_OPT_CONCURRENCY off the same kernels run on s0 in an order that respects these arrows.
   //  (B) in order on s0, attention after the compaction: everything else (large evicted sets, budgets
   //      beyond the fused front kernel, head shapes without the streaming attention kernel).
@@ -526,30 +526,27 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   const bool conc = defer && ctx->concurrent;
   call.defer = defer ? 1 : 0;
   ImLaunch L = make_launch(ctx, layer, s0);
-  ImLaunch L1 = L, L2 = L, L3 = L;
+  ImLaunch L1 = L, L2 = L, L3 = L, L4 = L;
+  const bool mem_write = due && ne_max > 0 && p.mem;
   if (conc) {
     L1.stream = ctx->side[0];
     L2.stream = ctx->side[1];
     L3.stream = ctx->side[2];
+    if (mem_write) L4.stream = ctx->side[3];
     CK(cudaEventRecord(ctx->ev[0], s0));
     CK(cudaStreamWaitEvent(L1.stream, ctx->ev[0], 0));
     CK(cudaStreamWaitEvent(L2.stream, ctx->ev[0], 0));
     CK(cudaStreamWaitEvent(L3.stream, ctx->ev[0], 0));
+    if (mem_write) CK(cudaStreamWaitEvent(L4.stream, ctx->ev[0], 0));
   }
   const bool prof = ctx->prof_target == 0 && ctx->prof_used + 2 <= ctx->prof_ev.size();
-  if (conc) {  // a5 first: it overlaps with everything below
-    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
-    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
-    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
-  }
-  const bool mem_write = due && ne_max > 0 && p.mem;
-  // s3: fold (reads the counters of before the call; the readout reads the folded state), key projection
+  // s4: fold (reads the counters of before the call; the readout reads the folded state); s3: key projection
   if (mem_write) {
-    CKL(im_launch_mem_fold(L3, call));
-    if (conc) CK(cudaEventRecord(ctx->ev[7], L3.stream));
+    CKL(im_launch_mem_fold(L4, call));
+    if (conc) CK(cudaEventRecord(ctx->ev[7], L4.stream));
   }
   CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
-  if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // fold and key projection done
+  if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // key projection done
   if (ctx->prefetch_next && ctx->fast_attn) {
     // warm L2 for the next layer's small kernels while this layer's attention streams K/V
     ImLaunch Lp = L3;
@@ -586,6 +583,20 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     g.job[1] = {L.w.wg, nullptr, 1, r.wg, 2};
     CKL(im_launch_gemm(L2, g));
   }
+  if (conc) {
+    // a5.  The three projections head every side chain and are latency bound (one memory round trip each);
+    // they get the first microseconds of the call to themselves, because a memory access issued while the
+    // attention kernel keeps the memory system's queues full takes several times longer.  Everything after
+    // them runs next to the attention kernel.
+    CK(cudaEventRecord(ctx->ev[1], L1.stream));
+    CK(cudaEventRecord(ctx->ev[6], L2.stream));
+    CK(cudaStreamWaitEvent(s0, ctx->ev[1], 0));
+    CK(cudaStreamWaitEvent(s0, ctx->ev[6], 0));
+    CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
+    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
+  }
   // an evicted set larger than the pending list is accumulated into Mhat itself, which the readout reads
   const bool readout_early = !(mem_write && ne_max > p.F);
   if (conc && mem_write) CK(cudaStreamWaitEvent(L2.stream, ctx->ev[7], 0));
@@ -593,7 +604,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   if (defer && p.mem) CKL(im_launch_readout_finish(L2, call));  // over the memory as it is before this call's write
   if (conc) {
     CK(cudaEventRecord(ctx->ev[4], L2.stream));  // s2 finished
-    CK(cudaStreamWaitEvent(L1.stream, ctx->ev[2], 0));  // the front kernel changes the counters the fold reads
+    CK(cudaStreamWaitEvent(L1.stream, ctx->ev[2], 0));
+    if (mem_write) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0));  // the front kernel changes the counters the fold reads
   }
   // append + a1 (+ a2 and the gather of the evicted pairs when the evicted set is small enough for one
   // block per sequence; a4 in the same kernel unless the compaction is deferred)

@@ -23,7 +23,7 @@ namespace {
 
 constexpr float NEG_INF = -__builtin_huge_valf();
 constexpr int TILE = IM_ATTN_TILE;       // keys per tile
-constexpr int STAGES = 3;                // ring depth per warp
+constexpr int STAGES = 2;                // ring depth per warp
 constexpr int WARPS = IM_ATTN_WARPS;     // consumer warps per CTA (each also issues its own TMA)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;  // try_wait attempts before a warp gives up and flags ST_TIMEOUT
 
@@ -524,11 +524,12 @@ __device__ __forceinline__ void softmax_push(float s, const float (&v)[CPL], flo
 // entries hold at most 90 % of the softmax mass (the error of the remainder grows by at most 10); beyond
 // that the warp recomputes its head over the retained entries from the cache, which is still uncompacted.
 template <int DH, typename OutT>
-__global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, ImScratch sc, ImCall call, int n_ctas,
+__global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st, ImScratch sc, ImCall call, int n_ctas,
                                                           OutT* __restrict__ out, const bf16* __restrict__ q,
                                                           const bf16* __restrict__ k_new, const bf16* __restrict__ v_new) {
   constexpr int CPL = DH / 32;  // columns per lane
   __shared__ int s_ev[IM_FRONT_MAX_NE], s_sv[IM_FRONT_MAX_NE];
+  __shared__ float s_q[8][DH];  // recompute path: the warp's query row
   const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
@@ -639,32 +640,79 @@ __global__ void __launch_bounds__(256) k_attn_merge_rows(ImDims p, ImState st, I
             for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[k] * en;
             M = Mn;
           } else {
-            // four keys per round so that their loads overlap; an evicted key gets the score -inf
-            for (int t0 = key0; t0 < key1; t0 += 4) {
-              float kk[4][CPL], vk[4][CPL], sc4[4];
+            // One key per lane, 32 keys per round: the lane forms its key's whole dot product (q from shared
+            // memory; 16 independent 16-byte loads), then the warp adds the 32 weighted V rows, lane l holding
+            // columns CPL l .. CPL l + CPL - 1 (32 independent loads).  An evicted key gets the weight 0.  The
+            // range's own softmax state is merged like a stored partial at the end.
+            float* sq = s_q[warp];
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const int t = min(t0 + j, key1 - 1);
+            for (int k = 0; k < CPL; ++k) sq[lane + 32 * k] = qv[k];
+            __syncwarp();
+            float Mr = NEG_INF, Lr = 0.f, racc[CPL];
 #pragma unroll
-                for (int k = 0; k < CPL; ++k) {
-                  kk[j][k] = __bfloat162float(Kb[(size_t)t * DH + lane + 32 * k]);
-                  vk[j][k] = __bfloat162float(Vb[(size_t)t * DH + lane + 32 * k]);
+            for (int k = 0; k < CPL; ++k) racc[k] = 0.f;
+            for (int t0 = key0; t0 < key1; t0 += 32) {
+              const int tk = t0 + lane;
+              bool valid = tk < key1;
+              for (int a = 0; a < ne; ++a) valid &= __shfl_sync(0xffffffffu, ev_l, a) != tk;
+              const uint4* kr = reinterpret_cast<const uint4*>(Kb + (size_t)min(tk, key1 - 1) * DH);
+              uint4 kw[DH / 8];
+#pragma unroll
+              for (int c = 0; c < DH / 8; ++c) kw[c] = kr[c];
+              uint2 vw[32];
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const bf16* vr = Vb + (size_t)min(t0 + j, key1 - 1) * DH + CPL * lane;
+                if (CPL == 4) vw[j] = *reinterpret_cast<const uint2*>(vr);
+                else { vw[j].x = *reinterpret_cast<const uint32_t*>(vr); vw[j].y = 0u; }
+              }
+              float sd = 0.f;
+#pragma unroll
+              for (int c = 0; c < DH / 8; ++c) {
+                const uint32_t ww[4] = {kw[c].x, kw[c].y, kw[c].z, kw[c].w};
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2) {
+                  sd = fmaf(sq[c * 8 + 2 * e2], __uint_as_float(ww[e2] << 16), sd);
+                  sd = fmaf(sq[c * 8 + 2 * e2 + 1], __uint_as_float(ww[e2] & 0xffff0000u), sd);
                 }
               }
+              sd = valid ? sd * sl2 : NEG_INF;
+              float mb = sd;
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                float dot = 0.f;
+              for (int o = 16; o > 0; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+              if (mb == NEG_INF) continue;  // (warp-uniform) nothing left in this round
+              const float Mn = fmaxf(Mr, mb);
+              const float eo = exp2f(Mr - Mn);
+              const float pl = valid ? exp2f(sd - Mn) : 0.f;
+              Lr = Lr * eo + warp_sum_f(pl);
 #pragma unroll
-                for (int k = 0; k < CPL; ++k) dot = fmaf(qv[k], kk[j][k], dot);
-                sc4[j] = warp_sum_f(dot) * sl2;
-                bool gone = t0 + j >= key1;
-                for (int a = 0; a < ne; ++a) gone |= __shfl_sync(0xffffffffu, ev_l, a) == t0 + j;
-                if (gone) sc4[j] = NEG_INF;
+              for (int k = 0; k < CPL; ++k) racc[k] *= eo;
+              Mr = Mn;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float pj = __shfl_sync(0xffffffffu, pl, j);
+                racc[0] = fmaf(pj, __uint_as_float(vw[j].x << 16), racc[0]);
+                racc[1] = fmaf(pj, __uint_as_float(vw[j].x & 0xffff0000u), racc[1]);
+                if (CPL == 4) {
+                  racc[2] = fmaf(pj, __uint_as_float(vw[j].y << 16), racc[2]);
+                  racc[3] = fmaf(pj, __uint_as_float(vw[j].y & 0xffff0000u), racc[3]);
+                }
               }
-#pragma unroll
-              for (int j = 0; j < 4; ++j)
-                if (sc4[j] > NEG_INF) softmax_push<CPL>(sc4[j], vk[j], M, L, res);
             }
+            // columns CPL l + k -> l + 32 k through the warp's shared row, then the usual merge
+            __syncwarp();
+#pragma unroll
+            for (int k = 0; k < CPL; ++k) sq[CPL * lane + k] = racc[k];
+            __syncwarp();
+            if (Lr > 0.f) {
+              const float Mn = fmaxf(M, Mr);
+              const float eo = exp2f(M - Mn), en = exp2f(Mr - Mn);
+              L = L * eo + Lr * en;
+#pragma unroll
+              for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + sq[lane + 32 * k] * en;
+              M = Mn;
+            }
+            __syncwarp();
           }
         }
       }

@@ -130,8 +130,16 @@ __global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
 // issues all loads of up to 4 chunks before the first MMA.
 // grid = (row tiles over all jobs, ksplit, ceil(NV / 32)), block = 256: the warps take the 32-wide chunks of
 // the K split round-robin and their accumulators are added through shared memory in warp order.
+// 16-byte read-only load that the compiler may neither reorder nor delay: the point of the direct variant is
+// that all loads of a batch are in flight together
+__device__ __forceinline__ uint4 ldg128_now(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
 constexpr int DG_DEPTH = 4;   // 32-wide chunks whose loads (weights and vectors) a warp has in flight
 constexpr int DG_WARPS = 8;
+template <bool TWO>  // TWO: the jobs have a second weight term
 __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
   __shared__ float red[DG_WARPS][16][33];
   int tile = blockIdx.x, j = 0;
@@ -158,31 +166,41 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
   for (int nt = 0; nt < 4; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
   const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
   for (int c0 = warp; c0 < n_chunks; c0 += DG_WARPS * DG_DEPTH) {
-    // every load of the batch is issued before the first MMA: one memory round trip per batch
+    // weights (the long round trip) first, then the vectors (L2: every block reads the same few vectors)
+    uint4 fa[TWO ? 2 : 1][DG_DEPTH], fb[TWO ? 2 : 1][DG_DEPTH];
+#pragma unroll
+    for (int term = 0; term < (TWO ? 2 : 1); ++term) {
+      const bf16* W = term ? job.W2 : job.W;
+      const bf16* wa = W + (size_t)rowA * a.K + kbeg + 8 * t;
+      const bf16* wb = W + (size_t)rowB * a.K + kbeg + 8 * t;
+#pragma unroll
+      for (int d = 0; d < DG_DEPTH; ++d) {
+        const int c = c0 + DG_WARPS * d;
+        fa[term][d] = c < n_chunks ? ldg128_now(wa + c * 32) : zero4;
+        fb[term][d] = c < n_chunks ? ldg128_now(wb + c * 32) : zero4;
+      }
+    }
     uint4 fx[DG_DEPTH][4];
 #pragma unroll
     for (int d = 0; d < DG_DEPTH; ++d) {
       const int c = c0 + DG_WARPS * d;
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt) fx[d][nt] = c < n_chunks ? *reinterpret_cast<const uint4*>(xb[nt] + c * 32) : zero4;
+      for (int nt = 0; nt < 4; ++nt) fx[d][nt] = c < n_chunks ? ldg128_now(xb[nt] + c * 32) : zero4;
     }
-    for (int term = 0; term < (job.W2 ? 2 : 1); ++term) {
-      const bf16* W = term ? job.W2 : job.W;
-      const bf16* wa = W + (size_t)rowA * a.K + kbeg + 8 * t;
-      const bf16* wb = W + (size_t)rowB * a.K + kbeg + 8 * t;
-      uint4 fa[DG_DEPTH], fb[DG_DEPTH];
+    asm volatile("" ::: "memory");  // every load of the batch is issued before the first MMA: one round trip
 #pragma unroll
-      for (int d = 0; d < DG_DEPTH; ++d) {
-        const int c = c0 + DG_WARPS * d;
-        fa[d] = c < n_chunks ? *reinterpret_cast<const uint4*>(wa + c * 32) : zero4;
-        fb[d] = c < n_chunks ? *reinterpret_cast<const uint4*>(wb + c * 32) : zero4;
+    for (int d = 0; d < DG_DEPTH; ++d) {
+      const uint4* x = fx[d];
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        mma_bf16(acc[nt], fa[0][d].x, fb[0][d].x, fa[0][d].y, fb[0][d].y, x[nt].x, x[nt].y);
+        mma_bf16(acc[nt], fa[0][d].z, fb[0][d].z, fa[0][d].w, fb[0][d].w, x[nt].z, x[nt].w);
       }
-#pragma unroll
-      for (int d = 0; d < DG_DEPTH; ++d) {
+      if (TWO) {
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
-          mma_bf16(acc[nt], fa[d].x, fb[d].x, fa[d].y, fb[d].y, fx[d][nt].x, fx[d][nt].y);
-          mma_bf16(acc[nt], fa[d].z, fb[d].z, fa[d].w, fb[d].w, fx[d][nt].z, fx[d][nt].w);
+          mma_bf16(acc[nt], fa[TWO ? 1 : 0][d].x, fb[TWO ? 1 : 0][d].x, fa[TWO ? 1 : 0][d].y, fb[TWO ? 1 : 0][d].y, x[nt].x, x[nt].y);
+          mma_bf16(acc[nt], fa[TWO ? 1 : 0][d].z, fb[TWO ? 1 : 0][d].z, fa[TWO ? 1 : 0][d].w, fb[TWO ? 1 : 0][d].w, x[nt].z, x[nt].w);
         }
       }
     }
@@ -268,11 +286,15 @@ cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
     attr_done = true;
   }
   ImGemmArgs a = a_in;
-  if (a.direct && a.ksplit > 0 && a.K % a.ksplit == 0 && (a.K / a.ksplit) % 32 == 0 && a.NV > 0) {
+  int n_w2 = 0;
+  for (int j = 0; j < a.n_jobs; ++j) n_w2 += a.job[j].W2 != nullptr;
+  if (a.direct && a.ksplit > 0 && a.K % a.ksplit == 0 && (a.K / a.ksplit) % 32 == 0 && a.NV > 0 &&
+      (n_w2 == 0 || n_w2 == a.n_jobs)) {
     int tiles = 0;
     for (int j = 0; j < a.n_jobs; ++j) tiles += (a.job[j].rows + 15) / 16;
     dim3 grid(tiles, a.ksplit, (unsigned)((a.NV + VB - 1) / VB));
-    k_direct_gemm<<<grid, DG_WARPS * 32, 0, L.stream>>>(a);
+    if (n_w2) k_direct_gemm<true><<<grid, DG_WARPS * 32, 0, L.stream>>>(a);
+    else k_direct_gemm<false><<<grid, DG_WARPS * 32, 0, L.stream>>>(a);
     ++*L.launches;
     return cudaGetLastError();
   }
