@@ -320,15 +320,54 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     h2d = sum(t.numel() * t.element_size() for t in host[0])
     d2h = hout.numel() * hout.element_size()
 
-    def step(s):
-        hx, hq, hk, hv = host[s % n_in]
+    cs, ds = torch.cuda.Stream(device), torch.cuda.Stream(device)   # host-to-device / device-to-host copies
+    ev_in = [torch.cuda.Event() for _ in range(L)]
+    ev_out = [torch.cuda.Event() for _ in range(L)]
+    ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
+
+    def enqueue(k):
+        """One step: the copies of layer l + 1's inputs and of layer l - 1's outputs run next to layer l's
+        kernels (three streams, forked from and joined back into `stream`, so that it can be captured)."""
+        hx, hq, hk, hv = host[k]
+        ev_fork.record(stream)
+        cs.wait_event(ev_fork)
+        ds.wait_event(ev_fork)
         for layer in range(L):
-            dx[layer].copy_(hx[layer], non_blocking=True)
-            dq[layer].copy_(hq[layer], non_blocking=True)
-            dk[layer].copy_(hk[layer], non_blocking=True)
-            dv[layer].copy_(hv[layer], non_blocking=True)
+            with torch.cuda.stream(cs):
+                dx[layer].copy_(hx[layer], non_blocking=True)
+                dq[layer].copy_(hq[layer], non_blocking=True)
+                dk[layer].copy_(hk[layer], non_blocking=True)
+                dv[layer].copy_(hv[layer], non_blocking=True)
+                ev_in[layer].record(cs)
+            stream.wait_event(ev_in[layer])
             g.decode_step(layer, ids, dx[layer], dq[layer], dq[layer], dk[layer], dv[layer], dout[layer])
-            hout[layer].copy_(dout[layer], non_blocking=True)
+            ev_out[layer].record(stream)
+            ds.wait_event(ev_out[layer])
+            with torch.cuda.stream(ds):
+                hout[layer].copy_(dout[layer], non_blocking=True)
+        ev_join.record(ds)
+        stream.wait_event(ev_join)
+
+    # The step as a user would run it in a serving loop: host-to-device copies, the 32 layer calls and the
+    # device-to-host copy of the outputs, captured once per input set into a CUDA graph (the pinned host
+    # buffers are the graph's sources and destination) and replayed; without --graph the same work is enqueued
+    # call by call.
+    graphs = None
+    if args.graph:
+        enqueue(0)                                               # one eager pass before capturing
+        stream.synchronize()
+        graphs = []
+        for k in range(n_in):
+            gk = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gk, stream=stream):
+                enqueue(k)
+            graphs.append(gk)
+
+    def step(s):
+        if graphs is not None:
+            graphs[s % n_in].replay()
+        else:
+            enqueue(s % n_in)
         stream.synchronize()                                     # the caller has the step's result on the host
 
     for s in range(min(3, args.warmup)):
@@ -344,7 +383,7 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     barrier(world)
     ms = max_over_ranks(ev0.elapsed_time(ev1), world, device)
     return {"value": wl.n_seq * args.steps * world / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "ms_per_step": ms / args.steps}
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms / args.steps, "cuda_graph": graphs is not None}
 
 
 # ----------------------------------------------------------------------------------------------
