@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(128) k_skinny_gemm(ImGemmArgs a) {
 // that all loads of a batch are in flight together
 __device__ __forceinline__ uint4 ldg128_now(const void* p) {
   uint4 v;
-  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
 constexpr int DG_DEPTH = 4;   // 32-wide chunks whose loads (weights and vectors) a warp has in flight
