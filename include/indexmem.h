@@ -193,7 +193,7 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *   IM_OPT_CONCURRENCY   1 (default where the streaming attention kernel is available): im_decode_step
  *                        starts the attention kernel at once over the entries cached before the call and
  *                        runs the rest of the call (projections, append / score / select, memory write,
- *                        readout) next to it on three internal side streams that fork from and join back
+ *                        readout) next to it on four internal side streams that fork from and join back
  *                        into `cuda_stream` inside the call (events only, so the pattern can be captured
  *                        into a CUDA graph); the merge adds the new token and removes the evicted entries
  *                        from the softmax sums again, so the result is the attention over the retained set.
