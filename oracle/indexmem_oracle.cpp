@@ -230,9 +230,13 @@ double gate_of(const Layer& L, const float* q) {
 }
 
 // Sec. 2.1 KV caching: o_j = sum_t softmax_t(scale q_j . k_t) v_t over the retained set.
-void attention(const Layer& L, const Seq& S, const float* q /*[H,d]*/, double* o /*[H,d]*/) {
+// `max_pos`: only entries at positions <= max_pos take part (the causal mask of a chunk's own queries);
+// entries are kept in ascending position, so these are a prefix of the list.
+void attention(const Layer& L, const Seq& S, const float* q /*[H,d]*/, double* o /*[H,d]*/,
+               int64_t max_pos = std::numeric_limits<int64_t>::max()) {
   const int d = L.c.d;
-  const size_t n = S.R.size();
+  size_t n = 0;
+  while (n < S.R.size() && (int64_t)S.R[n].pos <= max_pos) ++n;
   std::vector<double> logit(n);
   for (int j = 0; j < L.c.H; ++j) {
     const int g = j / L.Gq;
@@ -346,14 +350,37 @@ int orc_set_weights(void* h, int which, const float* data, int64_t n) {
 
 // Sec. 4 schedule, prefill side: append the chunk, pool the chunk's query scores over every cached
 // entry under the causal mask, then compress to the budget.
-int orc_prefill_chunk(void* h, int seq, int C, const float* X /*[C,D]*/, const float* Qpre /*[C,H,d]*/,
-                      const float* K /*[C,Hkv,d]*/, const float* V /*[C,Hkv,d]*/) {
+// Optional layer outputs of the chunk's own queries (Q != null; Eq. 4-5): query s attends to what is cached
+// when the chunk arrives plus the chunk's tokens up to itself (Sec. 2.1 causal attention; the chunk is
+// compressed only after it has been processed, Sec. 4), and reads the memory as the previous evict steps
+// left it.  out_bf16 / out_f64: [C,H,d], either may be null.
+int orc_prefill_chunk_out(void* h, int seq, int C, const float* X /*[C,D]*/, const float* Qpre /*[C,H,d]*/,
+                          const float* Q /*[C,H,d] or null*/, const float* K /*[C,Hkv,d]*/,
+                          const float* V /*[C,Hkv,d]*/, float* out_bf16, double* out_f64) {
   Layer* L = static_cast<Layer*>(h);
   Seq& S = L->seqs[seq];
   const int D = L->D, Dkv = L->Dkv, HI = L->c.HI, dI = L->c.dI;
   const int64_t T0 = S.T;
   for (int c = 0; c < C; ++c)
     append(*L, S, X + (size_t)c * D, K + (size_t)c * Dkv, V + (size_t)c * Dkv);
+  if (Q && (out_bf16 || out_f64)) {
+    std::vector<double> o(D), m(D);
+    for (int c = 0; c < C; ++c) {
+      const float* q = Q + (size_t)c * D;
+      attention(*L, S, q, o.data(), T0 + c);
+      double gate = 0.0;
+      std::fill(m.begin(), m.end(), 0.0);
+      if (L->c.enable_memory) {
+        mem_read(*L, S, q, m.data());
+        gate = gate_of(*L, q);
+      }
+      for (int j = 0; j < D; ++j) {
+        const double val = o[j] + gate * m[j];
+        if (out_f64) out_f64[(size_t)c * D + j] = val;
+        if (out_bf16) out_bf16[(size_t)c * D + j] = (float)bf16_round(val);
+      }
+    }
+  }
   std::vector<double> qf((size_t)C * HI * dI), alpha((size_t)C * HI);
   for (int c = 0; c < C; ++c)
     index_query(*L, X + (size_t)c * D, Qpre + (size_t)c * D, &qf[(size_t)c * HI * dI], &alpha[(size_t)c * HI]);
@@ -367,6 +394,9 @@ int orc_prefill_chunk(void* h, int seq, int C, const float* X /*[C,D]*/, const f
   }
   compress(*L, S);
   return 0;
+}
+int orc_prefill_chunk(void* h, int seq, int C, const float* X, const float* Qpre, const float* K, const float* V) {
+  return orc_prefill_chunk_out(h, seq, C, X, Qpre, nullptr, K, V, nullptr, nullptr);
 }
 
 // One decode token for one sequence (Sec. 4 schedule, decode side; Eq. 4-7).
@@ -412,15 +442,20 @@ int orc_decode_batch(void* h, int n_seq, const int32_t* seq_ids, const float* x,
                     out_bf16 ? out_bf16 + i * D : nullptr, out_f64 ? out_f64 + i * D : nullptr);
   return 0;
 }
-int orc_prefill_batch(void* h, int n_seq, const int32_t* seq_ids, int C, const float* X, const float* Qpre,
-                      const float* K, const float* V) {
+int orc_prefill_batch_out(void* h, int n_seq, const int32_t* seq_ids, int C, const float* X, const float* Qpre,
+                          const float* Q, const float* K, const float* V, float* out_bf16, double* out_f64) {
   Layer* L = static_cast<Layer*>(h);
   const size_t D = L->D, Dkv = L->Dkv;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int i = 0; i < n_seq; ++i)
-    orc_prefill_chunk(h, seq_ids[i], C, X + (size_t)i * C * D, Qpre + (size_t)i * C * D,
-                      K + (size_t)i * C * Dkv, V + (size_t)i * C * Dkv);
+    orc_prefill_chunk_out(h, seq_ids[i], C, X + (size_t)i * C * D, Qpre + (size_t)i * C * D,
+                          Q ? Q + (size_t)i * C * D : nullptr, K + (size_t)i * C * Dkv, V + (size_t)i * C * Dkv,
+                          out_bf16 ? out_bf16 + (size_t)i * C * D : nullptr, out_f64 ? out_f64 + (size_t)i * C * D : nullptr);
   return 0;
+}
+int orc_prefill_batch(void* h, int n_seq, const int32_t* seq_ids, int C, const float* X, const float* Qpre,
+                      const float* K, const float* V) {
+  return orc_prefill_batch_out(h, n_seq, seq_ids, C, X, Qpre, nullptr, K, V, nullptr, nullptr);
 }
 
 // ---- state export (entries in cache order = ascending position)

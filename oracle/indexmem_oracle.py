@@ -92,6 +92,8 @@ def _load():
     L.orc_decode_step.argtypes = [vp, C.c_int, vp, vp, vp, vp, vp, vp, vp]
     L.orc_decode_batch.argtypes = [vp, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp]
     L.orc_prefill_batch.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, vp, vp]
+    L.orc_prefill_chunk_out.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp, vp]
+    L.orc_prefill_batch_out.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, vp, vp, vp, vp, vp]
     L.orc_count.argtypes = [vp, C.c_int]
     L.orc_tokens_seen.argtypes = [vp, C.c_int]
     L.orc_tokens_seen.restype = i64
@@ -172,6 +174,28 @@ class OracleLayer:
         n, Cn = X.shape[0], X.shape[1]
         assert n == ids.size and X.shape == (n, Cn, self.D)
         self.lib.orc_prefill_batch(self.h, n, _p(ids), Cn, _p(X), _p(Qpre), _p(K), _p(V))
+
+    def prefill_chunk_out(self, seq: int, X, Qpre, Q, K, V):
+        """prefill_chunk that also returns the layer outputs of the chunk's own queries:
+        (out_bf16 [C,H,d] float32 holding bf16 values, out_f64 [C,H,d])."""
+        X, Qpre, Q, K, V = _f32(X), _f32(Qpre), _f32(Q), _f32(K), _f32(V)
+        Cn = X.shape[0]
+        assert X.shape == (Cn, self.D) and Qpre.size == Cn * self.D and Q.size == Cn * self.D
+        assert K.size == Cn * self.Dkv and V.size == K.size
+        ob = np.empty((Cn, self.cfg.H, self.cfg.d), dtype=np.float32)
+        od = np.empty((Cn, self.cfg.H, self.cfg.d), dtype=np.float64)
+        self.lib.orc_prefill_chunk_out(self.h, seq, Cn, _p(X), _p(Qpre), _p(Q), _p(K), _p(V), _p(ob), _p(od))
+        return ob, od
+
+    def prefill_batch_out(self, seq_ids, X, Qpre, Q, K, V):
+        X, Qpre, Q, K, V = _f32(X), _f32(Qpre), _f32(Q), _f32(K), _f32(V)
+        ids = np.ascontiguousarray(np.asarray(seq_ids, dtype=np.int32))
+        n, Cn = X.shape[0], X.shape[1]
+        assert n == ids.size and X.shape == (n, Cn, self.D) and Q.size == X.size
+        ob = np.empty((n, Cn, self.cfg.H, self.cfg.d), dtype=np.float32)
+        od = np.empty((n, Cn, self.cfg.H, self.cfg.d), dtype=np.float64)
+        self.lib.orc_prefill_batch_out(self.h, n, _p(ids), Cn, _p(X), _p(Qpre), _p(Q), _p(K), _p(V), _p(ob), _p(od))
+        return ob, od
 
     def decode_step(self, seq: int, x, q_pre, q, k_new, v_new):
         """Returns (out_bf16 [H,d] float32 holding bf16 values, out_f64 [H,d])."""

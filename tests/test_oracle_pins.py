@@ -395,3 +395,84 @@ def test_gate_bias_and_range():
         L.set_weights(w)
         _, g = L.mem_read(0, Q[5].reshape(-1))
         assert lo <= g <= hi
+
+
+# ------------------------------------------------------------------ layer outputs of a prefill chunk's own queries
+def test_chunk_outputs_with_infinite_budget_are_causal_softmax_attention():
+    """Nothing is ever evicted and the memory is off: the outputs of a prompt fed in three ragged chunks are
+    textbook causal attention over the whole prompt (numpy, float64), row by row."""
+    rng = np.random.default_rng(31)
+    L = orc.OracleLayer(small_cfg(B=10_000, enable_memory=0))
+    rand_weights(L, rng)
+    c = L.cfg
+    n = 23
+    X, Q, K, V = rand_tokens(L, rng, n)
+    outs = []
+    for a, b in ((0, 7), (7, 8), (8, 23)):
+        ob, od = L.prefill_chunk_out(0, X[a:b], Q[a:b], Q[a:b], K[a:b], V[a:b])
+        outs.append(od)
+        assert np.array_equal(ob, bf16(od))
+    got = np.concatenate(outs)
+    for s in range(n):
+        want = softmax_attention(Q[s], K[:s + 1], V[:s + 1], c.H // c.Hkv, 1.0 / math.sqrt(c.d))
+        np.testing.assert_allclose(got[s], want, rtol=1e-12, atol=1e-13)
+    # the mask is causal: a later token must not change an earlier row
+    L2 = orc.OracleLayer(small_cfg(B=10_000, enable_memory=0))
+    rand_weights(L2, np.random.default_rng(31))
+    K2 = K.copy()
+    K2[-1] += 1.0
+    _, od2 = L2.prefill_chunk_out(0, X, Q, Q, K2, V)
+    np.testing.assert_allclose(od2[:-1], got[:-1], rtol=1e-12, atol=1e-13)
+    assert not np.allclose(od2[-1], got[-1])
+
+
+def test_chunk_outputs_attend_to_the_retained_prefix_and_read_the_memory_of_before_the_chunk():
+    """After evictions: a chunk's query s sees exactly (entries retained when the chunk arrives) + (chunk tokens
+    up to s), and Eq. 4 adds g(q) m(q) with the memory as it was BEFORE the chunk's own evict step.  Expected
+    values: numpy softmax over the exported retained set plus the chunk, and Eq. 5 evaluated in numpy on the
+    exported (M, b); the evict step of the chunk itself must not leak into its outputs."""
+    rng = np.random.default_rng(32)
+    L = orc.OracleLayer(small_cfg(B=9, n_sink=1))
+    w = rand_weights(L, rng)
+    c = L.cfg
+    Gq = c.H // c.Hkv
+    X, Q, K, V = rand_tokens(L, rng, 30)
+    L.prefill_chunk(0, X[:14], Q[:14], K[:14], V[:14])          # evicts 5
+    assert L.count(0) == 9 and L.evict_steps(0) == 1
+    e = L.entries(0)
+    M, b = L.memory(0)
+    Cn = 11
+    xs, qs, ks, vs = X[14:14 + Cn], Q[14:14 + Cn], K[14:14 + Cn], V[14:14 + Cn]
+    ob, od = L.prefill_chunk_out(0, xs, qs, qs, ks, vs)
+    assert L.evict_steps(0) == 2                                   # the chunk was compressed afterwards
+    for s in range(Cn):
+        Ks = np.concatenate([e["K"], ks[:s + 1]])
+        Vs = np.concatenate([e["V"], vs[:s + 1]])
+        o = softmax_attention(qs[s], Ks, Vs, Gq, 1.0 / math.sqrt(c.d))
+        qd = qs[s].reshape(-1).astype(np.float64)
+        phi = w["W_theta"].astype(np.float64) @ qd
+        m = (phi @ M) / ((phi ** 2) @ b + c.eps)
+        gate = 1.0 / (1.0 + math.exp(-float(w["w_g"].astype(np.float64).reshape(-1) @ qd)))
+        want = o + gate * m.reshape(c.H, c.d)
+        np.testing.assert_allclose(od[s], want, rtol=1e-10, atol=1e-12)
+    # and the state after the call is the one the plain call leaves
+    L2 = orc.OracleLayer(small_cfg(B=9, n_sink=1))
+    L2.set_weights(w)
+    L2.prefill_chunk(0, X[:14], Q[:14], K[:14], V[:14])
+    L2.prefill_chunk(0, xs, qs, ks, vs)
+    assert np.array_equal(L2.positions(0), L.positions(0))
+    np.testing.assert_array_equal(L2.memory(0)[0], L.memory(0)[0])
+
+
+def test_single_token_chunk_output_equals_decode_output_when_nothing_is_evicted():
+    rng = np.random.default_rng(33)
+    La, Lb = orc.OracleLayer(small_cfg(B=50, tau=1)), orc.OracleLayer(small_cfg(B=50, tau=1))
+    w = rand_weights(La, rng)
+    Lb.set_weights(w)
+    X, Q, K, V = rand_tokens(La, rng, 12)
+    for L in (La, Lb):
+        L.prefill_chunk(0, X[:8], Q[:8], K[:8], V[:8])
+    for t in range(8, 12):
+        _, oa = La.prefill_chunk_out(0, X[t:t + 1], Q[t:t + 1], Q[t:t + 1], K[t:t + 1], V[t:t + 1])
+        _, ob = Lb.decode_step(0, X[t], Q[t], Q[t], K[t], V[t])
+        np.testing.assert_allclose(oa[0], ob, rtol=1e-13, atol=1e-14)
