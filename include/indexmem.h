@@ -60,6 +60,7 @@ typedef struct im_config {
   int32_t enable_memory;     /* 0: no memory write and no readout term         (Eq. 4 with g = 0)   */
   int32_t out_f32;           /* 0: `out` of im_decode_step is bf16; 1: float32                       */
   int32_t pending_slots;     /* rank-one writes folded lazily into M (0 => 16); see im_decode_step  */
+  int32_t chunk_outputs;     /* 1: reserve workspace for im_prefill_chunk_attend (max_seqs * max_chunk * D_kv floats) */
   float softmax_scale;       /* 0 => 1/sqrt(d)                                 (Sec. 2.1)           */
   float lambda;              /* decay of Eq. 6-7, (0,1]; 0 => 1                                      */
   float eta;                 /* write strength of Eq. 6-7, > 0; 0 => 1                               */
@@ -123,11 +124,28 @@ int im_reset(im_ctx* ctx, int layer, int seq, void* cuda_stream);
  * the importance of every cached entry, then compresses: if more than B entries are cached the B
  * best (importance descending, position ascending, sinks first) stay, the rest are written to the
  * latent memory (Eq. 6-7, one evict step) and the cache is compacted.  Attention outputs for the
- * chunk's own queries are not produced.
+ * chunk's own queries are not produced (see im_prefill_chunk_attend).
  * Errors: IM_ERR_ARG (bad ids, sizes, null pointers), IM_ERR_CAPACITY (n + C > capacity).
  */
 int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, int chunk_len,
                      const void* x, const void* q_pre, const void* k, const void* v, void* cuda_stream);
+
+/*
+ * im_prefill_chunk that also returns the layer outputs of the chunk's own queries (Eq. 4-5 during chunked
+ * prefill; the chunk is processed before it is compressed, Sec. 4 schedule).
+ *   q    dev bf16 [n_seq, C, H, d]  queries as the attention sees them (may alias q_pre)
+ *   out  dev [n_seq, C, H, d] bf16 (float32 when out_f32 = 1)
+ * Query s of the chunk attends to every entry cached when the call starts and to the chunk's tokens up to
+ * and including itself (Sec. 2.1, causal), and adds g(q_s) m(q_s) read from the memory as the evict steps of
+ * earlier calls left it (Eq. 5); the evict step of this chunk does not enter its own outputs.  The state
+ * after the call is the one im_prefill_chunk leaves.
+ * Needs chunk_outputs = 1 in the configuration (workspace) and head_dim 64 or 128 with at most 8 query heads
+ * per KV head; otherwise IM_ERR_ARG.  Other errors as for im_prefill_chunk; IM_ERR_TIMEOUT is reported through
+ * im_status if a bounded wait on a tile copy gave up.
+ */
+int im_prefill_chunk_attend(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, int chunk_len,
+                            const void* x, const void* q_pre, const void* q, const void* k, const void* v,
+                            void* out, void* cuda_stream);
 
 /*
  * One decode token per sequence for one layer (Sec. 4 schedule, decode side; Eq. 4-7).

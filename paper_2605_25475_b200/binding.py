@@ -34,7 +34,7 @@ WEIGHT_IDS = {"U_q": IM_W_UQ, "U_k": IM_W_UK, "G": IM_W_G, "W_theta": IM_W_THETA
 class im_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "max_seqs", "n_q_heads", "n_kv_heads", "head_dim", "n_index_heads", "index_dim", "mem_dim",
-        "budget", "compress_interval", "max_chunk", "n_sink", "act", "enable_memory", "out_f32", "pending_slots")] + \
+        "budget", "compress_interval", "max_chunk", "n_sink", "act", "enable_memory", "out_f32", "pending_slots", "chunk_outputs")] + \
         [(n, C.c_float) for n in ("softmax_scale", "lambda_", "eta", "eps", "norm_eps", "init_std")] + \
         [("seed", C.c_uint64)]
 
@@ -52,6 +52,7 @@ _lib.im_create.argtypes = [C.POINTER(im_config), _vp, _sz, C.POINTER(_vp)]
 _lib.im_destroy.argtypes = [_vp]
 _lib.im_reset.argtypes = [_vp, _i32, _i32, _vp]
 _lib.im_prefill_chunk.argtypes = [_vp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
+_lib.im_prefill_chunk_attend.argtypes = [_vp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.im_decode_step.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.im_set_weights.argtypes = [_vp, _i32, _i32, _vp, _sz]
 _lib.im_get_weights.argtypes = [_vp, _i32, _i32, _vp, _sz]
@@ -71,7 +72,7 @@ _lib.im_last_error.restype = C.c_char_p
 
 EXPORTED = ("im_workspace_bytes", "im_create", "im_destroy", "im_reset", "im_prefill_chunk", "im_decode_step",
             "im_set_weights", "im_get_weights", "im_state_export", "im_state_import", "im_topb_select",
-            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc", "im_event_count")
+            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc", "im_event_count", "im_prefill_chunk_attend")
 
 
 def _check(rc: int):
@@ -118,6 +119,13 @@ def im_prefill_chunk(ctx, layer, seq_ids, chunk_len, x, q_pre, k, v):
     ids = _ids(seq_ids)
     _check(_lib.im_prefill_chunk(ctx, layer, ids.size, ids.ctypes.data, chunk_len, x.data_ptr(), q_pre.data_ptr(),
                                  k.data_ptr(), v.data_ptr(), _stream()))
+
+
+def im_prefill_chunk_attend(ctx, layer, seq_ids, chunk_len, x, q_pre, q, k, v, out):
+    ids = _ids(seq_ids)
+    _check(_lib.im_prefill_chunk_attend(ctx, layer, ids.size, ids.ctypes.data, chunk_len, x.data_ptr(),
+                                        q_pre.data_ptr(), q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                        _stream()))
 
 
 def im_decode_step(ctx, layer, seq_ids, x, q_pre, q, k_new, v_new, out):
@@ -235,6 +243,7 @@ class Config:
     enable_memory: int = 1
     out_f32: int = 0
     pending_slots: int = 0
+    chunk_outputs: int = 0
     softmax_scale: float = 0.0
     lambda_: float = 0.0
     eta: float = 0.0
@@ -298,6 +307,18 @@ class IndexMem:
         _dev(x, bf, n * Cn * self.D, "x"); _dev(q_pre, bf, n * Cn * self.D, "q_pre")
         _dev(k, bf, n * Cn * self.Dkv, "k"); _dev(v, bf, n * Cn * self.Dkv, "v")
         im_prefill_chunk(self.ctx, layer, seq_ids, Cn, x, q_pre, k, v)
+
+    def prefill_chunk_attend(self, layer, seq_ids, x, q_pre, q, k, v, out=None):
+        """prefill_chunk that also returns the layer outputs [n, C, H, d] of the chunk's own queries."""
+        n, Cn = len(seq_ids), x.shape[-2]
+        bf = torch.bfloat16
+        _dev(x, bf, n * Cn * self.D, "x"); _dev(q_pre, bf, n * Cn * self.D, "q_pre"); _dev(q, bf, n * Cn * self.D, "q")
+        _dev(k, bf, n * Cn * self.Dkv, "k"); _dev(v, bf, n * Cn * self.Dkv, "v")
+        if out is None:
+            out = torch.empty((n, Cn, self.H, self.d), dtype=self.out_dtype, device=x.device)
+        _dev(out, self.out_dtype, n * Cn * self.D, "out")
+        im_prefill_chunk_attend(self.ctx, layer, seq_ids, Cn, x, q_pre, q, k, v, out)
+        return out
 
     def decode_step(self, layer, seq_ids, x, q_pre, q, k_new, v_new, out=None):
         n = len(seq_ids)

@@ -83,6 +83,7 @@ bool resolve(const im_config* in, im_config* c, ImDims* p) {
   q.B = c->budget; q.tau = c->compress_interval; q.cap = (int)cap; q.tail = q.cap - q.B;
   q.n_sink = c->n_sink; q.act = c->act; q.mem = c->enable_memory ? 1 : 0; q.F = c->pending_slots;
   q.out_f32 = c->out_f32 ? 1 : 0; q.max_chunk = std::max(c->max_chunk, 1);
+  q.chunk_out = c->chunk_outputs ? 1 : 0;
   q.R3 = q.HI * q.dI + q.dI + q.HI;
   q.R5 = q.R3 + q.dM + 1;
   q.max_splits = (q.cap + 255) / 256;
@@ -150,6 +151,8 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->sc.phiq = (float*)take((size_t)p.S * p.dM * 4);
   lo->sc.n_att = (int32_t*)take((size_t)p.S * 4);
   lo->sc.rpart = (float*)take((size_t)p.S * ((p.dM + IM_READOUT_ROWS - 1) / IM_READOUT_ROWS) * p.Dkv * 4);
+  lo->sc.mch = nullptr;
+  if (p.chunk_out) lo->sc.mch = (float*)take((size_t)p.S * p.max_chunk * p.Dkv * 4);
   lo->sc.qpack = nullptr;
   if (im_score_tc_supported(p))
     lo->sc.qpack = (uint8_t*)take((size_t)p.S * ((p.max_chunk + IM_TC_QT - 1) / IM_TC_QT) * IM_TC_TILE_BYTES);
@@ -221,6 +224,7 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
   call->C = 1;
   call->pack = 0;
   call->defer = 0;
+  call->fold_all = 0;
   return IM_OK;
 }
 
@@ -330,6 +334,7 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
     if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK, ctx->mapV);
     if (e == cudaSuccess) e = im_attn_prepare(p);
+    if (e == cudaSuccess) e = im_chunk_attn_prepare(p);
     ctx->n_ctas = std::max(1, std::min(sms, IM_ATTN_MAX_CTAS));
     ctx->fast_attn = (e == cudaSuccess);
   }
@@ -400,8 +405,10 @@ int im_reset(im_ctx* ctx, int layer, int seq, void* cuda_stream) {
   return IM_OK;
 }
 
-int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, int chunk_len, const void* x,
-                     const void* q_pre, const void* k, const void* v, void* cuda_stream) {
+// im_prefill_chunk (q = out = null) and im_prefill_chunk_attend
+static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, int chunk_len, const void* x,
+                        const void* q_pre, const void* q, const void* k, const void* v, void* out, bool attend,
+                        void* cuda_stream) {
   ImCall call;
   int rc = check_call(ctx, layer, n_seq, seq_ids, &call);
   if (rc) return rc;
@@ -409,6 +416,12 @@ int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, 
   if (chunk_len < 1 || chunk_len > p.max_chunk)
     return fail(IM_ERR_ARG, "chunk_len %d out of range [1,%d]", chunk_len, p.max_chunk);
   if (!x || !q_pre || !k || !v) return fail(IM_ERR_ARG, "null tensor");
+  if (attend) {
+    if (!q || !out) return fail(IM_ERR_ARG, "null tensor");
+    if (!p.chunk_out) return fail(IM_ERR_ARG, "im_prefill_chunk_attend needs chunk_outputs = 1 in the configuration");
+    if (!ctx->fast_attn)
+      return fail(IM_ERR_ARG, "im_prefill_chunk_attend needs head_dim 64 or 128 and at most 8 query heads per KV head");
+  }
   int n_max = 0, ne_max = 0;
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
@@ -423,10 +436,11 @@ int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, 
   call.ksplit_key = 1;
   call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
   call.pack = ctx->score_tc ? 1 : 0;
+  call.fold_all = attend && p.mem ? 1 : 0;
   ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
   const int NV = n_seq * chunk_len;
   // pending rank-one terms are folded into M before a compression that cannot append to the list
-  if (p.mem && ne_max > 0) CKL(im_launch_mem_fold(L, call));
+  if (p.mem && (ne_max > 0 || attend)) CKL(im_launch_mem_fold(L, call));
   // a0: indexer projections of every chunk token (Sec. 3.1)
   ImRows r = im_rows(p);
   ImGemmArgs g;
@@ -446,6 +460,30 @@ int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, 
   CKL(im_launch_gemm(L, g));
   CKL(im_launch_proj_key_split(L, x, NV, 1));
   CKL(im_launch_prefill_append(L, call, k, v));
+  if (attend) {
+    // layer outputs of the chunk's own queries, before the chunk is compressed: phi(q) and the gate logit of
+    // every chunk token (behind the indexer-side block of the projection scratch), Eq. 5 over the memory of
+    // before this chunk, then attention over (cached entries + causal chunk) with the readout added (Eq. 4)
+    if (p.mem) {
+      ImGemmArgs g2;
+      memset(&g2, 0, sizeof(g2));
+      g2.job[0] = {L.w.Wt, nullptr, p.dM, 0, 0};
+      g2.job[1] = {L.w.wg, nullptr, 1, p.dM, 0};
+      g2.n_jobs = 2;
+      g2.in[0] = (const bf16*)q;
+      g2.in_cnt[0] = 1;
+      g2.in_outer[0] = p.D;
+      g2.out = L.sc.raw + (size_t)p.S * p.max_chunk * p.R3;
+      g2.out_cnt = 1;
+      g2.out_outer = p.dM + 1;
+      g2.NV = NV;
+      g2.K = p.D;
+      g2.ksplit = 1;
+      CKL(im_launch_gemm(L, g2));
+      CKL(im_launch_chunk_readout(L, call));
+    }
+    CKL(im_launch_chunk_attention(L, call, ctx->mapK, ctx->mapV, q, out));
+  }
   // a1: pooled importance under the causal mask
   {
     const bool prof = ctx->prof_target == 1 && ctx->prof_used + 2 <= ctx->prof_ev.size();
@@ -468,12 +506,24 @@ int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, 
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
     const int ne = std::max(0, u.n + chunk_len - p.B);
+    if (call.fold_all) u.npend = 0;
     mirror_memory(p, u, ne);
     u.n = u.n + chunk_len - ne;
     u.T += chunk_len;
     u.since = 0;
   }
   return IM_OK;
+}
+
+int im_prefill_chunk(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, int chunk_len, const void* x,
+                     const void* q_pre, const void* k, const void* v, void* cuda_stream) {
+  return prefill_impl(ctx, layer, n_seq, seq_ids, chunk_len, x, q_pre, nullptr, k, v, nullptr, false, cuda_stream);
+}
+
+int im_prefill_chunk_attend(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, int chunk_len, const void* x,
+                            const void* q_pre, const void* q, const void* k, const void* v, void* out,
+                            void* cuda_stream) {
+  return prefill_impl(ctx, layer, n_seq, seq_ids, chunk_len, x, q_pre, q, k, v, out, true, cuda_stream);
 }
 
 int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, const void* x, const void* q_pre,

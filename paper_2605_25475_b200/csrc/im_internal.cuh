@@ -32,7 +32,7 @@ struct ImDims {
   int H, Hkv, d, D, Dkv, Gq;  // attention shape
   int HI, dI, dM;             // indexer / memory widths
   int B, tau, cap, tail;      // budget, interval, slots per sequence, tail = cap - B
-  int n_sink, act, mem, F, out_f32, max_chunk;
+  int n_sink, act, mem, F, out_f32, max_chunk, chunk_out;
   int R3, R5;                 // projection rows: indexer only / indexer + memory
   int max_splits;             // attention splits per (sequence, KV head)
   float scale, lambda, eta, eps, norm_eps;
@@ -104,6 +104,7 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
                      // the call's memory write (the merge adds the write's terms); otherwise the final m(q), gate, -
   float* phiq;       // [max_seqs][dM] phi(q) of the call (K-split partials summed)
   int32_t* n_att;    // [max_seqs] entries per sequence the streaming attention kernel of the call ran over
+  float* mch;        // [max_seqs][max_chunk][Dkv] gated memory readout of a chunk's own queries (im_prefill_chunk_attend)
   uint8_t* qpack;    // [n_seq][ceil(C / IM_TC_QT)][IM_TC_TILE_BYTES] query operand of the tensor-core prefill scoring
 };
 
@@ -113,6 +114,7 @@ struct ImCall {
   int defer;      // decode: 1 = the attention kernel runs over the entries cached before the call while the front
                   // kernel appends / scores / selects; the merge adds the new token and takes the evicted entries
                   // out again, and the holes are filled (and CTR_N advanced) by the call's last kernel
+  int fold_all;   // prefill with outputs: fold the pending list of every sequence first (the chunk readout reads Mhat alone)
   int pack;       // prefill: 1 = the append kernel also writes the operand records of the tensor-core scoring
   int phi_large;  // 1: phi of the evicted keys lives in ImScratch::phi, 0: in the K-split partials phip
   int ksplit, ksplit_key, ksplit_phi;  // K splits of the projections / key projection / phi partials of this call
@@ -176,6 +178,11 @@ bool im_score_tc_supported(const ImDims& p);
 cudaError_t im_score_tc_prepare();
 cudaError_t im_launch_prefill_score_tc(const ImLaunch& L, const ImCall& call, int n_max, int n_sm);
 cudaError_t im_launch_prefill_commit(const ImLaunch& L, const ImCall& call);
+// layer outputs of a prefill chunk's own queries
+cudaError_t im_chunk_attn_prepare(const ImDims& p);
+cudaError_t im_launch_chunk_readout(const ImLaunch& L, const ImCall& call);
+cudaError_t im_launch_chunk_attention(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
+                                      const void* q, void* out);
 cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const void* q, void* out, int n_max);
 bool im_attn_fast_supported(const ImDims& p);

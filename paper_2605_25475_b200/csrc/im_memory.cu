@@ -20,6 +20,7 @@ namespace {
 // does the coming compression of this sequence need the pending list folded first?
 __device__ __forceinline__ bool fold_needed(const ImDims& p, const ImCall& call, const int32_t* ctr, float cscale) {
   if (!p.mem) return false;
+  if (call.fold_all) return ctr[CTR_NPEND] > 0 || cscale != 1.0f;
   const int ne = im_upcoming_evictions(p, call.prefill, call.C, ctr[CTR_N], ctr[CTR_SINCE]);
   const int np = ctr[CTR_NPEND];
   if (ne <= 0) return false;

@@ -77,6 +77,22 @@ class Pair:
             self.check_selection()
             self.check_state()
 
+    def prefill_attend(self, chunk_idx: int, check=True):
+        """The chunk through im_prefill_chunk_attend: state checks as for prefill(), plus the layer outputs of
+        the chunk's own queries against the oracle (same bound as the decode outputs, row by row)."""
+        wl = self.wl
+        X, Q, K, V = synth.prefill_inputs(wl, self.layer, chunk_idx)
+        ob, od = self.o.prefill_batch_out(self.seq_ids, synth.f32(X), synth.f32(Q), synth.f32(Q), synth.f32(K), synth.f32(V))
+        dev = self.device
+        out = self.g.prefill_chunk_attend(0, self.seq_ids, X.to(dev), Q.to(dev), Q.to(dev), K.to(dev), V.to(dev))
+        assert self.g.status() == 0
+        if check:
+            self.check_selection()
+            self.check_state()
+            n, Cn = od.shape[0], od.shape[1]
+            self.check_out(out.reshape(n * Cn, wl.H, wl.d), ob.reshape(n * Cn, wl.H, wl.d), od.reshape(n * Cn, wl.H, wl.d))
+        return out, ob, od
+
     def decode(self, step: int, check=True):
         wl = self.wl
         x, q, k, v = synth.decode_inputs(wl, self.layer, step)

@@ -320,3 +320,52 @@ def test_decode_from_an_empty_cache(im):
     for s in range(wl.steps):
         p.decode(s)
     assert p.stats["max_out_err"] <= 2e-3
+
+
+# ------------------------------------------------------------------ layer outputs of a prefill chunk's own queries
+def test_chunk_outputs_llama_shape_several_chunks(im):
+    """32 q / 8 KV heads, d 128: four ragged chunks of 200 tokens into a budget of 256, two sequences; from the
+    second chunk on the queries see a retained prefix (holes filled in arbitrary slot order) plus the causal
+    chunk and read a non-empty memory; then decode steps continue from the same state."""
+    wl = synth.CONFIGS["llama8b_b1"].replace(name="chunk_out", n_seq=2, ctx=4 * 200, chunk=200, B=256, steps=3, n_needles=4)
+    p = _pair(wl, chunk_outputs=1)
+    for c in range(4):
+        p.prefill_attend(c)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
+
+
+def test_chunk_outputs_qwen_shape_and_pending_list(im):
+    """28 q / 4 KV heads (7 heads per KV head: 18 queries x 7 heads = 126 of a block's 128 rows), d_M 448;
+    decode steps in between leave rank-one writes pending, which the call folds before it reads the memory;
+    float32 outputs."""
+    wl = synth.CONFIGS["qwen7b_b8"].replace(name="chunk_out_q", n_seq=2, ctx=3 * 150, chunk=150, B=180, steps=5, n_needles=0)
+    p = _pair(wl, chunk_outputs=1, out_f32=1)
+    p.prefill_attend(0)
+    p.prefill_attend(1)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.g.counts(0, 0)["n_pending"] > 0
+    p.prefill_attend(2)
+    assert p.stats["max_out_err"] <= 1e-4
+
+
+def test_chunk_outputs_tiny_shape_no_memory_and_single_token_chunks(im):
+    wl = TINY.replace(name="chunk_out_t", ctx=3 * 70, chunk=70, B=90, steps=2, n_needles=0)
+    p = _pair(wl, chunk_outputs=1, enable_memory=0)
+    for c in range(3):
+        p.prefill_attend(c)
+    wl1 = TINY.replace(name="chunk_out_1", ctx=40, chunk=1, B=24, steps=1, n_needles=0)
+    p1 = _pair(wl1, chunk_outputs=1)
+    for c in range(40):
+        p1.prefill_attend(c)
+    assert p1.stats["max_out_err"] <= 2e-3
+
+
+def test_chunk_outputs_need_their_workspace(im):
+    wl = TINY.replace(name="chunk_out_e", ctx=32, chunk=32, B=64, steps=1)
+    p = _pair(wl)
+    X, Q, K, V = synth.prefill_inputs(wl, 0, 0)
+    with pytest.raises(im.IndexMemError):
+        p.g.prefill_chunk_attend(0, [0], X.cuda(), Q.cuda(), Q.cuda(), K.cuda(), V.cuda())
