@@ -264,6 +264,7 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
   g.K = p.Dkv;
   g.out_cnt = ne_max;
   g.out_inner = p.dM;
+  g.tensor = call.prefill ? 1 : 0;
   if (ne_max > p.F) {
     call.phi_large = 1;
     g.out = L.sc.phi;
@@ -457,6 +458,7 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   g.NV = NV;
   g.K = p.D;
   g.ksplit = 1;
+  g.tensor = 1;
   CKL(im_launch_gemm(L, g));
   CKL(im_launch_proj_key_split(L, x, NV, 1));
   CKL(im_launch_prefill_append(L, call, k, v));
@@ -479,6 +481,7 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
       g2.NV = NV;
       g2.K = p.D;
       g2.ksplit = 1;
+      g2.tensor = 1;
       CKL(im_launch_gemm(L, g2));
       CKL(im_launch_chunk_readout(L, call));
     }

@@ -286,6 +286,7 @@ cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
     attr_done = true;
   }
   ImGemmArgs a = a_in;
+  if (a.tensor && im_tc_gemm_usable(a)) return im_launch_tc_gemm(L, a);
   int n_w2 = 0;
   for (int j = 0; j < a.n_jobs; ++j) n_w2 += a.job[j].W2 != nullptr;
   if (a.direct && a.ksplit > 0 && a.K % a.ksplit == 0 && (a.K / a.ksplit) % 32 == 0 && a.NV > 0 &&

@@ -140,6 +140,7 @@ struct ImGemmArgs {
   int out_cnt;
   int NV, K, ksplit;
   int kc;      // K elements staged per round (0: the maximum, 512); small values keep the shared-memory footprint low
+  int tensor;  // 1: thousands of vectors (prefill) - the tcgen05 variant where it applies (im_tc_gemm_usable)
   int direct;  // 1: few vectors (decode) - the variant without shared-memory staging, if the K split is a multiple of 32
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
 };
@@ -164,6 +165,9 @@ int im_fail_message(int code, const char* msg);
 
 // ---- kernels' host launchers (each returns the cudaError of the launch)
 cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a);
+// tensor-core (tcgen05) variant for thousands of vectors and one K split (prefill)
+bool im_tc_gemm_usable(const ImGemmArgs& a);
+cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a);
 cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, int ksplit);
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
                                    int do_select, int n_max);
