@@ -151,6 +151,13 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->sc.phiq = (float*)take((size_t)p.S * p.dM * 4);
   lo->sc.n_att = (int32_t*)take((size_t)p.S * 4);
   lo->sc.rpart = (float*)take((size_t)p.S * ((p.dM + IM_READOUT_ROWS - 1) / IM_READOUT_ROWS) * p.Dkv * 4);
+  lo->sc.phiT = nullptr;
+  lo->sc.vT = nullptr;
+  if (p.tail > p.F) {
+    const size_t KE = ((size_t)p.tail + 63) / 64 * 64;
+    lo->sc.phiT = (bf16*)take(2 * (size_t)p.dM * KE * 2);
+    lo->sc.vT = (bf16*)take((size_t)p.Dkv * KE * 2);
+  }
   lo->sc.mch = nullptr;
   if (p.chunk_out) lo->sc.mch = (float*)take((size_t)p.S * p.max_chunk * p.Dkv * 4);
   lo->sc.qpack = nullptr;
@@ -248,6 +255,19 @@ void mirror_memory(const ImDims& p, HostUnit& u, int ne) {
   u.npend += ne;
 }
 
+// the state update of Eq. 6-7 with the per-sequence evicted counts of this call from the host mirror (must be
+// called before the mirror is advanced)
+cudaError_t launch_mem_update(im_ctx* ctx, const ImLaunch& L, const ImCall& call, int ne_max) {
+  const ImDims& p = ctx->p;
+  int ne_host[IM_MAX_CALL_SEQS];
+  for (int i = 0; i < call.n_seq; ++i) {
+    const HostUnit& u = ctx->hu[(size_t)call.layer * p.S + call.seq[i]];
+    const bool due = call.prefill || (u.since + 1 == p.tau);
+    ne_host[i] = due ? std::max(0, u.n + call.C - p.B) : 0;
+  }
+  return im_launch_mem_update(L, call, ne_max, ne_host);
+}
+
 // phi of the gathered evicted keys (skinny GEMM against the folded Linear_theta), then Eq. 6-7.
 // With `update` = false only the GEMM is launched (the caller launches im_launch_mem_update later).
 int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, bool update = true) {
@@ -281,7 +301,7 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
     g.direct = call.prefill ? 0 : 1;
   }
   CKL(im_launch_gemm(L, g));
-  if (update) CKL(im_launch_mem_update(L, call, ne_max));
+  if (update) CKL(launch_mem_update(ctx, L, call, ne_max));
   return IM_OK;
 }
 
@@ -674,7 +694,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[4], 0));  // s2 joins here
   if (defer && p.mem) CKL(im_launch_readout_apply(L1, call));
   if (conc) CK(cudaEventRecord(ctx->ev[3], L1.stream));  // everything the merge needs from s1
-  if (defer && mem_write) CKL(im_launch_mem_update(L1, call, ne_max));
+  if (defer && mem_write) CKL(launch_mem_update(ctx, L1, call, ne_max));
   if (mem_write && ctx->fast_attn && !readout_early) CKL(im_launch_readout(L1, call));
   int n_att = 0;
   for (int i = 0; i < n_seq; ++i) {

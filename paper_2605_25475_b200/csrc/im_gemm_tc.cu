@@ -98,6 +98,26 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 #pragma unroll
   for (int k = 0; k < 32; ++k) v[k] = __uint_as_float(r[k]);
 }
+// epilogue of one thread: 32 consecutive weight rows (c0 ..) of vector v
+__device__ __forceinline__ void store_columns(const ImGemmArgs& a, const ImGemmJob& job, int r0, int n_rows, int c0,
+                                              long long v, const float* acc) {
+  if (v >= a.NV) return;
+  if (a.gate && *a.gate <= a.gate_min) return;
+  if (a.out_t) {
+    float* o = a.out + (size_t)(job.row0 + r0 + c0) * a.out_outer + v;
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+      if (c0 + c < n_rows) {
+        float* q = o + (size_t)c * a.out_outer;
+        *q = a.rmw ? fmaf(a.beta, *q, a.alpha * acc[c]) : acc[c];
+      }
+  } else {
+    float* o = a.out + (v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0 + c0;
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+      if (c0 + c < n_rows) o[c] = a.rmw ? fmaf(a.beta, o[c], a.alpha * acc[c]) : acc[c];
+  }
+}
 __device__ __forceinline__ const bf16* vec_ptr(const ImGemmArgs& a, int sel, long long v) {
   return a.in[sel] + (v / a.in_cnt[sel]) * a.in_outer[sel] + (v % a.in_cnt[sel]) * a.in_inner[sel];
 }
@@ -190,15 +210,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_tc_gemm(ImGemmArgs a, int32_t*
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const long long v = v0 + warp * 32 + lane;
-      float* o = a.out + (v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0;
       for (int c0 = 0; c0 < n_cols; c0 += 32) {
         float acc[32];
         tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc);
-        if (v < a.NV) {
-#pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (c0 + c < n_rows) o[c0 + c] = acc[c];
-        }
+        store_columns(a, job, r0, n_rows, c0, v, acc);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
@@ -337,15 +352,10 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const long long v = v0 + qd * 32 + lane;
-      float* o = a.out + (v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0;
       for (int c0 = 0; c0 < n_cols; c0 += 32) {
         float acc[32];
         tmem_ld32(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)c0, acc);
-        if (v < a.NV) {
-#pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (c0 + c < n_rows) o[c0 + c] = acc[c];
-        }
+        store_columns(a, job, r0, n_rows, c0, v, acc);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }

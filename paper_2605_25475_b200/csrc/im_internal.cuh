@@ -104,6 +104,8 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
                      // the call's memory write (the merge adds the write's terms); otherwise the final m(q), gate, -
   float* phiq;       // [max_seqs][dM] phi(q) of the call (K-split partials summed)
   int32_t* n_att;    // [max_seqs] entries per sequence the streaming attention kernel of the call ran over
+  bf16* phiT;        // [2][dM][KE] phi of one sequence's evicted keys, transposed, as two bf16 terms (KE = tail rounded up to 64)
+  bf16* vT;          // [Dkv][KE] that sequence's evicted values, transposed
   float* mch;        // [max_seqs][max_chunk][Dkv] gated memory readout of a chunk's own queries (im_prefill_chunk_attend)
   uint8_t* qpack;    // [n_seq][ceil(C / IM_TC_QT)][IM_TC_TILE_BYTES] query operand of the tensor-core prefill scoring
 };
@@ -143,6 +145,12 @@ struct ImGemmArgs {
   int tensor;  // 1: thousands of vectors (prefill) - the tcgen05 variant where it applies (im_tc_gemm_usable)
   int direct;  // 1: few vectors (decode) - the variant without shared-memory staging, if the K split is a multiple of 32
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
+  // tensor-core variant only:
+  int out_t;            // 1: the result goes to out[(row0 + r) * out_outer + v] (vectors contiguous) instead
+  int rmw;              // 1: out = beta * out + alpha * result
+  float alpha, beta;
+  const int32_t* gate;  // if set, nothing is stored unless *gate > gate_min (a device-side counter decides)
+  int gate_min;
 };
 
 #define IM_NOALLOC_MAX_FLOATS (1u << 20) /* floats in the built-in scratch array of im_attention_noalloc (4 MiB) */
@@ -174,7 +182,8 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call);
-cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_max);
+// ne_host: per call sequence, the number of entries the compression of this call evicts (host mirror)
+cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_max, const int* ne_host);
 cudaError_t im_launch_prefill_append(const ImLaunch& L, const ImCall& call, const void* k, const void* v);
 cudaError_t im_launch_prefill_score(const ImLaunch& L, const ImCall& call, int n_max);
 // tensor-core (tcgen05) version of the prefill scoring; needs ImCall::pack set for the append kernel

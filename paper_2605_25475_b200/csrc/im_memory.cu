@@ -210,6 +210,65 @@ __global__ void __launch_bounds__(256) k_mem_accumulate(ImDims p, ImState st, Im
     }
 }
 
+// ---- large evicted sets on the tensor cores: Mhat <- lambda Mhat + eta Phi^T V as a GEMM over the evicted
+// entries.  The GEMM kernels want both operands K-major (K = evicted entry), so phi (float32, [e][m]) and the
+// evicted values ([e][col]) of one sequence are transposed first; phi becomes two bf16 terms (hi + lo
+// reproduces the float32 value to 2^-17).  Entries at or beyond the sequence's evicted count are zero.
+// grid = (KE / 32, (dM + Dkv) / 32), block = (32, 8).
+__global__ void __launch_bounds__(256) k_mem_pack(ImDims p, ImState st, ImScratch sc, ImCall call, int i, int KE) {
+  __shared__ float tile[32][33];
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
+  const int e0 = blockIdx.x * 32, tx = threadIdx.x, ty = threadIdx.y;
+  const int mt = (p.dM + 31) / 32;
+  const bool is_phi = (int)blockIdx.y < mt;
+  const int c0 = (is_phi ? blockIdx.y : blockIdx.y - mt) * 32;
+  const int width = is_phi ? p.dM : p.Dkv;
+  for (int r = ty; r < 32; r += 8) {  // rows = entries, threads along the contiguous column index
+    const int e = e0 + r, c = c0 + tx;
+    float v = 0.f;
+    if (e < ne && c < width)
+      v = is_phi ? sc.phi[((size_t)i * p.tail + e) * p.dM + c] : __bfloat162float(sc.evV[((size_t)i * p.tail + e) * p.Dkv + c]);
+    tile[r][tx] = v;
+  }
+  __syncthreads();
+  for (int r = ty; r < 32; r += 8) {  // rows = columns of the source, threads along the entries
+    const int c = c0 + r, e = e0 + tx;
+    if (c >= width || e >= KE) continue;
+    const float v = tile[tx][r];
+    const bf16 hi = __float2bfloat16_rn(v);
+    if (is_phi) {
+      sc.phiT[(size_t)c * KE + e] = hi;
+      sc.phiT[((size_t)p.dM + c) * KE + e] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    } else {
+      sc.vT[(size_t)c * KE + e] = hi;
+    }
+  }
+}
+
+// b <- lambda b + eta sum_e phi_e^2 (Eq. 7) for the sequences whose evicted set is larger than the pending list.
+// grid = (ceil(dM / 32), n_seq), block = (32, 8): eight partial sums per row, added in a fixed order.
+__global__ void __launch_bounds__(256) k_mem_bsum(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  __shared__ float part[8][32];
+  const int i = blockIdx.y;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
+  if (ne <= p.F) return;
+  const int m = blockIdx.x * 32 + threadIdx.x;
+  float s = 0.f;
+  if (m < p.dM)
+    for (int e = threadIdx.y; e < ne; e += 8) {
+      const float f = sc.phi[((size_t)i * p.tail + e) * p.dM + m];
+      s = fmaf(f, f, s);
+    }
+  part[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && m < p.dM) {
+    for (int k = 1; k < 8; ++k) s += part[k][threadIdx.x];
+    st.bvec[u * p.dM + m] = p.lambda * st.bvec[u * p.dM + m] + p.eta * s;
+  }
+}
+
 }  // namespace
 
 cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call) {
@@ -225,12 +284,50 @@ cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call) {
 }
 
 // after phi of the evicted keys is available (ImCall::phi_large says where)
-cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_max) {
+cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_max, const int* ne_host) {
   const ImDims& p = L.p;
   k_mem_small<<<call.n_seq, 256, 0, L.stream>>>(p, L.st, L.sc, call);
   ++*L.launches;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || ne_max <= p.F) return e;
+  // evicted sets larger than the pending list: Phi^T V on the tensor cores, one sequence at a time
+  const int KE = (ne_max + 63) / 64 * 64;
+  ImGemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.tensor = 1;
+  g.NV = p.Dkv;  // the GEMM's "vectors" are the columns of Mhat (rows of V^T), its "weight rows" the rows of Phi^T
+  g.K = KE;
+  g.ksplit = 1;
+  g.in[0] = L.sc.vT;
+  g.in_cnt[0] = 1;
+  g.in_outer[0] = KE;
+  g.job[0] = {L.sc.phiT, L.sc.phiT ? L.sc.phiT + (size_t)p.dM * KE : nullptr, p.dM, 0, 0};
+  g.n_jobs = 1;
+  g.out_t = 1;
+  g.out_outer = p.Dkv;
+  g.out_cnt = 1;
+  g.rmw = 1;
+  g.alpha = p.eta;
+  g.beta = p.lambda;
+  g.gate_min = p.F;
+  if (L.sc.phiT && call.phi_large && ne_host && im_tc_gemm_usable(g)) {
+    dim3 gb((p.dM + 31) / 32, call.n_seq);
+    k_mem_bsum<<<gb, dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call);
+    ++*L.launches;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    for (int i = 0; i < call.n_seq; ++i) {
+      if (ne_host[i] <= p.F) continue;
+      const size_t u = (size_t)call.layer * p.S + call.seq[i];
+      dim3 gp(KE / 32, (p.dM + 31) / 32 + (p.Dkv + 31) / 32);
+      k_mem_pack<<<gp, dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call, i, KE);
+      ++*L.launches;
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      g.out = L.st.Mhat + u * p.dM * p.Dkv;
+      g.gate = L.st.ctr + u * CTR_STRIDE + CTR_NEVICT;
+      if ((e = im_launch_tc_gemm(L, g)) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+  }
   dim3 grid((p.Dkv + 63) / 64, (p.dM + 63) / 64, call.n_seq);
   k_mem_accumulate<<<grid, 256, 0, L.stream>>>(p, L.st, L.sc, call);
   ++*L.launches;
