@@ -96,11 +96,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
-struct RowMap {        // tile bookkeeping shared by the attention and merge kernels
-  long long q;         // tiles per warp run
-  long long total;     // total tiles
-};
-
 // tiles of sequence i (all KV heads have the same count)
 __device__ __forceinline__ int tiles_of(int n) { return (n + TILE - 1) / TILE; }
 

@@ -6,12 +6,6 @@ namespace {
 
 constexpr float NEG_INF = -__builtin_huge_valf();
 
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
 // RMSNorm of one token's raw q features per indexer head, in place, and alpha = G x / sqrt(H_I d_I)
 // (Sec. 3.1).  Executed by one warp; lanes stride over heads.
 __device__ void finalize_features(const ImDims& p, float* raw, int lane) {
