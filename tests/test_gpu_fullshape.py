@@ -104,3 +104,37 @@ def test_stack_shape_sampled_units_under_graph_replay():
             assert len(set(pos.tolist())) == wl.B and set(range(wl.n_sink)) <= set(pos.tolist())
             assert pos.max() < wl.ctx + n_steps
     assert np.isfinite(results[-1]).all()
+
+
+def test_llama8b_b1_configuration_at_full_size():
+    """The Llama-3-8B-shaped single-sequence configuration as stated: 32 q / 8 KV heads, d 128, a 4096-token
+    context ingested in one chunk (3584 evictions in one evict step: the tensor-core scoring, selection,
+    phi and Phi^T V kernels at their full sizes), budget 512, lognormal key norms, 256 decode steps; every
+    state and every output checked against the oracle."""
+    from tests.parity import Pair
+    wl = synth.CONFIGS["llama8b_b1"]
+    p = Pair(wl)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    st = p.stats
+    assert st["steps"] == 256 and st["kidx_flips"] == 0
+    assert st["max_out_err"] <= 2e-3 and st["max_M_err"] <= 2e-3 and st["max_score_err"] <= 1e-5
+    assert st["cut_divergences"] <= 4
+
+
+def test_mistral_prefill_chunks_at_full_chunk_size():
+    """The Mistral-shaped chunked prefill at its stated chunk size and budget (2048 / 2048), prompt cut to three
+    chunks so that the oracle finishes in half a minute: the second and third chunk score 4096 cached keys
+    against 2048 queries (tcgen05 scoring GEMM at its benchmark size), evict 2048 entries each and write
+    them to the memory through the tensor-core GEMMs; selection, cached keys and memory against the oracle."""
+    from tests.parity import Pair
+    wl = synth.CONFIGS["mistral7b_prefill"].replace(name="mistral_full_chunk", ctx=3 * 2048, steps=2)
+    p = Pair(wl)
+    for c in range(3):
+        p.prefill(c)
+    assert p.o.evict_steps(0) == 2 and p.g.counts(0, 0)["n"] == 2048
+    for s in range(wl.steps):
+        p.decode(s)
+    st = p.stats
+    assert st["kidx_flips"] == 0 and st["max_M_err"] <= 2e-3 and st["max_score_err"] <= 1e-5 and st["max_out_err"] <= 2e-3
