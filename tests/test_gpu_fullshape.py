@@ -138,3 +138,19 @@ def test_mistral_prefill_chunks_at_full_chunk_size():
         p.decode(s)
     st = p.stats
     assert st["kidx_flips"] == 0 and st["max_M_err"] <= 2e-3 and st["max_score_err"] <= 1e-5 and st["max_out_err"] <= 2e-3
+
+
+def test_qwen_shape_one_shot_compression_of_a_long_context():
+    """Qwen2.5-7B shape (28 q / 4 KV heads, 7 indexer heads, d_M 448) with the one-shot compression of the
+    stated configuration at half its context (8192 tokens -> B = 1024 in a single evict step of 7168 entries,
+    two of the eight sequences, 64 needles each; the oracle needs about a minute for the full 16384), then
+    decode steps."""
+    from tests.parity import Pair
+    wl = synth.CONFIGS["qwen7b_b8"].replace(name="qwen_oneshot", n_seq=2, ctx=8192, chunk=8192, steps=8)
+    p = Pair(wl)
+    p.prefill(0)
+    assert p.g.counts(0, 1)["n"] == 1024 and p.g.counts(0, 1)["n_evicted"] == 7168
+    for s in range(wl.steps):
+        p.decode(s)
+    st = p.stats
+    assert st["kidx_flips"] == 0 and st["max_M_err"] <= 2e-3 and st["max_score_err"] <= 1e-5 and st["max_out_err"] <= 2e-3
