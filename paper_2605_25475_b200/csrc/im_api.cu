@@ -368,8 +368,12 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     // the short side kernels should be dispatched ahead of the long attention grid when both are ready
     int prio_lo = 0, prio_hi = 0;
     if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+    // (numerically lower = higher priority).  The readout stream (side[1]) one step below the others: its
+    // kernel has hundreds of blocks, and when it gets onto the SMs first the front kernel (one fat block per
+    // sequence, on the critical path) waits until those have drained.
     for (int k = 0; k < 4 && e == cudaSuccess; ++k)
-      e = cudaStreamCreateWithPriority(&ctx->side[k], cudaStreamNonBlocking, prio_hi);
+      e = cudaStreamCreateWithPriority(&ctx->side[k], cudaStreamNonBlocking,
+                                       (k == 1 && prio_hi + 1 <= prio_lo) ? prio_hi + 1 : prio_hi);
   }
   for (int k = 0; k < 10 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
