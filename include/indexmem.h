@@ -161,6 +161,12 @@ int im_prefill_chunk_attend(im_ctx* ctx, int layer, int n_seq, const int32_t* se
  * A compression that evicts at most `pending_slots` entries keeps them as rank-one terms next to M
  * and the readout adds them exactly; they are folded into M when the list fills.  This is Eq. 6-7
  * re-associated, not an approximation.
+ * CUDA graphs: the kernels of a call take entry counts, positions and pending writes from device memory, so a
+ * captured call can be replayed on later tokens; which kernels a call launches, however, is decided on the host
+ * (compression due or not, evicted set small or large).  With tau = 1 every call is alike and one captured
+ * step replays indefinitely (from the moment every sequence holds B entries); with tau > 1 capture one graph
+ * per phase of the interval or call eagerly.  A replay in the wrong phase leaves the cache uncompressed and is
+ * reported through im_status (count mismatch) once a sequence runs out of slots.
  * Errors: IM_ERR_ARG, IM_ERR_CAPACITY (a sequence has no free slot).
  */
 int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, const void* x,
