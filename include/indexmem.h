@@ -226,12 +226,13 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        im_decode_step prefetches into L2 what the small latency-bound kernels of layer
  *                        (l + 1) mod n_layers will read for the same sequences (weights, indexer key cache,
  *                        counters, pending memory terms); none of it depends on the output of layer l.
- *   IM_OPT_PREFILL_TENSOR 1 (default where n_index_heads <= 8 and index_dim is 8 or 16): im_prefill_chunk
- *                        evaluates the indexer scores of the chunk (Sec. 3.1, a dense [keys x d_I] x
- *                        [d_I x queries * heads] contraction) on the tensor cores, float32 features split
- *                        into three bf16 terms; 0: the CUDA-core kernel.  Both are within 1e-5 of a float32
- *                        evaluation; they need not agree to the last bit.  Setting 1 on an unsupported
- *                        shape returns IM_ERR_ARG.
+ *   IM_OPT_PREFILL_TENSOR 1 (default): the tcgen05 kernels of the prefill calls are used where they apply - the
+ *                        indexer scoring of the chunk (Sec. 3.1, a dense [keys x d_I] x [d_I x queries * heads]
+ *                        contraction; n_index_heads <= 8, index_dim 8 or 16; float32 features split into three
+ *                        bf16 terms) and the chunk attention of im_prefill_chunk_attend (head_dim 128); 0: the
+ *                        CUDA-core scoring kernel and the mma.sync attention kernel.  Both settings are within
+ *                        the stated tolerances of a float32 evaluation; they need not agree to the last bit.
+ *                        Setting 1 where neither kernel applies returns IM_ERR_ARG.
  *   IM_OPT_PROFILE_TARGET which kernel im_profile_begin / im_profile_end time: 0 (default) the attention
  *                        kernel of im_decode_step, 1 the scoring kernel of im_prefill_chunk.  Cannot be
  *                        changed while profiling is active (IM_ERR_STATE).

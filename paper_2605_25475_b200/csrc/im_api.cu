@@ -194,6 +194,7 @@ struct im_ctx {
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
   int n_sm = 1;                      // SMs of the device
   bool score_tc = false;             // prefill scoring runs on the tensor cores (tcgen05)
+  bool attend_tc = true;             // chunk attention of im_prefill_chunk_attend on tcgen05 where head_dim is 128
   int prof_target = 0;               // kernel timed by im_profile_*: 0 attention (decode), 1 prefill scoring
   std::vector<cudaEvent_t> prof_ev;  // pairs (start, stop)
   size_t prof_used = 0;              // events recorded so far
@@ -356,6 +357,7 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK, ctx->mapV);
     if (e == cudaSuccess) e = im_attn_prepare(p);
     if (e == cudaSuccess) e = im_chunk_attn_prepare(p);
+    if (e == cudaSuccess && im_chunk_attn_tc_supported(p)) e = im_chunk_attn_tc_prepare();
     ctx->n_ctas = std::max(1, std::min(sms, IM_ATTN_MAX_CTAS));
     ctx->fast_attn = (e == cudaSuccess);
   }
@@ -509,7 +511,8 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
       CKL(im_launch_gemm(L, g2));
       CKL(im_launch_chunk_readout(L, call));
     }
-    CKL(im_launch_chunk_attention(L, call, ctx->mapK, ctx->mapV, q, out));
+    if (ctx->attend_tc && im_chunk_attn_tc_supported(p)) CKL(im_launch_chunk_attention_tc(L, call, ctx->mapK, ctx->mapV, q, out));
+    else CKL(im_launch_chunk_attention(L, call, ctx->mapK, ctx->mapV, q, out));
   }
   // a1: pooled importance under the causal mask
   {
@@ -742,9 +745,10 @@ int im_set_option(im_ctx* ctx, int option, int value) {
     case IM_OPT_CONCURRENCY: ctx->concurrent = value != 0; return IM_OK;
     case IM_OPT_PREFETCH_NEXT: ctx->prefetch_next = value != 0; return IM_OK;
     case IM_OPT_PREFILL_TENSOR:
-      if (value && !im_score_tc_supported(ctx->p))
-        return fail(IM_ERR_ARG, "the tensor-core prefill scoring needs at most %d indexer heads of width 8 or 16", IM_TC_HP);
-      ctx->score_tc = value != 0;
+      if (value && !im_score_tc_supported(ctx->p) && !im_chunk_attn_tc_supported(ctx->p))
+        return fail(IM_ERR_ARG, "no tensor-core prefill kernel takes this shape (scoring: at most %d indexer heads of width 8 or 16; chunk attention: head_dim 128)", IM_TC_HP);
+      ctx->score_tc = value != 0 && im_score_tc_supported(ctx->p);
+      ctx->attend_tc = value != 0;
       return IM_OK;
     case IM_OPT_PROFILE_TARGET:
       if (value != 0 && value != 1) return fail(IM_ERR_ARG, "profile target %d: 0 = attention, 1 = prefill scoring", value);

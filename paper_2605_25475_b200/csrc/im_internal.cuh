@@ -196,6 +196,10 @@ cudaError_t im_chunk_attn_prepare(const ImDims& p);
 cudaError_t im_launch_chunk_readout(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_chunk_attention(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
                                       const void* q, void* out);
+bool im_chunk_attn_tc_supported(const ImDims& p);
+cudaError_t im_chunk_attn_tc_prepare();
+cudaError_t im_launch_chunk_attention_tc(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
+                                         const void* q, void* out);
 cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const void* q, void* out, int n_max);
 bool im_attn_fast_supported(const ImDims& p);

@@ -323,12 +323,14 @@ def test_decode_from_an_empty_cache(im):
 
 
 # ------------------------------------------------------------------ layer outputs of a prefill chunk's own queries
-def test_chunk_outputs_llama_shape_several_chunks(im):
+@pytest.mark.parametrize("tensor", [1, 0])
+def test_chunk_outputs_llama_shape_several_chunks(im, tensor):
     """32 q / 8 KV heads, d 128: four ragged chunks of 200 tokens into a budget of 256, two sequences; from the
     second chunk on the queries see a retained prefix (holes filled in arbitrary slot order) plus the causal
     chunk and read a non-empty memory; then decode steps continue from the same state."""
     wl = synth.CONFIGS["llama8b_b1"].replace(name="chunk_out", n_seq=2, ctx=4 * 200, chunk=200, B=256, steps=3, n_needles=4)
     p = _pair(wl, chunk_outputs=1)
+    im.im_set_option(p.g.ctx, im.IM_OPT_PREFILL_TENSOR, tensor)   # tcgen05 / mma.sync attention (and scoring)
     for c in range(4):
         p.prefill_attend(c)
     for s in range(wl.steps):
