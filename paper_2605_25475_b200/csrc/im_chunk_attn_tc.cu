@@ -9,11 +9,14 @@
 //   softmax        thread r reads its 64 scores with tcgen05.ld, masks (causal by chunk index), keeps the running
 //                  maximum and sum (base 2), and writes P as two bf16 terms (2^-17) into shared memory in the
 //                  K-major swizzled operand layout
-//   O_tile = P V   tcgen05.mma, N = d = 128, K = 64 keys (4 steps, both P terms); V is used as it lies in the
-//                  cache ([key][d], i.e. MN-major for this product: 8-key groups 1024 bytes apart, the two
-//                  64-column halves 8 KB apart); O_tile in tensor memory
-//   accumulate     thread r reads O_tile and adds it to its 128 float registers after rescaling them by
-//                  2^(m_old - m_new): no read-modify-write of tensor memory
+//   O += P V       tcgen05.mma, N = d = 128, K = 64 keys (4 steps, both P terms), accumulating in tensor memory
+//                  over the tiles; V is used as it lies in the cache ([key][d], i.e. MN-major for this product:
+//                  8-key groups 1024 bytes apart, the two 64-column halves 8 KB apart)
+//   rescale        P is formed relative to a reference maximum that is only raised when a row's maximum has
+//                  grown by more than 2^8 (or is seen for the first time): then the warp waits for the previous
+//                  P V product, multiplies its O rows in tensor memory (tcgen05.ld / st) and its row sums by
+//                  2^(m_ref_old - m_ref_new).  Between such events P (<= 2^8) and O need no correction, so the
+//                  softmax of tile j + 1 overlaps with the P V product of tile j (P is double buffered).
 // Warps 0-3: softmax / accumulate / epilogue; warp 4 lane 0: TMA; warp 5: tensor memory owner, lane 0 issues the
 // MMAs.  Every wait is bounded (ST_TIMEOUT).
 #include <cuda.h>
@@ -34,14 +37,14 @@ constexpr int Q_BYTES = ROWS * DH * 2;      // 32 KB: two halves of 128 rows x 1
 constexpr int P_BYTES = ROWS * KT * 2;      // 16 KB per term
 constexpr int THREADS = 192;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
-constexpr int TMEM_COLS = 256;              // S: 2 x 64, O_tile: 128
+constexpr int TMEM_COLS = 256;              // S: 2 x 64, O: 128
 
 struct Shared {
-  unsigned long long full[STAGES], empty[STAGES], sfull[2], sempty[2], pfull, ofull, oempty;
+  unsigned long long full[STAGES], empty[STAGES], sfull[2], sempty[2], pfull[2], pvdone[2];
   uint32_t tmem;
   int abort;
 };
-constexpr int SMEM_BYTES = Q_BYTES + 2 * P_BYTES + STAGES * STAGE_BYTES + (int)sizeof(Shared) + 1024;
+constexpr int SMEM_BYTES = Q_BYTES + 4 * P_BYTES + STAGES * STAGE_BYTES + (int)sizeof(Shared) + 1024;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -109,6 +112,21 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 #pragma unroll
   for (int k = 0; k < 32; ++k) v[k] = __uint_as_float(r[k]);
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n\t"
+      "tcgen05.wait::st.sync.aligned;" ::"r"(taddr),
+      "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+      "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+      "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+      "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+      "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+      "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+      "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+      "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -123,8 +141,8 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* s_q = smem;                       // [2 halves][128 rows][128 bytes]
-  uint8_t* s_p = smem + Q_BYTES;             // [2 terms][128 rows][128 bytes]
-  uint8_t* s_kv = s_p + 2 * P_BYTES;         // [STAGES][K: 2 halves x 64 rows x 128 bytes | V: the same]
+  uint8_t* s_p = smem + Q_BYTES;             // [2 buffers][2 terms][128 rows][128 bytes]
+  uint8_t* s_kv = s_p + 4 * P_BYTES;         // [STAGES][K: 2 halves x 64 rows x 128 bytes | V: the same]
   Shared* sh = reinterpret_cast<Shared*>(s_kv + STAGES * STAGE_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.y, i = blockIdx.z;
@@ -148,9 +166,10 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
       mbar_init(smem_u32(&sh->sfull[b]), 1);
       mbar_init(smem_u32(&sh->sempty[b]), ROWS);
     }
-    mbar_init(smem_u32(&sh->pfull), ROWS);
-    mbar_init(smem_u32(&sh->ofull), 1);
-    mbar_init(smem_u32(&sh->oempty), ROWS);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sh->pfull[b]), ROWS);
+      mbar_init(smem_u32(&sh->pvdone[b]), 1);
+    }
     sh->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -185,7 +204,7 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = sh->tmem;
-  const uint32_t t_o = tmem + 128;  // O_tile columns; S buffers at columns 0 and 64
+  const uint32_t t_o = tmem + 128;  // O columns; S buffers at columns 0 and 64
   bool ok = true;
 
   if (warp == 4) {
@@ -227,30 +246,25 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
       ok = issue_s(0);
       for (int j = 0; j < nt && ok; ++j) {
         if (j + 1 < nt && !issue_s(j + 1)) { ok = false; break; }
-        const int s = j % STAGES;
-        if (!mbar_wait(smem_u32(&sh->pfull), (uint32_t)(j & 1), abort_flag)) { ok = false; break; }
-        if (j >= 1 && !mbar_wait(smem_u32(&sh->oempty), (uint32_t)((j - 1) & 1), abort_flag)) { ok = false; break; }
+        const int s = j % STAGES, b = j & 1;
+        if (!mbar_wait(smem_u32(&sh->pfull[b]), (uint32_t)((j >> 1) & 1), abort_flag)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t va = smem_u32(s_kv + (size_t)s * STAGE_BYTES) + KV_TILE;
 #pragma unroll
         for (int term = 0; term < 2; ++term)
 #pragma unroll
           for (int ks = 0; ks < KT / 16; ++ks)
-            mma_bf16(t_o, desc_sw128(pa + term * P_BYTES + ks * 32, 16, 1024), desc_sw128(va + ks * 2048, HALF_BYTES, 1024),
-                     idesc_o, (term | ks) ? 1u : 0u);
-        mma_commit(smem_u32(&sh->ofull));
+            mma_bf16(t_o, desc_sw128(pa + (2 * b + term) * P_BYTES + ks * 32, 16, 1024), desc_sw128(va + ks * 2048, HALF_BYTES, 1024),
+                     idesc_o, (j | term | ks) ? 1u : 0u);
+        mma_commit(smem_u32(&sh->pvdone[b]));
         mma_commit(smem_u32(&sh->empty[s]));
       }
     }
   } else {
-    // ---- softmax, accumulation, epilogue: thread = row = TMEM lane
+    // ---- softmax, rescale, epilogue: thread = row = TMEM lane
     const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
     const float sl2 = p.scale * 1.4426950408889634f;  // softmax in base 2
-    float o[DH];
-#pragma unroll
-    for (int c = 0; c < DH; ++c) o[c] = 0.f;
-    float m = NEG_INF, l = 0.f;
-    uint8_t* prow = s_p + (tid >> 3) * 1024 + (tid & 7) * 128;
+    float m_ref = NEG_INF, l = 0.f;                    // reference maximum of P and O, row sum relative to it
     for (int j = 0; j < nt; ++j) {
       const int b = j & 1;
       if (!mbar_wait(smem_u32(&sh->sfull[b]), (uint32_t)((j >> 1) & 1), abort_flag)) { ok = false; break; }
@@ -267,12 +281,32 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
         sv[k] = key0 + k < lim ? sv[k] * sl2 : NEG_INF;
         tm = fmaxf(tm, sv[k]);
       }
-      const float mn = fmaxf(m, tm);
-      const float corr = mn == NEG_INF ? 1.f : exp2f(m - mn);  // a row that has seen no key yet keeps the factor 1
-      const float e = mn == NEG_INF ? 0.f : mn;
-      m = mn;
-      l *= corr;
-      // P of the previous tile has been consumed: its P V product completed before O_tile was read below
+      // raise the reference only for a first maximum or a jump of more than 8 (P stays below 2^8 otherwise)
+      const bool raise = tm > NEG_INF && (m_ref == NEG_INF || tm > m_ref + 8.0f);
+      if (__any_sync(0xffffffffu, raise)) {
+        const float corr = raise ? exp2f(m_ref - tm) : 1.0f;  // 0 for a first maximum: nothing accumulated yet
+        if (raise) {
+          m_ref = tm;
+          l *= corr;
+        }
+        if (j >= 1) {  // O holds the products up to tile j - 1: wait for the last one, then scale the rows
+          if (!mbar_wait(smem_u32(&sh->pvdone[(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+          for (int c0 = 0; c0 < DH; c0 += 32) {
+            float t[32];
+            tmem_ld32(t_o + lane_addr + (uint32_t)c0, t);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) t[c] *= corr;
+            tmem_st32(t_o + lane_addr + (uint32_t)c0, t);
+          }
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        }
+      }
+      // P buffer b was last read by the product of tile j - 2
+      if (j >= 2 && !mbar_wait(smem_u32(&sh->pvdone[b]), (uint32_t)(((j >> 1) - 1) & 1), abort_flag)) { ok = false; break; }
+      const float e = m_ref == NEG_INF ? 0.f : m_ref;
+      uint8_t* prow = s_p + (size_t)(2 * b) * P_BYTES + (tid >> 3) * 1024 + (tid & 7) * 128;
 #pragma unroll
       for (int c = 0; c < KT / 8; ++c) {
         uint32_t hi[4], lo[4];
@@ -288,34 +322,33 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
         *reinterpret_cast<uint4*>(dst + P_BYTES) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(smem_u32(&sh->pfull));
-      // O_tile = P V of this tile
-      if (!mbar_wait(smem_u32(&sh->ofull), (uint32_t)(j & 1), abort_flag)) { ok = false; break; }
+      mbar_arrive(smem_u32(&sh->pfull[b]));
+    }
+    // ---- epilogue: O / l + gated readout
+    if (ok && !mbar_wait(smem_u32(&sh->pvdone[(nt - 1) & 1]), (uint32_t)(((nt - 1) >> 1) & 1), abort_flag)) ok = false;
+    if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const float inv = l > 0.f ? 1.0f / l : 0.f;
+      const float* mr = sc.mch + ((size_t)i * C + (row_ok ? s_row : 0)) * p.Dkv + h * DH;
+      OutT* op = out + (((size_t)i * C + (row_ok ? s_row : 0)) * p.H + (size_t)h * p.Gq + hh) * DH;
 #pragma unroll
       for (int c0 = 0; c0 < DH; c0 += 32) {
         float t[32];
-        tmem_ld32(t_o + lane_addr + (uint32_t)c0, t);
+        tmem_ld32(t_o + lane_addr + (uint32_t)c0, t);  // (warp-collective: rows out of range load too, and skip the store)
+        if (row_ok) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[c0 + c] = fmaf(o[c0 + c], corr, t[c]);
-      }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(smem_u32(&sh->oempty));
-    }
-    if (ok && row_ok) {
-      const float inv = l > 0.f ? 1.0f / l : 0.f;
-      const float* mr = sc.mch + ((size_t)i * C + s_row) * p.Dkv + h * DH;
-      OutT* op = out + (((size_t)i * C + s_row) * p.H + (size_t)h * p.Gq + hh) * DH;
+          for (int c = 0; c < 32; c += 8) {
+            float v[8];
 #pragma unroll
-      for (int c = 0; c < DH; c += 8) {
-        float v[8];
+            for (int k = 0; k < 8; ++k) v[k] = t[c + k] * inv + (p.mem ? mr[c0 + c + k] : 0.f);
+            if constexpr (sizeof(OutT) == 2) {
+              *reinterpret_cast<uint4*>(op + c0 + c) =
+                  make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+            } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) v[k] = o[c + k] * inv + (p.mem ? mr[c + k] : 0.f);
-        if constexpr (sizeof(OutT) == 2) {
-          *reinterpret_cast<uint4*>(op + c) = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
-        } else {
-#pragma unroll
-          for (int k = 0; k < 8; ++k) op[c + k] = v[k];
+              for (int k = 0; k < 8; ++k) op[c0 + c + k] = v[k];
+            }
+          }
         }
       }
     }
