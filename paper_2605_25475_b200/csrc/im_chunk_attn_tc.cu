@@ -127,6 +127,12 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
       "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
       : "memory");
 }
+// 2^x, x <= 8 here; -inf gives 0
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -276,11 +282,13 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
       mbar_arrive(smem_u32(&sh->sempty[b]));
       const int key0 = j * KT;
       float tm = NEG_INF;
+      if (key0 + KT > lim) {  // only the row's last tiles need the causal mask
 #pragma unroll
-      for (int k = 0; k < KT; ++k) {
-        sv[k] = key0 + k < lim ? sv[k] * sl2 : NEG_INF;
-        tm = fmaxf(tm, sv[k]);
+        for (int k = 0; k < KT; ++k) sv[k] = key0 + k < lim ? sv[k] : NEG_INF;
       }
+#pragma unroll
+      for (int k = 0; k < KT; ++k) tm = fmaxf(tm, sv[k]);
+      tm *= sl2;  // the scale is positive: the maximum of the scaled scores
       // raise the reference only for a first maximum or a jump of more than 8 (P stays below 2^8 otherwise)
       const bool raise = tm > NEG_INF && (m_ref == NEG_INF || tm > m_ref + 8.0f);
       if (__any_sync(0xffffffffu, raise)) {
@@ -312,7 +320,7 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
         uint32_t hi[4], lo[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const float p0 = exp2f(sv[c * 8 + 2 * k] - e), p1 = exp2f(sv[c * 8 + 2 * k + 1] - e);
+          const float p0 = ex2(fmaf(sv[c * 8 + 2 * k], sl2, -e)), p1 = ex2(fmaf(sv[c * 8 + 2 * k + 1], sl2, -e));
           l += p0 + p1;
           hi[k] = pack_bf16(p0, p1);
           lo[k] = pack_bf16(p0 - __uint_as_float(hi[k] << 16), p1 - __uint_as_float(hi[k] & 0xffff0000u));
