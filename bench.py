@@ -338,11 +338,27 @@ ATTN_TRAFFIC_NCU = 272.0e6
 def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     L = wl.n_layers
     n_in = len(inputs)
-    host = [tuple(t.cpu().pin_memory() for t in inp) for inp in inputs]
-    dx, dq, dk, dv = [torch.empty_like(t) for t in inputs[0]]
+    # one pinned host buffer and one device buffer per input set / step: [L][x | q | k | v] (bf16), so that a
+    # layer's inputs travel in a single copy
+    sizes = [t[0].numel() for t in inputs[0]]                     # elements per layer of x, q, k, v
+    per_layer = sum(sizes)
+    host = []
+    for inp in inputs:
+        hb = torch.empty((L, per_layer), dtype=torch.bfloat16).pin_memory()
+        off = 0
+        for t, n in zip(inp, sizes):
+            hb[:, off:off + n].copy_(t.reshape(L, n).cpu())
+            off += n
+        host.append(hb)
+    dbuf = torch.empty((L, per_layer), dtype=torch.bfloat16, device=device)
+    views, off = [], 0
+    for t, n in zip(inputs[0], sizes):
+        views.append([dbuf[layer, off:off + n].view(t.shape[1:]) for layer in range(L)])
+        off += n
+    dx, dq, dk, dv = views
     dout = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=device)
     hout = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16).pin_memory()
-    h2d = sum(t.numel() * t.element_size() for t in host[0])
+    h2d = host[0].numel() * host[0].element_size()
     d2h = hout.numel() * hout.element_size()
 
     cs, ds = torch.cuda.Stream(device), torch.cuda.Stream(device)   # host-to-device / device-to-host copies
@@ -353,16 +369,13 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     def enqueue(k):
         """One step: the copies of layer l + 1's inputs and of layer l - 1's outputs run next to layer l's
         kernels (three streams, forked from and joined back into `stream`, so that it can be captured)."""
-        hx, hq, hk, hv = host[k]
+        hb = host[k]
         ev_fork.record(stream)
         cs.wait_event(ev_fork)
         ds.wait_event(ev_fork)
         for layer in range(L):
             with torch.cuda.stream(cs):
-                dx[layer].copy_(hx[layer], non_blocking=True)
-                dq[layer].copy_(hq[layer], non_blocking=True)
-                dk[layer].copy_(hk[layer], non_blocking=True)
-                dv[layer].copy_(hv[layer], non_blocking=True)
+                dbuf[layer].copy_(hb[layer], non_blocking=True)
                 ev_in[layer].record(cs)
             stream.wait_event(ev_in[layer])
             g.decode_step(layer, ids, dx[layer], dq[layer], dq[layer], dk[layer], dv[layer], dout[layer])
