@@ -122,6 +122,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   for (int k = 0; k < 32; ++k) v[k] = __uint_as_float(r[k]);
 }
 
+// the same load without the wait, and the pieces to use several of them at once: issue the loads, wait once,
+// then pass every destination register through an empty volatile statement placed after the wait, so that the
+// compiler cannot schedule a use of a loaded value before the wait
+#define IM_R32(r) "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), \
+    "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]),      \
+    "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]),      \
+    "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld32_landed(uint32_t* r) { asm volatile("" : IM_R32(r)::"memory"); }
+
 // imp = max(imp, v) for any mixture of signs (non-negative floats order as signed integers, negative
 // ones in reverse as unsigned integers); the result does not depend on the order of the updates
 __device__ __forceinline__ void atomic_max_float(float* addr, float v) {
@@ -260,11 +281,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_prefill_score_tc(ImDims p, Im
       const int sbase = jt * IM_TC_QT + half * 16;
       const bool masked = jt * IM_TC_QT < cmax;  // some key of the CTA is newer than the tile's first query
       const uint32_t taddr = tmem + ((uint32_t)lane_base << 16) + (uint32_t)(a * TC_N + half * 128);
-#pragma unroll 1
+      // the warp's 128 accumulator columns of the tile in one round trip
+      uint32_t rv[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32_issue(taddr + c * 32, rv[c]);
+      tmem_ld_wait();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32_landed(rv[c]);
+#pragma unroll
       for (int c = 0; c < 4; ++c) {
         if (sbase + c * 4 >= C) break;
         float v[32];
-        tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) v[k] = __uint_as_float(rv[c][k]);
 #pragma unroll
         for (int qq = 0; qq < 4; ++qq) {
           const int sq = sbase + c * 4 + qq;
