@@ -312,7 +312,11 @@ k_chunk_attention(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     }
   }
   if (!ok) {
-    if (lane == 0) atomicOr(st.status, ST_TIMEOUT);
+    if (lane == 0) {
+      atomicOr(st.status, ST_TIMEOUT);
+      // copies that this CTA still has in flight write into its shared memory: give them time to land (bounded)
+      for (int k = 0; k < 64; ++k) __nanosleep(1000);
+    }
     return;
   }
   // ---- normalise, add the gated readout, store

@@ -364,6 +364,8 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
   if (!ok && lane == 0) {
     sh->abort = 1;
     atomicOr(st.status, ST_TIMEOUT);
+    // copies that this CTA still has in flight write into its shared memory: give them time to land (bounded)
+    for (int k = 0; k < 64; ++k) __nanosleep(1000);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();

@@ -363,6 +363,8 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
   if (!ok && lane == 0) {
     sh->abort = 1;
     atomicOr(status, ST_TIMEOUT);
+    // copies that this CTA still has in flight write into its shared memory: give them time to land (bounded)
+    for (int k = 0; k < 64; ++k) __nanosleep(1000);
   }
   __syncthreads();
   if (warp == 1) {
