@@ -317,13 +317,14 @@ __global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, Im
 
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
                                    int do_select, int n_max) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done_dev[64] = {};
+  bool* attr_done = im_device_flag(attr_done_dev);
+  if (!attr_done || !*attr_done) {
     cudaError_t e = cudaFuncSetAttribute(k_decode_front<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    if (attr_done) *attr_done = true;
   }
   const int key_slots = do_select ? n_max : 0;
   const size_t smem = (size_t)key_slots * 8 + (size_t)L.p.HI * L.p.dI * 4;

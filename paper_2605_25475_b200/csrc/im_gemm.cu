@@ -279,11 +279,12 @@ __global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __
 }  // namespace
 
 cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done_dev[64] = {};
+  bool* attr_done = im_device_flag(attr_done_dev);
+  if (!attr_done || !*attr_done) {
     cudaError_t e = cudaFuncSetAttribute(k_skinny_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 64 * (KC_MAX * 2 + 16));
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    if (attr_done) *attr_done = true;
   }
   ImGemmArgs a = a_in;
   if (a.tensor && im_tc_gemm_usable(a)) return im_launch_tc_gemm(L, a);

@@ -408,11 +408,12 @@ bool im_tc_gemm_usable(const ImGemmArgs& a) {
 }
 
 cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done_dev[64] = {};
+  bool* attr_done = im_device_flag(attr_done_dev);
+  if (!attr_done || !*attr_done) {
     cudaError_t e = cudaFuncSetAttribute(k_tc_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    if (attr_done) *attr_done = true;
   }
   // vectors at a uniform stride: both operands by TMA, one launch per job
   bool uniform = true;
@@ -424,11 +425,12 @@ cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a) {
     else uniform = false;
   }
   if (uniform) {
-    static bool tma_attr_done = false;
-    if (!tma_attr_done) {
+    static bool tma_attr_done_dev[64] = {};
+    bool* tma_attr_done = im_device_flag(tma_attr_done_dev);
+    if (!tma_attr_done || !*tma_attr_done) {
       cudaError_t e = cudaFuncSetAttribute(k_tc_gemm_tma, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM);
       if (e != cudaSuccess) return e;
-      tma_attr_done = true;
+      if (tma_attr_done) *tma_attr_done = true;
     }
     CUtensorMap mA[4], mB0[4], mB1[4];
     bool enc_ok = true;

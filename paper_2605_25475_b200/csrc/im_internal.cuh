@@ -168,6 +168,14 @@ struct ImLaunch {
   int64_t* launches;
 };
 
+// Function attributes (dynamic shared-memory limits) are a per-device setting: launchers that set them lazily keep
+// one flag per device.  Returns the current device's flag (nullptr if the device id is out of range).
+inline bool* im_device_flag(bool (&flags)[64]) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  return &flags[dev];
+}
+
 // records `msg` as the calling thread's last error and returns `code` (defined next to im_last_error)
 int im_fail_message(int code, const char* msg);
 
