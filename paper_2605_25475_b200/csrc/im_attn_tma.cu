@@ -346,15 +346,31 @@ __global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const ImRows r = im_rows(p);
   const int m0 = rc * R_ROWS, mcnt = min(R_ROWS, p.dM - m0);
-  if (threadIdx.x < R_ROWS) s_phi[threadIdx.x] = threadIdx.x < mcnt ? im_raw_sum(p, sc, call, i, r.theta + m0 + threadIdx.x) : 0.f;
-  __syncthreads();
   const uint64_t pol = policy_evict_first();
   const float* Mh = st.Mhat + (u * p.dM + m0) * (size_t)p.Dkv;
+  // the first rows of Mhat do not depend on phi(q): their loads go out before the wait for it
+  const bool pre = (int)threadIdx.x < p.Dkv / 4 && mcnt >= 8;
+  float4 v0[8];
+  if (pre) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v0[k] = ldg_stream(reinterpret_cast<const float4*>(Mh + (size_t)k * p.Dkv) + threadIdx.x, pol);
+  }
+  if (threadIdx.x < R_ROWS) s_phi[threadIdx.x] = threadIdx.x < mcnt ? im_raw_sum(p, sc, call, i, r.theta + m0 + threadIdx.x) : 0.f;
+  __syncthreads();
   const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
   float* dst = sc.rpart + ((size_t)i * nchunk + rc) * p.Dkv;
   for (int c4 = threadIdx.x; c4 < p.Dkv / 4; c4 += blockDim.x) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     int m = 0;
+    if (pre && c4 == (int)threadIdx.x) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const float f = s_phi[k];
+        acc.x = fmaf(f, v0[k].x, acc.x); acc.y = fmaf(f, v0[k].y, acc.y);
+        acc.z = fmaf(f, v0[k].z, acc.z); acc.w = fmaf(f, v0[k].w, acc.w);
+      }
+      m = 8;
+    }
     for (; m + 8 <= mcnt; m += 8) {
       float4 v[8];
 #pragma unroll
