@@ -67,6 +67,15 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     }
   };
   load_batch(0);
+  // the new token's K / V rows (copied into slot n below): requested now, stored after the first barrier
+  const int dv = p.d / 8;
+  const bool kv_here = tid < p.Hkv * dv;
+  uint4 knew_c = make_uint4(0u, 0u, 0u, 0u), vnew_c = knew_c;
+  if (kv_here) {
+    const int h = tid / dv, c = tid % dv;
+    knew_c = reinterpret_cast<const uint4*>(k_new + (size_t)i * p.Dkv + h * p.d)[c];
+    vnew_c = reinterpret_cast<const uint4*>(v_new + (size_t)i * p.Dkv + h * p.d)[c];
+  }
   // ---- finish the projections: sum the K-split partials in a fixed order
   for (int k = tid; k < nq; k += FRONT_THREADS) {
     s_q[k] = im_raw_sum(p, sc, call, i, r.uq + k);
@@ -98,8 +107,13 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     sh.knew[k] = __bfloat162float(b);
   }
   // ---- append K / V / position in slot n
-  const int dv = p.d / 8;
-  for (int k = tid; k < p.Hkv * dv; k += FRONT_THREADS) {
+  if (kv_here) {
+    const int h = tid / dv, c = tid % dv;
+    const size_t row = ((u * p.Hkv + h) * p.cap + n) * p.d;
+    reinterpret_cast<uint4*>(st.Kc + row)[c] = knew_c;
+    reinterpret_cast<uint4*>(st.Vc + row)[c] = vnew_c;
+  }
+  for (int k = tid + FRONT_THREADS; k < p.Hkv * dv; k += FRONT_THREADS) {  // (more chunks than threads)
     const int h = k / dv, c = k % dv;
     const size_t row = ((u * p.Hkv + h) * p.cap + n) * p.d;
     reinterpret_cast<uint4*>(st.Kc + row)[c] = reinterpret_cast<const uint4*>(k_new + (size_t)i * p.Dkv + h * p.d)[c];
