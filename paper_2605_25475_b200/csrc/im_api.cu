@@ -188,7 +188,7 @@ struct im_ctx {
   // Independent pieces of one decode call run on three side streams that fork from and join back into
   // the caller's stream (plain event dependencies, so the pattern can be captured into a CUDA graph).
   cudaStream_t side[4] = {nullptr, nullptr, nullptr, nullptr};
-  cudaEvent_t ev[10] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t ev[12] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   bool concurrent = false;
   bool prefetch_next = true;         // warm L2 with the next layer's weights / index state during attention
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
@@ -377,12 +377,12 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
       e = cudaStreamCreateWithPriority(&ctx->side[k], cudaStreamNonBlocking,
                                        (k == 1 && prio_hi + 1 <= prio_lo) ? prio_hi + 1 : prio_hi);
   }
-  for (int k = 0; k < 10 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
+  for (int k = 0; k < 12 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
-    for (int k = 0; k < 10; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+    for (int k = 0; k < 12; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
     delete ctx;
     return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
   }
@@ -394,7 +394,7 @@ int im_destroy(im_ctx* ctx) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   cudaError_t e = cudaDeviceSynchronize();
   for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
-  for (int k = 0; k < 10; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+  for (int k = 0; k < 12; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   delete ctx;
   if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
   return IM_OK;
@@ -676,6 +676,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
     CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
+    CK(cudaEventRecord(ctx->ev[9], s0));  // the attention kernel has read the cache
   }
   // an evicted set larger than the pending list is accumulated into Mhat itself, which the readout reads
   const bool readout_early = !(mem_write && ne_max > p.F);
@@ -693,6 +694,15 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   if (due && !fused) {
     CKL(im_launch_select(L1, call));
     if (ne_max > 0) CKL(im_launch_gather_move(L1, call, ne_max));
+  }
+  if (conc) {
+    // a4 (fill the holes, publish the entry count) once the front kernel has listed the moves and the attention
+    // kernel has read the cache: next to the merge, on the stream the key projection has long left
+    CK(cudaEventRecord(ctx->ev[11], L1.stream));
+    CK(cudaStreamWaitEvent(L3.stream, ctx->ev[11], 0));
+    CK(cudaStreamWaitEvent(L3.stream, ctx->ev[9], 0));
+    CKL(im_launch_decode_commit(L3, call));
+    CK(cudaEventRecord(ctx->ev[10], L3.stream));
   }
   // a3: memory write (needs the gathered evicted pairs and the fold).  With deferred compaction the readout
   // of the state after the write is formed from phi of the evicted keys (k_readout_apply), and the state
@@ -726,6 +736,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
       CK(cudaStreamWaitEvent(s0, ctx->ev[8], 0));  // s3
     }
     CKL(im_launch_attention_merge(L, call, out, ctx->n_ctas, q, k_new, v_new));
+    if (defer && !conc) CKL(im_launch_decode_commit(L, call));
+    if (conc) CK(cudaStreamWaitEvent(s0, ctx->ev[10], 0));
     if (conc) {  // the memory write only has to end with the call
       CK(cudaEventRecord(ctx->ev[5], L1.stream));
       CK(cudaStreamWaitEvent(s0, ctx->ev[5], 0));

@@ -539,7 +539,6 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
                                                           OutT* __restrict__ out, const bf16* __restrict__ q,
                                                           const bf16* __restrict__ k_new, const bf16* __restrict__ v_new) {
   constexpr int CPL = DH / 32;  // columns per lane
-  __shared__ int s_ev[IM_FRONT_MAX_NE], s_sv[IM_FRONT_MAX_NE];
   __shared__ float s_q[8][DH];  // recompute path: the warp's query row
   const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
@@ -549,10 +548,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
   // on the critical path of the call and a dependent chain of loads costs a memory round trip per link
   const int na_lane = lane < call.n_seq ? sc.n_att[lane] : 0;
   const int ne_raw = st.ctr[u * CTR_STRIDE + CTR_NEVICT];
-  const int nh_raw = sc.nhole[i];
-  const int n_next = st.ctr[u * CTR_STRIDE + CTR_NNEXT];
   const int ev_l = lane < IM_FRONT_MAX_NE ? st.ev_slot[u * p.tail + min(lane, p.tail - 1)] : -1;
-  const int sv_l = lane < IM_FRONT_MAX_NE ? sc.surv[(size_t)i * p.tail + min(lane, p.tail - 1)] : -1;
   const float* mr = sc.mres + (size_t)i * (p.Dkv + 2);
   float gate = 0.f, mcol[CPL], qv[CPL], kn[CPL], vn[CPL], ek0[CPL], ev0[CPL];
   {
@@ -602,7 +598,6 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
   const long long row_first = pref + (long long)h * nt_i, row_last = row_first + nt_i - 1;
   const long long row_id = (long long)i * p.Hkv + h;
   const int ne = call.defer ? max(0, min(ne_raw, IM_FRONT_MAX_NE)) : 0;
-  if (warp == 0 && lane < IM_FRONT_MAX_NE) { s_ev[lane] = ev_l; s_sv[lane] = sv_l; }
   const float sl2 = p.scale * 1.4426950408889634f;
   // ---- one warp per query head of the group
   for (int hh = warp; hh < p.Gq; hh += nwarps) {
@@ -779,30 +774,6 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
       const float v = res[k] + gate * mcol[k];  // Eq. 4: attention over the retained set + gated memory readout
       if constexpr (sizeof(OutT) == 2) out[base + lane + 32 * k] = __float2bfloat16_rn(v);
       else out[base + lane + 32 * k] = v;
-    }
-  }
-  if (call.defer) {
-    // a4, deferred: the attention kernel has read the cache and every warp of this block is done with the
-    // rows of this KV head, so the holes below the budget can take the retained entries found above it
-    // (block h moves the K / V rows of its head; block 0 also the indexer keys and positions, and publishes
-    // the entry count, which no other block of this kernel reads)
-    __syncthreads();
-    const int nh = min(max(nh_raw, 0), ne);
-    constexpr int CH = DH / 8;  // 16-byte chunks per row
-    const size_t base = (u * p.Hkv + h) * (size_t)p.cap;
-    for (int k = tid; k < nh * CH; k += blockDim.x) {
-      const int j = k / CH, c = k % CH;
-      const int dst = s_ev[j], src = s_sv[j];
-      reinterpret_cast<uint4*>(st.Kc + (base + dst) * DH)[c] = reinterpret_cast<const uint4*>(st.Kc + (base + src) * DH)[c];
-      reinterpret_cast<uint4*>(st.Vc + (base + dst) * DH)[c] = reinterpret_cast<const uint4*>(st.Vc + (base + src) * DH)[c];
-    }
-    if (h == 0) {
-      for (int k = tid; k < nh * p.dI; k += blockDim.x) {
-        const int j = k / p.dI, c = k % p.dI;
-        st.kidx[(u * p.cap + s_ev[j]) * p.dI + c] = st.kidx[(u * p.cap + s_sv[j]) * p.dI + c];
-      }
-      for (int j = tid; j < nh; j += blockDim.x) st.pos[u * p.cap + s_ev[j]] = st.pos[u * p.cap + s_sv[j]];
-      if (tid == 0) st.ctr[u * CTR_STRIDE + CTR_N] = n_next;
     }
   }
 }

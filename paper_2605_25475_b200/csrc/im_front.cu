@@ -306,6 +306,9 @@ __global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, Im
   const int i = blockIdx.y;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
+  // deferred compaction: this kernel also publishes the entry count the call leaves (no kernel that runs next to
+  // it reads CTR_N: the merge kernel works from the attention kernel's snapshot)
+  if (call.defer && blockIdx.x == 0 && threadIdx.x == 0) st.ctr[u * CTR_STRIDE + CTR_N] = st.ctr[u * CTR_STRIDE + CTR_NNEXT];
   if (ne <= 0) return;
   const int nh = min(sc.nhole[i], ne);
   const int j0 = blockIdx.x * 4;
@@ -347,6 +350,15 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
   if (L.p.dI == 16) k_decode_front<16><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
   else if (L.p.dI == 8) k_decode_front<8><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
   else k_decode_front<0><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+// deferred compaction (a4): fills the holes and publishes the entry count once the attention kernel has read the
+// cache; may run next to the merge kernel, which reads neither the evicted slots nor CTR_N
+cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call) {
+  dim3 grid((IM_FRONT_MAX_NE + 3) / 4, call.n_seq);
+  k_move_survivors<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
 }

@@ -189,6 +189,7 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
                                    int do_select, int n_max);
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
+cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call);
 // ne_host: per call sequence, the number of entries the compression of this call evicts (host mirror)
 cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_max, const int* ne_host);
