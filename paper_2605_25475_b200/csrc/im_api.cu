@@ -147,10 +147,10 @@ void carve(const ImDims& p, char* base, Layout* lo) {
     const size_t stream = ((size_t)IM_ATTN_MAX_CTAS * IM_ATTN_WARPS + (size_t)p.S * p.Hkv) * p.Gq * (p.d + 2);
     lo->sc.part = (float*)take(std::max(generic, stream) * 4);
   }
-  lo->sc.mres = (float*)take((size_t)p.S * (p.Dkv + 2) * 4);
+  lo->sc.mres = (float*)take((size_t)p.S * IM_MRES_ROW(p) * 4);
   lo->sc.phiq = (float*)take((size_t)p.S * p.dM * 4);
   lo->sc.n_att = (int32_t*)take((size_t)p.S * 4);
-  lo->sc.rpart = (float*)take((size_t)p.S * ((p.dM + IM_READOUT_ROWS - 1) / IM_READOUT_ROWS) * p.Dkv * 4);
+  lo->sc.rpart = (float*)take((size_t)p.S * p.Dkv * 4);
   lo->sc.phiT = nullptr;
   lo->sc.vT = nullptr;
   if (p.tail > p.F) {
@@ -188,7 +188,7 @@ struct im_ctx {
   // Independent pieces of one decode call run on three side streams that fork from and join back into
   // the caller's stream (plain event dependencies, so the pattern can be captured into a CUDA graph).
   cudaStream_t side[4] = {nullptr, nullptr, nullptr, nullptr};
-  cudaEvent_t ev[12] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t ev[14] = {};
   bool concurrent = false;
   bool prefetch_next = true;         // warm L2 with the next layer's weights / index state during attention
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
@@ -271,7 +271,7 @@ cudaError_t launch_mem_update(im_ctx* ctx, const ImLaunch& L, const ImCall& call
 
 // phi of the gathered evicted keys (skinny GEMM against the folded Linear_theta), then Eq. 6-7.
 // With `update` = false only the GEMM is launched (the caller launches im_launch_mem_update later).
-int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, bool update = true) {
+int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, bool update = true, int smem_floor = 0) {
   const ImDims& p = ctx->p;
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
@@ -300,6 +300,7 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
     g.ks_stride = (long long)call.n_seq * p.F * p.dM;
     g.kc = 64;  // 18 KB of shared memory: fits next to the resident attention blocks
     g.direct = call.prefill ? 0 : 1;
+    g.smem_floor = smem_floor;
   }
   CKL(im_launch_gemm(L, g));
   if (update) CKL(launch_mem_update(ctx, L, call, ne_max));
@@ -356,6 +357,10 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
     if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK, ctx->mapV);
     if (e == cudaSuccess) e = im_attn_prepare(p);
+    if (e == cudaSuccess) e = im_gemm_prepare_decode();
+    if (e == cudaSuccess) e = im_memory_prepare_decode();
+    if (e == cudaSuccess) e = im_front_prepare_decode();
+    if (e == cudaSuccess) e = im_prefetch_prepare_decode();
     if (e == cudaSuccess) e = im_chunk_attn_prepare(p);
     if (e == cudaSuccess && im_chunk_attn_tc_supported(p)) e = im_chunk_attn_tc_prepare();
     ctx->n_ctas = std::max(1, std::min(sms, IM_ATTN_MAX_CTAS));
@@ -377,12 +382,12 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
       e = cudaStreamCreateWithPriority(&ctx->side[k], cudaStreamNonBlocking,
                                        (k == 1 && prio_hi + 1 <= prio_lo) ? prio_hi + 1 : prio_hi);
   }
-  for (int k = 0; k < 12 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
+  for (int k = 0; k < 14 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
-    for (int k = 0; k < 12; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+    for (int k = 0; k < 14; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
     delete ctx;
     return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
   }
@@ -394,7 +399,7 @@ int im_destroy(im_ctx* ctx) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   cudaError_t e = cudaDeviceSynchronize();
   for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
-  for (int k = 0; k < 12; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+  for (int k = 0; k < 14; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   delete ctx;
   if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
   return IM_OK;
@@ -590,11 +595,10 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   //      entries again (exactly, see k_attn_merge_rows), adds the terms of this call's memory write to the
   //      readout, and fills the holes.
   //        s0: (waits for the three projections) attention ------------------------> merge
-  //        s1: indexer projections -> front (append, score, select, gather) -> phi of the evicted keys ->
-  //            readout over the memory after the write (k_readout_apply)
+  //        s1: indexer projections -> front (append, score, select, gather) -> phi of the evicted keys
   //            [-> memory write: not needed by the merge, it only has to end with the call]
-  //        s2: phi(q) / gate projections -> readout partials -> readout over the memory as it is before
-  //            the write
+  //        s2: phi(q) / gate projections -> phi(q)^T Mhat (streams Mhat next to the attention kernel)
+  //        s4: fold -> the readout terms that do not go through Mhat, over the memory as it is before the write
   //        s3: float64 key projection (needed by front) -> L2 prefetch for the next layer
   //        s4: fold of the pending list (before front, which changes the counters, and before the readout)
   //      With IM_OPT_CONCURRENCY off the same kernels run on s0 in an order that respects these arrows.
@@ -608,16 +612,19 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   ImLaunch L = make_launch(ctx, layer, s0);
   ImLaunch L1 = L, L2 = L, L3 = L, L4 = L;
   const bool mem_write = due && ne_max > 0 && p.mem;
+  // concurrent schedule: the SMs left to the latency-bound chain (see IM_SMEM_FRONT)
+  const int n_res = conc ? im_reserved_sms(ctx->n_sm, n_seq) : 0;
+  const int n_ctas = n_res > 0 ? std::max(1, std::min(ctx->n_ctas, ctx->n_sm - n_res)) : ctx->n_ctas;
   if (conc) {
     L1.stream = ctx->side[0];
     L2.stream = ctx->side[1];
     L3.stream = ctx->side[2];
-    if (mem_write) L4.stream = ctx->side[3];
+    L4.stream = ctx->side[3];
     CK(cudaEventRecord(ctx->ev[0], s0));
     CK(cudaStreamWaitEvent(L1.stream, ctx->ev[0], 0));
     CK(cudaStreamWaitEvent(L2.stream, ctx->ev[0], 0));
     CK(cudaStreamWaitEvent(L3.stream, ctx->ev[0], 0));
-    if (mem_write) CK(cudaStreamWaitEvent(L4.stream, ctx->ev[0], 0));
+    CK(cudaStreamWaitEvent(L4.stream, ctx->ev[0], 0));
   }
   const bool prof = ctx->prof_target == 0 && ctx->prof_used + 2 <= ctx->prof_ev.size();
   // s4: fold (reads the counters of before the call; the readout reads the folded state); s3: key projection
@@ -627,15 +634,6 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   }
   CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
   if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // key projection done
-  if (ctx->prefetch_next && ctx->fast_attn) {
-    // warm L2 for the next layer's small kernels while this layer's attention streams K/V
-    ImLaunch Lp = L3;
-    ImCall nxt = call;
-    nxt.layer = (layer + 1) % p.L;
-    Lp.w = ctx->lo.w[nxt.layer];
-    CKL(im_launch_prefetch_layer(Lp, nxt));
-  }
-  if (conc) CK(cudaEventRecord(ctx->ev[8], L3.stream));  // s3 finished
   // a0: projections as K-split partial sums: indexer part (Sec. 3.1 features) on s1 ...
   ImRows r = im_rows(p);
   ImGemmArgs g;
@@ -664,55 +662,82 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CKL(im_launch_gemm(L2, g));
   }
   if (conc) {
-    // a5.  The three projections head every side chain and are latency bound (one memory round trip each);
-    // they get the first microseconds of the call to themselves, because a memory access issued while the
-    // attention kernel keeps the memory system's queues full takes several times longer.  Everything after
-    // them runs next to the attention kernel.
+    // a5.  The attention kernel needs nothing of the call but q.  Where the front kernel has SMs of its own
+    // (n_res > 0) it starts at once and streams the cache while the projections run.  Otherwise the three
+    // projections, which head every side chain and are latency bound (one memory round trip each), get the first
+    // microseconds of the call to themselves: a memory access issued on an SM that an attention CTA keeps busy
+    // takes several times longer, and every kernel of the chain would pay for it.
     CK(cudaEventRecord(ctx->ev[1], L1.stream));
     CK(cudaEventRecord(ctx->ev[6], L2.stream));
-    CK(cudaStreamWaitEvent(s0, ctx->ev[1], 0));
-    CK(cudaStreamWaitEvent(s0, ctx->ev[6], 0));
-    CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
+    if (n_res == 0) {
+      CK(cudaStreamWaitEvent(s0, ctx->ev[1], 0));
+      CK(cudaStreamWaitEvent(s0, ctx->ev[6], 0));
+      CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
+    }
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
-    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
+    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
     CK(cudaEventRecord(ctx->ev[9], s0));  // the attention kernel has read the cache
   }
   // an evicted set larger than the pending list is accumulated into Mhat itself, which the readout reads
   const bool readout_early = !(mem_write && ne_max > p.F);
   if (conc && mem_write) CK(cudaStreamWaitEvent(L2.stream, ctx->ev[7], 0));
-  if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call));
-  if (defer && p.mem) CKL(im_launch_readout_finish(L2, call));  // over the memory as it is before this call's write
+  // s4 again: the part of the readout that does not go through Mhat, over the memory as it is before this call's write
+  if (conc) CK(cudaStreamWaitEvent(L4.stream, ctx->ev[6], 0));
+  if (defer && p.mem) CKL(im_launch_readout_finish(L4, call));
+  if (conc) CK(cudaEventRecord(ctx->ev[4], L4.stream));
   if (conc) {
-    CK(cudaEventRecord(ctx->ev[4], L2.stream));  // s2 finished
     CK(cudaStreamWaitEvent(L1.stream, ctx->ev[2], 0));
     if (mem_write) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0));  // the front kernel changes the counters the fold reads
   }
   // append + a1 (+ a2 and the gather of the evicted pairs when the evicted set is small enough for one
   // block per sequence; a4 in the same kernel unless the compaction is deferred)
-  CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max));
+  CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max, n_res > 0 ? IM_SMEM_FRONT : 0));
   if (due && !fused) {
     CKL(im_launch_select(L1, call));
     if (ne_max > 0) CKL(im_launch_gather_move(L1, call, ne_max));
   }
   if (conc) {
-    // a4 (fill the holes, publish the entry count) once the front kernel has listed the moves and the attention
-    // kernel has read the cache: next to the merge, on the stream the key projection has long left
     CK(cudaEventRecord(ctx->ev[11], L1.stream));
     CK(cudaStreamWaitEvent(L3.stream, ctx->ev[11], 0));
+  }
+  // phi(q)^T Mhat on s2.  Where SMs are set aside for the front kernel it starts when that kernel has ended: its
+  // blocks would otherwise settle on just those SMs (the emptiest ones) and keep the front blocks out; the
+  // attention kernel has the memory system to itself meanwhile, so nothing is lost.
+  if (conc) {
+    if (n_res > 0) {
+      CK(cudaStreamWaitEvent(L2.stream, ctx->ev[11], 0));
+    } else {
+      CK(cudaStreamWaitEvent(L2.stream, ctx->ev[1], 0));
+      CK(cudaStreamWaitEvent(L2.stream, ctx->ev[2], 0));
+    }
+  }
+  if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call, n_res > 0 ? n_ctas : ctx->n_sm, conc && n_res == 0));
+  if (conc) CK(cudaEventRecord(ctx->ev[12], L2.stream));  // s2 finished: the merge needs phi(q)^T Mhat
+  if (ctx->prefetch_next && ctx->fast_attn) {
+    // warm L2 for the next layer's small kernels while this layer's attention streams K/V; after the front kernel,
+    // which should find its SMs free of other kernels' blocks
+    ImLaunch Lp = L3;
+    ImCall nxt = call;
+    nxt.layer = (layer + 1) % p.L;
+    Lp.w = ctx->lo.w[nxt.layer];
+    CKL(im_launch_prefetch_layer(Lp, nxt));
+  }
+  if (conc) {
+    // a4 (fill the holes, publish the entry count) once the front kernel has listed the moves and the attention
+    // kernel has read the cache: next to the merge, on the stream the key projection has long left
     CK(cudaStreamWaitEvent(L3.stream, ctx->ev[9], 0));
     CKL(im_launch_decode_commit(L3, call));
     CK(cudaEventRecord(ctx->ev[10], L3.stream));
   }
-  // a3: memory write (needs the gathered evicted pairs and the fold).  With deferred compaction the readout
-  // of the state after the write is formed from phi of the evicted keys (k_readout_apply), and the state
-  // update itself follows off the critical path, after the readout that wants the state from before it.
-  if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, !defer))) return rc;
-  if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[4], 0));  // s2 joins here
-  if (defer && p.mem) CKL(im_launch_readout_apply(L1, call));
+  // a3: memory write (needs the gathered evicted pairs and the fold).  With deferred compaction the merge kernel
+  // forms the readout of the state after the write from phi of the evicted keys, and the state update itself
+  // follows off the critical path, after the readout kernels that want the state from before it.
+  if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, !defer, n_res > 0 ? IM_SMEM_SIDE : 0))) return rc;
   if (conc) CK(cudaEventRecord(ctx->ev[3], L1.stream));  // everything the merge needs from s1
+  if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[4], 0));  // k_readout_finish reads what the update changes
   if (defer && mem_write) CKL(launch_mem_update(ctx, L1, call, ne_max));
-  if (mem_write && ctx->fast_attn && !readout_early) CKL(im_launch_readout(L1, call));
+  if (mem_write && ctx->fast_attn && !readout_early) CKL(im_launch_readout(L1, call, ctx->n_sm, 0));
   int n_att = 0;
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
@@ -727,15 +752,16 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   if (ctx->fast_attn) {
     if (!conc) {
       if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
-      CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, ctx->n_ctas));
+      CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas));
       if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
     }
     if (!defer && p.mem) CKL(im_launch_readout_finish(L, call));  // after the memory write
     if (conc) {
       CK(cudaStreamWaitEvent(s0, ctx->ev[3], 0));  // s1 (which waited for s2)
-      CK(cudaStreamWaitEvent(s0, ctx->ev[8], 0));  // s3
+      CK(cudaStreamWaitEvent(s0, ctx->ev[12], 0));  // s2
+      CK(cudaStreamWaitEvent(s0, ctx->ev[4], 0));   // s4
     }
-    CKL(im_launch_attention_merge(L, call, out, ctx->n_ctas, q, k_new, v_new));
+    CKL(im_launch_attention_merge(L, call, out, n_ctas, q, k_new, v_new));
     if (defer && !conc) CKL(im_launch_decode_commit(L, call));
     if (conc) CK(cudaStreamWaitEvent(s0, ctx->ev[10], 0));
     if (conc) {  // the memory write only has to end with the call

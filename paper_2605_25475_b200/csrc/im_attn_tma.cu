@@ -337,69 +337,104 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 }
 
 // ------------------------------------------------------------------------------------------------
-// Readout partials: rpart[i][rc][col] = sum over the 32 rows m of chunk rc of phi_q[m] * Mhat[m][col].
-// grid = (ceil(dM / 32), n_seq), block = 256; each thread owns 4 consecutive columns.
-constexpr int R_ROWS = IM_READOUT_ROWS;
-__global__ void __launch_bounds__(256) k_readout(ImDims p, ImState st, ImScratch sc, ImCall call) {
-  __shared__ float s_phi[R_ROWS];
-  const int rc = blockIdx.x, i = blockIdx.y;
-  const size_t u = (size_t)call.layer * p.S + call.seq[i];
-  const ImRows r = im_rows(p);
-  const int m0 = rc * R_ROWS, mcnt = min(R_ROWS, p.dM - m0);
+// Readout numerators (Eq. 5): rsum[i][col] = sum over all dM rows m of phi_q[m] * Mhat[m][col].
+// The kernel runs next to the attention kernel and shares an SM with one of its CTAs: a persistent grid of
+// 256-thread blocks, at most one per SM.  A block owns a contiguous run of items; an item is a 64-column slice
+// (256 bytes of every row) of one sequence's Mhat over all its rows, so that no partial sums go through memory
+// and the merge kernel reads one number per column.  A half warp reads one row slice per load, the 16 half warps
+// of the block take 16 consecutive rows per round, and every thread keeps DEPTH loads in flight across round,
+// batch and item boundaries (a consumed register is re-requested at once).  The loop body between two loads has
+// no branch: with branches there the compiler waits for every load in flight at each of them.
+// Two variants: DEPTH 32 (128 KB in flight per SM, 42 K registers: with an attention CTA it fills the SM's register
+// file, so it is used where the front kernel runs on SMs of its own and has ended before this kernel starts) and
+// DEPTH 8 (16 K registers: leaves room for a front block on the same SM).
+// grid = min(blocks wanted, items), block = RC_THREADS, smem = dM rounded up to RC_RPR * DEPTH floats.
+constexpr int RC_COLS = 64;
+constexpr int RC_THREADS = 256;
+constexpr int RC_RPR = RC_THREADS / 16;  // rows per round
+template <int RC_DEPTH>
+__device__ __forceinline__ void readout_cols_body(const ImDims& p, const ImState& st, const ImScratch& sc, const ImCall& call) {
+  extern __shared__ float s_phi[];  // phi(q) of the current sequence, zero beyond dM
+  __shared__ float4 s_red[RC_RPR][RC_COLS / 4];
+  const int tid = threadIdx.x;
+  const int rsub = tid >> 4, c4 = tid & 15;  // row within a round, float4 within the slice
+  const int nsl = p.Dkv / RC_COLS;
+  const int total = call.n_seq * nsl;
+  const int t0 = (int)((long long)blockIdx.x * total / gridDim.x);
+  const int t1 = (int)((long long)(blockIdx.x + 1) * total / gridDim.x);
+  if (t0 >= t1) return;
+  const int nb = (p.dM + RC_RPR * RC_DEPTH - 1) / (RC_RPR * RC_DEPTH);  // batches of RC_DEPTH rounds per item
   const uint64_t pol = policy_evict_first();
-  const float* Mh = st.Mhat + (u * p.dM + m0) * (size_t)p.Dkv;
-  // the first rows of Mhat do not depend on phi(q): their loads go out before the wait for it
-  const bool pre = (int)threadIdx.x < p.Dkv / 4 && mcnt >= 8;
-  float4 v0[8];
-  if (pre) {
+  const ImRows r = im_rows(p);
+  const size_t row_f4 = (size_t)p.Dkv / 4;
+  // first load of (item t, batch b) for this thread; round k of the batch is k * RC_RPR rows further
+  auto batch_ptr = [&](int t, int b) {
+    const size_t u = (size_t)call.layer * p.S + call.seq[t / nsl];
+    return reinterpret_cast<const float4*>(st.Mhat + u * p.dM * (size_t)p.Dkv + (size_t)(t % nsl) * RC_COLS) + c4;
+  };
+  float4 v[RC_DEPTH];
+  {
+    const float4* src = batch_ptr(t0, 0);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) v0[k] = ldg_stream(reinterpret_cast<const float4*>(Mh + (size_t)k * p.Dkv) + threadIdx.x, pol);
+    for (int k = 0; k < RC_DEPTH; ++k) v[k] = ldg_stream(src + (size_t)min(k * RC_RPR + rsub, p.dM - 1) * row_f4, pol);
   }
-  if (threadIdx.x < R_ROWS) s_phi[threadIdx.x] = threadIdx.x < mcnt ? im_raw_sum(p, sc, call, i, r.theta + m0 + threadIdx.x) : 0.f;
-  __syncthreads();
-  const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
-  float* dst = sc.rpart + ((size_t)i * nchunk + rc) * p.Dkv;
-  for (int c4 = threadIdx.x; c4 < p.Dkv / 4; c4 += blockDim.x) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    int m = 0;
-    if (pre && c4 == (int)threadIdx.x) {
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const float f = s_phi[k];
-        acc.x = fmaf(f, v0[k].x, acc.x); acc.y = fmaf(f, v0[k].y, acc.y);
-        acc.z = fmaf(f, v0[k].z, acc.z); acc.w = fmaf(f, v0[k].w, acc.w);
-      }
-      m = 8;
+  int cur = -1;
+  for (int t = t0; t < t1; ++t) {
+    const int i = t / nsl;
+    if (i != cur) {  // (block uniform)
+      if (cur >= 0) __syncthreads();
+      for (int m = tid; m < nb * RC_RPR * RC_DEPTH; m += RC_THREADS)
+        s_phi[m] = m < p.dM ? im_raw_sum(p, sc, call, i, r.theta + m) : 0.f;
+      cur = i;
+      __syncthreads();
     }
-    for (; m + 8 <= mcnt; m += 8) {
-      float4 v[8];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int b = 0; b < nb; ++b) {
+      const bool more = b + 1 < nb || t + 1 < t1;
+      const float4* src = more ? (b + 1 < nb ? batch_ptr(t, b + 1) : batch_ptr(t + 1, 0)) : nullptr;
+      const int row_next = b + 1 < nb ? (b + 1) * RC_RPR * RC_DEPTH + rsub : rsub;
+      const float* ph = s_phi + b * RC_RPR * RC_DEPTH + rsub;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = ldg_stream(reinterpret_cast<const float4*>(Mh + (size_t)(m + k) * p.Dkv) + c4, pol);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const float f = s_phi[m + k];
+      for (int k = 0; k < RC_DEPTH; ++k) {
+        const float f = ph[k * RC_RPR];
         acc.x = fmaf(f, v[k].x, acc.x); acc.y = fmaf(f, v[k].y, acc.y);
         acc.z = fmaf(f, v[k].z, acc.z); acc.w = fmaf(f, v[k].w, acc.w);
+        if (more) v[k] = ldg_stream(src + (size_t)min(row_next + k * RC_RPR, p.dM - 1) * row_f4, pol);
       }
     }
-    for (; m < mcnt; ++m) {
-      const float4 v = ldg_stream(reinterpret_cast<const float4*>(Mh + (size_t)m * p.Dkv) + c4, pol);
-      const float f = s_phi[m];
-      acc.x = fmaf(f, v.x, acc.x); acc.y = fmaf(f, v.y, acc.y);
-      acc.z = fmaf(f, v.z, acc.z); acc.w = fmaf(f, v.w, acc.w);
+    s_red[rsub][c4] = acc;
+    __syncthreads();
+    if (tid < RC_COLS / 4) {
+      float4 sum = s_red[0][tid];
+#pragma unroll
+      for (int j = 1; j < RC_RPR; ++j) {
+        const float4 o = s_red[j][tid];
+        sum.x += o.x; sum.y += o.y; sum.z += o.z; sum.w += o.w;
+      }
+      reinterpret_cast<float4*>(sc.rpart + (size_t)i * p.Dkv + (size_t)(t % nsl) * RC_COLS)[tid] = sum;
     }
-    reinterpret_cast<float4*>(dst)[c4] = acc;
+    __syncthreads();
   }
 }
 
+__global__ void __maxnreg__(168) k_readout_cols(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  readout_cols_body<32>(p, st, sc, call);
+}
+__global__ void __maxnreg__(64) k_readout_cols_light(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  readout_cols_body<8>(p, st, sc, call);
+}
+
 // ------------------------------------------------------------------------------------------------
-// Readout, second half (Eq. 5 and the gate of Eq. 4), once per sequence:
-//   mres[i][col] = cscale * ( sum_chunks rpart[col] + sum_p w_p (phi_q . phi_p) v_p[col] ) / ( sum_m phi_q[m]^2 b[m] + eps )
-//   mres[i][Dkv] = g(q)
-// Without deferred compaction it runs after the memory write of the call (it reads the pending list, b and
-// cscale).  With it (call.defer) it runs BEFORE the write and leaves numerator cscale * (...) and the
-// denominator sum apart; the merge kernel adds the terms of the entries written in this call, so that the
-// readout does not wait for the selection.  grid = n_seq, block = 256, smem = dM floats.
+// Readout, the part that does not go through Mhat (Eq. 5 and the gate of Eq. 4), once per sequence.  With
+// s = cscale / (sum_m phi_q[m]^2 b[m] + eps):
+//   mres[i][col]     = s * sum_p w_p (phi_q . phi_p) v_p[col]      (pending rank-one terms)
+//   mres[i][Dkv]     = g(q)
+//   mres[i][Dkv + 2] = s                                             (the merge kernel adds s * phi(q)^T Mhat[col])
+// It does not read the output of k_readout_cols and may run next to it.  Without deferred compaction it runs
+// after the memory write of the call (it reads the pending list, b and cscale).  With it (call.defer) it runs
+// BEFORE the write with s = cscale, leaving the denominator sum apart in mres[i][Dkv + 1]; the merge kernel
+// then adds the terms of the entries written in this call, so that the readout does not wait for the selection.
+// grid = n_seq, block = 256, smem = dM floats.
 __global__ void __launch_bounds__(256) k_readout_finish(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call) {
   extern __shared__ float phiq[];  // [dM] phi(q), summed over the K-split partials
   __shared__ float s_dot[64];
@@ -441,68 +476,17 @@ __global__ void __launch_bounds__(256) k_readout_finish(ImDims p, ImState st, Im
   for (int k = 0; k < 8; ++k) den += s_red[k];
   // deferred compaction: numerator and denominator sum over the state from before the call's memory write
   const float scale = call.defer ? st.cscale[u] : st.cscale[u] / den;
-  const int nchunk = (p.dM + R_ROWS - 1) / R_ROWS;
-  float* dst = sc.mres + (size_t)i * (p.Dkv + 2);
+  float* dst = sc.mres + (size_t)i * IM_MRES_ROW(p);
   for (int m = tid; m < p.dM; m += 256) sc.phiq[(size_t)i * p.dM + m] = phiq[m];
   for (int col = tid; col < p.Dkv; col += 256) {
-    const float* rp = sc.rpart + (size_t)i * nchunk * p.Dkv + col;
     float mv = 0.f;
-    for (int k = 0; k < nchunk; ++k) mv += rp[(size_t)k * p.Dkv];
     for (int pp = 0; pp < np; ++pp) mv = fmaf(s_dot[pp], __bfloat162float(st.pend_v[(u * p.F + pp) * p.Dkv + col]), mv);
     dst[col] = scale * mv;
   }
   if (tid == 0) {
     dst[p.Dkv] = 1.0f / (1.0f + expf(-(im_raw_sum(p, sc, call, i, r.wg) + w.bg[0])));
     dst[p.Dkv + 1] = den - p.eps;
-  }
-}
-
-// Deferred compaction, between the readout over the memory of before the call (k_readout_finish) and the
-// merge: Eq. 5 over the memory after this call's write (Eq. 6-7), M' = lambda M + eta sum_e phi_e v_e^T,
-// b' = lambda b + eta sum_e phi_e^2 (applied only if something was evicted):
-//   m[col] = (decay P[col] + eta sum_e (phi_q . phi_e) v_e[col]) / (eps + decay D + eta sum_e sum_m phi_q[m]^2 phi_e[m]^2)
-// in place over P.  Needs phi of the evicted keys (K-split partials) but not the state update itself.
-// grid = n_seq, block = 256.
-__global__ void __launch_bounds__(256) k_readout_apply(ImDims p, ImState st, ImScratch sc, ImCall call) {
-  __shared__ float s_dot[IM_FRONT_MAX_NE][8], s_sq[IM_FRONT_MAX_NE][8];
-  const int i = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const size_t u = (size_t)call.layer * p.S + call.seq[i];
-  const int ne = max(0, min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], min(IM_FRONT_MAX_NE, p.F)));
-  float* mr = sc.mres + (size_t)i * (p.Dkv + 2);
-  const float D = mr[p.Dkv + 1];
-  const float* pq = sc.phiq + (size_t)i * p.dM;
-  for (int e = 0; e < ne; ++e) {
-    float dot = 0.f, sq = 0.f;
-    for (int m = tid; m < p.dM; m += 256) {
-      float f = 0.f;
-      for (int ks = 0; ks < call.ksplit_phi; ++ks) f += sc.phip[(((size_t)ks * call.n_seq + i) * p.F + e) * p.dM + m];
-      const float qf = pq[m];
-      dot = fmaf(qf, f, dot);
-      sq = fmaf(qf * qf, f * f, sq);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      dot += __shfl_xor_sync(0xffffffffu, dot, o);
-      sq += __shfl_xor_sync(0xffffffffu, sq, o);
-    }
-    if (lane == 0) { s_dot[e][warp] = dot; s_sq[e][warp] = sq; }
-  }
-  __syncthreads();
-  const float decay = ne > 0 ? p.lambda : 1.0f;
-  float den = p.eps + decay * D;
-  for (int e = 0; e < ne; ++e) {
-    float sq = 0.f;
-    for (int w = 0; w < 8; ++w) sq += s_sq[e][w];
-    den = fmaf(p.eta, sq, den);
-  }
-  for (int col = tid; col < p.Dkv; col += 256) {
-    float num = decay * mr[col];
-    for (int e = 0; e < ne; ++e) {
-      float dot = 0.f;
-      for (int w = 0; w < 8; ++w) dot += s_dot[e][w];
-      num = fmaf(p.eta * dot, __bfloat162float(sc.evV[((size_t)i * p.tail + e) * p.Dkv + col]), num);
-    }
-    mr[col] = num / den;
+    dst[p.Dkv + 2] = scale;  // coefficient of phi(q)^T Mhat, which the merge kernel adds
   }
 }
 
@@ -540,6 +524,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
                                                           const bf16* __restrict__ k_new, const bf16* __restrict__ v_new) {
   constexpr int CPL = DH / 32;  // columns per lane
   __shared__ float s_q[8][DH];  // recompute path: the warp's query row
+  __shared__ float s_dot[IM_FRONT_MAX_NE][8], s_sq[IM_FRONT_MAX_NE][8];  // readout terms of this call's write, per warp
   const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
@@ -549,25 +534,94 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
   const int na_lane = lane < call.n_seq ? sc.n_att[lane] : 0;
   const int ne_raw = st.ctr[u * CTR_STRIDE + CTR_NEVICT];
   const int ev_l = lane < IM_FRONT_MAX_NE ? st.ev_slot[u * p.tail + min(lane, p.tail - 1)] : -1;
-  const float* mr = sc.mres + (size_t)i * (p.Dkv + 2);
-  float gate = 0.f, mcol[CPL], qv[CPL], kn[CPL], vn[CPL], ek0[CPL], ev0[CPL];
+  const float* mr = sc.mres + (size_t)i * IM_MRES_ROW(p);
+  const float* rs = sc.rpart + (size_t)i * p.Dkv;  // phi(q)^T Mhat (k_readout_cols)
+  float pf0[4], pq0[4];
+  float gate = 0.f, c_hat = 0.f, den_old = 0.f, mcol[CPL], qv[CPL], kn[CPL], vn[CPL], ek0[CPL], ev0[CPL];
   {
     const bf16* qrow = q + ((size_t)i * p.H + (size_t)h * p.Gq + hh0) * DH;
     const bf16* kr = k_new + (size_t)i * p.Dkv + h * DH;
     const bf16* vr = v_new + (size_t)i * p.Dkv + h * DH;
     const bf16* ekr = sc.evK + (size_t)i * p.tail * p.Dkv + h * DH;
     const bf16* evr = sc.evV + (size_t)i * p.tail * p.Dkv + h * DH;
-    if (p.mem) gate = mr[p.Dkv];
+    if (p.mem) { gate = mr[p.Dkv]; c_hat = mr[p.Dkv + 2]; den_old = mr[p.Dkv + 1]; }
+    if (p.mem && call.defer) {  // slot 0 of the evicted entries' phi is read before the evicted count is known
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int m = tid + j * blockDim.x;
+        pf0[j] = 0.f;
+        pq0[j] = 0.f;
+        if (m < p.dM) {
+          for (int ks = 0; ks < call.ksplit_phi; ++ks) pf0[j] += sc.phip[((size_t)ks * call.n_seq + i) * p.F * p.dM + m];
+          pq0[j] = sc.phiq[(size_t)i * p.dM + m];
+        }
+      }
+    }
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
       const int c = lane + 32 * k;
-      mcol[k] = p.mem ? mr[h * DH + c] : 0.f;
+      mcol[k] = p.mem ? fmaf(c_hat, rs[h * DH + c], mr[h * DH + c]) : 0.f;
       qv[k] = __bfloat162float(qrow[c]);
       kn[k] = __bfloat162float(kr[c]);
       vn[k] = __bfloat162float(vr[c]);
       ek0[k] = call.defer ? __bfloat162float(ekr[c]) : 0.f;
       ev0[k] = call.defer ? __bfloat162float(evr[c]) : 0.f;
     }
+  }
+  // ---- deferred compaction: Eq. 5 over the memory AFTER this call's write (Eq. 6-7), M' = lambda M + eta sum_e
+  // phi_e v_e^T, b' = lambda b + eta sum_e phi_e^2 (applied only if something was evicted), from the parts of
+  // before the write: with P = s (phi(q)^T Mhat + pending terms) and the denominator sum D that k_readout_finish
+  // left,  m[col] = (decay P[col] + eta sum_e (phi_q . phi_e) v_e[col]) / (eps + decay D + eta sum_e sum_m
+  // phi_q[m]^2 phi_e[m]^2).  Needs phi of the evicted keys (K-split partials), not the state update itself.
+  if (p.mem && call.defer) {  // (block uniform)
+    const int ne_m = max(0, min(ne_raw, min(IM_FRONT_MAX_NE, p.F)));
+    const float* pq = sc.phiq + (size_t)i * p.dM;
+    for (int e = 0; e < ne_m; ++e) {
+      float dot = 0.f, sq = 0.f;
+      int m_first = tid;
+      if (e == 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          dot = fmaf(pq0[j], pf0[j], dot);
+          sq = fmaf(pq0[j] * pq0[j], pf0[j] * pf0[j], sq);
+        }
+        m_first = tid + 4 * blockDim.x;
+      }
+      for (int m = m_first; m < p.dM; m += blockDim.x) {
+        float f = 0.f;
+        for (int ks = 0; ks < call.ksplit_phi; ++ks) f += sc.phip[(((size_t)ks * call.n_seq + i) * p.F + e) * p.dM + m];
+        const float qf = pq[m];
+        dot = fmaf(qf, f, dot);
+        sq = fmaf(qf * qf, f * f, sq);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      }
+      if (lane == 0) { s_dot[e][warp] = dot; s_sq[e][warp] = sq; }
+    }
+    __syncthreads();
+    const float decay = ne_m > 0 ? p.lambda : 1.0f;
+    float den = p.eps + decay * den_old;
+    for (int e = 0; e < ne_m; ++e) {
+      float sq = 0.f;
+      for (int w = 0; w < nwarps; ++w) sq += s_sq[e][w];
+      den = fmaf(p.eta, sq, den);
+    }
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) mcol[k] *= decay;
+    for (int e = 0; e < ne_m; ++e) {
+      float dot = 0.f;
+      for (int w = 0; w < nwarps; ++w) dot += s_dot[e][w];
+      const bf16* evr = sc.evV + ((size_t)i * p.tail + e) * p.Dkv + h * DH;
+#pragma unroll
+      for (int k = 0; k < CPL; ++k)
+        mcol[k] = fmaf(p.eta * dot, e == 0 ? ev0[k] : __bfloat162float(evr[lane + 32 * k]), mcol[k]);
+    }
+    const float inv = 1.0f / den;
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) mcol[k] *= inv;
   }
   // ---- rebuild the tile bookkeeping of the attention kernel (lanes stride over the sequences)
   long long pref = 0, total = 0;
@@ -820,26 +874,34 @@ size_t im_attn_smem_bytes(const ImDims& p) {
 cudaError_t im_attn_prepare(const ImDims& p) {
   const int smem = (int)im_attn_smem_bytes(p);
   cudaError_t e = cudaFuncSetAttribute(k_attn_stream<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_attn_stream<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_attn_stream<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_stream<64>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_stream<128>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_readout_cols);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_readout_cols_light);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_readout_finish);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_merge_rows<64, bf16>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_merge_rows<64, float>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_merge_rows<128, bf16>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_merge_rows<128, float>);
+  return e;
 }
 
-cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call) {
+cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call, int grid, int light) {
   const ImDims& p = L.p;
-  dim3 grid((p.dM + R_ROWS - 1) / R_ROWS, call.n_seq);
-  k_readout<<<grid, 256, 0, L.stream>>>(p, L.st, L.sc, call);
+  const int depth = light ? 8 : 32;
+  const int nb = (p.dM + RC_RPR * depth - 1) / (RC_RPR * depth);
+  const int items = call.n_seq * (p.Dkv / RC_COLS);
+  const size_t smem = (size_t)nb * RC_RPR * depth * 4;
+  const int blocks = std::max(1, std::min(grid, items));
+  if (light) k_readout_cols_light<<<blocks, RC_THREADS, smem, L.stream>>>(p, L.st, L.sc, call);
+  else k_readout_cols<<<blocks, RC_THREADS, smem, L.stream>>>(p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
 }
 
 cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call) {
   k_readout_finish<<<call.n_seq, 256, (size_t)L.p.dM * 4, L.stream>>>(L.p, L.st, L.w, L.sc, call);
-  ++*L.launches;
-  return cudaGetLastError();
-}
-
-cudaError_t im_launch_readout_apply(const ImLaunch& L, const ImCall& call) {
-  k_readout_apply<<<call.n_seq, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
 }

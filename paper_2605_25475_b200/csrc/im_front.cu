@@ -333,18 +333,19 @@ __global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, Im
 }  // namespace
 
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
-                                   int do_select, int n_max) {
+                                   int do_select, int n_max, int smem_floor) {
   static bool attr_done_dev[64] = {};
   bool* attr_done = im_device_flag(attr_done_dev);
   if (!attr_done || !*attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_decode_front<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_FRONT_MAX_N * 8 + 64 * 64 * 4);
+    cudaError_t e = cudaFuncSetAttribute(k_decode_front<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_FRONT);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_FRONT);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_decode_front<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_FRONT);
     if (e != cudaSuccess) return e;
     if (attr_done) *attr_done = true;
   }
   const int key_slots = do_select ? n_max : 0;
-  const size_t smem = (size_t)key_slots * 8 + (size_t)L.p.HI * L.p.dI * 4;
+  size_t smem = (size_t)key_slots * 8 + (size_t)L.p.HI * L.p.dI * 4;
+  if (smem < (size_t)smem_floor) smem = (size_t)smem_floor;  // keeps the streaming kernels' blocks off this block's SM
   const bf16* kn = (const bf16*)k_new;
   const bf16* vn = (const bf16*)v_new;
   if (L.p.dI == 16) k_decode_front<16><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
@@ -372,4 +373,12 @@ cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_
   k_move_survivors<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
+}
+
+cudaError_t im_front_prepare_decode() {
+  cudaError_t e = im_prefer_max_smem(k_decode_front<0>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_decode_front<8>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_decode_front<16>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_move_survivors);
+  return e;
 }

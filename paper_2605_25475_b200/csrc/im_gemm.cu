@@ -295,8 +295,8 @@ cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
     int tiles = 0;
     for (int j = 0; j < a.n_jobs; ++j) tiles += (a.job[j].rows + 15) / 16;
     dim3 grid(tiles, a.ksplit, (unsigned)((a.NV + VB - 1) / VB));
-    if (n_w2) k_direct_gemm<true><<<grid, DG_WARPS * 32, 0, L.stream>>>(a);
-    else k_direct_gemm<false><<<grid, DG_WARPS * 32, 0, L.stream>>>(a);
+    if (n_w2) k_direct_gemm<true><<<grid, DG_WARPS * 32, (size_t)std::max(0, a.smem_floor), L.stream>>>(a);
+    else k_direct_gemm<false><<<grid, DG_WARPS * 32, (size_t)std::max(0, a.smem_floor), L.stream>>>(a);
     ++*L.launches;
     return cudaGetLastError();
   }
@@ -317,4 +317,14 @@ cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, i
   k_proj_key_split<<<grid, 256, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
   ++*L.launches;
   return cudaGetLastError();
+}
+
+cudaError_t im_gemm_prepare_decode() {
+  cudaError_t e = im_prefer_max_smem(k_direct_gemm<false>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_direct_gemm<true>);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_direct_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_SIDE);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_direct_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_SIDE);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_skinny_gemm);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_split);
+  return e;
 }

@@ -13,7 +13,6 @@ typedef __nv_bfloat16 bf16;
 #define IM_ATTN_TILE 32      /* keys per attention tile (one TMA box is 32 rows x 128 bytes) */
 #define IM_ATTN_WARPS 4      /* warps per CTA of the streaming attention kernel */
 #define IM_ATTN_MAX_CTAS 512 /* upper bound of its grid (one CTA per SM) */
-#define IM_READOUT_ROWS 32   /* rows of M per readout partial */
 #define IM_TC_QT 32          /* queries per tile of the tensor-core prefill scoring */
 #define IM_TC_HP 8           /* head slots per query in its operand (indexer heads, zero padded) */
 #define IM_TC_TILE_BYTES 25600 /* one tile record: 3 bf16 terms x (256 rows x 32 bytes) + 256 alpha floats */
@@ -98,10 +97,10 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
   int32_t* nhole;    // [max_seqs]             compaction: number of evicted slots below the budget
   float* part;       // attention partials (acc[d], max, sum): generic kernel [max_seqs][H][max_splits][d + 2];
                      // streaming kernel [warps + rows][Gq][d + 2]
-  float* rpart;      // [max_seqs][ceil(dM / IM_READOUT_ROWS)][Dkv] readout partials
-  float* mres;       // [max_seqs][Dkv + 2] memory readout in KV space, the gate g(q), the denominator sum.  In a call
-                     // with deferred compaction: numerator and denominator sum of Eq. 5 over the state from before
-                     // the call's memory write (the merge adds the write's terms); otherwise the final m(q), gate, -
+  float* rpart;      // [max_seqs][Dkv] readout numerators: phi(q)^T Mhat
+  float* mres;       // [max_seqs][IM_MRES_ROW] per column the part of the memory readout (Eq. 5) that does not go
+                     // through Mhat (pending list, entries written in this call), then the gate g(q), the denominator
+                     // sum, and the coefficient c of the Mhat part: m(q)[col] = mres[col] + c * rpart[col]
   float* phiq;       // [max_seqs][dM] phi(q) of the call (K-split partials summed)
   int32_t* n_att;    // [max_seqs] entries per sequence the streaming attention kernel of the call ran over
   bf16* phiT;        // [2][dM][KE] phi of one sequence's evicted keys, transposed, as two bf16 terms (KE = tail rounded up to 64)
@@ -145,6 +144,7 @@ struct ImGemmArgs {
   int tensor;  // 1: thousands of vectors (prefill) - the tcgen05 variant where it applies (im_tc_gemm_usable)
   int direct;  // 1: few vectors (decode) - the variant without shared-memory staging, if the K split is a multiple of 32
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
+  int smem_floor;  // direct variant: dynamic shared memory to ask for although the kernel uses none (IM_SMEM_SIDE)
   // tensor-core variant only:
   int out_t;            // 1: the result goes to out[(row0 + r) * out_outer + v] (vectors contiguous) instead
   int rmw;              // 1: out = beta * out + alpha * result
@@ -176,6 +176,35 @@ inline bool* im_device_flag(bool (&flags)[64]) {
   return &flags[dev];
 }
 
+// An SM changes its shared-memory carveout only while it is idle.  The streaming attention kernel needs the largest
+// one; every kernel that runs next to it or shortly before it asks for the same, so that attention CTAs never wait
+// for resident blocks of a kernel with a smaller carveout to drain.
+template <typename F>
+inline cudaError_t im_prefer_max_smem(F* kernel) {
+  return cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel), cudaFuncAttributePreferredSharedMemoryCarveout,
+                              (int)cudaSharedmemCarveoutMaxShared);
+}
+cudaError_t im_gemm_prepare_decode();
+cudaError_t im_memory_prepare_decode();
+cudaError_t im_front_prepare_decode();
+cudaError_t im_prefetch_prepare_decode();
+
+#define IM_MRES_ROW(p) ((p).Dkv + 4)
+
+// Decode calls of few sequences split the SMs between the two kinds of work of a call: the streaming kernels
+// (attention over the cache, readout over Mhat), bound by HBM bandwidth, and the chain of small kernels that
+// decides what the call evicts (front kernel, phi of the evicted keys), bound by memory latency, which runs
+// several times slower on an SM whose load queues a streaming block keeps full.  The split is made by the
+// occupancy rules alone: a front block asks for so much shared memory that no attention CTA fits next to it,
+// and the attention grid is n_res blocks short of the SM count (n_res = number of front blocks), so that
+// wherever its CTAs land, n_res SMs are left to the front kernel.  The readout kernel, whose blocks would settle
+// on just those SMs (the emptiest), starts when the front kernel has ended; the phi GEMM that follows the front
+// kernel asks for more shared memory than an SM with an attention CTA has left and ends up on the SMs the front
+// kernel has just freed.
+#define IM_SMEM_FRONT (192 * 1024)   /* front block: excludes attention CTAs (>= 64 KB of shared memory each) */
+#define IM_SMEM_SIDE (38 * 1024)     /* phi GEMM block (+ 17 KB static): four per free SM, at most one next to an attention CTA */
+inline int im_reserved_sms(int n_sm, int n_seq) { return n_seq <= n_sm / 4 ? n_seq : 0; }
+
 // records `msg` as the calling thread's last error and returns `code` (defined next to im_last_error)
 int im_fail_message(int code, const char* msg);
 
@@ -186,7 +215,7 @@ bool im_tc_gemm_usable(const ImGemmArgs& a);
 cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a);
 cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, int ksplit);
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
-                                   int do_select, int n_max);
+                                   int do_select, int n_max, int smem_floor);
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call);
@@ -214,9 +243,9 @@ cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const voi
 bool im_attn_fast_supported(const ImDims& p);
 cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV);
 cudaError_t im_attn_prepare(const ImDims& p);
-cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call);
+// grid blocks (at most one per SM wanted); light: the variant that leaves room for a front block on its SM
+cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call, int grid, int light);
 cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call);
-cudaError_t im_launch_readout_apply(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
                                      const void* q, int n_ctas);
 cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas, const void* q,

@@ -333,3 +333,10 @@ cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_m
   ++*L.launches;
   return cudaGetLastError();
 }
+
+cudaError_t im_memory_prepare_decode() {
+  cudaError_t e = im_prefer_max_smem(k_mem_fold);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_mem_fold_commit);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_mem_small);
+  return e;
+}

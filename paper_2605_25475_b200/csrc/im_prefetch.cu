@@ -61,3 +61,5 @@ cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call) {
   ++*L.launches;
   return cudaGetLastError();
 }
+
+cudaError_t im_prefetch_prepare_decode() { return im_prefer_max_smem(k_prefetch_layer); }
