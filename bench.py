@@ -160,35 +160,32 @@ def run_ours(args, rank, world, device):
     L = wl.n_layers
     n_in = min(8, args.steps + args.warmup)                      # distinct input sets, cycled
     inputs = decode_inputs_all(wl, n_in, device)
-    sx, sq, sk, sv = [torch.empty_like(t) for t in inputs[0]]    # static buffers the graph reads
     out = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=device)
 
-    def one_step():
+    def one_step(k):
+        x, q, kk, v = inputs[k % n_in]
         for layer in range(L):
-            g.decode_step(layer, ids, sx[layer], sq[layer], sq[layer], sk[layer], sv[layer], out[layer])
-
-    def load(step):
-        x, q, k, v = inputs[step % n_in]
-        sx.copy_(x); sq.copy_(q); sk.copy_(k); sv.copy_(v)
+            g.decode_step(layer, ids, x[layer], q[layer], q[layer], kk[layer], v[layer], out[layer])
 
     stream = torch.cuda.Stream(device)
-    graph = None
+    graphs = None
     launches_per_step = None
     with torch.cuda.stream(stream):
-        load(0)
         c0 = g.launch_count()
-        one_step()                                               # reaches the steady state n = B
+        one_step(0)                                              # reaches the steady state n = B
         launches_per_step = g.launch_count() - c0
         stream.synchronize()
         if args.graph:
-            graph = torch.cuda.CUDAGraph()
-            load(1)
-            with torch.cuda.graph(graph, stream=stream):
-                one_step()
-        step_fn = graph.replay if graph is not None else one_step
+            # one captured step per input set: the graph reads the resident inputs where they are
+            graphs = []
+            for k in range(n_in):
+                gk = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gk, stream=stream):
+                    one_step(k)
+                graphs.append(gk)
+        step_fn = (lambda k: graphs[k % n_in].replay()) if graphs is not None else one_step
         for w in range(args.warmup):
-            load(w + 2)
-            step_fn()
+            step_fn(w + 1)
         stream.synchronize()
         barrier(world)
         sampler = ClockSampler(torch.cuda.current_device() if device.index is None else device.index)
@@ -199,8 +196,7 @@ def run_ours(args, rank, world, device):
         rec0 = im.im_event_count(g.ctx, im.IM_COUNT_MERGE_RECOMPUTE)
         ev0.record(stream)
         for s in range(args.steps):
-            load(args.warmup + 2 + s)
-            step_fn()
+            step_fn(args.warmup + 1 + s)
         ev1.record(stream)
         torch.cuda.synchronize()
         barrier(world)
@@ -216,8 +212,7 @@ def run_ours(args, rank, world, device):
         im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 0)
         im.im_profile_begin(g.ctx, args.steps * L)
         for s in range(args.steps):
-            load(s)
-            one_step()
+            one_step(s)
         attn_ms, attn_n = im.im_profile_end(g.ctx)
         im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 1)
 
@@ -236,7 +231,7 @@ def run_ours(args, rank, world, device):
         "config": {"workload": wl.name + ("" if not (args.layers or args.context) else " (reduced for profiling)"),
                    "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H,
                    "kv_heads": wl.Hkv, "head_dim": wl.d, "context": wl.ctx, "budget": wl.B, "tau": wl.tau,
-                   "cuda_graph": bool(args.graph),
+                   "cuda_graph": graphs is not None,
                    "l2": "inputs larger than L2 (each step streams %.1f GB)" % (ab["step"] / 1e9)},
         "hbm_gbs_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9,
         "hbm_frac_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"],

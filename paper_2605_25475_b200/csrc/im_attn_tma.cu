@@ -517,13 +517,16 @@ __device__ __forceinline__ void softmax_push(float s, const float (&v)[CPL], flo
 // (Eq. 4) is recovered exactly: the new token's term is added, the evicted entries' terms
 // exp(s_e) (1, v_e) are taken out of the sums again.  Taking out is safe in float32 while the evicted
 // entries hold at most 90 % of the softmax mass (the error of the remainder grows by at most 10); beyond
-// that the warp recomputes its head over the retained entries from the cache, which is still uncompacted.
+// that the block's warps together recompute, from the cache, which is still uncompacted, the partials of that
+// head whose key range holds an evicted entry.
 template <int DH, typename OutT>
 __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st, ImScratch sc, ImCall call, int n_ctas,
                                                           OutT* __restrict__ out, const bf16* __restrict__ q,
                                                           const bf16* __restrict__ k_new, const bf16* __restrict__ v_new) {
   constexpr int CPL = DH / 32;  // columns per lane
-  __shared__ float s_q[8][DH];  // recompute path: the warp's query row
+  __shared__ float s_q[8][DH];       // redo path: the query rows of the heads to redo
+  __shared__ float s_st[8][DH + 2];  // redo path: the warps' softmax states of a key range
+  __shared__ int s_redo[8];
   __shared__ float s_dot[IM_FRONT_MAX_NE][8], s_sq[IM_FRONT_MAX_NE][8];  // readout terms of this call's write, per warp
   const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
@@ -653,139 +656,66 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
   const long long row_id = (long long)i * p.Hkv + h;
   const int ne = call.defer ? max(0, min(ne_raw, IM_FRONT_MAX_NE)) : 0;
   const float sl2 = p.scale * 1.4426950408889634f;
-  // ---- one warp per query head of the group
-  for (int hh = warp; hh < p.Gq; hh += nwarps) {
+  // ---- one warp per query head of the group (the block has at least Gq warps)
+  const bf16* Kb = st.Kc + (u * p.Hkv + h) * (size_t)p.cap * DH;
+  const bf16* Vb = st.Vc + (u * p.Hkv + h) * (size_t)p.cap * DH;
+  const bool has_head = warp < p.Gq;
+  const int hh = hh0;
+  const long long w0 = nt_i > 0 ? row_first / qrun : 0, w1 = nt_i > 0 ? row_last / qrun : -1;
+  // keys of partial wv of this row: the tiles of the row that fall into run wv
+  auto partial_keys = [&](long long wv, int& key0, int& key1) {
+    const int lt0 = (int)(max(wv * qrun, row_first) - row_first);
+    const int lt1 = (int)(min((wv + 1) * qrun - 1, row_last) - row_first);
+    key0 = lt0 * TILE;
+    key1 = min((lt1 + 1) * TILE, n_old);
+  };
+  auto merge_stored = [&](long long wv, int head, float& M, float& L, float (&res)[CPL]) {
+    const float* ps = sc.part + ((size_t)(wv + row_id) * p.Gq + head) * (DH + 2);
+    const float mw = ps[DH], lw = ps[DH + 1];
+    float a[CPL];
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) a[k] = ps[lane + 32 * k];
+    const float Mn = fmaxf(M, mw);
+    const float eo = exp2f(M - Mn), en = exp2f(mw - Mn);  // exp2(-inf) = 0 for the first contributor
+    L = L * eo + lw * en;
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[k] * en;
+    M = Mn;
+  };
+  bool new_kept = true;
+  for (int a = 0; a < ne; ++a) new_kept &= __shfl_sync(0xffffffffu, ev_l, a) != n_old;
+  auto push_new = [&](float& M, float& L, float (&res)[CPL]) {
+    if (!new_kept) return;
+    float dot = 0.f;
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) dot = fmaf(qv[k], kn[k], dot);
+    softmax_push<CPL>(warp_sum_f(dot) * sl2, vn, M, L, res);
+  };
+  auto store_head = [&](float L, float (&res)[CPL]) {
+    if (L > 0.f) {
+      const float inv = 1.0f / L;
+#pragma unroll
+      for (int k = 0; k < CPL; ++k) res[k] *= inv;
+    }
+    const size_t base = ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH;
+#pragma unroll
+    for (int k = 0; k < CPL; ++k) {
+      const float v = res[k] + gate * mcol[k];  // Eq. 4: attention over the retained set + gated memory readout
+      if constexpr (sizeof(OutT) == 2) out[base + lane + 32 * k] = __float2bfloat16_rn(v);
+      else out[base + lane + 32 * k] = v;
+    }
+  };
+  // Pass 0 merges the stored partials and, with deferred compaction, takes the evicted entries' terms out of the
+  // sums.  A head whose evicted entries hold more than 90 % of the mass is redone below.
+  bool redo = false;
+  if (has_head) {
     float res[CPL];
 #pragma unroll
     for (int k = 0; k < CPL; ++k) res[k] = 0.f;
     float M = NEG_INF, L = 0.f;
-    if (call.defer && hh != hh0) {  // a warp with a second head (blocks with fewer warps than heads): its query row
-      const bf16* qrow = q + ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH;
-#pragma unroll
-      for (int k = 0; k < CPL; ++k) qv[k] = __bfloat162float(qrow[lane + 32 * k]);
-    }
-    const bf16* Kb = st.Kc + (u * p.Hkv + h) * (size_t)p.cap * DH;
-    const bf16* Vb = st.Vc + (u * p.Hkv + h) * (size_t)p.cap * DH;
-    // Pass 0 merges the stored partials; with deferred compaction it then takes the evicted entries' terms
-    // out of the sums.  If those hold more than 90 % of the mass, pass 1 starts over and recomputes, from the
-    // cache, the partials whose key range holds an evicted entry (without it); the others are exact already.
-    for (int pass = 0; pass < 2; ++pass) {
-      M = NEG_INF;
-      L = 0.f;
-#pragma unroll
-      for (int k = 0; k < CPL; ++k) res[k] = 0.f;
-      if (nt_i > 0) {
-        const long long w0 = row_first / qrun, w1 = row_last / qrun;
-        for (long long wv = w0; wv <= w1; ++wv) {
-          // keys of this partial: the tiles of the row that fall into run wv
-          const int lt0 = (int)(max(wv * qrun, row_first) - row_first);
-          const int lt1 = (int)(min((wv + 1) * qrun - 1, row_last) - row_first);
-          const int key0 = lt0 * TILE, key1 = min((lt1 + 1) * TILE, n_old);
-          bool dirty = false;
-          if (pass == 1)
-            for (int a = 0; a < ne; ++a) {
-              const int sl = __shfl_sync(0xffffffffu, ev_l, a);
-              dirty |= sl >= key0 && sl < key1;
-            }
-          if (!dirty) {
-            const float* ps = sc.part + ((size_t)(wv + row_id) * p.Gq + hh) * (DH + 2);
-            const float mw = ps[DH], lw = ps[DH + 1];
-            float a[CPL];
-#pragma unroll
-            for (int k = 0; k < CPL; ++k) a[k] = ps[lane + 32 * k];
-            const float Mn = fmaxf(M, mw);
-            const float eo = exp2f(M - Mn), en = exp2f(mw - Mn);  // exp2(-inf) = 0 for the first contributor
-            L = L * eo + lw * en;
-#pragma unroll
-            for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[k] * en;
-            M = Mn;
-          } else {
-            // One key per lane, 32 keys per round: the lane forms its key's whole dot product (q from shared
-            // memory; 16 independent 16-byte loads), then the warp adds the 32 weighted V rows, lane l holding
-            // columns CPL l .. CPL l + CPL - 1 (32 independent loads).  An evicted key gets the weight 0.  The
-            // range's own softmax state is merged like a stored partial at the end.
-            float* sq = s_q[warp];
-#pragma unroll
-            for (int k = 0; k < CPL; ++k) sq[lane + 32 * k] = qv[k];
-            __syncwarp();
-            float Mr = NEG_INF, Lr = 0.f, racc[CPL];
-#pragma unroll
-            for (int k = 0; k < CPL; ++k) racc[k] = 0.f;
-            for (int t0 = key0; t0 < key1; t0 += 32) {
-              const int tk = t0 + lane;
-              bool valid = tk < key1;
-              for (int a = 0; a < ne; ++a) valid &= __shfl_sync(0xffffffffu, ev_l, a) != tk;
-              const uint4* kr = reinterpret_cast<const uint4*>(Kb + (size_t)min(tk, key1 - 1) * DH);
-              uint4 kw[DH / 8];
-#pragma unroll
-              for (int c = 0; c < DH / 8; ++c) kw[c] = kr[c];
-              uint2 vw[32];
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const bf16* vr = Vb + (size_t)min(t0 + j, key1 - 1) * DH + CPL * lane;
-                if (CPL == 4) vw[j] = *reinterpret_cast<const uint2*>(vr);
-                else { vw[j].x = *reinterpret_cast<const uint32_t*>(vr); vw[j].y = 0u; }
-              }
-              float sd = 0.f;
-#pragma unroll
-              for (int c = 0; c < DH / 8; ++c) {
-                const uint32_t ww[4] = {kw[c].x, kw[c].y, kw[c].z, kw[c].w};
-#pragma unroll
-                for (int e2 = 0; e2 < 4; ++e2) {
-                  sd = fmaf(sq[c * 8 + 2 * e2], __uint_as_float(ww[e2] << 16), sd);
-                  sd = fmaf(sq[c * 8 + 2 * e2 + 1], __uint_as_float(ww[e2] & 0xffff0000u), sd);
-                }
-              }
-              sd = valid ? sd * sl2 : NEG_INF;
-              float mb = sd;
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, o));
-              if (mb == NEG_INF) continue;  // (warp-uniform) nothing left in this round
-              const float Mn = fmaxf(Mr, mb);
-              const float eo = exp2f(Mr - Mn);
-              const float pl = valid ? exp2f(sd - Mn) : 0.f;
-              Lr = Lr * eo + warp_sum_f(pl);
-#pragma unroll
-              for (int k = 0; k < CPL; ++k) racc[k] *= eo;
-              Mr = Mn;
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float pj = __shfl_sync(0xffffffffu, pl, j);
-                racc[0] = fmaf(pj, __uint_as_float(vw[j].x << 16), racc[0]);
-                racc[1] = fmaf(pj, __uint_as_float(vw[j].x & 0xffff0000u), racc[1]);
-                if (CPL == 4) {
-                  racc[2] = fmaf(pj, __uint_as_float(vw[j].y << 16), racc[2]);
-                  racc[3] = fmaf(pj, __uint_as_float(vw[j].y & 0xffff0000u), racc[3]);
-                }
-              }
-            }
-            // columns CPL l + k -> l + 32 k through the warp's shared row, then the usual merge
-            __syncwarp();
-#pragma unroll
-            for (int k = 0; k < CPL; ++k) sq[CPL * lane + k] = racc[k];
-            __syncwarp();
-            if (Lr > 0.f) {
-              const float Mn = fmaxf(M, Mr);
-              const float eo = exp2f(M - Mn), en = exp2f(Mr - Mn);
-              L = L * eo + Lr * en;
-#pragma unroll
-              for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + sq[lane + 32 * k] * en;
-              M = Mn;
-            }
-            __syncwarp();
-          }
-        }
-      }
-      if (!call.defer) break;
-      bool new_kept = true;
-      for (int a = 0; a < ne; ++a) new_kept &= __shfl_sync(0xffffffffu, ev_l, a) != n_old;
-      if (new_kept) {
-        float dot = 0.f;
-#pragma unroll
-        for (int k = 0; k < CPL; ++k) dot = fmaf(qv[k], kn[k], dot);
-        softmax_push<CPL>(warp_sum_f(dot) * sl2, vn, M, L, res);
-      }
-      if (pass == 1) break;
+    for (long long wv = w0; wv <= w1; ++wv) merge_stored(wv, hh, M, L, res);
+    if (call.defer) {
+      push_new(M, L, res);
       float Lsub = 0.f, sub[CPL];
 #pragma unroll
       for (int k = 0; k < CPL; ++k) sub[k] = 0.f;
@@ -813,24 +743,122 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
         L -= Lsub;
 #pragma unroll
         for (int k = 0; k < CPL; ++k) res[k] -= sub[k];
-        break;
+      } else {
+        redo = true;  // the evicted entries dominate this head's softmax
+        if (lane == 0) atomicAdd(st.status + 1, 1);
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) s_q[warp][lane + 32 * k] = qv[k];
       }
-      if (lane == 0) atomicAdd(st.status + 1, 1);  // the evicted entries dominate this head's softmax
     }
-    if (L > 0.f) {
-      const float inv = 1.0f / L;
+    if (!redo) store_head(L, res);
+  }
+  if (!call.defer) return;  // (block uniform)
+  if (lane == 0) s_redo[warp] = redo ? 1 : 0;
+  __syncthreads();
+  // Redo of a head, by all warps of the block: the partials whose key range holds an evicted entry are recomputed
+  // from the cache, which is still uncompacted, without that entry (the others are exact already).  The 32-key
+  // rounds of such a range go round-robin over the warps; within a round a lane forms its key's whole dot product
+  // (q from shared memory; 16 independent 16-byte loads), then the warp adds the 32 weighted V rows, lane l holding
+  // columns CPL l .. CPL l + CPL - 1 (32 independent loads).  The warps' softmax states are merged in warp order by
+  // the warp that owns the head, like stored partials.
+  for (int hq = 0; hq < p.Gq; ++hq) {
+    if (!s_redo[hq]) continue;  // (block uniform)
+    const bool owner = warp == hq;
+    float res[CPL];
 #pragma unroll
-      for (int k = 0; k < CPL; ++k) res[k] *= inv;
+    for (int k = 0; k < CPL; ++k) res[k] = 0.f;
+    float M = NEG_INF, L = 0.f;
+    for (long long wv = w0; wv <= w1; ++wv) {
+      int key0, key1;
+      partial_keys(wv, key0, key1);
+      bool dirty = false;
+      for (int a = 0; a < ne; ++a) {
+        const int sl = __shfl_sync(0xffffffffu, ev_l, a);
+        dirty |= sl >= key0 && sl < key1;
+      }
+      if (!dirty) {
+        if (owner) merge_stored(wv, hq, M, L, res);
+        continue;
+      }
+      const float* sq = s_q[hq];
+      float Mr = NEG_INF, Lr = 0.f, racc[CPL];
+#pragma unroll
+      for (int k = 0; k < CPL; ++k) racc[k] = 0.f;
+      for (int t0 = key0 + 32 * warp; t0 < key1; t0 += 32 * nwarps) {
+        const int tk = t0 + lane;
+        bool valid = tk < key1;
+        for (int a = 0; a < ne; ++a) valid &= __shfl_sync(0xffffffffu, ev_l, a) != tk;
+        const uint4* kr = reinterpret_cast<const uint4*>(Kb + (size_t)min(tk, key1 - 1) * DH);
+        uint4 kw[DH / 8];
+#pragma unroll
+        for (int c = 0; c < DH / 8; ++c) kw[c] = kr[c];
+        uint2 vw[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const bf16* vr = Vb + (size_t)min(t0 + j, key1 - 1) * DH + CPL * lane;
+          if (CPL == 4) vw[j] = *reinterpret_cast<const uint2*>(vr);
+          else { vw[j].x = *reinterpret_cast<const uint32_t*>(vr); vw[j].y = 0u; }
+        }
+        float sd = 0.f;
+#pragma unroll
+        for (int c = 0; c < DH / 8; ++c) {
+          const uint32_t ww[4] = {kw[c].x, kw[c].y, kw[c].z, kw[c].w};
+#pragma unroll
+          for (int e2 = 0; e2 < 4; ++e2) {
+            sd = fmaf(sq[c * 8 + 2 * e2], __uint_as_float(ww[e2] << 16), sd);
+            sd = fmaf(sq[c * 8 + 2 * e2 + 1], __uint_as_float(ww[e2] & 0xffff0000u), sd);
+          }
+        }
+        sd = valid ? sd * sl2 : NEG_INF;
+        float mb = sd;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+        if (mb == NEG_INF) continue;  // (warp-uniform) nothing left in this round
+        const float Mn = fmaxf(Mr, mb);
+        const float eo = exp2f(Mr - Mn);
+        const float pl = valid ? exp2f(sd - Mn) : 0.f;
+        Lr = Lr * eo + warp_sum_f(pl);
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) racc[k] *= eo;
+        Mr = Mn;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float pj = __shfl_sync(0xffffffffu, pl, j);
+          racc[0] = fmaf(pj, __uint_as_float(vw[j].x << 16), racc[0]);
+          racc[1] = fmaf(pj, __uint_as_float(vw[j].x & 0xffff0000u), racc[1]);
+          if (CPL == 4) {
+            racc[2] = fmaf(pj, __uint_as_float(vw[j].y << 16), racc[2]);
+            racc[3] = fmaf(pj, __uint_as_float(vw[j].y & 0xffff0000u), racc[3]);
+          }
+        }
+      }
+      // this warp's state of the range: columns CPL l + k -> l + 32 k through shared memory
+      float* stw = s_st[warp];
+#pragma unroll
+      for (int k = 0; k < CPL; ++k) stw[CPL * lane + k] = racc[k];
+      if (lane == 0) { stw[DH] = Mr; stw[DH + 1] = Lr; }
+      __syncthreads();
+      if (owner) {
+        for (int w = 0; w < nwarps; ++w) {
+          const float Mw = s_st[w][DH], Lw = s_st[w][DH + 1];
+          if (!(Lw > 0.f)) continue;
+          const float Mn = fmaxf(M, Mw);
+          const float eo = exp2f(M - Mn), en = exp2f(Mw - Mn);
+          L = L * eo + Lw * en;
+#pragma unroll
+          for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + s_st[w][lane + 32 * k] * en;
+          M = Mn;
+        }
+      }
+      __syncthreads();
     }
-    const size_t base = ((size_t)i * p.H + (size_t)h * p.Gq + hh) * DH;
-#pragma unroll
-    for (int k = 0; k < CPL; ++k) {
-      const float v = res[k] + gate * mcol[k];  // Eq. 4: attention over the retained set + gated memory readout
-      if constexpr (sizeof(OutT) == 2) out[base + lane + 32 * k] = __float2bfloat16_rn(v);
-      else out[base + lane + 32 * k] = v;
+    if (owner) {
+      push_new(M, L, res);
+      store_head(L, res);
     }
   }
 }
+
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
