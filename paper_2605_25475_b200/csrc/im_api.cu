@@ -675,7 +675,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
       CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
     }
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
-    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas));
+    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas, n_res > 0 ? 1 : 0));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
     CK(cudaEventRecord(ctx->ev[9], s0));  // the attention kernel has read the cache
   }
@@ -752,7 +752,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   if (ctx->fast_attn) {
     if (!conc) {
       if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
-      CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas));
+      CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas, 0));
       if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
     }
     if (!defer && p.mem) CKL(im_launch_readout_finish(L, call));  // after the memory write
@@ -761,7 +761,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
       CK(cudaStreamWaitEvent(s0, ctx->ev[12], 0));  // s2
       CK(cudaStreamWaitEvent(s0, ctx->ev[4], 0));   // s4
     }
-    CKL(im_launch_attention_merge(L, call, out, n_ctas, q, k_new, v_new));
+    CKL(im_launch_attention_merge(L, call, out, n_ctas, q, k_new, v_new, conc ? 1 : 0));
     if (defer && !conc) CKL(im_launch_decode_commit(L, call));
     if (conc) CK(cudaStreamWaitEvent(s0, ctx->ev[10], 0));
     if (conc) {  // the memory write only has to end with the call

@@ -125,7 +125,6 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   for (int i = threadIdx.x; i < call.n_seq; i += blockDim.x) {
     const size_t u = (size_t)call.layer * p.S + call.seq[i];
     s_n[i] = max(0, min(st.ctr[u * CTR_STRIDE + CTR_N], p.cap));
-    if (blockIdx.x == 0) sc.n_att[i] = s_n[i];  // what the merge kernel rebuilds the tile bookkeeping from
   }
   if (lane == 0) {
     for (int s = 0; s < STAGES; ++s) mbar_init(smem_u32(&bars[warp * STAGES + s]), 1);
@@ -147,11 +146,11 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   const long long qrun = (total + WT - 1) / WT;
   const long long wglob = (long long)blockIdx.x * WARPS + warp;
   const long long run0 = min(total, wglob * qrun), run1 = min(total, run0 + qrun);
-  if (run0 >= run1) return;
+  const bool has_work = run0 < run1;
 
   // ---- position of the first tile of the run: sequence i, KV head h, tile tt
   int i = 0;
-  {
+  if (has_work) {
     int lo = 0, hi = call.n_seq;  // last i with s_pref[i] <= run0
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
@@ -160,8 +159,8 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     i = lo;
     while (i < call.n_seq - 1 && tiles_of(s_n[i]) == 0) ++i;  // empty sequences own no tiles
   }
-  int nt = tiles_of(s_n[i]);
-  int h = (int)((run0 - s_pref[i]) / nt), tt = (int)((run0 - s_pref[i]) % nt);
+  int nt = max(1, tiles_of(s_n[i]));
+  int h = has_work ? (int)((run0 - s_pref[i]) / nt) : 0, tt = has_work ? (int)((run0 - s_pref[i]) % nt) : 0;
 
   const uint64_t pol = policy_evict_first();
   // iterator used by the producer side (runs STAGES tiles ahead of the consumer side)
@@ -192,6 +191,14 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   if (lane == 0) {
     for (int k = 0; k < STAGES && issued < run1; ++k) issue(issued++);
   }
+  // Launched as a programmatic dependent (of the previous call's merge kernel, or of whatever precedes the call in
+  // the caller's stream) the kernel may have come this far before that kernel has ended: the cache of this layer,
+  // which the first tiles are being fetched from, is not that kernel's business, but the query rows may be its
+  // output and the partials and entry counts of this call overwrite what the previous call's merge still reads.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (blockIdx.x == 0)  // what the merge kernel rebuilds the tile bookkeeping from
+    for (int k = threadIdx.x; k < call.n_seq; k += blockDim.x) sc.n_att[k] = s_n[k];
+  if (!has_work) return;
 
   const float sl2 = p.scale * 1.4426950408889634f;  // softmax in base 2
   bool ok = true;
@@ -291,7 +298,12 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
       // ---- the stage is free again: refill it
       __syncwarp();
-      if (lane == 0 && issued < run1) issue(issued++);
+      if (lane == 0 && issued < run1) {
+        issue(issued++);
+        // the last tile of this warp's run is requested: a kernel launched as programmatic dependent (the merge)
+        // may become resident and run the part of its prologue that does not read this kernel's output
+        if (issued == run1) asm volatile("griddepcontrol.launch_dependents;");
+      }
     }
     if (!ok) break;
     // ---- segment finished: write the partial (unnormalised O, max, sum) of this row
@@ -528,13 +540,14 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
   __shared__ float s_st[8][DH + 2];  // redo path: the warps' softmax states of a key range
   __shared__ int s_redo[8];
   __shared__ float s_dot[IM_FRONT_MAX_NE][8], s_sq[IM_FRONT_MAX_NE][8];  // readout terms of this call's write, per warp
+  // the next call's attention kernel may become resident and start fetching its first tiles
+  asm volatile("griddepcontrol.launch_dependents;");
   const int h = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int hh0 = min(warp, p.Gq - 1);  // the head this warp merges first (usually its only one)
   // ---- every load whose address depends on no other load is issued here, ahead of its use: this kernel is
   // on the critical path of the call and a dependent chain of loads costs a memory round trip per link
-  const int na_lane = lane < call.n_seq ? sc.n_att[lane] : 0;
   const int ne_raw = st.ctr[u * CTR_STRIDE + CTR_NEVICT];
   const int ev_l = lane < IM_FRONT_MAX_NE ? st.ev_slot[u * p.tail + min(lane, p.tail - 1)] : -1;
   const float* mr = sc.mres + (size_t)i * IM_MRES_ROW(p);
@@ -626,6 +639,10 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
 #pragma unroll
     for (int k = 0; k < CPL; ++k) mcol[k] *= inv;
   }
+  // ---- everything below reads what the attention kernel has written.  When this kernel was launched as its
+  // programmatic dependent it may have started before that kernel ended: wait for it (and its writes) here.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int na_lane = lane < call.n_seq ? sc.n_att[lane] : 0;
   // ---- rebuild the tile bookkeeping of the attention kernel (lanes stride over the sequences)
   long long pref = 0, total = 0;
   int nt_i = 0, n_old = 0;
@@ -935,32 +952,56 @@ cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call) {
 }
 
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
-                                     const void* q, int n_ctas) {
+                                     const void* q, int n_ctas, int programmatic) {
   const ImDims& p = L.p;
-  const size_t smem = im_attn_smem_bytes(p);
   const CUtensorMap& mk = *(const CUtensorMap*)mapK;
   const CUtensorMap& mv = *(const CUtensorMap*)mapV;
-  if (p.d == 64) k_attn_stream<64><<<n_ctas, WARPS * 32, smem, L.stream>>>(mk, mv, p, L.st, L.sc, call, (const bf16*)q);
-  else k_attn_stream<128><<<n_ctas, WARPS * 32, smem, L.stream>>>(mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(n_ctas);
+  cfg.blockDim = dim3(WARPS * 32);
+  cfg.dynamicSmemBytes = im_attn_smem_bytes(p);
+  cfg.stream = L.stream;
+  // programmatic: the kernel may start while the kernel before it in the stream is still running (it waits for it,
+  // griddepcontrol.wait, before it touches anything but this layer's cache)
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = programmatic ? 1 : 0;
+  cudaError_t e;
+  if (p.d == 64) e = cudaLaunchKernelEx(&cfg, k_attn_stream<64>, mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+  else e = cudaLaunchKernelEx(&cfg, k_attn_stream<128>, mk, mv, p, L.st, L.sc, call, (const bf16*)q);
   ++*L.launches;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas, const void* q,
-                                      const void* k_new, const void* v_new) {
+                                      const void* k_new, const void* v_new, int programmatic) {
   const bf16* qp = (const bf16*)q;
   const bf16* kp = (const bf16*)k_new;
   const bf16* vp = (const bf16*)v_new;
   const ImDims& p = L.p;
-  dim3 grid(p.Hkv, call.n_seq);
-  const int mthreads = 32 * std::max(p.Gq, p.d / 32);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(p.Hkv, call.n_seq);
+  cfg.blockDim = dim3(32 * std::max(p.Gq, p.d / 32));
+  cfg.stream = L.stream;
+  // programmatic: the kernel before this one in the stream is the attention kernel, which releases its dependents
+  // when its last tiles are requested; this kernel waits for it (griddepcontrol.wait) before it reads its output
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = programmatic ? 1 : 0;
+  cudaError_t e;
   if (p.d == 64) {
-    if (p.out_f32) k_attn_merge_rows<64, float><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (float*)out, qp, kp, vp);
-    else k_attn_merge_rows<64, bf16><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (bf16*)out, qp, kp, vp);
+    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, float>, p, L.st, L.sc, call, n_ctas, (float*)out, qp, kp, vp);
+    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, bf16>, p, L.st, L.sc, call, n_ctas, (bf16*)out, qp, kp, vp);
   } else {
-    if (p.out_f32) k_attn_merge_rows<128, float><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (float*)out, qp, kp, vp);
-    else k_attn_merge_rows<128, bf16><<<grid, mthreads, 0, L.stream>>>(p, L.st, L.sc, call, n_ctas, (bf16*)out, qp, kp, vp);
+    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, float>, p, L.st, L.sc, call, n_ctas, (float*)out, qp, kp, vp);
+    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, bf16>, p, L.st, L.sc, call, n_ctas, (bf16*)out, qp, kp, vp);
   }
   ++*L.launches;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }

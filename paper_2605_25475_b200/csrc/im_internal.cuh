@@ -247,9 +247,9 @@ cudaError_t im_attn_prepare(const ImDims& p);
 cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call, int grid, int light);
 cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
-                                     const void* q, int n_ctas);
+                                     const void* q, int n_ctas, int programmatic);
 cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas, const void* q,
-                                      const void* k_new, const void* v_new);
+                                      const void* k_new, const void* v_new, int programmatic);
 
 cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,
                            uint8_t* keep, int32_t* n_evict, cudaStream_t stream);
