@@ -313,6 +313,21 @@ def test_decode_schedules_agree_with_the_oracle(im, conc):
     assert p2.stats["max_out_err"] <= 2e-3
 
 
+def test_decode_many_sequences_without_sm_partition(im):
+    """More sequences than a quarter of the SMs: the concurrent schedule then sets no SMs aside for the front
+    kernel (attention waits for the projections, the readout runs in its light variant next to the front kernel).
+    40 and 64 sequences of a small shape (16 query / 4 KV heads of 64, 4 indexer heads, d_M = 128: readout rows
+    that do not fill a batch), evictions every step.  (With the tiny shape's single indexer head a sequence whose
+    alpha nearly cancels shows that float32 dot product's rounding in all its scores; more heads average it out.)"""
+    for n_seq in (40, 64):
+        wl = TINY.replace(name=f"many{n_seq}", n_seq=n_seq, H=16, Hkv=4, ctx=96, chunk=96, B=80, steps=6, n_needles=2)
+        p = _pair(wl)
+        p.prefill(0)
+        for s in range(wl.steps):
+            p.decode(s)
+        assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
+
+
 def test_decode_from_an_empty_cache(im):
     """No prefill at all: the first decode step attends to the new token alone."""
     wl = TINY.replace(name="empty_start", ctx=0, chunk=8, B=16, steps=24, n_needles=0)
