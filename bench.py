@@ -19,6 +19,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -50,7 +51,8 @@ def measured_peaks():
 # ----------------------------------------------------------------------------------------------
 # algorithmic bytes: what one decode step has to touch in HBM at tau = 1, n = B + 1
 def algorithmic_bytes(wl: synth.Workload):
-    n = wl.B + 1
+    # entries a step reads, averaged over the phases of a compression interval: B + 1 + p in phase p (tau = 1: B + 1)
+    n = wl.B + (wl.tau + 1) / 2
     weights = 2 * (wl.HI * wl.dI * wl.D + wl.dI * wl.D + wl.HI * wl.D + wl.dM * wl.D + wl.D) + 4 * wl.dM * wl.Dkv
     kv = n * 2 * wl.Dkv * 2
     state = 4 * wl.dM * wl.Dkv + 4 * wl.dM
@@ -59,8 +61,9 @@ def algorithmic_bytes(wl: synth.Workload):
     evict = 4 * wl.dM + 2 * wl.Dkv + 4 * wl.Dkv
     per_seq = kv + state + kidx + io + evict
     per_layer = weights + wl.n_seq * per_seq
-    # the attention kernel runs after the compaction: it streams exactly B retained entries per sequence
-    attn = wl.n_seq * wl.B * 2 * wl.Dkv * 2
+    # the attention kernel streams the entries cached before the call: B at tau = 1, B + p in phase p otherwise
+    # (B again in the phase that compresses, where it runs after the compaction)
+    attn = wl.n_seq * (wl.B + (wl.tau - 1) * (wl.tau - 2) / (2 * wl.tau)) * 2 * wl.Dkv * 2
     return {"step": wl.n_layers * per_layer, "attn_launch": attn, "readout_launch": wl.n_seq * state,
             "per_seq": per_seq, "weights": weights}
 
@@ -149,6 +152,8 @@ def pick_workload(args):
     wl = synth.CONFIGS[args.workload]
     if args.layers or args.context:
         wl = wl.replace(n_layers=args.layers or wl.n_layers, ctx=args.context or wl.ctx)
+    if getattr(args, "tau", 0):
+        wl = wl.replace(tau=args.tau)
     return wl
 
 
@@ -170,22 +175,26 @@ def run_ours(args, rank, world, device):
     stream = torch.cuda.Stream(device)
     graphs = None
     launches_per_step = None
+    tau = wl.tau
+    n_graphs = n_in * tau // math.gcd(n_in, tau)                 # every (input set, phase of the interval) pair that occurs
     with torch.cuda.stream(stream):
         c0 = g.launch_count()
-        one_step(0)                                              # reaches the steady state n = B
-        launches_per_step = g.launch_count() - c0
+        for k in range(tau):                                     # one whole interval, eagerly: ends with n = B, phase 0
+            one_step(k)
+        launches_per_step = (g.launch_count() - c0) / tau
         stream.synchronize()
         if args.graph:
-            # one captured step per input set: the graph reads the resident inputs where they are
+            # one captured step per input set and phase: the graph reads the resident inputs where they are; which
+            # kernels a step launches depends on its phase (the last step of an interval compresses)
             graphs = []
-            for k in range(n_in):
+            for k in range(n_graphs):
                 gk = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(gk, stream=stream):
                     one_step(k)
                 graphs.append(gk)
-        step_fn = (lambda k: graphs[k % n_in].replay()) if graphs is not None else one_step
+        step_fn = (lambda k: graphs[k % n_graphs].replay()) if graphs is not None else one_step
         for w in range(args.warmup):
-            step_fn(w + 1)
+            step_fn(w)
         stream.synchronize()
         barrier(world)
         sampler = ClockSampler(torch.cuda.current_device() if device.index is None else device.index)
@@ -196,7 +205,7 @@ def run_ours(args, rank, world, device):
         rec0 = im.im_event_count(g.ctx, im.IM_COUNT_MERGE_RECOMPUTE)
         ev0.record(stream)
         for s in range(args.steps):
-            step_fn(args.warmup + 1 + s)
+            step_fn(args.warmup + s)
         ev1.record(stream)
         torch.cuda.synchronize()
         barrier(world)
@@ -205,13 +214,18 @@ def run_ours(args, rank, world, device):
         clocks = sampler.stop() if rank == 0 else None
         assert g.status() == 0
         ms = max_over_ranks(ms, world, device)
+        done = args.warmup + args.steps
+        while done % tau:                                        # finish the interval (phase 0 again)
+            step_fn(done)
+            done += 1
 
         # per-launch time of the dominant kernel: the same steps again, un-graphed, with the
         # library recording CUDA events around the attention + readout launch on this stream
         # (side streams off for this pass, so that the kernel is timed alone against the burst peak)
         im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 0)
-        im.im_profile_begin(g.ctx, args.steps * L)
-        for s in range(args.steps):
+        im.im_profile_begin(g.ctx, (-(-args.steps // tau) * tau) * L)
+        prof_steps = -(-args.steps // tau) * tau                # whole intervals
+        for s in range(prof_steps):
             one_step(s)
         attn_ms, attn_n = im.im_profile_end(g.ctx)
         im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 1)
@@ -228,7 +242,8 @@ def run_ours(args, rank, world, device):
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.name + ("" if not (args.layers or args.context) else " (reduced for profiling)"),
+        "config": {"workload": wl.name + ("" if not (args.layers or args.context) else " (reduced for profiling)")
+                               + ("" if not args.tau else " (compression interval %d instead of the headline workload's)" % args.tau),
                    "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H,
                    "kv_heads": wl.Hkv, "head_dim": wl.d, "context": wl.ctx, "budget": wl.B, "tau": wl.tau,
                    "cuda_graph": graphs is not None,
@@ -237,10 +252,10 @@ def run_ours(args, rank, world, device):
         "hbm_frac_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"],
         "roofline": {"bound": "hbm", "kernel": "k_attn_stream", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     "traffic": args.traffic if wl.name == "llama8b_stack" else None, "bytes_per_launch": ab["attn_launch"],
+                     "traffic": args.traffic if wl.name == "llama8b_stack" and not args.tau else None, "bytes_per_launch": ab["attn_launch"],
                      "us_per_launch": attn_launch_s * 1e6},
         "merge_recomputes_per_step": recomputes / args.steps,
-        "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        "e2e": e2e, "gpu_launches": int(round(launches_per_step * args.steps)), "clocks": clocks,
     }
     return res, wl
 
@@ -390,32 +405,36 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     # device-to-host copy of the outputs, captured once per input set into a CUDA graph (the pinned host
     # buffers are the graph's sources and destination) and replayed; without --graph the same work is enqueued
     # call by call.
+    tau = wl.tau
+    n_graphs = n_in * tau // math.gcd(n_in, tau)                 # one per (input set, phase of the interval) pair
     graphs = None
     if args.graph:
-        enqueue(0)                                               # one eager pass before capturing
+        for k in range(tau):                                     # one whole interval eagerly before capturing
+            enqueue(k % n_in)
         stream.synchronize()
         graphs = []
-        for k in range(n_in):
+        for k in range(n_graphs):
             gk = torch.cuda.CUDAGraph()
             with torch.cuda.graph(gk, stream=stream):
-                enqueue(k)
+                enqueue(k % n_in)
             graphs.append(gk)
 
     def step(s):
         if graphs is not None:
-            graphs[s % n_in].replay()
+            graphs[s % n_graphs].replay()
         else:
             enqueue(s % n_in)
         stream.synchronize()                                     # the caller has the step's result on the host
 
-    for s in range(min(3, args.warmup)):
+    n_warm = min(3, args.warmup)
+    for s in range(n_warm):
         step(s)
     barrier(world)
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
     for s in range(args.steps):
-        step(s)
+        step(n_warm + s)
     ev1.record(stream)
     torch.cuda.synchronize()
     barrier(world)
@@ -506,6 +525,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: run only this many layers (not the headline workload)")
     ap.add_argument("--context", type=int, default=0, help="profiling aid: ingest only this many context tokens")
+    ap.add_argument("--tau", type=int, default=0,
+                    help="decode with this compression interval (the paper reports 128) instead of the workload's; "
+                         "one CUDA graph per phase of the interval is captured")
     ap.add_argument("--traffic", type=float, default=ATTN_TRAFFIC_NCU,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as is)")
     args = ap.parse_args()

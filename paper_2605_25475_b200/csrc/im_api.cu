@@ -153,10 +153,14 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->sc.rpart = (float*)take((size_t)p.S * p.Dkv * 4);
   lo->sc.phiT = nullptr;
   lo->sc.vT = nullptr;
+  lo->sc.pack_k = 0;
   if (p.tail > p.F) {
-    const size_t KE = ((size_t)p.tail + 63) / 64 * 64;
+    // one sequence's largest evicted set at least; 4096 entries so that the sequences of a decode call with a long
+    // compression interval go through one batched launch
+    const size_t KE = std::max<size_t>(((size_t)p.tail + 63) / 64 * 64, 4096);
     lo->sc.phiT = (bf16*)take(2 * (size_t)p.dM * KE * 2);
     lo->sc.vT = (bf16*)take((size_t)p.Dkv * KE * 2);
+    lo->sc.pack_k = (long long)KE;
   }
   lo->sc.mch = nullptr;
   if (p.chunk_out) lo->sc.mch = (float*)take((size_t)p.S * p.max_chunk * p.Dkv * 4);
@@ -285,7 +289,7 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
   g.K = p.Dkv;
   g.out_cnt = ne_max;
   g.out_inner = p.dM;
-  g.tensor = call.prefill ? 1 : 0;
+  g.tensor = (call.prefill || g.NV >= 1024) ? 1 : 0;  // thousands of evicted keys: the tensor-core variant
   if (ne_max > p.F) {
     call.phi_large = 1;
     g.out = L.sc.phi;

@@ -100,19 +100,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 }
 // epilogue of one thread: 32 consecutive weight rows (c0 ..) of vector v
 __device__ __forceinline__ void store_columns(const ImGemmArgs& a, const ImGemmJob& job, int r0, int n_rows, int c0,
-                                              long long v, const float* acc) {
+                                              long long v, const float* acc, float* out, const int32_t* gate) {
   if (v >= a.NV) return;
-  if (a.gate && *a.gate <= a.gate_min) return;
+  if (gate && *gate <= a.gate_min) return;
   if (a.out_t) {
-    float* o = a.out + (size_t)(job.row0 + r0 + c0) * a.out_outer + v;
+    float* o = out + (size_t)(job.row0 + r0 + c0) * a.out_outer + v;
+    if (a.rmw) {
+      // read-modify-write: all 32 old values are requested before the first store (a store between two loads
+      // would keep the compiler from overlapping them: it cannot know that the addresses differ)
+      float old[32];
 #pragma unroll
-    for (int c = 0; c < 32; ++c)
-      if (c0 + c < n_rows) {
-        float* q = o + (size_t)c * a.out_outer;
-        *q = a.rmw ? fmaf(a.beta, *q, a.alpha * acc[c]) : acc[c];
-      }
+      for (int c = 0; c < 32; ++c) old[c] = c0 + c < n_rows ? o[(size_t)c * a.out_outer] : 0.f;
+#pragma unroll
+      for (int c = 0; c < 32; ++c)
+        if (c0 + c < n_rows) o[(size_t)c * a.out_outer] = fmaf(a.beta, old[c], a.alpha * acc[c]);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c)
+        if (c0 + c < n_rows) o[(size_t)c * a.out_outer] = acc[c];
+    }
   } else {
-    float* o = a.out + (v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0 + c0;
+    float* o = out + (v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0 + c0;
 #pragma unroll
     for (int c = 0; c < 32; ++c)
       if (c0 + c < n_rows) o[c] = a.rmw ? fmaf(a.beta, o[c], a.alpha * acc[c]) : acc[c];
@@ -213,7 +221,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_tc_gemm(ImGemmArgs a, int32_t*
       for (int c0 = 0; c0 < n_cols; c0 += 32) {
         float acc[32];
         tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc);
-        store_columns(a, job, r0, n_rows, c0, v, acc);
+        store_columns(a, job, r0, n_rows, c0, v, acc, a.out, a.gate);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
@@ -281,7 +289,8 @@ __device__ __forceinline__ uint64_t operand_desc_sw128(uint32_t addr) {
 
 __global__ void __launch_bounds__(T_THREADS, 1)
 k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB0,
-              const __grid_constant__ CUtensorMap mapB1, ImGemmArgs a, int j, int32_t* status) {
+              const __grid_constant__ CUtensorMap mapB1, ImGemmArgs a, int j, int32_t* status,
+              const __grid_constant__ ImGemmBatch bt) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   TShared* sh = reinterpret_cast<TShared*>(smem + T_STAGES * T_STAGE);
@@ -293,6 +302,12 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
   const long long v0 = (long long)blockIdx.x * GM;
   const int KT = a.K / GK;
   const int KTOT = KT * (job.W2 ? 2 : 1);
+  // batched launch: this CTA's product
+  const int zb = bt.n > 1 ? (int)blockIdx.z : 0;
+  const long long zu = bt.n > 1 ? (long long)bt.unit0 + bt.seq[zb] : 0;
+  const int ya = (int)(v0 + zb * bt.zA_rows), yb = (int)(r0 + zb * bt.zB_rows);
+  float* out_z = a.out + zu * bt.z_out;
+  const int32_t* gate_z = a.gate ? a.gate + zu * bt.z_gate : nullptr;
   volatile int* abort_flag = &sh->abort;
   if (tid == 0) {
     for (int s = 0; s < T_STAGES; ++s) {
@@ -327,8 +342,8 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         const uint32_t sa = smem_u32(smem + (size_t)s * T_STAGE);
         const int k0 = (kt % KT) * GK;
         mbar_expect_tx(bar, T_STAGE);
-        tma_load_2d(sa, &mapA, k0, (int)v0, bar);
-        tma_load_2d(sa + T_TILE, kt < KT ? &mapB0 : &mapB1, k0, r0, bar);
+        tma_load_2d(sa, &mapA, k0, ya, bar);
+        tma_load_2d(sa + T_TILE, kt < KT ? &mapB0 : &mapB1, k0, yb, bar);
       }
     }
   } else if (warp == 1) {
@@ -355,7 +370,7 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       for (int c0 = 0; c0 < n_cols; c0 += 32) {
         float acc[32];
         tmem_ld32(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)c0, acc);
-        store_columns(a, job, r0, n_rows, c0, v, acc);
+        store_columns(a, job, r0, n_rows, c0, v, acc, out_z, gate_z);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
@@ -434,16 +449,23 @@ cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a) {
     }
     CUtensorMap mA[4], mB0[4], mB1[4];
     bool enc_ok = true;
+    static const ImGemmBatch no_batch = {};
+    const ImGemmBatch& bt = a.batch ? *a.batch : no_batch;
+    const int nb = bt.n > 1 ? bt.n : 1;
     for (int j = 0; j < a.n_jobs && enc_ok; ++j) {
       const ImGemmJob& jb = a.job[j];
-      enc_ok = encode_rows_map(&mA[j], a.in[jb.in_sel], a.NV, a.K, vstride[j]) &&
-               encode_rows_map(&mB0[j], jb.W, jb.rows, a.K, a.K) &&
-               encode_rows_map(&mB1[j], jb.W2 ? jb.W2 : jb.W, jb.rows, a.K, a.K);
+      // a batched launch addresses batch b's operands zA_rows / zB_rows rows further down the same maps; the second
+      // weight term starts (W2 - W) / K rows into the first batch's block
+      const long long rowsA = nb > 1 ? (nb - 1) * bt.zA_rows + a.NV : a.NV;
+      const long long rowsB = nb > 1 ? (nb - 1) * bt.zB_rows + jb.rows : jb.rows;
+      enc_ok = encode_rows_map(&mA[j], a.in[jb.in_sel], rowsA, a.K, vstride[j]) &&
+               encode_rows_map(&mB0[j], jb.W, rowsB, a.K, a.K) &&
+               encode_rows_map(&mB1[j], jb.W2 ? jb.W2 : jb.W, rowsB, a.K, a.K);
     }
     if (enc_ok) {
       for (int j = 0; j < a.n_jobs; ++j) {
-        dim3 grid((unsigned)((a.NV + GM - 1) / GM), (unsigned)((a.job[j].rows + GN - 1) / GN));
-        k_tc_gemm_tma<<<grid, T_THREADS, T_SMEM, L.stream>>>(mA[j], mB0[j], mB1[j], a, j, L.st.status);
+        dim3 grid((unsigned)((a.NV + GM - 1) / GM), (unsigned)((a.job[j].rows + GN - 1) / GN), (unsigned)nb);
+        k_tc_gemm_tma<<<grid, T_THREADS, T_SMEM, L.stream>>>(mA[j], mB0[j], mB1[j], a, j, L.st.status, bt);
         ++*L.launches;
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -451,6 +473,7 @@ cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a) {
       return cudaSuccess;
     }
   }
+  if (a.batch && a.batch->n > 1) return cudaErrorNotSupported;  // the batched form exists for the TMA variant only
   int tiles = 0;
   for (int j = 0; j < a.n_jobs; ++j) tiles += (a.job[j].rows + GN - 1) / GN;
   dim3 grid((unsigned)((a.NV + GM - 1) / GM), tiles);

@@ -103,8 +103,10 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
                      // sum, and the coefficient c of the Mhat part: m(q)[col] = mres[col] + c * rpart[col]
   float* phiq;       // [max_seqs][dM] phi(q) of the call (K-split partials summed)
   int32_t* n_att;    // [max_seqs] entries per sequence the streaming attention kernel of the call ran over
-  bf16* phiT;        // [2][dM][KE] phi of one sequence's evicted keys, transposed, as two bf16 terms (KE = tail rounded up to 64)
-  bf16* vT;          // [Dkv][KE] that sequence's evicted values, transposed
+  bf16* phiT;        // [seq][2][dM][KE] phi of the evicted keys, transposed, as two bf16 terms (KE = evicted count rounded
+                     // up to 64); room for pack_k entries in all (one sequence's tail at least)
+  bf16* vT;          // [seq][Dkv][KE] the evicted values, transposed
+  long long pack_k;  // entries phiT / vT have room for
   float* mch;        // [max_seqs][max_chunk][Dkv] gated memory readout of a chunk's own queries (im_prefill_chunk_attend)
   uint8_t* qpack;    // [n_seq][ceil(C / IM_TC_QT)][IM_TC_TILE_BYTES] query operand of the tensor-core prefill scoring
 };
@@ -130,6 +132,14 @@ struct ImGemmJob {
   const bf16* W2;  // optional second term of the weights (nullptr: none)
   int rows, row0, in_sel;
 };
+// Batched launch of the tensor-core TMA variant: n independent products, blockIdx.z = b.  Batch b reads its vectors
+// zA_rows rows and its weights zB_rows rows further down the operand arrays and writes to out + u * z_out with
+// u = unit0 + seq[b] (its gate is gate[u * z_gate]).  Travels as a kernel parameter of that variant alone.
+struct ImGemmBatch {
+  int n, unit0;
+  long long zA_rows, zB_rows, z_out, z_gate;
+  int seq[IM_MAX_CALL_SEQS];
+};
 struct ImGemmArgs {
   ImGemmJob job[4];
   int n_jobs;
@@ -145,6 +155,7 @@ struct ImGemmArgs {
   int direct;  // 1: few vectors (decode) - the variant without shared-memory staging, if the K split is a multiple of 32
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
   int smem_floor;  // direct variant: dynamic shared memory to ask for although the kernel uses none (IM_SMEM_SIDE)
+  const struct ImGemmBatch* batch;  // host pointer, tensor-core TMA variant only: several products in one launch
   // tensor-core variant only:
   int out_t;            // 1: the result goes to out[(row0 + r) * out_outer + v] (vectors contiguous) instead
   int rmw;              // 1: out = beta * out + alpha * result

@@ -214,9 +214,13 @@ __global__ void __launch_bounds__(256) k_mem_accumulate(ImDims p, ImState st, Im
 // entries.  The GEMM kernels want both operands K-major (K = evicted entry), so phi (float32, [e][m]) and the
 // evicted values ([e][col]) of one sequence are transposed first; phi becomes two bf16 terms (hi + lo
 // reproduces the float32 value to 2^-17).  Entries at or beyond the sequence's evicted count are zero.
-// grid = (KE / 32, (dM + Dkv) / 32), block = (32, 8).
-__global__ void __launch_bounds__(256) k_mem_pack(ImDims p, ImState st, ImScratch sc, ImCall call, int i, int KE) {
+// grid = (KE / 32, (dM + Dkv) / 32, sequences), block = (32, 8); sequence i0 + blockIdx.z goes to block blockIdx.z
+// of phiT / vT.
+__global__ void __launch_bounds__(256) k_mem_pack(ImDims p, ImState st, ImScratch sc, ImCall call, int i0, int KE) {
   __shared__ float tile[32][33];
+  const int i = i0 + blockIdx.z;
+  bf16* phiT = sc.phiT + (size_t)blockIdx.z * 2 * p.dM * KE;
+  bf16* vT = sc.vT + (size_t)blockIdx.z * p.Dkv * KE;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
   const int e0 = blockIdx.x * 32, tx = threadIdx.x, ty = threadIdx.y;
@@ -238,10 +242,10 @@ __global__ void __launch_bounds__(256) k_mem_pack(ImDims p, ImState st, ImScratc
     const float v = tile[tx][r];
     const bf16 hi = __float2bfloat16_rn(v);
     if (is_phi) {
-      sc.phiT[(size_t)c * KE + e] = hi;
-      sc.phiT[((size_t)p.dM + c) * KE + e] = __float2bfloat16_rn(v - __bfloat162float(hi));
+      phiT[(size_t)c * KE + e] = hi;
+      phiT[((size_t)p.dM + c) * KE + e] = __float2bfloat16_rn(v - __bfloat162float(hi));
     } else {
-      sc.vT[(size_t)c * KE + e] = hi;
+      vT[(size_t)c * KE + e] = hi;
     }
   }
 }
@@ -315,6 +319,26 @@ cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_m
     k_mem_bsum<<<gb, dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call);
     ++*L.launches;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    // all sequences of the call in one batched launch when their packed operands fit the scratch arrays
+    if (call.n_seq > 1 && (long long)call.n_seq * KE <= L.sc.pack_k) {
+      dim3 gp(KE / 32, (p.dM + 31) / 32 + (p.Dkv + 31) / 32, call.n_seq);
+      k_mem_pack<<<gp, dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call, 0, KE);
+      ++*L.launches;
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      ImGemmBatch bt;
+      memset(&bt, 0, sizeof(bt));
+      bt.n = call.n_seq;
+      bt.unit0 = call.layer * p.S;
+      for (int i = 0; i < call.n_seq; ++i) bt.seq[i] = call.seq[i];
+      bt.zA_rows = p.Dkv;
+      bt.zB_rows = 2 * (long long)p.dM;
+      bt.z_out = (long long)p.dM * p.Dkv;
+      bt.z_gate = CTR_STRIDE;
+      g.batch = &bt;
+      g.out = L.st.Mhat;
+      g.gate = L.st.ctr + CTR_NEVICT;
+      return im_launch_tc_gemm(L, g);
+    }
     for (int i = 0; i < call.n_seq; ++i) {
       if (ne_host[i] <= p.F) continue;
       const size_t u = (size_t)call.layer * p.S + call.seq[i];

@@ -328,6 +328,19 @@ def test_decode_many_sequences_without_sm_partition(im):
         assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
 
 
+def test_decode_long_interval_several_sequences_batched_memory_write(im):
+    """tau = 40 at Llama widths with three sequences: every 40th step evicts 40 entries per sequence, more than the
+    pending list or the fused front kernel hold, so the step runs in order and writes Phi^T V of all sequences
+    with one batched tensor-core launch; the 39 steps between attend to a growing cache without selecting."""
+    wl = synth.CONFIGS["llama8b_b1"].replace(name="tau40", n_seq=3, ctx=150, chunk=150, B=100, steps=85, tau=40, n_needles=2)
+    p = _pair(wl)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
+    assert p.o.evict_steps(0) == 1 + 2
+
+
 def test_decode_from_an_empty_cache(im):
     """No prefill at all: the first decode step attends to the new token alone."""
     wl = TINY.replace(name="empty_start", ctx=0, chunk=8, B=16, steps=24, n_needles=0)
