@@ -197,6 +197,12 @@ struct im_ctx {
   bool prefetch_next = true;         // warm L2 with the next layer's weights / index state during attention
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
   int n_sm = 1;                      // SMs of the device
+  // The last kernel this context put on a caller's stream, if that was the merge kernel of a concurrent decode
+  // call (which writes nothing but the call's output): only then may the next call's attention kernel be launched
+  // as its programmatic dependent and fetch cache tiles before that kernel has ended.  After a prefill call, an
+  // in-order decode call or a state import the stream's last kernel may have written the cache.
+  cudaStream_t tail_stream = nullptr;
+  bool tail_is_merge = false;
   bool score_tc = false;             // prefill scoring runs on the tensor cores (tcgen05)
   bool attend_tc = true;             // chunk attention of im_prefill_chunk_attend on tcgen05 where head_dim is 128
   int prof_target = 0;               // kernel timed by im_profile_*: 0 attention (decode), 1 prefill scoring
@@ -448,6 +454,7 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   ImCall call;
   int rc = check_call(ctx, layer, n_seq, seq_ids, &call);
   if (rc) return rc;
+  ctx->tail_is_merge = false;
   const ImDims& p = ctx->p;
   if (chunk_len < 1 || chunk_len > p.max_chunk)
     return fail(IM_ERR_ARG, "chunk_len %d out of range [1,%d]", chunk_len, p.max_chunk);
@@ -609,6 +616,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   //  (B) in order on s0, attention after the compaction: everything else (large evicted sets, budgets
   //      beyond the fused front kernel, head shapes without the streaming attention kernel).
   cudaStream_t s0 = (cudaStream_t)cuda_stream;
+  const bool after_merge = ctx->tail_is_merge && ctx->tail_stream == s0;
+  ctx->tail_is_merge = false;
   const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
   const bool defer = ctx->fast_attn && (!due || fused) && ne_max <= p.F;
   const bool conc = defer && ctx->concurrent;
@@ -679,7 +688,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
       CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
     }
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
-    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas, n_res > 0 ? 1 : 0));
+    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas, n_res > 0 && after_merge ? 1 : 0));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
     CK(cudaEventRecord(ctx->ev[9], s0));  // the attention kernel has read the cache
   }
@@ -778,6 +787,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
   }
   if (prof) ctx->prof_used += 2;
+  ctx->tail_is_merge = conc;
+  ctx->tail_stream = s0;
   return IM_OK;
 }
 
@@ -863,6 +874,7 @@ int im_set_weights(im_ctx* ctx, int layer, int which, const void* host_buf, size
   if (layer < 0 || layer >= ctx->p.L) return fail(IM_ERR_ARG, "layer out of range");
   size_t want = weight_bytes(ctx->p, which);
   if (want == 0 || want != bytes) return fail(IM_ERR_ARG, "weight %d: expected %zu bytes, got %zu", which, want, bytes);
+  ctx->tail_is_merge = false;
   CK(cudaDeviceSynchronize());
   CK(cudaMemcpy(weight_ptr(ctx->lo.w[layer], which), host_buf, bytes, cudaMemcpyHostToDevice));
   if (which == IM_W_THETA) {
@@ -886,6 +898,7 @@ int im_state_export(im_ctx* ctx, int layer, int seq, int which, void* host_buf, 
   if (!ctx || !host_buf) return fail(IM_ERR_ARG, "null argument");
   const ImDims& p = ctx->p;
   if (layer < 0 || layer >= p.L || seq < 0 || seq >= p.S) return fail(IM_ERR_ARG, "layer/seq out of range");
+  ctx->tail_is_merge = false;
   CK(cudaDeviceSynchronize());
   const size_t u = (size_t)layer * p.S + seq;
   const ImState& st = ctx->lo.st;
