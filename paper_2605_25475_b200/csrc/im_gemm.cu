@@ -276,6 +276,59 @@ __global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __
   }
 }
 
+// The same projection for the thousands of vectors of a prefill chunk, on the float64 tensor-core path
+// (mma.sync m8n8k4 f64): a warp takes 8 vectors x all d_I rows over a quarter of the K range, the four warps of a
+// block add their 8 x 8 tiles through shared memory in warp order.  Lane (r, q) = (lane / 4, lane % 4) loads 8
+// consecutive k of row r (vector r for A, weight row r of the n-tile for B) starting at 8 q inside a 32-wide
+// chunk; k-step s multiplies element s of every lane's vector: the contraction index is permuted identically for
+// both operands.  Every product and sum is formed in float64.
+// grid = ceil(NV / 8), block = 128; D a multiple of 128, d_I = 8 NT.
+__device__ __forceinline__ void dmma_884(double (&c)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(c[0]), "+d"(c[1]) : "d"(a), "d"(b));
+}
+__device__ __forceinline__ double bf16_elem(const uint4& v, int s) {
+  const uint32_t w = s < 2 ? v.x : s < 4 ? v.y : s < 6 ? v.z : v.w;
+  return (double)((s & 1) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16));
+}
+template <int NT>
+__global__ void __launch_bounds__(128) k_proj_key_mma(ImDims p, const bf16* __restrict__ Uk, const bf16* __restrict__ x,
+                                                       int NV, double* __restrict__ keyp) {
+  __shared__ double red[4][NT][64];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, q = lane & 3;
+  const long long v0 = (long long)blockIdx.x * 8;
+  const int kspan = p.D / 4, kbeg = warp * kspan;  // a multiple of 32 (checked by the launcher)
+  const bf16* xrow = x + (size_t)min(v0 + r, (long long)NV - 1) * p.D + kbeg + 8 * q;
+  const bf16* urow = Uk + (size_t)r * p.D + kbeg + 8 * q;
+  double c[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = 0.0;
+  for (int kb = 0; kb < kspan; kb += 32) {
+    const uint4 xa = *reinterpret_cast<const uint4*>(xrow + kb);
+    uint4 ub[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) ub[nt] = *reinterpret_cast<const uint4*>(urow + (size_t)nt * 8 * p.D + kb);
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const double a = bf16_elem(xa, s);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) dmma_884(c[nt], a, bf16_elem(ub[nt], s));
+    }
+  }
+  // C fragment: row r (vector), columns 2 q and 2 q + 1 (weight row of the n-tile)
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    red[warp][nt][r * 8 + 2 * q] = c[nt][0];
+    red[warp][nt][r * 8 + 2 * q + 1] = c[nt][1];
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < NT * 64; idx += 128) {
+    const int nt = idx >> 6, e = idx & 63;
+    const long long v = v0 + (e >> 3);
+    if (v < NV) keyp[(size_t)v * p.dI + nt * 8 + (e & 7)] = ((red[0][nt][e] + red[1][nt][e]) + red[2][nt][e]) + red[3][nt][e];
+  }
+}
+
 }  // namespace
 
 cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
@@ -313,6 +366,12 @@ cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
 }
 
 cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, int ksplit) {
+  if (ksplit == 1 && NV >= 64 && L.p.D % 128 == 0 && (L.p.dI == 8 || L.p.dI == 16)) {  // prefill chunks
+    if (L.p.dI == 8) k_proj_key_mma<1><<<(NV + 7) / 8, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, L.sc.keyp);
+    else k_proj_key_mma<2><<<(NV + 7) / 8, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, L.sc.keyp);
+    ++*L.launches;
+    return cudaGetLastError();
+  }
   dim3 grid(ksplit, (NV + 7) / 8);
   k_proj_key_split<<<grid, 256, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
   ++*L.launches;
