@@ -154,6 +154,7 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->sc.phiT = nullptr;
   lo->sc.vT = nullptr;
   lo->sc.pack_k = 0;
+  lo->sc.bpart = nullptr;
   if (p.tail > p.F) {
     // one sequence's largest evicted set at least; 4096 entries so that the sequences of a decode call with a long
     // compression interval go through one batched launch
@@ -161,6 +162,7 @@ void carve(const ImDims& p, char* base, Layout* lo) {
     lo->sc.phiT = (bf16*)take(2 * (size_t)p.dM * KE * 2);
     lo->sc.vT = (bf16*)take((size_t)p.Dkv * KE * 2);
     lo->sc.pack_k = (long long)KE;
+    lo->sc.bpart = (float*)take((KE / 32) * (size_t)p.dM * 4);
   }
   lo->sc.mch = nullptr;
   if (p.chunk_out) lo->sc.mch = (float*)take((size_t)p.S * p.max_chunk * p.Dkv * 4);

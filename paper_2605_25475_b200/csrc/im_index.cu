@@ -196,28 +196,67 @@ struct SelectShared {
   uint32_t digit, remaining;
 };
 
+// Key of rank k (k-th largest; keys are distinct) among n entries, by an 8-pass radix select over the 64-bit key,
+// most significant byte first.  Up to SEL_KPT keys per thread stay in registers over the passes (n beyond that:
+// re-read from memory); the digit of a pass is found by warp 0 (lane l sums the 8 bins 255 - 8 l down to
+// 248 - 8 l, a prefix over the lanes locates the lane, which then walks its own bins).
+constexpr int SEL_KPT = 8;
 __device__ uint64_t block_kth_largest_key(const float* __restrict__ score, const int32_t* __restrict__ pos, int n,
                                           int k, int n_sink, SelectShared* sh) {
   uint64_t prefix = 0, mask = 0;
+  const bool cached = n <= SEL_KPT * (int)blockDim.x;
+  uint64_t kreg[SEL_KPT];
+  if (cached) {
+#pragma unroll
+    for (int j = 0; j < SEL_KPT; ++j) {
+      const int t = threadIdx.x + j * blockDim.x;
+      kreg[j] = t < n ? im_select_key(score[t], pos[t], n_sink) : 0ull;
+    }
+  }
   if (threadIdx.x == 0) sh->remaining = (uint32_t)k;
   for (int shift = 56; shift >= 0; shift -= 8) {
     for (int b = threadIdx.x; b < 256; b += blockDim.x) sh->hist[b] = 0;
     __syncthreads();
-    for (int t = threadIdx.x; t < n; t += blockDim.x) {
-      const uint64_t key = im_select_key(score[t], pos[t], n_sink);
-      if ((key & mask) == prefix) atomicAdd(&sh->hist[(uint32_t)(key >> shift) & 255u], 1u);
+    if (cached) {
+#pragma unroll
+      for (int j = 0; j < SEL_KPT; ++j) {
+        const int t = threadIdx.x + j * blockDim.x;
+        if (t < n && (kreg[j] & mask) == prefix) atomicAdd(&sh->hist[(uint32_t)(kreg[j] >> shift) & 255u], 1u);
+      }
+    } else {
+      for (int t = threadIdx.x; t < n; t += blockDim.x) {
+        const uint64_t key = im_select_key(score[t], pos[t], n_sink);
+        if ((key & mask) == prefix) atomicAdd(&sh->hist[(uint32_t)(key >> shift) & 255u], 1u);
+      }
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      uint32_t rem = sh->remaining, cum = 0;
-      int b = 255;
-      for (; b > 0; --b) {
-        const uint32_t c = sh->hist[b];
-        if (cum + c >= rem) break;
-        cum += c;
+    if (threadIdx.x < 32) {
+      const int lane = threadIdx.x;
+      const uint32_t rem = sh->remaining;
+      uint32_t mine = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) mine += sh->hist[255 - 8 * lane - j];
+      uint32_t incl = mine;  // entries in the bins of lanes 0 .. lane (the highest bins)
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
       }
-      sh->digit = (uint32_t)b;
-      sh->remaining = rem - cum;
+      const uint32_t hit = __ballot_sync(0xffffffffu, incl >= rem);
+      // the rank lies in the bins of the first lane whose prefix reaches it (bin 0 takes what is left otherwise)
+      const int owner = hit ? __ffs(hit) - 1 : 31;
+      if (lane == owner) {
+        uint32_t cum = incl - mine;
+        int b = 255 - 8 * lane;
+        const int b_last = lane == 31 ? 0 : 255 - 8 * lane - 7;
+        for (; b > b_last; --b) {
+          const uint32_t c = sh->hist[b];
+          if (cum + c >= rem) break;
+          cum += c;
+        }
+        sh->digit = (uint32_t)b;
+        sh->remaining = rem - cum;
+      }
     }
     __syncthreads();
     prefix |= (uint64_t)sh->digit << shift;
@@ -259,7 +298,7 @@ __device__ int block_exclusive_scan(int v, int* out_excl, int* s_tmp /*[33]*/) {
 
 // Compression of every sequence in the call (Sec. 4 schedule): restart pooling; if over budget,
 // flag the retained entries and list the evicted slots in ascending slot order.
-// grid = n_seq, block = 256.
+// grid = n_seq, block = 1024.
 __global__ void k_select(ImDims p, ImState st, ImScratch sc, ImCall call) {
   __shared__ SelectShared sh;
   __shared__ int s_tmp[33];
@@ -407,7 +446,7 @@ cudaError_t im_launch_prefill_commit(const ImLaunch& L, const ImCall& call) {
 }
 
 cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call) {
-  k_select<<<call.n_seq, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
+  k_select<<<call.n_seq, 1024, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
 }

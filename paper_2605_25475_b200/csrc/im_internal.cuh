@@ -107,6 +107,7 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
                      // up to 64); room for pack_k entries in all (one sequence's tail at least)
   bf16* vT;          // [seq][Dkv][KE] the evicted values, transposed
   long long pack_k;  // entries phiT / vT have room for
+  float* bpart;      // [pack_k / 32][dM] sums of phi^2 over the 32 entries of a block of the packed operands
   float* mch;        // [max_seqs][max_chunk][Dkv] gated memory readout of a chunk's own queries (im_prefill_chunk_attend)
   uint8_t* qpack;    // [n_seq][ceil(C / IM_TC_QT)][IM_TC_TILE_BYTES] query operand of the tensor-core prefill scoring
 };

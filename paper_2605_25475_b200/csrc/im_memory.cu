@@ -236,6 +236,14 @@ __global__ void __launch_bounds__(256) k_mem_pack(ImDims p, ImState st, ImScratc
     tile[r][tx] = v;
   }
   __syncthreads();
+  if (is_phi && ty == 0 && c0 + tx < width) {
+    // sum of phi^2 over this block's 32 entries for column c0 + tx (Eq. 7), in a fixed order; k_mem_bsum adds the
+    // blocks' sums
+    float s2 = 0.f;
+#pragma unroll 8
+    for (int r = 0; r < 32; ++r) s2 = fmaf(tile[r][tx], tile[r][tx], s2);
+    sc.bpart[((size_t)blockIdx.z * (KE / 32) + blockIdx.x) * p.dM + c0 + tx] = s2;
+  }
   for (int r = ty; r < 32; r += 8) {  // rows = columns of the source, threads along the entries
     const int c = c0 + r, e = e0 + tx;
     if (c >= width || e >= KE) continue;
@@ -250,21 +258,19 @@ __global__ void __launch_bounds__(256) k_mem_pack(ImDims p, ImState st, ImScratc
   }
 }
 
-// b <- lambda b + eta sum_e phi_e^2 (Eq. 7) for the sequences whose evicted set is larger than the pending list.
-// grid = (ceil(dM / 32), n_seq), block = (32, 8): eight partial sums per row, added in a fixed order.
-__global__ void __launch_bounds__(256) k_mem_bsum(ImDims p, ImState st, ImScratch sc, ImCall call) {
+// b <- lambda b + eta sum_e phi_e^2 (Eq. 7) for the sequences whose evicted set is larger than the pending list,
+// from the sums over 32 entries that k_mem_pack left (block `slot` of the packed operands holds sequence i0 + slot).
+// grid = (ceil(dM / 32), sequences), block = (32, 8): eight partial sums per row, added in a fixed order.
+__global__ void __launch_bounds__(256) k_mem_bsum(ImDims p, ImState st, ImScratch sc, ImCall call, int i0, int KE) {
   __shared__ float part[8][32];
-  const int i = blockIdx.y;
+  const int i = i0 + blockIdx.y;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
   if (ne <= p.F) return;
   const int m = blockIdx.x * 32 + threadIdx.x;
   float s = 0.f;
   if (m < p.dM)
-    for (int e = threadIdx.y; e < ne; e += 8) {
-      const float f = sc.phi[((size_t)i * p.tail + e) * p.dM + m];
-      s = fmaf(f, f, s);
-    }
+    for (int j = threadIdx.y; j < KE / 32; j += 8) s += sc.bpart[((size_t)blockIdx.y * (KE / 32) + j) * p.dM + m];
   part[threadIdx.y][threadIdx.x] = s;
   __syncthreads();
   if (threadIdx.y == 0 && m < p.dM) {
@@ -315,14 +321,14 @@ cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_m
   g.beta = p.lambda;
   g.gate_min = p.F;
   if (L.sc.phiT && call.phi_large && ne_host && im_tc_gemm_usable(g)) {
-    dim3 gb((p.dM + 31) / 32, call.n_seq);
-    k_mem_bsum<<<gb, dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call);
-    ++*L.launches;
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     // all sequences of the call in one batched launch when their packed operands fit the scratch arrays
     if (call.n_seq > 1 && (long long)call.n_seq * KE <= L.sc.pack_k) {
       dim3 gp(KE / 32, (p.dM + 31) / 32 + (p.Dkv + 31) / 32, call.n_seq);
       k_mem_pack<<<gp, dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call, 0, KE);
+      ++*L.launches;
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      dim3 gb((p.dM + 31) / 32, call.n_seq);
+      k_mem_bsum<<<gb, dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call, 0, KE);
       ++*L.launches;
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       ImGemmBatch bt;
@@ -344,6 +350,9 @@ cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_m
       const size_t u = (size_t)call.layer * p.S + call.seq[i];
       dim3 gp(KE / 32, (p.dM + 31) / 32 + (p.Dkv + 31) / 32);
       k_mem_pack<<<gp, dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call, i, KE);
+      ++*L.launches;
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      k_mem_bsum<<<dim3((p.dM + 31) / 32, 1), dim3(32, 8), 0, L.stream>>>(p, L.st, L.sc, call, i, KE);
       ++*L.launches;
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       g.out = L.st.Mhat + u * p.dM * p.Dkv;
