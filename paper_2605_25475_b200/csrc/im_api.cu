@@ -607,13 +607,15 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   //      once over the entries cached before the call.  The merge adds the new token, removes the evicted
   //      entries again (exactly, see k_attn_merge_rows), adds the terms of this call's memory write to the
   //      readout, and fills the holes.
-  //        s0: (waits for the three projections) attention ------------------------> merge
+  //        s0: attention (with SMs set aside for the front kernel: from the start of the call, else after the three
+  //            projections) ---------------------------------------------------------> merge
   //        s1: indexer projections -> front (append, score, select, gather) -> phi of the evicted keys
   //            [-> memory write: not needed by the merge, it only has to end with the call]
-  //        s2: phi(q) / gate projections -> phi(q)^T Mhat (streams Mhat next to the attention kernel)
-  //        s4: fold -> the readout terms that do not go through Mhat, over the memory as it is before the write
-  //        s3: float64 key projection (needed by front) -> L2 prefetch for the next layer
-  //        s4: fold of the pending list (before front, which changes the counters, and before the readout)
+  //        s2: phi(q) / gate projections -> (front kernel ended) -> phi(q)^T Mhat next to the attention kernel
+  //        s3: float64 key projection (needed by front) -> L2 prefetch for the next layer -> filling of the holes
+  //            (once front has listed them and the attention kernel has read the cache)
+  //        s4: fold of the pending list (before front, which changes the counters, and before the readout) ->
+  //            the readout terms that do not go through Mhat, over the memory as it is before the write
   //      With IM_OPT_CONCURRENCY off the same kernels run on s0 in an order that respects these arrows.
   //  (B) in order on s0, attention after the compaction: everything else (large evicted sets, budgets
   //      beyond the fused front kernel, head shapes without the streaming attention kernel).
