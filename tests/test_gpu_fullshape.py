@@ -106,6 +106,93 @@ def test_stack_shape_sampled_units_under_graph_replay():
     assert np.isfinite(results[-1]).all()
 
 
+def test_stack_shape_long_interval_one_graph_per_phase():
+    """The benchmark's layer shape with a compression interval of 32 (`bench.py --tau`): one CUDA graph per phase of
+    the interval, captured in order and replayed in order with the inputs in place.  31 phases append and attend
+    over B + p entries; the last one selects 32 entries per sequence (more than the fused front kernel or the
+    pending list hold), writes Phi^T V of all 32 sequences with one batched tensor-core launch and compacts.  Two
+    sampled units follow the oracle through a whole eager interval and 34 replayed steps."""
+    from paper_2605_25475_b200 import binding as im
+    from tests.parity import bf16_ulp
+    tau = 32
+    wl = synth.CONFIGS["llama8b_stack"].replace(name="stack_tau", n_layers=2, ctx=4096, tau=tau)
+    dev = torch.device("cuda:0")
+    g = im.IndexMem(im.Config(n_layers=wl.n_layers, max_seqs=wl.n_seq, n_q_heads=wl.H, n_kv_heads=wl.Hkv,
+                              head_dim=wl.d, budget=wl.B, compress_interval=tau, max_chunk=wl.chunk,
+                              n_sink=wl.n_sink), dev)
+    ids = list(range(wl.n_seq))
+    sampled = [(0, 11), (1, 30)]
+    oracles = {}
+    for layer in range(wl.n_layers):
+        w = synth.make_weights(wl, layer)
+        g.set_weights(layer, w)
+        for (l, s) in sampled:
+            if l == layer:
+                o = orc.OracleLayer(orc.OracleConfig(H=wl.H, Hkv=wl.Hkv, d=wl.d, B=wl.B, tau=tau, n_sink=wl.n_sink), 1)
+                o.set_weights({k: synth.f32(v) for k, v in w.items()})
+                oracles[(l, s)] = o
+    for c in range(wl.ctx // wl.chunk):
+        for layer in range(wl.n_layers):
+            X, Q, K, V = synth.prefill_inputs(wl, layer, c)
+            g.prefill_chunk(layer, ids, X.to(dev), Q.to(dev), K.to(dev), V.to(dev))
+            for (l, s), o in oracles.items():
+                if l == layer:
+                    o.prefill_chunk(0, synth.f32(X[s]), synth.f32(Q[s]), synth.f32(K[s]), synth.f32(V[s]))
+    assert g.status() == 0
+
+    n_eager, n_replay = tau, tau + 2
+    n_steps = n_eager + n_replay
+    n_in = 4                                                     # input sets, cycled (tau is a multiple)
+    ins = [[synth.decode_inputs(wl, layer, st) for layer in range(wl.n_layers)] for st in range(n_in)]
+    dins = [[tuple(t.to(dev) for t in ins[k][layer]) for layer in range(wl.n_layers)] for k in range(n_in)]
+    out = torch.empty((wl.n_layers, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=dev)
+
+    def one_step(k):
+        for layer in range(wl.n_layers):
+            x, q, kk, v = dins[k % n_in][layer]
+            g.decode_step(layer, ids, x, q, q, kk, v, out[layer])
+
+    results = []
+    stream = torch.cuda.Stream(dev)
+    with torch.cuda.stream(stream):
+        for st in range(n_eager):                                # a whole interval eagerly: phase 0 again
+            one_step(st)
+            stream.synchronize()
+            results.append(out.float().cpu().numpy().copy())
+        graphs = []
+        for ph in range(tau):                                    # tau is a multiple of n_in: graph ph reads set ph % n_in
+            gk = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gk, stream=stream):
+                one_step(ph)
+            graphs.append(gk)
+        for st in range(n_replay):
+            graphs[st % tau].replay()
+            stream.synchronize()
+            results.append(out.float().cpu().numpy().copy())
+    assert g.status() == 0
+
+    for (l, s), o in oracles.items():
+        for st in range(n_steps):
+            x, q, k, v = ins[(st if st < n_eager else st - n_eager) % n_in][l]
+            ob, od = o.decode_step(0, synth.f32(x[s]), synth.f32(q[s]), synth.f32(q[s]), synth.f32(k[s]), synth.f32(v[s]))
+            got = results[st][l, s].astype(np.float64)
+            scale = np.abs(od).max()
+            half_ulp = 0.5 * bf16_ulp(np.maximum(np.abs(od), np.abs(got)))
+            assert np.all(np.abs(got - od) <= 2e-3 * scale + half_ulp), f"unit {(l, s)} step {st}"
+        assert o.evict_steps(0) == 1 + 2                         # the second prefill chunk, two full intervals
+        assert sorted(g.export(l, s, im.IM_S_POS).tolist()) == o.positions(0).tolist()
+        Mo, bo = o.memory_kv(0)
+        Mg = g.export(l, s, im.IM_S_M).astype(np.float64)
+        assert np.abs(Mg - Mo).max() <= 2e-3 * np.abs(Mo).max()
+        assert np.abs(g.export(l, s, im.IM_S_B) - bo).max() <= 2e-3 * np.abs(bo).max()
+    for layer in range(wl.n_layers):
+        for s in range(0, wl.n_seq, 7):
+            cnt = g.counts(layer, s)
+            assert cnt["n"] == wl.B + 2 and cnt["T"] == wl.ctx + n_steps
+            pos = g.export(layer, s, im.IM_S_POS)
+            assert len(set(pos.tolist())) == wl.B + 2 and set(range(wl.n_sink)) <= set(pos.tolist())
+
+
 def test_llama8b_b1_configuration_at_full_size():
     """The Llama-3-8B-shaped single-sequence configuration as stated: 32 q / 8 KV heads, d 128, a 4096-token
     context ingested in one chunk (3584 evictions in one evict step: the tensor-core scoring, selection,
