@@ -490,9 +490,7 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   ImRows r = im_rows(p);
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
-  g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
-  g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
-  g.n_jobs = 2;
+  g.n_jobs = 1;
   g.in[0] = (const bf16*)q_pre;
   g.in[1] = (const bf16*)x;
   for (int k = 0; k < 2; ++k) { g.in_cnt[k] = 1; g.in_outer[k] = p.D; g.in_inner[k] = 0; }
@@ -503,30 +501,67 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   g.K = p.D;
   g.ksplit = 1;
   g.tensor = 1;
+  // The projections of a chunk are independent of one another and each fills a fraction of the SMs (a launch is
+  // bound by the K loop of one CTA): with IM_OPT_CONCURRENCY they run next to one another on the side streams,
+  // forked from and joined back into the caller's stream with events.
+  const bool fork = ctx->concurrent;
+  const bool memside = attend && p.mem;
+  ImLaunch Lg = L, Lk = L, Lt = L, Lw = L;
+  if (fork) {
+    Lg.stream = ctx->side[0];
+    Lk.stream = ctx->side[1];
+    CK(cudaEventRecord(ctx->ev[0], L.stream));
+    CK(cudaStreamWaitEvent(Lg.stream, ctx->ev[0], 0));
+    CK(cudaStreamWaitEvent(Lk.stream, ctx->ev[0], 0));
+    if (memside) {
+      Lt.stream = ctx->side[2];
+      Lw.stream = ctx->side[3];
+      CK(cudaStreamWaitEvent(Lt.stream, ctx->ev[0], 0));
+      CK(cudaStreamWaitEvent(Lw.stream, ctx->ev[0], 0));
+    }
+  }
+  g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
   CKL(im_launch_gemm(L, g));
-  CKL(im_launch_proj_key_split(L, x, NV, 1));
+  g.job[0] = {L.w.G, nullptr, p.HI, r.g, 1};
+  CKL(im_launch_gemm(Lg, g));
+  CKL(im_launch_proj_key_split(Lk, x, NV, 1));
+  if (memside) {
+    // phi(q) and the gate logit of every chunk token (behind the indexer-side block of the projection scratch)
+    ImGemmArgs g2;
+    memset(&g2, 0, sizeof(g2));
+    g2.n_jobs = 1;
+    g2.in[0] = (const bf16*)q;
+    g2.in_cnt[0] = 1;
+    g2.in_outer[0] = p.D;
+    g2.out = L.sc.raw + (size_t)p.S * p.max_chunk * p.R3;
+    g2.out_cnt = 1;
+    g2.out_outer = p.dM + 1;
+    g2.NV = NV;
+    g2.K = p.D;
+    g2.ksplit = 1;
+    g2.tensor = 1;
+    g2.job[0] = {L.w.Wt, nullptr, p.dM, 0, 0};
+    CKL(im_launch_gemm(Lt, g2));
+    g2.job[0] = {L.w.wg, nullptr, 1, p.dM, 0};
+    CKL(im_launch_gemm(Lw, g2));
+  }
+  if (fork) {
+    CK(cudaEventRecord(ctx->ev[1], Lg.stream));
+    CK(cudaEventRecord(ctx->ev[2], Lk.stream));
+    CK(cudaStreamWaitEvent(L.stream, ctx->ev[1], 0));
+    CK(cudaStreamWaitEvent(L.stream, ctx->ev[2], 0));
+  }
   CKL(im_launch_prefill_append(L, call, k, v));
   if (attend) {
-    // layer outputs of the chunk's own queries, before the chunk is compressed: phi(q) and the gate logit of
-    // every chunk token (behind the indexer-side block of the projection scratch), Eq. 5 over the memory of
-    // before this chunk, then attention over (cached entries + causal chunk) with the readout added (Eq. 4)
-    if (p.mem) {
-      ImGemmArgs g2;
-      memset(&g2, 0, sizeof(g2));
-      g2.job[0] = {L.w.Wt, nullptr, p.dM, 0, 0};
-      g2.job[1] = {L.w.wg, nullptr, 1, p.dM, 0};
-      g2.n_jobs = 2;
-      g2.in[0] = (const bf16*)q;
-      g2.in_cnt[0] = 1;
-      g2.in_outer[0] = p.D;
-      g2.out = L.sc.raw + (size_t)p.S * p.max_chunk * p.R3;
-      g2.out_cnt = 1;
-      g2.out_outer = p.dM + 1;
-      g2.NV = NV;
-      g2.K = p.D;
-      g2.ksplit = 1;
-      g2.tensor = 1;
-      CKL(im_launch_gemm(L, g2));
+    // layer outputs of the chunk's own queries, before the chunk is compressed: Eq. 5 over the memory of before
+    // this chunk, then attention over (cached entries + causal chunk) with the readout added (Eq. 4)
+    if (memside) {
+      if (fork) {
+        CK(cudaEventRecord(ctx->ev[3], Lt.stream));
+        CK(cudaEventRecord(ctx->ev[4], Lw.stream));
+        CK(cudaStreamWaitEvent(L.stream, ctx->ev[3], 0));
+        CK(cudaStreamWaitEvent(L.stream, ctx->ev[4], 0));
+      }
       CKL(im_launch_chunk_readout(L, call));
     }
     if (ctx->attend_tc && im_chunk_attn_tc_supported(p)) CKL(im_launch_chunk_attention_tc(L, call, ctx->mapK, ctx->mapV, q, out));
