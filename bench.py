@@ -250,6 +250,7 @@ def run_ours(args, rank, world, device):
                    "l2": "inputs larger than L2 (each step streams %.1f GB)" % (ab["step"] / 1e9)},
         "hbm_gbs_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9,
         "hbm_frac_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "hbm_frac_step_nominal_8tbs": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / 8000.0,
         "roofline": {"bound": "hbm", "kernel": "k_attn_stream", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "traffic": args.traffic if wl.name == "llama8b_stack" and not args.tau else None, "bytes_per_launch": ab["attn_launch"],
