@@ -34,11 +34,6 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   const int i = blockIdx.x, tid = threadIdx.x;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   int32_t* ctr = st.ctr + u * CTR_STRIDE;
-  const int n = ctr[CTR_N], T = ctr[CTR_T], since = ctr[CTR_SINCE];
-  if (n < 0 || n >= p.cap) {  // never write out of bounds: flag and leave
-    if (tid == 0) atomicOr(st.status, ST_COUNT);
-    return;
-  }
   const ImRows r = im_rows(p);
   const int nq = p.HI * p.dI;
   const int dI = DI > 0 ? DI : p.dI;
@@ -46,6 +41,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   int32_t* pos = st.pos + u * p.cap;
   // ---- issue the loads of the first batch of cached entries (they depend on nothing of this call)
   constexpr int EPT = 4;
+  int n_lim = p.cap;  // entries a batch may read: the capacity until the count is known
   uint4 kraw[EPT][DI > 0 ? DI / 8 : 1];
   float imp_old[EPT];
   int pos_old[EPT];
@@ -55,7 +51,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
       const int t = b0 + e * FRONT_THREADS + tid;
       imp_old[e] = NEG_INF;
       pos_old[e] = 0;
-      if (t < n) {  // slot n is the token being appended
+      if (t < n_lim) {  // (entries at or beyond the count are read but never used; slot n is the token being appended)
         if (DI > 0) {
           const uint4* row = reinterpret_cast<const uint4*>(st.kidx + (u * p.cap + t) * dI);
 #pragma unroll
@@ -66,7 +62,14 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
       }
     }
   };
+  // the first batch goes out before the entry count is known: its addresses do not depend on it
   load_batch(0);
+  const int n = ctr[CTR_N], T = ctr[CTR_T], since = ctr[CTR_SINCE];
+  if (n < 0 || n >= p.cap) {  // never write out of bounds: flag and leave
+    if (tid == 0) atomicOr(st.status, ST_COUNT);
+    return;
+  }
+  n_lim = n;
   // the new token's K / V rows (copied into slot n below): requested now, stored after the first barrier
   const int dv = p.d / 8;
   const bool kv_here = tid < p.Hkv * dv;
