@@ -153,6 +153,8 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->sc.rpart = (float*)take((size_t)p.S * p.Dkv * 4);
   lo->sc.phiT = nullptr;
   lo->sc.vT = nullptr;
+  lo->sc.gpart_vecs = std::min<long long>((long long)p.S * p.max_chunk, 8192);
+  lo->sc.gpart = (float*)take((size_t)IM_TC_KSPLIT * lo->sc.gpart_vecs * p.R3 * 4);
   lo->sc.pack_k = 0;
   lo->sc.bpart = nullptr;
   if (p.tail > p.F) {
@@ -501,6 +503,13 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   g.K = p.D;
   g.ksplit = 1;
   g.tensor = 1;
+  // few output tiles: cut the K range over more CTAs (not next to the memory-side projections of a call with
+  // outputs, whose 80 CTAs already fill the SMs that the two indexer-side launches leave)
+  if (!(attend && p.mem) && NV <= L.sc.gpart_vecs && (p.D / 64) % IM_TC_KSPLIT == 0) {
+    g.tc_ksplit = IM_TC_KSPLIT;
+    g.part = L.sc.gpart;
+    g.part_stride = L.sc.gpart_vecs * p.R3;
+  }
   // The projections of a chunk are independent of one another and each fills a fraction of the SMs (a launch is
   // bound by the K loop of one CTA): with IM_OPT_CONCURRENCY they run next to one another on the side streams,
   // forked from and joined back into the caller's stream with events.

@@ -300,13 +300,17 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
   const int n_rows = min(GN, job.rows - r0);
   const int n_cols = (n_rows + 15) & ~15;
   const long long v0 = (long long)blockIdx.x * GM;
-  const int KT = a.K / GK;
+  // K split (not with a batched launch): this CTA's share of the K tiles and the partial buffer it writes
+  const int nks = (bt.n <= 1 && a.tc_ksplit > 1) ? a.tc_ksplit : 1;
+  const int ksi = nks > 1 ? (int)blockIdx.z : 0;
+  const int KT = a.K / GK / nks;          // K tiles of this CTA per weight term
+  const int kt0 = ksi * KT;
   const int KTOT = KT * (job.W2 ? 2 : 1);
   // batched launch: this CTA's product
   const int zb = bt.n > 1 ? (int)blockIdx.z : 0;
   const long long zu = bt.n > 1 ? (long long)bt.unit0 + bt.seq[zb] : 0;
   const int ya = (int)(v0 + zb * bt.zA_rows), yb = (int)(r0 + zb * bt.zB_rows);
-  float* out_z = a.out + zu * bt.z_out;
+  float* out_z = nks > 1 ? a.part + (long long)ksi * a.part_stride : a.out + zu * bt.z_out;
   const int32_t* gate_z = a.gate ? a.gate + zu * bt.z_gate : nullptr;
   volatile int* abort_flag = &sh->abort;
   if (tid == 0) {
@@ -340,7 +344,7 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         }
         const uint32_t bar = smem_u32(&sh->full[s]);
         const uint32_t sa = smem_u32(smem + (size_t)s * T_STAGE);
-        const int k0 = (kt % KT) * GK;
+        const int k0 = (kt0 + kt % KT) * GK;
         mbar_expect_tx(bar, T_STAGE);
         tma_load_2d(sa, &mapA, k0, ya, bar);
         tma_load_2d(sa + T_TILE, kt < KT ? &mapB0 : &mapB1, k0, yb, bar);
@@ -386,6 +390,21 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(128u) : "memory");
   }
+}
+
+// out = sum over the K splits of the partial buffers, in split order, for the rows of job j (vectors x rows, any
+// output layout: the partial buffers are laid out like `out`).  grid = ceil(NV * rows / 256), block = 256.
+__global__ void __launch_bounds__(256) k_ksplit_reduce(ImGemmArgs a, int j) {
+  const ImGemmJob job = a.job[j];
+  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= a.NV * (long long)job.rows) return;
+  const long long v = idx / job.rows;
+  const int r = (int)(idx % job.rows);
+  const long long off = a.out_t ? (long long)(job.row0 + r) * a.out_outer + v
+                                : (v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r;
+  float s = 0.f;
+  for (int k = 0; k < a.tc_ksplit; ++k) s += a.part[(long long)k * a.part_stride + off];
+  a.out[off] = s;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -464,11 +483,20 @@ cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a) {
     }
     if (enc_ok) {
       for (int j = 0; j < a.n_jobs; ++j) {
-        dim3 grid((unsigned)((a.NV + GM - 1) / GM), (unsigned)((a.job[j].rows + GN - 1) / GN), (unsigned)nb);
-        k_tc_gemm_tma<<<grid, T_THREADS, T_SMEM, L.stream>>>(mA[j], mB0[j], mB1[j], a, j, L.st.status, bt);
+        const int nks = (nb == 1 && a.tc_ksplit > 1 && !a.rmw && a.part && (a.K / GK) % a.tc_ksplit == 0) ? a.tc_ksplit : 1;
+        ImGemmArgs aj = a;
+        aj.tc_ksplit = nks;
+        dim3 grid((unsigned)((a.NV + GM - 1) / GM), (unsigned)((a.job[j].rows + GN - 1) / GN), (unsigned)(nb * nks));
+        k_tc_gemm_tma<<<grid, T_THREADS, T_SMEM, L.stream>>>(mA[j], mB0[j], mB1[j], aj, j, L.st.status, bt);
         ++*L.launches;
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
+        if (nks > 1) {
+          const long long total = a.NV * (long long)a.job[j].rows;
+          k_ksplit_reduce<<<(unsigned)((total + 255) / 256), 256, 0, L.stream>>>(aj, j);
+          ++*L.launches;
+          if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        }
       }
       return cudaSuccess;
     }

@@ -107,6 +107,8 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
                      // up to 64); room for pack_k entries in all (one sequence's tail at least)
   bf16* vT;          // [seq][Dkv][KE] the evicted values, transposed
   long long pack_k;  // entries phiT / vT have room for
+  float* gpart;      // partial results of K-split tensor-core projections: IM_TC_KSPLIT x [gpart_vecs][R3]
+  long long gpart_vecs;
   float* bpart;      // [pack_k / 32][dM] sums of phi^2 over the 32 entries of a block of the packed operands
   float* mch;        // [max_seqs][max_chunk][Dkv] gated memory readout of a chunk's own queries (im_prefill_chunk_attend)
   uint8_t* qpack;    // [n_seq][ceil(C / IM_TC_QT)][IM_TC_TILE_BYTES] query operand of the tensor-core prefill scoring
@@ -156,6 +158,12 @@ struct ImGemmArgs {
   int direct;  // 1: few vectors (decode) - the variant without shared-memory staging, if the K split is a multiple of 32
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
   int smem_floor;  // direct variant: dynamic shared memory to ask for although the kernel uses none (IM_SMEM_SIDE)
+  // tensor-core TMA variant only: tc_ksplit > 1 cuts the K range over that many CTAs per output tile (launches of
+  // few tiles are bound by the K loop of one CTA); split s writes to part + s * part_stride in the layout of `out`,
+  // and a second kernel adds the splits into `out` in a fixed order.  Not with rmw or a batched launch.
+  int tc_ksplit;
+  float* part;
+  long long part_stride;
   const struct ImGemmBatch* batch;  // host pointer, tensor-core TMA variant only: several products in one launch
   // tensor-core variant only:
   int out_t;            // 1: the result goes to out[(row0 + r) * out_outer + v] (vectors contiguous) instead
@@ -202,6 +210,7 @@ cudaError_t im_front_prepare_decode();
 cudaError_t im_prefetch_prepare_decode();
 
 #define IM_MRES_ROW(p) ((p).Dkv + 4)
+#define IM_TC_KSPLIT 4  /* K splits of the prefill projections on the tensor cores (chunks of up to 8192 vectors) */
 
 // Decode calls of few sequences split the SMs between the two kinds of work of a call: the streaming kernels
 // (attention over the cache, readout over Mhat), bound by HBM bandwidth, and the chain of small kernels that
