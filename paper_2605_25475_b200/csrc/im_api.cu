@@ -479,6 +479,7 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   }
   call.C = chunk_len;
   call.prefill = 1;
+  call.due = 1;
   call.ksplit = 1;
   call.ksplit_key = 1;
   call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
@@ -640,6 +641,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     return fail(IM_ERR_ARG, "sequences of one decode call must be at the same phase of the compression interval");
   const bool due = due_all;
   if (!due) ne_max = 0;
+  call.due = due ? 1 : 0;
   call.C = 1;
   call.prefill = 0;
   call.ksplit = pick_ksplit(p.D, IM_KSPLIT);
@@ -749,7 +751,6 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   if (conc) CK(cudaEventRecord(ctx->ev[4], L4.stream));
   if (conc) {
     CK(cudaStreamWaitEvent(L1.stream, ctx->ev[2], 0));
-    if (mem_write) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[7], 0));  // the front kernel changes the counters the fold reads
   }
   // append + a1 (+ a2 and the gather of the evicted pairs when the evicted set is small enough for one
   // block per sequence; a4 in the same kernel unless the compaction is deferred)

@@ -120,6 +120,8 @@ struct ImCall {
   int defer;      // decode: 1 = the attention kernel runs over the entries cached before the call while the front
                   // kernel appends / scores / selects; the merge adds the new token and takes the evicted entries
                   // out again, and the holes are filled (and CTR_N advanced) by the call's last kernel
+  int due;        // decode: 1 = this call compresses (the host checks that all its sequences are at that phase of the
+                  // interval); prefill calls always do
   int fold_all;   // prefill with outputs: fold the pending list of every sequence first (the chunk readout reads Mhat alone)
   int pack;       // prefill: 1 = the append kernel also writes the operand records of the tensor-core scoring
   int phi_large;  // 1: phi of the evicted keys lives in ImScratch::phi, 0: in the K-split partials phip
@@ -280,8 +282,7 @@ cudaError_t im_launch_fold_theta(const ImDims& p, const ImWeights& w, cudaStream
 
 // Evict-step bookkeeping shared by the memory kernels: number of entries the compression of this
 // call will evict for a sequence whose counters are still those from before the call.
-__host__ __device__ inline int im_upcoming_evictions(const ImDims& p, int prefill, int C, int n, int since) {
-  const bool due = prefill || (since + 1 == p.tau);
+__host__ __device__ inline int im_upcoming_evictions(const ImDims& p, int due, int C, int n) {
   const int over = n + C - p.B;
   return (due && over > 0) ? over : 0;
 }

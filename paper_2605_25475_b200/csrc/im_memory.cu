@@ -21,7 +21,9 @@ namespace {
 __device__ __forceinline__ bool fold_needed(const ImDims& p, const ImCall& call, const int32_t* ctr, float cscale) {
   if (!p.mem) return false;
   if (call.fold_all) return ctr[CTR_NPEND] > 0 || cscale != 1.0f;
-  const int ne = im_upcoming_evictions(p, call.prefill, call.C, ctr[CTR_N], ctr[CTR_SINCE]);
+  // (the phase of the interval comes from the host, not from the counter the decode front kernel advances, so
+  // that the fold kernels and the front kernel do not depend on one another)
+  const int ne = im_upcoming_evictions(p, call.prefill || call.due, call.C, ctr[CTR_N]);
   const int np = ctr[CTR_NPEND];
   if (ne <= 0) return false;
   if (ne > p.F) return np > 0 || cscale != 1.0f;  // a large set is accumulated into Mhat with cscale == 1
