@@ -77,68 +77,108 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // mch[i][s][col] = g(q_s) * cscale * (sum_m phi_s[m] Mhat[m][col]) / (eps + sum_m phi_s[m]^2 b[m])   (Eq. 5,
 // gate of Eq. 4).  The pending list is empty here (the call folds it first).  phi_s and the gate logit are
 // rows [0, dM) and dM of the chunk's memory-side projection, which the call writes behind the indexer-side
-// block of the projection scratch.  grid = (ceil(Dkv / 64), ceil(C / 64), n_seq), block = 256,
-// 64 x 64 tiles with 4 x 4 micro tiles.
+// block of the projection scratch.  A float32 GEMM on the CUDA cores ([C x d_M] x [d_M x D_kv], 2.1 GFLOP per
+// 2048-token chunk): 128 x 128 output tile per block, 8 x 8 micro tile per thread (two 4-wide halves 64 apart in
+// both directions, so that a warp's shared-memory reads are conflict free), K slices of 16 staged through
+// registers into shared memory while the previous slice is multiplied.
+// grid = (ceil(Dkv / 128), ceil(C / 128), n_seq), block = 256.
+constexpr int CR_T = 128, CR_K = 16;
 __global__ void __launch_bounds__(256) k_chunk_readout(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call) {
-  __shared__ float s_a[16][64 + 4];  // [m][query]
-  __shared__ float s_b[16][64 + 4];  // [m][col]
-  __shared__ float s_bv[16];
+  __shared__ __align__(16) float s_a[2][CR_K][CR_T + 4];  // [m][query] (padded: the staging stores of a warp spread over the banks)
+  __shared__ __align__(16) float s_b[2][CR_K][CR_T + 4];  // [m][col]
+  __shared__ float s_bv[2][CR_K];
   const int i = blockIdx.z;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const float* proj = sc.raw + (size_t)p.S * p.max_chunk * p.R3;  // [n_seq * C][dM + 1]
   const int ps = p.dM + 1;
-  const int q0 = blockIdx.y * 64, col0 = blockIdx.x * 64;
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int q0 = blockIdx.y * CR_T, col0 = blockIdx.x * CR_T;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const float* Mh = st.Mhat + u * p.dM * p.Dkv;
   const float* bv = st.bvec + u * p.dM;
-  float acc[4][4], den[4];
+  // staging roles: A - thread t loads m = t & 15 of queries (t >> 4) + 16 j, j < 8 (16 consecutive floats of a
+  // projection row per 16 threads); B - thread t loads float4 (t & 31) of rows (t >> 5) and (t >> 5) + 8
+  const int am = tid & 15, as = tid >> 4;
+  const int bc = (tid & 31) * 4, bm = tid >> 5;
+  const bool b_vec = (p.Dkv & 3) == 0;
+  float ra[8];
+  float4 rb[2];
+  float rbv = 0.f;
+  auto fetch = [&](int m0) {
 #pragma unroll
-  for (int a = 0; a < 4; ++a) {
+    for (int j = 0; j < 8; ++j) {
+      const int s = q0 + as + 16 * j, m = m0 + am;
+      ra[j] = (s < call.C && m < p.dM) ? proj[((size_t)i * call.C + s) * ps + m] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int m = m0 + bm + 8 * j, c = col0 + bc;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (m < p.dM) {
+        const float* src = Mh + (size_t)m * p.Dkv + c;
+        if (b_vec && c + 3 < p.Dkv) v = *reinterpret_cast<const float4*>(src);
+        else {
+          if (c < p.Dkv) v.x = src[0];
+          if (c + 1 < p.Dkv) v.y = src[1];
+          if (c + 2 < p.Dkv) v.z = src[2];
+          if (c + 3 < p.Dkv) v.w = src[3];
+        }
+      }
+      rb[j] = v;
+    }
+    if (tid < CR_K) rbv = m0 + tid < p.dM ? bv[m0 + tid] : 0.f;
+  };
+  auto stash = [&](int buf) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s_a[buf][am][as + 16 * j] = ra[j];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) *reinterpret_cast<float4*>(&s_b[buf][bm + 8 * j][bc]) = rb[j];
+    if (tid < CR_K) s_bv[buf][tid] = rbv;
+  };
+  float acc[8][8], den[8];
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
     den[a] = 0.f;
 #pragma unroll
-    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+    for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
   }
-  for (int m0 = 0; m0 < p.dM; m0 += 16) {
-    __syncthreads();
-    for (int k = threadIdx.x; k < 16 * 64; k += blockDim.x) {
-      const int s = k >> 4, m = k & 15;  // consecutive threads along m: contiguous in the projection row
-      float av = 0.f;
-      if (q0 + s < call.C && m0 + m < p.dM) av = proj[((size_t)i * call.C + q0 + s) * ps + m0 + m];
-      s_a[m][s] = av;
-      const int mm = k >> 6, c = k & 63;  // consecutive threads along the columns of Mhat
-      float bvv = 0.f;
-      if (m0 + mm < p.dM && col0 + c < p.Dkv) bvv = Mh[(size_t)(m0 + mm) * p.Dkv + col0 + c];
-      s_b[mm][c] = bvv;
-    }
-    if (threadIdx.x < 16) s_bv[threadIdx.x] = m0 + threadIdx.x < p.dM ? bv[m0 + threadIdx.x] : 0.f;
-    __syncthreads();
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  const int nk = (p.dM + CR_K - 1) / CR_K;
+  for (int kb = 0; kb < nk; ++kb) {
+    const int buf = kb & 1;
+    if (kb + 1 < nk) fetch((kb + 1) * CR_K);
 #pragma unroll
-    for (int m = 0; m < 16; ++m) {
-      float av[4], bb[4];
+    for (int m = 0; m < CR_K; ++m) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&s_a[buf][m][ty * 4]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&s_a[buf][m][64 + ty * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&s_b[buf][m][tx * 4]);
+      const float4 b1 = *reinterpret_cast<const float4*>(&s_b[buf][m][64 + tx * 4]);
+      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+      const float bmv = s_bv[buf][m];
 #pragma unroll
-      for (int a = 0; a < 4; ++a) av[a] = s_a[m][ty * 4 + a];
+      for (int a = 0; a < 8; ++a) {
+        den[a] = fmaf(av[a] * av[a], bmv, den[a]);
 #pragma unroll
-      for (int b = 0; b < 4; ++b) bb[b] = s_b[m][tx * 4 + b];
-      const float bm = s_bv[m];
-#pragma unroll
-      for (int a = 0; a < 4; ++a) {
-        den[a] = fmaf(av[a] * av[a], bm, den[a]);
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bb[b], acc[a][b]);
+        for (int b = 0; b < 8; ++b) acc[a][b] = fmaf(av[a], bb[b], acc[a][b]);
       }
     }
+    if (kb + 1 < nk) stash(buf ^ 1);  // (the other buffer: last read before the barrier that ended slice kb - 1)
+    __syncthreads();
   }
   const float cs = st.cscale[u];
 #pragma unroll
-  for (int a = 0; a < 4; ++a) {
-    const int s = q0 + ty * 4 + a;
+  for (int a = 0; a < 8; ++a) {
+    const int s = q0 + (a < 4 ? ty * 4 + a : 64 + ty * 4 + a - 4);
     if (s >= call.C) continue;
     const float logit = proj[((size_t)i * call.C + s) * ps + p.dM] + w.bg[0];
     const float f = cs / (1.0f + expf(-logit)) / (p.eps + den[a]);
+    float* dst = sc.mch + ((size_t)i * call.C + s) * p.Dkv;
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int col = col0 + tx * 4 + b;
-      if (col < p.Dkv) sc.mch[((size_t)i * call.C + s) * p.Dkv + col] = f * acc[a][b];
+    for (int b = 0; b < 8; ++b) {
+      const int col = col0 + (b < 4 ? tx * 4 + b : 64 + tx * 4 + b - 4);
+      if (col < p.Dkv) dst[col] = f * acc[a][b];
     }
   }
 }
@@ -363,7 +403,7 @@ cudaError_t im_chunk_attn_prepare(const ImDims& p) {
 }
 
 cudaError_t im_launch_chunk_readout(const ImLaunch& L, const ImCall& call) {
-  dim3 grid((L.p.Dkv + 63) / 64, (call.C + 63) / 64, call.n_seq);
+  dim3 grid((L.p.Dkv + CR_T - 1) / CR_T, (call.C + CR_T - 1) / CR_T, call.n_seq);
   k_chunk_readout<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.w, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
