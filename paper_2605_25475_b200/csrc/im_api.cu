@@ -306,6 +306,13 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
     g.out_outer = (long long)p.tail * p.dM;
     g.ksplit = 1;
     g.ks_stride = 0;
+    // a prefill chunk's few output tiles: two CTAs per tile over the K range, where the partial buffers have room
+    const long long extent = (long long)call.n_seq * p.tail * p.dM;
+    if (call.prefill && (p.Dkv / 64) % 2 == 0 && 2 * extent <= (long long)IM_TC_KSPLIT * L.sc.gpart_vecs * p.R3) {
+      g.tc_ksplit = 2;
+      g.part = L.sc.gpart;
+      g.part_stride = extent;
+    }
   } else {
     call.phi_large = 0;
     g.out = L.sc.phip;
@@ -592,9 +599,22 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   // a2: selection (also restarts the pooling); a4: gather the evicted pairs, fill the holes
   CKL(im_launch_select(L, call));
   if (ne_max > 0) {
-    CKL(im_launch_gather_move(L, call, ne_max));
-    // a3: memory write
-    if (p.mem && (rc = run_memory_write(ctx, L, call, ne_max))) return rc;
+    if (fork && p.mem) {
+      // the holes are filled next to the memory write, which works from the gathered copies
+      ImLaunch Lm = L;
+      Lm.stream = ctx->side[0];
+      CKL(im_launch_gather(L, call, ne_max));
+      CK(cudaEventRecord(ctx->ev[5], L.stream));
+      CK(cudaStreamWaitEvent(Lm.stream, ctx->ev[5], 0));
+      CKL(im_launch_move(Lm, call, ne_max));
+      CK(cudaEventRecord(ctx->ev[6], Lm.stream));
+      if ((rc = run_memory_write(ctx, L, call, ne_max))) return rc;  // a3
+      CK(cudaStreamWaitEvent(L.stream, ctx->ev[6], 0));
+    } else {
+      CKL(im_launch_gather_move(L, call, ne_max));
+      // a3: memory write
+      if (p.mem && (rc = run_memory_write(ctx, L, call, ne_max))) return rc;
+    }
   }
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];

@@ -367,15 +367,23 @@ cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call) {
   return cudaGetLastError();
 }
 
-cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max) {
+// gather of the evicted pairs / move of the retained entries into the holes: every gather must be done before a
+// move overwrites an evicted slot (stream order, or an event between the two launches)
+cudaError_t im_launch_gather(const ImLaunch& L, const ImCall& call, int ne_max) {
   dim3 grid((ne_max + 3) / 4, call.n_seq);
   k_gather_evicted<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  return cudaGetLastError();
+}
+cudaError_t im_launch_move(const ImLaunch& L, const ImCall& call, int ne_max) {
+  dim3 grid((ne_max + 3) / 4, call.n_seq);
   k_move_survivors<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
+}
+cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max) {
+  const cudaError_t e = im_launch_gather(L, call, ne_max);
+  return e != cudaSuccess ? e : im_launch_move(L, call, ne_max);
 }
 
 cudaError_t im_front_prepare_decode() {

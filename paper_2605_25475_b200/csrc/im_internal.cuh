@@ -241,6 +241,8 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
                                    int do_select, int n_max, int smem_floor);
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
+cudaError_t im_launch_gather(const ImLaunch& L, const ImCall& call, int ne_max);
+cudaError_t im_launch_move(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call);
 // ne_host: per call sequence, the number of entries the compression of this call evicts (host mirror)
