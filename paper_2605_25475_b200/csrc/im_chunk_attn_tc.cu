@@ -1,24 +1,29 @@
 // Layer outputs of a prefill chunk's own queries (Eq. 4-5 during chunked prefill): the flash attention of
 // im_chunk_attn.cu on the 5th-generation tensor cores, for head_dim 128.
 //
-// A CTA owns 128 rows = floor(128 / G_q) queries x G_q heads of one KV head; row r is TMEM lane r and belongs to
-// softmax thread r.  Per tile of 64 keys:
+// A CTA owns 128 rows = floor(128 / G_q) queries x G_q heads of one KV head; row r is TMEM lane r.  Per tile of 64 keys:
 //   S = Q K^T      tcgen05.mma, M = 128 rows, N = 64 keys, K = d = 128 (8 steps); Q and the K tile K-major in shared
 //                  memory (128-byte swizzle; the K/V tiles come by TMA through the tensor maps of the decode
 //                  attention kernel, two 32-row boxes per 64-column half), S in tensor memory (double buffered)
-//   softmax        thread r reads its 64 scores with tcgen05.ld, masks (causal by chunk index), keeps the running
-//                  maximum and sum (base 2), and writes P as two bf16 terms (2^-17) into shared memory in the
-//                  K-major swizzled operand layout
-//   O += P V       tcgen05.mma, N = d = 128, K = 64 keys (4 steps, both P terms), accumulating in tensor memory
-//                  over the tiles; V is used as it lies in the cache ([key][d], i.e. MN-major for this product:
-//                  8-key groups 1024 bytes apart, the two 64-column halves 8 KB apart)
+//   softmax        two threads per row (32 keys each) read their scores with tcgen05.ld, mask (causal by chunk
+//                  index), exchange the maxima, keep the running maximum and sum (base 2), and write P as two bf16
+//                  terms (upper 16 bits + rounded remainder: 2^-16) into TENSOR memory with tcgen05.st, two values per
+//                  32-bit column, row = lane: the layout of an A operand read from tensor memory
+//   O += P V       tcgen05.mma with A = P from tensor memory, N = d = 128, K = 64 keys (4 steps, both P terms),
+//                  accumulating in tensor memory over the tiles; V is used as it lies in the cache ([key][d], i.e.
+//                  MN-major for this product: 8-key groups 1024 bytes apart, the two 64-column halves 8 KB apart)
 //   rescale        P is formed relative to a reference maximum that is only raised when a row's maximum has
 //                  grown by more than 2^8 (or is seen for the first time): then the warp waits for the previous
 //                  P V product, multiplies its O rows in tensor memory (tcgen05.ld / st) and its row sums by
 //                  2^(m_ref_old - m_ref_new).  Between such events P (<= 2^8) and O need no correction, so the
 //                  softmax of tile j + 1 overlaps with the P V product of tile j (P is double buffered).
-// Warps 0-3: softmax / accumulate / epilogue; warp 4 lane 0: TMA; warp 5: tensor memory owner, lane 0 issues the
-// MMAs.  Every wait is bounded (ST_TIMEOUT).
+// Tensor memory (512 columns): S 0..127, O 128..255, P 256..383.
+// Warps 0-7: softmax / rescale / epilogue (two groups of four: each row's 64 keys of a tile and its 128 output
+// columns are split between two threads); warp 8 lane 0: TMA; warp 9: tensor memory owner and MMA issue.  The whole
+// of warp 9 runs the issue loop and one elected lane issues each instruction: with the loop inside an
+// `if (lane == 0)` the operand descriptors were per-thread values that had to be moved to uniform registers for every
+// instruction, and the issue itself (70-90 cycles per MMA of 32-64 cycles) bounded the kernel.
+// Every wait is bounded (ST_TIMEOUT).
 #include <cuda.h>
 
 #include "im_internal.cuh"
@@ -29,22 +34,24 @@ constexpr float NEG_INF = -__builtin_huge_valf();
 constexpr int DH = 128;
 constexpr int KT = 64;                      // keys per tile
 constexpr int ROWS = 128;
-constexpr int STAGES = 3;
+constexpr int STAGES = 5;
 constexpr int HALF_BYTES = KT * 128;        // one 64-column half of a K or V tile: 64 rows x 128 bytes
 constexpr int KV_TILE = 2 * HALF_BYTES;     // 16 KB
 constexpr int STAGE_BYTES = 2 * KV_TILE;    // K + V
 constexpr int Q_BYTES = ROWS * DH * 2;      // 32 KB: two halves of 128 rows x 128 bytes
-constexpr int P_BYTES = ROWS * KT * 2;      // 16 KB per term
-constexpr int THREADS = 192;
+constexpr int THREADS = 320;                // warps 0-7: softmax (two groups of four), 8: TMA, 9: tensor memory / MMA
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
-constexpr int TMEM_COLS = 256;              // S: 2 x 64, O: 128
+constexpr int TMEM_COLS = 512;              // S: 2 x 64, O: 128, P: 2 buffers x 2 terms x 32 (bf16 pairs); a power of two
+constexpr int P_COL = 256;                  // first column of P; buffer b, term t at P_COL + 64 b + 32 t
 
 struct Shared {
   unsigned long long full[STAGES], empty[STAGES], sfull[2], sempty[2], pfull[2], pvdone[2];
+  unsigned long long xch[2][4];   // row statistics of the two softmax groups exchanged: [tile parity][lane quarter]
+  float stat[2][2][ROWS];         // [tile parity][group][row]
   uint32_t tmem;
   int abort;
 };
-constexpr int SMEM_BYTES = Q_BYTES + 4 * P_BYTES + STAGES * STAGE_BYTES + (int)sizeof(Shared) + 1024;
+constexpr int SMEM_BYTES = Q_BYTES + STAGES * STAGE_BYTES + (int)sizeof(Shared) + 1024;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -88,14 +95,29 @@ __device__ __forceinline__ uint64_t desc_sw128(uint32_t addr, uint32_t lbo, uint
 }
 __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
       "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// the same with the A operand in tensor memory (row = lane, two bf16 per 32-bit column along K)
+__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar)
+      : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   uint32_t r[32];
@@ -127,6 +149,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
       "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+      "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
 // 2^x, x <= 8 here; -inf gives 0
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -139,7 +168,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
-// grid = (ceil(C / QB), Hkv, n_seq) with QB = 128 / Gq queries per CTA; block = 192.
+// grid = (ceil(C / QB), Hkv, n_seq) with QB = 128 / Gq queries per CTA; block = 320.
 template <typename OutT>
 __global__ void __launch_bounds__(THREADS, 1)
 k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, ImDims p, ImState st,
@@ -147,8 +176,7 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* s_q = smem;                       // [2 halves][128 rows][128 bytes]
-  uint8_t* s_p = smem + Q_BYTES;             // [2 buffers][2 terms][128 rows][128 bytes]
-  uint8_t* s_kv = s_p + 4 * P_BYTES;         // [STAGES][K: 2 halves x 64 rows x 128 bytes | V: the same]
+  uint8_t* s_kv = smem + Q_BYTES;            // [STAGES][K: 2 halves x 64 rows x 128 bytes | V: the same]
   Shared* sh = reinterpret_cast<Shared*>(s_kv + STAGES * STAGE_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.y, i = blockIdx.z;
@@ -170,18 +198,19 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&sh->sfull[b]), 1);
-      mbar_init(smem_u32(&sh->sempty[b]), ROWS);
+      mbar_init(smem_u32(&sh->sempty[b]), 2 * ROWS);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&sh->pfull[b]), ROWS);
+      mbar_init(smem_u32(&sh->pfull[b]), 2 * ROWS);
       mbar_init(smem_u32(&sh->pvdone[b]), 1);
+      for (int qd = 0; qd < 4; ++qd) mbar_init(smem_u32(&sh->xch[b][qd]), 64);
     }
     sh->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem)),
                  "r"((uint32_t)TMEM_COLS)
                  : "memory");
@@ -192,12 +221,15 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
   int lim = 0;          // this row sees slots [0, lim)
   bool row_ok = false;
   int s_row = s0, hh = 0;
-  if (tid < ROWS) {
-    const int sl = tid / p.Gq;
-    hh = tid % p.Gq;
+  const int row = tid & (ROWS - 1);  // softmax threads: the row (both groups), TMEM lane
+  if (tid < 2 * ROWS) {
+    const int sl = row / p.Gq;
+    hh = row % p.Gq;
     s_row = s0 + sl;
     row_ok = sl < QB && s_row < C;
     lim = row_ok ? n0 + s_row + 1 : 0;
+  }
+  if (tid < ROWS) {
     const uint4* src = reinterpret_cast<const uint4*>(q + (((size_t)i * C + (row_ok ? s_row : s0)) * p.H + (size_t)h * p.Gq + (row_ok ? hh : 0)) * DH);
 #pragma unroll
     for (int c = 0; c < 16; ++c) {
@@ -213,7 +245,7 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
   const uint32_t t_o = tmem + 128;  // O columns; S buffers at columns 0 and 64
   bool ok = true;
 
-  if (warp == 4) {
+  if (warp == 8) {
     if (lane == 0) {  // ---- TMA: K and V tiles of 64 keys, two 32-row boxes per 64-column half
       const int row_base = (int)((u * p.Hkv + h) * (size_t)p.cap);
       for (int j = 0; j < nt; ++j) {
@@ -231,11 +263,11 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
           }
       }
     }
-  } else if (warp == 5) {
-    if (lane == 0) {  // ---- MMA issue
+  } else if (warp == 9) {
+    {  // ---- MMA issue: the whole warp runs the loop (descriptors stay warp-uniform), one elected lane issues
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
       const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
-      const uint32_t qa = smem_u32(s_q), pa = smem_u32(s_p);
+      const uint32_t qa = smem_u32(s_q);
       auto issue_s = [&](int j) -> bool {  // S(j) = Q K_j^T into S buffer j & 1
         const int s = j % STAGES, b = j & 1;
         if (!mbar_wait(smem_u32(&sh->full[s]), (uint32_t)((j / STAGES) & 1), abort_flag)) return false;
@@ -260,34 +292,41 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
         for (int term = 0; term < 2; ++term)
 #pragma unroll
           for (int ks = 0; ks < KT / 16; ++ks)
-            mma_bf16(t_o, desc_sw128(pa + (2 * b + term) * P_BYTES + ks * 32, 16, 1024), desc_sw128(va + ks * 2048, HALF_BYTES, 1024),
-                     idesc_o, (j | term | ks) ? 1u : 0u);
+            mma_bf16_ts(t_o, tmem + (uint32_t)(P_COL + 64 * b + 32 * term + 8 * ks), desc_sw128(va + ks * 2048, HALF_BYTES, 1024),
+                        idesc_o, (j | term | ks) ? 1u : 0u);
         mma_commit(smem_u32(&sh->pvdone[b]));
         mma_commit(smem_u32(&sh->empty[s]));
       }
     }
   } else {
-    // ---- softmax, rescale, epilogue: thread = row = TMEM lane
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    // ---- softmax, rescale, epilogue.  Two groups of four warps: thread (group g, row r) owns keys 32 g .. 32 g + 31
+    // of every tile of row r = TMEM lane r (warps w and w + 4 may both read lane quarter w) and, for the rescale and
+    // the epilogue, columns 64 g .. 64 g + 63 of O.  The two threads of a row exchange their maxima (and at the end
+    // their sums) through shared memory and an mbarrier per lane quarter, and take every decision alike.
+    const int grp = warp >> 2, qd = warp & 3;
+    const uint32_t lane_addr = (uint32_t)(qd * 32) << 16;
     const float sl2 = p.scale * 1.4426950408889634f;  // softmax in base 2
-    float m_ref = NEG_INF, l = 0.f;                    // reference maximum of P and O, row sum relative to it
+    float m_ref = NEG_INF, l = 0.f;                    // reference maximum of P and O, this thread's share of the row sum
     for (int j = 0; j < nt; ++j) {
       const int b = j & 1;
       if (!mbar_wait(smem_u32(&sh->sfull[b]), (uint32_t)((j >> 1) & 1), abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      float sv[KT];
-      tmem_ld32(tmem + lane_addr + (uint32_t)(b * KT), sv);
-      tmem_ld32(tmem + lane_addr + (uint32_t)(b * KT + 32), sv + 32);
+      float sv[32];
+      tmem_ld32(tmem + lane_addr + (uint32_t)(b * KT + grp * 32), sv);
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       mbar_arrive(smem_u32(&sh->sempty[b]));
-      const int key0 = j * KT;
+      const int key0 = j * KT + grp * 32;
       float tm = NEG_INF;
-      if (key0 + KT > lim) {  // only the row's last tiles need the causal mask
+      if (key0 + 32 > lim) {  // only the row's last tiles need the causal mask
 #pragma unroll
-        for (int k = 0; k < KT; ++k) sv[k] = key0 + k < lim ? sv[k] : NEG_INF;
+        for (int k = 0; k < 32; ++k) sv[k] = key0 + k < lim ? sv[k] : NEG_INF;
       }
 #pragma unroll
-      for (int k = 0; k < KT; ++k) tm = fmaxf(tm, sv[k]);
+      for (int k = 0; k < 32; ++k) tm = fmaxf(tm, sv[k]);
+      sh->stat[b][grp][row] = tm;
+      mbar_arrive(smem_u32(&sh->xch[b][qd]));
+      if (!mbar_wait(smem_u32(&sh->xch[b][qd]), (uint32_t)((j >> 1) & 1), abort_flag)) { ok = false; break; }
+      tm = fmaxf(tm, sh->stat[b][grp ^ 1][row]);
       tm *= sl2;  // the scale is positive: the maximum of the scaled scores
       // raise the reference only for a first maximum or a jump of more than 8 (P stays below 2^8 otherwise)
       const bool raise = tm > NEG_INF && (m_ref == NEG_INF || tm > m_ref + 8.0f);
@@ -297,42 +336,50 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
           m_ref = tm;
           l *= corr;
         }
-        if (j >= 1) {  // O holds the products up to tile j - 1: wait for the last one, then scale the rows
+        if (j >= 1) {  // O holds the products up to tile j - 1: wait for the last one, then scale this thread's half row
           if (!mbar_wait(smem_u32(&sh->pvdone[(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-          for (int c0 = 0; c0 < DH; c0 += 32) {
+          for (int c0 = 0; c0 < DH / 2; c0 += 32) {
             float t[32];
-            tmem_ld32(t_o + lane_addr + (uint32_t)c0, t);
+            tmem_ld32(t_o + lane_addr + (uint32_t)(grp * (DH / 2) + c0), t);
 #pragma unroll
             for (int c = 0; c < 32; ++c) t[c] *= corr;
-            tmem_st32(t_o + lane_addr + (uint32_t)c0, t);
+            tmem_st32(t_o + lane_addr + (uint32_t)(grp * (DH / 2) + c0), t);
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         }
       }
       // P buffer b was last read by the product of tile j - 2
       if (j >= 2 && !mbar_wait(smem_u32(&sh->pvdone[b]), (uint32_t)(((j >> 1) - 1) & 1), abort_flag)) { ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const float e = m_ref == NEG_INF ? 0.f : m_ref;
-      uint8_t* prow = s_p + (size_t)(2 * b) * P_BYTES + (tid >> 3) * 1024 + (tid & 7) * 128;
+      uint32_t hi[16], lo[16];
 #pragma unroll
-      for (int c = 0; c < KT / 8; ++c) {
-        uint32_t hi[4], lo[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float p0 = ex2(fmaf(sv[c * 8 + 2 * k], sl2, -e)), p1 = ex2(fmaf(sv[c * 8 + 2 * k + 1], sl2, -e));
-          l += p0 + p1;
-          hi[k] = pack_bf16(p0, p1);
-          lo[k] = pack_bf16(p0 - __uint_as_float(hi[k] << 16), p1 - __uint_as_float(hi[k] & 0xffff0000u));
-        }
-        uint8_t* dst = prow + ((c ^ (tid & 7)) << 4);
-        *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(dst + P_BYTES) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      for (int k = 0; k < 16; ++k) {
+        const float p0 = ex2(fmaf(sv[2 * k], sl2, -e)), p1 = ex2(fmaf(sv[2 * k + 1], sl2, -e));
+        l += p0 + p1;
+        // bf16 split on the integer pipe: first term = the upper 16 bits, second = the remainder rounded half up
+        const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+        hi[k] = __byte_perm(b0, b1, 0x7632);
+        const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+        lo[k] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      const uint32_t t_p = tmem + lane_addr + (uint32_t)(P_COL + 64 * b + 16 * grp);
+      tmem_st16(t_p, hi);
+      tmem_st16(t_p + 32, lo);
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       mbar_arrive(smem_u32(&sh->pfull[b]));
     }
-    // ---- epilogue: O / l + gated readout
+    // ---- epilogue: O / l + gated readout; the row sum is the two threads' shares added
+    if (ok) {
+      const int b = nt & 1;  // the exchange barrier of the parity after the last tile: used (nt - b + 1) / 2 times so far
+      sh->stat[b][grp][row] = l;
+      mbar_arrive(smem_u32(&sh->xch[b][qd]));
+      if (!mbar_wait(smem_u32(&sh->xch[b][qd]), (uint32_t)((nt >> 1) & 1), abort_flag)) ok = false;
+      l += sh->stat[b][grp ^ 1][row];
+    }
     if (ok && !mbar_wait(smem_u32(&sh->pvdone[(nt - 1) & 1]), (uint32_t)(((nt - 1) >> 1) & 1), abort_flag)) ok = false;
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -340,7 +387,8 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
       const float* mr = sc.mch + ((size_t)i * C + (row_ok ? s_row : 0)) * p.Dkv + h * DH;
       OutT* op = out + (((size_t)i * C + (row_ok ? s_row : 0)) * p.H + (size_t)h * p.Gq + hh) * DH;
 #pragma unroll
-      for (int c0 = 0; c0 < DH; c0 += 32) {
+      for (int c1 = 0; c1 < DH / 2; c1 += 32) {
+        const int c0 = grp * (DH / 2) + c1;
         float t[32];
         tmem_ld32(t_o + lane_addr + (uint32_t)c0, t);  // (warp-collective: rows out of range load too, and skip the store)
         if (row_ok) {
@@ -369,7 +417,7 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
   }
