@@ -72,16 +72,23 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t addr) {
   d |= (uint64_t)1 << 46;  // descriptor version of this architecture
   return d;
 }
+// Called by a whole (converged) warp: one elected lane issues.  The operands then stay warp-uniform values; issued
+// from inside an `if (lane == 0)` they were per-thread values moved to uniform registers before every instruction.
 __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
       "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar)
+      : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   uint32_t r[32];
@@ -225,8 +232,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_tc_gemm(ImGemmArgs a, int32_t*
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
-  } else if (lane == 0) {
-    // ---- MMA issue: four K = 16 steps per stage
+  } else {
+    // ---- MMA issue (whole warp, one elected lane issues): four K = 16 steps per stage
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | ((uint32_t)(GM >> 4) << 24);
     for (int kt = 0; kt < KTOT; ++kt) {
       const int s = kt % G_STAGES;
@@ -351,7 +358,7 @@ k_tc_gemm_tma(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    {  // MMA issue: whole warp, one elected lane issues
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | ((uint32_t)(GM >> 4) << 24);
       for (int kt = 0; kt < KTOT; ++kt) {
         const int s = kt % T_STAGES;
