@@ -1,28 +1,31 @@
 // Layer outputs of a prefill chunk's own queries (Eq. 4-5 during chunked prefill): the flash attention of
 // im_chunk_attn.cu on the 5th-generation tensor cores, for head_dim 128.
 //
-// A CTA owns 128 rows = floor(128 / G_q) queries x G_q heads of one KV head; row r is TMEM lane r.  Per tile of 64 keys:
-//   S = Q K^T      tcgen05.mma, M = 128 rows, N = 64 keys, K = d = 128 (8 steps); Q and the K tile K-major in shared
+// A CTA owns two Q tiles of 128 rows each = 2 floor(128 / G_q) queries x G_q heads of one KV head; row r of tile g is
+// TMEM lane r and belongs to softmax thread (g, r).  Per tile of 64 keys and per Q tile g:
+//   S_g = Q_g K^T  tcgen05.mma, M = 128 rows, N = 64 keys, K = d = 128 (8 steps); Q_g and the K tile K-major in shared
 //                  memory (128-byte swizzle; the K/V tiles come by TMA through the tensor maps of the decode
-//                  attention kernel, two 32-row boxes per 64-column half), S in tensor memory (double buffered)
-//   softmax        two threads per row (32 keys each) read their scores with tcgen05.ld, mask (causal by chunk
-//                  index), exchange the maxima, keep the running maximum and sum (base 2), and write P as two bf16
-//                  terms (upper 16 bits + rounded remainder: 2^-16) into TENSOR memory with tcgen05.st, two values per
-//                  32-bit column, row = lane: the layout of an A operand read from tensor memory
-//   O += P V       tcgen05.mma with A = P from tensor memory, N = d = 128, K = 64 keys (4 steps, both P terms),
+//                  attention kernel, two 32-row boxes per 64-column half, and serve both Q tiles), S_g in tensor memory
+//   softmax        thread (g, r) reads its 64 scores with tcgen05.ld, masks (causal by chunk index), keeps the running
+//                  maximum and sum (base 2), and writes P as two bf16 terms (upper 16 bits + rounded remainder: 2^-16)
+//                  into TENSOR memory with tcgen05.st, two values per 32-bit column, row = lane: the layout of an A
+//                  operand read from tensor memory.  The split is integer arithmetic: the conversion instruction
+//                  shares the transcendental unit with ex2.
+//   O_g += P_g V   tcgen05.mma with A = P_g from tensor memory, N = d = 128, K = 64 keys (4 steps, both P terms),
 //                  accumulating in tensor memory over the tiles; V is used as it lies in the cache ([key][d], i.e.
 //                  MN-major for this product: 8-key groups 1024 bytes apart, the two 64-column halves 8 KB apart)
 //   rescale        P is formed relative to a reference maximum that is only raised when a row's maximum has
 //                  grown by more than 2^8 (or is seen for the first time): then the warp waits for the previous
 //                  P V product, multiplies its O rows in tensor memory (tcgen05.ld / st) and its row sums by
-//                  2^(m_ref_old - m_ref_new).  Between such events P (<= 2^8) and O need no correction, so the
-//                  softmax of tile j + 1 overlaps with the P V product of tile j (P is double buffered).
-// Tensor memory (512 columns): S 0..127, O 128..255, P 256..383.
-// Warps 0-7: softmax / rescale / epilogue (two groups of four: each row's 64 keys of a tile and its 128 output
-// columns are split between two threads); warp 8 lane 0: TMA; warp 9: tensor memory owner and MMA issue.  The whole
-// of warp 9 runs the issue loop and one elected lane issues each instruction: with the loop inside an
-// `if (lane == 0)` the operand descriptors were per-thread values that had to be moved to uniform registers for every
-// instruction, and the issue itself (70-90 cycles per MMA of 32-64 cycles) bounded the kernel.
+//                  2^(m_ref_old - m_ref_new).  Between such events P (<= 2^8) and O need no correction.
+// Tensor memory (512 columns): S_g at 64 g, P_g at 128 + 64 g, O_g at 256 + 128 g.  The two Q tiles are independent
+// but for the K/V tiles they share: while the threads of one are in their exponentials, the other's loads, maxima
+// and barrier round trips and both tiles' products run.  (One Q tile per CTA, with its rows' keys or its tiles dealt
+// to two warp groups, needs an exchange of maxima per tile and was no faster than one thread per row.)
+// Warps 0-3 / 4-7: softmax, rescale, epilogue of Q tile 0 / 1; warp 8 lane 0: TMA; warp 9: tensor memory owner and
+// MMA issue.  The whole of warp 9 runs the issue loop and one elected lane issues each instruction: with the loop
+// inside an `if (lane == 0)` the operand descriptors were per-thread values that had to be moved to uniform registers
+// for every instruction, and the issue itself (70-90 cycles per MMA of 32-64 cycles) bounded the kernel.
 // Every wait is bounded (ST_TIMEOUT).
 #include <cuda.h>
 
@@ -34,24 +37,25 @@ constexpr float NEG_INF = -__builtin_huge_valf();
 constexpr int DH = 128;
 constexpr int KT = 64;                      // keys per tile
 constexpr int ROWS = 128;
-constexpr int STAGES = 5;
+constexpr int STAGES = 4;
 constexpr int HALF_BYTES = KT * 128;        // one 64-column half of a K or V tile: 64 rows x 128 bytes
 constexpr int KV_TILE = 2 * HALF_BYTES;     // 16 KB
 constexpr int STAGE_BYTES = 2 * KV_TILE;    // K + V
-constexpr int Q_BYTES = ROWS * DH * 2;      // 32 KB: two halves of 128 rows x 128 bytes
+constexpr int Q_BYTES = ROWS * DH * 2;      // 32 KB per Q tile: two halves of 128 rows x 128 bytes
+constexpr int QTILES = 2;                   // Q tiles (row groups of 128) per CTA
 constexpr int THREADS = 320;                // warps 0-7: softmax (two groups of four), 8: TMA, 9: tensor memory / MMA
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
-constexpr int TMEM_COLS = 512;              // S: 2 x 64, O: 128, P: 2 buffers x 2 terms x 32 (bf16 pairs); a power of two
-constexpr int P_COL = 256;                  // first column of P; buffer b, term t at P_COL + 64 b + 32 t
+constexpr int TMEM_COLS = 512;              // per Q tile g: S 64, P 2 terms x 32 (bf16 pairs), O 128
+constexpr int S_COL = 0;                    // S of tile g at S_COL + 64 g
+constexpr int P_COL = 128;                  // P of tile g, term t at P_COL + 64 g + 32 t
+constexpr int O_COL = 256;                  // O of tile g at O_COL + 128 g
 
 struct Shared {
   unsigned long long full[STAGES], empty[STAGES], sfull[2], sempty[2], pfull[2], pvdone[2];
-  unsigned long long xch[2][4];   // row statistics of the two softmax groups exchanged: [tile parity][lane quarter]
-  float stat[2][2][ROWS];         // [tile parity][group][row]
   uint32_t tmem;
   int abort;
 };
-constexpr int SMEM_BYTES = Q_BYTES + STAGES * STAGE_BYTES + (int)sizeof(Shared) + 1024;
+constexpr int SMEM_BYTES = QTILES * Q_BYTES + STAGES * STAGE_BYTES + (int)sizeof(Shared) + 1024;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -168,26 +172,29 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
-// grid = (ceil(C / QB), Hkv, n_seq) with QB = 128 / Gq queries per CTA; block = 320.
+// grid = (Hkv, ceil(C / (2 QB)), n_seq) with QB = 128 / Gq queries per Q tile; block = 320.  Blocks are dispatched in
+// the order of their linear index (x fastest), so the query block is the slower dimension and counts down: block y
+// handles the queries from (gridDim.y - 1 - y) * 2 QB, and the blocks with the most keys (the latest queries) of all
+// heads start first.  With the shortest first, the last long blocks ran alone at the end (215 us against 186 us).
 template <typename OutT>
 __global__ void __launch_bounds__(THREADS, 1)
 k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, ImDims p, ImState st,
                      ImScratch sc, ImCall call, const bf16* __restrict__ q, OutT* __restrict__ out) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* s_q = smem;                       // [2 halves][128 rows][128 bytes]
-  uint8_t* s_kv = smem + Q_BYTES;            // [STAGES][K: 2 halves x 64 rows x 128 bytes | V: the same]
+  uint8_t* s_q = smem;                       // [2 Q tiles][2 halves][128 rows][128 bytes]
+  uint8_t* s_kv = smem + QTILES * Q_BYTES;   // [STAGES][K: 2 halves x 64 rows x 128 bytes | V: the same]
   Shared* sh = reinterpret_cast<Shared*>(s_kv + STAGES * STAGE_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int h = blockIdx.y, i = blockIdx.z;
+  const int h = blockIdx.x, i = blockIdx.z;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int n0 = st.ctr[u * CTR_STRIDE + CTR_N];  // entries cached before the chunk (the counters advance later)
   const int C = call.C;
   if (n0 < 0 || n0 + C > p.cap) return;  // flagged by the append kernel
   const int QB = ROWS / p.Gq;
-  const int s0 = blockIdx.x * QB;
+  const int s0 = (int)(gridDim.y - 1 - blockIdx.y) * QTILES * QB;
   if (s0 >= C) return;
-  const int s_last = min(C, s0 + QB) - 1;
+  const int s_last = min(C, s0 + QTILES * QB) - 1;
   const int n_keys = n0 + s_last + 1;  // slots the block's last query sees
   const int nt = (n_keys + KT - 1) / KT;
   volatile int* abort_flag = &sh->abort;
@@ -196,14 +203,11 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
       mbar_init(smem_u32(&sh->full[s]), 1);
       mbar_init(smem_u32(&sh->empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&sh->sfull[b]), 1);
-      mbar_init(smem_u32(&sh->sempty[b]), 2 * ROWS);
-    }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&sh->pfull[b]), 2 * ROWS);
-      mbar_init(smem_u32(&sh->pvdone[b]), 1);
-      for (int qd = 0; qd < 4; ++qd) mbar_init(smem_u32(&sh->xch[b][qd]), 64);
+    for (int g = 0; g < QTILES; ++g) {
+      mbar_init(smem_u32(&sh->sfull[g]), 1);
+      mbar_init(smem_u32(&sh->sempty[g]), ROWS);
+      mbar_init(smem_u32(&sh->pfull[g]), ROWS);
+      mbar_init(smem_u32(&sh->pvdone[g]), 1);
     }
     sh->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -217,24 +221,24 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
-  // ---- Q tile: thread r writes row r (query s0 + r / Gq, head r % Gq) into the swizzled K-major layout
+  // ---- Q tiles: softmax thread (g, r) writes row r of tile g (query s0 + (128 g + r) / Gq, head (128 g + r) % Gq) into
+  // the swizzled K-major layout
   int lim = 0;          // this row sees slots [0, lim)
   bool row_ok = false;
   int s_row = s0, hh = 0;
-  const int row = tid & (ROWS - 1);  // softmax threads: the row (both groups), TMEM lane
-  if (tid < 2 * ROWS) {
-    const int sl = row / p.Gq;
-    hh = row % p.Gq;
+  const int grp = warp >> 2;         // softmax warps: the Q tile
+  const int row = tid & (ROWS - 1);  // softmax threads: the row within the tile = TMEM lane
+  if (tid < QTILES * ROWS) {
+    const int sl = tid / p.Gq;
+    hh = tid % p.Gq;
     s_row = s0 + sl;
-    row_ok = sl < QB && s_row < C;
+    row_ok = sl < QTILES * QB && s_row < C;
     lim = row_ok ? n0 + s_row + 1 : 0;
-  }
-  if (tid < ROWS) {
     const uint4* src = reinterpret_cast<const uint4*>(q + (((size_t)i * C + (row_ok ? s_row : s0)) * p.H + (size_t)h * p.Gq + (row_ok ? hh : 0)) * DH);
 #pragma unroll
     for (int c = 0; c < 16; ++c) {
       const uint4 v = row_ok ? src[c] : make_uint4(0u, 0u, 0u, 0u);
-      uint8_t* dst = s_q + (c >> 3) * (ROWS * 128) + (tid >> 3) * 1024 + (tid & 7) * 128 + (((c & 7) ^ (tid & 7)) << 4);
+      uint8_t* dst = s_q + grp * Q_BYTES + (c >> 3) * (ROWS * 128) + (row >> 3) * 1024 + (row & 7) * 128 + (((c & 7) ^ (row & 7)) << 4);
       *reinterpret_cast<uint4*>(dst) = v;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -242,7 +246,6 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = sh->tmem;
-  const uint32_t t_o = tmem + 128;  // O columns; S buffers at columns 0 and 64
   bool ok = true;
 
   if (warp == 8) {
@@ -264,133 +267,140 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
       }
     }
   } else if (warp == 9) {
-    {  // ---- MMA issue: the whole warp runs the loop (descriptors stay warp-uniform), one elected lane issues
+    {  // ---- MMA issue: the whole warp runs the loop (descriptors stay warp-uniform), one elected lane issues.
+      // Order in the tensor pipe: S_0(0) S_1(0) | S_0(1) PV_0(0) S_1(1) PV_1(0) | S_0(2) PV_0(1) ...: the score tile
+      // j + 1 of a Q tile is issued as soon as its softmax threads have read tile j, ahead of the P V product of tile j
+      // (which waits for their P), so that they find it when they come back.
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
       const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(DH >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
       const uint32_t qa = smem_u32(s_q);
-      auto issue_s = [&](int j) -> bool {  // S(j) = Q K_j^T into S buffer j & 1
-        const int s = j % STAGES, b = j & 1;
-        if (!mbar_wait(smem_u32(&sh->full[s]), (uint32_t)((j / STAGES) & 1), abort_flag)) return false;
-        if (j >= 2 && !mbar_wait(smem_u32(&sh->sempty[b]), (uint32_t)(((j >> 1) - 1) & 1), abort_flag)) return false;
+      auto issue_s = [&](int j, int g) -> bool {  // S_g(j) = Q_g K_j^T
+        const int s = j % STAGES;
+        if (g == 0 && !mbar_wait(smem_u32(&sh->full[s]), (uint32_t)((j / STAGES) & 1), abort_flag)) return false;
+        if (j >= 1 && !mbar_wait(smem_u32(&sh->sempty[g]), (uint32_t)((j - 1) & 1), abort_flag)) return false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t ka = smem_u32(s_kv + (size_t)s * STAGE_BYTES);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks)
-          mma_bf16(tmem + (uint32_t)(b * KT), desc_sw128(qa + (ks >> 2) * (ROWS * 128) + (ks & 3) * 32, 16, 1024),
+          mma_bf16(tmem + (uint32_t)(S_COL + g * KT), desc_sw128(qa + g * Q_BYTES + (ks >> 2) * (ROWS * 128) + (ks & 3) * 32, 16, 1024),
                    desc_sw128(ka + (ks >> 2) * HALF_BYTES + (ks & 3) * 32, 16, 1024), idesc_s, ks ? 1u : 0u);
-        mma_commit(smem_u32(&sh->sfull[b]));
+        mma_commit(smem_u32(&sh->sfull[g]));
         return true;
       };
-      ok = issue_s(0);
+      ok = issue_s(0, 0) && issue_s(0, 1);
       for (int j = 0; j < nt && ok; ++j) {
-        if (j + 1 < nt && !issue_s(j + 1)) { ok = false; break; }
-        const int s = j % STAGES, b = j & 1;
-        if (!mbar_wait(smem_u32(&sh->pfull[b]), (uint32_t)((j >> 1) & 1), abort_flag)) { ok = false; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int s = j % STAGES;
         const uint32_t va = smem_u32(s_kv + (size_t)s * STAGE_BYTES) + KV_TILE;
+        for (int g = 0; g < QTILES && ok; ++g) {
+          if (j + 1 < nt && !issue_s(j + 1, g)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&sh->pfull[g]), (uint32_t)(j & 1), abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-        for (int term = 0; term < 2; ++term)
+          for (int term = 0; term < 2; ++term)
 #pragma unroll
-          for (int ks = 0; ks < KT / 16; ++ks)
-            mma_bf16_ts(t_o, tmem + (uint32_t)(P_COL + 64 * b + 32 * term + 8 * ks), desc_sw128(va + ks * 2048, HALF_BYTES, 1024),
-                        idesc_o, (j | term | ks) ? 1u : 0u);
-        mma_commit(smem_u32(&sh->pvdone[b]));
-        mma_commit(smem_u32(&sh->empty[s]));
+            for (int ks = 0; ks < KT / 16; ++ks)
+              mma_bf16_ts(tmem + (uint32_t)(O_COL + g * DH), tmem + (uint32_t)(P_COL + 64 * g + 32 * term + 8 * ks),
+                          desc_sw128(va + ks * 2048, HALF_BYTES, 1024), idesc_o, (j | term | ks) ? 1u : 0u);
+          mma_commit(smem_u32(&sh->pvdone[g]));
+        }
+        if (ok) mma_commit(smem_u32(&sh->empty[s]));
       }
     }
   } else {
-    // ---- softmax, rescale, epilogue.  Two groups of four warps: thread (group g, row r) owns keys 32 g .. 32 g + 31
-    // of every tile of row r = TMEM lane r (warps w and w + 4 may both read lane quarter w) and, for the rescale and
-    // the epilogue, columns 64 g .. 64 g + 63 of O.  The two threads of a row exchange their maxima (and at the end
-    // their sums) through shared memory and an mbarrier per lane quarter, and take every decision alike.
-    const int grp = warp >> 2, qd = warp & 3;
+    // ---- softmax, rescale, epilogue: warps 4 g .. 4 g + 3 own Q tile g, thread = row = TMEM lane (warp w reads lane
+    // quarter w % 4).  The two groups share nothing but the K/V tiles, so one group's loads, maxima and waits overlap
+    // with the other's exponentials and with the tensor pipe.
+    const int g = grp, qd = warp & 3;
     const uint32_t lane_addr = (uint32_t)(qd * 32) << 16;
+    const uint32_t t_s = tmem + lane_addr + (uint32_t)(S_COL + g * KT);
+    const uint32_t t_p = tmem + lane_addr + (uint32_t)(P_COL + 64 * g);
+    const uint32_t t_o = tmem + lane_addr + (uint32_t)(O_COL + g * DH);
     const float sl2 = p.scale * 1.4426950408889634f;  // softmax in base 2
-    float m_ref = NEG_INF, l = 0.f;                    // reference maximum of P and O, this thread's share of the row sum
+    float m_ref = NEG_INF, l = 0.f;                    // reference maximum of P and O, row sum
     for (int j = 0; j < nt; ++j) {
-      const int b = j & 1;
-      if (!mbar_wait(smem_u32(&sh->sfull[b]), (uint32_t)((j >> 1) & 1), abort_flag)) { ok = false; break; }
+      if (!mbar_wait(smem_u32(&sh->sfull[g]), (uint32_t)(j & 1), abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      float sv[32];
-      tmem_ld32(tmem + lane_addr + (uint32_t)(b * KT + grp * 32), sv);
+      float sv[KT];
+      tmem_ld32(t_s, sv);
+      tmem_ld32(t_s + 32, sv + 32);
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(smem_u32(&sh->sempty[b]));
-      const int key0 = j * KT + grp * 32;
-      float tm = NEG_INF;
-      if (key0 + 32 > lim) {  // only the row's last tiles need the causal mask
+      mbar_arrive(smem_u32(&sh->sempty[g]));
+      const int key0 = j * KT;
+      if (key0 + KT > lim) {  // only the row's last tiles need the causal mask
 #pragma unroll
-        for (int k = 0; k < 32; ++k) sv[k] = key0 + k < lim ? sv[k] : NEG_INF;
+        for (int k = 0; k < KT; ++k) sv[k] = key0 + k < lim ? sv[k] : NEG_INF;
       }
+      float t0 = sv[0], t1 = sv[1], t2 = sv[2], t3 = sv[3];
 #pragma unroll
-      for (int k = 0; k < 32; ++k) tm = fmaxf(tm, sv[k]);
-      sh->stat[b][grp][row] = tm;
-      mbar_arrive(smem_u32(&sh->xch[b][qd]));
-      if (!mbar_wait(smem_u32(&sh->xch[b][qd]), (uint32_t)((j >> 1) & 1), abort_flag)) { ok = false; break; }
-      tm = fmaxf(tm, sh->stat[b][grp ^ 1][row]);
-      tm *= sl2;  // the scale is positive: the maximum of the scaled scores
+      for (int k = 4; k < KT; k += 4) {
+        t0 = fmaxf(t0, sv[k]);
+        t1 = fmaxf(t1, sv[k + 1]);
+        t2 = fmaxf(t2, sv[k + 2]);
+        t3 = fmaxf(t3, sv[k + 3]);
+      }
+      const float tm = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3)) * sl2;  // the scale is positive: the maximum of the scaled scores
       // raise the reference only for a first maximum or a jump of more than 8 (P stays below 2^8 otherwise)
       const bool raise = tm > NEG_INF && (m_ref == NEG_INF || tm > m_ref + 8.0f);
+      bool pv_waited = false;
       if (__any_sync(0xffffffffu, raise)) {
         const float corr = raise ? exp2f(m_ref - tm) : 1.0f;  // 0 for a first maximum: nothing accumulated yet
         if (raise) {
           m_ref = tm;
           l *= corr;
         }
-        if (j >= 1) {  // O holds the products up to tile j - 1: wait for the last one, then scale this thread's half row
-          if (!mbar_wait(smem_u32(&sh->pvdone[(j - 1) & 1]), (uint32_t)(((j - 1) >> 1) & 1), abort_flag)) { ok = false; break; }
+        if (j >= 1) {  // O holds the products up to tile j - 1: wait for the last one, then scale the row
+          if (!mbar_wait(smem_u32(&sh->pvdone[g]), (uint32_t)((j - 1) & 1), abort_flag)) { ok = false; break; }
+          pv_waited = true;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-          for (int c0 = 0; c0 < DH / 2; c0 += 32) {
+          for (int c0 = 0; c0 < DH; c0 += 32) {
             float t[32];
-            tmem_ld32(t_o + lane_addr + (uint32_t)(grp * (DH / 2) + c0), t);
+            tmem_ld32(t_o + (uint32_t)c0, t);
 #pragma unroll
             for (int c = 0; c < 32; ++c) t[c] *= corr;
-            tmem_st32(t_o + lane_addr + (uint32_t)(grp * (DH / 2) + c0), t);
+            tmem_st32(t_o + (uint32_t)c0, t);
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         }
       }
-      // P buffer b was last read by the product of tile j - 2
-      if (j >= 2 && !mbar_wait(smem_u32(&sh->pvdone[b]), (uint32_t)(((j >> 1) - 1) & 1), abort_flag)) { ok = false; break; }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const float e = m_ref == NEG_INF ? 0.f : m_ref;
-      uint32_t hi[16], lo[16];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const float p0 = ex2(fmaf(sv[2 * k], sl2, -e)), p1 = ex2(fmaf(sv[2 * k + 1], sl2, -e));
-        l += p0 + p1;
-        // bf16 split on the integer pipe: first term = the upper 16 bits, second = the remainder rounded half up
-        const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
-        hi[k] = __byte_perm(b0, b1, 0x7632);
-        const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
-        lo[k] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t hi[16], lo[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const float p0 = ex2(fmaf(sv[32 * hf + 2 * k], sl2, -e)), p1 = ex2(fmaf(sv[32 * hf + 2 * k + 1], sl2, -e));
+          l += p0 + p1;
+          // bf16 split on the integer pipe (the conversion instruction shares the transcendental unit with ex2):
+          // first term = the upper 16 bits, second = the remainder rounded half up
+          const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+          hi[k] = __byte_perm(b0, b1, 0x7632);
+          const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+          lo[k] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);
+        }
+        if (hf == 0 && j >= 1 && !pv_waited) {  // P is single buffered: the product of tile j - 1 has to be through with it
+          if (!mbar_wait(smem_u32(&sh->pvdone[g]), (uint32_t)((j - 1) & 1), abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        }
+        tmem_st16(t_p + (uint32_t)(16 * hf), hi);
+        tmem_st16(t_p + (uint32_t)(32 + 16 * hf), lo);
       }
-      const uint32_t t_p = tmem + lane_addr + (uint32_t)(P_COL + 64 * b + 16 * grp);
-      tmem_st16(t_p, hi);
-      tmem_st16(t_p + 32, lo);
+      if (!ok) break;
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(smem_u32(&sh->pfull[b]));
+      mbar_arrive(smem_u32(&sh->pfull[g]));
     }
-    // ---- epilogue: O / l + gated readout; the row sum is the two threads' shares added
-    if (ok) {
-      const int b = nt & 1;  // the exchange barrier of the parity after the last tile: used (nt - b + 1) / 2 times so far
-      sh->stat[b][grp][row] = l;
-      mbar_arrive(smem_u32(&sh->xch[b][qd]));
-      if (!mbar_wait(smem_u32(&sh->xch[b][qd]), (uint32_t)((nt >> 1) & 1), abort_flag)) ok = false;
-      l += sh->stat[b][grp ^ 1][row];
-    }
-    if (ok && !mbar_wait(smem_u32(&sh->pvdone[(nt - 1) & 1]), (uint32_t)(((nt - 1) >> 1) & 1), abort_flag)) ok = false;
+    // ---- epilogue: O / l + gated readout
+    if (ok && !mbar_wait(smem_u32(&sh->pvdone[g]), (uint32_t)((nt - 1) & 1), abort_flag)) ok = false;
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const float inv = l > 0.f ? 1.0f / l : 0.f;
       const float* mr = sc.mch + ((size_t)i * C + (row_ok ? s_row : 0)) * p.Dkv + h * DH;
       OutT* op = out + (((size_t)i * C + (row_ok ? s_row : 0)) * p.H + (size_t)h * p.Gq + hh) * DH;
 #pragma unroll
-      for (int c1 = 0; c1 < DH / 2; c1 += 32) {
-        const int c0 = grp * (DH / 2) + c1;
+      for (int c0 = 0; c0 < DH; c0 += 32) {
         float t[32];
-        tmem_ld32(t_o + lane_addr + (uint32_t)c0, t);  // (warp-collective: rows out of range load too, and skip the store)
+        tmem_ld32(t_o + (uint32_t)c0, t);  // (warp-collective: rows out of range load too, and skip the store)
         if (row_ok) {
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
@@ -437,7 +447,7 @@ cudaError_t im_launch_chunk_attention_tc(const ImLaunch& L, const ImCall& call, 
                                          const void* q, void* out) {
   const ImDims& p = L.p;
   const int QB = ROWS / p.Gq;
-  dim3 grid((call.C + QB - 1) / QB, p.Hkv, call.n_seq);
+  dim3 grid(p.Hkv, (call.C + QTILES * QB - 1) / (QTILES * QB), call.n_seq);
   const CUtensorMap& mk = *(const CUtensorMap*)mapK;
   const CUtensorMap& mv = *(const CUtensorMap*)mapV;
   if (p.out_f32) k_chunk_attention_tc<float><<<grid, THREADS, SMEM_BYTES, L.stream>>>(mk, mv, p, L.st, L.sc, call, (const bf16*)q, (float*)out);
