@@ -393,6 +393,32 @@ def test_chunk_outputs_tiny_shape_no_memory_and_single_token_chunks(im):
     assert p1.stats["max_out_err"] <= 2e-3
 
 
+def test_chunk_outputs_head_dim_128_other_group_sizes_and_short_chunks(im):
+    """The tcgen05 chunk attention lays 2 x 128 rows = queries x heads of a KV head over two Q tiles: 8 heads per KV
+    head (16 queries per tile), 1 head per KV head (128 queries per tile, so a chunk of 100 leaves the second Q tile
+    without a valid row), and chunks of 1 and 3 tokens (one block, one key tile at first, the retained prefix
+    growing past a tile), all at head_dim 128."""
+    base = synth.CONFIGS["llama8b_b1"]
+    wl8 = base.replace(name="chunk_out_g8", H=8, Hkv=1, n_seq=2, ctx=3 * 90, chunk=90, B=120, steps=2, n_needles=0)
+    p8 = _pair(wl8, chunk_outputs=1)
+    for c in range(3):
+        p8.prefill_attend(c)
+    for s in range(wl8.steps):
+        p8.decode(s)
+    assert p8.stats["max_out_err"] <= 2e-3 and p8.stats["max_M_err"] <= 2e-3
+    wl1 = base.replace(name="chunk_out_g1", H=4, Hkv=4, n_seq=1, ctx=3 * 100, chunk=100, B=130, steps=2, n_needles=0)
+    p1 = _pair(wl1, chunk_outputs=1, out_f32=1)
+    for c in range(3):
+        p1.prefill_attend(c)
+    assert p1.stats["max_out_err"] <= 1e-4
+    for chunk, n in ((1, 70), (3, 30)):
+        wls = base.replace(name=f"chunk_out_c{chunk}", H=8, Hkv=2, n_seq=1, ctx=chunk * n, chunk=chunk, B=48, steps=1, n_needles=0)
+        ps = _pair(wls, chunk_outputs=1)
+        for c in range(n):
+            ps.prefill_attend(c)
+        assert ps.stats["max_out_err"] <= 2e-3 and ps.stats["max_M_err"] <= 2e-3
+
+
 def test_chunk_outputs_need_their_workspace(im):
     wl = TINY.replace(name="chunk_out_e", ctx=32, chunk=32, B=64, steps=1)
     p = _pair(wl)
