@@ -282,7 +282,9 @@ __global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __
 // consecutive k of row r (vector r for A, weight row r of the n-tile for B) starting at 8 q inside a 32-wide
 // chunk; k-step s multiplies element s of every lane's vector: the contraction index is permuted identically for
 // both operands.  Every product and sum is formed in float64.
-// grid = ceil(NV / 8), block = 128; D a multiple of 128, d_I = 8 NT.
+// grid = (ceil(NV / 8), ksplit), block = 128; D a multiple of 128 ksplit, d_I = 8 NT.  Block (., ks) takes the ks-th
+// part of the K range and writes the partial sums keyp[ks][v][.] (decode: the few vectors of a step would leave all
+// but a handful of SMs idle, and the consumer adds the parts in split order).
 __device__ __forceinline__ void dmma_884(double (&c)[2], double a, double b) {
   asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
                : "+d"(c[0]), "+d"(c[1]) : "d"(a), "d"(b));
@@ -293,11 +295,12 @@ __device__ __forceinline__ double bf16_elem(const uint4& v, int s) {
 }
 template <int NT>
 __global__ void __launch_bounds__(128) k_proj_key_mma(ImDims p, const bf16* __restrict__ Uk, const bf16* __restrict__ x,
-                                                       int NV, double* __restrict__ keyp) {
+                                                       int NV, int ksplit, double* __restrict__ keyp) {
   __shared__ double red[4][NT][64];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, q = lane & 3;
   const long long v0 = (long long)blockIdx.x * 8;
-  const int kspan = p.D / 4, kbeg = warp * kspan;  // a multiple of 32 (checked by the launcher)
+  const int kspan = p.D / (4 * ksplit), kbeg = ((int)blockIdx.y * 4 + warp) * kspan;  // a multiple of 32 (checked by the launcher)
+  keyp += (size_t)blockIdx.y * NV * p.dI;
   const bf16* xrow = x + (size_t)min(v0 + r, (long long)NV - 1) * p.D + kbeg + 8 * q;
   const bf16* urow = Uk + (size_t)r * p.D + kbeg + 8 * q;
   double c[NT][2];
@@ -366,9 +369,11 @@ cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
 }
 
 cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, int ksplit) {
-  if (ksplit == 1 && NV >= 64 && L.p.D % 128 == 0 && (L.p.dI == 8 || L.p.dI == 16)) {  // prefill chunks
-    if (L.p.dI == 8) k_proj_key_mma<1><<<(NV + 7) / 8, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, L.sc.keyp);
-    else k_proj_key_mma<2><<<(NV + 7) / 8, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, L.sc.keyp);
+  // float64 tensor-core path: prefill chunks whole, decode steps with the K range cut over `ksplit` blocks
+  if ((ksplit > 1 || NV >= 64) && L.p.D % (128 * ksplit) == 0 && (L.p.dI == 8 || L.p.dI == 16)) {
+    dim3 grid((NV + 7) / 8, ksplit);
+    if (L.p.dI == 8) k_proj_key_mma<1><<<grid, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
+    else k_proj_key_mma<2><<<grid, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
     ++*L.launches;
     return cudaGetLastError();
   }
@@ -385,5 +390,7 @@ cudaError_t im_gemm_prepare_decode() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_direct_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_SIDE);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_skinny_gemm);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_split);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_mma<1>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_mma<2>);
   return e;
 }
