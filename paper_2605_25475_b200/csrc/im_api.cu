@@ -285,7 +285,9 @@ cudaError_t launch_mem_update(im_ctx* ctx, const ImLaunch& L, const ImCall& call
 
 // phi of the gathered evicted keys (skinny GEMM against the folded Linear_theta), then Eq. 6-7.
 // With `update` = false only the GEMM is launched (the caller launches im_launch_mem_update later).
-int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, bool update = true, int smem_floor = 0) {
+// `before_update`: an event that the kernels changing the memory state wait for (a reader of the state of before)
+int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, bool update = true, int smem_floor = 0,
+                     cudaEvent_t before_update = nullptr) {
   const ImDims& p = ctx->p;
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
@@ -324,6 +326,7 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
     g.smem_floor = smem_floor;
   }
   CKL(im_launch_gemm(L, g));
+  if (update && before_update) CK(cudaStreamWaitEvent(L.stream, before_update, 0));
   if (update) CKL(launch_mem_update(ctx, L, call, ne_max));
   return IM_OK;
 }
@@ -570,19 +573,29 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   }
   CKL(im_launch_prefill_append(L, call, k, v));
   if (attend) {
-    // layer outputs of the chunk's own queries, before the chunk is compressed: Eq. 5 over the memory of before
-    // this chunk, then attention over (cached entries + causal chunk) with the readout added (Eq. 4)
+    // Layer outputs of the chunk's own queries, before the chunk is compressed: Eq. 5 over the memory of before
+    // this chunk, then attention over (cached entries + causal chunk) with the readout added (Eq. 4).  They read the
+    // cache and the memory as the append kernel left them (the entry count of before the chunk from CTR_NNEXT, which
+    // that kernel sets), so with IM_OPT_CONCURRENCY they run on a side stream NEXT TO the scoring, the selection,
+    // the gather and the GEMMs of the memory write; only the kernels that overwrite what they read wait for them:
+    // the filling of the holes for the attention kernel (ev[9]), the memory update for the readout (ev[8]).
+    ImLaunch La = L;
+    if (fork) {
+      La.stream = ctx->side[2];  // (the phi(q) projection runs there when there is a memory)
+      CK(cudaEventRecord(ctx->ev[7], L.stream));
+      CK(cudaStreamWaitEvent(La.stream, ctx->ev[7], 0));
+    }
     if (memside) {
       if (fork) {
-        CK(cudaEventRecord(ctx->ev[3], Lt.stream));
         CK(cudaEventRecord(ctx->ev[4], Lw.stream));
-        CK(cudaStreamWaitEvent(L.stream, ctx->ev[3], 0));
-        CK(cudaStreamWaitEvent(L.stream, ctx->ev[4], 0));
+        CK(cudaStreamWaitEvent(La.stream, ctx->ev[4], 0));
       }
-      CKL(im_launch_chunk_readout(L, call));
+      CKL(im_launch_chunk_readout(La, call));
+      if (fork) CK(cudaEventRecord(ctx->ev[8], La.stream));
     }
-    if (ctx->attend_tc && im_chunk_attn_tc_supported(p)) CKL(im_launch_chunk_attention_tc(L, call, ctx->mapK, ctx->mapV, q, out));
-    else CKL(im_launch_chunk_attention(L, call, ctx->mapK, ctx->mapV, q, out));
+    if (ctx->attend_tc && im_chunk_attn_tc_supported(p)) CKL(im_launch_chunk_attention_tc(La, call, ctx->mapK, ctx->mapV, q, out));
+    else CKL(im_launch_chunk_attention(La, call, ctx->mapK, ctx->mapV, q, out));
+    if (fork) CK(cudaEventRecord(ctx->ev[9], La.stream));
   }
   // a1: pooled importance under the causal mask
   {
@@ -606,16 +619,19 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
       CKL(im_launch_gather(L, call, ne_max));
       CK(cudaEventRecord(ctx->ev[5], L.stream));
       CK(cudaStreamWaitEvent(Lm.stream, ctx->ev[5], 0));
+      if (attend) CK(cudaStreamWaitEvent(Lm.stream, ctx->ev[9], 0));  // the chunk attention reads the slots that are filled
       CKL(im_launch_move(Lm, call, ne_max));
       CK(cudaEventRecord(ctx->ev[6], Lm.stream));
-      if ((rc = run_memory_write(ctx, L, call, ne_max))) return rc;  // a3
+      if ((rc = run_memory_write(ctx, L, call, ne_max, true, 0, memside ? ctx->ev[8] : nullptr))) return rc;  // a3
       CK(cudaStreamWaitEvent(L.stream, ctx->ev[6], 0));
     } else {
+      if (attend && fork) CK(cudaStreamWaitEvent(L.stream, ctx->ev[9], 0));  // the chunk attention reads the cache
       CKL(im_launch_gather_move(L, call, ne_max));
       // a3: memory write
       if (p.mem && (rc = run_memory_write(ctx, L, call, ne_max))) return rc;
     }
   }
+  if (attend && fork) CK(cudaStreamWaitEvent(L.stream, ctx->ev[9], 0));  // join (also when nothing was evicted)
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
     const int ne = std::max(0, u.n + chunk_len - p.B);

@@ -203,7 +203,7 @@ k_chunk_attention(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   const int g = lane >> 2, t = lane & 3;
   const int h = blockIdx.y, i = blockIdx.z;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
-  const int n0 = st.ctr[u * CTR_STRIDE + CTR_N];  // entries cached before the chunk (the counters advance later)
+  const int n0 = st.ctr[u * CTR_STRIDE + CTR_NNEXT];  // entries cached before the chunk (set by the append kernel; CTR_N advances meanwhile)
   const int C = call.C;
   if (n0 < 0 || n0 + C > p.cap) return;  // flagged by the append kernel
   const int QB = CA_ROWS / p.Gq;

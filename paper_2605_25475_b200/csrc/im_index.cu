@@ -35,7 +35,7 @@ __device__ __forceinline__ float index_score(const ImDims& p, const float* __res
 }
 
 // prefill: finalise the features of every chunk token, append K/V/kidx/pos.
-// grid = (C, n_seq), block = 128.  The counters are advanced by k_prefill_commit.
+// grid = (C, n_seq), block = 128.  The counters are advanced by k_prefill_commit (CTR_NNEXT keeps the old count).
 __global__ void k_prefill_append(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __restrict__ K,
                                  const bf16* __restrict__ V) {
   const int c = blockIdx.x, i = blockIdx.y;
@@ -47,6 +47,8 @@ __global__ void k_prefill_append(ImDims p, ImState st, ImScratch sc, ImCall call
     if (tid == 0 && c == 0) atomicOr(st.status, ST_COUNT);
     return;
   }
+  // the entry count of before the chunk, for the kernels that form the chunk's layer outputs while the counters advance
+  if (tid == 0 && c == 0) st.ctr[u * CTR_STRIDE + CTR_NNEXT] = n;
   const ImRows r = im_rows(p);
   float* raw = sc.raw + ((size_t)i * call.C + c) * p.R3;
   if (tid < 32) finalize_features(p, raw, tid);
