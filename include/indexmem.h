@@ -225,7 +225,9 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        launched as a programmatic dependent: it may request tiles of its own layer's cache
  *                        while that call's last kernel is still running, and waits for it before it reads `q`.
  *                        The prefill calls run the chunk's independent projections next to one another on the
- *                        same side streams.  0: everything is enqueued on `cuda_stream` in order.
+ *                        same side streams, and im_prefill_chunk_attend forms the layer outputs (readout and
+ *                        attention of the chunk's queries) next to the scoring, the selection and the memory
+ *                        write of the chunk.  0: everything is enqueued on `cuda_stream` in order.
  *   IM_OPT_PREFETCH_NEXT 1 (default): while the attention kernel of layer l streams the K/V cache,
  *                        im_decode_step prefetches into L2 what the small latency-bound kernels of layer
  *                        (l + 1) mod n_layers will read for the same sequences (weights, indexer key cache,
