@@ -277,12 +277,13 @@ __global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __
 }
 
 // The same projection for the thousands of vectors of a prefill chunk, on the float64 tensor-core path
-// (mma.sync m8n8k4 f64): a warp takes 8 vectors x all d_I rows over a quarter of the K range, the four warps of a
-// block add their 8 x 8 tiles through shared memory in warp order.  Lane (r, q) = (lane / 4, lane % 4) loads 8
+// (mma.sync m8n8k4 f64): a warp takes 8 vectors x all d_I rows over 1 / W of the K range, the W warps of a
+// block add their 8 x 8 tiles through shared memory in warp order (W = 8 for prefill chunks: the kernel is bound by
+// the latency of its load -> convert -> mma chains, and 256 blocks of 4 warps leave an SM 7 warps to hide it).  Lane (r, q) = (lane / 4, lane % 4) loads 8
 // consecutive k of row r (vector r for A, weight row r of the n-tile for B) starting at 8 q inside a 32-wide
 // chunk; k-step s multiplies element s of every lane's vector: the contraction index is permuted identically for
 // both operands.  Every product and sum is formed in float64.
-// grid = (ceil(NV / 8), ksplit), block = 128; D a multiple of 128 ksplit, d_I = 8 NT.  Block (., ks) takes the ks-th
+// grid = (ceil(NV / 8), ksplit), block = 32 W; D a multiple of 32 W ksplit, d_I = 8 NT.  Block (., ks) takes the ks-th
 // part of the K range and writes the partial sums keyp[ks][v][.] (decode: the few vectors of a step would leave all
 // but a handful of SMs idle, and the consumer adds the parts in split order).
 __device__ __forceinline__ void dmma_884(double (&c)[2], double a, double b) {
@@ -293,13 +294,13 @@ __device__ __forceinline__ double bf16_elem(const uint4& v, int s) {
   const uint32_t w = s < 2 ? v.x : s < 4 ? v.y : s < 6 ? v.z : v.w;
   return (double)((s & 1) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16));
 }
-template <int NT>
-__global__ void __launch_bounds__(128) k_proj_key_mma(ImDims p, const bf16* __restrict__ Uk, const bf16* __restrict__ x,
+template <int NT, int W>
+__global__ void __launch_bounds__(32 * W) k_proj_key_mma(ImDims p, const bf16* __restrict__ Uk, const bf16* __restrict__ x,
                                                        int NV, int ksplit, double* __restrict__ keyp) {
-  __shared__ double red[4][NT][64];
+  __shared__ double red[W][NT][64];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, q = lane & 3;
   const long long v0 = (long long)blockIdx.x * 8;
-  const int kspan = p.D / (4 * ksplit), kbeg = ((int)blockIdx.y * 4 + warp) * kspan;  // a multiple of 32 (checked by the launcher)
+  const int kspan = p.D / (W * ksplit), kbeg = ((int)blockIdx.y * W + warp) * kspan;  // a multiple of 32 (checked by the launcher)
   keyp += (size_t)blockIdx.y * NV * p.dI;
   const bf16* xrow = x + (size_t)min(v0 + r, (long long)NV - 1) * p.D + kbeg + 8 * q;
   const bf16* urow = Uk + (size_t)r * p.D + kbeg + 8 * q;
@@ -325,10 +326,15 @@ __global__ void __launch_bounds__(128) k_proj_key_mma(ImDims p, const bf16* __re
     red[warp][nt][r * 8 + 2 * q + 1] = c[nt][1];
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < NT * 64; idx += 128) {
+  for (int idx = threadIdx.x; idx < NT * 64; idx += 32 * W) {
     const int nt = idx >> 6, e = idx & 63;
     const long long v = v0 + (e >> 3);
-    if (v < NV) keyp[(size_t)v * p.dI + nt * 8 + (e & 7)] = ((red[0][nt][e] + red[1][nt][e]) + red[2][nt][e]) + red[3][nt][e];
+    if (v < NV) {
+      double sum = red[0][nt][e];
+#pragma unroll
+      for (int w = 1; w < W; ++w) sum += red[w][nt][e];
+      keyp[(size_t)v * p.dI + nt * 8 + (e & 7)] = sum;
+    }
   }
 }
 
@@ -372,8 +378,14 @@ cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, i
   // float64 tensor-core path: prefill chunks whole, decode steps with the K range cut over `ksplit` blocks
   if ((ksplit > 1 || NV >= 64) && L.p.D % (128 * ksplit) == 0 && (L.p.dI == 8 || L.p.dI == 16)) {
     dim3 grid((NV + 7) / 8, ksplit);
-    if (L.p.dI == 8) k_proj_key_mma<1><<<grid, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
-    else k_proj_key_mma<2><<<grid, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
+    const bool wide = ksplit == 1 && L.p.D % 256 == 0;  // prefill chunks
+    if (L.p.dI == 8) {
+      if (wide) k_proj_key_mma<1, 8><<<grid, 256, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
+      else k_proj_key_mma<1, 4><<<grid, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
+    } else {
+      if (wide) k_proj_key_mma<2, 8><<<grid, 256, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
+      else k_proj_key_mma<2, 4><<<grid, 128, 0, L.stream>>>(L.p, L.w.Uk, (const bf16*)x, NV, ksplit, L.sc.keyp);
+    }
     ++*L.launches;
     return cudaGetLastError();
   }
@@ -390,7 +402,7 @@ cudaError_t im_gemm_prepare_decode() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_direct_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_SIDE);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_skinny_gemm);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_split);
-  if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_mma<1>);
-  if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_mma<2>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_mma<1, 4>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_mma<2, 4>);
   return e;
 }
