@@ -580,18 +580,19 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
     // the gather and the GEMMs of the memory write; only the kernels that overwrite what they read wait for them:
     // the filling of the holes for the attention kernel (ev[9]), the memory update for the readout (ev[8]).
     ImLaunch La = L;
-    if (fork) {
-      La.stream = ctx->side[2];  // (the phi(q) projection runs there when there is a memory)
-      CK(cudaEventRecord(ctx->ev[7], L.stream));
-      CK(cudaStreamWaitEvent(La.stream, ctx->ev[7], 0));
-    }
+    if (fork) La.stream = ctx->side[2];  // (the phi(q) projection runs there when there is a memory)
     if (memside) {
+      // the readout needs the two memory-side projections only, not the appended chunk
       if (fork) {
         CK(cudaEventRecord(ctx->ev[4], Lw.stream));
         CK(cudaStreamWaitEvent(La.stream, ctx->ev[4], 0));
       }
       CKL(im_launch_chunk_readout(La, call));
       if (fork) CK(cudaEventRecord(ctx->ev[8], La.stream));
+    }
+    if (fork) {
+      CK(cudaEventRecord(ctx->ev[7], L.stream));  // the chunk is appended
+      CK(cudaStreamWaitEvent(La.stream, ctx->ev[7], 0));
     }
     if (ctx->attend_tc && im_chunk_attn_tc_supported(p)) CKL(im_launch_chunk_attention_tc(La, call, ctx->mapK, ctx->mapV, q, out));
     else CKL(im_launch_chunk_attention(La, call, ctx->mapK, ctx->mapV, q, out));
