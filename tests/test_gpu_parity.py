@@ -419,6 +419,32 @@ def test_chunk_outputs_head_dim_128_other_group_sizes_and_short_chunks(im):
         assert ps.stats["max_out_err"] <= 2e-3 and ps.stats["max_M_err"] <= 2e-3
 
 
+def test_chunk_outputs_call_captured_into_a_cuda_graph(im):
+    """im_prefill_chunk_attend forks onto the side streams (projections, the output kernels next to the compression
+    chain) and joins back with events only: the second chunk's call is captured into a CUDA graph, replayed once,
+    and outputs and state are compared with the oracle as for an eager call."""
+    wl = synth.CONFIGS["llama8b_b1"].replace(name="chunk_out_graph", n_seq=2, ctx=2 * 160, chunk=160, B=200, steps=1, n_needles=2)
+    p = _pair(wl, chunk_outputs=1)
+    p.prefill_attend(0)
+    X, Q, K, V = synth.prefill_inputs(wl, p.layer, 1)
+    ob, od = p.o.prefill_batch_out(p.seq_ids, synth.f32(X), synth.f32(Q), synth.f32(Q), synth.f32(K), synth.f32(V))
+    dev = p.device
+    Xd, Qd, Kd, Vd = X.to(dev), Q.to(dev), K.to(dev), V.to(dev)
+    stream = torch.cuda.Stream(dev)
+    with torch.cuda.stream(stream):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            out = p.g.prefill_chunk_attend(0, p.seq_ids, Xd, Qd, Qd, Kd, Vd)
+        graph.replay()
+        stream.synchronize()
+    assert p.g.status() == 0
+    p.check_selection()
+    p.check_state()
+    n, Cn = od.shape[0], od.shape[1]
+    p.check_out(out.reshape(n * Cn, wl.H, wl.d), ob.reshape(n * Cn, wl.H, wl.d), od.reshape(n * Cn, wl.H, wl.d))
+    assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_M_err"] <= 2e-3
+
+
 def test_chunk_outputs_need_their_workspace(im):
     wl = TINY.replace(name="chunk_out_e", ctx=32, chunk=32, B=64, steps=1)
     p = _pair(wl)
