@@ -77,44 +77,64 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // mch[i][s][col] = g(q_s) * cscale * (sum_m phi_s[m] Mhat[m][col]) / (eps + sum_m phi_s[m]^2 b[m])   (Eq. 5,
 // gate of Eq. 4).  The pending list is empty here (the call folds it first).  phi_s and the gate logit are
 // rows [0, dM) and dM of the chunk's memory-side projection, which the call writes behind the indexer-side
-// block of the projection scratch.  A float32 GEMM on the CUDA cores ([C x d_M] x [d_M x D_kv], 2.1 GFLOP per
-// 2048-token chunk): 128 x 128 output tile per block, 8 x 8 micro tile per thread (two 4-wide halves 64 apart in
-// both directions, so that a warp's shared-memory reads are conflict free), K slices of 16 staged through
-// registers into shared memory while the previous slice is multiplied.
-// grid = (ceil(Dkv / 128), ceil(C / 128), n_seq), block = 256.
-constexpr int CR_T = 128, CR_K = 16;
-__global__ void __launch_bounds__(256) k_chunk_readout(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call) {
-  __shared__ __align__(16) float s_a[2][CR_K][CR_T + 4];  // [m][query] (padded: the staging stores of a warp spread over the banks)
-  __shared__ __align__(16) float s_b[2][CR_K][CR_T + 4];  // [m][col]
-  __shared__ float s_bv[2][CR_K];
+// block of the projection scratch.  A float32 product ([C x d_M] x [d_M x D_kv], 2.1 GFLOP per 2048-token chunk) on
+// the tensor cores as three tf32 products: x = hi + lo with hi the upper 19 bits of x (what a tf32 operand keeps)
+// and lo the exact remainder, and phi Mhat ~ hi hi + hi lo + lo hi (the dropped lo lo term and the truncation of lo
+// are 2^-20 of a product).  64 queries x 128 columns per block, 8 warps of 32 queries x 32 columns (2 x 4
+// mma.sync.m16n8k8 tiles each), K slices of 16 staged through registers into shared memory while the previous slice
+// is multiplied; rows padded by 8 floats so that a warp's fragment loads (4 k x 8 rows) touch 32 different banks.
+// The loop is bound by the latency of the next slice's loads, not by the arithmetic (the float32 FMA version of the
+// same loop took the same 78 us): hence the small tile, two or three blocks per SM.  The denominators are summed by
+// the staging threads (each holds 4 queries x 1 m per slice) in float32.
+// grid = (ceil(Dkv / 128), ceil(C / 64), n_seq), block = 256.
+constexpr int CR_T = 128, CR_TQ = 64, CR_K = 16, CR_LD = CR_T + 8, CR_LDQ = CR_TQ + 8;
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+// x = hi + lo, both with the low 13 mantissa bits clear
+__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
+  hi = __float_as_uint(x) & 0xffffe000u;
+  lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
+}
+__global__ void __launch_bounds__(256, 3) k_chunk_readout(ImDims p, ImState st, ImWeights w, ImScratch sc, ImCall call) {
+  __shared__ __align__(16) float s_a[2][CR_K][CR_LDQ];  // [m][query]
+  __shared__ __align__(16) float s_b[2][CR_K][CR_LD];  // [m][col]
+  __shared__ float s_den[CR_TQ];
   const int i = blockIdx.z;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const float* proj = sc.raw + (size_t)p.S * p.max_chunk * p.R3;  // [n_seq * C][dM + 1]
   const int ps = p.dM + 1;
-  const int q0 = blockIdx.y * CR_T, col0 = blockIdx.x * CR_T;
-  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int q0 = blockIdx.y * CR_TQ, col0 = blockIdx.x * CR_T;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int wq = (warp & 1) * 32, wc = (warp >> 1) * 32;  // the warp's 32 queries x 32 columns of the tile
   const float* Mh = st.Mhat + u * p.dM * p.Dkv;
   const float* bv = st.bvec + u * p.dM;
-  // staging roles: A - thread t loads m = t & 15 of queries (t >> 4) + 16 j, j < 8 (16 consecutive floats of a
+  // staging roles: A - thread t loads m = t & 15 of queries (t >> 4) + 16 j, j < 4 (16 consecutive floats of a
   // projection row per 16 threads); B - thread t loads float4 (t & 31) of rows (t >> 5) and (t >> 5) + 8
   const int am = tid & 15, as = tid >> 4;
   const int bc = (tid & 31) * 4, bm = tid >> 5;
   const bool b_vec = (p.Dkv & 3) == 0;
-  float ra[8];
+  float ra[4], den[4];
   float4 rb[2];
-  float rbv = 0.f;
-  auto fetch = [&](int m0) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int s = q0 + as + 16 * j, m = m0 + am;
+  for (int j = 0; j < 4; ++j) den[j] = 0.f;
+  auto fetch = [&](int m0) {
+    const int m = m0 + am;
+    const float bm_ = m < p.dM ? bv[m] : 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int s = q0 + as + 16 * j;
       ra[j] = (s < call.C && m < p.dM) ? proj[((size_t)i * call.C + s) * ps + m] : 0.f;
+      den[j] = fmaf(ra[j] * ra[j], bm_, den[j]);
     }
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
-      const int m = m0 + bm + 8 * j, c = col0 + bc;
+      const int mm = m0 + bm + 8 * j, c = col0 + bc;
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (m < p.dM) {
-        const float* src = Mh + (size_t)m * p.Dkv + c;
+      if (mm < p.dM) {
+        const float* src = Mh + (size_t)mm * p.Dkv + c;
         if (b_vec && c + 3 < p.Dkv) v = *reinterpret_cast<const float4*>(src);
         else {
           if (c < p.Dkv) v.x = src[0];
@@ -125,22 +145,20 @@ __global__ void __launch_bounds__(256) k_chunk_readout(ImDims p, ImState st, ImW
       }
       rb[j] = v;
     }
-    if (tid < CR_K) rbv = m0 + tid < p.dM ? bv[m0 + tid] : 0.f;
   };
   auto stash = [&](int buf) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) s_a[buf][am][as + 16 * j] = ra[j];
+    for (int j = 0; j < 4; ++j) s_a[buf][am][as + 16 * j] = ra[j];
 #pragma unroll
     for (int j = 0; j < 2; ++j) *reinterpret_cast<float4*>(&s_b[buf][bm + 8 * j][bc]) = rb[j];
-    if (tid < CR_K) s_bv[buf][tid] = rbv;
   };
-  float acc[8][8], den[8];
+  float acc[2][4][4];
 #pragma unroll
-  for (int a = 0; a < 8; ++a) {
-    den[a] = 0.f;
+  for (int mi = 0; mi < 2; ++mi)
 #pragma unroll
-    for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
-  }
+    for (int ni = 0; ni < 4; ++ni)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[mi][ni][e] = 0.f;
   fetch(0);
   stash(0);
   __syncthreads();
@@ -149,38 +167,61 @@ __global__ void __launch_bounds__(256) k_chunk_readout(ImDims p, ImState st, ImW
     const int buf = kb & 1;
     if (kb + 1 < nk) fetch((kb + 1) * CR_K);
 #pragma unroll
-    for (int m = 0; m < CR_K; ++m) {
-      const float4 a0 = *reinterpret_cast<const float4*>(&s_a[buf][m][ty * 4]);
-      const float4 a1 = *reinterpret_cast<const float4*>(&s_a[buf][m][64 + ty * 4]);
-      const float4 b0 = *reinterpret_cast<const float4*>(&s_b[buf][m][tx * 4]);
-      const float4 b1 = *reinterpret_cast<const float4*>(&s_b[buf][m][64 + tx * 4]);
-      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-      const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-      const float bmv = s_bv[buf][m];
+    for (int kk = 0; kk < CR_K; kk += 8) {
+      // fragments: A (query row, m): a0 (g, t), a1 (g + 8, t), a2 (g, t + 4), a3 (g + 8, t + 4); B (m, column): b0 (t, g),
+      // b1 (t + 4, g)
+      uint32_t bh[4][2], bl[4][2];
 #pragma unroll
-      for (int a = 0; a < 8; ++a) {
-        den[a] = fmaf(av[a] * av[a], bmv, den[a]);
+      for (int ni = 0; ni < 4; ++ni) {
+        split_tf32(s_b[buf][kk + t][wc + ni * 8 + g], bh[ni][0], bl[ni][0]);
+        split_tf32(s_b[buf][kk + t + 4][wc + ni * 8 + g], bh[ni][1], bl[ni][1]);
+      }
 #pragma unroll
-        for (int b = 0; b < 8; ++b) acc[a][b] = fmaf(av[a], bb[b], acc[a][b]);
+      for (int mi = 0; mi < 2; ++mi) {
+        uint32_t ah[4], al[4];
+        const int qr = wq + mi * 16 + g;
+        split_tf32(s_a[buf][kk + t][qr], ah[0], al[0]);
+        split_tf32(s_a[buf][kk + t][qr + 8], ah[1], al[1]);
+        split_tf32(s_a[buf][kk + t + 4][qr], ah[2], al[2]);
+        split_tf32(s_a[buf][kk + t + 4][qr + 8], ah[3], al[3]);
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) {
+          mma_tf32(acc[mi][ni], al, bh[ni]);
+          mma_tf32(acc[mi][ni], ah, bl[ni]);
+          mma_tf32(acc[mi][ni], ah, bh[ni]);
+        }
       }
     }
     if (kb + 1 < nk) stash(buf ^ 1);  // (the other buffer: last read before the barrier that ended slice kb - 1)
     __syncthreads();
   }
-  const float cs = st.cscale[u];
+  // denominators: the 16 threads with the same query set (tid >> 4) hold one m each per slice
 #pragma unroll
-  for (int a = 0; a < 8; ++a) {
-    const int s = q0 + (a < 4 ? ty * 4 + a : 64 + ty * 4 + a - 4);
-    if (s >= call.C) continue;
-    const float logit = proj[((size_t)i * call.C + s) * ps + p.dM] + w.bg[0];
-    const float f = cs / (1.0f + expf(-logit)) / (p.eps + den[a]);
-    float* dst = sc.mch + ((size_t)i * call.C + s) * p.Dkv;
+  for (int j = 0; j < 4; ++j) {
+    float d = den[j];
 #pragma unroll
-    for (int b = 0; b < 8; ++b) {
-      const int col = col0 + (b < 4 ? tx * 4 + b : 64 + tx * 4 + b - 4);
-      if (col < p.Dkv) dst[col] = f * acc[a][b];
-    }
+    for (int o = 8; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+    if (am == 0) s_den[as + 16 * j] = d;
   }
+  __syncthreads();
+  const float cs = st.cscale[u];
+  // C fragment: c0, c1 (row g, columns 2 t, 2 t + 1), c2, c3 (row g + 8)
+#pragma unroll
+  for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      const int row = wq + mi * 16 + g + 8 * hf, s = q0 + row;
+      if (s >= call.C) continue;
+      const float logit = proj[((size_t)i * call.C + s) * ps + p.dM] + w.bg[0];
+      const float f = cs / (1.0f + expf(-logit)) / (p.eps + s_den[row]);
+      float* dst = sc.mch + ((size_t)i * call.C + s) * p.Dkv;
+#pragma unroll
+      for (int ni = 0; ni < 4; ++ni) {
+        const int col = col0 + wc + ni * 8 + 2 * t;
+        if (col < p.Dkv) dst[col] = f * acc[mi][ni][2 * hf];
+        if (col + 1 < p.Dkv) dst[col + 1] = f * acc[mi][ni][2 * hf + 1];
+      }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -403,7 +444,7 @@ cudaError_t im_chunk_attn_prepare(const ImDims& p) {
 }
 
 cudaError_t im_launch_chunk_readout(const ImLaunch& L, const ImCall& call) {
-  dim3 grid((L.p.Dkv + CR_T - 1) / CR_T, (call.C + CR_T - 1) / CR_T, call.n_seq);
+  dim3 grid((L.p.Dkv + CR_T - 1) / CR_T, (call.C + CR_TQ - 1) / CR_TQ, call.n_seq);
   k_chunk_readout<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.w, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
