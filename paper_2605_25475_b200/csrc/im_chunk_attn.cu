@@ -3,7 +3,7 @@
 // adds g(q_s) m(q_s) read from the memory as the previous evict steps left it.  Runs after the chunk has been
 // appended to the cache and before it is compressed.
 //
-//   k_chunk_readout    m(q_s) for every chunk query: [C x d_M] x [d_M x D_kv] on CUDA cores, gate applied
+//   k_chunk_readout    m(q_s) for every chunk query: [C x d_M] x [d_M x D_kv] as three tf32 products (mma.sync), gate applied
 //   k_chunk_attention  flash attention, queries on the M dimension of mma.sync m16n8k16: a CTA owns
 //                      128 rows = floor(128 / G_q) queries x G_q heads of one KV head (row = query * G_q + head),
 //                      8 warps x 16 rows, K/V tiles of 32 keys brought in by TMA (the tensor maps of the decode
