@@ -49,7 +49,7 @@ def measured_peaks():
 
 
 # ----------------------------------------------------------------------------------------------
-# algorithmic bytes: what one decode step has to touch in HBM at tau = 1, n = B + 1
+# algorithmic bytes: what one decode step has to touch in HBM (K/V cache, memory state, indexer keys, weights, inputs and outputs)
 def algorithmic_bytes(wl: synth.Workload):
     # entries a step reads, averaged over the phases of a compression interval: B + 1 + p in phase p (tau = 1: B + 1)
     n = wl.B + (wl.tau + 1) / 2
