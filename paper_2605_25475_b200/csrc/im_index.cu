@@ -195,13 +195,15 @@ __global__ void k_prefill_commit(ImDims p, ImState st, ImCall call) {
 // compare >= the threshold.
 struct SelectShared {
   uint32_t hist[256];
-  uint32_t digit, remaining;
+  uint32_t digit, remaining, single;
+  unsigned long long found;
 };
 
 // Key of rank k (k-th largest; keys are distinct) among n entries, by an 8-pass radix select over the 64-bit key,
 // most significant byte first.  Up to SEL_KPT keys per thread stay in registers over the passes (n beyond that:
 // re-read from memory); the digit of a pass is found by warp 0 (lane l sums the 8 bins 255 - 8 l down to
-// 248 - 8 l, a prefix over the lanes locates the lane, which then walks its own bins).
+// 248 - 8 l, a prefix over the lanes locates the lane, which then walks its own bins).  As soon as the chosen bin
+// holds a single key that key is the answer: with distinct scores that is after two or three passes, not eight.
 constexpr int SEL_KPT = 8;
 __device__ uint64_t block_kth_largest_key(const float* __restrict__ score, const int32_t* __restrict__ pos, int n,
                                           int k, int n_sink, SelectShared* sh) {
@@ -258,11 +260,30 @@ __device__ uint64_t block_kth_largest_key(const float* __restrict__ score, const
         }
         sh->digit = (uint32_t)b;
         sh->remaining = rem - cum;
+        sh->single = sh->hist[b] == 1u ? 1u : 0u;
       }
     }
     __syncthreads();
     prefix |= (uint64_t)sh->digit << shift;
     mask |= 0xFFull << shift;
+    if (sh->single) {  // (block uniform) exactly one key carries this prefix: find it
+      if (cached) {
+#pragma unroll
+        for (int j = 0; j < SEL_KPT; ++j) {
+          const int t = threadIdx.x + j * blockDim.x;
+          if (t < n && (kreg[j] & mask) == prefix) sh->found = kreg[j];
+        }
+      } else {
+        for (int t = threadIdx.x; t < n; t += blockDim.x) {
+          const uint64_t key = im_select_key(score[t], pos[t], n_sink);
+          if ((key & mask) == prefix) sh->found = key;
+        }
+      }
+      __syncthreads();
+      const uint64_t key = sh->found;
+      __syncthreads();  // (before a later call of this function writes the structure again)
+      return key;
+    }
     __syncthreads();
   }
   return prefix;
