@@ -694,7 +694,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   //            projections) ---------------------------------------------------------> merge
   //        s1: indexer projections -> front (append, score, select, gather) -> phi of the evicted keys
   //            [-> memory write: not needed by the merge, it only has to end with the call]
-  //        s2: phi(q) / gate projections -> (front kernel ended) -> phi(q)^T Mhat next to the attention kernel
+  //        s2: phi(q) / gate projections -> (front kernel's blocks resident) -> phi(q)^T Mhat next to the attention kernel
   //        s3: float64 key projection (needed by front) -> L2 prefetch for the next layer -> filling of the holes
   //            (once front has listed them and the attention kernel has read the cache)
   //        s4: fold of the pending list (before front, which changes the counters, and before the readout) ->
@@ -791,7 +791,10 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   }
   // append + a1 (+ a2 and the gather of the evicted pairs when the evicted set is small enough for one
   // block per sequence; a4 in the same kernel unless the compaction is deferred)
-  CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max, n_res > 0 ? IM_SMEM_FRONT : 0));
+  // (with SMs set aside: ev[13] triggers when all blocks of the front kernel have begun to run)
+  const bool front_started_ev = conc && n_res > 0;
+  CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max, n_res > 0 ? IM_SMEM_FRONT : 0,
+                             front_started_ev ? ctx->ev[13] : nullptr));
   if (due && !fused) {
     CKL(im_launch_select(L1, call));
     if (ne_max > 0) CKL(im_launch_gather_move(L1, call, ne_max));
@@ -800,12 +803,14 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CK(cudaEventRecord(ctx->ev[11], L1.stream));
     CK(cudaStreamWaitEvent(L3.stream, ctx->ev[11], 0));
   }
-  // phi(q)^T Mhat on s2.  Where SMs are set aside for the front kernel it starts when that kernel has ended: its
-  // blocks would otherwise settle on just those SMs (the emptiest ones) and keep the front blocks out; the
-  // attention kernel has the memory system to itself meanwhile, so nothing is lost.
+  // phi(q)^T Mhat on s2.  Where SMs are set aside for the front kernel it starts when every block of that kernel has
+  // BEGUN to run (a programmatic event that triggers at block start): launched earlier, its blocks would settle on
+  // just those SMs (the emptiest ones) and keep the front blocks out; once the front blocks are resident their
+  // registers leave no room for a readout block, so the readout runs beside the attention CTAs and the two streaming
+  // kernels end together.
   if (conc) {
     if (n_res > 0) {
-      CK(cudaStreamWaitEvent(L2.stream, ctx->ev[11], 0));
+      CK(cudaStreamWaitEvent(L2.stream, front_started_ev ? ctx->ev[13] : ctx->ev[11], 0));
     } else {
       CK(cudaStreamWaitEvent(L2.stream, ctx->ev[1], 0));
       CK(cudaStreamWaitEvent(L2.stream, ctx->ev[2], 0));

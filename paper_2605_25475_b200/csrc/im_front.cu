@@ -335,8 +335,10 @@ __global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, Im
 
 }  // namespace
 
+// `started`: an event (timing disabled) that triggers once every block of the kernel has begun to run; a stream that
+// waits for it launches its next kernel when this kernel's blocks are resident, not when they have ended.
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
-                                   int do_select, int n_max, int smem_floor) {
+                                   int do_select, int n_max, int smem_floor, cudaEvent_t started) {
   static bool attr_done_dev[64] = {};
   bool* attr_done = im_device_flag(attr_done_dev);
   if (!attr_done || !*attr_done) {
@@ -351,11 +353,27 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
   if (smem < (size_t)smem_floor) smem = (size_t)smem_floor;  // keeps the streaming kernels' blocks off this block's SM
   const bf16* kn = (const bf16*)k_new;
   const bf16* vn = (const bf16*)v_new;
-  if (L.p.dI == 16) k_decode_front<16><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
-  else if (L.p.dI == 8) k_decode_front<8><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
-  else k_decode_front<0><<<call.n_seq, FRONT_THREADS, smem, L.stream>>>(L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(call.n_seq);
+  cfg.blockDim = dim3(FRONT_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = L.stream;
+  cudaLaunchAttribute attr[1];
+  if (started) {
+    attr[0].id = cudaLaunchAttributeProgrammaticEvent;
+    attr[0].val.programmaticEvent.event = started;
+    attr[0].val.programmaticEvent.flags = 0;
+    attr[0].val.programmaticEvent.triggerAtBlockStart = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  cudaError_t e;
+  if (L.p.dI == 16) e = cudaLaunchKernelEx(&cfg, k_decode_front<16>, L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
+  else if (L.p.dI == 8) e = cudaLaunchKernelEx(&cfg, k_decode_front<8>, L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
+  else e = cudaLaunchKernelEx(&cfg, k_decode_front<0>, L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
   ++*L.launches;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // deferred compaction (a4): fills the holes and publishes the entry count once the attention kernel has read the

@@ -238,7 +238,7 @@ bool im_tc_gemm_usable(const ImGemmArgs& a);
 cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a);
 cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, int ksplit);
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
-                                   int do_select, int n_max, int smem_floor);
+                                   int do_select, int n_max, int smem_floor, cudaEvent_t started = nullptr);
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_gather(const ImLaunch& L, const ImCall& call, int ne_max);
