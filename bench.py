@@ -131,8 +131,8 @@ def build_context(wl: synth.Workload, device, ingest=True, log=lambda *a: None, 
         t0 = time.time()
         for c in range(wl.ctx // wl.chunk):
             for layer in range(wl.n_layers):
-                X, Q, K, V = synth.prefill_inputs(wl, layer, c, device)
-                g.prefill_chunk(layer, ids, X, Q, K, V)
+                X, Qp, _, K, V = synth.prefill_inputs(wl, layer, c, device)
+                g.prefill_chunk(layer, ids, X, Qp, K, V)
             torch.cuda.synchronize()
             log(f"ingested chunk {c + 1}/{wl.ctx // wl.chunk} ({time.time() - t0:.1f}s)")
         assert g.status() == 0
@@ -140,11 +140,11 @@ def build_context(wl: synth.Workload, device, ingest=True, log=lambda *a: None, 
 
 
 def decode_inputs_all(wl, n_steps, device):
-    """[n_steps][4] tensors stacked over layers: x [L, n, D], q [L, n, H, d], k, v [L, n, Hkv, d]."""
+    """[n_steps][5] tensors stacked over layers: x [L, n, D], q_pre, q [L, n, H, d], k, v [L, n, Hkv, d]."""
     steps = []
     for s in range(n_steps):
         parts = [synth.decode_inputs(wl, layer, s, device) for layer in range(wl.n_layers)]
-        steps.append(tuple(torch.stack([p[i] for p in parts]).contiguous() for i in range(4)))
+        steps.append(tuple(torch.stack([p[i] for p in parts]).contiguous() for i in range(5)))
     return steps
 
 
@@ -168,9 +168,9 @@ def run_ours(args, rank, world, device):
     out = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=device)
 
     def one_step(k):
-        x, q, kk, v = inputs[k % n_in]
+        x, qp, q, kk, v = inputs[k % n_in]
         for layer in range(L):
-            g.decode_step(layer, ids, x[layer], q[layer], q[layer], kk[layer], v[layer], out[layer])
+            g.decode_step(layer, ids, x[layer], qp[layer], q[layer], kk[layer], v[layer], out[layer])
 
     stream = torch.cuda.Stream(device)
     graphs = None
@@ -286,8 +286,8 @@ def run_prefill(args, device):
             def one_pass():
                 g.reset()
                 for c in range(n_chunks):
-                    X, Q, K, V = chunks[c % len(chunks)]
-                    g.prefill_chunk(0, ids, X, Q, K, V)
+                    X, Qp, _, K, V = chunks[c % len(chunks)]
+                    g.prefill_chunk(0, ids, X, Qp, K, V)
 
             for _ in range(args.warmup):
                 one_pass()
@@ -317,8 +317,8 @@ def run_prefill(args, device):
         def attend_pass():
             g.reset()
             for c in range(n_chunks):
-                X, Q, K, V = chunks[c % len(chunks)]
-                g.prefill_chunk_attend(0, ids, X, Q, Q, K, V, out)
+                X, Qp, Q, K, V = chunks[c % len(chunks)]
+                g.prefill_chunk_attend(0, ids, X, Qp, Q, K, V, out)
 
         for _ in range(args.warmup):
             attend_pass()
@@ -349,9 +349,9 @@ ATTN_TRAFFIC_NCU = 272.0e6
 def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     L = wl.n_layers
     n_in = len(inputs)
-    # one pinned host buffer and one device buffer per input set / step: [L][x | q | k | v] (bf16), so that a
+    # one pinned host buffer and one device buffer per input set / step: [L][x | q_pre | q | k | v] (bf16), so that a
     # layer's inputs travel in a single copy
-    sizes = [t[0].numel() for t in inputs[0]]                     # elements per layer of x, q, k, v
+    sizes = [t[0].numel() for t in inputs[0]]                     # elements per layer of x, q_pre, q, k, v
     per_layer = sum(sizes)
     host = []
     for inp in inputs:
@@ -366,7 +366,7 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     for t, n in zip(inputs[0], sizes):
         views.append([dbuf[layer, off:off + n].view(t.shape[1:]) for layer in range(L)])
         off += n
-    dx, dq, dk, dv = views
+    dx, dqp, dq, dk, dv = views
     dout = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=device)
     hout = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16).pin_memory()
     h2d = host[0].numel() * host[0].element_size()
@@ -394,7 +394,7 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device):
                 tick[layer:layer + 1].fill_(1.0)
                 ev_in[layer].record(cs)
             stream.wait_event(ev_in[layer])
-            g.decode_step(layer, ids, dx[layer], dq[layer], dq[layer], dk[layer], dv[layer], dout[layer])
+            g.decode_step(layer, ids, dx[layer], dqp[layer], dq[layer], dk[layer], dv[layer], dout[layer])
             ev_out[layer].record(stream)
             ds.wait_event(ev_out[layer])
             with torch.cuda.stream(ds):
@@ -456,14 +456,14 @@ def oracle_sample(wl, n_units, n_steps, log=lambda *a: None):
     ids = list(range(n_units))
     t0 = time.time()
     for c in range(2 if wl.ctx // wl.chunk >= 2 else 1):
-        X, Q, K, V = synth.prefill_inputs(sub, 0, c)
-        o.prefill_batch(ids, synth.f32(X), synth.f32(Q), synth.f32(K), synth.f32(V))
+        X, Qp, _, K, V = synth.prefill_inputs(sub, 0, c)
+        o.prefill_batch(ids, synth.f32(X), synth.f32(Qp), synth.f32(K), synth.f32(V))
     log(f"oracle sample set up in {time.time() - t0:.1f}s")
     ins = [tuple(synth.f32(t) for t in synth.decode_inputs(sub, 0, s)) for s in range(n_steps)]
     t0 = time.time()
     for s in range(n_steps):
-        x, q, k, v = ins[s]
-        o.decode_batch(ids, x, q, q, k, v)
+        x, qp, q, k, v = ins[s]
+        o.decode_batch(ids, x, qp, q, k, v)
     dt = time.time() - t0
     cores = min(n_units, len(os.sched_getaffinity(0)))
     unit_steps = n_units * n_steps

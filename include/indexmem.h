@@ -280,7 +280,7 @@ int im_get_config(im_ctx* ctx, im_config* out, int32_t* capacity);
  *   q    dev bf16 [n_q_heads, head_dim]
  *   k, v dev bf16 [n_kv_heads, n, head_dim]   (one contiguous slab per KV head)
  *   out  dev bf16 [n_q_heads, head_dim]       out_j = sum_t softmax_t(scale * q_j . k_t) v_t, KV head j / G_q
- *   softmax_scale 0 => 1/sqrt(head_dim);  head_dim <= 256;  n_q_heads a multiple of n_kv_heads
+ *   softmax_scale 0 => 1/sqrt(head_dim);  head_dim <= 256;  n_q_heads a multiple of n_kv_heads, at most 65535
  * Limit: n_q_heads * ceil(n / 256) * (head_dim + 2) <= 1,048,576 (the array's float count); larger
  * problems are rejected with IM_ERR_CAPACITY and a message naming both numbers.
  * The first call on a device looks up the array's device address (a host-side set-up step); make

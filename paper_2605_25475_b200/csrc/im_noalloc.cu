@@ -101,7 +101,9 @@ __global__ void k_noalloc_merge(const float* __restrict__ part, int splits, int 
 }
 
 // device address of the scratch array, looked up once per device (the array's name is only a
-// host-side handle in host code; kernels must be given the address that the runtime reports)
+// host-side handle in host code; kernels must be given the address that the runtime reports).
+// Host threads that make their first call on a device at the same time each look the address up
+// and store the same value: the cache needs no lock.
 constexpr int MAX_DEVICES = 64;
 float* g_scratch_addr[MAX_DEVICES] = {};
 
@@ -112,6 +114,8 @@ extern "C" int im_attention_noalloc(const void* q, const void* k, const void* v,
   if (!q || !k || !v || !out) return im_fail_message(IM_ERR_ARG, "im_attention_noalloc: null tensor");
   if (n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || head_dim < 1 || head_dim > 256 || n < 1)
     return im_fail_message(IM_ERR_ARG, "im_attention_noalloc: bad shape");
+  if (n_q_heads > 65535)  // the query heads ride on the grid's y axis
+    return im_fail_message(IM_ERR_ARG, "im_attention_noalloc: more than 65535 query heads");
   const int splits = (n + SPLIT - 1) / SPLIT;
   const size_t need = (size_t)n_q_heads * splits * (head_dim + 2);
   if (need > SCRATCH_FLOATS) {

@@ -130,21 +130,38 @@ def needle_positions(wl: Workload, layer: int) -> torch.Tensor:
     return torch.stack(rows)
 
 
+def rotate_queries(Q: torch.Tensor, positions: torch.Tensor, base: float = 10000.0) -> torch.Tensor:
+    """The backbone's rotary position embedding applied to query rows: Q [..., T, H, d] float32, positions [T].
+
+    Pairs (i, i + d/2) of every head are rotated by positions * base^(-2i/d).  This belongs to the backbone,
+    not to the method: it only makes the attention query a different tensor from the pre-RoPE query.
+    """
+    d = Q.shape[-1]
+    half = d // 2
+    inv = base ** (-torch.arange(half, device=Q.device, dtype=torch.float32) * 2.0 / d)
+    ang = positions.to(Q.device, torch.float32)[:, None] * inv[None, :]          # [T, d/2]
+    cos, sin = torch.cos(ang)[:, None, :], torch.sin(ang)[:, None, :]            # [T, 1, d/2]
+    a, b = Q[..., :half], Q[..., half:]
+    return torch.cat([a * cos - b * sin, a * sin + b * cos], dim=-1)
+
+
 def prefill_inputs(wl: Workload, layer: int, chunk_idx: int, device="cpu", seqs=None):
     """Inputs of ingestion chunk ``chunk_idx`` for sequences ``seqs`` (default all).
 
-    Returns bf16 tensors X [n, C, D], Q [n, C, H, d], K [n, C, Hkv, d], V [n, C, Hkv, d];
-    Q serves both as the pre-RoPE query of the indexer and as the attention query.
+    Returns bf16 tensors X [n, C, D], Q_pre [n, C, H, d], Q [n, C, H, d], K [n, C, Hkv, d], V [n, C, Hkv, d].
+    Q_pre is the pre-RoPE query (what the indexer reads), Q the same rows after the backbone's rotary
+    embedding at their positions (what attention, Linear_theta and the gate read).
     """
     seqs = list(range(wl.n_seq)) if seqs is None else list(seqs)
     C, t0 = wl.chunk, chunk_idx * wl.chunk
-    Xs, Qs, Ks, Vs = [], [], [], []
+    Xs, Qps, Qs, Ks, Vs = [], [], [], [], []
     npos = needle_positions(wl, layer)
     udir = needle_dirs(wl, layer, device) if wl.n_needles else None
     for s in seqs:
         tag = (wl.name, "prefill", layer, chunk_idx, s)
         X = _randn((C, wl.D), device, *tag, "x")
-        Q = _randn((C, wl.H, wl.d), device, *tag, "q")
+        Qp = _randn((C, wl.H, wl.d), device, *tag, "q")
+        Q = rotate_queries(Qp, torch.arange(t0, t0 + C))
         K = _randn((C, wl.Hkv, wl.d), device, *tag, "k")
         V = _randn((C, wl.Hkv, wl.d), device, *tag, "v")
         if wl.key_norm_sigma > 0:
@@ -154,21 +171,23 @@ def prefill_inputs(wl: Workload, layer: int, chunk_idx: int, device="cpu", seqs=
             for p in npos[s].tolist():
                 if t0 <= p < t0 + C:
                     K[p - t0] = 3.0 * math.sqrt(wl.d) * udir[s]
-        Xs.append(X); Qs.append(Q); Ks.append(K); Vs.append(V)
+        Xs.append(X); Qps.append(Qp); Qs.append(Q); Ks.append(K); Vs.append(V)
     bf = lambda ts: torch.stack(ts).to(torch.bfloat16)
-    return bf(Xs), bf(Qs), bf(Ks), bf(Vs)
+    return bf(Xs), bf(Qps), bf(Qs), bf(Ks), bf(Vs)
 
 
 def decode_inputs(wl: Workload, layer: int, step: int, device="cpu"):
     """Inputs of decode step ``step`` for all sequences.
 
-    Returns bf16 tensors x [n_seq, D], q [n_seq, H, d], k_new [n_seq, Hkv, d], v_new [n_seq, Hkv, d].
-    With needles, q = N(0,1) + sqrt(d) * u with u the planted direction of the query head's KV group.
+    Returns bf16 tensors x [n_seq, D], q_pre [n_seq, H, d], q [n_seq, H, d], k_new [n_seq, Hkv, d],
+    v_new [n_seq, Hkv, d].  q_pre ~ N(0,1) is the pre-RoPE query; q is q_pre rotated at position ctx + step,
+    plus, with needles, sqrt(d) * u with u the planted direction of the query head's KV group.
     """
     tag = (wl.name, "decode", layer, step)
     n = wl.n_seq
     x = _randn((n, wl.D), device, *tag, "x")
-    q = _randn((n, wl.H, wl.d), device, *tag, "q")
+    q_pre = _randn((n, wl.H, wl.d), device, *tag, "q")
+    q = rotate_queries(q_pre[:, None], torch.tensor([wl.ctx + step]))[:, 0]
     k = _randn((n, wl.Hkv, wl.d), device, *tag, "k")
     v = _randn((n, wl.Hkv, wl.d), device, *tag, "v")
     if wl.key_norm_sigma > 0:
@@ -178,7 +197,7 @@ def decode_inputs(wl: Workload, layer: int, step: int, device="cpu"):
         u = needle_dirs(wl, layer, device)                      # [n, Hkv, d]
         q = q + math.sqrt(wl.d) * u.repeat_interleave(wl.H // wl.Hkv, dim=1)
     bf = lambda t: t.to(torch.bfloat16)
-    return bf(x), bf(q), bf(k), bf(v)
+    return bf(x), bf(q_pre), bf(q), bf(k), bf(v)
 
 
 def f32(t: torch.Tensor):

@@ -174,10 +174,10 @@ def test_single_token_chunks_and_subset_of_sequences(im):
         p.prefill(c)
     dev = p.device
     # sequences 2 and 0 only, in that order
-    x, q, k, v = synth.decode_inputs(wl, 0, 0)
+    x, qp, q, k, v = synth.decode_inputs(wl, 0, 0)
     ids = [2, 0]
-    ob, od = p.o.decode_batch(ids, synth.f32(x[ids]), synth.f32(q[ids]), synth.f32(q[ids]), synth.f32(k[ids]), synth.f32(v[ids]))
-    out = p.g.decode_step(0, ids, x[ids].to(dev).contiguous(), q[ids].to(dev).contiguous(), q[ids].to(dev).contiguous(),
+    ob, od = p.o.decode_batch(ids, synth.f32(x[ids]), synth.f32(qp[ids]), synth.f32(q[ids]), synth.f32(k[ids]), synth.f32(v[ids]))
+    out = p.g.decode_step(0, ids, x[ids].to(dev).contiguous(), qp[ids].to(dev).contiguous(), q[ids].to(dev).contiguous(),
                           k[ids].to(dev).contiguous(), v[ids].to(dev).contiguous())
     assert p.g.status() == 0
     p.check_out(out, ob, od)
@@ -188,7 +188,7 @@ def test_errors_are_reported_not_fatal(im):
     wl = TINY.replace(name="errs", ctx=32, chunk=32, B=16, steps=0, n_needles=0)
     p = _pair(wl)
     dev = p.device
-    X, Q, K, V = [t.to(dev) for t in synth.prefill_inputs(wl, 0, 0)]
+    X, Q, _, K, V = [t.to(dev) for t in synth.prefill_inputs(wl, 0, 0)]
     with pytest.raises(im.IndexMemError) as e:
         im.im_prefill_chunk(p.g.ctx, 0, [5], 32, X, Q, K, V)
     assert e.value.code == im.IM_ERR_ARG
@@ -426,15 +426,15 @@ def test_chunk_outputs_call_captured_into_a_cuda_graph(im):
     wl = synth.CONFIGS["llama8b_b1"].replace(name="chunk_out_graph", n_seq=2, ctx=2 * 160, chunk=160, B=200, steps=1, n_needles=2)
     p = _pair(wl, chunk_outputs=1)
     p.prefill_attend(0)
-    X, Q, K, V = synth.prefill_inputs(wl, p.layer, 1)
-    ob, od = p.o.prefill_batch_out(p.seq_ids, synth.f32(X), synth.f32(Q), synth.f32(Q), synth.f32(K), synth.f32(V))
+    X, Qp, Q, K, V = synth.prefill_inputs(wl, p.layer, 1)
+    ob, od = p.o.prefill_batch_out(p.seq_ids, synth.f32(X), synth.f32(Qp), synth.f32(Q), synth.f32(K), synth.f32(V))
     dev = p.device
-    Xd, Qd, Kd, Vd = X.to(dev), Q.to(dev), K.to(dev), V.to(dev)
+    Xd, Qpd, Qd, Kd, Vd = X.to(dev), Qp.to(dev), Q.to(dev), K.to(dev), V.to(dev)
     stream = torch.cuda.Stream(dev)
     with torch.cuda.stream(stream):
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=stream):
-            out = p.g.prefill_chunk_attend(0, p.seq_ids, Xd, Qd, Qd, Kd, Vd)
+            out = p.g.prefill_chunk_attend(0, p.seq_ids, Xd, Qpd, Qd, Kd, Vd)
         graph.replay()
         stream.synchronize()
     assert p.g.status() == 0
@@ -448,6 +448,19 @@ def test_chunk_outputs_call_captured_into_a_cuda_graph(im):
 def test_chunk_outputs_need_their_workspace(im):
     wl = TINY.replace(name="chunk_out_e", ctx=32, chunk=32, B=64, steps=1)
     p = _pair(wl)
-    X, Q, K, V = synth.prefill_inputs(wl, 0, 0)
+    X, Qp, Q, K, V = synth.prefill_inputs(wl, 0, 0)
     with pytest.raises(im.IndexMemError):
-        p.g.prefill_chunk_attend(0, [0], X.cuda(), Q.cuda(), Q.cuda(), K.cuda(), V.cuda())
+        p.g.prefill_chunk_attend(0, [0], X.cuda(), Qp.cuda(), Q.cuda(), K.cuda(), V.cuda())
+
+
+def test_one_tensor_as_both_queries(im):
+    """The header allows q_pre to alias q: one device tensor passed for both (every other test passes two tensors
+    with different values, the pre-RoPE query for the indexer and the rotated one for attention, Linear_theta and
+    the gate)."""
+    wl = TINY.replace(name="alias", H=8, Hkv=2, ctx=200, chunk=100, B=64, steps=6, n_needles=4)
+    p = _pair(wl, alias_q=True, chunk_outputs=1)
+    p.prefill_attend(0)
+    p.prefill_attend(1)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_score_err"] <= 1e-5

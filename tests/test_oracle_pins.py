@@ -107,6 +107,76 @@ def test_index_features_against_numpy():
     assert not np.allclose(qf2, qf) and not np.allclose(alpha2, alpha)
 
 
+def test_index_query_invariants():
+    """What fixes the indexer query and the head gate without restating their formula (Sec. 3.1, Alg. 1): the
+    normalisation is per indexer head over d_I (unit RMS per head; a head's features depend only on its own rows of
+    U_q; rescaling q_pre changes nothing), and with one-hot rows the projections pick single inputs."""
+    rng = np.random.default_rng(11)
+    L = orc.OracleLayer(small_cfg(norm_eps=1e-12))
+    c = L.cfg
+    w = rand_weights(L, rng)
+    x = bf16(rng.standard_normal(L.D))
+    qp = bf16(rng.standard_normal(L.D))
+    qf, alpha = L.index_query(x, qp)
+    # unit RMS per indexer head, not over the whole H_I * d_I vector (the heads' raw norms differ)
+    np.testing.assert_allclose(np.sqrt((qf ** 2).mean(axis=1)), np.ones(c.HI), rtol=1e-9)
+    raw = (w["U_q"].astype(np.float64) @ qp).reshape(c.HI, c.dI)
+    assert abs(np.sqrt((raw[0] ** 2).mean()) / np.sqrt((raw[1] ** 2).mean()) - 1.0) > 1e-3
+    # scale invariance in q_pre (a power of two is exact in bf16); alpha does not depend on q_pre, nor qf on x
+    qf2, alpha2 = L.index_query(x, 4.0 * qp)
+    np.testing.assert_allclose(qf2, qf, rtol=1e-9)
+    np.testing.assert_array_equal(alpha2, alpha)
+    qf3, alpha3 = L.index_query(bf16(rng.standard_normal(L.D)), qp)
+    np.testing.assert_array_equal(qf3, qf)
+    assert not np.allclose(alpha3, alpha)
+    # heads are normalised independently: doubling head 0's rows of U_q leaves every head's features unchanged
+    w2 = dict(w)
+    w2["U_q"] = w["U_q"].copy()
+    w2["U_q"][: c.dI] *= 2.0
+    L.set_weights(w2)
+    qf4, _ = L.index_query(x, qp)
+    np.testing.assert_allclose(qf4, qf, rtol=1e-9)
+    # one-hot rows: feature r of head h reads q_pre[col], the gate reads x[col] / sqrt(H_I d_I)
+    Uq = np.zeros((c.HI * c.dI, L.D), np.float32)
+    cols = rng.permutation(L.D)[: c.HI * c.dI]
+    Uq[np.arange(c.HI * c.dI), cols] = 1.0
+    G = np.zeros((c.HI, L.D), np.float32)
+    gcols = rng.permutation(L.D)[: c.HI]
+    G[np.arange(c.HI), gcols] = 1.0
+    w3 = dict(w, U_q=Uq, G=G)
+    L.set_weights(w3)
+    qf5, alpha5 = L.index_query(x, qp)
+    picked = qp.astype(np.float64)[cols].reshape(c.HI, c.dI)
+    for h in range(c.HI):
+        np.testing.assert_allclose(qf5[h], picked[h] / np.sqrt((picked[h] ** 2).mean()), rtol=1e-9)
+    np.testing.assert_allclose(alpha5, x.astype(np.float64)[gcols] / math.sqrt(c.HI * c.dI), rtol=1e-12)
+    # flatten(Q) is head-major: column j * d + c of U_q reads component c of query head j
+    Q = qp.reshape(c.H, c.d)
+    j, cc = 2, 5
+    Uq1 = np.zeros_like(Uq)
+    Uq1[0, j * c.d + cc] = 1.0
+    Uq1[1, 0] = 1.0
+    L.set_weights(dict(w, U_q=Uq1))
+    qf6, _ = L.index_query(x, qp)
+    assert abs(qf6[0, 0] / qf6[0, 1] - float(Q[j, cc]) / float(Q[0, 0])) < 1e-9
+
+
+def test_score_relu_hand_computed_two_heads():
+    """A_t = sum_h alpha_h ReLU(q_h . k_t) on numbers small enough to do by hand (H_I = 2, d_I = 4)."""
+    L = orc.OracleLayer(small_cfg(act=0))
+    qf = np.array([[1.0, 2.0, 0.0, 0.0], [0.0, 0.0, -1.0, 1.0]])
+    alpha = np.array([0.5, -2.0])
+    kidx = np.array([[1, 1, 1, 1],      # head dots 3, 0   -> 0.5 * 3            = 1.5
+                     [-1, -1, 2, 0],    # head dots -3, -2 -> both clipped        = 0
+                     [0, 0, 0, 2],      # head dots 0, 2   -> -2 * 2              = -4
+                     [2, 0.5, -3, 1]],  # head dots 3, 4   -> 0.5 * 3 - 2 * 4     = -6.5
+                    np.float32)
+    np.testing.assert_array_equal(L.index_scores(qf, alpha, kidx), np.array([1.5, 0.0, -4.0, -6.5]))
+    # without the clipping the second key would score 0.5 * -3 - 2 * -2 = 2.5
+    Li = orc.OracleLayer(small_cfg(act=1))
+    np.testing.assert_array_equal(Li.index_scores(qf, alpha, kidx), np.array([1.5, 2.5, -4.0, -6.5]))
+
+
 def test_score_relu_and_identity_closed_form():
     rng = np.random.default_rng(2)
     for act in (0, 1):
