@@ -162,6 +162,8 @@ def run_ours(args, rank, world, device):
     wl = pick_workload(args)
     log = (lambda *a: print("[bench]", *a, file=sys.stderr, flush=True)) if rank == 0 else (lambda *a: None)
     g, ids = build_context(wl, device, log=log)
+    if args.decode_tensor >= 0:
+        im.im_set_option(g.ctx, im.IM_OPT_DECODE_TENSOR, args.decode_tensor)
     L = wl.n_layers
     n_in = min(8, args.steps + args.warmup)                      # distinct input sets, cycled
     inputs = decode_inputs_all(wl, n_in, device)
@@ -529,6 +531,8 @@ def main():
     ap.add_argument("--tau", type=int, default=0,
                     help="decode with this compression interval (the paper reports 128) instead of the workload's; "
                          "one CUDA graph per phase of the interval is captured")
+    ap.add_argument("--decode-tensor", type=int, default=-1,
+                    help="1 / 0: decode attention on the tcgen05 kernel / the mma.sync kernel (default: the library's choice)")
     ap.add_argument("--traffic", type=float, default=ATTN_TRAFFIC_NCU,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as is)")
     args = ap.parse_args()

@@ -242,12 +242,19 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *   IM_OPT_PROFILE_TARGET which kernel im_profile_begin / im_profile_end time: 0 (default) the attention
  *                        kernel of im_decode_step, 1 the scoring kernel of im_prefill_chunk.  Cannot be
  *                        changed while profiling is active (IM_ERR_STATE).
+ *   IM_OPT_DECODE_TENSOR 1: the attention over the retained entries of im_decode_step (Sec. 2.1, Eq. 4) runs as the
+ *                        warp-specialised tcgen05 kernel (head_dim 128, G_q <= 8: tiles of 128 keys on the M axis, the
+ *                        G_q query heads on N, accumulators in tensor memory, K and V tiles through TMA rings of their
+ *                        own); 0 (default): the mma.sync kernel with a TMA ring per warp, which also serves head_dim
+ *                        64.  Both are within the stated tolerances of a float32 evaluation; they need not agree to
+ *                        the last bit.  Setting 1 for a shape the tensor-core kernel does not take returns IM_ERR_ARG.
  */
 typedef enum im_option {
   IM_OPT_CONCURRENCY = 0,
   IM_OPT_PREFETCH_NEXT = 1,
   IM_OPT_PREFILL_TENSOR = 2,
-  IM_OPT_PROFILE_TARGET = 3
+  IM_OPT_PROFILE_TARGET = 3,
+  IM_OPT_DECODE_TENSOR = 4
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 

@@ -192,6 +192,12 @@ struct im_ctx {
   int device = 0;
   alignas(64) unsigned char mapK[128];  // TMA descriptors of the K / V caches
   alignas(64) unsigned char mapV[128];
+  alignas(64) unsigned char mapKs[128];    // the same caches with the boxes of the mma.sync streaming attention kernel
+  alignas(64) unsigned char mapVs[128];
+  alignas(64) unsigned char mapK128[128];  // the same caches with 128-row boxes (full tiles of the tensor-core attention)
+  alignas(64) unsigned char mapV128[128];
+  bool attn_tc_ready = false;        // the tensor-core streaming attention kernel takes this shape and is set up
+  bool attn_tc = false;              // ... and im_decode_step uses it (IM_OPT_DECODE_TENSOR)
   bool fast_attn = false;
   // Independent pieces of one decode call run on three side streams that fork from and join back into
   // the caller's stream (plain event dependencies, so the pattern can be captured into a CUDA graph).
@@ -379,8 +385,14 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
   if (e == cudaSuccess && im_attn_fast_supported(p)) {
     int sms = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
-    if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK, ctx->mapV);
+    if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK, ctx->mapV, IM_ATTN_TILE);
+    if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapKs, ctx->mapVs, IM_ATTN_STREAM_TILE);
     if (e == cudaSuccess) e = im_attn_prepare(p);
+    if (e == cudaSuccess && im_attn_tc_supported(p)) {
+      e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK128, ctx->mapV128, IM_ATTN_TC_TILE);
+      if (e == cudaSuccess) e = im_attn_tc_prepare();
+      ctx->attn_tc_ready = (e == cudaSuccess);
+    }
     if (e == cudaSuccess) e = im_gemm_prepare_decode();
     if (e == cudaSuccess) e = im_memory_prepare_decode();
     if (e == cudaSuccess) e = im_front_prepare_decode();
@@ -775,7 +787,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
       CK(cudaStreamWaitEvent(s0, ctx->ev[2], 0));
     }
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
-    CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas, n_res > 0 && after_merge ? 1 : 0));
+    if (ctx->attn_tc) CKL(im_launch_attention_tc(L, call, ctx->mapK, ctx->mapV, ctx->mapK128, ctx->mapV128, q, n_ctas, n_res > 0 && after_merge ? 1 : 0));
+    else CKL(im_launch_attention_fast(L, call, ctx->mapKs, ctx->mapVs, q, n_ctas, n_res > 0 && after_merge ? 1 : 0));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
     CK(cudaEventRecord(ctx->ev[9], s0));  // the attention kernel has read the cache
   }
@@ -856,7 +869,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   if (ctx->fast_attn) {
     if (!conc) {
       if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s0));
-      CKL(im_launch_attention_fast(L, call, ctx->mapK, ctx->mapV, q, n_ctas, 0));
+      if (ctx->attn_tc) CKL(im_launch_attention_tc(L, call, ctx->mapK, ctx->mapV, ctx->mapK128, ctx->mapV128, q, n_ctas, 0));
+      else CKL(im_launch_attention_fast(L, call, ctx->mapKs, ctx->mapVs, q, n_ctas, 0));
       if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
     }
     if (!defer && p.mem) CKL(im_launch_readout_finish(L, call));  // after the memory write
@@ -865,7 +879,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
       CK(cudaStreamWaitEvent(s0, ctx->ev[12], 0));  // s2
       CK(cudaStreamWaitEvent(s0, ctx->ev[4], 0));   // s4
     }
-    CKL(im_launch_attention_merge(L, call, out, n_ctas, q, k_new, v_new, conc ? 1 : 0));
+    CKL(im_launch_attention_merge(L, call, out, ctx->attn_tc ? n_ctas : n_ctas * IM_ATTN_WARPS,
+                                  ctx->attn_tc ? IM_ATTN_TC_TILE : IM_ATTN_STREAM_TILE, q, k_new, v_new, conc ? 1 : 0));
     if (defer && !conc) CKL(im_launch_decode_commit(L, call));
     if (conc) CK(cudaStreamWaitEvent(s0, ctx->ev[10], 0));
     if (conc) {  // the memory write only has to end with the call
@@ -898,6 +913,12 @@ int im_set_option(im_ctx* ctx, int option, int value) {
       if (value != 0 && value != 1) return fail(IM_ERR_ARG, "profile target %d: 0 = attention, 1 = prefill scoring", value);
       if (!ctx->prof_ev.empty()) return fail(IM_ERR_STATE, "profiling is active");
       ctx->prof_target = value;
+      return IM_OK;
+    case IM_OPT_DECODE_TENSOR:
+      if (value && !(ctx->fast_attn && ctx->attn_tc_ready))
+        return fail(IM_ERR_ARG, "the tensor-core decode attention kernel needs head_dim 128 and at most 8 query heads per KV head");
+      ctx->attn_tc = value != 0;
+      ctx->tail_is_merge = false;
       return IM_OK;
     default: return fail(IM_ERR_ARG, "unknown option %d", option);
   }

@@ -22,7 +22,8 @@
 namespace {
 
 constexpr float NEG_INF = -__builtin_huge_valf();
-constexpr int TILE = IM_ATTN_TILE;       // keys per tile
+constexpr int TILE = IM_ATTN_STREAM_TILE;  // keys per tile (48-key tiles with 6 KB boxes and a 192 KB ring measured slower
+                                           // in the full step: the readout kernel next to it then falls behind)
 constexpr int STAGES = 2;                // ring depth per warp
 constexpr int WARPS = IM_ATTN_WARPS;     // consumer warps per CTA (each also issues its own TMA)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;  // try_wait attempts before a warp gives up and flags ST_TIMEOUT
@@ -532,7 +533,7 @@ __device__ __forceinline__ void softmax_push(float s, const float (&v)[CPL], flo
 // that the block's warps together recompute, from the cache, which is still uncompacted, the partials of that
 // head whose key range holds an evicted entry.
 template <int DH, typename OutT>
-__global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st, ImScratch sc, ImCall call, int n_ctas,
+__global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st, ImScratch sc, ImCall call, int n_workers, int tile,
                                                           OutT* __restrict__ out, const bf16* __restrict__ q,
                                                           const bf16* __restrict__ k_new, const bf16* __restrict__ v_new) {
   constexpr int CPL = DH / 32;  // columns per lane
@@ -651,7 +652,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
     int na = 0;
     if (k0 == 0) na = na_lane;
     else if (k < call.n_seq) na = sc.n_att[k];
-    const int nk = tiles_of(na);
+    const int nk = (na + tile - 1) / tile;
     // inclusive prefix over the 32 lanes
     long long incl = (long long)nk * p.Hkv;
 #pragma unroll
@@ -667,7 +668,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
     total += __shfl_sync(0xffffffffu, incl, 31);
   }
   n_old = max(0, min(n_old, p.cap - 1));  // with deferred compaction: the slot of the new token
-  const long long WT = (long long)n_ctas * WARPS;
+  const long long WT = n_workers;  // runs the attention kernel cut the tiles into (warps or CTAs)
   const long long qrun = (total + WT - 1) / WT;
   const long long row_first = pref + (long long)h * nt_i, row_last = row_first + nt_i - 1;
   const long long row_id = (long long)i * p.Hkv + h;
@@ -683,8 +684,8 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
   auto partial_keys = [&](long long wv, int& key0, int& key1) {
     const int lt0 = (int)(max(wv * qrun, row_first) - row_first);
     const int lt1 = (int)(min((wv + 1) * qrun - 1, row_last) - row_first);
-    key0 = lt0 * TILE;
-    key1 = min((lt1 + 1) * TILE, n_old);
+    key0 = lt0 * tile;
+    key1 = min((lt1 + 1) * tile, n_old);
   };
   auto merge_stored = [&](long long wv, int head, float& M, float& L, float (&res)[CPL]) {
     const float* ps = sc.part + ((size_t)(wv + row_id) * p.Gq + head) * (DH + 2);
@@ -884,10 +885,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 }  // namespace
 
 // Encodes the tensor maps of the K and V caches: 2-D [rows = units * Hkv * cap, cols = d] bf16,
-// box = 64 columns x TILE rows, 128-byte swizzle.  Returns false if the fast path is unavailable.
+// box = 64 columns x box_rows rows, 128-byte swizzle.  Returns false if the fast path is unavailable.
 bool im_attn_fast_supported(const ImDims& p) { return (p.d == 64 || p.d == 128) && p.Gq <= 8 && p.Dkv % 4 == 0; }
 
-cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV) {
+cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV, int box_rows) {
   static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -898,7 +899,7 @@ cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, vo
   const cuuint64_t rows = (cuuint64_t)p.L * p.S * p.Hkv * p.cap;
   const cuuint64_t dims[2] = {(cuuint64_t)p.d, rows};
   const cuuint64_t strides[1] = {(cuuint64_t)p.d * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)TILE};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   void* bases[2] = {st.Kc, st.Vc};
   void* maps[2] = {mapK, mapV};
@@ -976,7 +977,7 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas, const void* q,
+cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_workers, int tile, const void* q,
                                       const void* k_new, const void* v_new, int programmatic) {
   const bf16* qp = (const bf16*)q;
   const bf16* kp = (const bf16*)k_new;
@@ -996,11 +997,11 @@ cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, voi
   cfg.numAttrs = programmatic ? 1 : 0;
   cudaError_t e;
   if (p.d == 64) {
-    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, float>, p, L.st, L.sc, call, n_ctas, (float*)out, qp, kp, vp);
-    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, bf16>, p, L.st, L.sc, call, n_ctas, (bf16*)out, qp, kp, vp);
+    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, float>, p, L.st, L.sc, call, n_workers, tile, (float*)out, qp, kp, vp);
+    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, bf16>, p, L.st, L.sc, call, n_workers, tile, (bf16*)out, qp, kp, vp);
   } else {
-    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, float>, p, L.st, L.sc, call, n_ctas, (float*)out, qp, kp, vp);
-    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, bf16>, p, L.st, L.sc, call, n_ctas, (bf16*)out, qp, kp, vp);
+    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, float>, p, L.st, L.sc, call, n_workers, tile, (float*)out, qp, kp, vp);
+    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, bf16>, p, L.st, L.sc, call, n_workers, tile, (bf16*)out, qp, kp, vp);
   }
   ++*L.launches;
   return e != cudaSuccess ? e : cudaGetLastError();

@@ -141,7 +141,9 @@ constexpr int DG_DEPTH = 4;   // 32-wide chunks whose loads (weights and vectors
 constexpr int DG_WARPS = 8;
 template <bool TWO>  // TWO: the jobs have a second weight term
 __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
-  __shared__ float red[DG_WARPS][16][33];
+  // the warps' partial tiles are added through shared memory in two rounds of four warps (half the buffer: the block
+  // fits next to a streaming attention CTA that leaves 12 KB of an SM's shared memory), in warp order: deterministic
+  __shared__ float red[DG_WARPS / 2][16][33];
   int tile = blockIdx.x, j = 0;
   while (j + 1 < a.n_jobs && tile >= (a.job[j].rows + 15) / 16) {
     tile -= (a.job[j].rows + 15) / 16;
@@ -206,24 +208,40 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
     }
   }
   // C fragment: rows g / g+8, columns 8 nt + 2t / + 1
+  constexpr int ITEMS = 16 * VB / (DG_WARPS * 32);  // outputs per thread
+  float sum[ITEMS];
 #pragma unroll
-  for (int nt = 0; nt < 4; ++nt) {
-    red[warp][g][nt * 8 + 2 * t] = acc[nt][0];
-    red[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1];
-    red[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2];
-    red[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3];
+  for (int k = 0; k < ITEMS; ++k) sum[k] = 0.f;
+#pragma unroll
+  for (int round = 0; round < 2; ++round) {
+    if ((warp >> 2) == round) {
+      const int w = warp & 3;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        red[w][g][nt * 8 + 2 * t] = acc[nt][0];
+        red[w][g][nt * 8 + 2 * t + 1] = acc[nt][1];
+        red[w][g + 8][nt * 8 + 2 * t] = acc[nt][2];
+        red[w][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3];
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < ITEMS; ++k) {
+      const int idx = threadIdx.x + k * DG_WARPS * 32;
+      const int r = idx & 15, vl = idx >> 4;
+#pragma unroll
+      for (int w = 0; w < DG_WARPS / 2; ++w) sum[k] += red[w][r][vl];
+    }
+    __syncthreads();
   }
-  __syncthreads();
   float* outk = a.out + (size_t)ks * a.ks_stride;
-  for (int idx = threadIdx.x; idx < 16 * VB; idx += DG_WARPS * 32) {
+#pragma unroll
+  for (int k = 0; k < ITEMS; ++k) {
+    const int idx = threadIdx.x + k * DG_WARPS * 32;
     const int r = idx & 15, vl = idx >> 4;
     const long long v = v0 + vl;
-    if (v < a.NV && r0 + r < job.rows) {
-      float sum = 0.f;
-#pragma unroll
-      for (int w = 0; w < DG_WARPS; ++w) sum += red[w][r][vl];  // warp order: deterministic
-      outk[(v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0 + r] = sum;
-    }
+    if (v < a.NV && r0 + r < job.rows)
+      outk[(v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0 + r] = sum[k];
   }
 }
 

@@ -10,8 +10,10 @@ typedef __nv_bfloat16 bf16;
 
 #define IM_MAX_CALL_SEQS 256 /* sequences per hot call (the id list travels as a kernel parameter) */
 #define IM_SLOT_ALIGN 64     /* slot capacity is a multiple of the attention tile */
-#define IM_ATTN_TILE 32      /* keys per attention tile (one TMA box is 32 rows x 128 bytes) */
+#define IM_ATTN_TILE 32      /* rows of the small TMA box of the cache's tensor maps (32 rows x 128 bytes) */
+#define IM_ATTN_STREAM_TILE 32 /* keys per tile (= rows of a TMA box) of the mma.sync streaming attention kernel */
 #define IM_ATTN_WARPS 4      /* warps per CTA of the streaming attention kernel */
+#define IM_ATTN_TC_TILE 128  /* keys per tile of the tensor-core streaming attention kernel (= the TMEM lanes) */
 #define IM_ATTN_MAX_CTAS 512 /* upper bound of its grid (one CTA per SM) */
 #define IM_TC_QT 32          /* queries per tile of the tensor-core prefill scoring */
 #define IM_TC_HP 8           /* head slots per query in its operand (indexer heads, zero padded) */
@@ -266,14 +268,21 @@ cudaError_t im_launch_chunk_attention_tc(const ImLaunch& L, const ImCall& call, 
 cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const void* q, void* out, int n_max);
 bool im_attn_fast_supported(const ImDims& p);
-cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV);
+cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV, int box_rows);
+// tcgen05 version of the streaming attention kernel (head_dim 128): one run of 128-key tiles per CTA; mapK / mapV
+// with 32-row boxes (ragged last tile of a row), mapK128 / mapV128 with 128-row boxes (full tiles)
+bool im_attn_tc_supported(const ImDims& p);
+cudaError_t im_attn_tc_prepare();
+cudaError_t im_launch_attention_tc(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
+                                   const void* mapK128, const void* mapV128, const void* q, int n_ctas, int programmatic);
 cudaError_t im_attn_prepare(const ImDims& p);
 // grid blocks (at most one per SM wanted); light: the variant that leaves room for a front block on its SM
 cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call, int grid, int light);
 cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
                                      const void* q, int n_ctas, int programmatic);
-cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_ctas, const void* q,
+// n_workers / tile: the runs the attention kernel of the call cut the tiles into, and its tile size
+cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_workers, int tile, const void* q,
                                       const void* k_new, const void* v_new, int programmatic);
 
 cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,

@@ -292,14 +292,16 @@ def test_peaked_attention_evicted_entry_dominates_softmax(im):
     assert im.im_event_count(p.g.ctx, im.IM_COUNT_MERGE_RECOMPUTE) > 0
 
 
-@pytest.mark.parametrize("conc", [0, 1])
-def test_decode_schedules_agree_with_the_oracle(im, conc):
-    """The in-order schedule and the concurrent one (attention first, evicted terms removed in the merge)
-    against the oracle on the same inputs: several sequences, evictions every step, needles, then steps on a
-    cache that is not full yet (nothing evicted, the new token only added)."""
+@pytest.mark.parametrize("conc,tensor", [(0, 1), (1, 1), (0, 0), (1, 0)])
+def test_decode_schedules_agree_with_the_oracle(im, conc, tensor):
+    """The in-order schedule and the concurrent one (attention first, evicted terms removed in the merge), each with
+    the tensor-core attention kernel and with the mma.sync one, against the oracle on the same inputs: several
+    sequences, evictions every step, needles, then steps on a cache that is not full yet (nothing evicted, the new
+    token only added)."""
     wl = synth.CONFIGS["llama8b_b1"].replace(name="sched", n_seq=3, ctx=333, chunk=333, B=300, steps=12, n_needles=4)
     p = _pair(wl)
     im.im_set_option(p.g.ctx, im.IM_OPT_CONCURRENCY, conc)
+    im.im_set_option(p.g.ctx, im.IM_OPT_DECODE_TENSOR, tensor)
     p.prefill(0)
     for s in range(wl.steps):
         p.decode(s)
@@ -307,6 +309,7 @@ def test_decode_schedules_agree_with_the_oracle(im, conc):
     wl2 = wl.replace(name="sched_notfull", ctx=40, chunk=40, B=64, steps=30)   # fills up at step 24
     p2 = _pair(wl2)
     im.im_set_option(p2.g.ctx, im.IM_OPT_CONCURRENCY, conc)
+    im.im_set_option(p2.g.ctx, im.IM_OPT_DECODE_TENSOR, tensor)
     p2.prefill(0)
     for s in range(wl2.steps):
         p2.decode(s)
@@ -464,3 +467,37 @@ def test_one_tensor_as_both_queries(im):
     for s in range(wl.steps):
         p.decode(s)
     assert p.stats["max_out_err"] <= 2e-3 and p.stats["max_score_err"] <= 1e-5
+
+
+@pytest.mark.parametrize("tensor", [1, 0])
+@pytest.mark.parametrize("shape", ["llama8b_b1", "qwen7b_b8"])
+def test_decode_attention_float32_ragged_rows_and_rising_maxima(im, tensor, shape):
+    """The streaming attention kernels with the float32 result exposed (bound 1e-4 of the tensor's max-abs) at
+    head_dim 128, G_q = 4 and 7: five sequences whose rows hold several 128-key tiles with ragged tails, a softmax
+    scale four times the usual one, so that a row's running maximum rises by more than 2^8 several times along the
+    row (the tensor-core kernel then rescales its accumulators in tensor memory) and the entry evicted in a step
+    often carries most of a head's mass (the merge then recomputes the head)."""
+    wl = synth.CONFIGS[shape].replace(name="attn_f32_" + shape, n_seq=5, ctx=700, chunk=700, B=645, steps=10, n_needles=6)
+    p = _pair(wl, out_f32=1, scale=4.0 / np.sqrt(wl.d))
+    im.im_set_option(p.g.ctx, im.IM_OPT_DECODE_TENSOR, tensor)
+    p.prefill(0)
+    for s in range(wl.steps):
+        p.decode(s)
+    assert p.stats["max_out_err"] <= 1e-4 and p.stats["max_M_err"] <= 2e-3
+    # rows of different lengths in one call, none of them full: 37, 131 and 257 entries (no eviction yet)
+    for k, ctx in enumerate((36, 130, 256)):
+        wl2 = wl.replace(name=f"attn_f32_short{k}", n_seq=2, ctx=ctx, chunk=ctx, B=400, steps=3, n_needles=0)
+        p2 = _pair(wl2, out_f32=1)
+        im.im_set_option(p2.g.ctx, im.IM_OPT_DECODE_TENSOR, tensor)
+        p2.prefill(0)
+        for s in range(wl2.steps):
+            p2.decode(s)
+        assert p2.stats["max_out_err"] <= 1e-4
+
+
+def test_decode_tensor_option_is_refused_for_other_head_dims(im):
+    p = _pair(TINY.replace(name="opt", ctx=32, chunk=32, B=16, steps=0))
+    with pytest.raises(im.IndexMemError) as e:
+        im.im_set_option(p.g.ctx, im.IM_OPT_DECODE_TENSOR, 1)
+    assert e.value.code == im.IM_ERR_ARG
+    im.im_set_option(p.g.ctx, im.IM_OPT_DECODE_TENSOR, 0)
