@@ -164,6 +164,8 @@ def run_ours(args, rank, world, device):
     g, ids = build_context(wl, device, log=log)
     if args.decode_tensor >= 0:
         im.im_set_option(g.ctx, im.IM_OPT_DECODE_TENSOR, args.decode_tensor)
+    if args.readout_stages >= 0:
+        im.im_set_option(g.ctx, im.IM_OPT_READOUT_STAGES, args.readout_stages)
     L = wl.n_layers
     n_in = min(8, args.steps + args.warmup)                      # distinct input sets, cycled
     inputs = decode_inputs_all(wl, n_in, device)
@@ -533,6 +535,8 @@ def main():
                          "one CUDA graph per phase of the interval is captured")
     ap.add_argument("--decode-tensor", type=int, default=-1,
                     help="1 / 0: decode attention on the tcgen05 kernel / the mma.sync kernel (default: the library's choice)")
+    ap.add_argument("--readout-stages", type=int, default=-1,
+                    help="0: readout on plain loads; k >= 1: on a ring of k 32 KB bulk copies per CTA (default: the library's choice)")
     ap.add_argument("--traffic", type=float, default=ATTN_TRAFFIC_NCU,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as is)")
     args = ap.parse_args()

@@ -248,13 +248,20 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        own); 0 (default): the mma.sync kernel with a TMA ring per warp, which also serves head_dim
  *                        64.  Both are within the stated tolerances of a float32 evaluation; they need not agree to
  *                        the last bit.  Setting 1 for a shape the tensor-core kernel does not take returns IM_ERR_ARG.
+ *   IM_OPT_READOUT_STAGES k >= 1: in concurrent decode calls with SMs set aside for
+ *                        the front kernel, phi(q)^T Mhat of Eq. 5 is formed by a persistent kernel that brings the rows of
+ *                        Mhat in through a ring of k 32 KB bulk copies per CTA, one CTA beside each attention CTA
+ *                        (k <= 6; D_kv a power of two of at most 1024 and d_M a multiple of 8192 / D_kv); 0 (default): by the
+ *                        kernel built on plain loads, which serves every shape and schedule.  The two add the rows in different
+ *                        orders (float32); both are within the stated tolerances.
  */
 typedef enum im_option {
   IM_OPT_CONCURRENCY = 0,
   IM_OPT_PREFETCH_NEXT = 1,
   IM_OPT_PREFILL_TENSOR = 2,
   IM_OPT_PROFILE_TARGET = 3,
-  IM_OPT_DECODE_TENSOR = 4
+  IM_OPT_DECODE_TENSOR = 4,
+  IM_OPT_READOUT_STAGES = 5
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 

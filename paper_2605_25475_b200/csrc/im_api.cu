@@ -150,7 +150,7 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->sc.mres = (float*)take((size_t)p.S * IM_MRES_ROW(p) * 4);
   lo->sc.phiq = (float*)take((size_t)p.S * p.dM * 4);
   lo->sc.n_att = (int32_t*)take((size_t)p.S * 4);
-  lo->sc.rpart = (float*)take((size_t)p.S * p.Dkv * 4);
+  lo->sc.rpart = (float*)take((size_t)(IM_ATTN_MAX_CTAS + p.S) * p.Dkv * 4);
   lo->sc.phiT = nullptr;
   lo->sc.vT = nullptr;
   lo->sc.gpart_vecs = std::min<long long>((long long)p.S * p.max_chunk, 8192);
@@ -196,6 +196,8 @@ struct im_ctx {
   alignas(64) unsigned char mapVs[128];
   alignas(64) unsigned char mapK128[128];  // the same caches with 128-row boxes (full tiles of the tensor-core attention)
   alignas(64) unsigned char mapV128[128];
+  bool ro_stream = false;            // phi(q)^T Mhat by the bulk-copy streaming kernel where it runs next to the attention kernel (IM_OPT_READOUT_STAGES)
+  int ro_stages = 2;                 // ... with this many 32 KB stages per CTA
   bool attn_tc_ready = false;        // the tensor-core streaming attention kernel takes this shape and is set up
   bool attn_tc = false;              // ... and im_decode_step uses it (IM_OPT_DECODE_TENSOR)
   bool fast_attn = false;
@@ -393,6 +395,7 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
       if (e == cudaSuccess) e = im_attn_tc_prepare();
       ctx->attn_tc_ready = (e == cudaSuccess);
     }
+    if (e == cudaSuccess && p.mem && im_readout_stream_supported(p)) e = im_readout_stream_prepare(p);
     if (e == cudaSuccess) e = im_gemm_prepare_decode();
     if (e == cudaSuccess) e = im_memory_prepare_decode();
     if (e == cudaSuccess) e = im_front_prepare_decode();
@@ -829,7 +832,16 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
       CK(cudaStreamWaitEvent(L2.stream, ctx->ev[2], 0));
     }
   }
-  if (ctx->fast_attn && p.mem && readout_early) CKL(im_launch_readout(L2, call, n_res > 0 ? n_ctas : ctx->n_sm, conc && n_res == 0));
+  // (with SMs set aside and the bulk-copy kernel: one CTA beside each attention CTA, its ring next to that CTA's)
+  int ro_workers = 0;
+  if (ctx->fast_attn && p.mem && readout_early) {
+    if (conc && n_res > 0 && ctx->ro_stream) {
+      ro_workers = (int)std::min<long long>(n_ctas, (long long)n_seq * im_readout_stream_chunks(p));
+      CKL(im_launch_readout_stream(L2, call, ro_workers, ctx->ro_stages));
+    } else {
+      CKL(im_launch_readout(L2, call, n_res > 0 ? n_ctas : ctx->n_sm, conc && n_res == 0));
+    }
+  }
   if (conc) CK(cudaEventRecord(ctx->ev[12], L2.stream));  // s2 finished: the merge needs phi(q)^T Mhat
   if (ctx->prefetch_next && ctx->fast_attn) {
     // warm L2 for the next layer's small kernels while this layer's attention streams K/V; after the front kernel,
@@ -880,7 +892,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
       CK(cudaStreamWaitEvent(s0, ctx->ev[4], 0));   // s4
     }
     CKL(im_launch_attention_merge(L, call, out, ctx->attn_tc ? n_ctas : n_ctas * IM_ATTN_WARPS,
-                                  ctx->attn_tc ? IM_ATTN_TC_TILE : IM_ATTN_STREAM_TILE, q, k_new, v_new, conc ? 1 : 0));
+                                  ctx->attn_tc ? IM_ATTN_TC_TILE : IM_ATTN_STREAM_TILE, ro_workers, q, k_new, v_new, conc ? 1 : 0));
     if (defer && !conc) CKL(im_launch_decode_commit(L, call));
     if (conc) CK(cudaStreamWaitEvent(s0, ctx->ev[10], 0));
     if (conc) {  // the memory write only has to end with the call
@@ -919,6 +931,13 @@ int im_set_option(im_ctx* ctx, int option, int value) {
         return fail(IM_ERR_ARG, "the tensor-core decode attention kernel needs head_dim 128 and at most 8 query heads per KV head");
       ctx->attn_tc = value != 0;
       ctx->tail_is_merge = false;
+      return IM_OK;
+    case IM_OPT_READOUT_STAGES:
+      if (value < 0 || value > 6) return fail(IM_ERR_ARG, "readout stages %d out of range [0,6]", value);
+      if (value > 0 && !(ctx->fast_attn && ctx->p.mem && im_readout_stream_supported(ctx->p)))
+        return fail(IM_ERR_ARG, "the bulk-copy readout kernel does not take this shape (D_kv a power of two of at most 1024, d_M a multiple of 8192 / D_kv)");
+      ctx->ro_stream = value > 0;
+      if (value > 0) ctx->ro_stages = value;
       return IM_OK;
     default: return fail(IM_ERR_ARG, "unknown option %d", option);
   }

@@ -534,7 +534,7 @@ __device__ __forceinline__ void softmax_push(float s, const float (&v)[CPL], flo
 // head whose key range holds an evicted entry.
 template <int DH, typename OutT>
 __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st, ImScratch sc, ImCall call, int n_workers, int tile,
-                                                          OutT* __restrict__ out, const bf16* __restrict__ q,
+                                                          int ro_workers, int ro_cs, OutT* __restrict__ out, const bf16* __restrict__ q,
                                                           const bf16* __restrict__ k_new, const bf16* __restrict__ v_new) {
   constexpr int CPL = DH / 32;  // columns per lane
   __shared__ float s_q[8][DH];       // redo path: the query rows of the heads to redo
@@ -552,7 +552,16 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
   const int ne_raw = st.ctr[u * CTR_STRIDE + CTR_NEVICT];
   const int ev_l = lane < IM_FRONT_MAX_NE ? st.ev_slot[u * p.tail + min(lane, p.tail - 1)] : -1;
   const float* mr = sc.mres + (size_t)i * IM_MRES_ROW(p);
-  const float* rs = sc.rpart + (size_t)i * p.Dkv;  // phi(q)^T Mhat (k_readout_cols)
+  // phi(q)^T Mhat: one vector per sequence (k_readout_cols), or - ro_workers > 0 - the partial vectors of the CTAs of
+  // k_readout_stream whose runs of ro_cs chunks per sequence hold chunks of this sequence, added in CTA order
+  const float* rs = sc.rpart + (size_t)i * p.Dkv;
+  int rw0 = 0, rw1 = 0;
+  if (ro_workers > 0) {
+    const long long rq = ((long long)call.n_seq * ro_cs + ro_workers - 1) / ro_workers;
+    rw0 = (int)(((long long)i * ro_cs) / rq);
+    rw1 = (int)(((long long)(i + 1) * ro_cs - 1) / rq);
+    rs = sc.rpart + (size_t)(rw0 + i) * p.Dkv;
+  }
   float pf0[4], pq0[4];
   float gate = 0.f, c_hat = 0.f, den_old = 0.f, mcol[CPL], qv[CPL], kn[CPL], vn[CPL], ek0[CPL], ev0[CPL];
   {
@@ -577,7 +586,9 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
 #pragma unroll
     for (int k = 0; k < CPL; ++k) {
       const int c = lane + 32 * k;
-      mcol[k] = p.mem ? fmaf(c_hat, rs[h * DH + c], mr[h * DH + c]) : 0.f;
+      float rv = p.mem ? rs[h * DH + c] : 0.f;
+      for (int w = rw0 + 1; w <= rw1; ++w) rv += rs[(size_t)(w - rw0) * p.Dkv + h * DH + c];
+      mcol[k] = p.mem ? fmaf(c_hat, rv, mr[h * DH + c]) : 0.f;
       qv[k] = __bfloat162float(qrow[c]);
       kn[k] = __bfloat162float(kr[c]);
       vn[k] = __bfloat162float(vr[c]);
@@ -977,8 +988,9 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_workers, int tile, const void* q,
-                                      const void* k_new, const void* v_new, int programmatic) {
+cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_workers, int tile, int ro_workers,
+                                      const void* q, const void* k_new, const void* v_new, int programmatic) {
+  const int ro_cs = ro_workers > 0 ? im_readout_stream_chunks(L.p) : 0;
   const bf16* qp = (const bf16*)q;
   const bf16* kp = (const bf16*)k_new;
   const bf16* vp = (const bf16*)v_new;
@@ -997,11 +1009,11 @@ cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, voi
   cfg.numAttrs = programmatic ? 1 : 0;
   cudaError_t e;
   if (p.d == 64) {
-    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, float>, p, L.st, L.sc, call, n_workers, tile, (float*)out, qp, kp, vp);
-    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, bf16>, p, L.st, L.sc, call, n_workers, tile, (bf16*)out, qp, kp, vp);
+    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, float>, p, L.st, L.sc, call, n_workers, tile, ro_workers, ro_cs, (float*)out, qp, kp, vp);
+    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<64, bf16>, p, L.st, L.sc, call, n_workers, tile, ro_workers, ro_cs, (bf16*)out, qp, kp, vp);
   } else {
-    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, float>, p, L.st, L.sc, call, n_workers, tile, (float*)out, qp, kp, vp);
-    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, bf16>, p, L.st, L.sc, call, n_workers, tile, (bf16*)out, qp, kp, vp);
+    if (p.out_f32) e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, float>, p, L.st, L.sc, call, n_workers, tile, ro_workers, ro_cs, (float*)out, qp, kp, vp);
+    else e = cudaLaunchKernelEx(&cfg, k_attn_merge_rows<128, bf16>, p, L.st, L.sc, call, n_workers, tile, ro_workers, ro_cs, (bf16*)out, qp, kp, vp);
   }
   ++*L.launches;
   return e != cudaSuccess ? e : cudaGetLastError();

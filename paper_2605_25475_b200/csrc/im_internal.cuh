@@ -99,7 +99,8 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
   int32_t* nhole;    // [max_seqs]             compaction: number of evicted slots below the budget
   float* part;       // attention partials (acc[d], max, sum): generic kernel [max_seqs][H][max_splits][d + 2];
                      // streaming kernel [warps + rows][Gq][d + 2]
-  float* rpart;      // [max_seqs][Dkv] readout numerators: phi(q)^T Mhat
+  float* rpart;      // readout numerators phi(q)^T Mhat: [max_seqs][Dkv] (k_readout_cols), or partial vectors
+                     // [CTAs + max_seqs][Dkv] (k_readout_stream)
   float* mres;       // [max_seqs][IM_MRES_ROW] per column the part of the memory readout (Eq. 5) that does not go
                      // through Mhat (pending list, entries written in this call), then the gate g(q), the denominator
                      // sum, and the coefficient c of the Mhat part: m(q)[col] = mres[col] + c * rpart[col]
@@ -281,9 +282,15 @@ cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call, int grid, i
 cudaError_t im_launch_readout_finish(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, const void* mapK, const void* mapV,
                                      const void* q, int n_ctas, int programmatic);
-// n_workers / tile: the runs the attention kernel of the call cut the tiles into, and its tile size
-cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_workers, int tile, const void* q,
-                                      const void* k_new, const void* v_new, int programmatic);
+// n_workers / tile: the runs the attention kernel of the call cut the tiles into, and its tile size; ro_workers: CTAs
+// of the streaming readout kernel whose partial vectors are to be added (0: one vector per sequence from k_readout_cols)
+cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, void* out, int n_workers, int tile, int ro_workers,
+                                      const void* q, const void* k_new, const void* v_new, int programmatic);
+// phi(q)^T Mhat as a persistent kernel fed by bulk copies (ring of `stages` 32 KB stages per CTA)
+bool im_readout_stream_supported(const ImDims& p);
+int im_readout_stream_chunks(const ImDims& p);
+cudaError_t im_readout_stream_prepare(const ImDims& p);
+cudaError_t im_launch_readout_stream(const ImLaunch& L, const ImCall& call, int grid, int stages);
 
 cudaError_t im_launch_topb(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink,
                            uint8_t* keep, int32_t* n_evict, cudaStream_t stream);

@@ -501,3 +501,25 @@ def test_decode_tensor_option_is_refused_for_other_head_dims(im):
         im.im_set_option(p.g.ctx, im.IM_OPT_DECODE_TENSOR, 1)
     assert e.value.code == im.IM_ERR_ARG
     im.im_set_option(p.g.ctx, im.IM_OPT_DECODE_TENSOR, 0)
+
+
+@pytest.mark.parametrize("tensor,stages", [(0, 1), (0, 3), (1, 2), (1, 6)])
+def test_decode_readout_through_bulk_copy_ring(im, tensor, stages):
+    """phi(q)^T Mhat formed by the persistent bulk-copy kernel (a ring of 32 KB stages per CTA next to the attention
+    kernel, partial vectors per CTA added by the merge) instead of the kernel on plain loads: Llama widths (D_kv 1024,
+    8 rows per chunk) and Qwen widths (D_kv 512, d_M 448: 16 rows per chunk, two row groups per column), several
+    sequences, evictions every step with decay, float32 outputs held to 1e-4, the memory to 2e-3."""
+    for shape, n_seq in (("llama8b_b1", 3), ("qwen7b_b8", 5)):
+        wl = synth.CONFIGS[shape].replace(name=f"ro_ring_{shape}", n_seq=n_seq, ctx=300, chunk=300, B=200, steps=24, n_needles=3)
+        p = _pair(wl, out_f32=1, lambda_=0.95, eta=0.5)
+        im.im_set_option(p.g.ctx, im.IM_OPT_DECODE_TENSOR, tensor)
+        im.im_set_option(p.g.ctx, im.IM_OPT_READOUT_STAGES, stages)
+        p.prefill(0)
+        for s in range(wl.steps):
+            p.decode(s)
+        assert p.stats["max_out_err"] <= 1e-4 and p.stats["max_M_err"] <= 2e-3
+    # shapes the ring kernel does not take are refused
+    p = _pair(TINY.replace(name="ro_ring_refused", H=12, Hkv=3, ctx=32, chunk=32, B=16, steps=0))   # D_kv = 192
+    with pytest.raises(im.IndexMemError) as e:
+        im.im_set_option(p.g.ctx, im.IM_OPT_READOUT_STAGES, 2)
+    assert e.value.code == im.IM_ERR_ARG
