@@ -109,7 +109,8 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
 /* Releases the host object.  The workspace stays with the caller.  Synchronises the device. */
 int im_destroy(im_ctx* ctx);
 
-/* Clears the state of one sequence in one layer (layer = -1: all layers; seq = -1: all sequences). Enqueued on the stream. */
+/* Clears the state of one sequence in one layer (layer = -1: all layers; seq = -1: all sequences); with both -1 also the
+ * sticky device status word that im_status reports.  Enqueued on the stream. */
 int im_reset(im_ctx* ctx, int layer, int seq, void* cuda_stream);
 
 /*
@@ -254,6 +255,13 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        (k <= 6; D_kv a power of two of at most 1024 and d_M a multiple of 8192 / D_kv); 0 (default): by the
  *                        kernel built on plain loads, which serves every shape and schedule.  The two add the rows in different
  *                        orders (float32); both are within the stated tolerances.
+ *   IM_OPT_WAIT_LIMIT    (test aid) attempts of the bounded device-side waits in which a consumer waits for its copies to
+ *                        arrive (TMA / bulk-copy rings of the decode attention kernels, the bulk-copy readout kernel and
+ *                        the tcgen05 chunk attention kernel): 0 restores the default (2^22), k >= 1 allows k - 1 attempts,
+ *                        so 1 makes every such wait give up at once.  A wait that gives up sets the sticky status word
+ *                        (im_status then returns IM_ERR_TIMEOUT), the CTA still waits, with the full default limit, for
+ *                        the copies it has in flight, frees its tensor memory and returns; the outputs of that call are
+ *                        undefined, the context stays usable.
  */
 typedef enum im_option {
   IM_OPT_CONCURRENCY = 0,
@@ -261,7 +269,8 @@ typedef enum im_option {
   IM_OPT_PREFILL_TENSOR = 2,
   IM_OPT_PROFILE_TARGET = 3,
   IM_OPT_DECODE_TENSOR = 4,
-  IM_OPT_READOUT_STAGES = 5
+  IM_OPT_READOUT_STAGES = 5,
+  IM_OPT_WAIT_LIMIT = 6
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 

@@ -89,6 +89,7 @@ bool resolve(const im_config* in, im_config* c, ImDims* p) {
   q.max_splits = (q.cap + 255) / 256;
   q.scale = c->softmax_scale; q.lambda = c->lambda; q.eta = c->eta; q.eps = c->eps; q.norm_eps = c->norm_eps;
   if (q.Gq > 16) return false;
+  p->wait_limit = IM_WAIT_LIMIT;
   return true;
 }
 
@@ -473,6 +474,8 @@ int im_reset(im_ctx* ctx, int layer, int seq, void* cuda_stream) {
       ctx->hu[u] = HostUnit();
     }
   }
+  // a reset of everything also clears the sticky device status word
+  if (layer < 0 && seq < 0) CK(cudaMemsetAsync(ctx->lo.st.status, 0, 4, s));
   return IM_OK;
 }
 
@@ -931,6 +934,10 @@ int im_set_option(im_ctx* ctx, int option, int value) {
         return fail(IM_ERR_ARG, "the tensor-core decode attention kernel needs head_dim 128 and at most 8 query heads per KV head");
       ctx->attn_tc = value != 0;
       ctx->tail_is_merge = false;
+      return IM_OK;
+    case IM_OPT_WAIT_LIMIT:
+      if (value < 0) return fail(IM_ERR_ARG, "wait limit %d: 0 = default, k >= 1 = k - 1 attempts", value);
+      ctx->p.wait_limit = value == 0 ? IM_WAIT_LIMIT : (uint32_t)(value - 1);
       return IM_OK;
     case IM_OPT_READOUT_STAGES:
       if (value < 0 || value > 6) return fail(IM_ERR_ARG, "readout stages %d out of range [0,6]", value);

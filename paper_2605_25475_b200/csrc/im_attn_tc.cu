@@ -63,7 +63,7 @@ constexpr int OP_HALF = 8 * 128;             // one 64-element half of a B opera
 constexpr int Q_BYTES = 2 * OP_HALF;         // Q^T of one segment: rows = heads, 128 elements per row
 constexpr int P_BYTES = 2 * OP_HALF;         // one bf16 term of P^T of one tile: rows = heads, 128 keys per row
 constexpr int THREADS = 192;                 // warps 0-3 softmax, 4 TMA, 5 tensor memory / MMA issue
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = IM_WAIT_LIMIT;
 constexpr int TMEM_COLS = 64;                // S^T double buffered at 0 / 16, O^T at 32
 constexpr int S_COL = 0, O_COL = 32;
 
@@ -91,8 +91,8 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // bounded wait; gives up early when another role of the CTA has given up
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit = WAIT_LIMIT) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -498,7 +498,8 @@ k_attn_stream_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
         if (progressed) idle = 0;
         else {
-          if (++idle >= WAIT_LIMIT || ((idle & 63) == 0 && *abort_flag)) { ok = false; break; }  // (warp uniform)
+          if (idle >= p.wait_limit || ((idle & 63) == 63 && *abort_flag)) { ok = false; break; }  // (warp uniform)
+          ++idle;
           __nanosleep(40);  // this warp shares its scheduler with a softmax warp: do not spin at full rate
         }
       }
@@ -522,7 +523,7 @@ k_attn_stream_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       long long j = run0;
       bool fail = false;
       auto wait = [&](unsigned long long* bar, uint32_t parity) {
-        const bool got = mbar_wait(smem_u32(bar), parity, abort_flag);
+        const bool got = mbar_wait(smem_u32(bar), parity, abort_flag, p.wait_limit);
         if (!got) { fail = true; sh->abort = 1; }
         return got;
       };

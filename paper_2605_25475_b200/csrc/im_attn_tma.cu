@@ -26,7 +26,7 @@ constexpr int TILE = IM_ATTN_STREAM_TILE;  // keys per tile (48-key tiles with 6
                                            // in the full step: the readout kernel next to it then falls behind)
 constexpr int STAGES = 2;                // ring depth per warp
 constexpr int WARPS = IM_ATTN_WARPS;     // consumer warps per CTA (each also issues its own TMA)
-constexpr uint32_t WAIT_LIMIT = 1u << 22;  // try_wait attempts before a warp gives up and flags ST_TIMEOUT
+constexpr uint32_t WAIT_LIMIT = IM_WAIT_LIMIT;  // try_wait attempts before a warp gives up and flags ST_TIMEOUT
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -36,9 +36,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// bounded wait: returns false if the phase did not complete within the limit
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+// bounded wait: returns false if the phase did not complete within `limit` attempts
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = WAIT_LIMIT) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -226,7 +226,8 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     for (; tt < nt && j < run1; ++tt, ++j) {
       const int s = (int)((j - run0) % STAGES);
       const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
-      if (!mbar_wait(bar, (uint32_t)(((j - run0) / STAGES) & 1))) { ok = false; break; }
+      // (the outcome is made warp-uniform: the lanes poll on their own and could disagree at the limit)
+      if (!__all_sync(0xffffffffu, mbar_wait(bar, (uint32_t)(((j - run0) / STAGES) & 1), p.wait_limit))) { ok = false; break; }
       const uint32_t Ks = smem_u32(ring + (size_t)s * STAGE_BYTES), Vs = Ks + TILE_BYTES;
       // ---- S^T = K Q^T : [32 keys] x [8 heads]
       float sacc[TILE / 16][4];
@@ -346,7 +347,14 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
     }
   }
-  if (!ok && lane == 0) atomicOr(st.status, ST_TIMEOUT);
+  if (!ok && lane == 0) {
+    // The warp gives up.  The copies it has requested and not consumed (tiles j .. issued - 1) still write into this
+    // CTA's shared memory, which the SM hands to another CTA when this one ends: wait for each of them, with the full
+    // limit, before returning.
+    atomicOr(st.status, ST_TIMEOUT);
+    for (long long t2 = j; t2 < issued; ++t2)
+      mbar_wait(smem_u32(&bars[warp * STAGES + (int)((t2 - run0) % STAGES)]), (uint32_t)(((t2 - run0) / STAGES) & 1));
+  }
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -44,7 +44,7 @@ constexpr int STAGE_BYTES = 2 * KV_TILE;    // K + V
 constexpr int Q_BYTES = ROWS * DH * 2;      // 32 KB per Q tile: two halves of 128 rows x 128 bytes
 constexpr int QTILES = 2;                   // Q tiles (row groups of 128) per CTA
 constexpr int THREADS = 320;                // warps 0-7: softmax (two groups of four), 8: TMA, 9: tensor memory / MMA
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = IM_WAIT_LIMIT;
 constexpr int TMEM_COLS = 512;              // per Q tile g: S 64, P 2 terms x 32 (bf16 pairs), O 128
 constexpr int S_COL = 0;                    // S of tile g at S_COL + 64 g
 constexpr int P_COL = 128;                  // P of tile g, term t at P_COL + 64 g + 32 t
@@ -67,8 +67,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit = WAIT_LIMIT) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -276,7 +276,7 @@ k_chunk_attention_tc(const __grid_constant__ CUtensorMap tmK, const __grid_const
       const uint32_t qa = smem_u32(s_q);
       auto issue_s = [&](int j, int g) -> bool {  // S_g(j) = Q_g K_j^T
         const int s = j % STAGES;
-        if (g == 0 && !mbar_wait(smem_u32(&sh->full[s]), (uint32_t)((j / STAGES) & 1), abort_flag)) return false;
+        if (g == 0 && !mbar_wait(smem_u32(&sh->full[s]), (uint32_t)((j / STAGES) & 1), abort_flag, p.wait_limit)) return false;
         if (j >= 1 && !mbar_wait(smem_u32(&sh->sempty[g]), (uint32_t)((j - 1) & 1), abort_flag)) return false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t ka = smem_u32(s_kv + (size_t)s * STAGE_BYTES);

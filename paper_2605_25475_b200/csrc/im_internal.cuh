@@ -37,7 +37,10 @@ struct ImDims {
   int R3, R5;                 // projection rows: indexer only / indexer + memory
   int max_splits;             // attention splits per (sequence, KV head)
   float scale, lambda, eta, eps, norm_eps;
+  uint32_t wait_limit;        // attempts of a consumer's bounded wait for data to arrive (IM_OPT_WAIT_LIMIT; the waits for
+                              // a CTA's own copies to land before it ends always get the full IM_WAIT_LIMIT)
 };
+#define IM_WAIT_LIMIT (1u << 22)
 
 // projection row offsets inside one raw output vector
 struct ImRows {

@@ -25,7 +25,7 @@ constexpr int RO_CHUNK = 32 * 1024;          // bytes per stage
 constexpr int RO_CONSUMERS = 256;
 constexpr int RO_THREADS = RO_CONSUMERS + 32;
 constexpr int RO_MAX_STAGES = 6;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = IM_WAIT_LIMIT;
 
 struct RoShared {
   unsigned long long full[RO_MAX_STAGES], empty[RO_MAX_STAGES];
@@ -42,8 +42,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit = WAIT_LIMIT) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -137,7 +137,7 @@ k_readout_stream(ImDims p, ImState st, ImScratch sc, ImCall call, int stages) {
       for (; j < seq_end; ++j) {
         const long long k = j - run0;
         const int s = (int)(k % stages);
-        if (!fail && !mbar_wait(smem_u32(&sh->full[s]), (uint32_t)((k / stages) & 1), abort_flag)) {
+        if (!fail && !mbar_wait(smem_u32(&sh->full[s]), (uint32_t)((k / stages) & 1), abort_flag, p.wait_limit)) {
           fail = true;
           sh->abort = 1;
         }
