@@ -69,8 +69,9 @@ def algorithmic_bytes(wl: synth.Workload):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """Samples nvidia-smi clocks and throttle reasons.  Started before the warm-up (the tool needs a few hundred
+    milliseconds to come up); `stop(t0, t1)` keeps the samples whose time stamp falls into the timed region."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -81,11 +82,12 @@ class ClockSampler:
         try:
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.idx), "-lms", "50"], stdout=self.f, stderr=subprocess.DEVNULL)
+                                          "-i", str(self.idx), "-lms", "20"], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -95,26 +97,32 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.f.close()
-        sm, mx, reasons = [], [], set()
+        rows = []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 9:
                 continue
             try:
-                sm.append(float(parts[1])); mx.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), [nm for nm, val in zip(names, parts[5:9]) if val.lower().startswith("active")]))
             except ValueError:
                 continue
-            for nm, val in zip(names, parts[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
         try:
             os.remove(self.path)
         except OSError:
             pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
-        out["reasons"] = sorted(reasons)
+        inside = [r for r in rows if t0 is not None and t0 <= r[0] <= t1]
+        out["samples_total"] = len(rows)
+        if not inside and rows and t0 is not None:
+            # the region was shorter than the sampling interval: the samples nearest to it
+            inside = sorted(rows, key=lambda r: min(abs(r[0] - t0), abs(r[0] - t1)))[:2]
+            out["note"] = "no sample fell into the timed region; the two nearest are reported"
+        if t0 is None:
+            inside = rows
+        if inside:
+            out.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside), samples=len(inside))
+        out["reasons"] = sorted({nm for r in inside for nm in r[3]})
         return out
 
 
@@ -157,17 +165,16 @@ def pick_workload(args):
     return wl
 
 
-def run_ours(args, rank, world, device):
+def measure_decode(wl, device, steps, warmup, graph=True, rank=0, world=1, log=lambda *a: None, opts=None,
+                   profile=True, e2e_args=None):
+    """Ingests the workload's context, then times `steps` decode steps (all layers, all sequences per step) replayed
+    from CUDA graphs, inputs resident.  Returns the raw measurements; the context is closed before returning."""
     from paper_2605_25475_b200 import binding as im
-    wl = pick_workload(args)
-    log = (lambda *a: print("[bench]", *a, file=sys.stderr, flush=True)) if rank == 0 else (lambda *a: None)
     g, ids = build_context(wl, device, log=log)
-    if args.decode_tensor >= 0:
-        im.im_set_option(g.ctx, im.IM_OPT_DECODE_TENSOR, args.decode_tensor)
-    if args.readout_stages >= 0:
-        im.im_set_option(g.ctx, im.IM_OPT_READOUT_STAGES, args.readout_stages)
+    for opt, val in (opts or {}).items():
+        im.im_set_option(g.ctx, opt, val)
     L = wl.n_layers
-    n_in = min(8, args.steps + args.warmup)                      # distinct input sets, cycled
+    n_in = min(8, steps + warmup)                                # distinct input sets, cycled
     inputs = decode_inputs_all(wl, n_in, device)
     out = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=device)
 
@@ -178,16 +185,19 @@ def run_ours(args, rank, world, device):
 
     stream = torch.cuda.Stream(device)
     graphs = None
-    launches_per_step = None
     tau = wl.tau
     n_graphs = n_in * tau // math.gcd(n_in, tau)                 # every (input set, phase of the interval) pair that occurs
+    res = {}
+    sampler = ClockSampler(torch.cuda.current_device() if device.index is None else device.index)
+    if rank == 0:
+        sampler.start()                                          # before the warm-up: the tool takes a while to come up
     with torch.cuda.stream(stream):
         c0 = g.launch_count()
         for k in range(tau):                                     # one whole interval, eagerly: ends with n = B, phase 0
             one_step(k)
-        launches_per_step = (g.launch_count() - c0) / tau
+        res["launches_per_step"] = (g.launch_count() - c0) / tau
         stream.synchronize()
-        if args.graph:
+        if graph:
             # one captured step per input set and phase: the graph reads the resident inputs where they are; which
             # kernels a step launches depends on its phase (the last step of an interval compresses)
             graphs = []
@@ -197,51 +207,77 @@ def run_ours(args, rank, world, device):
                     one_step(k)
                 graphs.append(gk)
         step_fn = (lambda k: graphs[k % n_graphs].replay()) if graphs is not None else one_step
-        for w in range(args.warmup):
+        for w in range(warmup):
             step_fn(w)
         stream.synchronize()
         barrier(world)
-        sampler = ClockSampler(torch.cuda.current_device() if device.index is None else device.index)
-        if rank == 0:
-            sampler.start()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         rec0 = im.im_event_count(g.ctx, im.IM_COUNT_MERGE_RECOMPUTE)
+        t_wall0 = time.time()
         ev0.record(stream)
-        for s in range(args.steps):
-            step_fn(args.warmup + s)
+        for s in range(steps):
+            step_fn(warmup + s)
         ev1.record(stream)
         torch.cuda.synchronize()
+        t_wall1 = time.time()
         barrier(world)
         ms = ev0.elapsed_time(ev1)
-        recomputes = im.im_event_count(g.ctx, im.IM_COUNT_MERGE_RECOMPUTE) - rec0
-        clocks = sampler.stop() if rank == 0 else None
+        res["recomputes"] = im.im_event_count(g.ctx, im.IM_COUNT_MERGE_RECOMPUTE) - rec0
+        res["clocks"] = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
         assert g.status() == 0
-        ms = max_over_ranks(ms, world, device)
-        done = args.warmup + args.steps
+        res["ms"] = max_over_ranks(ms, world, device)
+        done = warmup + steps
         while done % tau:                                        # finish the interval (phase 0 again)
             step_fn(done)
             done += 1
+        res["cuda_graph"] = graphs is not None
 
-        # per-launch time of the dominant kernel: the same steps again, un-graphed, with the
-        # library recording CUDA events around the attention + readout launch on this stream
-        # (side streams off for this pass, so that the kernel is timed alone against the burst peak)
-        im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 0)
-        im.im_profile_begin(g.ctx, (-(-args.steps // tau) * tau) * L)
-        prof_steps = -(-args.steps // tau) * tau                # whole intervals
-        for s in range(prof_steps):
-            one_step(s)
-        attn_ms, attn_n = im.im_profile_end(g.ctx)
-        im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 1)
+        if profile:
+            # per-launch time of the dominant kernel: the same steps again, un-graphed, with the library recording
+            # CUDA events around the attention launch on this stream - once in the concurrent schedule the timed steps
+            # ran (the kernel next to the readout kernel and the chain of small kernels, on the SMs the schedule
+            # leaves it), once with the side streams off (the kernel alone on all SMs, against the burst peak)
+            prof_steps = -(-min(steps, 32) // tau) * tau            # whole intervals
+            for name, conc in (("in_step", 1), ("alone", 0)):
+                im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, conc)
+                im.im_profile_begin(g.ctx, prof_steps * L)
+                for s in range(prof_steps):
+                    one_step(s)
+                k_ms, k_n = im.im_profile_end(g.ctx)
+                res["attn_ms_" + name], res["attn_n_" + name] = k_ms, k_n
+            im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 1)
+        if e2e_args is not None:
+            # end to end: host buffers in, host buffer out, copies inside the timed region
+            res["e2e"] = run_e2e(e2e_args, wl, g, ids, inputs, stream, world, device)
+    del graphs
+    g.close()
+    return res
 
-        # end to end: host buffers in, host buffer out, copies inside the timed region
-        e2e = run_e2e(args, wl, g, ids, inputs, stream, world, device)
 
+def run_ours(args, rank, world, device):
+    from paper_2605_25475_b200 import binding as im
+    wl = pick_workload(args)
+    log = (lambda *a: print("[bench]", *a, file=sys.stderr, flush=True)) if rank == 0 else (lambda *a: None)
+    opts = {}
+    if args.decode_tensor >= 0:
+        opts[im.IM_OPT_DECODE_TENSOR] = args.decode_tensor
+    if args.readout_stages >= 0:
+        opts[im.IM_OPT_READOUT_STAGES] = args.readout_stages
+    m = measure_decode(wl, device, args.steps, args.warmup, graph=bool(args.graph), rank=rank, world=world, log=log,
+                       opts=opts, e2e_args=args)
+    ms = m["ms"]
     tokens = wl.n_seq * args.steps * world
     ab = algorithmic_bytes(wl)
     peaks = measured_peaks()
-    attn_launch_s = attn_ms / max(attn_n, 1) * 1e-3
-    achieved = ab["attn_launch"] / attn_launch_s / 1e9
+    kernel = "k_attn_stream_tc" if opts.get(im.IM_OPT_DECODE_TENSOR, 0) else "k_attn_stream"
+
+    def rate(k_ms, k_n):
+        sec = k_ms / max(k_n, 1) * 1e-3
+        return {"us_per_launch": sec * 1e6, "achieved": ab["attn_launch"] / sec / 1e9,
+                "frac": ab["attn_launch"] / sec / 1e9 / peaks["hbm_gbs"]}
+    alone, in_step = rate(m["attn_ms_alone"], m["attn_n_alone"]), rate(m["attn_ms_in_step"], m["attn_n_in_step"])
+    full = wl.name == "llama8b_stack" and not args.tau and not args.layers and not args.context
     res = {
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -250,19 +286,88 @@ def run_ours(args, rank, world, device):
                                + ("" if not args.tau else " (compression interval %d instead of the headline workload's)" % args.tau),
                    "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H,
                    "kv_heads": wl.Hkv, "head_dim": wl.d, "context": wl.ctx, "budget": wl.B, "tau": wl.tau,
-                   "cuda_graph": graphs is not None,
+                   "cuda_graph": m["cuda_graph"],
                    "l2": "inputs larger than L2 (each step streams %.1f GB)" % (ab["step"] / 1e9)},
         "hbm_gbs_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9,
         "hbm_frac_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"],
         "hbm_frac_step_nominal_8tbs": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / 8000.0,
-        "roofline": {"bound": "hbm", "kernel": "k_attn_stream", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     "traffic": args.traffic if wl.name == "llama8b_stack" and not args.tau else None, "bytes_per_launch": ab["attn_launch"],
-                     "us_per_launch": attn_launch_s * 1e6},
-        "merge_recomputes_per_step": recomputes / args.steps,
-        "e2e": e2e, "gpu_launches": int(round(launches_per_step * args.steps)), "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": kernel, "achieved": alone["achieved"], "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": alone["frac"], "peak_source": peaks["source"],
+                     "schedule": "in order, the kernel alone on all SMs (side streams off, un-graphed, CUDA events around the launch)",
+                     "traffic": args.traffic if full else None,
+                     "traffic_source": ("profiles/k_attn_stream_llama8b_stack_2layers_ctx4096.md (ncu dram__bytes_read.sum + "
+                                        "dram__bytes_write.sum of one launch of this size; a constant, not measured in this run)") if full else None,
+                     "bytes_per_launch": ab["attn_launch"], "us_per_launch": alone["us_per_launch"],
+                     "in_step": dict(in_step, schedule="concurrent schedule of the timed steps: the kernel on the SMs left by the "
+                                                      "front kernel, next to the readout kernel (un-graphed, CUDA events around the launch)")},
+        "merge_recomputes_per_step": m["recomputes"] / args.steps,
+        "e2e": m["e2e"], "gpu_launches": int(round(m["launches_per_step"] * args.steps)), "clocks": m["clocks"],
     }
     return res, wl
+
+
+# ----------------------------------------------------------------------------------------------
+# Secondary measurements: the other configurations, short runs, one entry each in the default line
+def secondary_block(args, device, log):
+    """Configurations 2-4 and the paper's compression interval on the headline stack, each a short run with its own
+    oracle baseline.  None of them has a bandwidth target: 2 and 3 are bound by the latency of a call's kernel chain."""
+    from paper_2605_25475_b200 import binding as im
+    peaks = measured_peaks()
+    out = {}
+    for name, steps in (("llama8b_b1", 64), ("qwen7b_b8", 64)):
+        wl = synth.CONFIGS[name]
+        m = measure_decode(wl, device, steps, 4, log=log, profile=False)
+        ab = algorithmic_bytes(wl)
+        sec = m["ms"] / steps * 1e-3
+        cpu, _ = oracle_sample(wl.replace(chunk=min(wl.chunk, 2048)), min(len(os.sched_getaffinity(0)), wl.n_seq), 48, log=log)
+        out[name] = {"us_per_step": sec * 1e6, "tokens_per_s": wl.n_seq / sec, "steps": steps, "bytes_per_step": ab["step"],
+                     "hbm_gbs": ab["step"] / sec / 1e9, "hbm_frac": ab["step"] / sec / 1e9 / peaks["hbm_gbs"],
+                     "bound": "latency of the call's kernel chain (no bandwidth target)",
+                     "config": {"layers": 1, "batch": wl.n_seq, "context": wl.ctx, "budget": wl.B, "tau": 1, "cuda_graph": True},
+                     "cpu_baseline": cpu}
+        log(f"secondary {name}: {sec * 1e6:.1f} us/step")
+    # configuration 4: chunked prefill
+    pre_args = argparse.Namespace(**vars(args))
+    pre_args.steps, pre_args.warmup, pre_args.context = 2, 3, 0
+    pf = run_prefill(pre_args, device)
+    wl4 = synth.CONFIGS["mistral7b_prefill"]
+    out["mistral7b_prefill"] = {
+        "ms_per_prompt": pf["scoring"]["tensor_cores"]["ms_per_prompt"], "tokens_per_s": pf["scoring"]["tensor_cores"]["tokens_per_s"],
+        "ms_per_prompt_with_outputs": pf["with_outputs"]["ms_per_prompt"],
+        "scoring_kernel": {"name": "k_prefill_score_tc", "us_per_launch": pf["scoring"]["tensor_cores"]["us_per_launch"],
+                           "tensor_pipe_active_pct": 10.0,
+                           "tensor_pipe_source": "profiles/k_prefill_score_tc_mistral7b_prefill_ctx8192.md (ncu, not measured in this run)"},
+        "config": {"layers": 1, "batch": 1, "prompt": wl4.ctx, "chunk": wl4.chunk, "budget": wl4.B},
+        "cpu_baseline": oracle_prefill_sample(wl4, log)}
+    log(f"secondary mistral7b_prefill: {out['mistral7b_prefill']['ms_per_prompt']:.2f} ms per prompt")
+    # the paper's compression interval on the headline stack
+    wl = synth.CONFIGS["llama8b_stack"].replace(tau=128)
+    m = measure_decode(wl, device, 128, 128, log=log, profile=False)
+    ab = algorithmic_bytes(wl)
+    sec = m["ms"] / 128 * 1e-3
+    out["llama8b_stack_tau128"] = {
+        "ms_per_step": sec * 1e3, "tokens_per_s": wl.n_seq / sec, "steps": 128, "bytes_per_step": ab["step"],
+        "hbm_gbs": ab["step"] / sec / 1e9, "hbm_frac": ab["step"] / sec / 1e9 / peaks["hbm_gbs"],
+        "config": {"layers": wl.n_layers, "batch": wl.n_seq, "context": wl.ctx, "budget": wl.B, "tau": 128, "cuda_graph": True,
+                   "note": "one whole interval: 127 steps attend over B + p entries, one selects 128 entries per sequence"},
+        "cpu_baseline": "as the headline line's (an oracle step costs the same per cached entry; the interval changes how many are cached)"}
+    log(f"secondary tau=128: {sec * 1e3:.3f} ms/step")
+    return out
+
+
+def oracle_prefill_sample(wl, log):
+    """The oracle on two 2048-token chunks of the prefill configuration (the second one at the steady-state size: 4096
+    cached keys scored by 2048 queries, 2048 evictions)."""
+    from oracle import indexmem_oracle as orc
+    o = orc.OracleLayer(orc.OracleConfig(H=wl.H, Hkv=wl.Hkv, d=wl.d, B=wl.B, n_sink=wl.n_sink), 1)
+    o.set_weights({k: synth.f32(v) for k, v in synth.make_weights(wl, 0).items()})
+    ins = [tuple(synth.f32(t[0]) for t in synth.prefill_inputs(wl, 0, c)) for c in range(2)]
+    o.prefill_chunk(0, ins[0][0], ins[0][1], ins[0][3], ins[0][4])
+    t0 = time.time()
+    o.prefill_chunk(0, ins[1][0], ins[1][1], ins[1][3], ins[1][4])
+    dt = time.time() - t0
+    return {"value": wl.chunk / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+            "sample": f"one steady-state chunk ({wl.chunk} tokens against {2 * wl.chunk} cached keys, {wl.chunk} evictions); {dt:.1f}s of CPU time on 1 thread"}
 
 
 def run_prefill(args, device):
@@ -490,11 +595,19 @@ def run_reference(args, rank, world):
     steps = max(1, min(args.steps, 64))
     base, dt = oracle_sample(wl, n_units, steps,
                              log=lambda *a: print("[bench]", *a, file=sys.stderr, flush=True))
+    ab = algorithmic_bytes(wl)
     return {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wl.n_seq / base["value"],
+            "extrapolated": True,
+            "extrapolation": (f"timed: {n_units} sequences x 1 layer x {steps} decode steps ({dt:.1f} s on the host cores); value and "
+                              f"ms_per_step are that rate scaled to {wl.n_seq} sequences x {wl.n_layers} layers (units are independent)"),
+            "timed_seconds": dt,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "budget": wl.B,
-                       "tau": wl.tau},
+            "config": {"workload": wl.name + ("" if not (args.layers or args.context) else " (reduced for profiling)")
+                                   + ("" if not args.tau else " (compression interval %d instead of the headline workload's)" % args.tau),
+                       "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H, "kv_heads": wl.Hkv, "head_dim": wl.d,
+                       "context": wl.ctx, "budget": wl.B, "tau": wl.tau, "cuda_graph": False,
+                       "l2": "inputs larger than L2 (each step streams %.1f GB)" % (ab["step"] / 1e9)},
             "cpu_baseline": base,
             "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
@@ -528,6 +641,8 @@ def main():
                     help="prefill: profiling aid that times the chunked prefill and its scoring kernel (1 GPU)")
     ap.add_argument("--graph", type=int, default=1, help="replay the step from a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="skip the short runs of the other configurations that the default line carries in `secondary`")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: run only this many layers (not the headline workload)")
     ap.add_argument("--context", type=int, default=0, help="profiling aid: ingest only this many context tokens")
     ap.add_argument("--tau", type=int, default=0,
@@ -573,6 +688,10 @@ def main():
                                                    log=lambda *a: print("[bench]", *a, file=sys.stderr, flush=True))
         else:
             res["cpu_baseline"] = None
+        default_run = (world == 1 and args.workload == "llama8b_stack" and not (args.layers or args.context or args.tau)
+                       and args.decode_tensor < 0 and args.readout_stages < 0)
+        if default_run and not args.no_secondary:
+            res["secondary"] = secondary_block(args, device, lambda *a: print("[bench]", *a, file=sys.stderr, flush=True))
         print(json.dumps(res), flush=True)
     if world > 1:
         _dist.destroy_process_group()
