@@ -299,6 +299,54 @@ void append(const Layer& L, Seq& S, const float* x, const float* k, const float*
   S.T += 1;
 }
 
+// App. B "From Running Mean to IndexCache": a layer that reuses the indexer scores of a neighbouring layer computes
+// no indexer features of its own; its cached entries carry no indexer key.
+void append_without_index(const Layer& L, Seq& S, const float* k, const float* v) {
+  Entry e;
+  e.pos = (int32_t)S.T;
+  e.k.assign(k, k + L.Dkv);
+  e.v.assign(v, v + L.Dkv);
+  e.kidx.assign(L.c.dI, 0.f);
+  e.acc = -std::numeric_limits<float>::infinity();
+  S.R.push_back(std::move(e));
+  S.T += 1;
+}
+
+// App. B: "compute the indexer scores once within a short group of neighbouring layers and reuse the resulting
+// scores ... for the remaining layers in the group".  The scores reused are the pooled importances the leading
+// layer's latest compression chose among, matched by token position.  Returns false if the leading layer has no
+// score for one of this layer's entries (the two layers must have seen the same tokens and made the same calls).
+bool adopt_scores(Seq& S, const Seq& lead) {
+  for (Entry& e : S.R) {
+    bool found = false;
+    for (size_t i = 0; i < lead.sel_pos.size(); ++i)
+      if (lead.sel_pos[i] == e.pos) {
+        e.acc = lead.sel_acc[i];
+        found = true;
+        break;
+      }
+    if (!found) return false;
+  }
+  return true;
+}
+
+// Eq. 4-5 for one query: attention over the retained set plus the gated memory readout
+void layer_output(const Layer& L, const Seq& S, const float* q, int64_t max_pos, float* out_bf16, double* out_f64) {
+  const int D = L.D;
+  std::vector<double> o(D), m(D, 0.0);
+  attention(L, S, q, o.data(), max_pos);
+  double gate = 0.0;
+  if (L.c.enable_memory) {
+    mem_read(L, S, q, m.data());
+    gate = gate_of(L, q);
+  }
+  for (int j = 0; j < D; ++j) {
+    const double val = o[j] + gate * m[j];
+    if (out_f64) out_f64[j] = val;
+    if (out_bf16) out_bf16[j] = (float)bf16_round(val);
+  }
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------ C API
@@ -428,6 +476,44 @@ int orc_decode_step(void* h, int seq, const float* x, const float* q_pre, const 
       if (out_f64) out_f64[j * d + c] = val;
       if (out_bf16) out_bf16[j * d + c] = (float)bf16_round(val);
     }
+  return 0;
+}
+
+// The two calls for a layer that reuses the indexer scores of the leading layer of its group (App. B, IndexCache-style
+// reuse; the paper reuses scores "across every four consecutive layers").  `lead` / `lead_seq`: the leading layer's
+// handle and sequence, which must already have made the same call for the same tokens.  The layer appends its own
+// K / V, adopts the leading layer's pooled importances when a compression is due, and does everything else - selection
+// under its own budget and sinks, memory write from its own evicted pairs (Eq. 6-7), attention over its own retained
+// entries and readout of its own memory (Eq. 4-5) - as any layer does.  Returns -1 if the leading layer's scores do
+// not cover this layer's entries.
+int orc_decode_step_follow(void* h, int seq, void* lead, int lead_seq, const float* q, const float* k_new,
+                           const float* v_new, float* out_bf16, double* out_f64) {
+  Layer* L = static_cast<Layer*>(h);
+  Seq& S = L->seqs[seq];
+  const Seq& LS = static_cast<Layer*>(lead)->seqs[lead_seq];
+  append_without_index(*L, S, k_new, v_new);
+  S.since += 1;
+  if (S.since == L->c.tau) {
+    if (!adopt_scores(S, LS)) return -1;
+    compress(*L, S);
+  }
+  layer_output(*L, S, q, std::numeric_limits<int64_t>::max(), out_bf16, out_f64);
+  return 0;
+}
+int orc_prefill_chunk_follow(void* h, int seq, void* lead, int lead_seq, int C, const float* Q /*[C,H,d] or null*/,
+                             const float* K, const float* V, float* out_bf16, double* out_f64) {
+  Layer* L = static_cast<Layer*>(h);
+  Seq& S = L->seqs[seq];
+  const Seq& LS = static_cast<Layer*>(lead)->seqs[lead_seq];
+  const int D = L->D, Dkv = L->Dkv;
+  const int64_t T0 = S.T;
+  for (int c = 0; c < C; ++c) append_without_index(*L, S, K + (size_t)c * Dkv, V + (size_t)c * Dkv);
+  if (Q && (out_bf16 || out_f64))
+    for (int c = 0; c < C; ++c)
+      layer_output(*L, S, Q + (size_t)c * D, T0 + c, out_bf16 ? out_bf16 + (size_t)c * D : nullptr,
+                   out_f64 ? out_f64 + (size_t)c * D : nullptr);
+  if (!adopt_scores(S, LS)) return -1;
+  compress(*L, S);
   return 0;
 }
 

@@ -94,6 +94,8 @@ def _load():
     L.orc_prefill_batch.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, vp, vp]
     L.orc_prefill_chunk_out.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp, vp]
     L.orc_prefill_batch_out.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, vp, vp, vp, vp, vp]
+    L.orc_decode_step_follow.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, vp, vp, vp]
+    L.orc_prefill_chunk_follow.argtypes = [vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp, vp, vp]
     L.orc_count.argtypes = [vp, C.c_int]
     L.orc_tokens_seen.argtypes = [vp, C.c_int]
     L.orc_tokens_seen.restype = i64
@@ -215,6 +217,34 @@ class OracleLayer:
         ob = np.empty((n, self.cfg.H, self.cfg.d), np.float32)
         od = np.empty((n, self.cfg.H, self.cfg.d), np.float64)
         self.lib.orc_decode_batch(self.h, n, _p(ids), _p(x), _p(q_pre), _p(q), _p(k_new), _p(v_new), _p(ob), _p(od))
+        return ob, od
+
+    # ---- a layer that reuses the indexer scores of the leading layer of its group (App. B, IndexCache-style reuse)
+    def decode_step_follow(self, seq: int, lead: "OracleLayer", lead_seq: int, q, k_new, v_new):
+        """decode_step for a layer that adopts `lead`'s pooled importances (matched by token position) instead of
+        scoring with an indexer of its own; `lead` must already have made the call for the same token."""
+        q, k_new, v_new = _f32(q), _f32(k_new), _f32(v_new)
+        assert q.size == self.D and k_new.size == self.Dkv and v_new.size == self.Dkv
+        ob = np.empty((self.cfg.H, self.cfg.d), np.float32)
+        od = np.empty((self.cfg.H, self.cfg.d), np.float64)
+        rc = self.lib.orc_decode_step_follow(self.h, seq, lead.h, lead_seq, _p(q), _p(k_new), _p(v_new), _p(ob), _p(od))
+        assert rc == 0, "the leading layer's scores do not cover this layer's entries"
+        return ob, od
+
+    def prefill_chunk_follow(self, seq: int, lead: "OracleLayer", lead_seq: int, K, V, Q=None):
+        """prefill_chunk for such a layer; with Q [C,H,d] also returns the layer outputs of the chunk's own queries."""
+        K, V = _f32(K), _f32(V)
+        Cn = K.size // self.Dkv
+        assert K.size == Cn * self.Dkv and V.size == K.size
+        ob = od = None
+        if Q is not None:
+            Q = _f32(Q)
+            assert Q.size == Cn * self.D
+            ob = np.empty((Cn, self.cfg.H, self.cfg.d), dtype=np.float32)
+            od = np.empty((Cn, self.cfg.H, self.cfg.d), dtype=np.float64)
+        rc = self.lib.orc_prefill_chunk_follow(self.h, seq, lead.h, lead_seq, Cn, _p(Q) if Q is not None else None, _p(K), _p(V),
+                                               _p(ob) if ob is not None else None, _p(od) if od is not None else None)
+        assert rc == 0, "the leading layer's scores do not cover this layer's entries"
         return ob, od
 
     # ---- state

@@ -546,3 +546,98 @@ def test_single_token_chunk_output_equals_decode_output_when_nothing_is_evicted(
         _, oa = La.prefill_chunk_out(0, X[t:t + 1], Q[t:t + 1], Q[t:t + 1], K[t:t + 1], V[t:t + 1])
         _, ob = Lb.decode_step(0, X[t], Q[t], Q[t], K[t], V[t])
         np.testing.assert_allclose(oa[0], ob, rtol=1e-13, atol=1e-14)
+
+
+# ------------------------------------------------------------------ score reuse across neighbouring layers (App. B)
+def _leader_and_follower(rng, same=False, **kw):
+    lead = orc.OracleLayer(small_cfg(**kw))
+    foll = orc.OracleLayer(small_cfg(**kw))
+    wl = rand_weights(lead, rng)
+    if same:
+        foll.set_weights(wl)
+        wf = wl
+    else:
+        wf = rand_weights(foll, rng)
+    return lead, foll, wl, wf
+
+
+def test_score_reuse_follower_keeps_the_leaders_positions_and_attends_to_its_own_cache():
+    """IndexCache-style reuse: the following layer makes the leading layer's decisions (same retained positions
+    after every call) but everything it computes comes from its own keys, values and queries: with the memory
+    disabled its output is the textbook softmax attention over its own K / V at the positions the leader kept."""
+    rng = np.random.default_rng(21)
+    lead, foll, _, _ = _leader_and_follower(rng, B=9, tau=3, n_sink=2, enable_memory=0)
+    n0, steps = 14, 13
+    X, Q, K, V = rand_tokens(lead, rng, n0 + steps)
+    _, Q2, K2, V2 = rand_tokens(foll, rng, n0 + steps)
+    lead.prefill_chunk(0, X[:n0], Q[:n0], K[:n0], V[:n0])
+    foll.prefill_chunk_follow(0, lead, 0, K2[:n0], V2[:n0])
+    assert foll.positions().tolist() == lead.positions().tolist() and len(lead.positions()) == 9
+    for s in range(n0, n0 + steps):
+        lead.decode_step(0, X[s], Q[s].reshape(-1), Q[s], K[s], V[s])
+        _, od = foll.decode_step_follow(0, lead, 0, Q2[s], K2[s], V2[s])
+        pos = lead.positions()
+        assert foll.positions().tolist() == pos.tolist()
+        assert foll.since() == lead.since() and foll.evict_steps() == lead.evict_steps()
+        want = softmax_attention(Q2[s], K2[pos], V2[pos], foll.Gq, foll.cfg.scale)
+        np.testing.assert_allclose(od, want, rtol=1e-11, atol=1e-13)
+        # the follower's cache holds its OWN rows at those positions
+        e = foll.entries()
+        assert np.array_equal(e["K"], K2[pos]) and np.array_equal(e["V"], V2[pos])
+    assert lead.evict_steps() == 1 + steps // 3
+
+
+def test_score_reuse_follower_writes_its_own_evicted_pairs_to_its_own_memory():
+    """lambda = 1: the follower's (M, b) is the sum over every position evicted so far of phi(k) v^T / phi(k)^2 formed
+    with the follower's weights, keys and values - the leader decides which positions, nothing else."""
+    rng = np.random.default_rng(22)
+    lead, foll, _, wf = _leader_and_follower(rng, B=7, tau=1, n_sink=1)
+    n = 22
+    X, Q, K, V = rand_tokens(lead, rng, n)
+    _, Q2, K2, V2 = rand_tokens(foll, rng, n)
+    lead.prefill_chunk(0, X[:10], Q[:10], K[:10], V[:10])
+    foll.prefill_chunk_follow(0, lead, 0, K2[:10], V2[:10])
+    for s in range(10, n):
+        lead.decode_step(0, X[s], Q[s].reshape(-1), Q[s], K[s], V[s])
+        foll.decode_step_follow(0, lead, 0, Q2[s], K2[s], V2[s])
+    gone = sorted(set(range(n)) - set(lead.positions().tolist()))
+    assert len(gone) == n - 7
+    Wt = wf["W_theta"].astype(np.float64)
+    Phi = model_space(K2[gone], foll.Gq).astype(np.float64) @ Wt.T
+    M, b = foll.memory()
+    np.testing.assert_allclose(M, Phi.T @ model_space(V2[gone], foll.Gq).astype(np.float64), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(b, (Phi ** 2).sum(axis=0), rtol=1e-10, atol=1e-12)
+    Ml, _ = lead.memory()
+    assert not np.allclose(M, Ml)
+
+
+def test_score_reuse_follower_with_the_leaders_inputs_reproduces_the_leader():
+    """A follower given the leader's weights, keys, values and queries is the leader: outputs, cache and memory agree
+    to the last bit (reusing the scores changes who computes them, not what is selected), also for the layer outputs
+    of a prefill chunk's own queries."""
+    rng = np.random.default_rng(23)
+    lead, foll, _, _ = _leader_and_follower(rng, same=True, B=8, tau=2, n_sink=2, lambda_=0.9, eta=0.5)
+    X, Q, K, V = rand_tokens(lead, rng, 30)
+    for c in range(2):
+        sl = slice(6 * c, 6 * c + 6)
+        _, od_l = lead.prefill_chunk_out(0, X[sl], Q[sl], Q[sl], K[sl], V[sl])
+        _, od_f = foll.prefill_chunk_follow(0, lead, 0, K[sl], V[sl], Q=Q[sl])
+        assert np.array_equal(od_l, od_f)
+    for s in range(12, 30):
+        _, od_l = lead.decode_step(0, X[s], Q[s].reshape(-1), Q[s], K[s], V[s])
+        _, od_f = foll.decode_step_follow(0, lead, 0, Q[s], K[s], V[s])
+        assert np.array_equal(od_l, od_f)
+    for a, b in zip(lead.memory(), foll.memory()):
+        assert np.array_equal(a, b)
+    el, ef = lead.entries(), foll.entries()
+    assert np.array_equal(el["pos"], ef["pos"]) and np.array_equal(el["K"], ef["K"]) and np.array_equal(el["V"], ef["V"])
+
+
+def test_score_reuse_needs_the_leaders_call_first():
+    rng = np.random.default_rng(24)
+    lead, foll, _, _ = _leader_and_follower(rng, B=5, tau=1)
+    X, Q, K, V = rand_tokens(lead, rng, 8)
+    lead.prefill_chunk(0, X[:7], Q[:7], K[:7], V[:7])
+    foll.prefill_chunk_follow(0, lead, 0, K[:7], V[:7])
+    with pytest.raises(AssertionError):            # the leader has not seen token 7 yet
+        foll.decode_step_follow(0, lead, 0, Q[7], K[7], V[7])
