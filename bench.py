@@ -127,11 +127,11 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------
-def build_context(wl: synth.Workload, device, ingest=True, log=lambda *a: None, chunk_outputs=0):
+def build_context(wl: synth.Workload, device, ingest=True, log=lambda *a: None, chunk_outputs=0, score_share=0):
     from paper_2605_25475_b200 import binding as im
     g = im.IndexMem(im.Config(n_layers=wl.n_layers, max_seqs=wl.n_seq, n_q_heads=wl.H, n_kv_heads=wl.Hkv,
                               head_dim=wl.d, budget=wl.B, compress_interval=wl.tau, max_chunk=wl.chunk,
-                              n_sink=wl.n_sink, chunk_outputs=chunk_outputs), device)
+                              n_sink=wl.n_sink, chunk_outputs=chunk_outputs, score_share=score_share), device)
     ids = list(range(wl.n_seq))
     for layer in range(wl.n_layers):
         g.set_weights(layer, {k: v.cpu() for k, v in synth.make_weights(wl, layer, device).items()})
@@ -166,11 +166,11 @@ def pick_workload(args):
 
 
 def measure_decode(wl, device, steps, warmup, graph=True, rank=0, world=1, log=lambda *a: None, opts=None,
-                   profile=True, e2e_args=None):
+                   profile=True, e2e_args=None, score_share=0):
     """Ingests the workload's context, then times `steps` decode steps (all layers, all sequences per step) replayed
     from CUDA graphs, inputs resident.  Returns the raw measurements; the context is closed before returning."""
     from paper_2605_25475_b200 import binding as im
-    g, ids = build_context(wl, device, log=log)
+    g, ids = build_context(wl, device, log=log, score_share=score_share)
     for opt, val in (opts or {}).items():
         im.im_set_option(g.ctx, opt, val)
     L = wl.n_layers
@@ -265,7 +265,7 @@ def run_ours(args, rank, world, device):
     if args.readout_stages >= 0:
         opts[im.IM_OPT_READOUT_STAGES] = args.readout_stages
     m = measure_decode(wl, device, args.steps, args.warmup, graph=bool(args.graph), rank=rank, world=world, log=log,
-                       opts=opts, e2e_args=args)
+                       opts=opts, e2e_args=args, score_share=args.score_share)
     ms = m["ms"]
     tokens = wl.n_seq * args.steps * world
     ab = algorithmic_bytes(wl)
@@ -286,7 +286,7 @@ def run_ours(args, rank, world, device):
                                + ("" if not args.tau else " (compression interval %d instead of the headline workload's)" % args.tau),
                    "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H,
                    "kv_heads": wl.Hkv, "head_dim": wl.d, "context": wl.ctx, "budget": wl.B, "tau": wl.tau,
-                   "cuda_graph": m["cuda_graph"],
+                   "cuda_graph": m["cuda_graph"], "score_share": args.score_share,
                    "l2": "inputs larger than L2 (each step streams %.1f GB)" % (ab["step"] / 1e9)},
         "hbm_gbs_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9,
         "hbm_frac_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -352,6 +352,16 @@ def secondary_block(args, device, log):
                    "note": "one whole interval: 127 steps attend over B + p entries, one selects 128 entries per sequence"},
         "cpu_baseline": "as the headline line's (an oracle step costs the same per cached entry; the interval changes how many are cached)"}
     log(f"secondary tau=128: {sec * 1e3:.3f} ms/step")
+    # reuse of one layer's indexer scores by the three layers that follow it (App. B of the paper)
+    wl = synth.CONFIGS["llama8b_stack"]
+    m = measure_decode(wl, device, 64, 4, log=log, profile=False, score_share=4)
+    sec = m["ms"] / 64 * 1e-3
+    out["llama8b_stack_score_share4"] = {
+        "ms_per_step": sec * 1e3, "tokens_per_s": wl.n_seq / sec, "steps": 64,
+        "config": {"layers": wl.n_layers, "batch": wl.n_seq, "context": wl.ctx, "budget": wl.B, "tau": 1, "cuda_graph": True,
+                   "score_share": 4,
+                   "note": "layers 4k+1 .. 4k+3 make layer 4k's selection: no indexer projections, keys or scoring in 24 of 32 layers"}}
+    log(f"secondary score_share=4: {sec * 1e3:.3f} ms/step")
     return out
 
 
@@ -650,6 +660,8 @@ def main():
                          "one CUDA graph per phase of the interval is captured")
     ap.add_argument("--decode-tensor", type=int, default=-1,
                     help="1 / 0: decode attention on the tcgen05 kernel / the mma.sync kernel (default: the library's choice)")
+    ap.add_argument("--score-share", type=int, default=0,
+                    help="g >= 2: layers l with l %% g != 0 reuse the indexer scores of layer l - l %% g (the paper's appendix uses 4)")
     ap.add_argument("--readout-stages", type=int, default=-1,
                     help="0: readout on plain loads; k >= 1: on a ring of k 32 KB bulk copies per CTA (default: the library's choice)")
     ap.add_argument("--traffic", type=float, default=ATTN_TRAFFIC_NCU,
@@ -689,7 +701,7 @@ def main():
         else:
             res["cpu_baseline"] = None
         default_run = (world == 1 and args.workload == "llama8b_stack" and not (args.layers or args.context or args.tau)
-                       and args.decode_tensor < 0 and args.readout_stages < 0)
+                       and args.decode_tensor < 0 and args.readout_stages < 0 and not args.score_share)
         if default_run and not args.no_secondary:
             res["secondary"] = secondary_block(args, device, lambda *a: print("[bench]", *a, file=sys.stderr, flush=True))
         print(json.dumps(res), flush=True)

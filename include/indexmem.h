@@ -61,6 +61,8 @@ typedef struct im_config {
   int32_t out_f32;           /* 0: `out` of im_decode_step is bf16; 1: float32                       */
   int32_t pending_slots;     /* rank-one writes folded lazily into M (0 => 16); see im_decode_step  */
   int32_t chunk_outputs;     /* 1: reserve workspace for im_prefill_chunk_attend (max_seqs * max_chunk * D_kv floats) */
+  int32_t score_share;       /* g >= 2: layers l with l % g != 0 reuse the indexer scores of layer l - l % g (App. B,
+                                IndexCache-style reuse; the paper uses 4); 0 or 1: every layer scores for itself      */
   float softmax_scale;       /* 0 => 1/sqrt(d)                                 (Sec. 2.1)           */
   float lambda;              /* decay of Eq. 6-7, (0,1]; 0 => 1                                      */
   float eta;                 /* write strength of Eq. 6-7, > 0; 0 => 1                               */

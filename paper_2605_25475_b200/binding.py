@@ -34,7 +34,7 @@ WEIGHT_IDS = {"U_q": IM_W_UQ, "U_k": IM_W_UK, "G": IM_W_G, "W_theta": IM_W_THETA
 class im_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "max_seqs", "n_q_heads", "n_kv_heads", "head_dim", "n_index_heads", "index_dim", "mem_dim",
-        "budget", "compress_interval", "max_chunk", "n_sink", "act", "enable_memory", "out_f32", "pending_slots", "chunk_outputs")] + \
+        "budget", "compress_interval", "max_chunk", "n_sink", "act", "enable_memory", "out_f32", "pending_slots", "chunk_outputs", "score_share")] + \
         [(n, C.c_float) for n in ("softmax_scale", "lambda_", "eta", "eps", "norm_eps", "init_std")] + \
         [("seed", C.c_uint64)]
 
@@ -244,6 +244,7 @@ class Config:
     out_f32: int = 0
     pending_slots: int = 0
     chunk_outputs: int = 0
+    score_share: int = 0
     softmax_scale: float = 0.0
     lambda_: float = 0.0
     eta: float = 0.0

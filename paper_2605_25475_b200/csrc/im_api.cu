@@ -84,6 +84,8 @@ bool resolve(const im_config* in, im_config* c, ImDims* p) {
   q.n_sink = c->n_sink; q.act = c->act; q.mem = c->enable_memory ? 1 : 0; q.F = c->pending_slots;
   q.out_f32 = c->out_f32 ? 1 : 0; q.max_chunk = std::max(c->max_chunk, 1);
   q.chunk_out = c->chunk_outputs ? 1 : 0;
+  if (c->score_share < 0 || c->score_share > c->n_layers) return false;
+  q.share = c->score_share >= 2 ? c->score_share : 0;
   q.R3 = q.HI * q.dI + q.dI + q.HI;
   q.R5 = q.R3 + q.dM + 1;
   q.max_splits = (q.cap + 255) / 256;
@@ -252,6 +254,7 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
   }
   call->layer = layer;
   call->n_seq = n_seq;
+  call->lead = (ctx->p.share >= 2 && layer % ctx->p.share) ? layer - layer % ctx->p.share : -1;
   call->C = 1;
   call->pack = 0;
   call->defer = 0;
@@ -505,13 +508,22 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
     n_max = std::max(n_max, u.n + chunk_len);
     ne_max = std::max(ne_max, u.n + chunk_len - p.B);
   }
+  const bool follow = call.lead >= 0;
+  if (follow)  // the leading layer of the group must already have ingested this chunk
+    for (int i = 0; i < n_seq; ++i) {
+      const HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+      const HostUnit& ul = ctx->hu[(size_t)call.lead * p.S + call.seq[i]];
+      if (ul.T != u.T + chunk_len || ul.n != std::min(u.n + chunk_len, p.B))
+        return fail(IM_ERR_STATE, "layer %d reuses the scores of layer %d, which has to make this call first (sequence %d)",
+                    layer, call.lead, call.seq[i]);
+    }
   call.C = chunk_len;
   call.prefill = 1;
   call.due = 1;
   call.ksplit = 1;
   call.ksplit_key = 1;
   call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
-  call.pack = ctx->score_tc ? 1 : 0;
+  call.pack = (ctx->score_tc && !follow) ? 1 : 0;
   call.fold_all = attend && p.mem ? 1 : 0;
   ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
   const int NV = n_seq * chunk_len;
@@ -558,11 +570,13 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
       CK(cudaStreamWaitEvent(Lw.stream, ctx->ev[0], 0));
     }
   }
-  g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
-  CKL(im_launch_gemm(L, g));
-  g.job[0] = {L.w.G, nullptr, p.HI, r.g, 1};
-  CKL(im_launch_gemm(Lg, g));
-  CKL(im_launch_proj_key_split(Lk, x, NV, 1));
+  if (!follow) {  // (a layer that reuses another layer's scores has no indexer work)
+    g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
+    CKL(im_launch_gemm(L, g));
+    g.job[0] = {L.w.G, nullptr, p.HI, r.g, 1};
+    CKL(im_launch_gemm(Lg, g));
+    CKL(im_launch_proj_key_split(Lk, x, NV, 1));
+  }
   if (memside) {
     // phi(q) and the gate logit of every chunk token (behind the indexer-side block of the projection scratch)
     ImGemmArgs g2;
@@ -620,7 +634,8 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   {
     const bool prof = ctx->prof_target == 1 && ctx->prof_used + 2 <= ctx->prof_ev.size();
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], L.stream));
-    if (call.pack) CKL(im_launch_prefill_score_tc(L, call, n_max, ctx->n_sm));
+    if (follow) {}  // the scores come from the leading layer, after the commit below
+    else if (call.pack) CKL(im_launch_prefill_score_tc(L, call, n_max, ctx->n_sm));
     else CKL(im_launch_prefill_score(L, call, n_max));
     if (prof) {
       CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], L.stream));
@@ -628,6 +643,7 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
     }
   }
   CKL(im_launch_prefill_commit(L, call));
+  if (follow) CKL(im_launch_follow_scores(L, call));
   // a2: selection (also restarts the pooling); a4: gather the evicted pairs, fill the holes
   CKL(im_launch_select(L, call));
   if (ne_max > 0) {
@@ -696,6 +712,16 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     return fail(IM_ERR_ARG, "sequences of one decode call must be at the same phase of the compression interval");
   const bool due = due_all;
   if (!due) ne_max = 0;
+  const bool follow = call.lead >= 0;
+  if (follow)  // the leading layer of the group must already have taken this token
+    for (int i = 0; i < n_seq; ++i) {
+      const HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+      const HostUnit& ul = ctx->hu[(size_t)call.lead * p.S + call.seq[i]];
+      const int n_after = due ? std::min(u.n + 1, p.B) : u.n + 1;
+      if (ul.T != u.T + 1 || ul.n != n_after)
+        return fail(IM_ERR_STATE, "layer %d reuses the scores of layer %d, which has to make this call first (sequence %d)",
+                    layer, call.lead, call.seq[i]);
+    }
   call.due = due ? 1 : 0;
   call.C = 1;
   call.prefill = 0;
@@ -750,7 +776,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CKL(im_launch_mem_fold(L4, call));
     if (conc) CK(cudaEventRecord(ctx->ev[7], L4.stream));
   }
-  CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
+  if (!follow) CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
   if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // key projection done
   // a0: projections as K-split partial sums: indexer part (Sec. 3.1 features) on s1 ...
   ImRows r = im_rows(p);
@@ -772,7 +798,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
   g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
   g.n_jobs = 2;
-  CKL(im_launch_gemm(L1, g));
+  if (!follow) CKL(im_launch_gemm(L1, g));  // (a layer that reuses another layer's scores has no indexer work)
   // ... memory part (phi(q) of Eq. 5, gate logit of Eq. 4) on s2, followed by the readout
   if (p.mem) {
     g.job[0] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
@@ -1227,7 +1253,9 @@ int im_status(im_ctx* ctx, void* cuda_stream, int32_t* device_status) {
   CK(cudaStreamSynchronize((cudaStream_t)cuda_stream));
   CK(cudaMemcpy(device_status, ctx->lo.st.status, 4, cudaMemcpyDeviceToHost));
   if (*device_status & ST_TIMEOUT) return fail(IM_ERR_TIMEOUT, "a bounded device wait gave up (status %d)", *device_status);
-  if (*device_status) return fail(IM_ERR_STATE, "device status %d (1: non-finite score, 2: count mismatch)", *device_status);
+  if (*device_status)
+    return fail(IM_ERR_STATE, "device status %d (1: non-finite score, 2: count mismatch, 8: a layer that reuses another layer's scores holds other positions than that layer)",
+                *device_status);
   return IM_OK;
 }
 

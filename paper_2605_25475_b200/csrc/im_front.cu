@@ -39,6 +39,10 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   const int dI = DI > 0 ? DI : p.dI;
   float* imp = st.imp + u * p.cap;
   int32_t* pos = st.pos + u * p.cap;
+  // A layer that reuses the scores of the leading layer of its group (App. B) computes no indexer features and caches
+  // no indexer key: the pooled importances are those the leading layer's selection saw in this step, slot by slot.
+  const bool follow = call.lead >= 0;
+  const size_t ul = follow ? (size_t)call.lead * p.S + call.seq[i] : u;
   // ---- issue the loads of the first batch of cached entries (they depend on nothing of this call)
   constexpr int EPT = 4;
   int n_lim = p.cap;  // entries a batch may read: the capacity until the count is known
@@ -52,12 +56,12 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
       imp_old[e] = NEG_INF;
       pos_old[e] = 0;
       if (t < n_lim) {  // (entries at or beyond the count are read but never used; slot n is the token being appended)
-        if (DI > 0) {
+        if (DI > 0 && !follow) {
           const uint4* row = reinterpret_cast<const uint4*>(st.kidx + (u * p.cap + t) * dI);
 #pragma unroll
           for (int c = 0; c < (DI > 0 ? DI / 8 : 1); ++c) kraw[e][c] = row[c];
         }
-        imp_old[e] = imp[t];
+        imp_old[e] = follow ? NEG_INF : imp[t];
         pos_old[e] = pos[t];
       }
     }
@@ -80,27 +84,29 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     vnew_c = reinterpret_cast<const uint4*>(v_new + (size_t)i * p.Dkv + h * p.d)[c];
   }
   // ---- finish the projections: sum the K-split partials in a fixed order
-  for (int k = tid; k < nq; k += FRONT_THREADS) {
-    s_q[k] = im_raw_sum(p, sc, call, i, r.uq + k);
-  }
-  for (int k = tid; k < p.HI; k += FRONT_THREADS) {
-    sh.alpha[k] = im_raw_sum(p, sc, call, i, r.g + k) * (1.0f / sqrtf((float)p.HI * (float)p.dI));
-  }
-  for (int k = tid; k < p.dI; k += FRONT_THREADS) {
-    double s = 0.0;
-    for (int ks = 0; ks < call.ksplit_key; ++ks) s += sc.keyp[((size_t)ks * call.n_seq + i) * p.dI + k];
-    sh.kd[k] = s;
+  if (!follow) {
+    for (int k = tid; k < nq; k += FRONT_THREADS) {
+      s_q[k] = im_raw_sum(p, sc, call, i, r.uq + k);
+    }
+    for (int k = tid; k < p.HI; k += FRONT_THREADS) {
+      sh.alpha[k] = im_raw_sum(p, sc, call, i, r.g + k) * (1.0f / sqrtf((float)p.HI * (float)p.dI));
+    }
+    for (int k = tid; k < p.dI; k += FRONT_THREADS) {
+      double s = 0.0;
+      for (int ks = 0; ks < call.ksplit_key; ++ks) s += sc.keyp[((size_t)ks * call.n_seq + i) * p.dI + k];
+      sh.kd[k] = s;
+    }
   }
   __syncthreads();
   // RMSNorm of the q features per indexer head (float32) and of the key (float64, then bf16)
-  for (int h = tid; h < p.HI; h += FRONT_THREADS) {
+  for (int h = tid; h < (follow ? 0 : p.HI); h += FRONT_THREADS) {
     float* y = s_q + h * p.dI;
     float ms = 0.f;
     for (int k = 0; k < p.dI; ++k) ms = fmaf(y[k], y[k], ms);
     const float inv = 1.0f / sqrtf(ms / (float)p.dI + p.norm_eps);
     for (int k = 0; k < p.dI; ++k) y[k] *= inv;
   }
-  if (tid >= 64 && tid < 64 + p.dI) {
+  if (!follow && tid >= 64 && tid < 64 + p.dI) {
     const int k = tid - 64;
     double ms = 0.0;
     for (int j = 0; j < p.dI; ++j) ms += sh.kd[j] * sh.kd[j];
@@ -130,13 +136,30 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   const int n1 = n + 1;
   const bool due = (since + 1 == p.tau);
   const bool select_here = do_select && due;
-  bool bad = false;
+  bool bad = false, layout_bad = false;
   for (int b0 = 0; b0 < n1; b0 += EPT * FRONT_THREADS) {
     if (b0 > 0) load_batch(b0);
 #pragma unroll
     for (int e = 0; e < EPT; ++e) {
       const int t = b0 + e * FRONT_THREADS + tid;
       if (t >= n1) continue;
+      if (follow) {
+        // the leading layer scored the same entries in the same slots (checked: same position in the same slot)
+        const int ps = (t == n) ? T : pos_old[e];
+        if (due) {
+          const float pooled = st.sel_imp[ul * p.cap + t];
+          if (st.sel_pos[ul * p.cap + t] != ps) layout_bad = true;
+          st.sel_pos[u * p.cap + t] = ps;
+          st.sel_imp[u * p.cap + t] = pooled;
+          if (select_here) {
+            s_key[t] = im_select_key(pooled, ps, p.n_sink);
+            imp[t] = NEG_INF;
+          } else {
+            imp[t] = pooled;
+          }
+        }
+        continue;
+      }
       float kk[DI > 0 ? DI : 64];
       if (t == n) {
 #pragma unroll
@@ -179,6 +202,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     }
   }
   if (bad) atomicOr(st.status, ST_NONFINITE);
+  if (layout_bad) atomicOr(st.status, ST_LAYOUT);
   if (!select_here) {
     // either not due, or the selection runs in the kernels that follow (they read imp / pos)
     if (tid == 0) {

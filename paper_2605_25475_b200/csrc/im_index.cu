@@ -51,9 +51,10 @@ __global__ void k_prefill_append(ImDims p, ImState st, ImScratch sc, ImCall call
   if (tid == 0 && c == 0) st.ctr[u * CTR_STRIDE + CTR_NNEXT] = n;
   const ImRows r = im_rows(p);
   float* raw = sc.raw + ((size_t)i * call.C + c) * p.R3;
-  if (tid < 32) finalize_features(p, raw, tid);
+  const bool follow = call.lead >= 0;  // the layer reuses another layer's scores: no indexer features, no indexer key
+  if (tid < 32 && !follow) finalize_features(p, raw, tid);
   __syncthreads();
-  if (call.pack) {
+  if (call.pack && !follow) {
     // operand record of the tensor-core scoring: the token's features as three bf16 terms (their sum is the
     // float32 value to 2^-24), each 16-byte row (8 features of one head slot) at its place in the
     // shared-memory layout of a K-major operand without swizzle; alpha follows the three terms
@@ -86,7 +87,7 @@ __global__ void k_prefill_append(ImDims p, ImState st, ImScratch sc, ImCall call
   const int slot = n + c;
   bf16* kid = st.kidx + (u * p.cap + slot) * p.dI;
   // k = bf16(RMSNorm(U_k x)) from the float64 projection (one K split in prefill)
-  if (tid >= 32 && tid < 32 + p.dI) {
+  if (!follow && tid >= 32 && tid < 32 + p.dI) {
     const double* ud = sc.keyp + ((size_t)i * call.C + c) * p.dI;
     double ms = 0.0;
     for (int j = 0; j < p.dI; ++j) ms += ud[j] * ud[j];
@@ -187,6 +188,23 @@ __global__ void k_prefill_commit(ImDims p, ImState st, ImCall call) {
     ctr[CTR_T] = ctr[CTR_T] + call.C;
     ctr[CTR_NEVICT] = 0;
   }
+}
+
+// A layer that reuses the scores of the leading layer of its group (App. B, IndexCache-style reuse): its pooled
+// importances are those the leading layer's latest selection saw, slot by slot.  The two layers have made the same
+// calls, so their slot layouts agree; the kernel checks it position by position (ST_LAYOUT otherwise).
+// grid = n_seq, block = 256; after k_prefill_commit (CTR_N counts the appended chunk).
+__global__ void k_follow_scores(ImDims p, ImState st, ImCall call) {
+  const size_t u = (size_t)call.layer * p.S + call.seq[blockIdx.x];
+  const size_t ul = (size_t)call.lead * p.S + call.seq[blockIdx.x];
+  const int n = st.ctr[u * CTR_STRIDE + CTR_N];
+  if (n < 0 || n > p.cap) return;  // flagged elsewhere
+  bool bad = n != st.ctr[ul * CTR_STRIDE + CTR_NSEL];
+  for (int t = threadIdx.x; t < n && !bad; t += blockDim.x) {
+    bad |= st.sel_pos[ul * p.cap + t] != st.pos[u * p.cap + t];
+    st.imp[u * p.cap + t] = st.sel_imp[ul * p.cap + t];
+  }
+  if (bad) atomicOr(st.status, ST_LAYOUT);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -458,6 +476,12 @@ cudaError_t im_launch_prefill_score(const ImLaunch& L, const ImCall& call, int n
   dim3 grid((n_max + 31) / 32, call.n_seq);
   const size_t smem = ((size_t)PS_QT * (L.p.HI * L.p.dI + L.p.HI) + 256) * 4;
   k_prefill_score<<<grid, 256, smem, L.stream>>>(L.p, L.st, L.sc, call);
+  ++*L.launches;
+  return cudaGetLastError();
+}
+
+cudaError_t im_launch_follow_scores(const ImLaunch& L, const ImCall& call) {
+  k_follow_scores<<<call.n_seq, 256, 0, L.stream>>>(L.p, L.st, call);
   ++*L.launches;
   return cudaGetLastError();
 }

@@ -26,7 +26,7 @@ enum { CTR_N = 0, CTR_T = 1, CTR_SINCE = 2, CTR_EVSTEPS = 3, CTR_NEVICT = 4, CTR
 // count from before the call until the call's last kernel (the attention and merge kernels read it).
 
 // device status bits (sticky)
-enum { ST_NONFINITE = 1, ST_COUNT = 2, ST_TIMEOUT = 4 };
+enum { ST_NONFINITE = 1, ST_COUNT = 2, ST_TIMEOUT = 4, ST_LAYOUT = 8 };
 
 struct ImDims {
   int L, S;                   // layers, sequences per layer
@@ -34,6 +34,7 @@ struct ImDims {
   int HI, dI, dM;             // indexer / memory widths
   int B, tau, cap, tail;      // budget, interval, slots per sequence, tail = cap - B
   int n_sink, act, mem, F, out_f32, max_chunk, chunk_out;
+  int share;                  // >= 2: layers l with l % share != 0 reuse the scores of layer l - l % share
   int R3, R5;                 // projection rows: indexer only / indexer + memory
   int max_splits;             // attention splits per (sequence, KV head)
   float scale, lambda, eta, eps, norm_eps;
@@ -132,6 +133,8 @@ struct ImCall {
   int pack;       // prefill: 1 = the append kernel also writes the operand records of the tensor-core scoring
   int phi_large;  // 1: phi of the evicted keys lives in ImScratch::phi, 0: in the K-split partials phip
   int ksplit, ksplit_key, ksplit_phi;  // K splits of the projections / key projection / phi partials of this call
+  int lead;       // >= 0: the layer whose pooled importances this call's layer reuses instead of scoring with an
+                  // indexer of its own (App. B); that layer has already made this call for the same sequences
   int seq[IM_MAX_CALL_SEQS];
 };
 
@@ -260,6 +263,9 @@ bool im_score_tc_supported(const ImDims& p);
 cudaError_t im_score_tc_prepare();
 cudaError_t im_launch_prefill_score_tc(const ImLaunch& L, const ImCall& call, int n_max, int n_sm);
 cudaError_t im_launch_prefill_commit(const ImLaunch& L, const ImCall& call);
+// a layer that reuses another layer's scores: copy the pooled importances that layer's selection saw (slot by slot; the
+// two layers' slot layouts agree, which the kernel checks position by position)
+cudaError_t im_launch_follow_scores(const ImLaunch& L, const ImCall& call);
 // layer outputs of a prefill chunk's own queries
 cudaError_t im_chunk_attn_prepare(const ImDims& p);
 cudaError_t im_launch_chunk_readout(const ImLaunch& L, const ImCall& call);

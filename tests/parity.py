@@ -173,12 +173,13 @@ class Pair:
 
 
 # ---------------------------------------------------------------------- one (layer, sequence) unit against its oracle
-def check_unit_state(g, layer: int, seq: int, o, oseq: int, stats: dict) -> bool:
+def check_unit_state(g, layer: int, seq: int, o, oseq: int, stats: dict, indexer: bool = True) -> bool:
     """State of library unit (layer, seq) against sequence ``oseq`` of oracle ``o``: counters, retained
     positions, cached indexer keys, pooled scores, K/V copies, M and b.  A divergence the parity rules
     allow (a selection decided inside the 1e-5 cut gap, an isolated one-ulp flip of a cached indexer key) is
     counted in ``stats`` and the unit re-synchronised from the oracle; the function then returns False (the
-    outputs of the step just made are not comparable).  Anything else fails."""
+    outputs of the step just made are not comparable).  Anything else fails.  indexer = False: the unit belongs to a
+    layer that reuses another layer's scores and keeps no indexer keys or pooled scores of its own."""
     e = o.entries(oseq)
     cnt = g.counts(layer, seq)
     assert cnt["n"] == len(e["pos"]), f"unit {(layer, seq)}: {cnt['n']} entries vs oracle {len(e['pos'])}"
@@ -192,7 +193,7 @@ def check_unit_state(g, layer: int, seq: int, o, oseq: int, stats: dict) -> bool
         stats["cut_divergences"] = stats.get("cut_divergences", 0) + 1
         resync = True
     else:
-        gk = g.export(layer, seq, im.IM_S_KIDX)[order]
+        gk = g.export(layer, seq, im.IM_S_KIDX)[order] if indexer else e["kidx"]
         diff = gk != e["kidx"]
         if diff.any():
             ulp = bf16_ulp(e["kidx"].astype(np.float64))
@@ -200,8 +201,8 @@ def check_unit_state(g, layer: int, seq: int, o, oseq: int, stats: dict) -> bool
             assert diff.sum() <= max(2, diff.size // 1000), f"unit {(layer, seq)}: {diff.sum()} kidx flips"
             stats["kidx_flips"] = stats.get("kidx_flips", 0) + int(diff.sum())
             resync = True
-        gimp = g.export(layer, seq, im.IM_S_IMP)[order]
-        if not resync:
+        if not resync and indexer:
+            gimp = g.export(layer, seq, im.IM_S_IMP)[order]
             check_scores(gimp, e["acc"], f"unit {(layer, seq)}", stats)
         # K / V are copies: bit-exact
         assert np.array_equal(g.export(layer, seq, im.IM_S_K)[order], e["K"]), f"unit {(layer, seq)}: K cache differs"
