@@ -19,11 +19,17 @@
 // brute-force top-B on tiny inputs; order invariance of (M,b) at lambda = 1;
 // identity activation closed form; alpha == 0 tie case; single-pair rank-one
 // closed form; lambda^j decay; the 19.92M indexer parameter count of the
-// efficiency paragraph.
+// efficiency paragraph; score reuse by a following layer (App. B): the leader's
+// positions, a numpy attention over the follower's own cache, the clone
+// identity; per-KV-head retained sets (Sec. 2.2): brute-force Knorm selection
+// per head, the assembled memory write against numpy, and the reduction to
+// the shared-row path when every head is handed the same scores.
 // Parity unpinned (no value in the paper fixes them): the memory widths under
 // GQA (the printed 0.52M parameter count matches no stated width), act = ReLU,
 // RMSNorm epsilon, the scalar sigmoid form of the gate g(q), softmax scale
-// 1/sqrt(d_head), sinks counted inside the budget.
+// 1/sqrt(d_head), sinks counted inside the budget, and - with a retained set per
+// KV head - how the slices a token loses in one evict step enter the memory
+// (assembled into one model-space pair, zeros at the heads that keep the token).
 //
 // One handle = one layer.  Sequences inside a handle are independent.
 
@@ -44,7 +50,8 @@ struct Cfg {
   int32_t n_sink;             // always-kept first tokens                 (Sec. 4 setup)
   int32_t act;                // 0 ReLU, 1 identity
   int32_t enable_memory;      // 0: no write, readout contributes nothing
-  int32_t pad_;
+  int32_t scorer;             // 0: the learnable indexer (one score row per sequence, Sec. 3.1); per-KV-head retained sets
+                              // (Sec. 2.2 framework, S in R^{B x H_kv x L}): 1 Knorm S_t = ||K_t||_2, 2 scores given by the caller
   double scale;               // softmax scale
   double lambda, eta, eps, norm_eps;
 };
@@ -76,8 +83,18 @@ struct Entry {
   float acc;                   // pooled importance since the last compression
 };
 
+struct HEntry {                // one KV head's slice of a cached token (per-KV-head retained sets)
+  int32_t pos;
+  std::vector<float> k, v;     // [d] each (bf16 values)
+  float score;                 // importance of the token for this head
+};
+
 struct Seq {
   std::vector<Entry> R;
+  std::vector<std::vector<HEntry>> RH;           // per-KV-head mode: [Hkv] lists, ascending position
+  std::vector<std::vector<int32_t>> h_evicted;   // [Hkv] positions evicted by the latest COMPRESS, ascending
+  std::vector<std::vector<int32_t>> h_sel_pos;   // [Hkv] what the latest COMPRESS chose among ...
+  std::vector<std::vector<float>> h_sel_score;   // ... and the scores it saw
   std::vector<double> M;       // [dM x D]  model space, Eq. 6
   std::vector<double> b;       // [dM]      Eq. 7
   int64_t T = 0;               // tokens appended so far (next position)
@@ -330,6 +347,161 @@ bool adopt_scores(Seq& S, const Seq& lead) {
   return true;
 }
 
+// ---------------------------------------------------------------- per-KV-head retained sets (Sec. 2.2)
+// Sec. 2.2 states eviction as S = f(.) in R^{B x H_kv x L}, I = TopK(S, L'), [K', V'] = Gather(K, V, I): every KV head keeps
+// its own set of token positions.  Two scorers with a head axis: Knorm (S_t = ||K_t||_2, Sec. 2.2) and scores handed in
+// by the caller (the memory module on top of another eviction policy, Sec. 5 ablation "SnapKV+Memory").
+
+// Knorm, Sec. 2.2: the key's magnitude for this head, kept as float32
+float knorm_score(const float* k, int d) {
+  double s = 0.0;
+  for (int c = 0; c < d; ++c) s += (double)k[c] * (double)k[c];
+  return (float)std::sqrt(s);
+}
+
+void ph_init(const Layer& L, Seq& S) {
+  if ((int)S.RH.size() != L.c.Hkv) {
+    S.RH.assign(L.c.Hkv, {});
+    S.h_evicted.assign(L.c.Hkv, {});
+    S.h_sel_pos.assign(L.c.Hkv, {});
+    S.h_sel_score.assign(L.c.Hkv, {});
+  }
+}
+
+void ph_append(const Layer& L, Seq& S, const float* k /*[Hkv,d]*/, const float* v) {
+  ph_init(L, S);
+  const int d = L.c.d;
+  for (int h = 0; h < L.c.Hkv; ++h) {
+    HEntry e;
+    e.pos = (int32_t)S.T;
+    e.k.assign(k + (size_t)h * d, k + (size_t)(h + 1) * d);
+    e.v.assign(v + (size_t)h * d, v + (size_t)(h + 1) * d);
+    e.score = L.c.scorer == 1 ? knorm_score(e.k.data(), d) : -std::numeric_limits<float>::infinity();
+    S.RH[h].push_back(std::move(e));
+  }
+  S.T += 1;
+}
+
+// Eq. 6-7 over model-space pairs (k~_i, v~_i)
+void mem_write_model(const Layer& L, Seq& S, const std::vector<std::vector<double>>& ku, const std::vector<std::vector<double>>& vu) {
+  const int dM = L.c.dM, D = L.D;
+  std::vector<double> sumM((size_t)dM * D, 0.0), sumb(dM, 0.0), phi(dM);
+  for (size_t i = 0; i < ku.size(); ++i) {
+    phi_of(L, ku[i].data(), phi.data());
+    for (int m = 0; m < dM; ++m) {
+      const double p = phi[m];
+      double* row = &sumM[(size_t)m * D];
+      for (int c = 0; c < D; ++c) row[c] += p * vu[i][c];
+      sumb[m] += p * p;
+    }
+  }
+  for (size_t i = 0; i < S.M.size(); ++i) S.M[i] = L.c.lambda * S.M[i] + L.c.eta * sumM[i];
+  for (int m = 0; m < dM; ++m) S.b[m] = L.c.lambda * S.b[m] + L.c.eta * sumb[m];
+}
+
+// Compression with a set of retained positions per KV head.  ext: scores handed in by the caller, [Hkv][n_pos] indexed
+// by token position (scorer 2), else null.  The memory write of this evict step (Alg. 1: "evicted_v is summed across
+// heads per token"): for every token that loses at least one head slice in this step, the evicted slices are assembled
+// into ONE model-space key and value - the slice of KV head g at the places of its query heads, zeros at the heads
+// that keep the token - and written as one pair of Eq. 6-7.
+bool ph_compress(const Layer& L, Seq& S, const float* ext, int64_t n_pos) {
+  const int Hkv = L.c.Hkv, d = L.c.d;
+  S.since = 0;
+  std::vector<std::vector<uint8_t>> keep(Hkv);
+  bool any = false;
+  for (int h = 0; h < Hkv; ++h) {
+    std::vector<HEntry>& R = S.RH[h];
+    const int n = (int)R.size();
+    if (L.c.scorer == 2) {
+      if (!ext) return false;
+      for (HEntry& e : R) {
+        if (e.pos >= n_pos) return false;
+        e.score = ext[(size_t)h * n_pos + e.pos];
+      }
+    }
+    S.h_evicted[h].clear();
+    S.h_sel_pos[h].resize(n);
+    S.h_sel_score[h].resize(n);
+    std::vector<float> sc(n);
+    std::vector<int32_t> ps(n);
+    for (int i = 0; i < n; ++i) { S.h_sel_pos[h][i] = ps[i] = R[i].pos; S.h_sel_score[h][i] = sc[i] = R[i].score; }
+    keep[h].assign(n, 1);
+    if (n > L.c.B) {
+      select_top_b(sc.data(), ps.data(), n, L.c.B, L.c.n_sink, keep[h].data());
+      any = true;
+    }
+  }
+  if (any) {
+    // tokens that lose a slice, ascending position, with the heads that evict them
+    std::vector<int32_t> toks;
+    for (int h = 0; h < Hkv; ++h)
+      for (size_t i = 0; i < S.RH[h].size(); ++i)
+        if (!keep[h][i]) { toks.push_back(S.RH[h][i].pos); S.h_evicted[h].push_back(S.RH[h][i].pos); }
+    std::sort(toks.begin(), toks.end());
+    toks.erase(std::unique(toks.begin(), toks.end()), toks.end());
+    if (L.c.enable_memory) {
+      std::vector<std::vector<double>> ku(toks.size(), std::vector<double>(L.D, 0.0)), vu(toks.size(), std::vector<double>(L.D, 0.0));
+      for (int h = 0; h < Hkv; ++h)
+        for (size_t i = 0; i < S.RH[h].size(); ++i) {
+          if (keep[h][i]) continue;
+          const HEntry& e = S.RH[h][i];
+          const size_t r = std::lower_bound(toks.begin(), toks.end(), e.pos) - toks.begin();
+          for (int j = h * L.Gq; j < (h + 1) * L.Gq; ++j)       // the query heads that read KV head h
+            for (int c = 0; c < d; ++c) { ku[r][(size_t)j * d + c] = (double)e.k[c]; vu[r][(size_t)j * d + c] = (double)e.v[c]; }
+        }
+      mem_write_model(L, S, ku, vu);
+    }
+    for (int h = 0; h < Hkv; ++h) {
+      std::vector<HEntry> kept;
+      for (size_t i = 0; i < S.RH[h].size(); ++i) if (keep[h][i]) kept.push_back(std::move(S.RH[h][i]));
+      S.RH[h].swap(kept);
+    }
+    S.n_evict_steps++;
+  }
+  return true;
+}
+
+// Sec. 2.1 attention with every KV head's own retained set
+void ph_attention(const Layer& L, const Seq& S, const float* q /*[H,d]*/, double* o /*[H,d]*/, int64_t max_pos) {
+  const int d = L.c.d;
+  for (int j = 0; j < L.c.H; ++j) {
+    const std::vector<HEntry>& R = S.RH[j / L.Gq];
+    size_t n = 0;
+    while (n < R.size() && (int64_t)R[n].pos <= max_pos) ++n;
+    std::vector<double> logit(n);
+    double mx = -std::numeric_limits<double>::infinity();
+    for (size_t t = 0; t < n; ++t) {
+      double s = 0.0;
+      for (int c = 0; c < d; ++c) s += (double)q[j * d + c] * (double)R[t].k[c];
+      logit[t] = s * L.c.scale;
+      mx = std::max(mx, logit[t]);
+    }
+    double den = 0.0;
+    for (size_t t = 0; t < n; ++t) { logit[t] = std::exp(logit[t] - mx); den += logit[t]; }
+    for (int c = 0; c < d; ++c) o[j * d + c] = 0.0;
+    for (size_t t = 0; t < n; ++t) {
+      const double p = logit[t] / den;
+      for (int c = 0; c < d; ++c) o[j * d + c] += p * (double)R[t].v[c];
+    }
+  }
+}
+
+void ph_layer_output(const Layer& L, const Seq& S, const float* q, int64_t max_pos, float* out_bf16, double* out_f64) {
+  const int D = L.D;
+  std::vector<double> o(D), m(D, 0.0);
+  ph_attention(L, S, q, o.data(), max_pos);
+  double gate = 0.0;
+  if (L.c.enable_memory) {
+    mem_read(L, S, q, m.data());
+    gate = gate_of(L, q);
+  }
+  for (int j = 0; j < D; ++j) {
+    const double val = o[j] + gate * m[j];
+    if (out_f64) out_f64[j] = val;
+    if (out_bf16) out_bf16[j] = (float)bf16_round(val);
+  }
+}
+
 // Eq. 4-5 for one query: attention over the retained set plus the gated memory readout
 void layer_output(const Layer& L, const Seq& S, const float* q, int64_t max_pos, float* out_bf16, double* out_f64) {
   const int D = L.D;
@@ -353,7 +525,7 @@ void layer_output(const Layer& L, const Seq& S, const float* q, int64_t max_pos,
 extern "C" {
 
 struct orc_config {          // mirrors Cfg; kept separate so the ABI is explicit
-  int32_t H, Hkv, d, HI, dI, dM, B, tau, n_sink, act, enable_memory, pad_;
+  int32_t H, Hkv, d, HI, dI, dM, B, tau, n_sink, act, enable_memory, scorer;
   double scale, lambda, eta, eps, norm_eps;
 };
 
@@ -515,6 +687,62 @@ int orc_prefill_chunk_follow(void* h, int seq, void* lead, int lead_seq, int C, 
   if (!adopt_scores(S, LS)) return -1;
   compress(*L, S);
   return 0;
+}
+
+// The two calls with a retained set per KV head (configuration scorer = 1 Knorm, 2 scores from the caller).  ext: float32
+// [Hkv][n_pos], the importance of token position p for KV head h at ext[h * n_pos + p]; it must cover every position
+// cached after the call's append (scorer 2; ignored by Knorm).  Returns -1 if scores are missing.
+int orc_ph_decode_step(void* h, int seq, const float* q, const float* k_new, const float* v_new, const float* ext,
+                       int64_t n_pos, float* out_bf16, double* out_f64) {
+  Layer* L = static_cast<Layer*>(h);
+  Seq& S = L->seqs[seq];
+  ph_append(*L, S, k_new, v_new);
+  S.since += 1;
+  if (S.since == L->c.tau && !ph_compress(*L, S, ext, n_pos)) return -1;
+  ph_layer_output(*L, S, q, std::numeric_limits<int64_t>::max(), out_bf16, out_f64);
+  return 0;
+}
+int orc_ph_prefill_chunk(void* h, int seq, int C, const float* Q /*[C,H,d] or null*/, const float* K, const float* V,
+                         const float* ext, int64_t n_pos, float* out_bf16, double* out_f64) {
+  Layer* L = static_cast<Layer*>(h);
+  Seq& S = L->seqs[seq];
+  const int D = L->D, Dkv = L->Dkv;
+  const int64_t T0 = S.T;
+  for (int c = 0; c < C; ++c) ph_append(*L, S, K + (size_t)c * Dkv, V + (size_t)c * Dkv);
+  if (Q && (out_bf16 || out_f64))
+    for (int c = 0; c < C; ++c)
+      ph_layer_output(*L, S, Q + (size_t)c * D, T0 + c, out_bf16 ? out_bf16 + (size_t)c * D : nullptr,
+                      out_f64 ? out_f64 + (size_t)c * D : nullptr);
+  return ph_compress(*L, S, ext, n_pos) ? 0 : -1;
+}
+int orc_ph_count(void* h, int seq, int head) {
+  Seq& S = static_cast<Layer*>(h)->seqs[seq];
+  return head < (int)S.RH.size() ? (int)S.RH[head].size() : 0;
+}
+void orc_ph_export(void* h, int seq, int head, int32_t* pos, float* score, float* K, float* V) {
+  Layer* L = static_cast<Layer*>(h);
+  const std::vector<HEntry>& R = L->seqs[seq].RH[head];
+  const int d = L->c.d;
+  for (size_t i = 0; i < R.size(); ++i) {
+    if (pos) pos[i] = R[i].pos;
+    if (score) score[i] = R[i].score;
+    if (K) std::memcpy(K + i * d, R[i].k.data(), sizeof(float) * d);
+    if (V) std::memcpy(V + i * d, R[i].v.data(), sizeof(float) * d);
+  }
+}
+int orc_ph_last_evicted(void* h, int seq, int head, int32_t* pos, int cap) {
+  const std::vector<int32_t>& e = static_cast<Layer*>(h)->seqs[seq].h_evicted[head];
+  if (pos) for (size_t i = 0; i < e.size() && (int)i < cap; ++i) pos[i] = e[i];
+  return (int)e.size();
+}
+int orc_ph_last_selection(void* h, int seq, int head, int32_t* pos, float* score, int cap) {
+  const Seq& S = static_cast<Layer*>(h)->seqs[seq];
+  const int n = (int)S.h_sel_pos[head].size();
+  for (int i = 0; i < n && i < cap; ++i) {
+    if (pos) pos[i] = S.h_sel_pos[head][i];
+    if (score) score[i] = S.h_sel_score[head][i];
+  }
+  return n;
 }
 
 // The same two calls over several independent sequences (one OpenMP thread per sequence).

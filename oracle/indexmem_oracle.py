@@ -33,7 +33,7 @@ def build(force: bool = False) -> str:
 
 class _Cfg(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
-                ("H", "Hkv", "d", "HI", "dI", "dM", "B", "tau", "n_sink", "act", "enable_memory", "pad_")] + \
+                ("H", "Hkv", "d", "HI", "dI", "dM", "B", "tau", "n_sink", "act", "enable_memory", "scorer")] + \
                [(n, C.c_double) for n in ("scale", "lambda_", "eta", "eps", "norm_eps")]
 
 
@@ -55,6 +55,7 @@ class OracleConfig:
     n_sink: int = 4
     act: int = 0
     enable_memory: int = 1
+    scorer: int = 0          # 0 the learnable indexer; retained sets per KV head: 1 Knorm (Sec. 2.2), 2 scores from the caller
     scale: float = 0.0
     lambda_: float = 1.0
     eta: float = 1.0
@@ -96,6 +97,12 @@ def _load():
     L.orc_prefill_batch_out.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, vp, vp, vp, vp, vp]
     L.orc_decode_step_follow.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, vp, vp, vp]
     L.orc_prefill_chunk_follow.argtypes = [vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp, vp, vp]
+    L.orc_ph_decode_step.argtypes = [vp, C.c_int, vp, vp, vp, vp, i64, vp, vp]
+    L.orc_ph_prefill_chunk.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, vp, i64, vp, vp]
+    L.orc_ph_count.argtypes = [vp, C.c_int, C.c_int]
+    L.orc_ph_export.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, vp]
+    L.orc_ph_last_evicted.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int]
+    L.orc_ph_last_selection.argtypes = [vp, C.c_int, C.c_int, vp, vp, C.c_int]
     L.orc_count.argtypes = [vp, C.c_int]
     L.orc_tokens_seen.argtypes = [vp, C.c_int]
     L.orc_tokens_seen.restype = i64
@@ -140,7 +147,7 @@ class OracleLayer:
         c = self.cfg
         assert c.H % c.Hkv == 0
         self.D, self.Dkv, self.Gq = c.H * c.d, c.Hkv * c.d, c.H // c.Hkv
-        raw = _Cfg(c.H, c.Hkv, c.d, c.HI, c.dI, c.dM, c.B, c.tau, c.n_sink, c.act, c.enable_memory, 0,
+        raw = _Cfg(c.H, c.Hkv, c.d, c.HI, c.dI, c.dM, c.B, c.tau, c.n_sink, c.act, c.enable_memory, c.scorer,
                    c.scale, c.lambda_, c.eta, c.eps, c.norm_eps)
         self.n_seq = n_seq
         self.h = self.lib.orc_create(C.byref(raw), n_seq)
@@ -246,6 +253,65 @@ class OracleLayer:
                                                _p(ob) if ob is not None else None, _p(od) if od is not None else None)
         assert rc == 0, "the leading layer's scores do not cover this layer's entries"
         return ob, od
+
+    # ---- a retained set per KV head (Sec. 2.2 framework; configuration scorer = 1 Knorm, 2 scores from the caller)
+    def _ext(self, ext):
+        if ext is None:
+            return None, 0
+        ext = np.ascontiguousarray(np.asarray(ext, dtype=np.float32))
+        assert ext.ndim == 2 and ext.shape[0] == self.cfg.Hkv, "scores are [Hkv, positions]"
+        return ext, ext.shape[1]
+
+    def ph_decode_step(self, seq: int, q, k_new, v_new, ext=None):
+        """One decode token; ext: float32 [Hkv, positions] scores by token position (scorer 2), used if the call compresses."""
+        q, k_new, v_new = _f32(q), _f32(k_new), _f32(v_new)
+        assert q.size == self.D and k_new.size == self.Dkv and v_new.size == self.Dkv
+        ext, n_pos = self._ext(ext)
+        ob = np.empty((self.cfg.H, self.cfg.d), np.float32)
+        od = np.empty((self.cfg.H, self.cfg.d), np.float64)
+        rc = self.lib.orc_ph_decode_step(self.h, seq, _p(q), _p(k_new), _p(v_new), _p(ext) if ext is not None else None, n_pos, _p(ob), _p(od))
+        assert rc == 0, "scores from the caller are missing or do not cover the cached positions"
+        return ob, od
+
+    def ph_prefill_chunk(self, seq: int, K, V, Q=None, ext=None):
+        K, V = _f32(K), _f32(V)
+        Cn = K.size // self.Dkv
+        assert K.size == Cn * self.Dkv and V.size == K.size
+        ext, n_pos = self._ext(ext)
+        ob = od = None
+        if Q is not None:
+            Q = _f32(Q)
+            assert Q.size == Cn * self.D
+            ob = np.empty((Cn, self.cfg.H, self.cfg.d), dtype=np.float32)
+            od = np.empty((Cn, self.cfg.H, self.cfg.d), dtype=np.float64)
+        rc = self.lib.orc_ph_prefill_chunk(self.h, seq, Cn, _p(Q) if Q is not None else None, _p(K), _p(V),
+                                           _p(ext) if ext is not None else None, n_pos,
+                                           _p(ob) if ob is not None else None, _p(od) if od is not None else None)
+        assert rc == 0, "scores from the caller are missing or do not cover the cached positions"
+        return ob, od
+
+    def ph_entries(self, seq: int, head: int):
+        """dict(pos int32[n], score f32[n], K f32[n,d], V f32[n,d]) of one KV head's retained set; ascending pos."""
+        n, c = self.lib.orc_ph_count(self.h, seq, head), self.cfg
+        pos = np.empty(n, np.int32)
+        score = np.empty(n, np.float32)
+        K = np.empty((n, c.d), np.float32)
+        V = np.empty((n, c.d), np.float32)
+        self.lib.orc_ph_export(self.h, seq, head, _p(pos), _p(score), _p(K), _p(V))
+        return {"pos": pos, "score": score, "K": K, "V": V}
+
+    def ph_last_evicted(self, seq: int, head: int) -> np.ndarray:
+        cap = max(1, self.lib.orc_ph_last_evicted(self.h, seq, head, None, 0))
+        buf = np.empty(cap, np.int32)
+        n = self.lib.orc_ph_last_evicted(self.h, seq, head, _p(buf), cap)
+        return buf[:n]
+
+    def ph_last_selection(self, seq: int, head: int):
+        n = self.lib.orc_ph_last_selection(self.h, seq, head, None, None, 0)
+        pos = np.empty(max(n, 1), np.int32)
+        score = np.empty(max(n, 1), np.float32)
+        self.lib.orc_ph_last_selection(self.h, seq, head, _p(pos), _p(score), n)
+        return pos[:n], score[:n]
 
     # ---- state
     def count(self, seq=0) -> int:

@@ -641,3 +641,131 @@ def test_score_reuse_needs_the_leaders_call_first():
     foll.prefill_chunk_follow(0, lead, 0, K[:7], V[:7])
     with pytest.raises(AssertionError):            # the leader has not seen token 7 yet
         foll.decode_step_follow(0, lead, 0, Q[7], K[7], V[7])
+
+
+# ------------------------------------------------------------------ a retained set per KV head (Sec. 2.2 framework)
+def _dense_scores(pos, acc, n_pos, Hkv):
+    """[Hkv, n_pos] score table by token position with the same row for every head."""
+    row = np.full(n_pos, -np.inf, np.float32)
+    row[pos] = acc
+    return np.tile(row, (Hkv, 1))
+
+
+def test_per_head_knorm_keeps_the_largest_key_norms_of_every_head():
+    """Knorm (Sec. 2.2: S_t = ||K_t||_2): every KV head keeps its sinks and then the B - n_sink entries with the
+    largest key norm of THAT head (ties to the lower position) - a brute-force sort per head; the heads' sets differ."""
+    rng = np.random.default_rng(31)
+    L = orc.OracleLayer(small_cfg(Hkv=2, B=7, tau=3, n_sink=2, scorer=1, enable_memory=0))
+    rand_weights(L, rng)
+    _, Q, K, V = rand_tokens(L, rng, 40)
+    K = bf16(K * np.exp(0.6 * rng.standard_normal((40, 2, 1))))          # norms differ between heads
+    L.ph_prefill_chunk(0, K[:12], V[:12])
+    alive = [list(range(12)) for _ in range(2)]
+
+    def compress(h):
+        norm = lambda t: np.float32(np.sqrt((K[t, h].astype(np.float64) ** 2).sum()))
+        order = sorted(alive[h], key=lambda t: (-(math.inf if t < 2 else float(norm(t))), t))
+        alive[h] = sorted(order[:7])
+
+    for h in range(2):
+        compress(h)
+        assert L.ph_entries(0, h)["pos"].tolist() == alive[h]
+    for s in range(12, 40):
+        _, od = L.ph_decode_step(0, Q[s], K[s], V[s])
+        for h in range(2):
+            alive[h].append(s)
+            if (s - 12 + 1) % 3 == 0:
+                compress(h)
+            e = L.ph_entries(0, h)
+            assert e["pos"].tolist() == alive[h]
+            assert np.array_equal(e["K"], K[alive[h], h]) and np.array_equal(e["V"], V[alive[h], h])
+        # attention of query head j over the set of ITS KV head (memory disabled): textbook softmax per head
+        for j in range(L.cfg.H):
+            g = j // L.Gq
+            sc = (K[alive[g], g].astype(np.float64) @ Q[s, j].astype(np.float64)) * L.cfg.scale
+            pr = np.exp(sc - sc.max())
+            np.testing.assert_allclose(od[j], (pr / pr.sum()) @ V[alive[g], g].astype(np.float64), rtol=1e-11, atol=1e-13)
+    assert alive[0] != alive[1]
+
+
+def test_per_head_memory_write_assembles_the_evicted_slices_of_a_token():
+    """The evict step's memory write with per-head sets (Alg. 1, "summed across heads per token"): a token that loses
+    the slices of some heads in this step contributes ONE pair (k~, v~) in model space, holding those slices at their
+    query heads' places and zeros elsewhere.  Scores from the caller make head 0 evict positions {1, 3} and head 1
+    evict {3, 4}: three pairs - position 1 (head 0 only), 3 (both), 4 (head 1 only) - against numpy."""
+    rng = np.random.default_rng(32)
+    L = orc.OracleLayer(small_cfg(Hkv=2, B=3, n_sink=0, scorer=2, lambda_=0.5, eta=2.0))
+    w = rand_weights(L, rng)
+    c = L.cfg
+    _, Q, K, V = rand_tokens(L, rng, 6)
+    ext = np.array([[5, 0, 4, 1, 3], [5, 4, 3, 0, 1]], np.float32)        # by position, per head
+    L.ph_prefill_chunk(0, K[:5], V[:5], ext=ext)
+    assert L.ph_entries(0, 0)["pos"].tolist() == [0, 2, 4] and L.ph_entries(0, 1)["pos"].tolist() == [0, 1, 2]
+    assert L.ph_last_evicted(0, 0).tolist() == [1, 3] and L.ph_last_evicted(0, 1).tolist() == [3, 4]
+    Wt = w["W_theta"].astype(np.float64)
+    M_want, b_want = np.zeros((c.dM, L.D)), np.zeros(c.dM)
+    for t, heads in ((1, [0]), (3, [0, 1]), (4, [1])):
+        ku, vu = np.zeros((c.H, c.d)), np.zeros((c.H, c.d))
+        for h in heads:
+            ku[h * L.Gq:(h + 1) * L.Gq] = K[t, h]
+            vu[h * L.Gq:(h + 1) * L.Gq] = V[t, h]
+        phi = Wt @ ku.reshape(-1)
+        M_want += np.outer(phi, vu.reshape(-1))
+        b_want += phi ** 2
+    M, b = L.memory()
+    np.testing.assert_allclose(M, 2.0 * M_want, rtol=1e-11, atol=1e-13)     # eta = 2, first evict step: lambda * 0
+    np.testing.assert_allclose(b, 2.0 * b_want, rtol=1e-11, atol=1e-13)
+    # a second evict step decays the first: one more token, every head evicts its lowest score
+    ext2 = np.array([[5, 0, 4, 1, 3, 2], [5, 4, 3, 0, 1, 9]], np.float32)
+    L.ph_decode_step(0, Q[5], K[5], V[5], ext=ext2)
+    assert L.ph_last_evicted(0, 0).tolist() == [5] and L.ph_last_evicted(0, 1).tolist() == [2]
+    M2_want, b2_want = 0.5 * 2.0 * M_want, 0.5 * 2.0 * b_want
+    for t, h in ((2, 1), (5, 0)):
+        ku, vu = np.zeros((c.H, c.d)), np.zeros((c.H, c.d))
+        ku[h * L.Gq:(h + 1) * L.Gq] = K[t, h]
+        vu[h * L.Gq:(h + 1) * L.Gq] = V[t, h]
+        phi = Wt @ ku.reshape(-1)
+        M2_want += 2.0 * np.outer(phi, vu.reshape(-1))
+        b2_want += 2.0 * phi ** 2
+    M, b = L.memory()
+    np.testing.assert_allclose(M, M2_want, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(b, b2_want, rtol=1e-11, atol=1e-13)
+
+
+def test_per_head_sets_with_identical_rows_reduce_to_the_shared_row_path():
+    """Handed the indexer's own pooled scores as the row of every head, the per-head path makes the indexer path's
+    selections, memory writes and outputs to the last bit (a token then loses all its slices at once and the
+    assembled pair is the plain lifted key / value)."""
+    rng = np.random.default_rng(33)
+    kw = dict(B=8, tau=2, n_sink=1, lambda_=0.9, eta=0.7)
+    A = orc.OracleLayer(small_cfg(**kw))
+    P = orc.OracleLayer(small_cfg(scorer=2, **kw))
+    w = rand_weights(A, rng)
+    P.set_weights(w)
+    X, Q, K, V = rand_tokens(A, rng, 34)
+    Hkv = A.cfg.Hkv
+    _, od_a = A.prefill_chunk_out(0, X[:14], Q[:14], Q[:14], K[:14], V[:14])
+    _, od_p = P.ph_prefill_chunk(0, K[:14], V[:14], Q=Q[:14], ext=_dense_scores(*A.last_selection(), 14, Hkv))
+    assert np.array_equal(od_a, od_p)
+    for s in range(14, 34):
+        _, od_a = A.decode_step(0, X[s], Q[s].reshape(-1), Q[s], K[s], V[s])
+        ext = _dense_scores(*A.last_selection(), s + 1, Hkv) if A.since() == 0 else None
+        _, od_p = P.ph_decode_step(0, Q[s], K[s], V[s], ext=ext)
+        assert np.array_equal(od_a, od_p), s
+        for h in range(Hkv):
+            assert P.ph_entries(0, h)["pos"].tolist() == A.positions().tolist()
+    for a, b in zip(A.memory(), P.memory()):
+        assert np.array_equal(a, b)
+    assert A.evict_steps() == P.evict_steps() == 1 + 10
+
+
+def test_per_head_scores_from_the_caller_are_required():
+    rng = np.random.default_rng(34)
+    L = orc.OracleLayer(small_cfg(B=3, scorer=2))
+    rand_weights(L, rng)
+    _, Q, K, V = rand_tokens(L, rng, 5)
+    with pytest.raises(AssertionError):
+        L.ph_prefill_chunk(0, K[:5], V[:5])                               # no scores
+    L2 = orc.OracleLayer(small_cfg(B=3, scorer=2))
+    with pytest.raises(AssertionError):
+        L2.ph_prefill_chunk(0, K[:5], V[:5], ext=np.zeros((2, 4), np.float32))   # position 4 not covered
