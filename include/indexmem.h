@@ -63,6 +63,9 @@ typedef struct im_config {
   int32_t chunk_outputs;     /* 1: reserve workspace for im_prefill_chunk_attend (max_seqs * max_chunk * D_kv floats) */
   int32_t score_share;       /* g >= 2: layers l with l % g != 0 reuse the indexer scores of layer l - l % g (App. B,
                                 IndexCache-style reuse; the paper uses 4); 0 or 1: every layer scores for itself      */
+  int32_t scorer;            /* 0: the learnable indexer, one score row per sequence (Sec. 3.1).  A retained set per KV head
+                                (Sec. 2.2, S in R^{B x H_kv x L}): 1 Knorm, S_t = ||K_t||_2 (Sec. 2.2); 2 scores handed in
+                                by the caller with im_set_scores (Sec. 5 ablation: the memory on another eviction policy) */
   float softmax_scale;       /* 0 => 1/sqrt(d)                                 (Sec. 2.1)           */
   float lambda;              /* decay of Eq. 6-7, (0,1]; 0 => 1                                      */
   float eta;                 /* write strength of Eq. 6-7, > 0; 0 => 1                               */
@@ -316,6 +319,35 @@ int im_get_config(im_ctx* ctx, im_config* out, int32_t* capacity);
  */
 int im_attention_noalloc(const void* q, const void* k, const void* v, int n_q_heads, int n_kv_heads, int head_dim,
                          int n, float softmax_scale, void* out, void* cuda_stream);
+
+/*
+ * Retained sets per KV head (configuration scorer = 1 or 2; Sec. 2.2 frames eviction as S = f(.) in R^{B x H_kv x L},
+ * I = TopK(S, L'), [K', V'] = Gather(K, V, I)).  im_prefill_chunk and im_decode_step then keep, for every KV head of a
+ * sequence, the B entries with the largest score of THAT head (score descending, position ascending, the first n_sink
+ * positions first); x and q_pre are ignored (there is no indexer), im_prefill_chunk_attend and score_share are not
+ * available.  All heads hold the same number of entries; which positions they are differs per head.
+ * The memory write of an evict step (Eq. 6-7; Alg. 1: "evicted_v is summed across heads per token"): every token that
+ * loses at least one head slice in the step contributes ONE pair (k~, v~) in model space, the evicted slices at the
+ * places of their query heads and zeros at the heads that keep the token.  With the same scores for every head this
+ * is the shared-row path.
+ *
+ * im_set_scores (scorer = 2): `scores` is dev float32 [n_seq][H_kv][n_positions]; scores[i][h][t] is the importance of
+ * token position t of the i-th sequence of the NEXT compressing call on `layer` for KV head h.  n_positions must cover
+ * every position cached after that call's append, the call must name the same number of sequences, and the array must
+ * stay valid until that call's kernels have run.  The scores are consumed by that call; a compressing call without
+ * scores returns IM_ERR_STATE.  Non-finite scores set the status word.
+ */
+int im_set_scores(im_ctx* ctx, int layer, int n_seq, const float* scores, int64_t n_positions);
+
+/*
+ * Per-head pieces of the state in per-head mode (head in [0, H_kv)): IM_S_POS int32[n], IM_S_IMP float32[n] (the head's
+ * scores), IM_S_K / IM_S_V bf16 [n][d] (the head's slab, slot order), IM_S_EVICTED int32[n_evicted] (ascending),
+ * IM_S_SEL_POS / IM_S_SEL_IMP (what the head's latest selection chose among).  Import: IM_S_POS, IM_S_IMP, IM_S_K,
+ * IM_S_V.  IM_S_COUNTS, IM_S_M and IM_S_B go through im_state_export / im_state_import in either mode; the pieces
+ * above are refused there in per-head mode (and here otherwise).  Both synchronise the device.
+ */
+int im_state_export_head(im_ctx* ctx, int layer, int seq, int head, int which, void* host_buf, size_t bytes);
+int im_state_import_head(im_ctx* ctx, int layer, int seq, int head, int which, const void* host_buf, size_t bytes);
 
 /* Thread-local description of the last error returned on this thread ("" if none). */
 const char* im_last_error(void);

@@ -34,7 +34,7 @@ WEIGHT_IDS = {"U_q": IM_W_UQ, "U_k": IM_W_UK, "G": IM_W_G, "W_theta": IM_W_THETA
 class im_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "max_seqs", "n_q_heads", "n_kv_heads", "head_dim", "n_index_heads", "index_dim", "mem_dim",
-        "budget", "compress_interval", "max_chunk", "n_sink", "act", "enable_memory", "out_f32", "pending_slots", "chunk_outputs", "score_share")] + \
+        "budget", "compress_interval", "max_chunk", "n_sink", "act", "enable_memory", "out_f32", "pending_slots", "chunk_outputs", "score_share", "scorer")] + \
         [(n, C.c_float) for n in ("softmax_scale", "lambda_", "eta", "eps", "norm_eps", "init_std")] + \
         [("seed", C.c_uint64)]
 
@@ -59,6 +59,9 @@ _lib.im_get_weights.argtypes = [_vp, _i32, _i32, _vp, _sz]
 _lib.im_state_export.argtypes = [_vp, _i32, _i32, _i32, _vp, _sz]
 _lib.im_state_import.argtypes = [_vp, _i32, _i32, _i32, _vp, _sz]
 _lib.im_topb_select.argtypes = [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp]
+_lib.im_set_scores.argtypes = [_vp, _i32, _i32, _vp, C.c_int64]
+_lib.im_state_export_head.argtypes = [_vp, _i32, _i32, _i32, _i32, _vp, _sz]
+_lib.im_state_import_head.argtypes = [_vp, _i32, _i32, _i32, _i32, _vp, _sz]
 _lib.im_status.argtypes = [_vp, _vp, C.POINTER(C.c_int32)]
 _lib.im_launch_count.argtypes = [_vp]
 _lib.im_launch_count.restype = C.c_int64
@@ -72,7 +75,8 @@ _lib.im_last_error.restype = C.c_char_p
 
 EXPORTED = ("im_workspace_bytes", "im_create", "im_destroy", "im_reset", "im_prefill_chunk", "im_decode_step",
             "im_set_weights", "im_get_weights", "im_state_export", "im_state_import", "im_topb_select",
-            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc", "im_event_count", "im_prefill_chunk_attend")
+            "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc", "im_event_count", "im_prefill_chunk_attend",
+            "im_set_scores", "im_state_export_head", "im_state_import_head")
 
 
 def _check(rc: int):
@@ -115,9 +119,13 @@ def im_reset(ctx: int, layer: int = -1, seq: int = -1):
     _check(_lib.im_reset(ctx, layer, seq, _stream()))
 
 
+def _ptr(t):
+    return 0 if t is None else t.data_ptr()
+
+
 def im_prefill_chunk(ctx, layer, seq_ids, chunk_len, x, q_pre, k, v):
     ids = _ids(seq_ids)
-    _check(_lib.im_prefill_chunk(ctx, layer, ids.size, ids.ctypes.data, chunk_len, x.data_ptr(), q_pre.data_ptr(),
+    _check(_lib.im_prefill_chunk(ctx, layer, ids.size, ids.ctypes.data, chunk_len, _ptr(x), _ptr(q_pre),
                                  k.data_ptr(), v.data_ptr(), _stream()))
 
 
@@ -130,7 +138,7 @@ def im_prefill_chunk_attend(ctx, layer, seq_ids, chunk_len, x, q_pre, q, k, v, o
 
 def im_decode_step(ctx, layer, seq_ids, x, q_pre, q, k_new, v_new, out):
     ids = _ids(seq_ids)
-    _check(_lib.im_decode_step(ctx, layer, ids.size, ids.ctypes.data, x.data_ptr(), q_pre.data_ptr(), q.data_ptr(),
+    _check(_lib.im_decode_step(ctx, layer, ids.size, ids.ctypes.data, _ptr(x), _ptr(q_pre), q.data_ptr(),
                                k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(), _stream()))
 
 
@@ -150,6 +158,23 @@ def im_state_export(ctx, layer, seq, which, host: np.ndarray):
 def im_state_import(ctx, layer, seq, which, host: np.ndarray):
     host = np.ascontiguousarray(host)
     _check(_lib.im_state_import(ctx, layer, seq, which, host.ctypes.data, host.nbytes))
+
+
+def im_set_scores(ctx, layer, scores: torch.Tensor):
+    """scores float32 [n_seq, Hkv, n_positions] (CUDA, contiguous): the importance of every token position per KV head
+    for the next compressing call on `layer`; must stay alive until that call's kernels have run."""
+    n_seq, _, n_pos = scores.shape
+    _dev(scores, torch.float32, scores.numel(), "scores")
+    _check(_lib.im_set_scores(ctx, layer, n_seq, scores.data_ptr(), n_pos))
+
+
+def im_state_export_head(ctx, layer, seq, head, which, host: np.ndarray):
+    _check(_lib.im_state_export_head(ctx, layer, seq, head, which, host.ctypes.data, host.nbytes))
+
+
+def im_state_import_head(ctx, layer, seq, head, which, host: np.ndarray):
+    host = np.ascontiguousarray(host)
+    _check(_lib.im_state_import_head(ctx, layer, seq, head, which, host.ctypes.data, host.nbytes))
 
 
 def im_topb_select(scores: torch.Tensor, pos: torch.Tensor, budget: int, n_sink: int):
@@ -245,6 +270,7 @@ class Config:
     pending_slots: int = 0
     chunk_outputs: int = 0
     score_share: int = 0
+    scorer: int = 0
     softmax_scale: float = 0.0
     lambda_: float = 0.0
     eta: float = 0.0
@@ -303,9 +329,11 @@ class IndexMem:
 
     # ---- hot calls
     def prefill_chunk(self, layer, seq_ids, x, q_pre, k, v):
-        n, Cn = len(seq_ids), x.shape[-2]
+        """x and q_pre feed the indexer; with a retained set per KV head (cfg.scorer != 0) they may be None."""
+        n, Cn = len(seq_ids), k.shape[-3]
         bf = torch.bfloat16
-        _dev(x, bf, n * Cn * self.D, "x"); _dev(q_pre, bf, n * Cn * self.D, "q_pre")
+        if not self.ccfg.scorer:
+            _dev(x, bf, n * Cn * self.D, "x"); _dev(q_pre, bf, n * Cn * self.D, "q_pre")
         _dev(k, bf, n * Cn * self.Dkv, "k"); _dev(v, bf, n * Cn * self.Dkv, "v")
         im_prefill_chunk(self.ctx, layer, seq_ids, Cn, x, q_pre, k, v)
 
@@ -324,7 +352,9 @@ class IndexMem:
     def decode_step(self, layer, seq_ids, x, q_pre, q, k_new, v_new, out=None):
         n = len(seq_ids)
         bf = torch.bfloat16
-        _dev(x, bf, n * self.D, "x"); _dev(q_pre, bf, n * self.D, "q_pre"); _dev(q, bf, n * self.D, "q")
+        if not self.ccfg.scorer:
+            _dev(x, bf, n * self.D, "x"); _dev(q_pre, bf, n * self.D, "q_pre")
+        _dev(q, bf, n * self.D, "q")
         _dev(k_new, bf, n * self.Dkv, "k_new"); _dev(v_new, bf, n * self.Dkv, "v_new")
         if out is None:
             out = torch.empty((n, self.H, self.d), dtype=self.out_dtype, device=self.device)
@@ -403,6 +433,52 @@ class IndexMem:
         if a.dtype == np.int16:
             return _from_bf16_bits(a).to(torch.float32).numpy().reshape(a.shape)
         return a
+
+    # ---- a retained set per KV head (cfg.scorer != 0)
+    def set_scores(self, layer, scores: torch.Tensor):
+        im_set_scores(self.ctx, layer, scores)
+
+    def export_head(self, layer, seq, head, which):
+        """One KV head's piece of the state: IM_S_POS, IM_S_IMP (scores), IM_S_K / IM_S_V ([n, d]), IM_S_EVICTED,
+        IM_S_SEL_POS, IM_S_SEL_IMP."""
+        c = self.counts(layer, seq)
+        n = c["n"]
+        if which == IM_S_POS:
+            a = np.empty(n, np.int32)
+        elif which == IM_S_IMP:
+            a = np.empty(n, np.float32)
+        elif which in (IM_S_K, IM_S_V):
+            a = np.empty((n, self.d), np.int16)
+        elif which == IM_S_EVICTED:
+            a = np.empty(c["n_evicted"], np.int32)
+        elif which == IM_S_SEL_POS:
+            a = np.empty(c["n_sel"], np.int32)
+        elif which == IM_S_SEL_IMP:
+            a = np.empty(c["n_sel"], np.float32)
+        else:
+            raise ValueError(which)
+        if a.size:
+            im_state_export_head(self.ctx, layer, seq, head, which, a)
+        if a.dtype == np.int16:
+            return _from_bf16_bits(a).to(torch.float32).numpy().reshape(a.shape)
+        return a
+
+    def import_head_state(self, layer, seq, *, heads, M_kv, b, T, since=0, evict_steps=0):
+        """Replaces one sequence's state in per-head mode.  heads: one dict(pos, score, K [n, d], V [n, d]) per KV head,
+        all with the same number of entries."""
+        n = len(heads[0]["pos"])
+        ctr = np.zeros(8, np.int32)
+        ctr[0], ctr[1], ctr[2], ctr[3] = n, T, since, evict_steps
+        im_state_import(self.ctx, layer, seq, IM_S_M, np.asarray(M_kv, np.float32))
+        im_state_import(self.ctx, layer, seq, IM_S_B, np.asarray(b, np.float32))
+        im_state_import(self.ctx, layer, seq, IM_S_COUNTS, ctr)
+        for h, e in enumerate(heads):
+            assert len(e["pos"]) == n
+            if n:
+                im_state_import_head(self.ctx, layer, seq, h, IM_S_POS, np.asarray(e["pos"], np.int32))
+                im_state_import_head(self.ctx, layer, seq, h, IM_S_IMP, np.asarray(e["score"], np.float32))
+                im_state_import_head(self.ctx, layer, seq, h, IM_S_K, _bf16_bits(torch.from_numpy(np.asarray(e["K"], np.float32))))
+                im_state_import_head(self.ctx, layer, seq, h, IM_S_V, _bf16_bits(torch.from_numpy(np.asarray(e["V"], np.float32))))
 
     def import_state(self, layer, seq, *, pos, imp, kidx, K, V, M_kv, b, T, since=0, evict_steps=0):
         """Replaces one sequence's state.  kidx/K/V are float arrays holding bf16 values."""

@@ -86,6 +86,10 @@ bool resolve(const im_config* in, im_config* c, ImDims* p) {
   q.chunk_out = c->chunk_outputs ? 1 : 0;
   if (c->score_share < 0 || c->score_share > c->n_layers) return false;
   q.share = c->score_share >= 2 ? c->score_share : 0;
+  if (c->scorer < 0 || c->scorer > 2) return false;
+  if (c->scorer && (q.share || c->chunk_outputs || c->n_kv_heads > 4096)) return false;  // per-head sets: neither score reuse nor chunk outputs
+  q.scorer = c->scorer;
+  q.evr = q.tail * (q.scorer ? q.Hkv : 1);
   q.R3 = q.HI * q.dI + q.dI + q.HI;
   q.R5 = q.R3 + q.dM + 1;
   q.max_splits = (q.cap + 255) / 256;
@@ -124,6 +128,19 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->st.pend_w = (float*)take(U * p.F * 4);
   lo->st.ctr = (int32_t*)take(U * CTR_STRIDE * 4);
   lo->st.status = (int32_t*)take(256);
+  lo->st.hpos = lo->st.hsel_pos = lo->st.hev_slot = lo->st.hev_pos = nullptr;
+  lo->st.hscore = lo->st.hsel_score = nullptr;
+  lo->st.hkeep = nullptr;
+  if (p.scorer) {  // a retained set per KV head: position / score / selection bookkeeping per (unit, head) row
+    const size_t R = U * p.Hkv;
+    lo->st.hpos = (int32_t*)take(R * p.cap * 4);
+    lo->st.hscore = (float*)take(R * p.cap * 4);
+    lo->st.hsel_pos = (int32_t*)take(R * p.cap * 4);
+    lo->st.hsel_score = (float*)take(R * p.cap * 4);
+    lo->st.hev_slot = (int32_t*)take(R * p.tail * 4);
+    lo->st.hev_pos = (int32_t*)take(R * p.tail * 4);
+    lo->st.hkeep = (uint8_t*)take(R * p.cap);
+  }
   lo->state_end = off;
   lo->w.resize(p.L);
   for (int l = 0; l < p.L; ++l) {
@@ -139,9 +156,16 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   }
   lo->sc.raw = (float*)take((size_t)p.S * std::max(p.max_chunk, IM_KSPLIT) * p.R5 * 4);
   lo->sc.keyp = (double*)take((size_t)p.S * std::max(p.max_chunk, IM_KSPLIT_KEY) * p.dI * 8);
-  lo->sc.evK = (bf16*)take((size_t)p.S * p.tail * p.Dkv * 2);
-  lo->sc.evV = (bf16*)take((size_t)p.S * p.tail * p.Dkv * 2);
-  lo->sc.phi = (float*)take((size_t)p.S * p.tail * p.dM * 4);
+  lo->sc.evK = (bf16*)take((size_t)p.S * p.evr * p.Dkv * 2);
+  lo->sc.evV = (bf16*)take((size_t)p.S * p.evr * p.Dkv * 2);
+  lo->sc.phi = (float*)take((size_t)p.S * p.evr * p.dM * 4);
+  lo->sc.hsurv = lo->sc.hnhole = lo->sc.hrowmap = lo->sc.hntok = nullptr;
+  if (p.scorer) {
+    lo->sc.hsurv = (int32_t*)take((size_t)p.S * p.Hkv * p.tail * 4);
+    lo->sc.hnhole = (int32_t*)take((size_t)p.S * p.Hkv * 4);
+    lo->sc.hrowmap = (int32_t*)take((size_t)p.S * p.Hkv * p.tail * 4);
+    lo->sc.hntok = (int32_t*)take((size_t)p.S * 4);
+  }
   lo->sc.phip = (float*)take((size_t)IM_KSPLIT * p.S * p.F * p.dM * 4);
   lo->sc.surv = (int32_t*)take((size_t)p.S * p.tail * 4);
   lo->sc.nhole = (int32_t*)take((size_t)p.S * 4);
@@ -199,6 +223,8 @@ struct im_ctx {
   alignas(64) unsigned char mapVs[128];
   alignas(64) unsigned char mapK128[128];  // the same caches with 128-row boxes (full tiles of the tensor-core attention)
   alignas(64) unsigned char mapV128[128];
+  struct ExtScores { const float* ptr = nullptr; long long n_pos = 0; int n_seq = 0; };
+  std::vector<ExtScores> ext;        // per layer: scores handed in by the caller for the next compressing call (scorer = 2)
   bool ro_stream = false;            // phi(q)^T Mhat by the bulk-copy streaming kernel where it runs next to the attention kernel (IM_OPT_READOUT_STAGES)
   int ro_stages = 2;                 // ... with this many 32 KB stages per CTA
   bool attn_tc_ready = false;        // the tensor-core streaming attention kernel takes this shape and is set up
@@ -343,6 +369,157 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
   return IM_OK;
 }
 
+// ---- a retained set per KV head (scorer = 1 Knorm, 2 the caller's scores): both calls in order on the caller's stream.
+// Append; if due: scores in, selection per head, the evict step's memory write (rows assembled per token, phi by the
+// skinny / tensor-core GEMM against the folded Linear_theta, accumulation straight into Mhat), hole filling; decode
+// then attends per head slab and adds the readout (Eq. 4-5).
+int perhead_compress(im_ctx* ctx, const ImLaunch& L, ImCall& call, int layer, int ne_max, long long T_after) {
+  const ImDims& p = ctx->p;
+  const float* ext = nullptr;
+  long long n_pos = 0;
+  if (p.scorer == 2) {
+    im_ctx::ExtScores& x = ctx->ext[layer];
+    if (!x.ptr) return fail(IM_ERR_STATE, "layer %d compresses with the caller's scores: call im_set_scores first", layer);
+    if (x.n_seq != call.n_seq) return fail(IM_ERR_ARG, "im_set_scores named %d sequences, this call %d", x.n_seq, call.n_seq);
+    if (x.n_pos < T_after) return fail(IM_ERR_ARG, "the caller's scores cover %lld positions, %lld are cached", x.n_pos, T_after);
+    ext = x.ptr;
+    n_pos = x.n_pos;
+    x = im_ctx::ExtScores();  // consumed
+  }
+  CKL(im_ph_launch_select(L, call, ext, n_pos));
+  if (ne_max > 0) {
+    if (p.mem) {
+      CKL(im_ph_launch_assemble(L, call, ne_max));
+      ImGemmArgs g;
+      memset(&g, 0, sizeof(g));
+      g.job[0] = {L.w.Wfh, L.w.Wfl, p.dM, 0, 0};
+      g.n_jobs = 1;
+      g.in[0] = L.sc.evK;
+      g.in_cnt[0] = ne_max * p.Hkv;
+      g.in_outer[0] = (long long)p.evr * p.Dkv;
+      g.in_inner[0] = p.Dkv;
+      g.NV = call.n_seq * ne_max * p.Hkv;
+      g.K = p.Dkv;
+      g.out = L.sc.phi;
+      g.out_cnt = ne_max * p.Hkv;
+      g.out_outer = (long long)p.evr * p.dM;
+      g.out_inner = p.dM;
+      g.ksplit = 1;
+      g.tensor = g.NV >= 1024 ? 1 : 0;
+      CKL(im_launch_gemm(L, g));
+      CKL(im_ph_launch_mem_write(L, call));
+    }
+    CKL(im_ph_launch_move(L, call));
+  }
+  return IM_OK;
+}
+
+int perhead_prefill(im_ctx* ctx, ImCall& call, int layer, int chunk_len, const void* k, const void* v, void* cuda_stream) {
+  const ImDims& p = ctx->p;
+  int ne_max = 0;
+  long long T_after = 0;
+  for (int i = 0; i < call.n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    if (u.n + chunk_len > p.cap)
+      return fail(IM_ERR_CAPACITY, "sequence %d: %d cached + chunk %d exceeds capacity %d", call.seq[i], u.n, chunk_len, p.cap);
+    ne_max = std::max(ne_max, u.n + chunk_len - p.B);
+    T_after = std::max(T_after, u.T + chunk_len);
+  }
+  if ((long long)ne_max * p.Hkv > IM_PH_MAX_PAIRS)
+    return fail(IM_ERR_CAPACITY, "per-head sets: %d evicted entries x %d heads exceed %d pairs per evict step", ne_max, p.Hkv, IM_PH_MAX_PAIRS);
+  call.C = chunk_len;
+  call.prefill = 1;
+  call.due = 1;
+  ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
+  CKL(im_ph_launch_append(L, call, k, v));
+  int rc = perhead_compress(ctx, L, call, layer, ne_max, T_after);
+  if (rc) return rc;
+  for (int i = 0; i < call.n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    const int ne = std::max(0, u.n + chunk_len - p.B);
+    u.n = u.n + chunk_len - ne;
+    u.T += chunk_len;
+    u.since = 0;
+  }
+  return IM_OK;
+}
+
+int perhead_decode(im_ctx* ctx, ImCall& call, int layer, const void* q, const void* k_new, const void* v_new, void* out,
+                   void* cuda_stream) {
+  const ImDims& p = ctx->p;
+  bool due_any = false, due_all = true;
+  int ne_max = 0, n_att = 0;
+  long long T_after = 0;
+  for (int i = 0; i < call.n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    if (u.n + 1 > p.cap) return fail(IM_ERR_CAPACITY, "sequence %d has no free slot (capacity %d)", call.seq[i], p.cap);
+    const bool due = (u.since + 1 == p.tau);
+    due_any |= due;
+    due_all &= due;
+    ne_max = std::max(ne_max, u.n + 1 - p.B);
+    T_after = std::max(T_after, u.T + 1);
+  }
+  if (due_any != due_all)
+    return fail(IM_ERR_ARG, "sequences of one decode call must be at the same phase of the compression interval");
+  const bool due = due_all;
+  if (!due) ne_max = 0;
+  if ((long long)ne_max * p.Hkv > IM_PH_MAX_PAIRS)
+    return fail(IM_ERR_CAPACITY, "per-head sets: %d evicted entries x %d heads exceed %d pairs per evict step", ne_max, p.Hkv, IM_PH_MAX_PAIRS);
+  call.due = due ? 1 : 0;
+  call.C = 1;
+  call.prefill = 0;
+  call.ksplit = pick_ksplit(p.D, IM_KSPLIT);
+  call.ksplit_key = 1;
+  call.ksplit_phi = 1;
+  ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
+  CKL(im_ph_launch_append(L, call, k_new, v_new));
+  if (p.mem) {  // phi(q) of Eq. 5 and the gate logit of Eq. 4 (K-split partials, summed by their consumers)
+    ImRows r = im_rows(p);
+    ImGemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.in[2] = (const bf16*)q;
+    g.in_cnt[2] = 1;
+    g.in_outer[2] = p.D;
+    g.out = L.sc.raw;
+    g.out_cnt = 1;
+    g.out_outer = p.R5;
+    g.ks_stride = (long long)call.n_seq * p.R5;
+    g.NV = call.n_seq;
+    g.K = p.D;
+    g.ksplit = call.ksplit;
+    g.direct = 1;
+    g.job[0] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
+    g.job[1] = {L.w.wg, nullptr, 1, r.wg, 2};
+    g.n_jobs = 2;
+    CKL(im_launch_gemm(L, g));
+  }
+  if (due) {
+    int rc = perhead_compress(ctx, L, call, layer, ne_max, T_after);
+    if (rc) return rc;
+  }
+  for (int i = 0; i < call.n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    const int ne = due ? std::max(0, u.n + 1 - p.B) : 0;
+    u.n = u.n + 1 - ne;
+    u.T += 1;
+    u.since = due ? 0 : u.since + 1;
+    n_att = std::max(n_att, u.n);
+  }
+  // a5 / a6 over the heads' own slabs (all heads of a sequence hold the same number of entries)
+  if (ctx->fast_attn) {
+    CKL(im_launch_attention_fast(L, call, ctx->mapKs, ctx->mapVs, q, ctx->n_ctas, 0));
+    if (p.mem) {
+      CKL(im_launch_readout(L, call, ctx->n_sm, 0));
+      CKL(im_launch_readout_finish(L, call));
+    }
+    CKL(im_launch_attention_merge(L, call, out, ctx->n_ctas * IM_ATTN_WARPS, IM_ATTN_STREAM_TILE, 0, q, k_new, v_new, 0));
+  } else {
+    CKL(im_launch_attention(L, call, q, out, n_att));
+  }
+  ctx->tail_stream = L.stream;
+  return IM_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -409,6 +586,8 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     ctx->n_ctas = std::max(1, std::min(sms, IM_ATTN_MAX_CTAS));
     ctx->fast_attn = (e == cudaSuccess);
   }
+  ctx->ext.resize(p.L);
+  if (e == cudaSuccess && p.scorer) e = im_perhead_prepare(p);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, ctx->device);
   if (e == cudaSuccess && im_score_tc_supported(p)) {
     e = im_score_tc_prepare();
@@ -493,6 +672,11 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   const ImDims& p = ctx->p;
   if (chunk_len < 1 || chunk_len > p.max_chunk)
     return fail(IM_ERR_ARG, "chunk_len %d out of range [1,%d]", chunk_len, p.max_chunk);
+  if (p.scorer) {  // a retained set per KV head: no indexer inputs
+    if (attend) return fail(IM_ERR_ARG, "im_prefill_chunk_attend is not available with a retained set per KV head");
+    if (!k || !v) return fail(IM_ERR_ARG, "null tensor");
+    return perhead_prefill(ctx, call, layer, chunk_len, k, v, cuda_stream);
+  }
   if (!x || !q_pre || !k || !v) return fail(IM_ERR_ARG, "null tensor");
   if (attend) {
     if (!q || !out) return fail(IM_ERR_ARG, "null tensor");
@@ -696,6 +880,11 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   int rc = check_call(ctx, layer, n_seq, seq_ids, &call);
   if (rc) return rc;
   const ImDims& p = ctx->p;
+  if (p.scorer) {  // a retained set per KV head: no indexer inputs
+    if (!q || !k_new || !v_new || !out) return fail(IM_ERR_ARG, "null tensor");
+    ctx->tail_is_merge = false;
+    return perhead_decode(ctx, call, layer, q, k_new, v_new, out, cuda_stream);
+  }
   if (!x || !q_pre || !q || !k_new || !v_new || !out) return fail(IM_ERR_ARG, "null tensor");
   bool due_any = false, due_all = true;
   int n_max = 0, ne_max = 0;
@@ -1075,6 +1264,8 @@ int im_state_export(im_ctx* ctx, int layer, int seq, int which, void* host_buf, 
     return IM_OK;
   };
   int rc;
+  if (p.scorer && which != IM_S_COUNTS && which != IM_S_M && which != IM_S_B)
+    return fail(IM_ERR_ARG, "state piece %d is kept per KV head in this configuration: use im_state_export_head", which);
   switch (which) {
     case IM_S_COUNTS:
       if ((rc = need(sizeof(ctr)))) return rc;
@@ -1168,6 +1359,8 @@ int im_state_import(im_ctx* ctx, int layer, int seq, int which, const void* host
   };
   int rc;
   const int n = hu.n;
+  if (p.scorer && which != IM_S_COUNTS && which != IM_S_M && which != IM_S_B)
+    return fail(IM_ERR_ARG, "state piece %d is kept per KV head in this configuration: use im_state_import_head", which);
   switch (which) {
     case IM_S_COUNTS: {
       if ((rc = exact(CTR_STRIDE * 4))) return rc;
@@ -1227,6 +1420,71 @@ int im_state_import(im_ctx* ctx, int layer, int seq, int which, const void* host
     default:
       return fail(IM_ERR_ARG, "state piece %d cannot be imported", which);
   }
+}
+
+int im_set_scores(im_ctx* ctx, int layer, int n_seq, const float* scores, int64_t n_positions) {
+  if (!ctx) return fail(IM_ERR_ARG, "null context");
+  const ImDims& p = ctx->p;
+  if (p.scorer != 2) return fail(IM_ERR_ARG, "im_set_scores needs scorer = 2 in the configuration");
+  if (layer < 0 || layer >= p.L) return fail(IM_ERR_ARG, "layer %d out of range [0,%d)", layer, p.L);
+  if (!scores || n_seq < 1 || n_seq > p.S || n_positions < 1) return fail(IM_ERR_ARG, "bad scores");
+  ctx->ext[layer].ptr = scores;
+  ctx->ext[layer].n_pos = n_positions;
+  ctx->ext[layer].n_seq = n_seq;
+  return IM_OK;
+}
+
+static int head_piece(im_ctx* ctx, int layer, int seq, int head, int which, void* host_buf, size_t bytes, bool import) {
+  if (!ctx || !host_buf) return fail(IM_ERR_ARG, "null argument");
+  const ImDims& p = ctx->p;
+  if (!p.scorer) return fail(IM_ERR_ARG, "per-head state pieces need scorer = 1 or 2 in the configuration");
+  if (layer < 0 || layer >= p.L || seq < 0 || seq >= p.S || head < 0 || head >= p.Hkv) return fail(IM_ERR_ARG, "layer/seq/head out of range");
+  ctx->tail_is_merge = false;
+  CK(cudaDeviceSynchronize());
+  const size_t u = (size_t)layer * p.S + seq;
+  const ImState& st = ctx->lo.st;
+  int32_t ctr[CTR_STRIDE];
+  CK(cudaMemcpy(ctr, st.ctr + u * CTR_STRIDE, sizeof(ctr), cudaMemcpyDeviceToHost));
+  const int n = import ? ctx->hu[u].n : ctr[CTR_N];
+  if (n < 0 || n > p.cap) return fail(IM_ERR_STATE, "entry count %d outside [0,%d]", n, p.cap);
+  const size_t row = (u * p.Hkv + head) * (size_t)p.cap, erow = (u * p.Hkv + head) * (size_t)p.tail;
+  void* dev = nullptr;
+  size_t want = 0;
+  switch (which) {
+    case IM_S_POS: dev = st.hpos + row; want = (size_t)n * 4; break;
+    case IM_S_IMP: dev = st.hscore + row; want = (size_t)n * 4; break;
+    case IM_S_K: dev = st.Kc + row * p.d; want = (size_t)n * p.d * 2; break;
+    case IM_S_V: dev = st.Vc + row * p.d; want = (size_t)n * p.d * 2; break;
+    case IM_S_EVICTED: {
+      if (import) return fail(IM_ERR_ARG, "state piece %d cannot be imported", which);
+      const int ne = ctr[CTR_NEVICT];
+      if (ne < 0 || ne > p.tail) return fail(IM_ERR_STATE, "device evicted count %d outside [0,%d]", ne, p.tail);
+      dev = st.hev_pos + erow;
+      want = (size_t)ne * 4;
+      break;
+    }
+    case IM_S_SEL_POS:
+    case IM_S_SEL_IMP: {
+      if (import) return fail(IM_ERR_ARG, "state piece %d cannot be imported", which);
+      const int ns = ctr[CTR_NSEL];
+      if (ns < 0 || ns > p.cap) return fail(IM_ERR_STATE, "device selection count %d outside [0,%d]", ns, p.cap);
+      dev = which == IM_S_SEL_POS ? (void*)(st.hsel_pos + row) : (void*)(st.hsel_score + row);
+      want = (size_t)ns * 4;
+      break;
+    }
+    default: return fail(IM_ERR_ARG, "state piece %d has no per-head form", which);
+  }
+  if (import ? bytes != want : bytes < want) return fail(IM_ERR_ARG, "state %d: buffer of %zu bytes, need %zu", which, bytes, want);
+  if (import) CK(cudaMemcpy(dev, host_buf, want, cudaMemcpyHostToDevice));
+  else CK(cudaMemcpy(host_buf, dev, want, cudaMemcpyDeviceToHost));
+  if (!import && which == IM_S_EVICTED) std::sort((int32_t*)host_buf, (int32_t*)host_buf + want / 4);
+  return IM_OK;
+}
+int im_state_export_head(im_ctx* ctx, int layer, int seq, int head, int which, void* host_buf, size_t bytes) {
+  return head_piece(ctx, layer, seq, head, which, host_buf, bytes, false);
+}
+int im_state_import_head(im_ctx* ctx, int layer, int seq, int head, int which, const void* host_buf, size_t bytes) {
+  return head_piece(ctx, layer, seq, head, which, const_cast<void*>(host_buf), bytes, true);
 }
 
 int im_topb_select(const float* scores, const int32_t* pos, int rows, int n, int budget, int n_sink, uint8_t* keep,

@@ -35,6 +35,8 @@ struct ImDims {
   int B, tau, cap, tail;      // budget, interval, slots per sequence, tail = cap - B
   int n_sink, act, mem, F, out_f32, max_chunk, chunk_out;
   int share;                  // >= 2: layers l with l % share != 0 reuse the scores of layer l - l % share
+  int scorer;                 // 0 indexer (one row per sequence); a retained set per KV head: 1 Knorm, 2 caller's scores
+  int evr;                    // rows per sequence of the evicted-pair scratch (evK / evV / phi): tail, per head tail * Hkv
   int R3, R5;                 // projection rows: indexer only / indexer + memory
   int max_splits;             // attention splits per (sequence, KV head)
   float scale, lambda, eta, eps, norm_eps;
@@ -77,6 +79,14 @@ struct ImState {
   float* pend_w;    // [U][F]
   int32_t* ctr;     // [U][CTR_STRIDE]
   int32_t* status;  // [1]
+  // a retained set per KV head (ImDims::scorer != 0): row = (u * Hkv + h)
+  int32_t* hpos;       // [U][Hkv][cap]  position held by a slot of the head's slab
+  float* hscore;       // [U][Hkv][cap]  the head's score of that entry
+  int32_t* hsel_pos;   // [U][Hkv][cap]  what the head's latest selection chose among
+  float* hsel_score;   // [U][Hkv][cap]
+  int32_t* hev_slot;   // [U][Hkv][tail] slots the head evicted in the latest compression, ascending
+  int32_t* hev_pos;    // [U][Hkv][tail] their positions
+  uint8_t* hkeep;      // [U][Hkv][cap]
 };
 
 struct ImWeights {  // one layer
@@ -119,6 +129,11 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
   float* bpart;      // [pack_k / 32][dM] sums of phi^2 over the 32 entries of a block of the packed operands
   float* mch;        // [max_seqs][max_chunk][Dkv] gated memory readout of a chunk's own queries (im_prefill_chunk_attend)
   uint8_t* qpack;    // [n_seq][ceil(C / IM_TC_QT)][IM_TC_TILE_BYTES] query operand of the tensor-core prefill scoring
+  // a retained set per KV head
+  int32_t* hsurv;    // [max_seqs][Hkv][tail] retained entries above the budget, ascending, per head
+  int32_t* hnhole;   // [max_seqs][Hkv]       holes below the budget per head
+  int32_t* hrowmap;  // [max_seqs][Hkv][tail] row of the memory write that an evicted (head, entry) pair belongs to
+  int32_t* hntok;    // [max_seqs]            rows (tokens that lose a slice) of the evict step
 };
 
 struct ImCall {
@@ -221,6 +236,14 @@ cudaError_t im_front_prepare_decode();
 cudaError_t im_prefetch_prepare_decode();
 
 #define IM_MRES_ROW(p) ((p).Dkv + 4)
+#define IM_PH_MAX_PAIRS 16384 /* evicted (head, entry) pairs per sequence and evict step in per-head mode (sorted in shared memory) */
+// a retained set per KV head (im_perhead.cu)
+cudaError_t im_perhead_prepare(const ImDims& p);
+cudaError_t im_ph_launch_append(const ImLaunch& L, const ImCall& call, const void* k, const void* v);
+cudaError_t im_ph_launch_select(const ImLaunch& L, const ImCall& call, const float* ext, long long n_pos);
+cudaError_t im_ph_launch_assemble(const ImLaunch& L, const ImCall& call, int ne_max);
+cudaError_t im_ph_launch_mem_write(const ImLaunch& L, const ImCall& call);
+cudaError_t im_ph_launch_move(const ImLaunch& L, const ImCall& call);
 #define IM_TC_KSPLIT 4  /* K splits of the prefill projections on the tensor cores (chunks of up to 8192 vectors) */
 
 // Decode calls of few sequences split the SMs between the two kinds of work of a call: the streaming kernels

@@ -51,9 +51,9 @@ def test_workspace_bytes_and_validation(im):
 
 
 def test_config_struct_layout(im):
-    # 18 int32, 6 float, one uint64
-    assert C.sizeof(im.im_config) == 104
-    assert im.im_config.seed.offset == 96 and im.im_config.score_share.offset == 68
+    # 19 int32, 6 float, padding to 8, one uint64
+    assert C.sizeof(im.im_config) == 112
+    assert im.im_config.seed.offset == 104 and im.im_config.score_share.offset == 68 and im.im_config.scorer.offset == 72
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-device error path")
