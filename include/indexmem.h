@@ -260,6 +260,10 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        (k <= 6; D_kv a power of two of at most 1024 and d_M a multiple of 8192 / D_kv); 0 (default): by the
  *                        kernel built on plain loads, which serves every shape and schedule.  The two add the rows in different
  *                        orders (float32); both are within the stated tolerances.
+ *   IM_OPT_LAYER_OVERLAP 1 (default): in the concurrent schedule the attention kernel of a decode call on ANOTHER layer than
+ *                        the call before it on the same stream is launched as programmatic dependent of that call's last
+ *                        kernel: it requests its first cache tiles while that kernel still runs and waits for it before it
+ *                        touches anything else.  0: it is launched in plain stream order.
  *   IM_OPT_WAIT_LIMIT    (test aid) attempts of the bounded device-side waits in which a consumer waits for its copies to
  *                        arrive (TMA / bulk-copy rings of the decode attention kernels, the bulk-copy readout kernel and
  *                        the tcgen05 chunk attention kernel): 0 restores the default (2^22), k >= 1 allows k - 1 attempts,
@@ -275,7 +279,8 @@ typedef enum im_option {
   IM_OPT_PROFILE_TARGET = 3,
   IM_OPT_DECODE_TENSOR = 4,
   IM_OPT_READOUT_STAGES = 5,
-  IM_OPT_WAIT_LIMIT = 6
+  IM_OPT_WAIT_LIMIT = 6,
+  IM_OPT_LAYER_OVERLAP = 7
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 

@@ -239,11 +239,17 @@ struct im_ctx {
   int n_ctas = 1;                    // grid of the streaming attention kernel (SM count)
   int n_sm = 1;                      // SMs of the device
   // The last kernel this context put on a caller's stream, if that was the merge kernel of a concurrent decode
-  // call (which writes nothing but the call's output): only then may the next call's attention kernel be launched
-  // as its programmatic dependent and fetch cache tiles before that kernel has ended.  After a prefill call, an
-  // in-order decode call or a state import the stream's last kernel may have written the cache.
+  // call (which writes the call's output and fills the holes of layer `tail_layer`'s cache): only then, and only for
+  // another layer, may the next call's attention kernel be launched as its programmatic dependent and fetch cache
+  // tiles before that kernel has ended.  After a prefill call, an in-order decode call or a state import the stream's
+  // last kernel may have written any layer's cache.
   cudaStream_t tail_stream = nullptr;
   bool tail_is_merge = false;
+  int tail_layer = -1;
+  bool layer_overlap = true;         // IM_OPT_LAYER_OVERLAP
+#ifdef IM_TRACE
+  int tune[8] = {0, -1, -1, 0, 0, 0, 0, 0};  // development builds: knobs set through options 100 + k
+#endif
   bool score_tc = false;             // prefill scoring runs on the tensor cores (tcgen05)
   bool attend_tc = true;             // chunk attention of im_prefill_chunk_attend on tcgen05 where head_dim is 128
   int prof_target = 0;               // kernel timed by im_profile_*: 0 attention (decode), 1 prefill scoring
@@ -285,6 +291,7 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
   call->pack = 0;
   call->defer = 0;
   call->fold_all = 0;
+  for (int k = 0; k < 5; ++k) { call->warm[k] = nullptr; call->warm_bytes[k] = 0; }
   return IM_OK;
 }
 
@@ -340,6 +347,7 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
   g.out_cnt = ne_max;
   g.out_inner = p.dM;
   g.tensor = (call.prefill || g.NV >= 1024) ? 1 : 0;  // thousands of evicted keys: the tensor-core variant
+  IM_TRACE_GEMM(g, L, call.layer, 2);
   if (ne_max > p.F) {
     call.phi_large = 1;
     g.out = L.sc.phi;
@@ -547,6 +555,14 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
   ctx->cfg = c;
   ctx->p = p;
   carve(p, (char*)dev_workspace, &ctx->lo);
+#ifdef IM_TRACE
+  {
+    void* tr = nullptr;
+    const size_t bytes = (size_t)p.L * IM_TRACE_KERNELS * IM_TRACE_MARKS * 8;
+    if (cudaMalloc(&tr, bytes) == cudaSuccess) cudaMemset(tr, 0, bytes);
+    ctx->lo.sc.trace = (unsigned long long*)tr;
+  }
+#endif
   if (ctx->lo.total > workspace_bytes) {
     size_t need = ctx->lo.total;
     delete ctx;
@@ -917,6 +933,9 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   call.ksplit = pick_ksplit(p.D, IM_KSPLIT);
   call.ksplit_key = (p.D % (8 * IM_KSPLIT_KEY) == 0) ? IM_KSPLIT_KEY : 1;
   call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
+#ifdef IM_TRACE
+  if (ctx->tune[0] > 0) call.ksplit_phi = pick_ksplit(p.Dkv, ctx->tune[0]);
+#endif
   // Two schedules.
   //  (A) deferred compaction - the streaming attention kernel is available and the selection, if one is
   //      due, fits the fused front kernel: attention needs nothing of this call but q, so it starts at
@@ -928,15 +947,23 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   //        s1: indexer projections -> front (append, score, select, gather) -> phi of the evicted keys
   //            [-> memory write: not needed by the merge, it only has to end with the call]
   //        s2: phi(q) / gate projections -> (front kernel's blocks resident) -> phi(q)^T Mhat next to the attention kernel
-  //        s3: float64 key projection (needed by front) -> L2 prefetch for the next layer -> filling of the holes
-  //            (once front has listed them and the attention kernel has read the cache)
+  //        s3: float64 key projection (needed by front) -> L2 prefetch for the next layer
+  //      The holes of the cache are filled by the merge kernel (the front kernel has listed the moves; the attention
+  //      kernel has read the cache by then).
   //        s4: fold of the pending list (before front, which changes the counters, and before the readout) ->
   //            the readout terms that do not go through Mhat, over the memory as it is before the write
   //      With IM_OPT_CONCURRENCY off the same kernels run on s0 in an order that respects these arrows.
   //  (B) in order on s0, attention after the compaction: everything else (large evicted sets, budgets
   //      beyond the fused front kernel, head shapes without the streaming attention kernel).
+  {
+    const void* in[5] = {x, q_pre, q, k_new, v_new};
+    const size_t by[5] = {(size_t)p.D * 2, (size_t)p.D * 2, (size_t)p.D * 2, (size_t)p.Dkv * 2, (size_t)p.Dkv * 2};
+    for (int k = 0; k < 5; ++k) { call.warm[k] = in[k]; call.warm_bytes[k] = (unsigned)(by[k] * n_seq); }
+  }
   cudaStream_t s0 = (cudaStream_t)cuda_stream;
-  const bool after_merge = ctx->tail_is_merge && ctx->tail_stream == s0;
+  // (the merge kernel also fills the holes of ITS layer's cache, after its own wait: a programmatic dependent on the
+  // same layer would request tiles of that cache too early)
+  const bool after_merge = ctx->layer_overlap && ctx->tail_is_merge && ctx->tail_stream == s0 && ctx->tail_layer != layer;
   ctx->tail_is_merge = false;
   const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
   const bool defer = ctx->fast_attn && (!due || fused) && ne_max <= p.F;
@@ -960,14 +987,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     CK(cudaStreamWaitEvent(L4.stream, ctx->ev[0], 0));
   }
   const bool prof = ctx->prof_target == 0 && ctx->prof_used + 2 <= ctx->prof_ev.size();
-  // s4: fold (reads the counters of before the call; the readout reads the folded state); s3: key projection
-  if (mem_write) {
-    CKL(im_launch_mem_fold(L4, call));
-    if (conc) CK(cudaEventRecord(ctx->ev[7], L4.stream));
-  }
-  if (!follow) CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
-  if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // key projection done
-  // a0: projections as K-split partial sums: indexer part (Sec. 3.1 features) on s1 ...
+  // a0: projections as K-split partial sums: indexer part (Sec. 3.1 features) on s1, launched first: it heads the
+  // longest chain of the call ...
   ImRows r = im_rows(p);
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
@@ -987,7 +1008,22 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
   g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
   g.n_jobs = 2;
+  IM_TRACE_GEMM(g, L, layer, 3);
+  g.smem_floor = n_res > 0 ? IM_SMEM_HEAD : 0;  // on the SMs without an attention CTA: its loads are not queued behind a stream's
+#ifdef IM_TRACE
+  if (ctx->tune[1] >= 0) g.smem_floor = ctx->tune[1] * 1024;
+  g.trace_skip = ctx->tune[3];
+#endif
   if (!follow) CKL(im_launch_gemm(L1, g));  // (a layer that reuses another layer's scores has no indexer work)
+  g.smem_floor = 0;
+  IM_TRACE_GEMM_OFF(g);
+  // s3: key projection; s4: fold (reads the counters of before the call; the readout reads the folded state)
+  if (!follow) CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
+  if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // key projection done
+  if (mem_write) {
+    CKL(im_launch_mem_fold(L4, call));
+    if (conc) CK(cudaEventRecord(ctx->ev[7], L4.stream));
+  }
   // ... memory part (phi(q) of Eq. 5, gate logit of Eq. 4) on s2, followed by the readout
   if (p.mem) {
     g.job[0] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
@@ -1011,7 +1047,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     if (ctx->attn_tc) CKL(im_launch_attention_tc(L, call, ctx->mapK, ctx->mapV, ctx->mapK128, ctx->mapV128, q, n_ctas, n_res > 0 && after_merge ? 1 : 0));
     else CKL(im_launch_attention_fast(L, call, ctx->mapKs, ctx->mapVs, q, n_ctas, n_res > 0 && after_merge ? 1 : 0));
     if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s0));
-    CK(cudaEventRecord(ctx->ev[9], s0));  // the attention kernel has read the cache
+    CK(cudaEventRecord(ctx->ev[9], s0));  // the attention kernel has ended
   }
   // an evicted set larger than the pending list is accumulated into Mhat itself, which the readout reads
   const bool readout_early = !(mem_write && ne_max > p.F);
@@ -1028,7 +1064,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   // (with SMs set aside: ev[13] triggers when all blocks of the front kernel have begun to run)
   const bool front_started_ev = conc && n_res > 0;
   CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max, n_res > 0 ? IM_SMEM_FRONT : 0,
-                             front_started_ev ? ctx->ev[13] : nullptr));
+                             front_started_ev ? ctx->ev[13] : nullptr, conc && !follow ? 1 : 0));
   if (due && !fused) {
     CKL(im_launch_select(L1, call));
     if (ne_max > 0) CKL(im_launch_gather_move(L1, call, ne_max));
@@ -1070,13 +1106,21 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     Lp.w = ctx->lo.w[nxt.layer];
     CKL(im_launch_prefetch_layer(Lp, nxt));
   }
-  if (conc) {
-    // a4 (fill the holes, publish the entry count) once the front kernel has listed the moves and the attention
-    // kernel has read the cache: next to the merge, on the stream the key projection has long left
+  if (conc && ctx->prefetch_next && p.mem && n_res > 0) {
+    // Half of the next layer's memory matrices go into L2 while this call's merge runs: the streaming kernels have
+    // ended, nothing else asks for HBM, and the next call's readout then finds these rows in L2 while its attention
+    // kernel has the DRAM channels (measured: a step of the 32-layer benchmark takes 2.26 ms with half of each
+    // matrix, 2.30 ms with a quarter, 2.37 ms with none, 2.40 ms with all of it, which the streams evict again)
+    int eighths = IM_PREFETCH_MEM_EIGHTHS;
+#ifdef IM_TRACE
+    if (ctx->tune[2] >= 0) eighths = ctx->tune[2];
+#endif
+    ImCall nxt = call;
+    nxt.layer = (layer + 1) % p.L;
     CK(cudaStreamWaitEvent(L3.stream, ctx->ev[9], 0));
-    CKL(im_launch_decode_commit(L3, call));
-    CK(cudaEventRecord(ctx->ev[10], L3.stream));
+    CKL(im_launch_prefetch_memory(L3, nxt, eighths));
   }
+  if (conc) CK(cudaEventRecord(ctx->ev[10], L3.stream));  // s3 has to end with the call
   // a3: memory write (needs the gathered evicted pairs and the fold).  With deferred compaction the merge kernel
   // forms the readout of the state after the write from phi of the evicted keys, and the state update itself
   // follows off the critical path, after the readout kernels that want the state from before it.
@@ -1111,7 +1155,6 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     }
     CKL(im_launch_attention_merge(L, call, out, ctx->attn_tc ? n_ctas : n_ctas * IM_ATTN_WARPS,
                                   ctx->attn_tc ? IM_ATTN_TC_TILE : IM_ATTN_STREAM_TILE, ro_workers, q, k_new, v_new, conc ? 1 : 0));
-    if (defer && !conc) CKL(im_launch_decode_commit(L, call));
     if (conc) CK(cudaStreamWaitEvent(s0, ctx->ev[10], 0));
     if (conc) {  // the memory write only has to end with the call
       CK(cudaEventRecord(ctx->ev[5], L1.stream));
@@ -1125,8 +1168,17 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   if (prof) ctx->prof_used += 2;
   ctx->tail_is_merge = conc;
   ctx->tail_stream = s0;
+  ctx->tail_layer = layer;
   return IM_OK;
 }
+
+#ifdef IM_TRACE
+extern "C" int im_trace_read(im_ctx* ctx, unsigned long long* host, long long n) {
+  cudaDeviceSynchronize();
+  const long long have = (long long)ctx->p.L * IM_TRACE_KERNELS * IM_TRACE_MARKS;
+  return cudaMemcpy(host, ctx->lo.sc.trace, (size_t)std::min(n, have) * 8, cudaMemcpyDeviceToHost) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 int im_set_option(im_ctx* ctx, int option, int value) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
@@ -1150,6 +1202,10 @@ int im_set_option(im_ctx* ctx, int option, int value) {
       ctx->attn_tc = value != 0;
       ctx->tail_is_merge = false;
       return IM_OK;
+    case IM_OPT_LAYER_OVERLAP: ctx->layer_overlap = value != 0; return IM_OK;
+#ifdef IM_TRACE
+    case 100: case 101: case 102: case 103: case 104: case 105: case 106: case 107: ctx->tune[option - 100] = value; return IM_OK;
+#endif
     case IM_OPT_WAIT_LIMIT:
       if (value < 0) return fail(IM_ERR_ARG, "wait limit %d: 0 = default, k >= 1 = k - 1 attempts", value);
       ctx->p.wait_limit = value == 0 ? IM_WAIT_LIMIT : (uint32_t)(value - 1);

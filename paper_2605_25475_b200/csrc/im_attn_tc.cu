@@ -513,6 +513,7 @@ k_attn_stream_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // A wait that runs out does not leave the loop on its own (the other threads would wait for this one at the next
     // named barrier): it is recorded in `fail`, the abort flag makes every later wait of the CTA return at once,
     // and the threads leave together where the per-tile reduction shows the failure to all of them.
+    im_warm_inputs(call, blockIdx.x, tid, KT);  // (the first CTAs: one input tensor each)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (blockIdx.x == 0)  // what the merge kernel rebuilds the tile bookkeeping from
       for (int k = tid; k < call.n_seq; k += KT) sc.n_att[k] = sh->n[k];

@@ -192,6 +192,7 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   if (lane == 0) {
     for (int k = 0; k < STAGES && issued < run1; ++k) issue(issued++);
   }
+  im_warm_inputs(call, blockIdx.x, threadIdx.x, blockDim.x);  // (the first CTAs: one input tensor each)
   // Launched as a programmatic dependent (of the previous call's merge kernel, or of whatever precedes the call in
   // the caller's stream) the kernel may have come this far before that kernel has ended: the cache of this layer,
   // which the first tiles are being fetched from, is not that kernel's business, but the query rows may be its
@@ -555,10 +556,21 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
   const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int hh0 = min(warp, p.Gq - 1);  // the head this warp merges first (usually its only one)
+  IM_MARK(sc, call.layer, 1, 0);
   // ---- every load whose address depends on no other load is issued here, ahead of its use: this kernel is
   // on the critical path of the call and a dependent chain of loads costs a memory round trip per link
   const int ne_raw = st.ctr[u * CTR_STRIDE + CTR_NEVICT];
   const int ev_l = lane < IM_FRONT_MAX_NE ? st.ev_slot[u * p.tail + min(lane, p.tail - 1)] : -1;
+  // (deferred compaction) the moves the front kernel listed, and the entry counts the attention kernel ran over: the
+  // counts of before the call, which the front kernel left as CTR_NNEXT + CTR_NEVICT - 1 (CTR_N itself is advanced by
+  // this kernel further down)
+  const int nh_raw = call.defer ? sc.nhole[i] : 0;
+  const int surv_l = (call.defer && lane < IM_FRONT_MAX_NE) ? sc.surv[(size_t)i * p.tail + min(lane, p.tail - 1)] : 0;
+  auto count_before = [&](int k) {
+    const int32_t* c = st.ctr + ((size_t)call.layer * p.S + call.seq[k]) * CTR_STRIDE;
+    return max(0, min(c[CTR_NNEXT] + c[CTR_NEVICT] - 1, p.cap));
+  };
+  int na_lane = (call.defer && lane < call.n_seq) ? count_before(lane) : 0;
   const float* mr = sc.mres + (size_t)i * IM_MRES_ROW(p);
   // phi(q)^T Mhat: one vector per sequence (k_readout_cols), or - ro_workers > 0 - the partial vectors of the CTAs of
   // k_readout_stream whose runs of ro_cs chunks per sequence hold chunks of this sequence, added in CTA order
@@ -580,15 +592,20 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
     const bf16* evr = sc.evV + (size_t)i * p.tail * p.Dkv + h * DH;
     if (p.mem) { gate = mr[p.Dkv]; c_hat = mr[p.Dkv + 2]; den_old = mr[p.Dkv + 1]; }
     if (p.mem && call.defer) {  // slot 0 of the evicted entries' phi is read before the evicted count is known
+      float pk[4][IM_KSPLIT];  // (all requested before the first sum: one round trip)
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int m = tid + j * blockDim.x;
+        pq0[j] = m < p.dM ? sc.phiq[(size_t)i * p.dM + m] : 0.f;
+#pragma unroll
+        for (int ks = 0; ks < IM_KSPLIT; ++ks)
+          pk[j][ks] = (m < p.dM && ks < call.ksplit_phi) ? sc.phip[((size_t)ks * call.n_seq + i) * p.F * p.dM + m] : 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
         pf0[j] = 0.f;
-        pq0[j] = 0.f;
-        if (m < p.dM) {
-          for (int ks = 0; ks < call.ksplit_phi; ++ks) pf0[j] += sc.phip[((size_t)ks * call.n_seq + i) * p.F * p.dM + m];
-          pq0[j] = sc.phiq[(size_t)i * p.dM + m];
-        }
+#pragma unroll
+        for (int ks = 0; ks < IM_KSPLIT; ++ks) pf0[j] += pk[j][ks];
       }
     }
 #pragma unroll
@@ -659,32 +676,100 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
 #pragma unroll
     for (int k = 0; k < CPL; ++k) mcol[k] *= inv;
   }
+  // ---- a4 with deferred compaction: this block fills the holes of head h's slabs (block h == 0 also those of the
+  // index-key and position arrays).  The retained entries above the budget are read here, the holes are overwritten
+  // once the attention kernel, which streams the evicted entries like any other, has ended.
+  constexpr int MV = 4, DV = DH / 8;
+  IM_MARK(sc, call.layer, 1, 1);
+  uint4 mv[MV];
+  bf16 mx[MV];
+  int n_mv = 0, n_mx = 0, nh = 0, pos_surv = 0, n_next = 0;
+  int hole[MV], hole_x[MV], hole_p = 0;
+  bf16* Kw = st.Kc + (u * p.Hkv + h) * (size_t)p.cap * DH;
+  bf16* Vw = st.Vc + (u * p.Hkv + h) * (size_t)p.cap * DH;
+  if (call.defer) {
+    const int ne_c = min(ne_raw, min(p.tail, IM_FRONT_MAX_NE));
+    nh = ne_c > 0 ? max(0, min(nh_raw, ne_c)) : 0;
+    n_mv = nh * 2 * DV;
+    n_mx = h == 0 ? nh * p.dI : 0;
+#pragma unroll
+    for (int r = 0; r < MV; ++r) {
+      const int k = tid + r * blockDim.x;
+      const int j = min(k / (2 * DV), IM_FRONT_MAX_NE - 1), rem = k % (2 * DV);
+      const int sj = __shfl_sync(0xffffffffu, surv_l, j), ej = __shfl_sync(0xffffffffu, ev_l, j);
+      if (k < n_mv) {
+        mv[r] = reinterpret_cast<const uint4*>((rem < DV ? Kw : Vw) + (size_t)sj * DH)[rem % DV];
+        hole[r] = ej;
+      }
+      const int jx = min(k / p.dI, IM_FRONT_MAX_NE - 1);
+      const int sx = __shfl_sync(0xffffffffu, surv_l, jx), ex = __shfl_sync(0xffffffffu, ev_l, jx);
+      if (k < n_mx) {
+        mx[r] = st.kidx[(u * p.cap + sx) * p.dI + k % p.dI];
+        hole_x[r] = ex;
+      }
+    }
+    if (h == 0 && warp == 0) {
+      if (lane < nh) pos_surv = st.pos[u * p.cap + surv_l];
+      hole_p = ev_l;
+    }
+    if (h == 0 && tid == 0) n_next = st.ctr[u * CTR_STRIDE + CTR_NNEXT];
+  }
+  // ---- the tile bookkeeping of the attention kernel, rebuilt (lanes stride over the sequences).  With deferred
+  // compaction it needs nothing that the attention kernel writes and runs ahead of the wait.
+  long long pref = 0, total = 0;
+  int nt_i = 0, n_old = 0;
+  auto bookkeeping = [&]() {
+    for (int k0 = 0; k0 < call.n_seq; k0 += 32) {
+      const int k = k0 + lane;
+      int na = 0;
+      if (k0 == 0) na = na_lane;
+      else if (k < call.n_seq) na = call.defer ? count_before(k) : sc.n_att[k];
+      const int nk = (na + tile - 1) / tile;
+      // inclusive prefix over the 32 lanes
+      long long incl = (long long)nk * p.Hkv;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const long long v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (i >= k0 && i < k0 + 32) {
+        pref = total + __shfl_sync(0xffffffffu, incl, i - k0) - (long long)__shfl_sync(0xffffffffu, nk, i - k0) * p.Hkv;
+        nt_i = __shfl_sync(0xffffffffu, nk, i - k0);
+        n_old = __shfl_sync(0xffffffffu, na, i - k0);
+      }
+      total += __shfl_sync(0xffffffffu, incl, 31);
+    }
+  };
+  if (call.defer) bookkeeping();
+  IM_MARK(sc, call.layer, 1, 2);
   // ---- everything below reads what the attention kernel has written.  When this kernel was launched as its
   // programmatic dependent it may have started before that kernel ended: wait for it (and its writes) here.
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int na_lane = lane < call.n_seq ? sc.n_att[lane] : 0;
-  // ---- rebuild the tile bookkeeping of the attention kernel (lanes stride over the sequences)
-  long long pref = 0, total = 0;
-  int nt_i = 0, n_old = 0;
-  for (int k0 = 0; k0 < call.n_seq; k0 += 32) {
-    const int k = k0 + lane;
-    int na = 0;
-    if (k0 == 0) na = na_lane;
-    else if (k < call.n_seq) na = sc.n_att[k];
-    const int nk = (na + tile - 1) / tile;
-    // inclusive prefix over the 32 lanes
-    long long incl = (long long)nk * p.Hkv;
+  if (call.defer) {
+    // (the recomputation below reads the slabs too: never a hole with a weight, and no entry that is moved away)
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const long long v = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += v;
+    for (int r = 0; r < MV; ++r) {
+      const int k = tid + r * blockDim.x;
+      if (k < n_mv) {
+        const int rem = k % (2 * DV);
+        reinterpret_cast<uint4*>((rem < DV ? Kw : Vw) + (size_t)hole[r] * DH)[rem % DV] = mv[r];
+      }
+      if (k < n_mx) st.kidx[(u * p.cap + hole_x[r]) * p.dI + k % p.dI] = mx[r];
     }
-    if (i >= k0 && i < k0 + 32) {
-      pref = total + __shfl_sync(0xffffffffu, incl, i - k0) - (long long)__shfl_sync(0xffffffffu, nk, i - k0) * p.Hkv;
-      nt_i = __shfl_sync(0xffffffffu, nk, i - k0);
-      n_old = __shfl_sync(0xffffffffu, na, i - k0);
+    for (int k = tid + MV * blockDim.x; k < n_mx; k += blockDim.x) {  // (index keys wider than MV elements per thread)
+      const int32_t* evs = st.ev_slot + u * p.tail;
+      const int32_t* surv = sc.surv + (size_t)i * p.tail;
+      st.kidx[(u * p.cap + evs[k / p.dI]) * p.dI + k % p.dI] = st.kidx[(u * p.cap + surv[k / p.dI]) * p.dI + k % p.dI];
     }
-    total += __shfl_sync(0xffffffffu, incl, 31);
+    if (h == 0 && warp == 0 && lane < nh) st.pos[u * p.cap + hole_p] = pos_surv;
+    // the entry count the call leaves (nothing that runs next to this kernel reads it: the merge below works from
+    // the attention kernel's snapshot)
+    if (h == 0 && tid == 0) st.ctr[u * CTR_STRIDE + CTR_N] = n_next;
+  }
+  IM_MARK(sc, call.layer, 1, 3);
+  if (!call.defer) {
+    na_lane = lane < call.n_seq ? sc.n_att[lane] : 0;
+    bookkeeping();
   }
   n_old = max(0, min(n_old, p.cap - 1));  // with deferred compaction: the slot of the new token
   const long long WT = n_workers;  // runs the attention kernel cut the tiles into (warps or CTAs)
@@ -789,6 +874,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
     }
     if (!redo) store_head(L, res);
   }
+  IM_MARK(sc, call.layer, 1, 4);
   if (!call.defer) return;  // (block uniform)
   if (lane == 0) s_redo[warp] = redo ? 1 : 0;
   __syncthreads();
@@ -894,6 +980,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
       store_head(L, res);
     }
   }
+  IM_MARK(sc, call.layer, 1, 5);
 }
 
 

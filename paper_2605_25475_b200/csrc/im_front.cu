@@ -30,7 +30,9 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
                const bf16* __restrict__ v_new, int do_select, int key_slots) {
   extern __shared__ __align__(16) unsigned long long s_key[];
   __shared__ FrontShared sh;
-  float* s_q = reinterpret_cast<float*>(s_key + key_slots);
+  float* s_q = reinterpret_cast<float*>(s_key + key_slots);                         // [HI][dI], 16-byte aligned
+  double* s_pk = reinterpret_cast<double*>(s_q + ((p.HI * p.dI + 3) & ~3));         // [ksplit_key][dI] key partials
+  float* s_pf = reinterpret_cast<float*>(s_pk + IM_KSPLIT_KEY * p.dI);              // [ksplit][HI dI + HI] partials
   const int i = blockIdx.x, tid = threadIdx.x;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   int32_t* ctr = st.ctr + u * CTR_STRIDE;
@@ -43,6 +45,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   // no indexer key: the pooled importances are those the leading layer's selection saw in this step, slot by slot.
   const bool follow = call.lead >= 0;
   const size_t ul = follow ? (size_t)call.lead * p.S + call.seq[i] : u;
+  IM_MARK(sc, call.layer, 0, 0);
   // ---- issue the loads of the first batch of cached entries (they depend on nothing of this call)
   constexpr int EPT = 4;
   int n_lim = p.cap;  // entries a batch may read: the capacity until the count is known
@@ -59,10 +62,10 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
         if (DI > 0 && !follow) {
           const uint4* row = reinterpret_cast<const uint4*>(st.kidx + (u * p.cap + t) * dI);
 #pragma unroll
-          for (int c = 0; c < (DI > 0 ? DI / 8 : 1); ++c) kraw[e][c] = row[c];
+          for (int c = 0; c < (DI > 0 ? DI / 8 : 1); ++c) kraw[e][c] = im_ld_now_u4(row + c);
         }
-        imp_old[e] = follow ? NEG_INF : imp[t];
-        pos_old[e] = pos[t];
+        imp_old[e] = follow ? NEG_INF : im_ld_now_f32(imp + t);
+        pos_old[e] = im_ld_now_s32(pos + t);
       }
     }
   };
@@ -74,6 +77,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     return;
   }
   n_lim = n;
+  IM_MARK(sc, call.layer, 0, 1);
   // the new token's K / V rows (copied into slot n below): requested now, stored after the first barrier
   const int dv = p.d / 8;
   const bool kv_here = tid < p.Hkv * dv;
@@ -83,18 +87,39 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     knew_c = reinterpret_cast<const uint4*>(k_new + (size_t)i * p.Dkv + h * p.d)[c];
     vnew_c = reinterpret_cast<const uint4*>(v_new + (size_t)i * p.Dkv + h * p.d)[c];
   }
-  // ---- finish the projections: sum the K-split partials in a fixed order
+  // ---- finish the projections: sum the K-split partials in a fixed order.  Launched as programmatic dependent of
+  // the projection kernel this block may have come this far while that kernel still runs: wait for its partial sums.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  IM_MARK(sc, call.layer, 0, 2);
   if (!follow) {
-    for (int k = tid; k < nq; k += FRONT_THREADS) {
-      s_q[k] = im_raw_sum(p, sc, call, i, r.uq + k);
+    // every partial is requested before the first one is used (one memory round trip), staged in shared memory,
+    // then added in K-split order
+    const int nrow = nq + p.HI, n_pf = call.ksplit * nrow, n_pk = call.ksplit_key * p.dI;
+    auto raw_at = [&](int k) {
+      const int ks = k / nrow, row = k % nrow;
+      return sc.raw[((size_t)ks * call.n_seq + i) * p.R5 + (row < nq ? r.uq + row : r.g + (row - nq))];
+    };
+    auto key_at = [&](int k) { return sc.keyp[((size_t)(k / p.dI) * call.n_seq + i) * p.dI + k % p.dI]; };
+    for (int k0 = tid; k0 < max(n_pf, n_pk); k0 += 2 * FRONT_THREADS) {
+      const int k1 = k0 + FRONT_THREADS;
+      const float f0 = k0 < n_pf ? raw_at(k0) : 0.f, f1 = k1 < n_pf ? raw_at(k1) : 0.f;
+      const double d0 = k0 < n_pk ? key_at(k0) : 0.0, d1 = k1 < n_pk ? key_at(k1) : 0.0;
+      if (k0 < n_pf) s_pf[k0] = f0;
+      if (k1 < n_pf) s_pf[k1] = f1;
+      if (k0 < n_pk) s_pk[k0] = d0;
+      if (k1 < n_pk) s_pk[k1] = d1;
     }
-    for (int k = tid; k < p.HI; k += FRONT_THREADS) {
-      sh.alpha[k] = im_raw_sum(p, sc, call, i, r.g + k) * (1.0f / sqrtf((float)p.HI * (float)p.dI));
+    __syncthreads();
+    for (int k = tid; k < nrow; k += FRONT_THREADS) {
+      float v = 0.f;
+      for (int ks = 0; ks < call.ksplit; ++ks) v += s_pf[ks * nrow + k];
+      if (k < nq) s_q[k] = v;
+      else sh.alpha[k - nq] = v * (1.0f / sqrtf((float)p.HI * (float)p.dI));
     }
     for (int k = tid; k < p.dI; k += FRONT_THREADS) {
-      double s = 0.0;
-      for (int ks = 0; ks < call.ksplit_key; ++ks) s += sc.keyp[((size_t)ks * call.n_seq + i) * p.dI + k];
-      sh.kd[k] = s;
+      double v = 0.0;
+      for (int ks = 0; ks < call.ksplit_key; ++ks) v += s_pk[ks * p.dI + k];
+      sh.kd[k] = v;
     }
   }
   __syncthreads();
@@ -130,6 +155,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   }
   if (tid == 0) st.pos[u * p.cap + n] = T;
   __syncthreads();
+  IM_MARK(sc, call.layer, 0, 4);
   // ---- a1: A_t = sum_h alpha_h act(q_h . k_t), pooled by max into the importance.
   // Entries are handled in batches of EPT per thread; the loads of a batch are all issued before its
   // arithmetic (the first batch was issued before the feature finalisation above).
@@ -139,57 +165,9 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
   bool bad = false, layout_bad = false;
   for (int b0 = 0; b0 < n1; b0 += EPT * FRONT_THREADS) {
     if (b0 > 0) load_batch(b0);
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) {
-      const int t = b0 + e * FRONT_THREADS + tid;
-      if (t >= n1) continue;
-      if (follow) {
-        // the leading layer scored the same entries in the same slots (checked: same position in the same slot)
-        const int ps = (t == n) ? T : pos_old[e];
-        if (due) {
-          const float pooled = st.sel_imp[ul * p.cap + t];
-          if (st.sel_pos[ul * p.cap + t] != ps) layout_bad = true;
-          st.sel_pos[u * p.cap + t] = ps;
-          st.sel_imp[u * p.cap + t] = pooled;
-          if (select_here) {
-            s_key[t] = im_select_key(pooled, ps, p.n_sink);
-            imp[t] = NEG_INF;
-          } else {
-            imp[t] = pooled;
-          }
-        }
-        continue;
-      }
-      float kk[DI > 0 ? DI : 64];
-      if (t == n) {
-#pragma unroll
-        for (int k = 0; k < dI; ++k) kk[k] = sh.knew[k];
-      } else if (DI > 0) {
-#pragma unroll
-        for (int c = 0; c < (DI > 0 ? DI / 8 : 1); ++c) {
-          const uint32_t ww[4] = {kraw[e][c].x, kraw[e][c].y, kraw[e][c].z, kraw[e][c].w};
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            kk[c * 8 + 2 * k] = __uint_as_float(ww[k] << 16);
-            kk[c * 8 + 2 * k + 1] = __uint_as_float(ww[k] & 0xffff0000u);
-          }
-        }
-      } else {
-        const bf16* row = st.kidx + (u * p.cap + t) * dI;
-        for (int k = 0; k < dI; ++k) kk[k] = __bfloat162float(row[k]);
-      }
-      float A = 0.f;
-      for (int h = 0; h < p.HI; ++h) {
-        float z = 0.f;
-#pragma unroll
-        for (int k = 0; k < dI; ++k) z = fmaf(s_q[h * dI + k], kk[k], z);
-        if (p.act == 0) z = fmaxf(z, 0.f);
-        A = fmaf(sh.alpha[h], z, A);
-      }
-      bad |= !isfinite(A);
-      const float pooled = fmaxf((t == n) ? NEG_INF : imp_old[e], A);
+    auto publish = [&](int e, int t, float pooled) {  // what the selection sees (parity export), then the pooling restarts
       const int ps = (t == n) ? T : pos_old[e];
-      if (due) {  // what the selection sees (parity export), then the pooling restarts
+      if (due) {
         st.sel_pos[u * p.cap + t] = ps;
         st.sel_imp[u * p.cap + t] = pooled;
       }
@@ -199,10 +177,93 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
       } else {
         imp[t] = pooled;
       }
+    };
+    if (follow) {
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const int t = b0 + e * FRONT_THREADS + tid;
+        if (t >= n1) continue;
+        // the leading layer scored the same entries in the same slots (checked: same position in the same slot)
+        const int ps = (t == n) ? T : pos_old[e];
+        if (due) {
+          const float pooled = st.sel_imp[ul * p.cap + t];
+          if (st.sel_pos[ul * p.cap + t] != ps) layout_bad = true;
+          publish(e, t, pooled);
+        }
+      }
+      continue;
+    }
+    // two entries at a time: a head's query features are read from shared memory once (as 16-byte words) for both
+#pragma unroll
+    for (int e0 = 0; e0 < EPT; e0 += 2) {
+      constexpr int KD = DI > 0 ? DI : 64;
+      float kk[2][KD];
+      int tt[2];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int e = e0 + j, t = b0 + e * FRONT_THREADS + tid;
+        tt[j] = t;
+        if (t == n) {
+#pragma unroll
+          for (int k = 0; k < dI; ++k) kk[j][k] = sh.knew[k];
+        } else if (DI > 0) {
+#pragma unroll
+          for (int c = 0; c < (DI > 0 ? DI / 8 : 1); ++c) {
+            const uint32_t ww[4] = {kraw[e][c].x, kraw[e][c].y, kraw[e][c].z, kraw[e][c].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              kk[j][c * 8 + 2 * k] = __uint_as_float(ww[k] << 16);
+              kk[j][c * 8 + 2 * k + 1] = __uint_as_float(ww[k] & 0xffff0000u);
+            }
+          }
+        } else if (t < n1) {
+          const bf16* row = st.kidx + (u * p.cap + t) * dI;
+          for (int k = 0; k < dI; ++k) kk[j][k] = __bfloat162float(row[k]);
+        }
+      }
+      if (tt[0] >= n1) continue;  // (then tt[1] >= n1 as well)
+      float A[2] = {0.f, 0.f};
+      for (int h = 0; h < p.HI; ++h) {
+        float z[2] = {0.f, 0.f};
+        if (DI > 0) {
+          const float4* q4 = reinterpret_cast<const float4*>(s_q + h * dI);
+#pragma unroll
+          for (int c = 0; c < (DI > 0 ? DI / 4 : 1); ++c) {
+            const float4 qv = q4[c];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              z[j] = fmaf(qv.x, kk[j][4 * c], z[j]);
+              z[j] = fmaf(qv.y, kk[j][4 * c + 1], z[j]);
+              z[j] = fmaf(qv.z, kk[j][4 * c + 2], z[j]);
+              z[j] = fmaf(qv.w, kk[j][4 * c + 3], z[j]);
+            }
+          }
+        } else {
+          for (int k = 0; k < dI; ++k) {
+            const float qv = s_q[h * dI + k];
+            z[0] = fmaf(qv, kk[0][k], z[0]);
+            z[1] = fmaf(qv, kk[1][k], z[1]);
+          }
+        }
+        const float al = sh.alpha[h];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          if (p.act == 0) z[j] = fmaxf(z[j], 0.f);
+          A[j] = fmaf(al, z[j], A[j]);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int e = e0 + j, t = tt[j];
+        if (t >= n1) continue;
+        bad |= !isfinite(A[j]);
+        publish(e, t, fmaxf((t == n) ? NEG_INF : imp_old[e], A[j]));
+      }
     }
   }
   if (bad) atomicOr(st.status, ST_NONFINITE);
   if (layout_bad) atomicOr(st.status, ST_LAYOUT);
+  IM_MARK(sc, call.layer, 0, 5);
   if (!select_here) {
     // either not due, or the selection runs in the kernels that follow (they read imp / pos)
     if (tid == 0) {
@@ -244,6 +305,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     }
     __syncthreads();
   }
+  IM_MARK(sc, call.layer, 0, 6);
   if (tid == 0) {
     // ascending slot order; holes below the budget pair with the retained entries above it
     for (int a = 1; a < ne; ++a) {
@@ -272,6 +334,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     }
   }
   __syncthreads();
+  IM_MARK(sc, call.layer, 0, 7);
   // ---- gather the evicted pairs for the memory write (a3) and, in the same pass, a4: a hole below
   // the budget (the first nh evicted slots) receives the retained entry found above it.  A thread
   // reads the evicted chunk before it overwrites it; the sources of the moves are never written.
@@ -292,6 +355,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     reinterpret_cast<uint4*>(sc.evV + dst)[c] = ve;
     if (e < nh) { *krow = ks; *vrow = vs; }
   }
+  IM_MARK(sc, call.layer, 0, 8);
   for (int k = tid; k < nh * p.dI; k += FRONT_THREADS) {
     const int j = k / p.dI, c = k % p.dI;
     st.kidx[(u * p.cap + sh.ev[j]) * p.dI + c] = st.kidx[(u * p.cap + sh.surv[j]) * p.dI + c];
@@ -305,6 +369,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
     ctr[CTR_NEVICT] = ne;
     if (ne > 0) ctr[CTR_EVSTEPS] = ctr[CTR_EVSTEPS] + 1;
   }
+  IM_MARK(sc, call.layer, 0, 9);
 }
 
 // Stand-alone versions for large evicted sets (after k_select): gather the evicted pairs, then move
@@ -333,9 +398,6 @@ __global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, Im
   const int i = blockIdx.y;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int ne = min(st.ctr[u * CTR_STRIDE + CTR_NEVICT], p.tail);
-  // deferred compaction: this kernel also publishes the entry count the call leaves (no kernel that runs next to
-  // it reads CTR_N: the merge kernel works from the attention kernel's snapshot)
-  if (call.defer && blockIdx.x == 0 && threadIdx.x == 0) st.ctr[u * CTR_STRIDE + CTR_N] = st.ctr[u * CTR_STRIDE + CTR_NNEXT];
   if (ne <= 0) return;
   const int nh = min(sc.nhole[i], ne);
   const int j0 = blockIdx.x * 4;
@@ -361,8 +423,10 @@ __global__ void __launch_bounds__(256) k_move_survivors(ImDims p, ImState st, Im
 
 // `started`: an event (timing disabled) that triggers once every block of the kernel has begun to run; a stream that
 // waits for it launches its next kernel when this kernel's blocks are resident, not when they have ended.
+// `programmatic`: the kernel before this one in the stream releases its dependents early; this kernel's blocks then read
+// the cache, the counters and the new token's K / V while it still runs, and wait for it before they read its output.
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
-                                   int do_select, int n_max, int smem_floor, cudaEvent_t started) {
+                                   int do_select, int n_max, int smem_floor, cudaEvent_t started, int programmatic) {
   static bool attr_done_dev[64] = {};
   bool* attr_done = im_device_flag(attr_done_dev);
   if (!attr_done || !*attr_done) {
@@ -372,8 +436,9 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
     if (e != cudaSuccess) return e;
     if (attr_done) *attr_done = true;
   }
-  const int key_slots = do_select ? n_max : 0;
-  size_t smem = (size_t)key_slots * 8 + (size_t)L.p.HI * L.p.dI * 4;
+  const int key_slots = do_select ? (n_max + 1) & ~1 : 0;  // (even: what follows the keys is 16-byte aligned)
+  size_t smem = (size_t)key_slots * 8 + (size_t)((L.p.HI * L.p.dI + 3) & ~3) * 4 + (size_t)IM_KSPLIT_KEY * L.p.dI * 8 +
+                (size_t)IM_KSPLIT * (L.p.HI * L.p.dI + L.p.HI) * 4;
   if (smem < (size_t)smem_floor) smem = (size_t)smem_floor;  // keeps the streaming kernels' blocks off this block's SM
   const bf16* kn = (const bf16*)k_new;
   const bf16* vn = (const bf16*)v_new;
@@ -383,30 +448,28 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
   cfg.blockDim = dim3(FRONT_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = L.stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
+  int na = 0;
   if (started) {
-    attr[0].id = cudaLaunchAttributeProgrammaticEvent;
-    attr[0].val.programmaticEvent.event = started;
-    attr[0].val.programmaticEvent.flags = 0;
-    attr[0].val.programmaticEvent.triggerAtBlockStart = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    attr[na].id = cudaLaunchAttributeProgrammaticEvent;
+    attr[na].val.programmaticEvent.event = started;
+    attr[na].val.programmaticEvent.flags = 0;
+    attr[na].val.programmaticEvent.triggerAtBlockStart = 1;
+    ++na;
   }
+  if (programmatic) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
   cudaError_t e;
   if (L.p.dI == 16) e = cudaLaunchKernelEx(&cfg, k_decode_front<16>, L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
   else if (L.p.dI == 8) e = cudaLaunchKernelEx(&cfg, k_decode_front<8>, L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
   else e = cudaLaunchKernelEx(&cfg, k_decode_front<0>, L.p, L.st, L.sc, call, kn, vn, do_select, key_slots);
   ++*L.launches;
   return e != cudaSuccess ? e : cudaGetLastError();
-}
-
-// deferred compaction (a4): fills the holes and publishes the entry count once the attention kernel has read the
-// cache; may run next to the merge kernel, which reads neither the evicted slots nor CTR_N
-cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call) {
-  dim3 grid((IM_FRONT_MAX_NE + 3) / 4, call.n_seq);
-  k_move_survivors<<<grid, 256, 0, L.stream>>>(L.p, L.st, L.sc, call);
-  ++*L.launches;
-  return cudaGetLastError();
 }
 
 // gather of the evicted pairs / move of the retained entries into the holes: every gather must be done before a

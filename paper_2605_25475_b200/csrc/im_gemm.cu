@@ -144,6 +144,9 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
   // the warps' partial tiles are added through shared memory in two rounds of four warps (half the buffer: the block
   // fits next to a streaming attention CTA that leaves 12 KB of an SM's shared memory), in warp order: deterministic
   __shared__ float red[DG_WARPS / 2][16][33];
+  // a kernel launched as programmatic dependent of this one may start its own preamble now
+  asm volatile("griddepcontrol.launch_dependents;");
+  IM_MARK_GEMM(a, 0);
   int tile = blockIdx.x, j = 0;
   while (j + 1 < a.n_jobs && tile >= (a.job[j].rows + 15) / 16) {
     tile -= (a.job[j].rows + 15) / 16;
@@ -163,6 +166,10 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
   const bf16* xb[4];
 #pragma unroll
   for (int nt = 0; nt < 4; ++nt) xb[nt] = vec_ptr(a, job.in_sel, min(v0 + nt * 8 + g, (long long)a.NV - 1)) + kbeg + 8 * t;
+#ifdef IM_TRACE
+  if (a.trace_skip & 4)  // timing experiment: the vectors are read from the (L2-resident) weights instead
+    for (int nt = 0; nt < 4; ++nt) xb[nt] = job.W + (size_t)min(nt * 8 + g, job.rows - 1) * a.K + kbeg + 8 * t;
+#endif
   float acc[4][4];
 #pragma unroll
   for (int nt = 0; nt < 4; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
@@ -178,6 +185,9 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
 #pragma unroll
       for (int d = 0; d < DG_DEPTH; ++d) {
         const int c = c0 + DG_WARPS * d;
+#ifdef IM_TRACE
+        if (a.trace_skip & 1) { fa[term][d] = zero4; fb[term][d] = zero4; continue; }
+#endif
         fa[term][d] = c < n_chunks ? ldg128_now(wa + c * 32) : zero4;
         fb[term][d] = c < n_chunks ? ldg128_now(wb + c * 32) : zero4;
       }
@@ -187,7 +197,12 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
     for (int d = 0; d < DG_DEPTH; ++d) {
       const int c = c0 + DG_WARPS * d;
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt) fx[d][nt] = c < n_chunks ? ldg128_now(xb[nt] + c * 32) : zero4;
+      for (int nt = 0; nt < 4; ++nt) {
+#ifdef IM_TRACE
+        if (a.trace_skip & 2) { fx[d][nt] = zero4; continue; }
+#endif
+        fx[d][nt] = c < n_chunks ? ldg128_now(xb[nt] + c * 32) : zero4;
+      }
     }
     asm volatile("" ::: "memory");  // every load of the batch is issued before the first MMA: one round trip
 #pragma unroll
@@ -207,6 +222,7 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
       }
     }
   }
+  IM_MARK_GEMM(a, 1);
   // C fragment: rows g / g+8, columns 8 nt + 2t / + 1
   constexpr int ITEMS = 16 * VB / (DG_WARPS * 32);  // outputs per thread
   float sum[ITEMS];
@@ -234,6 +250,7 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
     }
     __syncthreads();
   }
+  IM_MARK_GEMM(a, 2);
   float* outk = a.out + (size_t)ks * a.ks_stride;
 #pragma unroll
   for (int k = 0; k < ITEMS; ++k) {
@@ -243,6 +260,7 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
     if (v < a.NV && r0 + r < job.rows)
       outk[(v / a.out_cnt) * a.out_outer + (v % a.out_cnt) * a.out_inner + job.row0 + r0 + r] = sum[k];
   }
+  IM_MARK_GEMM(a, 3);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -416,7 +434,7 @@ cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, i
 cudaError_t im_gemm_prepare_decode() {
   cudaError_t e = im_prefer_max_smem(k_direct_gemm<false>);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_direct_gemm<true>);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_direct_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_SIDE);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_direct_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_HEAD);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_direct_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, IM_SMEM_SIDE);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_skinny_gemm);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_proj_key_split);

@@ -134,7 +134,27 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
   int32_t* hnhole;   // [max_seqs][Hkv]       holes below the budget per head
   int32_t* hrowmap;  // [max_seqs][Hkv][tail] row of the memory write that an evicted (head, entry) pair belongs to
   int32_t* hntok;    // [max_seqs]            rows (tokens that lose a slice) of the evict step
+#ifdef IM_TRACE
+  unsigned long long* trace;  // [n_layers][IM_TRACE_KERNELS][IM_TRACE_MARKS] nanosecond time stamps (development builds)
+#endif
 };
+
+// Development aid, compiled out of the library build: with IM_TRACE defined, thread 0 of block (0, 0) of an instrumented
+// kernel writes the global nanosecond timer at its marks; im_trace_read() copies the stamps to the host.
+#define IM_TRACE_KERNELS 8
+#define IM_TRACE_MARKS 16
+#ifdef IM_TRACE
+#define IM_MARK(sc_, layer_, kern_, mark_)                                                                      \
+  do {                                                                                                          \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {                                               \
+      unsigned long long t_;                                                                                    \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                                    \
+      (sc_).trace[((size_t)(layer_) * IM_TRACE_KERNELS + (kern_)) * IM_TRACE_MARKS + (mark_)] = t_;             \
+    }                                                                                                           \
+  } while (0)
+#else
+#define IM_MARK(sc_, layer_, kern_, mark_) do {} while (0)
+#endif
 
 struct ImCall {
   int layer, n_seq, C;
@@ -150,8 +170,21 @@ struct ImCall {
   int ksplit, ksplit_key, ksplit_phi;  // K splits of the projections / key projection / phi partials of this call
   int lead;       // >= 0: the layer whose pooled importances this call's layer reuses instead of scoring with an
                   // indexer of its own (App. B); that layer has already made this call for the same sequences
+  // decode: the call's input tensors (x, q_pre, q, k_new, v_new; null entries are skipped) and their size in bytes.
+  // The attention kernel, which may start before the kernel ahead of it in the stream has ended, requests them into L2
+  // at once: where the caller keeps them resident in HBM the call's latency-bound kernels would each pay a DRAM round
+  // trip behind the streams' queued requests (about 7 us against 2 us for a line found in L2).  A line that its
+  // producer has yet to write is simply written later: L2 is where the device's writes meet.
+  const void* warm[5];
+  unsigned warm_bytes[5];
   int seq[IM_MAX_CALL_SEQS];
 };
+__device__ __forceinline__ void im_warm_inputs(const ImCall& call, int part, int tid, int nthreads) {
+  if (part >= 5 || !call.warm[part]) return;
+  const char* b = static_cast<const char*>(call.warm[part]);
+  for (size_t off = (size_t)tid * 128; off < call.warm_bytes[part]; off += (size_t)nthreads * 128)
+    asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(b + off));
+}
 
 // Skinny GEMM arguments: out[v][row0 + r] (+)= sum_k (W[r][k] + W2[r][k]) * in[v][k].
 // Vector v of input set s starts at in[s] + (v / in_cnt[s]) * in_outer[s] + (v % in_cnt[s]) * in_inner[s]
@@ -197,7 +230,20 @@ struct ImGemmArgs {
   float alpha, beta;
   const int32_t* gate;  // if set, nothing is stored unless *gate > gate_min (a device-side counter decides)
   int gate_min;
+#ifdef IM_TRACE
+  ImScratch trace_sc;  // development builds: where IM_MARK writes (trace_sc.trace == nullptr: nowhere)
+  int trace_layer, trace_kern, trace_skip;
+#endif
 };
+#ifdef IM_TRACE
+#define IM_MARK_GEMM(a_, mark_) do { if ((a_).trace_sc.trace && blockIdx.z == 0) IM_MARK((a_).trace_sc, (a_).trace_layer, (a_).trace_kern, mark_); } while (0)
+#define IM_TRACE_GEMM(g_, L_, layer_, kern_) do { (g_).trace_sc = (L_).sc; (g_).trace_layer = (layer_); (g_).trace_kern = (kern_); } while (0)
+#define IM_TRACE_GEMM_OFF(g_) do { (g_).trace_sc.trace = nullptr; } while (0)
+#else
+#define IM_MARK_GEMM(a_, mark_) do {} while (0)
+#define IM_TRACE_GEMM(g_, L_, layer_, kern_) do {} while (0)
+#define IM_TRACE_GEMM_OFF(g_) do {} while (0)
+#endif
 
 #define IM_NOALLOC_MAX_FLOATS (1u << 20) /* floats in the built-in scratch array of im_attention_noalloc (4 MiB) */
 #define IM_KSPLIT 4       /* K splits of the decode projections (partials summed by the consumer) */
@@ -258,6 +304,9 @@ cudaError_t im_ph_launch_move(const ImLaunch& L, const ImCall& call);
 // kernel has just freed.
 #define IM_SMEM_FRONT (192 * 1024)   /* front block: excludes attention CTAs (>= 64 KB of shared memory each) */
 #define IM_SMEM_SIDE (38 * 1024)     /* phi GEMM block (+ 17 KB static): four per free SM, at most one next to an attention CTA */
+#define IM_PREFETCH_MEM_EIGHTHS 4   /* eighths of the next layer's memory matrices requested into L2 at the end of a decode call */
+#define IM_SMEM_HEAD (100 * 1024)    /* indexer projection block, which heads the call's longest chain: two per free SM, none next
+                                        to an attention CTA (which leaves 96 KB of an SM's shared memory) */
 inline int im_reserved_sms(int n_sm, int n_seq) { return n_seq <= n_sm / 4 ? n_seq : 0; }
 
 // records `msg` as the calling thread's last error and returns `code` (defined next to im_last_error)
@@ -270,12 +319,12 @@ bool im_tc_gemm_usable(const ImGemmArgs& a);
 cudaError_t im_launch_tc_gemm(const ImLaunch& L, const ImGemmArgs& a);
 cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, int ksplit);
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
-                                   int do_select, int n_max, int smem_floor, cudaEvent_t started = nullptr);
+                                   int do_select, int n_max, int smem_floor, cudaEvent_t started = nullptr, int programmatic = 0);
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call);
+cudaError_t im_launch_prefetch_memory(const ImLaunch& L, const ImCall& call, int eighths);
 cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_gather(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_move(const ImLaunch& L, const ImCall& call, int ne_max);
-cudaError_t im_launch_decode_commit(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call);
 // ne_host: per call sequence, the number of entries the compression of this call evicts (host mirror)
 cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_max, const int* ne_host);
@@ -342,6 +391,24 @@ __device__ __forceinline__ float im_raw_sum(const ImDims& p, const ImScratch& sc
   float s = 0.f;
   for (int ks = 0; ks < call.ksplit; ++ks) s += sc.raw[((size_t)ks * call.n_seq + i) * p.R5 + row];
   return s;
+}
+
+// Loads that the compiler may neither reorder nor delay to their first use: for values that are requested long before
+// they are needed, so that the round trip overlaps what lies in between.
+__device__ __forceinline__ uint4 im_ld_now_u4(const void* p) {
+  uint4 v;
+  asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float im_ld_now_f32(const float* p) {
+  float v;
+  asm volatile("ld.volatile.global.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ int im_ld_now_s32(const int32_t* p) {
+  int v;
+  asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
 }
 
 // ---- small device helpers

@@ -52,7 +52,25 @@ __global__ void __launch_bounds__(256) k_prefetch_layer(ImDims p, ImState st, Im
   }
 }
 
+// The memory matrices of layer `call.layer` (the NEXT layer) for the call's sequences, requested into L2 as bulk
+// prefetches of 4 KB: grid = (n_seq), block = 512; the first `eighths` eighths of each matrix.
+__global__ void __launch_bounds__(512) k_prefetch_memory(ImDims p, ImState st, ImCall call, int eighths) {
+  const size_t u = (size_t)call.layer * p.S + call.seq[blockIdx.x];
+  const size_t bytes = (size_t)p.dM * p.Dkv * 4 / 8 * eighths;
+  const char* base = reinterpret_cast<const char*>(st.Mhat + u * p.dM * p.Dkv);
+  for (size_t off = (size_t)threadIdx.x * 4096; off + 4096 <= bytes; off += (size_t)blockDim.x * 4096)
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(4096) : "memory");
+}
+
 }  // namespace
+
+// `call.layer` names the layer to warm up.  Needs 16-byte aligned matrices whose eighth is a multiple of 4 KB.
+cudaError_t im_launch_prefetch_memory(const ImLaunch& L, const ImCall& call, int eighths) {
+  if (!L.p.mem || eighths <= 0 || ((size_t)L.p.dM * L.p.Dkv * 4 / 8) % 4096) return cudaSuccess;
+  k_prefetch_memory<<<call.n_seq, 512, 0, L.stream>>>(L.p, L.st, call, eighths > 8 ? 8 : eighths);
+  ++*L.launches;
+  return cudaGetLastError();
+}
 
 // `L.w` and `call.layer` must describe the layer to warm up (not the one being computed).
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call) {
