@@ -1118,7 +1118,11 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     ImCall nxt = call;
     nxt.layer = (layer + 1) % p.L;
     CK(cudaStreamWaitEvent(L3.stream, ctx->ev[9], 0));
-    CKL(im_launch_prefetch_memory(L3, nxt, eighths));
+    int pm_blocks = 1;
+#ifdef IM_TRACE
+    if (ctx->tune[4] > 0) pm_blocks = ctx->tune[4];
+#endif
+    CKL(im_launch_prefetch_memory(L3, nxt, eighths, pm_blocks));
   }
   if (conc) CK(cudaEventRecord(ctx->ev[10], L3.stream));  // s3 has to end with the call
   // a3: memory write (needs the gathered evicted pairs and the fold).  With deferred compaction the merge kernel

@@ -222,6 +222,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
         }
       }
       if (tt[0] >= n1) continue;  // (then tt[1] >= n1 as well)
+      if (b0 == 0) IM_MARK(sc, call.layer, 0, 10 + e0);
       float A[2] = {0.f, 0.f};
       for (int h = 0; h < p.HI; ++h) {
         float z[2] = {0.f, 0.f};
@@ -252,6 +253,7 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
           A[j] = fmaf(al, z[j], A[j]);
         }
       }
+      if (b0 == 0) IM_MARK(sc, call.layer, 0, 11 + e0);
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int e = e0 + j, t = tt[j];

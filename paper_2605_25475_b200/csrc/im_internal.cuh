@@ -11,7 +11,9 @@ typedef __nv_bfloat16 bf16;
 #define IM_MAX_CALL_SEQS 256 /* sequences per hot call (the id list travels as a kernel parameter) */
 #define IM_SLOT_ALIGN 64     /* slot capacity is a multiple of the attention tile */
 #define IM_ATTN_TILE 32      /* rows of the small TMA box of the cache's tensor maps (32 rows x 128 bytes) */
+#ifndef IM_ATTN_STREAM_TILE
 #define IM_ATTN_STREAM_TILE 32 /* keys per tile (= rows of a TMA box) of the mma.sync streaming attention kernel */
+#endif
 #define IM_ATTN_WARPS 4      /* warps per CTA of the streaming attention kernel */
 #define IM_ATTN_TC_TILE 128  /* keys per tile of the tensor-core streaming attention kernel (= the TMEM lanes) */
 #define IM_ATTN_MAX_CTAS 512 /* upper bound of its grid (one CTA per SM) */
@@ -321,7 +323,7 @@ cudaError_t im_launch_proj_key_split(const ImLaunch& L, const void* x, int NV, i
 cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const void* k_new, const void* v_new,
                                    int do_select, int n_max, int smem_floor, cudaEvent_t started = nullptr, int programmatic = 0);
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call);
-cudaError_t im_launch_prefetch_memory(const ImLaunch& L, const ImCall& call, int eighths);
+cudaError_t im_launch_prefetch_memory(const ImLaunch& L, const ImCall& call, int eighths, int per_block = 1);
 cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_gather(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_move(const ImLaunch& L, const ImCall& call, int ne_max);

@@ -53,21 +53,27 @@ __global__ void __launch_bounds__(256) k_prefetch_layer(ImDims p, ImState st, Im
 }
 
 // The memory matrices of layer `call.layer` (the NEXT layer) for the call's sequences, requested into L2 as bulk
-// prefetches of 4 KB: grid = (n_seq), block = 512; the first `eighths` eighths of each matrix.
-__global__ void __launch_bounds__(512) k_prefetch_memory(ImDims p, ImState st, ImCall call, int eighths) {
-  const size_t u = (size_t)call.layer * p.S + call.seq[blockIdx.x];
+// prefetches of 4 KB, the first `eighths` eighths of each matrix.  grid = ceil(n_seq / per_block), block = 512.  An
+// SM's copy engine takes these requests at a bounded rate, so the number of blocks paces the whole prefetch: it is
+// meant to trickle in next to the merge kernel and the next call's projections, not to compete with them
+// (measured on the 32-layer benchmark: one block per sequence 2.24 ms per step, eight 2.33 ms).
+__global__ void __launch_bounds__(512) k_prefetch_memory(ImDims p, ImState st, ImCall call, int eighths, int per_block) {
   const size_t bytes = (size_t)p.dM * p.Dkv * 4 / 8 * eighths;
-  const char* base = reinterpret_cast<const char*>(st.Mhat + u * p.dM * p.Dkv);
-  for (size_t off = (size_t)threadIdx.x * 4096; off + 4096 <= bytes; off += (size_t)blockDim.x * 4096)
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(4096) : "memory");
+  for (int i = blockIdx.x * per_block; i < min(call.n_seq, (blockIdx.x + 1) * per_block); ++i) {
+    const size_t u = (size_t)call.layer * p.S + call.seq[i];
+    const char* base = reinterpret_cast<const char*>(st.Mhat + u * p.dM * p.Dkv);
+    for (size_t off = (size_t)threadIdx.x * 4096; off + 4096 <= bytes; off += (size_t)blockDim.x * 4096)
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(4096) : "memory");
+  }
 }
 
 }  // namespace
 
 // `call.layer` names the layer to warm up.  Needs 16-byte aligned matrices whose eighth is a multiple of 4 KB.
-cudaError_t im_launch_prefetch_memory(const ImLaunch& L, const ImCall& call, int eighths) {
+cudaError_t im_launch_prefetch_memory(const ImLaunch& L, const ImCall& call, int eighths, int per_block) {
   if (!L.p.mem || eighths <= 0 || ((size_t)L.p.dM * L.p.Dkv * 4 / 8) % 4096) return cudaSuccess;
-  k_prefetch_memory<<<call.n_seq, 512, 0, L.stream>>>(L.p, L.st, call, eighths > 8 ? 8 : eighths);
+  if (per_block <= 0) per_block = 1;
+  k_prefetch_memory<<<(call.n_seq + per_block - 1) / per_block, 512, 0, L.stream>>>(L.p, L.st, call, eighths > 8 ? 8 : eighths, per_block);
   ++*L.launches;
   return cudaGetLastError();
 }
