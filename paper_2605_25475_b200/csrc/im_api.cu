@@ -332,7 +332,7 @@ cudaError_t launch_mem_update(im_ctx* ctx, const ImLaunch& L, const ImCall& call
 // With `update` = false only the GEMM is launched (the caller launches im_launch_mem_update later).
 // `before_update`: an event that the kernels changing the memory state wait for (a reader of the state of before)
 int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, bool update = true, int smem_floor = 0,
-                     cudaEvent_t before_update = nullptr) {
+                     cudaEvent_t before_update = nullptr, int programmatic = 0) {
   const ImDims& p = ctx->p;
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
@@ -370,6 +370,7 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
     g.kc = 64;  // 18 KB of shared memory: fits next to the resident attention blocks
     g.direct = call.prefill ? 0 : 1;
     g.smem_floor = smem_floor;
+    g.programmatic = programmatic;
   }
   CKL(im_launch_gemm(L, g));
   if (update && before_update) CK(cudaStreamWaitEvent(L.stream, before_update, 0));
@@ -974,7 +975,17 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   const bool mem_write = due && ne_max > 0 && p.mem;
   // concurrent schedule: the SMs left to the latency-bound chain (see IM_SMEM_FRONT)
   const int n_res = conc ? im_reserved_sms(ctx->n_sm, n_seq) : 0;
-  const int n_ctas = n_res > 0 ? std::max(1, std::min(ctx->n_ctas, ctx->n_sm - n_res)) : ctx->n_ctas;
+  const int n_ctas_max = n_res > 0 ? std::max(1, std::min(ctx->n_ctas, ctx->n_sm - n_res)) : ctx->n_ctas;
+  // the attention grid: no more CTAs than give every warp a run of IM_ATTN_MIN_RUN tiles (a small call cut into
+  // one-tile runs leaves the merge kernel a long row of partial results to add per head)
+  int n_ctas = n_ctas_max;
+  if (!ctx->attn_tc) {
+    long long tiles = 0;
+    for (int i = 0; i < n_seq; ++i)
+      tiles += (long long)((ctx->hu[(size_t)layer * p.S + call.seq[i]].n + IM_ATTN_STREAM_TILE - 1) / IM_ATTN_STREAM_TILE) * p.Hkv;
+    const long long want = (tiles + IM_ATTN_WARPS * IM_ATTN_MIN_RUN - 1) / (IM_ATTN_WARPS * IM_ATTN_MIN_RUN);
+    n_ctas = (int)std::max<long long>(1, std::min<long long>(n_ctas_max, want));
+  }
   if (conc) {
     L1.stream = ctx->side[0];
     L2.stream = ctx->side[1];
@@ -1008,6 +1019,23 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
   g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
   g.n_jobs = 2;
+  // (the float64 key projection rides along in the same launch where its K range divides: the front kernel then
+  // depends on one kernel only and starts behind it as its programmatic dependent)
+  // (small calls only: in a large one the projection's blocks share the SMs set aside for the chain with the front
+  // blocks, which then find no room to start early)
+  int key_ride = 0;
+  if (conc && !follow && (p.dI == 8 || p.dI == 16) && (n_res == 0 || (long long)n_seq * (p.Dkv / 64) < ctx->n_sm - n_res))
+    for (int ks = 8; ks >= 1 && !key_ride; --ks)
+      if (p.D % (256 * ks) == 0) key_ride = ks;
+  if (key_ride) {
+    g.key_W = L.w.Uk;
+    g.key_x = (const bf16*)x;
+    g.key_out = L.sc.keyp;
+    g.key_nv = n_seq;
+    g.key_ksplit = key_ride;
+    g.key_dI = p.dI;
+    call.ksplit_key = key_ride;
+  }
   IM_TRACE_GEMM(g, L, layer, 3);
   g.smem_floor = n_res > 0 ? IM_SMEM_HEAD : 0;  // on the SMs without an attention CTA: its loads are not queued behind a stream's
 #ifdef IM_TRACE
@@ -1016,9 +1044,10 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
 #endif
   if (!follow) CKL(im_launch_gemm(L1, g));  // (a layer that reuses another layer's scores has no indexer work)
   g.smem_floor = 0;
+  g.key_W = nullptr;
   IM_TRACE_GEMM_OFF(g);
   // s3: key projection; s4: fold (reads the counters of before the call; the readout reads the folded state)
-  if (!follow) CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
+  if (!follow && !key_ride) CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
   if (conc) CK(cudaEventRecord(ctx->ev[2], L3.stream));  // key projection done
   if (mem_write) {
     CKL(im_launch_mem_fold(L4, call));
@@ -1063,8 +1092,12 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   // block per sequence; a4 in the same kernel unless the compaction is deferred)
   // (with SMs set aside: ev[13] triggers when all blocks of the front kernel have begun to run)
   const bool front_started_ev = conc && n_res > 0;
+  int front_pdl = conc && !follow ? 1 : 0;
+#ifdef IM_TRACE
+  if (ctx->tune[5]) front_pdl = 0;
+#endif
   CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max, n_res > 0 ? IM_SMEM_FRONT : 0,
-                             front_started_ev ? ctx->ev[13] : nullptr, conc && !follow ? 1 : 0));
+                             front_started_ev ? ctx->ev[13] : nullptr, front_pdl));
   if (due && !fused) {
     CKL(im_launch_select(L1, call));
     if (ne_max > 0) CKL(im_launch_gather_move(L1, call, ne_max));
@@ -1079,7 +1112,10 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   // registers leave no room for a readout block, so the readout runs beside the attention CTAs and the two streaming
   // kernels end together.
   if (conc) {
-    if (n_res > 0) {
+    // (a readout with fewer blocks than there are other SMs cannot keep the front blocks out: no need to hold it back)
+    const bool few_blocks = (long long)n_seq * (p.Dkv / 64) < ctx->n_sm - n_res;
+    if (n_res > 0 && few_blocks) {
+    } else if (n_res > 0) {
       CK(cudaStreamWaitEvent(L2.stream, front_started_ev ? ctx->ev[13] : ctx->ev[11], 0));
     } else {
       CK(cudaStreamWaitEvent(L2.stream, ctx->ev[1], 0));
@@ -1090,10 +1126,10 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   int ro_workers = 0;
   if (ctx->fast_attn && p.mem && readout_early) {
     if (conc && n_res > 0 && ctx->ro_stream) {
-      ro_workers = (int)std::min<long long>(n_ctas, (long long)n_seq * im_readout_stream_chunks(p));
+      ro_workers = (int)std::min<long long>(n_ctas_max, (long long)n_seq * im_readout_stream_chunks(p));
       CKL(im_launch_readout_stream(L2, call, ro_workers, ctx->ro_stages));
     } else {
-      CKL(im_launch_readout(L2, call, n_res > 0 ? n_ctas : ctx->n_sm, conc && n_res == 0));
+      CKL(im_launch_readout(L2, call, n_res > 0 ? n_ctas_max : ctx->n_sm, conc && n_res == 0));
     }
   }
   if (conc) CK(cudaEventRecord(ctx->ev[12], L2.stream));  // s2 finished: the merge needs phi(q)^T Mhat
@@ -1128,7 +1164,10 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   // a3: memory write (needs the gathered evicted pairs and the fold).  With deferred compaction the merge kernel
   // forms the readout of the state after the write from phi of the evicted keys, and the state update itself
   // follows off the critical path, after the readout kernels that want the state from before it.
-  if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, !defer, n_res > 0 ? IM_SMEM_SIDE : 0))) return rc;
+  // (a small call on an idle device: the phi GEMM starts behind the front kernel as its programmatic dependent; in a
+  // large one its blocks would wait on SMs that a streaming kernel keeps busy)
+  const bool phi_pdl = conc && fused && n_res > 0 && (long long)n_seq * (p.Dkv / 64) < ctx->n_sm - n_res;
+  if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, !defer, n_res > 0 ? IM_SMEM_SIDE : 0, nullptr, phi_pdl ? 1 : 0))) return rc;
   if (conc) CK(cudaEventRecord(ctx->ev[3], L1.stream));  // everything the merge needs from s1
   if (conc) CK(cudaStreamWaitEvent(L1.stream, ctx->ev[4], 0));  // k_readout_finish reads what the update changes
   if (defer && mem_write) CKL(launch_mem_update(ctx, L1, call, ne_max));

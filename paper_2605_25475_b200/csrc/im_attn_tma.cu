@@ -804,6 +804,30 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
     for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[k] * en;
     M = Mn;
   };
+  // the stored partials wa .. wb of a head, four at a time: their loads are all requested before the first is added
+  auto merge_stored_range = [&](long long wa, long long wb, int head, float& M, float& L, float (&res)[CPL]) {
+    for (long long w4 = wa; w4 <= wb; w4 += 4) {
+      float a[4][CPL], mw[4], lw[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float* ps = sc.part + ((size_t)(min(w4 + j, wb) + row_id) * p.Gq + head) * (DH + 2);
+        mw[j] = ps[DH];
+        lw[j] = ps[DH + 1];
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) a[j][k] = ps[lane + 32 * k];
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (w4 + j > wb) break;
+        const float Mn = fmaxf(M, mw[j]);
+        const float eo = exp2f(M - Mn), en = exp2f(mw[j] - Mn);  // exp2(-inf) = 0 for the first contributor
+        L = L * eo + lw[j] * en;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) res[k] = res[k] * eo + a[j][k] * en;
+        M = Mn;
+      }
+    }
+  };
   bool new_kept = true;
   for (int a = 0; a < ne; ++a) new_kept &= __shfl_sync(0xffffffffu, ev_l, a) != n_old;
   auto push_new = [&](float& M, float& L, float (&res)[CPL]) {
@@ -835,7 +859,7 @@ __global__ void __launch_bounds__(256, 1) k_attn_merge_rows(ImDims p, ImState st
 #pragma unroll
     for (int k = 0; k < CPL; ++k) res[k] = 0.f;
     float M = NEG_INF, L = 0.f;
-    for (long long wv = w0; wv <= w1; ++wv) merge_stored(wv, hh, M, L, res);
+    merge_stored_range(w0, w1, hh, M, L, res);
     if (call.defer) {
       push_new(M, L, res);
       float Lsub = 0.f, sub[CPL];

@@ -30,6 +30,8 @@ k_decode_front(ImDims p, ImState st, ImScratch sc, ImCall call, const bf16* __re
                const bf16* __restrict__ v_new, int do_select, int key_slots) {
   extern __shared__ __align__(16) unsigned long long s_key[];
   __shared__ FrontShared sh;
+  // a kernel launched as programmatic dependent of this one (phi of the evicted keys) may request its weights now
+  asm volatile("griddepcontrol.launch_dependents;");
   float* s_q = reinterpret_cast<float*>(s_key + key_slots);                         // [HI][dI], 16-byte aligned
   double* s_pk = reinterpret_cast<double*>(s_q + ((p.HI * p.dI + 3) & ~3));         // [ksplit_key][dI] key partials
   float* s_pf = reinterpret_cast<float*>(s_pk + IM_KSPLIT_KEY * p.dI);              // [ksplit][HI dI + HI] partials

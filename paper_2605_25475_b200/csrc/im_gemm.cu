@@ -137,16 +137,84 @@ __device__ __forceinline__ uint4 ldg128_now(const void* p) {
   asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
+__device__ __forceinline__ void dmma_884(double (&c)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(c[0]), "+d"(c[1]) : "d"(a), "d"(b));
+}
+__device__ __forceinline__ double bf16_elem(const uint4& v, int s) {
+  const uint32_t w = s < 2 ? v.x : s < 4 ? v.y : s < 6 ? v.z : v.w;
+  return (double)((s & 1) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16));
+}
+// One block's share of the float64 key projection (see k_proj_key_mma): block (bx, by) of a (ceil(NV / 8), ksplit)
+// grid, W warps, `red` = W * NT * 64 doubles of shared memory.
+template <int NT, int W>
+__device__ __forceinline__ void proj_key_mma_block(int D, int dI, const bf16* __restrict__ Uk, const bf16* __restrict__ x, int NV,
+                                                   int ksplit, double* __restrict__ keyp, int bx, int by, double* red) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, q = lane & 3;
+  const long long v0 = (long long)bx * 8;
+  const int kspan = D / (W * ksplit), kbeg = (by * W + warp) * kspan;  // a multiple of 32 (checked by the launcher)
+  keyp += (size_t)by * NV * dI;
+  const bf16* xrow = x + (size_t)min(v0 + r, (long long)NV - 1) * D + kbeg + 8 * q;
+  const bf16* urow = Uk + (size_t)r * D + kbeg + 8 * q;
+  double c[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = 0.0;
+  for (int kb = 0; kb < kspan; kb += 32) {
+    const uint4 xa = *reinterpret_cast<const uint4*>(xrow + kb);
+    uint4 ub[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) ub[nt] = *reinterpret_cast<const uint4*>(urow + (size_t)nt * 8 * D + kb);
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const double a = bf16_elem(xa, s);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) dmma_884(c[nt], a, bf16_elem(ub[nt], s));
+    }
+  }
+  // C fragment: row r (vector), columns 2 q and 2 q + 1 (weight row of the n-tile)
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    red[(warp * NT + nt) * 64 + r * 8 + 2 * q] = c[nt][0];
+    red[(warp * NT + nt) * 64 + r * 8 + 2 * q + 1] = c[nt][1];
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < NT * 64; idx += 32 * W) {
+    const int nt = idx >> 6, e = idx & 63;
+    const long long v = v0 + (e >> 3);
+    if (v < NV) {
+      double sum = red[nt * 64 + e];
+#pragma unroll
+      for (int w = 1; w < W; ++w) sum += red[(w * NT + nt) * 64 + e];
+      keyp[(size_t)v * dI + nt * 8 + (e & 7)] = sum;
+    }
+  }
+}
+
 constexpr int DG_DEPTH = 4;   // 32-wide chunks whose loads (weights and vectors) a warp has in flight
 constexpr int DG_WARPS = 8;
 template <bool TWO>  // TWO: the jobs have a second weight term
 __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
   // the warps' partial tiles are added through shared memory in two rounds of four warps (half the buffer: the block
   // fits next to a streaming attention CTA that leaves 12 KB of an SM's shared memory), in warp order: deterministic
-  __shared__ float red[DG_WARPS / 2][16][33];
+  constexpr int RED_BYTES = (DG_WARPS / 2) * 16 * 33 * 4 > DG_WARPS * 2 * 64 * 8 ? (DG_WARPS / 2) * 16 * 33 * 4 : DG_WARPS * 2 * 64 * 8;
+  __shared__ __align__(16) unsigned char red_raw[RED_BYTES];  // the float tiles below, or the key projection's doubles
+  float (*red)[16][33] = reinterpret_cast<float (*)[16][33]>(red_raw);
   // a kernel launched as programmatic dependent of this one may start its own preamble now
   asm volatile("griddepcontrol.launch_dependents;");
   IM_MARK_GEMM(a, 0);
+  if ((int)blockIdx.x >= a.tiles) {
+    // the float64 indexer-key projection of the same vectors, in the same launch (blocks behind the tiles' blocks)
+    if (blockIdx.z == 0) {
+      const int kid = ((int)blockIdx.x - a.tiles) * (int)gridDim.y + (int)blockIdx.y;
+      const int nbx = (a.key_nv + 7) / 8;
+      if (kid < nbx * a.key_ksplit) {
+        double* redd = reinterpret_cast<double*>(red_raw);
+        if (a.key_dI == 8) proj_key_mma_block<1, DG_WARPS>(a.K, 8, a.key_W, a.key_x, a.key_nv, a.key_ksplit, a.key_out, kid % nbx, kid / nbx, redd);
+        else proj_key_mma_block<2, DG_WARPS>(a.K, 16, a.key_W, a.key_x, a.key_nv, a.key_ksplit, a.key_out, kid % nbx, kid / nbx, redd);
+      }
+    }
+    return;
+  }
   int tile = blockIdx.x, j = 0;
   while (j + 1 < a.n_jobs && tile >= (a.job[j].rows + 15) / 16) {
     tile -= (a.job[j].rows + 15) / 16;
@@ -192,6 +260,8 @@ __global__ void __launch_bounds__(DG_WARPS * 32) k_direct_gemm(ImGemmArgs a) {
         fb[term][d] = c < n_chunks ? ldg128_now(wb + c * 32) : zero4;
       }
     }
+    // (the vectors may be the output of the kernel this one was launched behind as a programmatic dependent)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     uint4 fx[DG_DEPTH][4];
 #pragma unroll
     for (int d = 0; d < DG_DEPTH; ++d) {
@@ -322,56 +392,11 @@ __global__ void __launch_bounds__(256) k_proj_key_split(ImDims p, const bf16* __
 // grid = (ceil(NV / 8), ksplit), block = 32 W; D a multiple of 32 W ksplit, d_I = 8 NT.  Block (., ks) takes the ks-th
 // part of the K range and writes the partial sums keyp[ks][v][.] (decode: the few vectors of a step would leave all
 // but a handful of SMs idle, and the consumer adds the parts in split order).
-__device__ __forceinline__ void dmma_884(double (&c)[2], double a, double b) {
-  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-               : "+d"(c[0]), "+d"(c[1]) : "d"(a), "d"(b));
-}
-__device__ __forceinline__ double bf16_elem(const uint4& v, int s) {
-  const uint32_t w = s < 2 ? v.x : s < 4 ? v.y : s < 6 ? v.z : v.w;
-  return (double)((s & 1) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16));
-}
 template <int NT, int W>
 __global__ void __launch_bounds__(32 * W) k_proj_key_mma(ImDims p, const bf16* __restrict__ Uk, const bf16* __restrict__ x,
                                                        int NV, int ksplit, double* __restrict__ keyp) {
-  __shared__ double red[W][NT][64];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, q = lane & 3;
-  const long long v0 = (long long)blockIdx.x * 8;
-  const int kspan = p.D / (W * ksplit), kbeg = ((int)blockIdx.y * W + warp) * kspan;  // a multiple of 32 (checked by the launcher)
-  keyp += (size_t)blockIdx.y * NV * p.dI;
-  const bf16* xrow = x + (size_t)min(v0 + r, (long long)NV - 1) * p.D + kbeg + 8 * q;
-  const bf16* urow = Uk + (size_t)r * p.D + kbeg + 8 * q;
-  double c[NT][2];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = 0.0;
-  for (int kb = 0; kb < kspan; kb += 32) {
-    const uint4 xa = *reinterpret_cast<const uint4*>(xrow + kb);
-    uint4 ub[NT];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) ub[nt] = *reinterpret_cast<const uint4*>(urow + (size_t)nt * 8 * p.D + kb);
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      const double a = bf16_elem(xa, s);
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) dmma_884(c[nt], a, bf16_elem(ub[nt], s));
-    }
-  }
-  // C fragment: row r (vector), columns 2 q and 2 q + 1 (weight row of the n-tile)
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    red[warp][nt][r * 8 + 2 * q] = c[nt][0];
-    red[warp][nt][r * 8 + 2 * q + 1] = c[nt][1];
-  }
-  __syncthreads();
-  for (int idx = threadIdx.x; idx < NT * 64; idx += 32 * W) {
-    const int nt = idx >> 6, e = idx & 63;
-    const long long v = v0 + (e >> 3);
-    if (v < NV) {
-      double sum = red[0][nt][e];
-#pragma unroll
-      for (int w = 1; w < W; ++w) sum += red[w][nt][e];
-      keyp[(size_t)v * p.dI + nt * 8 + (e & 7)] = sum;
-    }
-  }
+  __shared__ double red[W * NT * 64];
+  proj_key_mma_block<NT, W>(p.D, p.dI, Uk, x, NV, ksplit, keyp, blockIdx.x, blockIdx.y, red);
 }
 
 }  // namespace
@@ -392,11 +417,26 @@ cudaError_t im_launch_gemm(const ImLaunch& L, const ImGemmArgs& a_in) {
       (n_w2 == 0 || n_w2 == a.n_jobs)) {
     int tiles = 0;
     for (int j = 0; j < a.n_jobs; ++j) tiles += (a.job[j].rows + 15) / 16;
-    dim3 grid(tiles, a.ksplit, (unsigned)((a.NV + VB - 1) / VB));
-    if (n_w2) k_direct_gemm<true><<<grid, DG_WARPS * 32, (size_t)std::max(0, a.smem_floor), L.stream>>>(a);
-    else k_direct_gemm<false><<<grid, DG_WARPS * 32, (size_t)std::max(0, a.smem_floor), L.stream>>>(a);
+    a.tiles = tiles;
+    int key_cols = 0;  // columns of blocks behind the tiles' for the key projection riding along
+    if (a.key_W) {
+      if ((a.key_dI != 8 && a.key_dI != 16) || a.key_ksplit < 1 || a.K % (32 * DG_WARPS * a.key_ksplit)) return cudaErrorInvalidValue;
+      key_cols = (((a.key_nv + 7) / 8) * a.key_ksplit + a.ksplit - 1) / a.ksplit;
+    }
+    dim3 grid(tiles + key_cols, a.ksplit, (unsigned)((a.NV + VB - 1) / VB));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(DG_WARPS * 32);
+    cfg.dynamicSmemBytes = (size_t)std::max(0, a.smem_floor);
+    cfg.stream = L.stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = a.programmatic ? 1 : 0;
+    const cudaError_t e = n_w2 ? cudaLaunchKernelEx(&cfg, k_direct_gemm<true>, a) : cudaLaunchKernelEx(&cfg, k_direct_gemm<false>, a);
     ++*L.launches;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
   }
   a.any_w2 = 0;
   for (int j = 0; j < a.n_jobs; ++j) a.any_w2 |= a.job[j].W2 != nullptr;

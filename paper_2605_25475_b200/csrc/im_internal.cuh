@@ -11,6 +11,7 @@ typedef __nv_bfloat16 bf16;
 #define IM_MAX_CALL_SEQS 256 /* sequences per hot call (the id list travels as a kernel parameter) */
 #define IM_SLOT_ALIGN 64     /* slot capacity is a multiple of the attention tile */
 #define IM_ATTN_TILE 32      /* rows of the small TMA box of the cache's tensor maps (32 rows x 128 bytes) */
+#define IM_ATTN_MIN_RUN 4 /* tiles a warp of the streaming attention kernel should at least get (bounds the grid of small calls) */
 #ifndef IM_ATTN_STREAM_TILE
 #define IM_ATTN_STREAM_TILE 32 /* keys per tile (= rows of a TMA box) of the mma.sync streaming attention kernel */
 #endif
@@ -219,6 +220,15 @@ struct ImGemmArgs {
   int direct;  // 1: few vectors (decode) - the variant without shared-memory staging, if the K split is a multiple of 32
   int any_w2;  // set by the launcher: some job has a second weight term (decides the smem layout)
   int smem_floor;  // direct variant: dynamic shared memory to ask for although the kernel uses none (IM_SMEM_SIDE)
+  // direct variant: the float64 indexer-key projection of key_nv vectors (rows of key_x, K elements each) rides along in
+  // the same launch if key_W is set: key_out[ks][v][key_dI] receives key_ksplit partial sums (K a multiple of
+  // 256 key_ksplit, key_dI 8 or 16); `tiles` is set by the launcher
+  const bf16* key_W;
+  const bf16* key_x;
+  double* key_out;
+  int key_nv, key_ksplit, key_dI, tiles;
+  int programmatic;  // direct variant: launched as programmatic dependent of the kernel ahead of it in the stream, whose
+                     // output the vectors are: the weights are requested while that kernel still runs
   // tensor-core TMA variant only: tc_ksplit > 1 cuts the K range over that many CTAs per output tile (launches of
   // few tiles are bound by the K loop of one CTA); split s writes to part + s * part_stride in the layout of `out`,
   // and a second kernel adds the splits into `out` in a fixed order.  Not with rmw or a batched launch.
