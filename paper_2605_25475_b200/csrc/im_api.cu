@@ -292,6 +292,7 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
   call->defer = 0;
   call->fold_all = 0;
   for (int k = 0; k < 5; ++k) { call->warm[k] = nullptr; call->warm_bytes[k] = 0; }
+  call->early_cache = 0;
   return IM_OK;
 }
 
@@ -963,8 +964,9 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   }
   cudaStream_t s0 = (cudaStream_t)cuda_stream;
   // (the merge kernel also fills the holes of ITS layer's cache, after its own wait: a programmatic dependent on the
-  // same layer would request tiles of that cache too early)
-  const bool after_merge = ctx->layer_overlap && ctx->tail_is_merge && ctx->tail_stream == s0 && ctx->tail_layer != layer;
+  // same layer waits for it before it reads anything, see ImCall::early_cache)
+  const bool after_merge = ctx->layer_overlap && ctx->tail_is_merge && ctx->tail_stream == s0;
+  call.early_cache = (after_merge && ctx->tail_layer != layer) ? 1 : 0;
   ctx->tail_is_merge = false;
   const bool fused = due && n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE;
   const bool defer = ctx->fast_attn && (!due || fused) && ne_max <= p.F;

@@ -256,6 +256,8 @@ k_attn_stream_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   if (tid == 0) im_attn_span[blockIdx.x][0] = im_gtimer();
 #endif
 
+  // (behind the merge kernel of a call on the same layer nothing of this cache may be read before that kernel has ended)
+  if (!call.early_cache) asm volatile("griddepcontrol.wait;" ::: "memory");
   // ---- tile prefix over the sequences of the call (every CTA computes the same table)
   for (int i = tid; i < call.n_seq; i += THREADS) {
     const size_t u = (size_t)call.layer * p.S + call.seq[i];

@@ -122,6 +122,9 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   long long* s_pref = reinterpret_cast<long long*>(bars + WARPS * STAGES);  // [n_seq + 1]
   int* s_n = reinterpret_cast<int*>(s_pref + IM_MAX_CALL_SEQS + 1);         // [n_seq]
 
+  // (launched behind the merge kernel of a call on the SAME layer, which advances the counters and fills the holes of
+  // this very cache: nothing of it may be read before that kernel has ended)
+  if (!call.early_cache) asm volatile("griddepcontrol.wait;" ::: "memory");
   // ---- tile prefix over the sequences of the call (every CTA computes the same table)
   for (int i = threadIdx.x; i < call.n_seq; i += blockDim.x) {
     const size_t u = (size_t)call.layer * p.S + call.seq[i];

@@ -180,6 +180,9 @@ struct ImCall {
   // producer has yet to write is simply written later: L2 is where the device's writes meet.
   const void* warm[5];
   unsigned warm_bytes[5];
+  // decode: 1 = the attention kernel may read this layer's counters and cache before the kernel ahead of it in the
+  // stream has ended (that kernel is the merge of a call on another layer); 0 = it waits for that kernel first
+  int early_cache;
   int seq[IM_MAX_CALL_SEQS];
 };
 __device__ __forceinline__ void im_warm_inputs(const ImCall& call, int part, int tid, int nthreads) {
