@@ -247,6 +247,13 @@ struct im_ctx {
   bool tail_is_merge = false;
   int tail_layer = -1;
   bool layer_overlap = true;         // IM_OPT_LAYER_OVERLAP
+  // A prefill call that evicts more than the pending list holds leaves the state update of its memory write (Eq. 6-7:
+  // pack, sums, Phi^T V) running on `late` when it returns: it needs nothing of the next chunk's projections, append
+  // and scoring and runs next to them.  The next call of the context, whatever it is, first makes its stream wait
+  // for `ev_late` (a prefill call: just before its own commit kernel, the first that writes a word the update reads).
+  cudaStream_t late = nullptr;
+  cudaEvent_t ev_late = nullptr, ev_phi = nullptr;
+  bool late_pending = false;
 #ifdef IM_TRACE
   int tune[8] = {0, -1, -1, 0, 0, 0, 0, 0};  // development builds: knobs set through options 100 + k
 #endif
@@ -268,6 +275,13 @@ ImLaunch make_launch(im_ctx* ctx, int layer, cudaStream_t s) {
   L.stream = s;
   L.launches = &ctx->launches;
   return L;
+}
+
+// makes `s` wait for a state update that an earlier prefill call left running (see im_ctx::late)
+cudaError_t join_late(im_ctx* ctx, cudaStream_t s) {
+  if (!ctx->late_pending) return cudaSuccess;
+  ctx->late_pending = false;
+  return cudaStreamWaitEvent(s, ctx->ev_late, 0);
 }
 
 int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall* call) {
@@ -623,11 +637,22 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
                                        (k == 1 && prio_hi + 1 <= prio_lo) ? prio_hi + 1 : prio_hi);
   }
   for (int k = 0; k < 14 && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&ctx->ev[k], cudaEventDisableTiming);
+  {
+    // (lowest priority: where its blocks and those of the next call's projections are ready together, the next call's go first)
+    int prio_lo = 0, prio_hi = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+    if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&ctx->late, cudaStreamNonBlocking, prio_lo);
+  }
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_late, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_phi, cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
     for (int k = 0; k < 14; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+    if (ctx->late) cudaStreamDestroy(ctx->late);
+    if (ctx->ev_late) cudaEventDestroy(ctx->ev_late);
+    if (ctx->ev_phi) cudaEventDestroy(ctx->ev_phi);
     delete ctx;
     return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
   }
@@ -640,6 +665,9 @@ int im_destroy(im_ctx* ctx) {
   cudaError_t e = cudaDeviceSynchronize();
   for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
   for (int k = 0; k < 14; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+  if (ctx->late) cudaStreamDestroy(ctx->late);
+  if (ctx->ev_late) cudaEventDestroy(ctx->ev_late);
+  if (ctx->ev_phi) cudaEventDestroy(ctx->ev_phi);
   delete ctx;
   if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
   return IM_OK;
@@ -659,6 +687,7 @@ int im_reset(im_ctx* ctx, int layer, int seq, void* cuda_stream) {
   const ImDims& p = ctx->p;
   if (layer < -1 || layer >= p.L || seq < -1 || seq >= p.S) return fail(IM_ERR_ARG, "layer/seq out of range");
   cudaStream_t s = (cudaStream_t)cuda_stream;
+  CK(join_late(ctx, s));
   for (int l = 0; l < p.L; ++l) {
     if (layer >= 0 && l != layer) continue;
     for (int q = 0; q < p.S; ++q) {
@@ -693,6 +722,7 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   if (p.scorer) {  // a retained set per KV head: no indexer inputs
     if (attend) return fail(IM_ERR_ARG, "im_prefill_chunk_attend is not available with a retained set per KV head");
     if (!k || !v) return fail(IM_ERR_ARG, "null tensor");
+    CK(join_late(ctx, (cudaStream_t)cuda_stream));
     return perhead_prefill(ctx, call, layer, chunk_len, k, v, cuda_stream);
   }
   if (!x || !q_pre || !k || !v) return fail(IM_ERR_ARG, "null tensor");
@@ -728,6 +758,11 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   call.pack = (ctx->score_tc && !follow) ? 1 : 0;
   call.fold_all = attend && p.mem ? 1 : 0;
   ImLaunch L = make_launch(ctx, layer, (cudaStream_t)cuda_stream);
+  // A state update that the previous prefill call left running (im_ctx::late): the projections, the append and the
+  // scoring of this chunk touch nothing that it reads or writes (after a write of that size the pending list of its
+  // sequences is empty, so the fold kernel below only looks at their counters), and this call waits for it just before
+  // its commit kernel.  A call with outputs reads the memory early: it waits at once.
+  if (attend || !ctx->concurrent) CK(join_late(ctx, L.stream));
   const int NV = n_seq * chunk_len;
   // pending rank-one terms are folded into M before a compression that cannot append to the list
   if (p.mem && (ne_max > 0 || attend)) CKL(im_launch_mem_fold(L, call));
@@ -844,6 +879,7 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
       ctx->prof_used += 2;
     }
   }
+  CK(join_late(ctx, L.stream));
   CKL(im_launch_prefill_commit(L, call));
   if (follow) CKL(im_launch_follow_scores(L, call));
   // a2: selection (also restarts the pooling); a4: gather the evicted pairs, fill the holes
@@ -859,7 +895,28 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
       if (attend) CK(cudaStreamWaitEvent(Lm.stream, ctx->ev[9], 0));  // the chunk attention reads the slots that are filled
       CKL(im_launch_move(Lm, call, ne_max));
       CK(cudaEventRecord(ctx->ev[6], Lm.stream));
-      if ((rc = run_memory_write(ctx, L, call, ne_max, true, 0, memside ? ctx->ev[8] : nullptr))) return rc;  // a3
+      // a3.  When every sequence of the call evicts more than the pending list holds, the state update runs on a
+      // stream of its own behind phi of the evicted keys and is left running (im_ctx::late); not under stream capture,
+      // which every stream that was forked has to rejoin
+      bool late = !attend && ne_max > p.F;
+      for (int i = 0; i < n_seq && late; ++i)
+        late = ctx->hu[(size_t)layer * p.S + call.seq[i]].n + chunk_len - p.B > p.F;
+      if (late) {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(L.stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) late = false;
+      }
+      if (late) {
+        if ((rc = run_memory_write(ctx, L, call, ne_max, false))) return rc;  // phi of the evicted keys
+        CK(cudaEventRecord(ctx->ev_phi, L.stream));
+        ImLaunch Ll = L;
+        Ll.stream = ctx->late;
+        CK(cudaStreamWaitEvent(Ll.stream, ctx->ev_phi, 0));
+        CKL(launch_mem_update(ctx, Ll, call, ne_max));
+        CK(cudaEventRecord(ctx->ev_late, Ll.stream));
+        ctx->late_pending = true;
+      } else if ((rc = run_memory_write(ctx, L, call, ne_max, true, 0, memside ? ctx->ev[8] : nullptr))) {
+        return rc;
+      }
       CK(cudaStreamWaitEvent(L.stream, ctx->ev[6], 0));
     } else {
       if (attend && fork) CK(cudaStreamWaitEvent(L.stream, ctx->ev[9], 0));  // the chunk attention reads the cache
@@ -898,6 +955,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   int rc = check_call(ctx, layer, n_seq, seq_ids, &call);
   if (rc) return rc;
   const ImDims& p = ctx->p;
+  CK(join_late(ctx, (cudaStream_t)cuda_stream));
   if (p.scorer) {  // a retained set per KV head: no indexer inputs
     if (!q || !k_new || !v_new || !out) return fail(IM_ERR_ARG, "null tensor");
     ctx->tail_is_merge = false;
@@ -1609,6 +1667,7 @@ int im_event_count(im_ctx* ctx, int counter, int64_t* value) {
 
 int im_status(im_ctx* ctx, void* cuda_stream, int32_t* device_status) {
   if (!ctx || !device_status) return fail(IM_ERR_ARG, "null argument");
+  CK(join_late(ctx, (cudaStream_t)cuda_stream));
   CK(cudaStreamSynchronize((cudaStream_t)cuda_stream));
   CK(cudaMemcpy(device_status, ctx->lo.st.status, 4, cudaMemcpyDeviceToHost));
   if (*device_status & ST_TIMEOUT) return fail(IM_ERR_TIMEOUT, "a bounded device wait gave up (status %d)", *device_status);

@@ -159,16 +159,27 @@ __device__ __forceinline__ void proj_key_mma_block(int D, int dI, const bf16* __
   double c[NT][2];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = 0.0;
-  for (int kb = 0; kb < kspan; kb += 32) {
-    const uint4 xa = *reinterpret_cast<const uint4*>(xrow + kb);
-    uint4 ub[NT];
+  // the loads of four 32-wide chunks are requested before the first of them is converted and multiplied: the loop is
+  // bound by the latency of its load -> convert -> mma chains, not by arithmetic
+  constexpr int PF = 4;
+  for (int kb0 = 0; kb0 < kspan; kb0 += 32 * PF) {
+    uint4 xa[PF], ub[PF][NT];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) ub[nt] = *reinterpret_cast<const uint4*>(urow + (size_t)nt * 8 * D + kb);
+    for (int i = 0; i < PF; ++i) {
+      const int kb = min(kb0 + 32 * i, kspan - 32);  // (a chunk past the end is loaded again and skipped below)
+      xa[i] = *reinterpret_cast<const uint4*>(xrow + kb);
 #pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      const double a = bf16_elem(xa, s);
+      for (int nt = 0; nt < NT; ++nt) ub[i][nt] = *reinterpret_cast<const uint4*>(urow + (size_t)nt * 8 * D + kb);
+    }
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) dmma_884(c[nt], a, bf16_elem(ub[nt], s));
+    for (int i = 0; i < PF; ++i) {
+      if (kb0 + 32 * i >= kspan) break;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        const double a = bf16_elem(xa[i], s);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) dmma_884(c[nt], a, bf16_elem(ub[i][nt], s));
+      }
     }
   }
   // C fragment: row r (vector), columns 2 q and 2 q + 1 (weight row of the n-tile)
