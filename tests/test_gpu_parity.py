@@ -108,6 +108,36 @@ def test_chunked_prefill_reduced():
     assert p.stats["max_M_err"] <= 2e-3
 
 
+def test_prefill_chunks_and_decode_steps_enqueued_back_to_back():
+    """Nothing waits for the device between the calls: a prefill call leaves the state update of its memory write
+    running on a stream of the library's own, and whatever call comes next has to order itself behind it.  Six chunks
+    whose evicted sets exceed the pending list, then decode steps, all enqueued at once; the final state and the outputs
+    against the oracle."""
+    wl = synth.CONFIGS["mistral7b_prefill"].replace(name="mistral_b2b", ctx=6 * 256, chunk=256, B=320, steps=3)
+    p = _pair(wl)
+    dev = p.device
+    ins = [tuple(t.to(dev) for t in synth.prefill_inputs(wl, 0, c)) for c in range(6)]
+    dec = [tuple(t.to(dev) for t in synth.decode_inputs(wl, 0, s)) for s in range(wl.steps)]
+    torch.cuda.synchronize()
+    outs = []
+    for X, Qp, _, K, V in ins:
+        p.g.prefill_chunk(0, p.seq_ids, X, Qp, K, V)
+    for x, qp, q, k, v in dec[:-1]:
+        outs.append(p.g.decode_step(0, p.seq_ids, x, qp, q, k, v))
+    torch.cuda.synchronize()
+    assert p.g.status() == 0
+    for c in range(6):
+        X, Qp, _, K, V = synth.prefill_inputs(wl, 0, c)
+        p.o.prefill_batch(p.seq_ids, synth.f32(X), synth.f32(Qp), synth.f32(K), synth.f32(V))
+    for s in range(wl.steps - 1):
+        x, qp, q, k, v = synth.decode_inputs(wl, 0, s)
+        ob, od = p.o.decode_batch(p.seq_ids, synth.f32(x), synth.f32(qp), synth.f32(q), synth.f32(k), synth.f32(v))
+        p.check_out(outs[s], ob, od)
+    assert p.check_state()
+    p.decode(wl.steps - 1)                       # and one more step, checked in full
+    assert p.stats["max_M_err"] <= 2e-3 and p.stats["cut_divergences"] == 0
+
+
 # ------------------------------------------------------------------ edge cases of the method
 def test_budget_never_reached_is_exact_attention(im):
     wl = TINY.replace(name="nobudget", ctx=100, chunk=100, B=4096, steps=5, n_needles=2)
