@@ -13,7 +13,11 @@
  *   - bf16 means the 16-bit brain-float bit pattern (upper half of an IEEE float32).
  *   - The two hot calls only enqueue kernels on `cuda_stream` (a cudaStream_t passed as void*, NULL =
  *     the legacy default stream) and return without synchronising; they allocate nothing.  All calls
- *     on one context must be issued in stream order on one stream at a time.
+ *     on one context must be issued in stream order on one stream at a time.  A prefill call may leave the last
+ *     part of its work (the state update of its memory write) running on a stream of the context's own when it
+ *     returns; every later call on the context orders itself behind that work, and im_destroy synchronises the
+ *     device, so the caller sees no difference as long as the workspace is touched through this interface only
+ *     (under stream capture nothing is left running: a capture has to end with every stream rejoined).
  *   - Return value: IM_OK (0) or a negative im_error.  No exception, abort or device trap crosses the
  *     boundary.  im_last_error() describes the most recent failure on the calling thread.  Problems
  *     that only the device can see (for example a non-finite score) set a sticky device status word
@@ -237,7 +241,9 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *   IM_OPT_PREFETCH_NEXT 1 (default): while the attention kernel of layer l streams the K/V cache,
  *                        im_decode_step prefetches into L2 what the small latency-bound kernels of layer
  *                        (l + 1) mod n_layers will read for the same sequences (weights, indexer key cache,
- *                        counters, pending memory terms); none of it depends on the output of layer l.
+ *                        counters, pending memory terms), and, once the attention kernel has ended, the first half
+ *                        of that layer's memory matrices (HBM has little else to do while the merge kernel runs);
+ *                        none of it depends on the output of layer l.
  *   IM_OPT_PREFILL_TENSOR 1 (default): the tcgen05 kernels of the prefill calls are used where they apply - the
  *                        indexer scoring of the chunk (Sec. 3.1, a dense [keys x d_I] x [d_I x queries * heads]
  *                        contraction; n_index_heads <= 8, index_dim 8 or 16; float32 features split into three
