@@ -1090,8 +1090,7 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   const ImDims& p = L.p;
   const CUtensorMap& mk = *(const CUtensorMap*)mapK;
   const CUtensorMap& mv = *(const CUtensorMap*)mapV;
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
+  cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_ctas);
   cfg.blockDim = dim3(WARPS * 32);
   cfg.dynamicSmemBytes = im_attn_smem_bytes(p);
@@ -1117,8 +1116,7 @@ cudaError_t im_launch_attention_merge(const ImLaunch& L, const ImCall& call, voi
   const bf16* kp = (const bf16*)k_new;
   const bf16* vp = (const bf16*)v_new;
   const ImDims& p = L.p;
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
+  cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.Hkv, call.n_seq);
   cfg.blockDim = dim3(32 * std::max(p.Gq, p.d / 32));
   cfg.stream = L.stream;

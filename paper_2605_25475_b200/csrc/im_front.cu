@@ -446,8 +446,7 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
   if (smem < (size_t)smem_floor) smem = (size_t)smem_floor;  // keeps the streaming kernels' blocks off this block's SM
   const bf16* kn = (const bf16*)k_new;
   const bf16* vn = (const bf16*)v_new;
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
+  cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(call.n_seq);
   cfg.blockDim = dim3(FRONT_THREADS);
   cfg.dynamicSmemBytes = smem;
