@@ -533,7 +533,7 @@ def test_decode_tensor_option_is_refused_for_other_head_dims(im):
     im.im_set_option(p.g.ctx, im.IM_OPT_DECODE_TENSOR, 0)
 
 
-@pytest.mark.parametrize("tensor,stages", [(0, 1), (0, 3), (1, 2), (1, 6)])
+@pytest.mark.parametrize("tensor,stages", [(0, 0), (0, 1), (0, 3), (1, 2), (1, 6)])
 def test_decode_readout_through_bulk_copy_ring(im, tensor, stages):
     """phi(q)^T Mhat formed by the persistent bulk-copy kernel (a ring of 32 KB stages per CTA next to the attention
     kernel, partial vectors per CTA added by the merge) instead of the kernel on plain loads: Llama widths (D_kv 1024,
