@@ -166,7 +166,7 @@ def pick_workload(args):
 
 
 def measure_decode(wl, device, steps, warmup, graph=True, rank=0, world=1, log=lambda *a: None, opts=None,
-                   profile=True, e2e_args=None, score_share=0, steps_per_graph=1):
+                   profile=True, e2e_args=None, score_share=0, steps_per_graph=1, stack_call=False):
     """Ingests the workload's context, then times `steps` decode steps (all layers, all sequences per step) replayed
     from CUDA graphs, inputs resident.  Returns the raw measurements; the context is closed before returning."""
     from paper_2605_25475_b200 import binding as im
@@ -178,8 +178,13 @@ def measure_decode(wl, device, steps, warmup, graph=True, rank=0, world=1, log=l
     inputs = decode_inputs_all(wl, n_in, device)
     out = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=device)
 
-    def one_step(k):
+    all_layers = list(range(L))
+
+    def one_step(k, stack=stack_call):
         x, qp, q, kk, v = inputs[k % n_in]
+        if stack:        # the step's layers in one call (im_decode_stack): their inputs are all there, the layers overlap
+            g.decode_stack(all_layers, ids, x, qp, q, kk, v, out)
+            return
         for layer in range(L):
             g.decode_step(layer, ids, x[layer], qp[layer], q[layer], kk[layer], v[layer], out[layer])
 
@@ -252,7 +257,7 @@ def measure_decode(wl, device, steps, warmup, graph=True, rank=0, world=1, log=l
                 im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, conc)
                 im.im_profile_begin(g.ctx, prof_steps * L)
                 for s in range(prof_steps):
-                    one_step(s)
+                    one_step(s, stack=False)          # (the library times the attention launch of a layer call)
                 k_ms, k_n = im.im_profile_end(g.ctx)
                 res["attn_ms_" + name], res["attn_n_" + name] = k_ms, k_n
             im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 1)
@@ -273,8 +278,10 @@ def run_ours(args, rank, world, device):
         opts[im.IM_OPT_DECODE_TENSOR] = args.decode_tensor
     if args.readout_stages >= 0:
         opts[im.IM_OPT_READOUT_STAGES] = args.readout_stages
+    if args.stack_reserved >= 0:
+        opts[im.IM_OPT_STACK_RESERVED] = args.stack_reserved
     m = measure_decode(wl, device, args.steps, args.warmup, graph=bool(args.graph), rank=rank, world=world, log=log,
-                       opts=opts, e2e_args=args, score_share=args.score_share)
+                       opts=opts, e2e_args=args, score_share=args.score_share, stack_call=bool(args.stack_call))
     ms = m["ms"]
     tokens = wl.n_seq * args.steps * world
     ab = algorithmic_bytes(wl)
@@ -674,6 +681,10 @@ def main():
                     help="g >= 2: layers l with l %% g != 0 reuse the indexer scores of layer l - l %% g (the paper's appendix uses 4)")
     ap.add_argument("--readout-stages", type=int, default=-1,
                     help="0: readout on plain loads; k >= 1: on a ring of k 32 KB bulk copies per CTA (default: the library's choice)")
+    ap.add_argument("--stack-call", type=int, default=0,
+                    help="1: a step is one im_decode_stack call over all layers (the layers overlap); 0: one im_decode_step call per layer")
+    ap.add_argument("--stack-reserved", type=int, default=-1,
+                    help="SMs a pipelined stack call keeps free of streaming blocks (default: the library's choice)")
     ap.add_argument("--traffic", type=float, default=ATTN_TRAFFIC_NCU,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as is)")
     args = ap.parse_args()

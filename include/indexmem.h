@@ -183,6 +183,35 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
                    const void* q_pre, const void* q, const void* k_new, const void* v_new, void* out,
                    void* cuda_stream);
 
+/*
+ * One decode token per sequence for several layers in one call: the same computation, layer by layer, as
+ * im_decode_step(layers[j], ..., x[j], q_pre[j], q[j], k_new[j], v_new[j], out[j]) for j = 0 .. n_layers - 1 (Sec. 4
+ * schedule, decode side; Eq. 4-7), for callers that hold the inputs of all those layers when they make the call: a
+ * stack of per-layer states driven from recorded or synthetic activations, layers of independent models that share a
+ * context.  Inside a transformer the query of layer l + 1 depends on the output of layer l, and the layers are then
+ * called one by one with im_decode_step.
+ *   layers           host int32 [n_layers], distinct
+ *   x, q_pre, q, k_new, v_new, out   host arrays of n_layers device pointers, shapes as for im_decode_step
+ * No input of the call may be written by the call (no out[j] overlaps an input of any layer): the layers overlap in
+ * time.  The (layer, sequence) states of different layers are independent, so the call keeps several layers in
+ * flight: the attention kernels of consecutive layers follow one another without a gap on one internal stream, the
+ * readout kernels on a second one, and each layer's projections, front kernel, phi of the evicted keys and merge
+ * run on the streams of one of three lanes with a scratch set per lane, next to the streams of the layers ahead of
+ * it.  All internal streams fork from `cuda_stream` when the call starts and join it when it ends: every output is
+ * complete in stream order after the call, and the call can be captured into a CUDA graph like im_decode_step.
+ * The streaming kernels are kept to a fixed subset of the SMs by SM id (a block that finds itself on an SM set
+ * aside for the small kernels hands its work to a block that is still to come), since with layers overlapping the
+ * occupancy rules that make this split in im_decode_step no longer hold.
+ * The pipelined schedule needs every layer of the call to qualify for im_decode_step's concurrent schedule with
+ * SMs set aside (at most n_SM / 4 sequences, evicted sets of at most min(16, pending_slots) entries, budgets of at
+ * most 6144 entries, the indexer as scorer, no score reuse, memory enabled); otherwise, and with
+ * IM_OPT_STACK_PIPELINE = 0, the layers are simply called in order.  Results are those of im_decode_step either way.
+ * Errors: as for im_decode_step; IM_ERR_ARG also for a repeated layer or a null entry.
+ */
+int im_decode_stack(im_ctx* ctx, int n_layers, const int32_t* layers, int n_seq, const int32_t* seq_ids,
+                    const void* const* x, const void* const* q_pre, const void* const* q, const void* const* k_new,
+                    const void* const* v_new, void* const* out, void* cuda_stream);
+
 /* Copies one weight tensor of a layer from / to host memory (bytes must equal the tensor size). Synchronous. */
 int im_set_weights(im_ctx* ctx, int layer, int which, const void* host_buf, size_t bytes);
 int im_get_weights(im_ctx* ctx, int layer, int which, void* host_buf, size_t bytes);
@@ -270,6 +299,15 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        the call before it on the same stream is launched as programmatic dependent of that call's last
  *                        kernel: it requests its first cache tiles while that kernel still runs and waits for it before it
  *                        touches anything else.  0: it is launched in plain stream order.
+ *   IM_OPT_STACK_PIPELINE 1 (default): im_decode_stack overlaps the layers of a call where they qualify; 0: it calls
+ *                        im_decode_step layer by layer.
+ *   IM_OPT_STACK_RESERVED k >= 1: SMs that a pipelined im_decode_stack keeps free of streaming blocks, for the small
+ *                        kernels of the layers in flight; 0 (default): one per sequence of the call.
+ *   IM_OPT_STACK_SPREAD  which SMs a pipelined im_decode_stack sets aside: 2 (default) pairs of neighbouring SM ids at even
+ *                        distances over the id range, 1 single SMs at even distances, 0 the highest ids.
+ *   IM_OPT_STACK_CHUNKS  k in [1, 16] (default 4): a pipelined im_decode_stack cuts the tiles of a layer's attention into k
+ *                        runs per warp, which the warps take from a counter.  With k = 1 the runs, and with them the
+ *                        order of every float32 sum, are those of im_decode_step: the two then agree bit for bit.
  *   IM_OPT_WAIT_LIMIT    (test aid) attempts of the bounded device-side waits in which a consumer waits for its copies to
  *                        arrive (TMA / bulk-copy rings of the decode attention kernels, the bulk-copy readout kernel and
  *                        the tcgen05 chunk attention kernel): 0 restores the default (2^22), k >= 1 allows k - 1 attempts,
@@ -286,7 +324,11 @@ typedef enum im_option {
   IM_OPT_DECODE_TENSOR = 4,
   IM_OPT_READOUT_STAGES = 5,
   IM_OPT_WAIT_LIMIT = 6,
-  IM_OPT_LAYER_OVERLAP = 7
+  IM_OPT_LAYER_OVERLAP = 7,
+  IM_OPT_STACK_PIPELINE = 8,
+  IM_OPT_STACK_RESERVED = 9,
+  IM_OPT_STACK_CHUNKS = 10,
+  IM_OPT_STACK_SPREAD = 11
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 

@@ -54,6 +54,7 @@ _lib.im_reset.argtypes = [_vp, _i32, _i32, _vp]
 _lib.im_prefill_chunk.argtypes = [_vp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.im_prefill_chunk_attend.argtypes = [_vp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.im_decode_step.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.im_decode_stack.argtypes = [_vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.im_set_weights.argtypes = [_vp, _i32, _i32, _vp, _sz]
 _lib.im_get_weights.argtypes = [_vp, _i32, _i32, _vp, _sz]
 _lib.im_state_export.argtypes = [_vp, _i32, _i32, _i32, _vp, _sz]
@@ -76,7 +77,7 @@ _lib.im_last_error.restype = C.c_char_p
 EXPORTED = ("im_workspace_bytes", "im_create", "im_destroy", "im_reset", "im_prefill_chunk", "im_decode_step",
             "im_set_weights", "im_get_weights", "im_state_export", "im_state_import", "im_topb_select",
             "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc", "im_event_count", "im_prefill_chunk_attend",
-            "im_set_scores", "im_state_export_head", "im_state_import_head")
+            "im_set_scores", "im_state_export_head", "im_state_import_head", "im_decode_stack")
 
 
 def _check(rc: int):
@@ -140,6 +141,15 @@ def im_decode_step(ctx, layer, seq_ids, x, q_pre, q, k_new, v_new, out):
     ids = _ids(seq_ids)
     _check(_lib.im_decode_step(ctx, layer, ids.size, ids.ctypes.data, _ptr(x), _ptr(q_pre), q.data_ptr(),
                                k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(), _stream()))
+
+
+def im_decode_stack(ctx, layers, seq_ids, x, q_pre, q, k_new, v_new, out):
+    """x .. out: one tensor per layer (sequences of tensors, or tensors stacked over the layers)."""
+    ids, lay = _ids(seq_ids), _ids(layers)
+    lists = [np.asarray([t.data_ptr() for t in ts], dtype=np.uint64) for ts in (x, q_pre, q, k_new, v_new, out)]
+    assert all(a.size == lay.size for a in lists)
+    _check(_lib.im_decode_stack(ctx, lay.size, lay.ctypes.data, ids.size, ids.ctypes.data, *[a.ctypes.data for a in lists],
+                                _stream()))
 
 
 def im_set_weights(ctx, layer, which, host: np.ndarray):
@@ -207,6 +217,7 @@ def im_profile_end(ctx):
 
 
 IM_OPT_CONCURRENCY, IM_OPT_PREFETCH_NEXT, IM_OPT_PREFILL_TENSOR, IM_OPT_PROFILE_TARGET, IM_OPT_DECODE_TENSOR, IM_OPT_READOUT_STAGES, IM_OPT_WAIT_LIMIT, IM_OPT_LAYER_OVERLAP = 0, 1, 2, 3, 4, 5, 6, 7
+IM_OPT_STACK_PIPELINE, IM_OPT_STACK_RESERVED, IM_OPT_STACK_CHUNKS, IM_OPT_STACK_SPREAD = 8, 9, 10, 11
 
 
 def im_set_option(ctx, option: int, value: int):
@@ -361,6 +372,20 @@ class IndexMem:
         else:
             _dev(out, self.out_dtype, n * self.D, "out")
         im_decode_step(self.ctx, layer, seq_ids, x, q_pre, q, k_new, v_new, out)
+        return out
+
+    def decode_stack(self, layers, seq_ids, x, q_pre, q, k_new, v_new, out=None):
+        """One decode token for every layer of `layers` in one call; x .. v_new (and out) hold one tensor per layer."""
+        n, nl = len(seq_ids), len(layers)
+        bf = torch.bfloat16
+        for j in range(nl):
+            _dev(x[j], bf, n * self.D, "x"); _dev(q_pre[j], bf, n * self.D, "q_pre"); _dev(q[j], bf, n * self.D, "q")
+            _dev(k_new[j], bf, n * self.Dkv, "k_new"); _dev(v_new[j], bf, n * self.Dkv, "v_new")
+        if out is None:
+            out = torch.empty((nl, n, self.H, self.d), dtype=self.out_dtype, device=self.device)
+        for j in range(nl):
+            _dev(out[j], self.out_dtype, n * self.D, "out")
+        im_decode_stack(self.ctx, layers, seq_ids, x, q_pre, q, k_new, v_new, out)
         return out
 
     def reset(self, layer=-1, seq=-1):

@@ -43,6 +43,8 @@ namespace {
 struct Layout {
   ImState st;
   ImScratch sc;
+  ImScratch lane[IM_STACK_LANES];  // decode scratch of the layers in flight in a pipelined stack call (see carve)
+  int32_t* claims;                 // the lanes' claim counters, IM_STACK_LANES x 8 (zeroed at create)
   std::vector<ImWeights> w;
   size_t state_begin, state_end;  // byte range holding per-unit state (zeroed at create)
   size_t total;
@@ -198,6 +200,36 @@ void carve(const ImDims& p, char* base, Layout* lo) {
   lo->sc.qpack = nullptr;
   if (im_score_tc_supported(p))
     lo->sc.qpack = (uint8_t*)take((size_t)p.S * ((p.max_chunk + IM_TC_QT - 1) / IM_TC_QT) * IM_TC_TILE_BYTES);
+  // Pipelined stack calls keep IM_STACK_LANES layers in flight, each with the scratch a deferred-compaction decode
+  // call writes: projection partials, gathered evicted pairs, phi partials, moves, attention / readout partials, the
+  // readout's small vectors, entry counts, claim counters.  A lane's gathered evicted pairs are at most
+  // IM_FRONT_MAX_NE rows per sequence; where a sequence's region of evK / evV has room (row stride `tail`), lane k
+  // uses rows [k, k + 1) * IM_FRONT_MAX_NE of the shared arrays, else arrays of its own.
+  lo->sc.claim = (int32_t*)take(256);
+  lo->claims = (int32_t*)take((size_t)IM_STACK_LANES * 8 * 4);
+  for (int k = 0; k < IM_STACK_LANES; ++k) {
+    ImScratch& ln = lo->lane[k];
+    ln = lo->sc;
+    if (p.scorer) continue;
+    ln.raw = (float*)take((size_t)p.S * IM_KSPLIT * p.R5 * 4);
+    ln.keyp = (double*)take((size_t)p.S * IM_KSPLIT_KEY * p.dI * 8);
+    if (p.tail >= IM_FRONT_MAX_NE * IM_STACK_LANES) {
+      ln.evK = base ? lo->sc.evK + (size_t)k * IM_FRONT_MAX_NE * p.Dkv : nullptr;
+      ln.evV = base ? lo->sc.evV + (size_t)k * IM_FRONT_MAX_NE * p.Dkv : nullptr;
+    } else {
+      ln.evK = (bf16*)take((size_t)p.S * p.evr * p.Dkv * 2);
+      ln.evV = (bf16*)take((size_t)p.S * p.evr * p.Dkv * 2);
+    }
+    ln.phip = (float*)take((size_t)IM_KSPLIT * p.S * p.F * p.dM * 4);
+    ln.surv = (int32_t*)take((size_t)p.S * p.tail * 4);
+    ln.nhole = (int32_t*)take((size_t)p.S * 4);
+    ln.part = (float*)take(((size_t)IM_ATTN_MAX_CTAS * IM_ATTN_WARPS + (size_t)p.S * p.Hkv) * p.Gq * (p.d + 2) * 4);
+    ln.mres = (float*)take((size_t)p.S * IM_MRES_ROW(p) * 4);
+    ln.phiq = (float*)take((size_t)p.S * p.dM * 4);
+    ln.n_att = (int32_t*)take((size_t)p.S * 4);
+    ln.rpart = (float*)take((size_t)p.S * p.Dkv * 4);
+    ln.claim = base ? lo->claims + k * 8 : nullptr;
+  }
   lo->total = align_up(off, 256);
 }
 
@@ -254,6 +286,24 @@ struct im_ctx {
   cudaStream_t late = nullptr;
   cudaEvent_t ev_late = nullptr, ev_phi = nullptr;
   bool late_pending = false;
+  // Pipelined stack calls (im_decode_stack): the attention kernels of the call's layers follow one another on
+  // `st_attn`, the readout kernels on `st_ro`; everything else of layer j runs on the streams of lane j %
+  // IM_STACK_LANES (main: merge; side: the four chains of a decode call), with the lane's events and scratch set.
+  struct Lane {
+    cudaStream_t main = nullptr, side[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ev[16] = {};
+    cudaEvent_t done = nullptr;  // everything of the lane's latest layer has been enqueued behind this
+    bool used = false;           // (within the current call)
+  } lane[IM_STACK_LANES];
+  cudaStream_t st_attn = nullptr, st_ro = nullptr;
+  cudaEvent_t st_fork = nullptr, st_attn_done = nullptr, st_ro_done = nullptr;
+  std::vector<int> sm_ids;           // ids of the device's SMs (ascending) as a probe kernel saw them; empty: unknown
+  bool stack_pipeline = true;        // IM_OPT_STACK_PIPELINE
+  int stack_reserved = 0;            // IM_OPT_STACK_RESERVED: SMs kept free of streaming blocks (0: one per sequence)
+  int stack_spread = 2;              // IM_OPT_STACK_SPREAD: where the SMs set aside lie in the id range
+  int stack_ro_workers = 0;          // (development) blocks of the readout kernel that work (0: one per streaming SM)
+  int stack_floors = 0;              // (development) the small kernels of a stack call ask for their shared-memory floors
+  int stack_chunks = 4;              // IM_OPT_STACK_CHUNKS: runs per warp the attention kernel's tiles are cut into
 #ifdef IM_TRACE
   int tune[8] = {0, -1, -1, 0, 0, 0, 0, 0};  // development builds: knobs set through options 100 + k
 #endif
@@ -284,6 +334,21 @@ cudaError_t join_late(im_ctx* ctx, cudaStream_t s) {
   return cudaStreamWaitEvent(s, ctx->ev_late, 0);
 }
 
+void destroy_lanes(im_ctx* ctx) {
+  for (int k = 0; k < IM_STACK_LANES; ++k) {
+    im_ctx::Lane& ln = ctx->lane[k];
+    if (ln.main) cudaStreamDestroy(ln.main);
+    for (int j = 0; j < 4; ++j) if (ln.side[j]) cudaStreamDestroy(ln.side[j]);
+    for (int j = 0; j < 16; ++j) if (ln.ev[j]) cudaEventDestroy(ln.ev[j]);
+    if (ln.done) cudaEventDestroy(ln.done);
+  }
+  if (ctx->st_attn) cudaStreamDestroy(ctx->st_attn);
+  if (ctx->st_ro) cudaStreamDestroy(ctx->st_ro);
+  if (ctx->st_fork) cudaEventDestroy(ctx->st_fork);
+  if (ctx->st_attn_done) cudaEventDestroy(ctx->st_attn_done);
+  if (ctx->st_ro_done) cudaEventDestroy(ctx->st_ro_done);
+}
+
 int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall* call) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   if (layer < 0 || layer >= ctx->p.L) return fail(IM_ERR_ARG, "layer %d out of range [0,%d)", layer, ctx->p.L);
@@ -307,6 +372,9 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
   call->fold_all = 0;
   for (int k = 0; k < 5; ++k) { call->warm[k] = nullptr; call->warm_bytes[k] = 0; }
   call->early_cache = 0;
+  call->stack = 0;
+  call->att_workers = call->ro_claim = call->att_chunks = 0;
+  for (int k = 0; k < 4; ++k) call->sm_stream[k] = 0;
   return IM_OK;
 }
 
@@ -646,8 +714,36 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_late, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_phi, cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
+  if (e == cudaSuccess && ctx->fast_attn && !p.scorer) {
+    // streams, events and the SM ids of pipelined stack calls
+    int prio_lo = 0, prio_hi = 0;
+    e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+    for (int k = 0; k < IM_STACK_LANES && e == cudaSuccess; ++k) {
+      im_ctx::Lane& ln = ctx->lane[k];
+      e = cudaStreamCreateWithPriority(&ln.main, cudaStreamNonBlocking, prio_lo);
+      for (int j = 0; j < 4 && e == cudaSuccess; ++j) e = cudaStreamCreateWithPriority(&ln.side[j], cudaStreamNonBlocking, prio_lo);
+      for (int j = 0; j < 16 && e == cudaSuccess; ++j) e = cudaEventCreateWithFlags(&ln.ev[j], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ln.done, cudaEventDisableTiming);
+    }
+    // (the two streaming kernels above the lanes' small kernels: where a block of either kind could take the registers
+    // or the shared memory that a streaming block of the previous layer has just released, the next layer's streaming
+    // block, which is already waiting, gets them; the small kernels run on the SMs set aside and in what is left)
+    if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&ctx->st_attn, cudaStreamNonBlocking, prio_hi);
+    if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&ctx->st_ro, cudaStreamNonBlocking, prio_hi);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->st_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->st_attn_done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->st_ro_done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->lo.claims, 0, (size_t)IM_STACK_LANES * 8 * 4, 0);
+    if (e == cudaSuccess && ctx->n_sm <= 256) {
+      std::vector<int> ids(ctx->n_sm);
+      int n = 0;
+      e = im_probe_sm_ids(ctx->lo.sc.raw, ctx->n_sm, ids.data(), &n, 0);
+      if (e == cudaSuccess && n == ctx->n_sm) ctx->sm_ids = ids;
+    }
+  }
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
+    destroy_lanes(ctx);
     for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
     for (int k = 0; k < 14; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
     if (ctx->late) cudaStreamDestroy(ctx->late);
@@ -663,6 +759,7 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
 int im_destroy(im_ctx* ctx) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   cudaError_t e = cudaDeviceSynchronize();
+  destroy_lanes(ctx);
   for (int k = 0; k < 4; ++k) if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
   for (int k = 0; k < 14; ++k) if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   if (ctx->late) cudaStreamDestroy(ctx->late);
@@ -1275,6 +1372,268 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   return IM_OK;
 }
 
+namespace {
+
+// What a decode call on `layer` would do, from the host mirror: phase of the interval, largest entry count after the
+// append and largest evicted set among the call's sequences.  Returns false where im_decode_step would refuse the call.
+bool decode_plan(im_ctx* ctx, int layer, const ImCall& call, bool* due, int* n_max, int* ne_max) {
+  const ImDims& p = ctx->p;
+  bool due_any = false, due_all = true;
+  *n_max = 0;
+  *ne_max = 0;
+  for (int i = 0; i < call.n_seq; ++i) {
+    const HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    if (u.n + 1 > p.cap) return false;
+    const bool d = (u.since + 1 == p.tau);
+    due_any |= d;
+    due_all &= d;
+    *n_max = std::max(*n_max, u.n + 1);
+    *ne_max = std::max(*ne_max, u.n + 1 - p.B);
+  }
+  if (due_any != due_all) return false;
+  *due = due_all;
+  if (!*due) *ne_max = 0;
+  return true;
+}
+
+// One layer of a pipelined stack call (see im_decode_stack): the kernels of im_decode_step's concurrent schedule with
+// deferred compaction, enqueued on the lane's streams, the call's attention stream and its readout stream.
+int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids, int n_res, const unsigned long long* sm_stream,
+                const void* x, const void* q_pre, const void* q, const void* k_new, const void* v_new, void* out) {
+  const ImDims& p = ctx->p;
+  ImCall call;
+  int rc = check_call(ctx, layer, n_seq, seq_ids, &call);
+  if (rc) return rc;
+  bool due = false;
+  int n_max = 0, ne_max = 0;
+  if (!decode_plan(ctx, layer, call, &due, &n_max, &ne_max)) return fail(IM_ERR_STATE, "layer %d: the call's plan changed under it", layer);
+  const int k = j % IM_STACK_LANES;
+  im_ctx::Lane& ln = ctx->lane[k];
+  call.due = due ? 1 : 0;
+  call.C = 1;
+  call.prefill = 0;
+  call.ksplit = pick_ksplit(p.D, IM_KSPLIT);
+  call.ksplit_key = (p.D % (8 * IM_KSPLIT_KEY) == 0) ? IM_KSPLIT_KEY : 1;
+  call.ksplit_phi = pick_ksplit(p.Dkv, IM_KSPLIT);
+  call.defer = 1;
+  call.early_cache = 1;
+  call.stack = 1;
+  for (int w = 0; w < 4; ++w) call.sm_stream[w] = sm_stream[w];
+  const bool fused = due;
+  const bool mem_write = due && ne_max > 0;
+  // workers of the two streaming kernels
+  const int n_wk_max = std::max(1, std::min(ctx->n_ctas, ctx->n_sm - n_res));
+  long long tiles = 0;
+  for (int i = 0; i < n_seq; ++i)
+    tiles += (long long)((ctx->hu[(size_t)layer * p.S + call.seq[i]].n + IM_ATTN_STREAM_TILE - 1) / IM_ATTN_STREAM_TILE) * p.Hkv;
+  const long long want = (tiles + IM_ATTN_WARPS * IM_ATTN_MIN_RUN - 1) / (IM_ATTN_WARPS * IM_ATTN_MIN_RUN);
+  call.att_workers = (int)std::max<long long>(1, std::min<long long>(n_wk_max, want));
+  call.ro_claim = (int)std::max<long long>(1, std::min<long long>(n_wk_max, (long long)n_seq * (p.Dkv / 64)));
+  if (ctx->stack_ro_workers > 0) call.ro_claim = std::min(call.ro_claim, ctx->stack_ro_workers);
+  // runs the attention kernel's tiles are cut into: a few per warp, so that a block that starts late takes fewer
+  call.att_chunks = std::min(call.att_workers * IM_ATTN_WARPS * ctx->stack_chunks, IM_ATTN_MAX_CTAS * IM_ATTN_WARPS);
+  // streams: the lane's own wait for the lane's previous layer (its scratch set), or for the start of the call
+  ImLaunch L = make_launch(ctx, layer, ln.main);
+  L.sc = ctx->lo.lane[k];
+  ImLaunch L1 = L, L2 = L, L3 = L, L4 = L, LA = L, LR = L;
+  L1.stream = ln.side[0];
+  L2.stream = ln.side[1];
+  L3.stream = ln.side[2];
+  L4.stream = ln.side[3];
+  LA.stream = ctx->st_attn;
+  LR.stream = ctx->st_ro;
+  if (!ln.used) {
+    CK(cudaStreamWaitEvent(ln.main, ctx->st_fork, 0));
+    for (int w = 0; w < 4; ++w) CK(cudaStreamWaitEvent(ln.side[w], ctx->st_fork, 0));
+  } else {
+    for (int w = 0; w < 4; ++w) CK(cudaStreamWaitEvent(ln.side[w], ln.done, 0));
+    CK(cudaStreamWaitEvent(LA.stream, ln.done, 0));
+    CK(cudaStreamWaitEvent(LR.stream, ln.done, 0));
+  }
+  // a0: projections.  s1: indexer part (heads the chain that decides the eviction)
+  ImRows r = im_rows(p);
+  ImGemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.in[0] = (const bf16*)q_pre;
+  g.in[1] = (const bf16*)x;
+  g.in[2] = (const bf16*)q;
+  for (int w = 0; w < 3; ++w) { g.in_cnt[w] = 1; g.in_outer[w] = p.D; g.in_inner[w] = 0; }
+  g.out = L.sc.raw;
+  g.out_cnt = 1;
+  g.out_outer = p.R5;
+  g.ks_stride = (long long)n_seq * p.R5;
+  g.NV = n_seq;
+  g.K = p.D;
+  g.ksplit = call.ksplit;
+  g.kc = 64;
+  g.direct = 1;
+  g.job[0] = {L.w.Uq, nullptr, p.HI * p.dI, r.uq, 0};
+  g.job[1] = {L.w.G, nullptr, p.HI, r.g, 1};
+  g.n_jobs = 2;
+  int key_ride = 0;
+  if ((p.dI == 8 || p.dI == 16) && (long long)n_seq * (p.Dkv / 64) < ctx->n_sm - n_res)
+    for (int ks = 8; ks >= 1 && !key_ride; --ks)
+      if (p.D % (256 * ks) == 0) key_ride = ks;
+  if (key_ride) {
+    g.key_W = L.w.Uk;
+    g.key_x = (const bf16*)x;
+    g.key_out = L.sc.keyp;
+    g.key_nv = n_seq;
+    g.key_ksplit = key_ride;
+    g.key_dI = p.dI;
+    call.ksplit_key = key_ride;
+  }
+  g.smem_floor = ctx->stack_floors ? IM_SMEM_HEAD : 0;
+  CKL(im_launch_gemm(L1, g));
+  g.smem_floor = 0;
+  g.key_W = nullptr;
+  // s3: key projection; s4: fold of the pending list
+  if (!key_ride) CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
+  CK(cudaEventRecord(ln.ev[2], L3.stream));
+  if (mem_write) {
+    CKL(im_launch_mem_fold(L4, call));
+    CK(cudaEventRecord(ln.ev[7], L4.stream));
+  }
+  // s2: phi(q) and the gate logit
+  g.job[0] = {L.w.Wt, nullptr, p.dM, r.theta, 2};
+  g.job[1] = {L.w.wg, nullptr, 1, r.wg, 2};
+  CKL(im_launch_gemm(L2, g));
+  CK(cudaEventRecord(ln.ev[6], L2.stream));
+  // a5 on the call's attention stream: behind the previous layer's attention kernel as its programmatic dependent
+  // (it becomes resident as that kernel's blocks end, and waits for nothing)
+  CKL(im_launch_attention_fast(LA, call, ctx->mapKs, ctx->mapVs, q, std::max(ctx->n_sm, call.att_workers), j > 0 ? 1 : 0));
+  CK(cudaEventRecord(ln.ev[9], LA.stream));
+  // s4: the part of the readout that does not go through Mhat, over the memory as it is before this call's write
+  CK(cudaStreamWaitEvent(L4.stream, ln.ev[6], 0));
+  CKL(im_launch_readout_finish(L4, call));
+  CK(cudaEventRecord(ln.ev[4], L4.stream));
+  // s1: append, score, select, gather, list the moves
+  CK(cudaStreamWaitEvent(L1.stream, ln.ev[2], 0));
+  CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max, ctx->stack_floors ? IM_SMEM_FRONT : 0, nullptr, 1));
+  // phi(q)^T Mhat on the call's readout stream
+  CK(cudaStreamWaitEvent(LR.stream, ln.ev[6], 0));
+  if (mem_write) CK(cudaStreamWaitEvent(LR.stream, ln.ev[7], 0));
+  CKL(im_launch_readout(LR, call, std::max(ctx->n_sm, call.ro_claim), 0));
+  CK(cudaEventRecord(ln.ev[12], LR.stream));
+  // a3: phi of the evicted keys, then (off the path to the merge) the state update
+  if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, false, ctx->stack_floors ? IM_SMEM_SIDE : 0, nullptr, 0))) return rc;
+  CK(cudaEventRecord(ln.ev[3], L1.stream));
+  CK(cudaStreamWaitEvent(L1.stream, ln.ev[4], 0));
+  if (mem_write) CKL(launch_mem_update(ctx, L1, call, ne_max));
+  CK(cudaEventRecord(ln.ev[5], L1.stream));
+  for (int i = 0; i < n_seq; ++i) {
+    HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
+    const int ne = due ? std::max(0, u.n + 1 - p.B) : 0;
+    mirror_memory(p, u, ne);
+    u.n = u.n + 1 - ne;
+    u.T += 1;
+    u.since = due ? 0 : u.since + 1;
+  }
+  // a6: merge, gate, fuse; a4: the merge fills the holes
+  CK(cudaStreamWaitEvent(ln.main, ln.ev[9], 0));
+  CK(cudaStreamWaitEvent(ln.main, ln.ev[3], 0));
+  CK(cudaStreamWaitEvent(ln.main, ln.ev[12], 0));
+  CK(cudaStreamWaitEvent(ln.main, ln.ev[4], 0));
+  CKL(im_launch_attention_merge(L, call, out, call.att_chunks, IM_ATTN_STREAM_TILE, 0, q, k_new, v_new, 0));
+  CK(cudaStreamWaitEvent(ln.main, ln.ev[5], 0));
+  CK(cudaStreamWaitEvent(ln.main, ln.ev[2], 0));
+  CK(cudaEventRecord(ln.done, ln.main));
+  ln.used = true;
+  return IM_OK;
+}
+
+}  // namespace
+
+extern "C" int im_decode_stack(im_ctx* ctx, int n_layers, const int32_t* layers, int n_seq, const int32_t* seq_ids,
+                               const void* const* x, const void* const* q_pre, const void* const* q, const void* const* k_new,
+                               const void* const* v_new, void* const* out, void* cuda_stream) {
+  if (!ctx) return fail(IM_ERR_ARG, "null context");
+  const ImDims& p = ctx->p;
+  if (n_layers < 1 || n_layers > p.L) return fail(IM_ERR_ARG, "n_layers %d out of range [1,%d]", n_layers, p.L);
+  if (!layers || !q || !k_new || !v_new || !out || (!p.scorer && (!x || !q_pre))) return fail(IM_ERR_ARG, "null pointer list");
+  {
+    std::vector<char> seen(p.L, 0);
+    for (int j = 0; j < n_layers; ++j) {
+      if (layers[j] < 0 || layers[j] >= p.L) return fail(IM_ERR_ARG, "layer %d out of range [0,%d)", layers[j], p.L);
+      if (seen[layers[j]]) return fail(IM_ERR_ARG, "layer %d repeated in one call", layers[j]);
+      seen[layers[j]] = 1;
+    }
+  }
+  // The pipelined schedule takes calls whose every layer runs im_decode_step's concurrent schedule with deferred
+  // compaction and SMs set aside for the chain of small kernels; anything else goes layer by layer.
+  bool pipe = ctx->stack_pipeline && n_layers >= 2 && ctx->fast_attn && ctx->concurrent && !ctx->attn_tc && !ctx->ro_stream &&
+              !p.scorer && !p.share && p.mem && !ctx->sm_ids.empty() && ctx->st_attn != nullptr;
+  int n_res = 0;
+  if (pipe) {
+    // (far fewer than im_decode_step sets aside: the small kernels are off the path that bounds the call, and while
+    // a layer's readout block is absent from a streaming SM they find registers there as well)
+    n_res = ctx->stack_reserved > 0 ? ctx->stack_reserved : std::min(im_reserved_sms(ctx->n_sm, n_seq), 8);
+    pipe = n_res > 0 && n_res < ctx->n_sm;
+  }
+  for (int j = 0; j < n_layers && pipe; ++j) {
+    ImCall call;
+    if (check_call(ctx, layers[j], n_seq, seq_ids, &call)) { pipe = false; break; }
+    bool due = false;
+    int n_max = 0, ne_max = 0;
+    if (!decode_plan(ctx, layers[j], call, &due, &n_max, &ne_max)) { pipe = false; break; }
+    if (due && !(n_max <= IM_FRONT_MAX_N && ne_max <= IM_FRONT_MAX_NE)) pipe = false;
+    if (ne_max > p.F) pipe = false;
+  }
+  if (!pipe) {
+    for (int j = 0; j < n_layers; ++j) {
+      const int rc = im_decode_step(ctx, layers[j], n_seq, seq_ids, x ? x[j] : nullptr, q_pre ? q_pre[j] : nullptr, q[j], k_new[j],
+                                    v_new[j], out[j], cuda_stream);
+      if (rc) return rc;
+    }
+    return IM_OK;
+  }
+  for (int j = 0; j < n_layers; ++j)
+    if (!x[j] || !q_pre[j] || !q[j] || !k_new[j] || !v_new[j] || !out[j]) return fail(IM_ERR_ARG, "null tensor (layer %d)", layers[j]);
+  cudaStream_t s0 = (cudaStream_t)cuda_stream;
+  CK(join_late(ctx, s0));
+  ctx->tail_is_merge = false;
+  // SMs for the streaming kernels: all but n_res, which are taken at even distances over the id range so that every
+  // part of the chip keeps streaming blocks (ids that lie together share a path to the memory system; with the n_res
+  // highest ids set aside the streams reached three quarters of their rate).  IM_OPT_STACK_SPREAD 2: whole pairs
+  // (2k, 2k + 1) at even distances; 1: single SMs; 0: the highest ids.
+  unsigned long long sm_stream[4] = {0, 0, 0, 0};
+  {
+    const int n = ctx->n_sm;
+    std::vector<char> res(n, 0);
+    if (ctx->stack_spread == 0) {
+      for (int w = n - n_res; w < n; ++w) res[w] = 1;
+    } else if (ctx->stack_spread == 1 || n_res < 2) {
+      for (int k = 0; k < n_res; ++k) res[(int)(((long long)(2 * k + 1) * n) / (2 * n_res))] = 1;
+    } else {
+      const int pairs = n / 2, want = n_res / 2;
+      for (int k = 0; k < want; ++k) {
+        const int t = (int)(((long long)(2 * k + 1) * pairs) / (2 * want));
+        res[2 * t] = res[2 * t + 1] = 1;
+      }
+      if (n_res & 1)  // one more: the first free SM
+        for (int w = 0; w < n; ++w)
+          if (!res[w]) { res[w] = 1; break; }
+    }
+    for (int w = 0; w < n; ++w)
+      if (!res[w]) sm_stream[ctx->sm_ids[w] >> 6] |= 1ull << (ctx->sm_ids[w] & 63);
+  }
+  CK(cudaEventRecord(ctx->st_fork, s0));
+  CK(cudaStreamWaitEvent(ctx->st_attn, ctx->st_fork, 0));
+  CK(cudaStreamWaitEvent(ctx->st_ro, ctx->st_fork, 0));
+  for (int k = 0; k < IM_STACK_LANES; ++k) ctx->lane[k].used = false;
+  for (int j = 0; j < n_layers; ++j) {
+    const int rc = stack_layer(ctx, j, layers[j], n_seq, seq_ids, n_res, sm_stream, x[j], q_pre[j], q[j], k_new[j], v_new[j], out[j]);
+    if (rc) return rc;  // (streams forked so far are rejoined by the caller's next synchronisation only: the call has failed)
+  }
+  CK(cudaEventRecord(ctx->st_attn_done, ctx->st_attn));
+  CK(cudaEventRecord(ctx->st_ro_done, ctx->st_ro));
+  CK(cudaStreamWaitEvent(s0, ctx->st_attn_done, 0));
+  CK(cudaStreamWaitEvent(s0, ctx->st_ro_done, 0));
+  for (int k = 0; k < IM_STACK_LANES; ++k)
+    if (ctx->lane[k].used) CK(cudaStreamWaitEvent(s0, ctx->lane[k].done, 0));
+  return IM_OK;
+}
+
 #ifdef IM_TRACE
 extern "C" int im_trace_read(im_ctx* ctx, unsigned long long* host, long long n) {
   cudaDeviceSynchronize();
@@ -1306,6 +1665,21 @@ int im_set_option(im_ctx* ctx, int option, int value) {
       ctx->tail_is_merge = false;
       return IM_OK;
     case IM_OPT_LAYER_OVERLAP: ctx->layer_overlap = value != 0; return IM_OK;
+    case IM_OPT_STACK_PIPELINE: ctx->stack_pipeline = value != 0; return IM_OK;
+    case IM_OPT_STACK_SPREAD:
+      if (value < 0 || value > 2) return fail(IM_ERR_ARG, "placement %d: 0 highest ids, 1 single SMs at even distances, 2 pairs at even distances", value);
+      ctx->stack_spread = value;
+      return IM_OK;
+    case 12: ctx->stack_floors = value; return IM_OK;
+    case 13: ctx->stack_ro_workers = value; return IM_OK;
+    case IM_OPT_STACK_CHUNKS:
+      if (value < 1 || value > 16) return fail(IM_ERR_ARG, "runs per warp %d out of range [1,16]", value);
+      ctx->stack_chunks = value;
+      return IM_OK;
+    case IM_OPT_STACK_RESERVED:
+      if (value < 0 || value >= ctx->n_sm) return fail(IM_ERR_ARG, "reserved SMs %d out of range [0,%d)", value, ctx->n_sm);
+      ctx->stack_reserved = value;
+      return IM_OK;
 #ifdef IM_TRACE
     case 100: case 101: case 102: case 103: case 104: case 105: case 106: case 107: ctx->tune[option - 100] = value; return IM_OK;
 #endif

@@ -19,6 +19,15 @@
 
 #include "im_internal.cuh"
 
+#ifdef IM_DBG_STACK
+__device__ unsigned long long g_dbg[32 * 160 * 8];
+extern "C" int im_dbg_read(unsigned long long* host) {
+  cudaDeviceSynchronize();
+  return (int)cudaMemcpyFromSymbol(host, g_dbg, sizeof(g_dbg));
+}
+__device__ __forceinline__ unsigned long long dbg_now() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#endif
+
 namespace {
 
 constexpr float NEG_INF = -__builtin_huge_valf();
@@ -104,7 +113,12 @@ __device__ __forceinline__ int tiles_of(int n) { return (n + TILE - 1) / TILE; }
 // Persistent attention kernel.  grid = #SMs (or fewer), block = WARPS * 32.
 // Shared memory: per warp STAGES x 16 KB (1024-byte aligned), then barriers and the per-sequence
 // prefix of tile counts.
-template <int DH>
+// DYN (pipelined stack calls): the tiles are cut into call.att_chunks equal runs and a warp takes runs from a
+// counter until none is left, instead of owning the one run its index names.  With layers overlapping, a block of
+// this kernel may find its SM busy for a while with blocks of a neighbouring layer's small kernels; with fixed runs
+// the whole kernel, and every layer behind it, would wait for that one block.  The merge kernel only needs to know
+// how the tiles were cut (run r writes partial slot r + row), not who computed a run.
+template <int DH, bool DYN>
 __global__ void __launch_bounds__(WARPS * 32, 1)
 k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, ImDims p, ImState st,
               ImScratch sc, ImCall call, const bf16* __restrict__ q) {
@@ -121,7 +135,33 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)WARPS * STAGES * STAGE_BYTES);
   long long* s_pref = reinterpret_cast<long long*>(bars + WARPS * STAGES);  // [n_seq + 1]
   int* s_n = reinterpret_cast<int*>(s_pref + IM_MAX_CALL_SEQS + 1);         // [n_seq]
+  int* s_misc = s_n + IM_MAX_CALL_SEQS;                                     // [1 + WARPS * 4] (DYN)
+  int* s_fifo = s_misc + 1 + warp * 4;  // runs this warp's producer side has taken, in order (-1: none left)
 
+  // Pipelined stack call: the block claims a worker id (blocks on SMs that are set aside for the call's small
+  // kernels, and blocks beyond the worker count, leave).  Nothing that this kernel reads or writes belongs to the
+  // kernel ahead of it in its stream (the attention kernel of the previous layer, with a scratch set of its own), so
+  // a programmatic dependent never waits for it.
+  int wid = blockIdx.x;
+#ifdef IM_DBG_STACK
+  unsigned long long* dbg = g_dbg + ((size_t)(call.layer % 32) * 160 + blockIdx.x % 160) * 8;
+  if (DYN && threadIdx.x == 0) { unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); dbg[0] = smid; dbg[1] = dbg_now(); dbg[5] = 0; }
+#endif
+  if (DYN) {
+    if (threadIdx.x == 0) s_misc[0] = im_claim_worker(call, sc.claim, call.att_workers);
+    __syncthreads();
+    wid = s_misc[0];
+#ifdef IM_DBG_STACK
+    if (threadIdx.x == 0) { dbg[2] = (unsigned long long)(long long)wid; dbg[3] = dbg_now(); dbg[4] = dbg[3]; }
+#endif
+    if (wid < 0) {
+      if (threadIdx.x == 0) im_claim_exit(sc.claim);
+      return;
+    }
+    __syncthreads();
+  }
+  int next_run = 0;  // DYN, lane 0: the run this warp's producer side starts next
+  if (DYN && lane == 0) next_run = atomicAdd(sc.claim + 3, 1);
   // (launched behind the merge kernel of a call on the SAME layer, which advances the counters and fills the holes of
   // this very cache: nothing of it may be read before that kernel has ended)
   if (!call.early_cache) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -146,32 +186,60 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   }
   __syncthreads();
   const long long total = s_pref[call.n_seq];
-  const long long WT = (long long)gridDim.x * WARPS;
+  const long long WT = DYN ? (long long)call.att_chunks : (long long)gridDim.x * WARPS;  // runs the tiles are cut into
   const long long qrun = (total + WT - 1) / WT;
-  const long long wglob = (long long)blockIdx.x * WARPS + warp;
-  const long long run0 = min(total, wglob * qrun), run1 = min(total, run0 + qrun);
-  const bool has_work = run0 < run1;
 
-  // ---- position of the first tile of the run: sequence i, KV head h, tile tt
-  int i = 0;
-  if (has_work) {
-    int lo = 0, hi = call.n_seq;  // last i with s_pref[i] <= run0
+  // position of global tile `tile`: sequence i_, KV head h_, tile tt_ of nt_
+  auto locate = [&](long long tile, int& i_, int& h_, int& tt_, int& nt_) {
+    int lo = 0, hi = call.n_seq;  // last i with s_pref[i] <= tile
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (s_pref[mid] <= run0) lo = mid; else hi = mid;
+      if (s_pref[mid] <= tile) lo = mid; else hi = mid;
     }
-    i = lo;
-    while (i < call.n_seq - 1 && tiles_of(s_n[i]) == 0) ++i;  // empty sequences own no tiles
-  }
-  int nt = max(1, tiles_of(s_n[i]));
-  int h = has_work ? (int)((run0 - s_pref[i]) / nt) : 0, tt = has_work ? (int)((run0 - s_pref[i]) % nt) : 0;
+    i_ = lo;
+    while (i_ < call.n_seq - 1 && tiles_of(s_n[i_]) == 0) ++i_;  // empty sequences own no tiles
+    nt_ = max(1, tiles_of(s_n[i_]));
+    h_ = (int)((tile - s_pref[i_]) / nt_);
+    tt_ = (int)((tile - s_pref[i_]) % nt_);
+  };
 
   const uint64_t pol = policy_evict_first();
-  // iterator used by the producer side (runs STAGES tiles ahead of the consumer side)
-  int pi = i, ph = h, ptt = tt, pnt = nt;
-  long long issued = run0;
-  auto issue = [&](long long j) {  // lane 0 only: load global tile j (== issued) into stage j % STAGES
-    const int s = (int)((j - run0) % STAGES);
+  // ---- producer side (lane 0): runs STAGES tiles ahead of the consumer side.  The k-th tile this warp requests goes
+  // to stage k % STAGES, whichever run it belongs to.
+  long long p_pos = 0, p_end = 0;  // next tile to request, end of the producer's current run
+  long long n_issued = 0;          // tiles requested so far
+  int pi = 0, ph = 0, ptt = 0, pnt = 1, n_pushed = 0;
+  bool p_done = false, released = false;
+  auto take_run = [&]() {  // the producer's next run (DYN: from the counter, recorded for the consumer side)
+    long long r = -1;
+    if (DYN) {
+      // (the run was taken from the counter when the previous one was started, and the one after it is taken now:
+      // the add's round trip, microseconds while the streams keep the memory system busy, is off the warp's path)
+      const int c = next_run;
+      next_run = atomicAdd(sc.claim + 3, 1);
+      if (c < WT && (long long)c * qrun < total) r = c;
+      s_fifo[n_pushed & 3] = (int)r;
+      ++n_pushed;
+    } else if (n_pushed == 0) {
+      const long long w = (long long)wid * WARPS + warp;
+      if (w * qrun < total) r = w;
+      ++n_pushed;
+    }
+    if (r < 0) { p_done = true; return; }
+    p_pos = r * qrun;
+    p_end = min(total, p_pos + qrun);
+    locate(p_pos, pi, ph, ptt, pnt);
+  };
+  auto issue = [&]() {  // lane 0 only: request the next tile, if one is left
+    if (!p_done && p_pos == p_end) take_run();
+    if (p_done) {
+      // nothing left to request: a kernel launched as programmatic dependent (the merge, or the next layer's attention
+      // kernel) may become resident and run what does not read this kernel's output
+      if (!released) asm volatile("griddepcontrol.launch_dependents;");
+      released = true;
+      return;
+    }
+    const int s = (int)(n_issued % STAGES);
     const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
     const uint32_t dst = smem_u32(ring + (size_t)s * STAGE_BYTES);
     const size_t u = (size_t)call.layer * p.S + call.seq[pi];
@@ -182,6 +250,8 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       tma_load_2d(dst + b * (TILE * 128), &tmK, b * 64, row, bar, pol);
       tma_load_2d(dst + TILE_BYTES + b * (TILE * 128), &tmV, b * 64, row, bar, pol);
     }
+    ++n_issued;
+    ++p_pos;
     // advance the producer iterator
     if (++ptt == pnt) {
       ptt = 0;
@@ -191,22 +261,43 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         pnt = pi < call.n_seq ? tiles_of(s_n[pi]) : 1;
       }
     }
+    if (!DYN && p_pos == p_end) {  // (a fixed run: its last tile is requested)
+      asm volatile("griddepcontrol.launch_dependents;");
+      released = true;
+      p_done = true;
+    }
   };
   if (lane == 0) {
-    for (int k = 0; k < STAGES && issued < run1; ++k) issue(issued++);
+    for (int k = 0; k < STAGES; ++k) issue();
   }
-  im_warm_inputs(call, blockIdx.x, threadIdx.x, blockDim.x);  // (the first CTAs: one input tensor each)
+  if (!DYN) im_warm_inputs(call, wid, threadIdx.x, blockDim.x);  // (the first CTAs: one input tensor each)
   // Launched as a programmatic dependent (of the previous call's merge kernel, or of whatever precedes the call in
   // the caller's stream) the kernel may have come this far before that kernel has ended: the cache of this layer,
   // which the first tiles are being fetched from, is not that kernel's business, but the query rows may be its
   // output and the partials and entry counts of this call overwrite what the previous call's merge still reads.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (blockIdx.x == 0)  // what the merge kernel rebuilds the tile bookkeeping from
+  if (!DYN) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (wid == 0)  // what the merge kernel rebuilds the tile bookkeeping from
     for (int k = threadIdx.x; k < call.n_seq; k += blockDim.x) sc.n_att[k] = s_n[k];
-  if (!has_work) return;
 
   const float sl2 = p.scale * 1.4426950408889634f;  // softmax in base 2
   bool ok = true;
+  long long n_done = 0;  // tiles consumed so far (tile k sits in stage k % STAGES)
+  int n_popped = 0;
+  while (ok) {
+    // ---- the consumer side's next run
+    long long run_id = -1;
+    if (DYN) {
+      __syncwarp();  // (the producer side, lane 0, has recorded the run before it requested the run's first tile)
+      run_id = s_fifo[n_popped & 3];
+    } else if (n_popped == 0) {
+      const long long w = (long long)wid * WARPS + warp;
+      if (w * qrun < total) run_id = w;
+    }
+    ++n_popped;
+    if (run_id < 0) break;
+    const long long run0 = run_id * qrun, run1 = min(total, run0 + qrun);
+    int i, h, tt, nt;
+    locate(run0, i, h, tt, nt);
   long long j = run0;
   while (j < run1 && ok) {
     // ---- one (sequence, KV head) segment of the run
@@ -228,10 +319,11 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     float m0 = NEG_INF, m1 = NEG_INF, l0 = 0.f, l1 = 0.f;  // heads 2t, 2t+1 (l: this thread's share)
 
     for (; tt < nt && j < run1; ++tt, ++j) {
-      const int s = (int)((j - run0) % STAGES);
+      const int s = (int)(n_done % STAGES);
       const uint32_t bar = smem_u32(&bars[warp * STAGES + s]);
       // (the outcome is made warp-uniform: the lanes poll on their own and could disagree at the limit)
-      if (!__all_sync(0xffffffffu, mbar_wait(bar, (uint32_t)(((j - run0) / STAGES) & 1), p.wait_limit))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(bar, (uint32_t)((n_done / STAGES) & 1), p.wait_limit))) { ok = false; break; }
+      ++n_done;
       const uint32_t Ks = smem_u32(ring + (size_t)s * STAGE_BYTES), Vs = Ks + TILE_BYTES;
       // ---- S^T = K Q^T : [32 keys] x [8 heads]
       float sacc[TILE / 16][4];
@@ -304,12 +396,7 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
       // ---- the stage is free again: refill it
       __syncwarp();
-      if (lane == 0 && issued < run1) {
-        issue(issued++);
-        // the last tile of this warp's run is requested: a kernel launched as programmatic dependent (the merge)
-        // may become resident and run the part of its prologue that does not read this kernel's output
-        if (issued == run1) asm volatile("griddepcontrol.launch_dependents;");
-      }
+      if (lane == 0) issue();
     }
     if (!ok) break;
     // ---- segment finished: write the partial (unnormalised O, max, sum) of this row
@@ -319,9 +406,9 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       l1 += __shfl_xor_sync(0xffffffffu, l1, off);
     }
     {
-      // Rows are served by consecutive warps and consecutive rows share at most one warp, so
-      // (warp index + row index) is a collision-free slot id below WT + rows.
-      const long long slot = wglob + row_id;
+      // Rows are served by consecutive runs and consecutive rows share at most one run, so
+      // (run index + row index) is a collision-free slot id below WT + rows.
+      const long long slot = run_id + row_id;
       float* dst = sc.part + (size_t)slot * p.Gq * (DH + 2);
       const int hh0 = 2 * t, hh1 = 2 * t + 1;
 #pragma unroll
@@ -351,13 +438,25 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       }
     }
   }
+    if (!DYN) break;
+  }
   if (!ok && lane == 0) {
-    // The warp gives up.  The copies it has requested and not consumed (tiles j .. issued - 1) still write into this
-    // CTA's shared memory, which the SM hands to another CTA when this one ends: wait for each of them, with the full
-    // limit, before returning.
+    // The warp gives up.  The copies it has requested and not consumed (tiles n_done .. n_issued - 1 of its own count)
+    // still write into this CTA's shared memory, which the SM hands to another CTA when this one ends: wait for each
+    // of them, with the full limit, before returning.
     atomicOr(st.status, ST_TIMEOUT);
-    for (long long t2 = j; t2 < issued; ++t2)
-      mbar_wait(smem_u32(&bars[warp * STAGES + (int)((t2 - run0) % STAGES)]), (uint32_t)(((t2 - run0) / STAGES) & 1));
+    for (long long t2 = n_done; t2 < n_issued; ++t2)
+      mbar_wait(smem_u32(&bars[warp * STAGES + (int)(t2 % STAGES)]), (uint32_t)((t2 / STAGES) & 1));
+  }
+#ifdef IM_DBG_STACK
+  if (DYN && lane == 0) atomicAdd(dbg + 5, (unsigned long long)n_done);
+#endif
+  if (DYN) {
+    __syncthreads();
+#ifdef IM_DBG_STACK
+    if (threadIdx.x == 0) dbg[4] = dbg_now();
+#endif
+    if (threadIdx.x == 0) im_claim_exit(sc.claim);
   }
 }
 
@@ -377,17 +476,37 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 constexpr int RC_COLS = 64;
 constexpr int RC_THREADS = 256;
 constexpr int RC_RPR = RC_THREADS / 16;  // rows per round
-template <int RC_DEPTH>
+// DYN (pipelined stack calls): a block claims a worker id and then takes items from a counter, always one item
+// ahead of the one it works on (the first loads of the next item are requested while the current one is added up),
+// instead of owning the run of items its index names; see k_attn_stream for why.
+template <int RC_DEPTH, bool DYN>
 __device__ __forceinline__ void readout_cols_body(const ImDims& p, const ImState& st, const ImScratch& sc, const ImCall& call) {
   extern __shared__ float s_phi[];  // phi(q) of the current sequence, zero beyond dM
   __shared__ float4 s_red[RC_RPR][RC_COLS / 4];
+  __shared__ int s_take[2];
   const int tid = threadIdx.x;
   const int rsub = tid >> 4, c4 = tid & 15;  // row within a round, float4 within the slice
   const int nsl = p.Dkv / RC_COLS;
   const int total = call.n_seq * nsl;
-  const int t0 = (int)((long long)blockIdx.x * total / gridDim.x);
-  const int t1 = (int)((long long)(blockIdx.x + 1) * total / gridDim.x);
-  if (t0 >= t1) return;
+  int t = 0, t_next = 0, t_end = total;  // current item, the one after it, end of the items (of this block's run)
+  if (DYN) {
+    if (tid == 0) {
+      const int wid = im_claim_worker(call, sc.claim + 4, call.ro_claim);
+      s_take[0] = wid < 0 ? total : atomicAdd(sc.claim + 7, 1);
+      s_take[1] = wid < 0 ? total : atomicAdd(sc.claim + 7, 1);
+    }
+    __syncthreads();
+    t = s_take[0];
+    t_next = s_take[1];
+  } else {
+    t = (int)((long long)blockIdx.x * total / gridDim.x);
+    t_end = (int)((long long)(blockIdx.x + 1) * total / gridDim.x);
+    t_next = t + 1;
+  }
+  if (t >= t_end) {
+    if (DYN && tid == 0) im_claim_exit(sc.claim + 4);
+    return;
+  }
   const int nb = (p.dM + RC_RPR * RC_DEPTH - 1) / (RC_RPR * RC_DEPTH);  // batches of RC_DEPTH rounds per item
   const uint64_t pol = policy_evict_first();
   const ImRows r = im_rows(p);
@@ -399,12 +518,12 @@ __device__ __forceinline__ void readout_cols_body(const ImDims& p, const ImState
   };
   float4 v[RC_DEPTH];
   {
-    const float4* src = batch_ptr(t0, 0);
+    const float4* src = batch_ptr(t, 0);
 #pragma unroll
     for (int k = 0; k < RC_DEPTH; ++k) v[k] = ldg_stream(src + (size_t)min(k * RC_RPR + rsub, p.dM - 1) * row_f4, pol);
   }
   int cur = -1;
-  for (int t = t0; t < t1; ++t) {
+  while (t < t_end) {
     const int i = t / nsl;
     if (i != cur) {  // (block uniform)
       if (cur >= 0) __syncthreads();
@@ -413,10 +532,11 @@ __device__ __forceinline__ void readout_cols_body(const ImDims& p, const ImState
       cur = i;
       __syncthreads();
     }
+    if (DYN && tid == 0) s_take[0] = t_next < total ? atomicAdd(sc.claim + 7, 1) : total;  // the item after the next
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int b = 0; b < nb; ++b) {
-      const bool more = b + 1 < nb || t + 1 < t1;
-      const float4* src = more ? (b + 1 < nb ? batch_ptr(t, b + 1) : batch_ptr(t + 1, 0)) : nullptr;
+      const bool more = b + 1 < nb || t_next < t_end;
+      const float4* src = more ? (b + 1 < nb ? batch_ptr(t, b + 1) : batch_ptr(t_next, 0)) : nullptr;
       const int row_next = b + 1 < nb ? (b + 1) * RC_RPR * RC_DEPTH + rsub : rsub;
       const float* ph = s_phi + b * RC_RPR * RC_DEPTH + rsub;
 #pragma unroll
@@ -438,15 +558,22 @@ __device__ __forceinline__ void readout_cols_body(const ImDims& p, const ImState
       }
       reinterpret_cast<float4*>(sc.rpart + (size_t)i * p.Dkv + (size_t)(t % nsl) * RC_COLS)[tid] = sum;
     }
+    const int t_after = DYN ? s_take[0] : t_next + 1;  // (written by thread 0 before the barrier above)
     __syncthreads();
+    t = t_next;
+    t_next = t_after;
   }
+  if (DYN && tid == 0) im_claim_exit(sc.claim + 4);
 }
 
 __global__ void __maxnreg__(168) k_readout_cols(ImDims p, ImState st, ImScratch sc, ImCall call) {
-  readout_cols_body<32>(p, st, sc, call);
+  readout_cols_body<32, false>(p, st, sc, call);
+}
+__global__ void __maxnreg__(168) k_readout_cols_dyn(ImDims p, ImState st, ImScratch sc, ImCall call) {
+  readout_cols_body<32, true>(p, st, sc, call);
 }
 __global__ void __maxnreg__(64) k_readout_cols_light(ImDims p, ImState st, ImScratch sc, ImCall call) {
-  readout_cols_body<8>(p, st, sc, call);
+  readout_cols_body<8, false>(p, st, sc, call);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1047,16 +1174,21 @@ cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, vo
 
 size_t im_attn_smem_bytes(const ImDims& p) {
   const size_t stage = (size_t)2 * TILE * p.d * 2;
-  return (size_t)WARPS * STAGES * stage + (size_t)WARPS * STAGES * 8 + (IM_MAX_CALL_SEQS + 1) * 8 + IM_MAX_CALL_SEQS * 4 + 64;
+  return (size_t)WARPS * STAGES * stage + (size_t)WARPS * STAGES * 8 + (IM_MAX_CALL_SEQS + 1) * 8 + IM_MAX_CALL_SEQS * 4 + (1 + WARPS * 4) * 4 + 64;
 }
 
 cudaError_t im_attn_prepare(const ImDims& p) {
   const int smem = (int)im_attn_smem_bytes(p);
-  cudaError_t e = cudaFuncSetAttribute(k_attn_stream<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_attn_stream<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_stream<64>);
-  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_stream<128>);
+  cudaError_t e = cudaFuncSetAttribute(k_attn_stream<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_attn_stream<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_attn_stream<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_attn_stream<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_stream<64, false>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_stream<128, false>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_stream<64, true>);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_stream<128, true>);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_readout_cols);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_readout_cols_dyn);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_readout_cols_light);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_readout_finish);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_attn_merge_rows<64, bf16>);
@@ -1073,7 +1205,8 @@ cudaError_t im_launch_readout(const ImLaunch& L, const ImCall& call, int grid, i
   const int items = call.n_seq * (p.Dkv / RC_COLS);
   const size_t smem = (size_t)nb * RC_RPR * depth * 4;
   const int blocks = std::max(1, std::min(grid, items));
-  if (light) k_readout_cols_light<<<blocks, RC_THREADS, smem, L.stream>>>(p, L.st, L.sc, call);
+  if (call.stack) k_readout_cols_dyn<<<blocks, RC_THREADS, smem, L.stream>>>(p, L.st, L.sc, call);
+  else if (light) k_readout_cols_light<<<blocks, RC_THREADS, smem, L.stream>>>(p, L.st, L.sc, call);
   else k_readout_cols<<<blocks, RC_THREADS, smem, L.stream>>>(p, L.st, L.sc, call);
   ++*L.launches;
   return cudaGetLastError();
@@ -1103,8 +1236,13 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   cfg.attrs = &attr;
   cfg.numAttrs = programmatic ? 1 : 0;
   cudaError_t e;
-  if (p.d == 64) e = cudaLaunchKernelEx(&cfg, k_attn_stream<64>, mk, mv, p, L.st, L.sc, call, (const bf16*)q);
-  else e = cudaLaunchKernelEx(&cfg, k_attn_stream<128>, mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+  if (call.stack) {
+    if (p.d == 64) e = cudaLaunchKernelEx(&cfg, k_attn_stream<64, true>, mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+    else e = cudaLaunchKernelEx(&cfg, k_attn_stream<128, true>, mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+  } else {
+    if (p.d == 64) e = cudaLaunchKernelEx(&cfg, k_attn_stream<64, false>, mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+    else e = cudaLaunchKernelEx(&cfg, k_attn_stream<128, false>, mk, mv, p, L.st, L.sc, call, (const bf16*)q);
+  }
   ++*L.launches;
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -137,6 +137,9 @@ struct ImScratch {   // per call, shared by all layers, stream ordered
   int32_t* hnhole;   // [max_seqs][Hkv]       holes below the budget per head
   int32_t* hrowmap;  // [max_seqs][Hkv][tail] row of the memory write that an evicted (head, entry) pair belongs to
   int32_t* hntok;    // [max_seqs]            rows (tokens that lose a slice) of the evict step
+  int32_t* claim;    // [8] worker claiming of the persistent streaming kernels in a pipelined stack call (im_claim_worker):
+                     // (arrivals and ids, -, blocks ended, next piece of work) of the attention kernel at [0..3], of the readout
+                     // kernel at [4..7]; zero between launches
 #ifdef IM_TRACE
   unsigned long long* trace;  // [n_layers][IM_TRACE_KERNELS][IM_TRACE_MARKS] nanosecond time stamps (development builds)
 #endif
@@ -183,13 +186,68 @@ struct ImCall {
   // decode: 1 = the attention kernel may read this layer's counters and cache before the kernel ahead of it in the
   // stream has ended (that kernel is the merge of a call on another layer); 0 = it waits for that kernel first
   int early_cache;
+  // Pipelined stack call (im_decode_stack): the layers of the call overlap, so the occupancy rules that keep the
+  // streaming kernels off the SMs set aside for the chain of small kernels no longer hold (a streaming kernel of the
+  // next layer starts when SMs of either kind happen to be free).  The split is made by SM id instead: the persistent
+  // streaming kernels are launched with one block per SM, a block reads %smid and claims a worker id only on an SM
+  // whose bit is set in sm_stream; see im_claim_worker.
+  int stack;                        // 1 = the streaming kernels claim their worker ids
+  int att_workers, ro_claim;        // blocks of the attention / readout kernel of the call that are to work
+  int att_chunks;                   // runs the attention kernel's tiles are cut into (taken from a counter)
+  unsigned long long sm_stream[4];  // bit s set: SM s runs streaming blocks
   int seq[IM_MAX_CALL_SEQS];
 };
+#define IM_STACK_LANES 3     /* layers of a pipelined stack call in flight (scratch sets, stream sets) */
+#define IM_CLAIM_POLLS 12    /* one-microsecond naps of a block that stays off the workers' SMs until the workers are placed */
 __device__ __forceinline__ void im_warm_inputs(const ImCall& call, int part, int tid, int nthreads) {
   if (part >= 5 || !call.warm[part]) return;
   const char* b = static_cast<const char*>(call.warm[part]);
   for (size_t off = (size_t)tid * 128; off < call.warm_bytes[part]; off += (size_t)nthreads * 128)
     asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(b + off));
+}
+
+// Worker claiming (ImCall::stack).  The grid has at least n_workers blocks; tk[0] holds (blocks arrived << 16 | ids
+// claimed) and tk[2] the blocks that have ended, both zero when the launch starts.  Called by one thread of a block, it
+// returns the block's worker id in [0, n_workers) or -1 (the block has nothing to do).  A block on a streaming SM
+// arrives and claims in one atomic add and works if its id is below n_workers.  A block on another SM arrives with an
+// add of its own and leaves without an id, but only if, by the counts that add returned, the blocks still to come
+// could claim every id that is left; otherwise it claims like a streaming block.  The count of blocks to come thus
+// never falls below the count of ids left (a claim lowers both; a block leaves only where the inequality holds
+// after its arrival, and it judges by a claim count that can only be too low): whatever the block scheduler does,
+// every id is claimed by exactly one block, and the SM split only decides where.  No add is ever retried: a
+// compare-and-swap loop here cost every launch 60 us, one memory round trip per block, one block after the other.
+// A block that leaves stays resident for a moment (until the ids are gone, IM_CLAIM_POLLS naps at most) so that the
+// blocks still queued are not all dispatched to its SM, one after the other, while the workers' SMs are still busy
+// with the previous launch.  Every block, with or without an id, ends with im_claim_exit; the last one clears the
+// counters.
+__device__ __forceinline__ int im_claim_worker(const ImCall& call, int32_t* tk, int n_workers) {
+  unsigned smid;
+  asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+  const bool streaming = smid < 256u && ((call.sm_stream[smid >> 6] >> (smid & 63u)) & 1ull);
+  unsigned* word = reinterpret_cast<unsigned*>(tk);
+  if (streaming) {
+    const int id = (int)(atomicAdd(word, (1u << 16) + 1u) & 0xffffu);
+    return id < n_workers ? id : -1;
+  }
+  const unsigned old = atomicAdd(word, 1u << 16);
+  const int arrived = (int)(old >> 16), claimed = (int)(old & 0xffffu);
+  if (claimed >= n_workers) return -1;
+  if ((int)gridDim.x - 1 - arrived >= n_workers - claimed) {
+    for (int it = 0; it < IM_CLAIM_POLLS; ++it) {
+      __nanosleep(1000);
+      if ((int)(*reinterpret_cast<volatile unsigned*>(word) & 0xffffu) >= n_workers) break;
+    }
+    return -1;
+  }
+  const int id = (int)(atomicAdd(word, 1u) & 0xffffu);
+  return id < n_workers ? id : -1;
+}
+__device__ __forceinline__ void im_claim_exit(int32_t* tk) {
+  if (atomicAdd(tk + 2, 1) == (int)gridDim.x - 1) {
+    tk[0] = 0;
+    tk[2] = 0;
+    tk[3] = 0;  // (the kernel's work counter)
+  }
 }
 
 // Skinny GEMM arguments: out[v][row0 + r] (+)= sum_k (W[r][k] + W2[r][k]) * in[v][k].
@@ -337,6 +395,7 @@ cudaError_t im_launch_decode_front(const ImLaunch& L, const ImCall& call, const 
                                    int do_select, int n_max, int smem_floor, cudaEvent_t started = nullptr, int programmatic = 0);
 cudaError_t im_launch_prefetch_layer(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_prefetch_memory(const ImLaunch& L, const ImCall& call, int eighths, int per_block = 1);
+cudaError_t im_probe_sm_ids(void* map, int n_sm, int* ids, int* n, cudaStream_t stream);
 cudaError_t im_launch_gather_move(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_gather(const ImLaunch& L, const ImCall& call, int ne_max);
 cudaError_t im_launch_move(const ImLaunch& L, const ImCall& call, int ne_max);

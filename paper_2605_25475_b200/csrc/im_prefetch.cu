@@ -67,7 +67,42 @@ __global__ void __launch_bounds__(512) k_prefetch_memory(ImDims p, ImState st, I
   }
 }
 
+// Marks the id of the SM a block runs on in a 256-bit map (ids beyond 255: bit 31 of word 8).  Blocks of 1024 threads
+// that nap for a while, several waves of them, so that every SM gets one.
+__global__ void __launch_bounds__(1024) k_probe_sm_ids(uint32_t* map) {
+  if (threadIdx.x == 0) {
+    unsigned smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    if (smid < 256u) atomicOr(map + (smid >> 5), 1u << (smid & 31u));
+    else atomicOr(map + 8, 0x80000000u);
+    __nanosleep(8000);
+  }
+  __syncthreads();
+}
+
 }  // namespace
+
+// The ids (%smid) of the device's SMs, ascending, as blocks of a probe kernel report them; `map` is device scratch of
+// at least 64 bytes.  *n = 0 if the ids do not number n_sm distinct values below 256 (the caller then does without).
+cudaError_t im_probe_sm_ids(void* map, int n_sm, int* ids, int* n, cudaStream_t stream) {
+  *n = 0;
+  cudaError_t e = cudaMemsetAsync(map, 0, 64, stream);
+  if (e != cudaSuccess) return e;
+  k_probe_sm_ids<<<8 * n_sm, 1024, 0, stream>>>(static_cast<uint32_t*>(map));
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  uint32_t host[16];
+  if ((e = cudaMemcpyAsync(host, map, 64, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return e;
+  if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return e;
+  if (host[8]) return cudaSuccess;
+  int k = 0;
+  for (int s = 0; s < 256; ++s)
+    if ((host[s >> 5] >> (s & 31)) & 1u) {
+      if (k < n_sm) ids[k] = s;
+      ++k;
+    }
+  if (k == n_sm) *n = k;
+  return cudaSuccess;
+}
 
 // `call.layer` names the layer to warm up.  Needs 16-byte aligned matrices whose eighth is a multiple of 4 KB.
 cudaError_t im_launch_prefetch_memory(const ImLaunch& L, const ImCall& call, int eighths, int per_block) {

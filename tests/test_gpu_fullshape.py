@@ -131,7 +131,7 @@ class SampledUnits:
                 assert pos.max() < T_expect
 
 
-def _decode_under_graph_replay(su, n_steps, full_check_every=16):
+def _decode_under_graph_replay(su, n_steps, full_check_every=16, stack_call=False):
     """bench.py's launch configuration: static input buffers, the step of all layers captured once into a CUDA graph
     and replayed, the library's side streams on.  After every replay the sampled units' outputs and retained sets
     are compared with the oracle; every `full_check_every` steps and at the end, their whole state."""
@@ -154,6 +154,9 @@ def _decode_under_graph_replay(su, n_steps, full_check_every=16):
         return ins
 
     def one_step():
+        if stack_call:   # all layers in one call, the layers overlapping
+            g.decode_stack(list(range(L)), su.ids, sx, sqp, sq, sk, sv, out)
+            return
         for layer in range(L):
             g.decode_step(layer, su.ids, sx[layer], sqp[layer], sq[layer], sk[layer], sv[layer], out[layer])
 
