@@ -252,18 +252,42 @@ def measure_decode(wl, device, steps, warmup, graph=True, rank=0, world=1, log=l
             # CUDA events around the attention launch on this stream - once in the concurrent schedule the timed steps
             # ran (the kernel next to the readout kernel and the chain of small kernels, on the SMs the schedule
             # leaves it), once with the side streams off (the kernel alone on all SMs, against the burst peak)
+            # (with a stack call per step the first pass makes stack calls: the events then sit on the stream that
+            # carries the attention kernels of all layers back to back)
             prof_steps = -(-min(steps, 32) // tau) * tau            # whole intervals
             for name, conc in (("in_step", 1), ("alone", 0)):
                 im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, conc)
                 im.im_profile_begin(g.ctx, prof_steps * L)
                 for s in range(prof_steps):
-                    one_step(s, stack=False)          # (the library times the attention launch of a layer call)
+                    one_step(s, stack=stack_call and conc == 1)
                 k_ms, k_n = im.im_profile_end(g.ctx)
                 res["attn_ms_" + name], res["attn_n_" + name] = k_ms, k_n
             im.im_set_option(g.ctx, im.IM_OPT_CONCURRENCY, 1)
+        if stack_call and graph and tau == 1:
+            # the same steps as one im_decode_step call per layer (what a model whose layers depend on one another
+            # would run), replayed from graphs of their own, for comparison in the same process
+            lgraphs = []
+            for k in range(n_in):
+                gk = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gk, stream=stream):
+                    one_step(k, stack=False)
+                lgraphs.append(gk)
+            n_cmp = min(steps, 64)
+            for k in range(3):
+                lgraphs[k % n_in].replay()
+            stream.synchronize()
+            ev0.record(stream)
+            for k in range(n_cmp):
+                lgraphs[k % n_in].replay()
+            ev1.record(stream)
+            stream.synchronize()
+            res["layer_calls_ms"] = max_over_ranks(ev0.elapsed_time(ev1), world, device) / n_cmp
+            res["layer_calls_steps"] = n_cmp
+            del lgraphs
+            assert g.status() == 0
         if e2e_args is not None:
             # end to end: host buffers in, host buffer out, copies inside the timed region
-            res["e2e"] = run_e2e(e2e_args, wl, g, ids, inputs, stream, world, device)
+            res["e2e"] = run_e2e(e2e_args, wl, g, ids, inputs, stream, world, device, stack_call=stack_call)
     del graphs
     g.close()
     return res
@@ -294,6 +318,7 @@ def run_ours(args, rank, world, device):
                 "frac": ab["attn_launch"] / sec / 1e9 / peaks["hbm_gbs"]}
     alone, in_step = rate(m["attn_ms_alone"], m["attn_n_alone"]), rate(m["attn_ms_in_step"], m["attn_n_in_step"])
     full = wl.name == "llama8b_stack" and not args.tau and not args.layers and not args.context
+    stack = bool(args.stack_call) and wl.n_layers >= 2 and not args.score_share
     res = {
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -303,6 +328,9 @@ def run_ours(args, rank, world, device):
                    "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H,
                    "kv_heads": wl.Hkv, "head_dim": wl.d, "context": wl.ctx, "budget": wl.B, "tau": wl.tau,
                    "cuda_graph": m["cuda_graph"], "score_share": args.score_share,
+                   "call": ("one im_decode_stack call per step: the inputs of all layers are resident when the step starts "
+                            "(a stack driven from synthetic activations), so the call overlaps the layers"
+                            if stack else "one im_decode_step call per layer"),
                    "l2": "inputs larger than L2 (each step streams %.1f GB)" % (ab["step"] / 1e9)},
         "hbm_gbs_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9,
         "hbm_frac_step": ab["step"] / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -314,9 +342,18 @@ def run_ours(args, rank, world, device):
                      "traffic_source": ("profiles/k_attn_stream_llama8b_stack_2layers_ctx4096.md (ncu dram__bytes_read.sum + "
                                         "dram__bytes_write.sum of one launch of this size; a constant, not measured in this run)") if full else None,
                      "bytes_per_launch": ab["attn_launch"], "us_per_launch": alone["us_per_launch"],
-                     "in_step": dict(in_step, schedule="concurrent schedule of the timed steps: the kernel on the SMs left by the "
-                                                      "front kernel, next to the readout kernel (un-graphed, CUDA events around the launch)")},
+                     "in_step": dict(in_step, schedule=(
+                         "schedule of the timed steps: the attention kernels of the step's layers back to back on one stream, "
+                         "next to the readout kernels and the small kernels of the layers in flight (un-graphed, CUDA events "
+                         "around each launch on that stream)" if stack else
+                         "concurrent schedule of the timed steps: the kernel on the SMs left by the front kernel, next to the "
+                         "readout kernel (un-graphed, CUDA events around the launch)"))},
         "merge_recomputes_per_step": m["recomputes"] / args.steps,
+        "layer_calls": ({"ms_per_step": m["layer_calls_ms"], "tokens_per_s": wl.n_seq * world / (m["layer_calls_ms"] * 1e-3),
+                         "steps": m["layer_calls_steps"],
+                         "note": "the same steps as one im_decode_step call per layer (layers in sequence, as in a model "
+                                 "whose layers depend on one another), graph replay, same process"}
+                        if "layer_calls_ms" in m else None),
         "e2e": m["e2e"], "gpu_launches": int(round(m["launches_per_step"] * args.steps)), "clocks": m["clocks"],
     }
     return res, wl
@@ -359,7 +396,7 @@ def secondary_block(args, device, log):
     log(f"secondary mistral7b_prefill: {out['mistral7b_prefill']['ms_per_prompt']:.2f} ms per prompt")
     # the paper's compression interval on the headline stack
     wl = synth.CONFIGS["llama8b_stack"].replace(tau=128)
-    m = measure_decode(wl, device, 128, 128, log=log, profile=False)
+    m = measure_decode(wl, device, 128, 128, log=log, profile=False, stack_call=True)
     ab = algorithmic_bytes(wl)
     sec = m["ms"] / 128 * 1e-3
     out["llama8b_stack_tau128"] = {
@@ -482,7 +519,7 @@ def run_prefill(args, device):
 ATTN_TRAFFIC_NCU = 272.0e6
 
 
-def run_e2e(args, wl, g, ids, inputs, stream, world, device):
+def run_e2e(args, wl, g, ids, inputs, stream, world, device, stack_call=False):
     L = wl.n_layers
     n_in = len(inputs)
     # one pinned host buffer and one device buffer per input set / step: [L][x | q_pre | q | k | v] (bf16), so that a
@@ -514,9 +551,36 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     ev_out = [torch.cuda.Event() for _ in range(L)]
     ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
 
+    n_groups = 4 if (stack_call and L % 4 == 0 and L >= 8) else 0
+
+    def enqueue_groups(k):
+        """One step made of stack calls over groups of L / 4 consecutive layers: the inputs of group g + 1 are copied
+        in and the outputs of group g - 1 copied out while the stack call of group g runs."""
+        hb = host[k]
+        per = L // n_groups
+        ev_fork.record(stream)
+        cs.wait_event(ev_fork)
+        ds.wait_event(ev_fork)
+        for gi in range(n_groups):
+            a, b = gi * per, (gi + 1) * per
+            with torch.cuda.stream(cs):
+                dbuf[a:b].copy_(hb[a:b], non_blocking=True)
+                tick[gi:gi + 1].fill_(1.0)           # (see below: the calls depend on a kernel, not on the copy node)
+                ev_in[gi].record(cs)
+            stream.wait_event(ev_in[gi])
+            g.decode_stack(list(range(a, b)), ids, dx[a:b], dqp[a:b], dq[a:b], dk[a:b], dv[a:b], dout[a:b])
+            ev_out[gi].record(stream)
+            ds.wait_event(ev_out[gi])
+            with torch.cuda.stream(ds):
+                hout[a:b].copy_(dout[a:b], non_blocking=True)
+        ev_join.record(ds)
+        stream.wait_event(ev_join)
+
     def enqueue(k):
         """One step: the copies of layer l + 1's inputs and of layer l - 1's outputs run next to layer l's
         kernels (three streams, forked from and joined back into `stream`, so that it can be captured)."""
+        if n_groups:
+            return enqueue_groups(k)
         hb = host[k]
         ev_fork.record(stream)
         cs.wait_event(ev_fork)
@@ -577,7 +641,9 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device):
     barrier(world)
     ms = max_over_ranks(ev0.elapsed_time(ev1), world, device)
     return {"value": wl.n_seq * args.steps * world / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "ms_per_step": ms / args.steps, "cuda_graph": graphs is not None}
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms / args.steps, "cuda_graph": graphs is not None,
+            "calls_per_step": ("%d im_decode_stack calls over %d layers each" % (n_groups, L // n_groups)) if n_groups
+                              else "%d im_decode_step calls" % L}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -681,7 +747,7 @@ def main():
                     help="g >= 2: layers l with l %% g != 0 reuse the indexer scores of layer l - l %% g (the paper's appendix uses 4)")
     ap.add_argument("--readout-stages", type=int, default=-1,
                     help="0: readout on plain loads; k >= 1: on a ring of k 32 KB bulk copies per CTA (default: the library's choice)")
-    ap.add_argument("--stack-call", type=int, default=0,
+    ap.add_argument("--stack-call", type=int, default=1,
                     help="1: a step is one im_decode_stack call over all layers (the layers overlap); 0: one im_decode_step call per layer")
     ap.add_argument("--stack-reserved", type=int, default=-1,
                     help="SMs a pipelined stack call keeps free of streaming blocks (default: the library's choice)")

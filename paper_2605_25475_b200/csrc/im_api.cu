@@ -237,7 +237,6 @@ struct HostUnit {
   int n = 0;       // cached entries
   long long T = 0; // tokens seen
   int since = 0;   // decode tokens since the last compression
-  int npend = 0;   // pending rank-one writes
 };
 
 }  // namespace
@@ -388,14 +387,6 @@ int pick_ksplit(int K, int want) {
   for (int s = want; s > 1; --s)
     if (K % (16 * s) == 0) return s;
   return 1;
-}
-
-// Host mirror of the pending-list bookkeeping the memory kernels do on the device.
-void mirror_memory(const ImDims& p, HostUnit& u, int ne) {
-  if (!p.mem || ne <= 0) return;
-  if (ne > p.F) { u.npend = 0; return; }
-  if (u.npend + ne > p.F) u.npend = 0;
-  u.npend += ne;
 }
 
 // the state update of Eq. 6-7 with the per-sequence evicted counts of this call from the host mirror (must be
@@ -1026,8 +1017,6 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
     const int ne = std::max(0, u.n + chunk_len - p.B);
-    if (call.fold_all) u.npend = 0;
-    mirror_memory(p, u, ne);
     u.n = u.n + chunk_len - ne;
     u.T += chunk_len;
     u.since = 0;
@@ -1333,7 +1322,6 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
     const int ne = due ? std::max(0, u.n + 1 - p.B) : 0;
-    mirror_memory(p, u, ne);
     u.n = u.n + 1 - ne;
     u.T += 1;
     u.since = due ? 0 : u.since + 1;
@@ -1501,7 +1489,13 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
   CK(cudaEventRecord(ln.ev[6], L2.stream));
   // a5 on the call's attention stream: behind the previous layer's attention kernel as its programmatic dependent
   // (it becomes resident as that kernel's blocks end, and waits for nothing)
+  const bool prof = ctx->prof_target == 0 && ctx->prof_used + 2 <= ctx->prof_ev.size();
+  if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], LA.stream));
   CKL(im_launch_attention_fast(LA, call, ctx->mapKs, ctx->mapVs, q, std::max(ctx->n_sm, call.att_workers), j > 0 ? 1 : 0));
+  if (prof) {
+    CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], LA.stream));
+    ctx->prof_used += 2;
+  }
   CK(cudaEventRecord(ln.ev[9], LA.stream));
   // s4: the part of the readout that does not go through Mhat, over the memory as it is before this call's write
   CK(cudaStreamWaitEvent(L4.stream, ln.ev[6], 0));
@@ -1524,7 +1518,6 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
   for (int i = 0; i < n_seq; ++i) {
     HostUnit& u = ctx->hu[(size_t)layer * p.S + call.seq[i]];
     const int ne = due ? std::max(0, u.n + 1 - p.B) : 0;
-    mirror_memory(p, u, ne);
     u.n = u.n + 1 - ne;
     u.T += 1;
     u.since = due ? 0 : u.since + 1;
@@ -1912,7 +1905,6 @@ int im_state_import(im_ctx* ctx, int layer, int seq, int which, const void* host
       hu.n = ctr[CTR_N];
       hu.T = ctr[CTR_T];
       hu.since = ctr[CTR_SINCE];
-      hu.npend = 0;
       return IM_OK;
     }
     case IM_S_POS:
@@ -1943,7 +1935,6 @@ int im_state_import(im_ctx* ctx, int layer, int seq, int which, const void* host
       const int32_t zero = 0;
       CK(cudaMemcpy(st.cscale + u, &one, 4, cudaMemcpyHostToDevice));
       CK(cudaMemcpy(st.ctr + u * CTR_STRIDE + CTR_NPEND, &zero, 4, cudaMemcpyHostToDevice));
-      hu.npend = 0;
       return IM_OK;
     }
     case IM_S_B:

@@ -28,7 +28,9 @@ def test_decode_line_has_the_contract_keys():
     assert d["value"] > 0 and d["ms_per_step"] > 0 and d["gpu_launches"] >= 6 * 2 * 10
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and 0 < r["frac"] < 1.5 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
-    assert "alone" in r["schedule"] and r["in_step"]["us_per_launch"] > 0 and "concurrent" in r["in_step"]["schedule"]
+    assert "alone" in r["schedule"] and r["in_step"]["us_per_launch"] > 0 and "schedule of the timed steps" in r["in_step"]["schedule"]
+    # the step is one stack call over the layers; the layer-by-layer figure is reported next to it
+    assert "im_decode_stack" in d["config"]["call"] and d["layer_calls"]["ms_per_step"] > 0
     assert d["clocks"]["samples"] >= 1
     e = d["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0

@@ -185,17 +185,19 @@ def _decode_under_graph_replay(su, n_steps, full_check_every=16, stack_call=Fals
     assert np.isfinite(out.float().cpu().numpy()).all()
 
 
-def test_stack_config_at_full_size_under_graph_replay():
+@pytest.mark.parametrize("stack_call", [1, 0])
+def test_stack_config_at_full_size_under_graph_replay(stack_call):
     """The headline configuration as stated: 32 layers x 32 sequences, 32 q / 8 KV heads of 128, 16384-token context
     ingested in eight 2048-token chunks with eviction to B = 2048 after each, then its 64 decode steps replayed from
     one CUDA graph (one eviction per sequence and step; the 16-entry pending list of every unit is folded into the
-    memory four times).  Four units in four layers follow the oracle through all chunks and steps."""
+    memory four times).  Four units in four layers follow the oracle through all chunks and steps.  Once with the step
+    as one im_decode_stack call over the 32 layers (what the benchmark times), once as 32 im_decode_step calls."""
     wl = synth.CONFIGS["llama8b_stack"]
-    su = SampledUnits(wl, [(0, 5), (13, 29), (22, 0), (31, 18)])
+    su = SampledUnits(wl, [(0, 5), (13, 29), (22, 0), (31, 18)] if stack_call else [(1, 30), (12, 3), (23, 16), (30, 9)])
     for c in range(wl.ctx // wl.chunk):
         su.prefill(c)
     su.check_properties(wl.B, wl.ctx, n_evicted=wl.chunk, stride=11)
-    _decode_under_graph_replay(su, wl.steps)
+    _decode_under_graph_replay(su, wl.steps, stack_call=bool(stack_call))
     su.check_properties(wl.B, wl.ctx + wl.steps, n_evicted=1, stride=11)
     for o in su.oracles.values():
         assert o.evict_steps(0) == wl.ctx // wl.chunk - 1 + wl.steps
