@@ -303,8 +303,6 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        im_decode_step layer by layer.
  *   IM_OPT_STACK_RESERVED k >= 1: SMs that a pipelined im_decode_stack keeps free of streaming blocks, for the small
  *                        kernels of the layers in flight; 0 (default): one per sequence of the call.
- *   IM_OPT_STACK_SPREAD  which SMs a pipelined im_decode_stack sets aside: 2 (default) pairs of neighbouring SM ids at even
- *                        distances over the id range, 1 single SMs at even distances, 0 the highest ids.
  *   IM_OPT_STACK_CHUNKS  k in [1, 16] (default 4): a pipelined im_decode_stack cuts the tiles of a layer's attention into k
  *                        runs per warp, which the warps take from a counter.  With k = 1 the runs, and with them the
  *                        order of every float32 sum, are those of im_decode_step: the two then agree bit for bit.
@@ -327,8 +325,7 @@ typedef enum im_option {
   IM_OPT_LAYER_OVERLAP = 7,
   IM_OPT_STACK_PIPELINE = 8,
   IM_OPT_STACK_RESERVED = 9,
-  IM_OPT_STACK_CHUNKS = 10,
-  IM_OPT_STACK_SPREAD = 11
+  IM_OPT_STACK_CHUNKS = 10
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 

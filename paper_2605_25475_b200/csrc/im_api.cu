@@ -299,9 +299,6 @@ struct im_ctx {
   std::vector<int> sm_ids;           // ids of the device's SMs (ascending) as a probe kernel saw them; empty: unknown
   bool stack_pipeline = true;        // IM_OPT_STACK_PIPELINE
   int stack_reserved = 0;            // IM_OPT_STACK_RESERVED: SMs kept free of streaming blocks (0: one per sequence)
-  int stack_spread = 2;              // IM_OPT_STACK_SPREAD: where the SMs set aside lie in the id range
-  int stack_ro_workers = 0;          // (development) blocks of the readout kernel that work (0: one per streaming SM)
-  int stack_floors = 0;              // (development) the small kernels of a stack call ask for their shared-memory floors
   int stack_chunks = 4;              // IM_OPT_STACK_CHUNKS: runs per warp the attention kernel's tiles are cut into
 #ifdef IM_TRACE
   int tune[8] = {0, -1, -1, 0, 0, 0, 0, 0};  // development builds: knobs set through options 100 + k
@@ -660,7 +657,7 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     int sms = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
     if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK, ctx->mapV, IM_ATTN_TILE);
-    if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapKs, ctx->mapVs, IM_ATTN_STREAM_TILE);
+    if (e == cudaSuccess) e = im_attn_make_maps(p, ctx->lo.st, ctx->mapKs, ctx->mapVs, IM_ATTN_STREAM_TILE, p.d == 128 ? 1 : 0);
     if (e == cudaSuccess) e = im_attn_prepare(p);
     if (e == cudaSuccess && im_attn_tc_supported(p)) {
       e = im_attn_make_maps(p, ctx->lo.st, ctx->mapK128, ctx->mapV128, IM_ATTN_TC_TILE);
@@ -1417,7 +1414,6 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
   const long long want = (tiles + IM_ATTN_WARPS * IM_ATTN_MIN_RUN - 1) / (IM_ATTN_WARPS * IM_ATTN_MIN_RUN);
   call.att_workers = (int)std::max<long long>(1, std::min<long long>(n_wk_max, want));
   call.ro_claim = (int)std::max<long long>(1, std::min<long long>(n_wk_max, (long long)n_seq * (p.Dkv / 64)));
-  if (ctx->stack_ro_workers > 0) call.ro_claim = std::min(call.ro_claim, ctx->stack_ro_workers);
   // runs the attention kernel's tiles are cut into: a few per warp, so that a block that starts late takes fewer
   call.att_chunks = std::min(call.att_workers * IM_ATTN_WARPS * ctx->stack_chunks, IM_ATTN_MAX_CTAS * IM_ATTN_WARPS);
   // streams: the lane's own wait for the lane's previous layer (its scratch set), or for the start of the call
@@ -1471,9 +1467,9 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
     g.key_dI = p.dI;
     call.ksplit_key = key_ride;
   }
-  g.smem_floor = ctx->stack_floors ? IM_SMEM_HEAD : 0;
+  // (no shared-memory floors here: in im_decode_step they keep the small kernels' blocks off the SMs of the attention
+  // blocks, in a stack call they would keep an attention block off an SM it finds free between two layers)
   CKL(im_launch_gemm(L1, g));
-  g.smem_floor = 0;
   g.key_W = nullptr;
   // s3: key projection; s4: fold of the pending list
   if (!key_ride) CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
@@ -1503,14 +1499,14 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
   CK(cudaEventRecord(ln.ev[4], L4.stream));
   // s1: append, score, select, gather, list the moves
   CK(cudaStreamWaitEvent(L1.stream, ln.ev[2], 0));
-  CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max, ctx->stack_floors ? IM_SMEM_FRONT : 0, nullptr, 1));
+  CKL(im_launch_decode_front(L1, call, k_new, v_new, fused ? 1 : 0, n_max, 0, nullptr, 1));
   // phi(q)^T Mhat on the call's readout stream
   CK(cudaStreamWaitEvent(LR.stream, ln.ev[6], 0));
   if (mem_write) CK(cudaStreamWaitEvent(LR.stream, ln.ev[7], 0));
   CKL(im_launch_readout(LR, call, std::max(ctx->n_sm, call.ro_claim), 0));
   CK(cudaEventRecord(ln.ev[12], LR.stream));
   // a3: phi of the evicted keys, then (off the path to the merge) the state update
-  if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, false, ctx->stack_floors ? IM_SMEM_SIDE : 0, nullptr, 0))) return rc;
+  if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, false, 0, nullptr, 0))) return rc;
   CK(cudaEventRecord(ln.ev[3], L1.stream));
   CK(cudaStreamWaitEvent(L1.stream, ln.ev[4], 0));
   if (mem_write) CKL(launch_mem_update(ctx, L1, call, ne_max));
@@ -1585,28 +1581,20 @@ extern "C" int im_decode_stack(im_ctx* ctx, int n_layers, const int32_t* layers,
   cudaStream_t s0 = (cudaStream_t)cuda_stream;
   CK(join_late(ctx, s0));
   ctx->tail_is_merge = false;
-  // SMs for the streaming kernels: all but n_res, which are taken at even distances over the id range so that every
-  // part of the chip keeps streaming blocks (ids that lie together share a path to the memory system; with the n_res
-  // highest ids set aside the streams reached three quarters of their rate).  IM_OPT_STACK_SPREAD 2: whole pairs
-  // (2k, 2k + 1) at even distances; 1: single SMs; 0: the highest ids.
+  // SMs for the streaming kernels: all but n_res, taken as pairs of neighbouring ids at even distances over the id
+  // range, so that every part of the chip keeps both kinds of SMs
   unsigned long long sm_stream[4] = {0, 0, 0, 0};
   {
     const int n = ctx->n_sm;
     std::vector<char> res(n, 0);
-    if (ctx->stack_spread == 0) {
-      for (int w = n - n_res; w < n; ++w) res[w] = 1;
-    } else if (ctx->stack_spread == 1 || n_res < 2) {
-      for (int k = 0; k < n_res; ++k) res[(int)(((long long)(2 * k + 1) * n) / (2 * n_res))] = 1;
-    } else {
-      const int pairs = n / 2, want = n_res / 2;
-      for (int k = 0; k < want; ++k) {
-        const int t = (int)(((long long)(2 * k + 1) * pairs) / (2 * want));
-        res[2 * t] = res[2 * t + 1] = 1;
-      }
-      if (n_res & 1)  // one more: the first free SM
-        for (int w = 0; w < n; ++w)
-          if (!res[w]) { res[w] = 1; break; }
+    const int pairs = n / 2, want = n_res / 2;
+    for (int k = 0; k < want; ++k) {
+      const int t = (int)(((long long)(2 * k + 1) * pairs) / (2 * want));
+      res[2 * t] = res[2 * t + 1] = 1;
     }
+    if (n_res & 1)  // one more: the first SM that is still free
+      for (int w = 0; w < n; ++w)
+        if (!res[w]) { res[w] = 1; break; }
     for (int w = 0; w < n; ++w)
       if (!res[w]) sm_stream[ctx->sm_ids[w] >> 6] |= 1ull << (ctx->sm_ids[w] & 63);
   }
@@ -1659,12 +1647,6 @@ int im_set_option(im_ctx* ctx, int option, int value) {
       return IM_OK;
     case IM_OPT_LAYER_OVERLAP: ctx->layer_overlap = value != 0; return IM_OK;
     case IM_OPT_STACK_PIPELINE: ctx->stack_pipeline = value != 0; return IM_OK;
-    case IM_OPT_STACK_SPREAD:
-      if (value < 0 || value > 2) return fail(IM_ERR_ARG, "placement %d: 0 highest ids, 1 single SMs at even distances, 2 pairs at even distances", value);
-      ctx->stack_spread = value;
-      return IM_OK;
-    case 12: ctx->stack_floors = value; return IM_OK;
-    case 13: ctx->stack_ro_workers = value; return IM_OK;
     case IM_OPT_STACK_CHUNKS:
       if (value < 1 || value > 16) return fail(IM_ERR_ARG, "runs per warp %d out of range [1,16]", value);
       ctx->stack_chunks = value;

@@ -19,14 +19,6 @@
 
 #include "im_internal.cuh"
 
-#ifdef IM_DBG_STACK
-__device__ unsigned long long g_dbg[32 * 160 * 8];
-extern "C" int im_dbg_read(unsigned long long* host) {
-  cudaDeviceSynchronize();
-  return (int)cudaMemcpyFromSymbol(host, g_dbg, sizeof(g_dbg));
-}
-__device__ __forceinline__ unsigned long long dbg_now() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#endif
 
 namespace {
 
@@ -71,6 +63,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(pol)
+      : "memory");
+}
+// one copy for a whole tile of a cache with 256-byte rows: box (64 columns, rows, 2 halves), see im_attn_make_maps
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(pol)
       : "memory");
 }
 __device__ __forceinline__ float4 ldg_stream(const float4* ptr, uint64_t pol) {
@@ -143,17 +142,10 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   // kernel ahead of it in its stream (the attention kernel of the previous layer, with a scratch set of its own), so
   // a programmatic dependent never waits for it.
   int wid = blockIdx.x;
-#ifdef IM_DBG_STACK
-  unsigned long long* dbg = g_dbg + ((size_t)(call.layer % 32) * 160 + blockIdx.x % 160) * 8;
-  if (DYN && threadIdx.x == 0) { unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); dbg[0] = smid; dbg[1] = dbg_now(); dbg[5] = 0; }
-#endif
   if (DYN) {
     if (threadIdx.x == 0) s_misc[0] = im_claim_worker(call, sc.claim, call.att_workers);
     __syncthreads();
     wid = s_misc[0];
-#ifdef IM_DBG_STACK
-    if (threadIdx.x == 0) { dbg[2] = (unsigned long long)(long long)wid; dbg[3] = dbg_now(); dbg[4] = dbg[3]; }
-#endif
     if (wid < 0) {
       if (threadIdx.x == 0) im_claim_exit(sc.claim);
       return;
@@ -245,10 +237,15 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const size_t u = (size_t)call.layer * p.S + call.seq[pi];
     const int row = (int)((u * p.Hkv + ph) * (size_t)p.cap) + ptt * TILE;
     mbar_expect_tx(bar, STAGE_BYTES);
-#pragma unroll
-    for (int b = 0; b < BOXES; ++b) {
-      tma_load_2d(dst + b * (TILE * 128), &tmK, b * 64, row, bar, pol);
-      tma_load_2d(dst + TILE_BYTES + b * (TILE * 128), &tmV, b * 64, row, bar, pol);
+    if (BOXES == 1) {
+      tma_load_2d(dst, &tmK, 0, row, bar, pol);
+      tma_load_2d(dst + TILE_BYTES, &tmV, 0, row, bar, pol);
+    } else {
+      // (one copy per tile and cache: the 128-byte halves of the rows are the map's third dimension, and the box lands
+      // in shared memory half by half, each half the 128-byte-swizzled rows that two 2-D boxes would leave; an SM's
+      // copy unit takes requests at a bounded rate, and with 4 KB boxes that rate, not the memory, bounded the kernel)
+      tma_load_3d(dst, &tmK, 0, row, 0, bar, pol);
+      tma_load_3d(dst + TILE_BYTES, &tmV, 0, row, 0, bar, pol);
     }
     ++n_issued;
     ++p_pos;
@@ -448,14 +445,8 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     for (long long t2 = n_done; t2 < n_issued; ++t2)
       mbar_wait(smem_u32(&bars[warp * STAGES + (int)(t2 % STAGES)]), (uint32_t)((t2 / STAGES) & 1));
   }
-#ifdef IM_DBG_STACK
-  if (DYN && lane == 0) atomicAdd(dbg + 5, (unsigned long long)n_done);
-#endif
   if (DYN) {
     __syncthreads();
-#ifdef IM_DBG_STACK
-    if (threadIdx.x == 0) dbg[4] = dbg_now();
-#endif
     if (threadIdx.x == 0) im_claim_exit(sc.claim);
   }
 }
@@ -1148,7 +1139,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 // box = 64 columns x box_rows rows, 128-byte swizzle.  Returns false if the fast path is unavailable.
 bool im_attn_fast_supported(const ImDims& p) { return (p.d == 64 || p.d == 128) && p.Gq <= 8 && p.Dkv % 4 == 0; }
 
-cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV, int box_rows) {
+// halves3d (head_dim 128 only): the 256-byte rows as two 128-byte halves on a third dimension, dims (64 columns, rows,
+// 2 halves) with strides (256, 128) bytes and box (64, box_rows, 2): one copy brings a whole tile, laid out in shared
+// memory as the two 2-D boxes of its halves would be.
+cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV, int box_rows, int halves3d) {
   static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -1163,10 +1157,19 @@ cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, vo
   const cuuint32_t estr[2] = {1, 1};
   void* bases[2] = {st.Kc, st.Vc};
   void* maps[2] = {mapK, mapV};
+  const cuuint64_t dims3[3] = {64, rows, 2};
+  const cuuint64_t strides3[2] = {(cuuint64_t)p.d * 2, 128};
+  const cuuint32_t box3[3] = {64, (cuuint32_t)box_rows, 2};
+  const cuuint32_t estr3[3] = {1, 1, 1};
+  if (halves3d && p.d != 128) return cudaErrorInvalidValue;
   for (int k = 0; k < 2; ++k) {
-    CUresult r = enc((CUtensorMap*)maps[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bases[k], dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = halves3d
+        ? enc((CUtensorMap*)maps[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, bases[k], dims3, strides3, box3, estr3,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE)
+        : enc((CUtensorMap*)maps[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bases[k], dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
   return cudaSuccess;

@@ -424,7 +424,7 @@ cudaError_t im_launch_chunk_attention_tc(const ImLaunch& L, const ImCall& call, 
 cudaError_t im_launch_select(const ImLaunch& L, const ImCall& call);
 cudaError_t im_launch_attention(const ImLaunch& L, const ImCall& call, const void* q, void* out, int n_max);
 bool im_attn_fast_supported(const ImDims& p);
-cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV, int box_rows);
+cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, void* mapV, int box_rows, int halves3d = 0);
 // tcgen05 version of the streaming attention kernel (head_dim 128): one run of 128-key tiles per CTA; mapK / mapV
 // with 32-row boxes (ragged last tile of a row), mapK128 / mapV128 with 128-row boxes (full tiles)
 bool im_attn_tc_supported(const ImDims& p);
