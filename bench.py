@@ -127,11 +127,12 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------
-def build_context(wl: synth.Workload, device, ingest=True, log=lambda *a: None, chunk_outputs=0, score_share=0):
+def build_context(wl: synth.Workload, device, ingest=True, log=lambda *a: None, chunk_outputs=0, score_share=0, pending_slots=0):
     from paper_2605_25475_b200 import binding as im
     g = im.IndexMem(im.Config(n_layers=wl.n_layers, max_seqs=wl.n_seq, n_q_heads=wl.H, n_kv_heads=wl.Hkv,
                               head_dim=wl.d, budget=wl.B, compress_interval=wl.tau, max_chunk=wl.chunk,
-                              n_sink=wl.n_sink, chunk_outputs=chunk_outputs, score_share=score_share), device)
+                              n_sink=wl.n_sink, chunk_outputs=chunk_outputs, score_share=score_share,
+                              pending_slots=pending_slots), device)
     ids = list(range(wl.n_seq))
     for layer in range(wl.n_layers):
         g.set_weights(layer, {k: v.cpu() for k, v in synth.make_weights(wl, layer, device).items()})

@@ -165,3 +165,42 @@ def test_stack_call_falls_back_and_refuses_bad_arguments():
         gb.decode_stack([0, 1, 7], ids, x, qp, q, k, v)
     _same_state(im, ga, gb, wl, "after the refused calls")
     ga.close(); gb.close()
+
+
+def test_stack_call_with_a_wait_that_runs_out_leaves_its_counters_clean():
+    """The give-up path of the attention kernel inside a stack call (IM_OPT_WAIT_LIMIT = 1: a consumer gets no attempt
+    to wait for its tile copies, nothing is broken or left to hang).  Every block, with or without a worker id, must
+    still hand the claim counters back: the status reads IM_ERR_TIMEOUT, and after the limit is restored and both
+    contexts are reset and fed the same context again, stack calls on the context that saw the time-out agree with
+    im_decode_step on its twin bit for bit."""
+    wl = _stack(n_layers=4, n_seq=3, ctx=512, chunk=256, B=256, steps=5)
+    im, (ga, gb), ids, dev = _twin(wl)
+    layers = list(range(wl.n_layers))
+    x, qp, q, k, v = _step_inputs(wl, 0, dev)
+    gb.decode_stack(layers, ids, x, qp, q, k, v)             # a good step first
+    torch.cuda.synchronize()
+    assert gb.status() == 0
+    im.im_set_option(gb.ctx, im.IM_OPT_WAIT_LIMIT, 1)
+    x, qp, q, k, v = _step_inputs(wl, 1, dev)
+    gb.decode_stack(layers, ids, x, qp, q, k, v)
+    torch.cuda.synchronize()
+    with pytest.raises(im.IndexMemError) as e:
+        gb.status()
+    assert e.value.code == im.IM_ERR_TIMEOUT, str(e.value)
+    im.im_set_option(gb.ctx, im.IM_OPT_WAIT_LIMIT, 0)
+    for g in (ga, gb):
+        g.reset()
+        assert g.status() == 0
+        for c in range(wl.ctx // wl.chunk):
+            for layer in layers:
+                X, Qp, _, K, V = synth.prefill_inputs(wl, layer, c, dev)
+                g.prefill_chunk(layer, ids, X, Qp, K, V)
+    for st in range(wl.steps):
+        x, qp, q, k, v = _step_inputs(wl, st, dev)
+        ref = torch.stack([ga.decode_step(l, ids, x[l], qp[l], q[l], k[l], v[l]) for l in layers])
+        got = gb.decode_stack(layers, ids, x, qp, q, k, v)
+        torch.cuda.synchronize()
+        assert torch.equal(ref, got), f"step {st}: outputs differ in {int((ref != got).sum())} elements"
+    assert ga.status() == 0 and gb.status() == 0
+    _same_state(im, ga, gb, wl, "after the time-out and the reset")
+    ga.close(); gb.close()
