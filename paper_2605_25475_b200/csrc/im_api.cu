@@ -1276,7 +1276,10 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     }
   }
   if (conc) CK(cudaEventRecord(ctx->ev[12], L2.stream));  // s2 finished: the merge needs phi(q)^T Mhat
-  if (ctx->prefetch_next && ctx->fast_attn) {
+  // (a context of one layer has no next layer to warm L2 for: what the next call reads is what this one has just read,
+  // and the two kernels, which end after the merge, would only hold the next call back: 7 us of a 31 us step)
+  const bool warm_next = ctx->prefetch_next && p.L > 1;
+  if (warm_next && ctx->fast_attn) {
     // warm L2 for the next layer's small kernels while this layer's attention streams K/V; after the front kernel,
     // which should find its SMs free of other kernels' blocks
     ImLaunch Lp = L3;
@@ -1285,7 +1288,7 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
     Lp.w = ctx->lo.w[nxt.layer];
     CKL(im_launch_prefetch_layer(Lp, nxt));
   }
-  if (conc && ctx->prefetch_next && p.mem && n_res > 0) {
+  if (conc && warm_next && p.mem && n_res > 0) {
     // Half of the next layer's memory matrices go into L2 while this call's merge runs: the streaming kernels have
     // ended, nothing else asks for HBM, and the next call's readout then finds these rows in L2 while its attention
     // kernel has the DRAM channels (measured: a step of the 32-layer benchmark takes 2.26 ms with half of each
