@@ -700,7 +700,8 @@ def run_reference(args, rank, world):
             "config": {"workload": wl.name + ("" if not (args.layers or args.context) else " (reduced for profiling)")
                                    + ("" if not args.tau else " (compression interval %d instead of the headline workload's)" % args.tau),
                        "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H, "kv_heads": wl.Hkv, "head_dim": wl.d,
-                       "context": wl.ctx, "budget": wl.B, "tau": wl.tau, "cuda_graph": False,
+                       "context": wl.ctx, "budget": wl.B, "tau": wl.tau, "cuda_graph": False, "score_share": args.score_share,
+                       "call": "the CPU oracle's decode step, one (layer, sequence) unit after the other on the host cores",
                        "l2": "inputs larger than L2 (each step streams %.1f GB)" % (ab["step"] / 1e9)},
             "cpu_baseline": base,
             "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
