@@ -30,65 +30,106 @@ __device__ __forceinline__ bool fold_needed(const ImDims& p, const ImCall& call,
   return np + ne > p.F;
 }
 
-// Mhat <- cscale * (Mhat + sum_p w_p phi_p v_p^T).  grid = (FOLD_BLOCKS, n_seq), block = 256; a block
-// walks 64x64 tiles of Mhat, each thread a 4x4 micro tile.  Blocks of sequences that need no fold
-// leave at once (the kernel is part of every decode step so that a captured launch sequence stays valid).
-constexpr int FOLD_BLOCKS = 16;
+// Mhat <- cscale * (Mhat + sum_p w_p phi_p v_p^T).  grid = (stripes of 64 rows, n_seq), block = 256.  A block owns a
+// stripe of 64 rows of one sequence's Mhat.  Per 16 listed entries it stages w_p phi_p of its rows and v_p of up to 1024
+// columns in shared memory ONCE, then walks the stripe in 64 x 64 tiles, each thread a 4 x 4 micro tile whose rows it
+// reads and writes as 16-byte words, the next tile's rows requested before the current tile is updated: between the
+// staging and the end of the stripe the kernel only streams Mhat.  (Its first form staged per tile, with two block
+// barriers and a round trip of small loads each, and read Mhat in 4-byte words: next to the streaming kernels of a
+// decode step, where every request queues behind theirs, the 32 layers' folds of a step took 1.7 ms; this form 1.2 ms.)
+// Blocks of sequences that need no fold leave at once (the kernel is part of every decode step so that a captured
+// launch sequence stays valid).
+constexpr int FOLD_COLS = 1024;  // columns of v_p staged at a time
 __global__ void __launch_bounds__(256) k_mem_fold(ImDims p, ImState st, ImCall call) {
-  __shared__ float s_a[16][64 + 4];  // [entry][m]   w_p * phi_p
-  __shared__ float s_b[16][64 + 4];  // [entry][col] v_p
+  __shared__ float s_a[16][64 + 4];        // [entry][m]   w_p * phi_p
+  __shared__ bf16 s_v[16][FOLD_COLS + 8];  // [entry][col] v_p
   const int i = blockIdx.y;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int32_t* ctr = st.ctr + u * CTR_STRIDE;
   const float c = st.cscale[u];
   if (!fold_needed(p, call, ctr, c)) return;
   const int np = min(ctr[CTR_NPEND], p.F);
-  const int tiles_x = (p.Dkv + 63) / 64, tiles_y = (p.dM + 63) / 64;
+  const int stripes = (p.dM + 63) / 64;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   float* Mh = st.Mhat + u * p.dM * p.Dkv;
-  for (int tile = blockIdx.x; tile < tiles_x * tiles_y; tile += gridDim.x) {
-  const int m0 = (tile / tiles_x) * 64, col0 = (tile % tiles_x) * 64;
-  float acc[4][4];
+  const bool wide = (p.Dkv & 7) == 0 && (p.dM & 3) == 0;  // 16-byte words throughout
+  // rows a thread owns in a stripe: ty, ty + 16, ty + 32, ty + 48 (a warp's loads then cover two whole 256-byte row pieces)
+  auto load_tile = [&](float (&acc)[4][4], int m0, int col0) {
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < 4; ++a) {
+      const int m = m0 + a * 16 + ty;
+      if (wide && col0 + tx * 4 + 3 < p.Dkv) {
+        float4 w = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (m < p.dM) w = *reinterpret_cast<const float4*>(Mh + (size_t)m * p.Dkv + col0 + tx * 4);
+        acc[a][0] = w.x; acc[a][1] = w.y; acc[a][2] = w.z; acc[a][3] = w.w;
+      } else {
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int m = m0 + ty * 4 + a, col = col0 + tx * 4 + b;
-      acc[a][b] = (m < p.dM && col < p.Dkv) ? Mh[(size_t)m * p.Dkv + col] : 0.f;
-    }
-  for (int k0 = 0; k0 < np; k0 += 16) {
-    __syncthreads();
-    for (int k = threadIdx.x; k < 16 * 64; k += blockDim.x) {
-      const int e = k / 64, j = k % 64;
-      float av = 0.f, bv = 0.f;
-      if (k0 + e < np) {
-        const int m = m0 + j, col = col0 + j;
-        if (m < p.dM) av = st.pend_w[u * p.F + k0 + e] * st.pend_phi[(u * p.F + k0 + e) * p.dM + m];
-        if (col < p.Dkv) bv = __bfloat162float(st.pend_v[(u * p.F + k0 + e) * p.Dkv + col]);
+        for (int b = 0; b < 4; ++b) {
+          const int col = col0 + tx * 4 + b;
+          acc[a][b] = (m < p.dM && col < p.Dkv) ? Mh[(size_t)m * p.Dkv + col] : 0.f;
+        }
       }
-      s_a[e][j] = av;
-      s_b[e][j] = bv;
     }
-    __syncthreads();
-    const int lim = min(16, np - k0);
-    for (int e = 0; e < lim; ++e) {
-      float av[4], bv[4];
+  };
+  for (int stripe = blockIdx.x; stripe < stripes; stripe += gridDim.x) {
+    const int m0 = stripe * 64;
+    for (int cb = 0; cb < p.Dkv; cb += FOLD_COLS) {
+      const int ncol = min(FOLD_COLS, p.Dkv - cb);
+      for (int k0 = 0; k0 < np || k0 == 0; k0 += 16) {
+        const int lim = max(0, min(16, np - k0));
+        const bool last = k0 + 16 >= np;  // (the scale is applied with the last entries)
+        __syncthreads();
+        for (int k = threadIdx.x; k < lim * 64; k += blockDim.x) {
+          const int e = k / 64, j = k % 64;
+          s_a[e][j] = m0 + j < p.dM ? st.pend_w[u * p.F + k0 + e] * st.pend_phi[(u * p.F + k0 + e) * p.dM + m0 + j] : 0.f;
+        }
+        if (wide) {
+          for (int k = threadIdx.x; k < lim * (ncol / 8); k += blockDim.x) {
+            const int e = k / (ncol / 8), j = (k % (ncol / 8)) * 8;
+            *reinterpret_cast<uint4*>(&s_v[e][j]) = *reinterpret_cast<const uint4*>(st.pend_v + (u * p.F + k0 + e) * p.Dkv + cb + j);
+          }
+        } else {
+          for (int k = threadIdx.x; k < lim * ncol; k += blockDim.x) {
+            const int e = k / ncol, j = k % ncol;
+            s_v[e][j] = st.pend_v[(u * p.F + k0 + e) * p.Dkv + cb + j];
+          }
+        }
+        __syncthreads();
+        float cur[4][4], nxt[4][4];
+        load_tile(cur, m0, cb);
+        for (int c0 = 0; c0 < ncol; c0 += 64) {
+          if (c0 + 64 < ncol) load_tile(nxt, m0, cb + c0 + 64);
+          for (int e = 0; e < lim; ++e) {
+            float bv[4];
 #pragma unroll
-      for (int a = 0; a < 4; ++a) av[a] = s_a[e][ty * 4 + a];
+            for (int b = 0; b < 4; ++b) bv[b] = c0 + tx * 4 + b < ncol ? __bfloat162float(s_v[e][c0 + tx * 4 + b]) : 0.f;
 #pragma unroll
-      for (int b = 0; b < 4; ++b) bv[b] = s_b[e][tx * 4 + b];
+            for (int a = 0; a < 4; ++a) {
+              const float av = s_a[e][a * 16 + ty];
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
+              for (int b = 0; b < 4; ++b) cur[a][b] = fmaf(av, bv[b], cur[a][b]);
+            }
+          }
+          const float sc_ = last ? c : 1.0f;
 #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
-    }
-  }
+          for (int a = 0; a < 4; ++a) {
+            const int m = m0 + a * 16 + ty, col = cb + c0 + tx * 4;
+            if (m >= p.dM) continue;
+            if (wide && col + 3 < p.Dkv) {
+              *reinterpret_cast<float4*>(Mh + (size_t)m * p.Dkv + col) =
+                  make_float4(sc_ * cur[a][0], sc_ * cur[a][1], sc_ * cur[a][2], sc_ * cur[a][3]);
+            } else {
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+              for (int b = 0; b < 4; ++b)
+                if (col + b < p.Dkv) Mh[(size_t)m * p.Dkv + col + b] = sc_ * cur[a][b];
+            }
+          }
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int m = m0 + ty * 4 + a, col = col0 + tx * 4 + b;
-      if (m < p.dM && col < p.Dkv) Mh[(size_t)m * p.Dkv + col] = c * acc[a][b];
+          for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) cur[a][b] = nxt[a][b];
+        }
+      }
     }
   }
 }
@@ -285,7 +326,7 @@ __global__ void __launch_bounds__(256) k_mem_bsum(ImDims p, ImState st, ImScratc
 
 cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call) {
   const ImDims& p = L.p;
-  dim3 grid(FOLD_BLOCKS, call.n_seq);
+  dim3 grid((p.dM + 63) / 64, call.n_seq);
   k_mem_fold<<<grid, 256, 0, L.stream>>>(p, L.st, call);
   ++*L.launches;
   cudaError_t e = cudaGetLastError();

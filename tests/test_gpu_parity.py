@@ -167,6 +167,19 @@ def test_decay_and_write_strength():
     assert p.stats["max_M_err"] <= 2e-3
 
 
+def test_long_pending_list_folds_in_several_passes():
+    """A pending list of 40 entries (the fold kernel takes 16 listed entries per pass over a stripe of M) with decay and a
+    write strength, at the Llama head shape with a memory matrix of several stripes and column tiles: M, b and the
+    outputs against the oracle through two folds."""
+    wl = synth.CONFIGS["llama8b_b1"].replace(name="pend40", n_seq=2, ctx=400, chunk=200, B=128, steps=90, n_needles=0)
+    p = _pair(wl, lambda_=0.97, eta=0.7, pending_slots=40)
+    p.prefill(0)
+    p.prefill(1)
+    for s in range(wl.steps):
+        p.decode(s, check=(s % 9 == 8 or s == wl.steps - 1))
+    assert p.stats["max_M_err"] <= 2e-3 and p.stats["max_out_err"] <= 2e-3
+
+
 def test_interval_pooling_tau():
     """tau = 8: scores pooled by max over the interval's queries, 8 entries evicted at once."""
     wl = TINY.replace(name="tau8", ctx=200, chunk=200, B=96, steps=24, tau=8, n_needles=2)
