@@ -140,6 +140,22 @@ def test_stack_call_against_the_oracle():
     assert su.stats["kidx_flips"] == 0 and su.stats["cut_divergences"] <= 2
 
 
+@pytest.mark.parametrize("shape", ["qwen7b_b8", "tiny"])
+def test_stack_call_other_head_shapes_against_the_oracle(shape):
+    """The stack call at the Qwen head shape (7 query heads per KV head, 4 KV heads, memory width 448: eight column
+    slices per readout item row) and at head_dim 64 with one KV head (the other instance of the attention kernel),
+    three layers, sampled units against the oracle under graph replay."""
+    base = synth.CONFIGS[shape]
+    wl = base.replace(name="stack_" + shape, n_layers=3, n_seq=4, ctx=600, chunk=300, B=256, steps=10,
+                      n_needles=min(base.n_needles, 4))
+    su = SampledUnits(wl, [(0, 3), (1, 0), (2, 2)])
+    for c in range(wl.ctx // wl.chunk):
+        su.prefill(c)
+    _decode_under_graph_replay(su, wl.steps, full_check_every=5, stack_call=True)
+    su.check_properties(wl.B, wl.ctx + wl.steps, n_evicted=1, stride=2)
+    assert su.stats["kidx_flips"] == 0 and su.stats["cut_divergences"] <= 2
+
+
 def test_stack_call_falls_back_and_refuses_bad_arguments():
     """Calls that do not qualify for the pipelined schedule (it is switched off; one layer only) run layer by layer
     with the same results; a repeated layer and a layer out of range are refused."""
