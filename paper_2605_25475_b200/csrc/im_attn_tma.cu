@@ -273,7 +273,14 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   // which the first tiles are being fetched from, is not that kernel's business, but the query rows may be its
   // output and the partials and entry counts of this call overwrite what the previous call's merge still reads.
   if (!DYN) asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (wid == 0)  // what the merge kernel rebuilds the tile bookkeeping from
+  // DYN: the kernel is launched as programmatic dependent so that its blocks follow those of the previous layer's
+  // attention kernel without a gap.  Among the launch's other prerequisites is the layer that used this lane's scratch
+  // set before (the stream waits for its event), and a prerequisite that releases its dependents early - that layer's
+  // merge kernel does - may still be running when this kernel starts.  So nothing is written to the scratch set before
+  // `griddepcontrol.wait` has returned; a warp calls it just ahead of its first store, a run's worth of streaming into
+  // the kernel, when it returns at once.
+  bool scratch_free = !DYN;
+  if (!DYN && wid == 0)  // what the merge kernel rebuilds the tile bookkeeping from
     for (int k = threadIdx.x; k < call.n_seq; k += blockDim.x) sc.n_att[k] = s_n[k];
 
   const float sl2 = p.scale * 1.4426950408889634f;  // softmax in base 2
@@ -401,6 +408,12 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     for (int off = 4; off < 32; off <<= 1) {
       l0 += __shfl_xor_sync(0xffffffffu, l0, off);
       l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+    }
+    if (!scratch_free) {  // (warp uniform)
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      scratch_free = true;
+      if (wid == 0 && warp == 0)
+        for (int k = lane; k < call.n_seq; k += 32) sc.n_att[k] = s_n[k];
     }
     {
       // Rows are served by consecutive runs and consecutive rows share at most one run, so
