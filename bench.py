@@ -558,18 +558,19 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device, stack_call=False):
     ev_out = [torch.cuda.Event() for _ in range(L)]
     ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
 
-    n_groups = 4 if (stack_call and L % 4 == 0 and L >= 8) else 0
+    # groups of consecutive layers, one stack call each: a short first group (its copy is the only one nothing hides)
+    bounds = ([0, 2, 8] + list(range(16, L + 1, 8))) if (stack_call and L % 8 == 0 and L >= 16) else []
+    n_groups = max(len(bounds) - 1, 0)
 
     def enqueue_groups(k):
-        """One step made of stack calls over groups of L / 4 consecutive layers: the inputs of group g + 1 are copied
-        in and the outputs of group g - 1 copied out while the stack call of group g runs."""
+        """One step made of stack calls over groups of consecutive layers: the inputs of group g + 1 are copied in and
+        the outputs of group g - 1 copied out while the stack call of group g runs."""
         hb = host[k]
-        per = L // n_groups
         ev_fork.record(stream)
         cs.wait_event(ev_fork)
         ds.wait_event(ev_fork)
         for gi in range(n_groups):
-            a, b = gi * per, (gi + 1) * per
+            a, b = bounds[gi], bounds[gi + 1]
             with torch.cuda.stream(cs):
                 dbuf[a:b].copy_(hb[a:b], non_blocking=True)
                 tick[gi:gi + 1].fill_(1.0)           # (see below: the calls depend on a kernel, not on the copy node)
@@ -649,8 +650,8 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device, stack_call=False):
     ms = max_over_ranks(ev0.elapsed_time(ev1), world, device)
     return {"value": wl.n_seq * args.steps * world / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms / args.steps, "cuda_graph": graphs is not None,
-            "calls_per_step": ("%d im_decode_stack calls over %d layers each" % (n_groups, L // n_groups)) if n_groups
-                              else "%d im_decode_step calls" % L}
+            "calls_per_step": ("%d im_decode_stack calls over %s layers" % (n_groups, ", ".join(str(bounds[i + 1] - bounds[i]) for i in range(n_groups))))
+                              if n_groups else "%d im_decode_step calls" % L}
 
 
 # ----------------------------------------------------------------------------------------------
