@@ -201,7 +201,8 @@ int im_decode_step(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, co
  * complete in stream order after the call, and the call can be captured into a CUDA graph like im_decode_step.
  * The streaming kernels are kept to a fixed subset of the SMs by SM id (a block that finds itself on an SM set
  * aside for the small kernels hands its work to a block that is still to come), since with layers overlapping the
- * occupancy rules that make this split in im_decode_step no longer hold.
+ * occupancy rules that make this split in im_decode_step no longer hold.  phi(q)^T Mhat is formed by the bulk-copy
+ * readout kernel where it serves the shape (see IM_OPT_READOUT_STAGES).
  * The pipelined schedule needs every layer of the call to qualify for im_decode_step's concurrent schedule with
  * SMs set aside (at most n_SM / 4 sequences, evicted sets of at most min(16, pending_slots) entries, budgets of at
  * most 6144 entries, the indexer as scorer, no score reuse, memory enabled); otherwise, and with
@@ -294,7 +295,9 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        Mhat in through a ring of k 32 KB bulk copies per CTA, one CTA beside each attention CTA
  *                        (k <= 6; D_kv a power of two of at most 1024 and d_M a multiple of 8192 / D_kv); 0 (default): by the
  *                        kernel built on plain loads, which serves every shape and schedule.  The two add the rows in different
- *                        orders (float32); both are within the stated tolerances.
+ *                        orders (float32); both are within the stated tolerances.  While the option has not been set, a
+ *                        pipelined im_decode_stack uses the bulk-copy kernel with two stages where it serves the shape
+ *                        and im_decode_step the plain-load kernel; once set, the value holds for both.
  *   IM_OPT_LAYER_OVERLAP 1 (default): in the concurrent schedule the attention kernel of a decode call on ANOTHER layer than
  *                        the call before it on the same stream is launched as programmatic dependent of that call's last
  *                        kernel: it requests its first cache tiles while that kernel still runs and waits for it before it
@@ -303,7 +306,7 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        im_decode_step layer by layer.
  *   IM_OPT_STACK_RESERVED k >= 1: SMs that a pipelined im_decode_stack keeps free of streaming blocks, for the small
  *                        kernels of the layers in flight; 0 (default): one per sequence of the call.
- *   IM_OPT_STACK_CHUNKS  k in [1, 16] (default 4): a pipelined im_decode_stack cuts the tiles of a layer's attention into k
+ *   IM_OPT_STACK_CHUNKS  k in [1, 16] (default 2): a pipelined im_decode_stack cuts the tiles of a layer's attention into k
  *                        runs per warp, which the warps take from a counter.  With k = 1 the runs, and with them the
  *                        order of every float32 sum, are those of im_decode_step: the two then agree bit for bit.
  *   IM_OPT_WAIT_LIMIT    (test aid) attempts of the bounded device-side waits in which a consumer waits for its copies to

@@ -227,7 +227,7 @@ void carve(const ImDims& p, char* base, Layout* lo) {
     ln.mres = (float*)take((size_t)p.S * IM_MRES_ROW(p) * 4);
     ln.phiq = (float*)take((size_t)p.S * p.dM * 4);
     ln.n_att = (int32_t*)take((size_t)p.S * 4);
-    ln.rpart = (float*)take((size_t)p.S * p.Dkv * 4);
+    ln.rpart = (float*)take((size_t)(IM_ATTN_MAX_CTAS + p.S) * p.Dkv * 4);
     ln.claim = base ? lo->claims + k * 8 : nullptr;
   }
   lo->total = align_up(off, 256);
@@ -258,6 +258,8 @@ struct im_ctx {
   std::vector<ExtScores> ext;        // per layer: scores handed in by the caller for the next compressing call (scorer = 2)
   bool ro_stream = false;            // phi(q)^T Mhat by the bulk-copy streaming kernel where it runs next to the attention kernel (IM_OPT_READOUT_STAGES)
   int ro_stages = 2;                 // ... with this many 32 KB stages per CTA
+  bool ro_explicit = false;          // IM_OPT_READOUT_STAGES has been set: it rules stack calls too (which otherwise take
+                                     // the bulk-copy kernel with two stages where it serves the shape)
   bool attn_tc_ready = false;        // the tensor-core streaming attention kernel takes this shape and is set up
   bool attn_tc = false;              // ... and im_decode_step uses it (IM_OPT_DECODE_TENSOR)
   bool fast_attn = false;
@@ -299,7 +301,7 @@ struct im_ctx {
   std::vector<int> sm_ids;           // ids of the device's SMs (ascending) as a probe kernel saw them; empty: unknown
   bool stack_pipeline = true;        // IM_OPT_STACK_PIPELINE
   int stack_reserved = 0;            // IM_OPT_STACK_RESERVED: SMs kept free of streaming blocks (0: one per sequence)
-  int stack_chunks = 4;              // IM_OPT_STACK_CHUNKS: runs per warp the attention kernel's tiles are cut into
+  int stack_chunks = 2;              // IM_OPT_STACK_CHUNKS: runs per warp the attention kernel's tiles are cut into
 #ifdef IM_TRACE
   int tune[8] = {0, -1, -1, 0, 0, 0, 0, 0};  // development builds: knobs set through options 100 + k
 #endif
@@ -1384,6 +1386,11 @@ bool decode_plan(im_ctx* ctx, int layer, const ImCall& call, bool* due, int* n_m
   return true;
 }
 
+// does a pipelined stack call form phi(q)^T Mhat with the bulk-copy kernel?
+bool stack_bulk_readout(const im_ctx* ctx) {
+  return (ctx->ro_explicit ? ctx->ro_stream : true) && ctx->p.mem && im_readout_stream_supported(ctx->p);
+}
+
 // One layer of a pipelined stack call (see im_decode_stack): the kernels of im_decode_step's concurrent schedule with
 // deferred compaction, enqueued on the lane's streams, the call's attention stream and its readout stream.
 int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids, int n_res, const unsigned long long* sm_stream,
@@ -1506,7 +1513,18 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
   // phi(q)^T Mhat on the call's readout stream
   CK(cudaStreamWaitEvent(LR.stream, ln.ev[6], 0));
   if (mem_write) CK(cudaStreamWaitEvent(LR.stream, ln.ev[7], 0));
-  CKL(im_launch_readout(LR, call, std::max(ctx->n_sm, call.ro_claim), 0));
+  // The bulk-copy kernel by default (fixed runs of 32 KB chunks, a partial vector per block, two stages per block): it
+  // needs a few registers where the plain-load kernel fills the SM's register file next to an attention block, so the
+  // small kernels of the layers in flight find room on the streaming SMs at all times, and the memory system serves
+  // its few large copies better than the other's many small loads (1.87 against 1.96 ms per step of the 32-layer
+  // benchmark, with 24 against 8 SMs set aside).
+  int ro_workers = 0;
+  if (stack_bulk_readout(ctx)) {
+    ro_workers = (int)std::min<long long>(n_wk_max, (long long)n_seq * im_readout_stream_chunks(p));
+    CKL(im_launch_readout_stream(LR, call, ro_workers, ctx->ro_explicit ? ctx->ro_stages : 2));
+  } else {
+    CKL(im_launch_readout(LR, call, std::max(ctx->n_sm, call.ro_claim), 0));
+  }
   CK(cudaEventRecord(ln.ev[12], LR.stream));
   // a3: phi of the evicted keys, then (off the path to the merge) the state update
   if (mem_write && (rc = run_memory_write(ctx, L1, call, ne_max, false, 0, nullptr, 0))) return rc;
@@ -1526,7 +1544,7 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
   CK(cudaStreamWaitEvent(ln.main, ln.ev[3], 0));
   CK(cudaStreamWaitEvent(ln.main, ln.ev[12], 0));
   CK(cudaStreamWaitEvent(ln.main, ln.ev[4], 0));
-  CKL(im_launch_attention_merge(L, call, out, call.att_chunks, IM_ATTN_STREAM_TILE, 0, q, k_new, v_new, 0));
+  CKL(im_launch_attention_merge(L, call, out, call.att_chunks, IM_ATTN_STREAM_TILE, ro_workers, q, k_new, v_new, 0));
   CK(cudaStreamWaitEvent(ln.main, ln.ev[5], 0));
   CK(cudaStreamWaitEvent(ln.main, ln.ev[2], 0));
   CK(cudaEventRecord(ln.done, ln.main));
@@ -1553,13 +1571,17 @@ extern "C" int im_decode_stack(im_ctx* ctx, int n_layers, const int32_t* layers,
   }
   // The pipelined schedule takes calls whose every layer runs im_decode_step's concurrent schedule with deferred
   // compaction and SMs set aside for the chain of small kernels; anything else goes layer by layer.
-  bool pipe = ctx->stack_pipeline && n_layers >= 2 && ctx->fast_attn && ctx->concurrent && !ctx->attn_tc && !ctx->ro_stream &&
+  bool pipe = ctx->stack_pipeline && n_layers >= 2 && ctx->fast_attn && ctx->concurrent && !ctx->attn_tc &&
               !p.scorer && !p.share && p.mem && !ctx->sm_ids.empty() && ctx->st_attn != nullptr;
   int n_res = 0;
   if (pipe) {
     // (far fewer than im_decode_step sets aside: the small kernels are off the path that bounds the call, and while
     // a layer's readout block is absent from a streaming SM they find registers there as well)
-    n_res = ctx->stack_reserved > 0 ? ctx->stack_reserved : std::min(im_reserved_sms(ctx->n_sm, n_seq), 8);
+    // (with the bulk-copy readout kernel, whose shared-memory ring leaves little room for the small kernels' blocks next
+    // to an attention block, a few more: 24 measured best on the 32-layer benchmark, 16: +2 %, 32: +4 %; with the
+    // plain-load kernel 8)
+    n_res = ctx->stack_reserved > 0 ? ctx->stack_reserved
+                                    : std::min(im_reserved_sms(ctx->n_sm, n_seq), stack_bulk_readout(ctx) ? 24 : 8);
     pipe = n_res > 0 && n_res < ctx->n_sm;
   }
   for (int j = 0; j < n_layers && pipe; ++j) {
@@ -1670,6 +1692,7 @@ int im_set_option(im_ctx* ctx, int option, int value) {
       if (value > 0 && !(ctx->fast_attn && ctx->p.mem && im_readout_stream_supported(ctx->p)))
         return fail(IM_ERR_ARG, "the bulk-copy readout kernel does not take this shape (D_kv a power of two of at most 1024, d_M a multiple of 8192 / D_kv)");
       ctx->ro_stream = value > 0;
+      ctx->ro_explicit = true;
       if (value > 0) ctx->ro_stages = value;
       return IM_OK;
     default: return fail(IM_ERR_ARG, "unknown option %d", option);

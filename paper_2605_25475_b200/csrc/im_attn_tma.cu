@@ -132,9 +132,11 @@ k_attn_stream(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   const int g = lane >> 2, t = lane & 3;
   unsigned char* ring = smem + (size_t)warp * STAGES * STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)WARPS * STAGES * STAGE_BYTES);
+  // (sized by the call's sequences, not by the most a call may have: next to this block and a readout block an SM has
+  // some 25 KB of shared memory left, which the small kernels of the layers in flight need every KB of)
   long long* s_pref = reinterpret_cast<long long*>(bars + WARPS * STAGES);  // [n_seq + 1]
-  int* s_n = reinterpret_cast<int*>(s_pref + IM_MAX_CALL_SEQS + 1);         // [n_seq]
-  int* s_misc = s_n + IM_MAX_CALL_SEQS;                                     // [1 + WARPS * 4] (DYN)
+  int* s_n = reinterpret_cast<int*>(s_pref + call.n_seq + 1);               // [n_seq]
+  int* s_misc = s_n + call.n_seq;                                           // [1 + WARPS * 4] (DYN)
   int* s_fifo = s_misc + 1 + warp * 4;  // runs this warp's producer side has taken, in order (-1: none left)
 
   // Pipelined stack call: the block claims a worker id (blocks on SMs that are set aside for the call's small
@@ -1188,13 +1190,13 @@ cudaError_t im_attn_make_maps(const ImDims& p, const ImState& st, void* mapK, vo
   return cudaSuccess;
 }
 
-size_t im_attn_smem_bytes(const ImDims& p) {
+size_t im_attn_smem_bytes(const ImDims& p, int n_seq) {
   const size_t stage = (size_t)2 * TILE * p.d * 2;
-  return (size_t)WARPS * STAGES * stage + (size_t)WARPS * STAGES * 8 + (IM_MAX_CALL_SEQS + 1) * 8 + IM_MAX_CALL_SEQS * 4 + (1 + WARPS * 4) * 4 + 64;
+  return (size_t)WARPS * STAGES * stage + (size_t)WARPS * STAGES * 8 + (size_t)(n_seq + 1) * 8 + (size_t)n_seq * 4 + (1 + WARPS * 4) * 4 + 64;
 }
 
 cudaError_t im_attn_prepare(const ImDims& p) {
-  const int smem = (int)im_attn_smem_bytes(p);
+  const int smem = (int)im_attn_smem_bytes(p, IM_MAX_CALL_SEQS);
   cudaError_t e = cudaFuncSetAttribute(k_attn_stream<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_attn_stream<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_attn_stream<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -1242,7 +1244,7 @@ cudaError_t im_launch_attention_fast(const ImLaunch& L, const ImCall& call, cons
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_ctas);
   cfg.blockDim = dim3(WARPS * 32);
-  cfg.dynamicSmemBytes = im_attn_smem_bytes(p);
+  cfg.dynamicSmemBytes = im_attn_smem_bytes(p, call.n_seq);
   cfg.stream = L.stream;
   // programmatic: the kernel may start while the kernel before it in the stream is still running (it waits for it,
   // griddepcontrol.wait, before it touches anything but this layer's cache)

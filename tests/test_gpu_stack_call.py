@@ -30,11 +30,16 @@ def _twin(wl, **over):
     dev = torch.device("cuda:0")
     cfg = dict(n_layers=wl.n_layers, max_seqs=wl.n_seq, n_q_heads=wl.H, n_kv_heads=wl.Hkv, head_dim=wl.d, budget=wl.B,
                compress_interval=wl.tau, max_chunk=wl.chunk, n_sink=wl.n_sink)
+    bulk = over.pop("bulk_readout", False)
     cfg.update(over)
     gs = [im.IndexMem(im.Config(**cfg), dev) for _ in range(2)]
     # (one run per warp: the attention kernel then cuts its tiles exactly as im_decode_step's does, and every sum is
     # formed in the same order)
     im.im_set_option(gs[1].ctx, im.IM_OPT_STACK_CHUNKS, 1)
+    # (and phi(q)^T Mhat by the plain-load kernel in both: the bulk-copy kernel a stack call would take cuts the rows
+    # into per-block partial vectors, as many as there are blocks)
+    for g in gs:
+        im.im_set_option(g.ctx, im.IM_OPT_READOUT_STAGES, 2 if bulk else 0)
     ids = list(range(wl.n_seq))
     for layer in range(wl.n_layers):
         w = synth.make_weights(wl, layer)
@@ -90,6 +95,23 @@ def test_stack_call_equals_layer_calls_bit_for_bit(tau):
         assert torch.equal(ref, got), f"step {st}: outputs differ in {int((ref != got).sum())} elements"
         if st % 4 == 3 or st == wl.steps - 1:
             _same_state(im, ga, gb, wl, f"step {st}")
+    ga.close(); gb.close()
+
+
+def test_stack_call_with_the_bulk_copy_readout_equals_layer_calls():
+    """One sequence per call: the bulk-copy readout kernel then cuts a sequence's rows into the same runs in a stack
+    call and in a layer call (fewer chunks than blocks in both), so the two agree bit for bit with that kernel too."""
+    wl = _stack(n_layers=5, n_seq=1, steps=8)
+    im, (ga, gb), ids, dev = _twin(wl, bulk_readout=True)
+    layers = list(range(wl.n_layers))
+    for st in range(wl.steps):
+        x, qp, q, k, v = _step_inputs(wl, st, dev)
+        ref = torch.stack([ga.decode_step(l, ids, x[l], qp[l], q[l], k[l], v[l]) for l in layers])
+        got = gb.decode_stack(layers, ids, x, qp, q, k, v)
+        torch.cuda.synchronize()
+        assert torch.equal(ref, got), f"step {st}: outputs differ in {int((ref != got).sum())} elements"
+    assert ga.status() == 0 and gb.status() == 0
+    _same_state(im, ga, gb, wl, "with the bulk-copy readout")
     ga.close(); gb.close()
 
 
