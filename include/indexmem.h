@@ -305,7 +305,8 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *   IM_OPT_STACK_PIPELINE 1 (default): im_decode_stack overlaps the layers of a call where they qualify; 0: it calls
  *                        im_decode_step layer by layer.
  *   IM_OPT_STACK_RESERVED k >= 1: SMs that a pipelined im_decode_stack keeps free of streaming blocks, for the small
- *                        kernels of the layers in flight; 0 (default): one per sequence of the call.
+ *                        kernels of the layers in flight; 0 (default): one per sequence of the call, at most 24 with
+ *                        the bulk-copy readout kernel and 8 with the plain-load one.
  *   IM_OPT_STACK_CHUNKS  k in [1, 16] (default 2): a pipelined im_decode_stack cuts the tiles of a layer's attention into k
  *                        runs per warp, which the warps take from a counter.  With k = 1 the runs, and with them the
  *                        order of every float32 sum, are those of im_decode_step: the two then agree bit for bit.

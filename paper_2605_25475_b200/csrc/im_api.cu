@@ -300,7 +300,7 @@ struct im_ctx {
   cudaEvent_t st_fork = nullptr, st_attn_done = nullptr, st_ro_done = nullptr;
   std::vector<int> sm_ids;           // ids of the device's SMs (ascending) as a probe kernel saw them; empty: unknown
   bool stack_pipeline = true;        // IM_OPT_STACK_PIPELINE
-  int stack_reserved = 0;            // IM_OPT_STACK_RESERVED: SMs kept free of streaming blocks (0: one per sequence)
+  int stack_reserved = 0;            // IM_OPT_STACK_RESERVED: SMs kept free of streaming blocks (0: one per sequence, at most 24 / 8)
   int stack_chunks = 2;              // IM_OPT_STACK_CHUNKS: runs per warp the attention kernel's tiles are cut into
 #ifdef IM_TRACE
   int tune[8] = {0, -1, -1, 0, 0, 0, 0, 0};  // development builds: knobs set through options 100 + k
