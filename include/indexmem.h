@@ -63,7 +63,7 @@ typedef struct im_config {
   int32_t act;               /* indexer activation: 0 ReLU, 1 identity         (Sec. 3.1, z = act(q.k)) */
   int32_t enable_memory;     /* 0: no memory write and no readout term         (Eq. 4 with g = 0)   */
   int32_t out_f32;           /* 0: `out` of im_decode_step is bf16; 1: float32                       */
-  int32_t pending_slots;     /* rank-one writes folded lazily into M (0 => 16); see im_decode_step  */
+  int32_t pending_slots;     /* rank-one writes folded lazily into M (0 => 32); see im_decode_step  */
   int32_t chunk_outputs;     /* 1: reserve workspace for im_prefill_chunk_attend (max_seqs * max_chunk * D_kv floats) */
   int32_t score_share;       /* g >= 2: layers l with l % g != 0 reuse the indexer scores of layer l - l % g (App. B,
                                 IndexCache-style reuse; the paper uses 4); 0 or 1: every layer scores for itself      */
@@ -310,6 +310,10 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *   IM_OPT_STACK_CHUNKS  k in [1, 16] (default 2): a pipelined im_decode_stack cuts the tiles of a layer's attention into k
  *                        runs per warp, which the warps take from a counter.  With k = 1 the runs, and with them the
  *                        order of every float32 sum, are those of im_decode_step: the two then agree bit for bit.
+ *   IM_OPT_FOLD_TENSOR   1 (default): where d_M and D_kv are multiples of 64, the listed rank-one terms are folded into M on
+ *                        the tensor cores (w_p phi_p as three bf16 terms, v_p as stored: exact products, float32 sums); 0:
+ *                        by float32 multiply-adds in list order, as for every other shape.  The two differ by rounding
+ *                        order only.
  *   IM_OPT_WAIT_LIMIT    (test aid) attempts of the bounded device-side waits in which a consumer waits for its copies to
  *                        arrive (TMA / bulk-copy rings of the decode attention kernels, the bulk-copy readout kernel and
  *                        the tcgen05 chunk attention kernel): 0 restores the default (2^22), k >= 1 allows k - 1 attempts,
@@ -329,7 +333,8 @@ typedef enum im_option {
   IM_OPT_LAYER_OVERLAP = 7,
   IM_OPT_STACK_PIPELINE = 8,
   IM_OPT_STACK_RESERVED = 9,
-  IM_OPT_STACK_CHUNKS = 10
+  IM_OPT_STACK_CHUNKS = 10,
+  IM_OPT_FOLD_TENSOR = 11
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 

@@ -65,7 +65,7 @@ bool resolve(const im_config* in, im_config* c, ImDims* p) {
   if (c->max_chunk < 0) return false;
   if (c->n_sink < 0 || c->budget <= c->n_sink || c->budget < 1) return false;
   if (c->act != 0 && c->act != 1) return false;
-  if (c->pending_slots == 0) c->pending_slots = 16;
+  if (c->pending_slots == 0) c->pending_slots = 32;
   if (c->pending_slots < 1 || c->pending_slots > 64) return false;
   if (c->softmax_scale == 0.f) c->softmax_scale = 1.0f / sqrtf((float)c->head_dim);
   if (c->lambda == 0.f) c->lambda = 1.f;
@@ -301,6 +301,7 @@ struct im_ctx {
   std::vector<int> sm_ids;           // ids of the device's SMs (ascending) as a probe kernel saw them; empty: unknown
   bool stack_pipeline = true;        // IM_OPT_STACK_PIPELINE
   int stack_reserved = 0;            // IM_OPT_STACK_RESERVED: SMs kept free of streaming blocks (0: one per sequence, at most 24 / 8)
+  bool fold_tensor = true;           // IM_OPT_FOLD_TENSOR
   int stack_chunks = 2;              // IM_OPT_STACK_CHUNKS: runs per warp the attention kernel's tiles are cut into
 #ifdef IM_TRACE
   int tune[8] = {0, -1, -1, 0, 0, 0, 0, 0};  // development builds: knobs set through options 100 + k
@@ -372,6 +373,7 @@ int check_call(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_ids, ImCall
   call->early_cache = 0;
   call->stack = 0;
   call->att_workers = call->ro_claim = call->att_chunks = 0;
+  call->fold_ffma = ctx->fold_tensor ? 0 : 1;
   for (int k = 0; k < 4; ++k) call->sm_stream[k] = 0;
   return IM_OK;
 }
@@ -1672,6 +1674,7 @@ int im_set_option(im_ctx* ctx, int option, int value) {
       return IM_OK;
     case IM_OPT_LAYER_OVERLAP: ctx->layer_overlap = value != 0; return IM_OK;
     case IM_OPT_STACK_PIPELINE: ctx->stack_pipeline = value != 0; return IM_OK;
+    case IM_OPT_FOLD_TENSOR: ctx->fold_tensor = value != 0; return IM_OK;
     case IM_OPT_STACK_CHUNKS:
       if (value < 1 || value > 16) return fail(IM_ERR_ARG, "runs per warp %d out of range [1,16]", value);
       ctx->stack_chunks = value;

@@ -194,6 +194,7 @@ struct ImCall {
   int stack;                        // 1 = the streaming kernels claim their worker ids
   int att_workers, ro_claim;        // blocks of the attention / readout kernel of the call that are to work
   int att_chunks;                   // runs the attention kernel's tiles are cut into (taken from a counter)
+  int fold_ffma;                    // 1 = the fold of the pending list by the FFMA kernel whatever the shape (IM_OPT_FOLD_TENSOR 0)
   unsigned long long sm_stream[4];  // bit s set: SM s runs streaming blocks
   int seq[IM_MAX_CALL_SEQS];
 };

@@ -31,18 +31,19 @@ __device__ __forceinline__ bool fold_needed(const ImDims& p, const ImCall& call,
 }
 
 // Mhat <- cscale * (Mhat + sum_p w_p phi_p v_p^T).  grid = (stripes of 64 rows, n_seq), block = 256.  A block owns a
-// stripe of 64 rows of one sequence's Mhat.  Per 16 listed entries it stages w_p phi_p of its rows and v_p of up to 1024
-// columns in shared memory ONCE, then walks the stripe in 64 x 64 tiles, each thread a 4 x 4 micro tile whose rows it
+// stripe of 64 rows of one sequence's Mhat.  Per FOLD_ENT listed entries it stages w_p phi_p of its rows and v_p of up to
+// FOLD_COLS columns in shared memory ONCE, then walks the stripe in 64 x 64 tiles, each thread a 4 x 4 micro tile whose rows it
 // reads and writes as 16-byte words, the next tile's rows requested before the current tile is updated: between the
 // staging and the end of the stripe the kernel only streams Mhat.  (Its first form staged per tile, with two block
 // barriers and a round trip of small loads each, and read Mhat in 4-byte words: next to the streaming kernels of a
 // decode step, where every request queues behind theirs, the 32 layers' folds of a step took 1.7 ms; this form 1.2 ms.)
 // Blocks of sequences that need no fold leave at once (the kernel is part of every decode step so that a captured
 // launch sequence stays valid).
-constexpr int FOLD_COLS = 1024;  // columns of v_p staged at a time
+constexpr int FOLD_COLS = 512;  // columns of v_p staged at a time
+constexpr int FOLD_ENT = 32;    // listed entries folded per pass over a stripe (a list of up to FOLD_ENT entries: one pass)
 __global__ void __launch_bounds__(256) k_mem_fold(ImDims p, ImState st, ImCall call) {
-  __shared__ float s_a[16][64 + 4];        // [entry][m]   w_p * phi_p
-  __shared__ bf16 s_v[16][FOLD_COLS + 8];  // [entry][col] v_p
+  __shared__ float s_a[FOLD_ENT][64 + 4];        // [entry][m]   w_p * phi_p
+  __shared__ bf16 s_v[FOLD_ENT][FOLD_COLS + 8];  // [entry][col] v_p
   const int i = blockIdx.y;
   const size_t u = (size_t)call.layer * p.S + call.seq[i];
   const int32_t* ctr = st.ctr + u * CTR_STRIDE;
@@ -75,9 +76,9 @@ __global__ void __launch_bounds__(256) k_mem_fold(ImDims p, ImState st, ImCall c
     const int m0 = stripe * 64;
     for (int cb = 0; cb < p.Dkv; cb += FOLD_COLS) {
       const int ncol = min(FOLD_COLS, p.Dkv - cb);
-      for (int k0 = 0; k0 < np || k0 == 0; k0 += 16) {
-        const int lim = max(0, min(16, np - k0));
-        const bool last = k0 + 16 >= np;  // (the scale is applied with the last entries)
+      for (int k0 = 0; k0 < np || k0 == 0; k0 += FOLD_ENT) {
+        const int lim = max(0, min(FOLD_ENT, np - k0));
+        const bool last = k0 + FOLD_ENT >= np;  // (the scale is applied with the last entries)
         __syncthreads();
         for (int k = threadIdx.x; k < lim * 64; k += blockDim.x) {
           const int e = k / 64, j = k % 64;
@@ -128,6 +129,134 @@ __global__ void __launch_bounds__(256) k_mem_fold(ImDims p, ImState st, ImCall c
           for (int a = 0; a < 4; ++a)
 #pragma unroll
             for (int b = 0; b < 4; ++b) cur[a][b] = nxt[a][b];
+        }
+      }
+    }
+  }
+}
+
+// The same fold with the rank-one terms added by the tensor cores, for shapes whose d_M and D_kv are multiples of 64.
+// Per element the fold is one multiply-add per listed entry: 17 GFLOP for the 32 layers x 32 sequences of the decode
+// benchmark at 16 entries, which the FFMA form above spends on the few SMs the streaming kernels leave it (a quarter
+// of a fold step's extra time, and all of what a longer list adds).  Here a warp owns 16 rows x FOLDT_W columns of the
+// block's 64 x 2 FOLDT_W tile as FOLDT_NJ m16n8 accumulators that it loads from and stores to Mhat directly in the accumulator
+// layout (8-byte words: a warp's access covers whole 32-byte sectors), A = w_p phi_p of its rows as THREE bf16 terms
+// (hi + mid + lo reproduce the float32 value to 2^-24), B = v_p, which is bf16 as stored, through ldmatrix.trans from
+// the staged [entry][column] rows: the products are exact and the sums are float32, so the result differs from the
+// FFMA form by rounding order only.  Entries are staged FOLDT_ENT at a time (a list of up to 32: one pass over Mhat).
+constexpr int FOLDT_COLS = 512;
+constexpr int FOLDT_ENT = 32;
+#ifndef FOLDT_NJ
+#define FOLDT_NJ 4        /* m16n8 accumulators per warp and step */
+#define FOLDT_BLOCKS 3    /* blocks per SM the register budget allows */
+#endif
+constexpr int FOLDT_W = FOLDT_NJ * 8;  // columns of a warp's step
+__device__ __forceinline__ void fold_ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void fold_mma(float2& c01, float2& c23, const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c01.x), "+f"(c01.y), "+f"(c23.x), "+f"(c23.y)
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// x0, x1 -> three packed bf16 pairs (x0 in the low half) whose sum is x to 2^-24
+__device__ __forceinline__ void fold_split3(float x0, float x1, uint32_t& hi, uint32_t& mid, uint32_t& lo) {
+  const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+  const float r0 = x0 - __bfloat162float(h0), r1 = x1 - __bfloat162float(h1);
+  const __nv_bfloat16 m0 = __float2bfloat16_rn(r0), m1 = __float2bfloat16_rn(r1);
+  const float q0 = r0 - __bfloat162float(m0), q1 = r1 - __bfloat162float(m1);
+  const __nv_bfloat16 l0 = __float2bfloat16_rn(q0), l1 = __float2bfloat16_rn(q1);
+  hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+  mid = (uint32_t)__bfloat16_as_ushort(m0) | ((uint32_t)__bfloat16_as_ushort(m1) << 16);
+  lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+}
+__global__ void __launch_bounds__(256, FOLDT_BLOCKS) k_mem_fold_tc(ImDims p, ImState st, ImCall call) {
+  __shared__ __align__(16) float s_a[FOLDT_ENT][64 + 4];        // [entry][m]   w_p * phi_p
+  __shared__ __align__(16) bf16 s_v[FOLDT_ENT][FOLDT_COLS + 8];  // [entry][col] v_p
+  const int i = blockIdx.y;
+  const size_t u = (size_t)call.layer * p.S + call.seq[i];
+  const int32_t* ctr = st.ctr + u * CTR_STRIDE;
+  const float c = st.cscale[u];
+  if (!fold_needed(p, call, ctr, c)) return;
+  const int np = min(ctr[CTR_NPEND], p.F);
+  const int stripes = p.dM / 64;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int wr = warp & 3, wc = warp >> 2;  // the warp's 16-row slab of the stripe; which FOLDT_W columns of a 2 FOLDT_W-column step
+  float* Mh = st.Mhat + u * p.dM * p.Dkv;
+  for (int stripe = blockIdx.x; stripe < stripes; stripe += gridDim.x) {
+    const int m0 = stripe * 64;
+    float* rowp = Mh + (size_t)(m0 + wr * 16 + g) * p.Dkv + 2 * t;  // the thread's upper row; the lower one is 8 rows on
+    for (int cb = 0; cb < p.Dkv; cb += FOLDT_COLS) {
+      const int ncol = min(FOLDT_COLS, p.Dkv - cb);
+      const int ngroups = ncol / FOLDT_W;
+      for (int k0 = 0; k0 < np || k0 == 0; k0 += FOLDT_ENT) {
+        const int lim = max(0, min(FOLDT_ENT, np - k0));
+        const int limr = (lim + 15) & ~15;            // entries staged: whole k-steps, zeros past the list's end
+        const bool last = k0 + FOLDT_ENT >= np;       // (the scale is applied with the last entries)
+        __syncthreads();
+        for (int k = threadIdx.x; k < limr * 64; k += blockDim.x) {
+          const int e = k / 64, j = k % 64;
+          s_a[e][j] = e < lim ? st.pend_w[u * p.F + k0 + e] * st.pend_phi[(u * p.F + k0 + e) * p.dM + m0 + j] : 0.f;
+        }
+        for (int k = threadIdx.x; k < limr * (ncol / 8); k += blockDim.x) {
+          const int e = k / (ncol / 8), j = (k % (ncol / 8)) * 8;
+          *reinterpret_cast<uint4*>(&s_v[e][j]) =
+              e < lim ? *reinterpret_cast<const uint4*>(st.pend_v + (u * p.F + k0 + e) * p.Dkv + cb + j) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        __syncthreads();
+        // A of the warp's rows: [k-step][term][register]
+        uint32_t af[FOLDT_ENT / 16][3][4];
+#pragma unroll
+        for (int ks = 0; ks < FOLDT_ENT / 16; ++ks)
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            af[ks][0][r] = af[ks][1][r] = af[ks][2][r] = 0u;
+            if (ks * 16 < limr) {
+              const int row = wr * 16 + g + (r & 1) * 8, kk = ks * 16 + 2 * t + (r >> 1) * 8;
+              fold_split3(s_a[kk][row], s_a[kk + 1][row], af[ks][0][r], af[ks][1][r], af[ks][2][r]);
+            }
+          }
+        // ldmatrix row address of this lane: entry (lane & 7) + 8 * ((lane >> 3) & 1) of a k-step, 8 columns on for lanes 16-31
+        const uint32_t sv_lane = (uint32_t)__cvta_generic_to_shared(&s_v[(lane & 7) + ((lane >> 3) & 1) * 8][(lane >> 4) * 8]);
+        float2 cur[2 * FOLDT_NJ], nxt[2 * FOLDT_NJ];
+        auto load_group = [&](float2 (&a)[2 * FOLDT_NJ], int grp) {
+          const float* q = rowp + cb + grp * FOLDT_W;
+#pragma unroll
+          for (int j = 0; j < FOLDT_NJ; ++j) {
+            a[2 * j] = *reinterpret_cast<const float2*>(q + j * 8);
+            a[2 * j + 1] = *reinterpret_cast<const float2*>(q + (size_t)8 * p.Dkv + j * 8);
+          }
+        };
+        int grp = wc;
+        if (grp < ngroups) load_group(cur, grp);
+        for (; grp < ngroups; grp += 2) {
+          if (grp + 2 < ngroups) load_group(nxt, grp + 2);
+#pragma unroll
+          for (int ks = 0; ks < FOLDT_ENT / 16; ++ks) {
+            if (ks * 16 < limr) {
+#pragma unroll
+              for (int jp = 0; jp < FOLDT_NJ / 2; ++jp) {
+                uint32_t b0, b1, b2, b3;
+                fold_ldsm_x4_t(sv_lane + (uint32_t)((ks * 16 * (FOLDT_COLS + 8) + grp * FOLDT_W + jp * 16) * 2), b0, b1, b2, b3);
+#pragma unroll
+                for (int term = 2; term >= 0; --term) {
+                  fold_mma(cur[4 * jp], cur[4 * jp + 1], af[ks][term], b0, b1);
+                  fold_mma(cur[4 * jp + 2], cur[4 * jp + 3], af[ks][term], b2, b3);
+                }
+              }
+            }
+          }
+          const float sc_ = last ? c : 1.0f;
+          float* q = rowp + cb + grp * FOLDT_W;
+#pragma unroll
+          for (int j = 0; j < FOLDT_NJ; ++j) {
+            *reinterpret_cast<float2*>(q + j * 8) = make_float2(sc_ * cur[2 * j].x, sc_ * cur[2 * j].y);
+            *reinterpret_cast<float2*>(q + (size_t)8 * p.Dkv + j * 8) = make_float2(sc_ * cur[2 * j + 1].x, sc_ * cur[2 * j + 1].y);
+          }
+#pragma unroll
+          for (int j = 0; j < 2 * FOLDT_NJ; ++j) cur[j] = nxt[j];
         }
       }
     }
@@ -327,7 +456,8 @@ __global__ void __launch_bounds__(256) k_mem_bsum(ImDims p, ImState st, ImScratc
 cudaError_t im_launch_mem_fold(const ImLaunch& L, const ImCall& call) {
   const ImDims& p = L.p;
   dim3 grid((p.dM + 63) / 64, call.n_seq);
-  k_mem_fold<<<grid, 256, 0, L.stream>>>(p, L.st, call);
+  if (!call.fold_ffma && p.dM % 64 == 0 && p.Dkv % 64 == 0) k_mem_fold_tc<<<grid, 256, 0, L.stream>>>(p, L.st, call);
+  else k_mem_fold<<<grid, 256, 0, L.stream>>>(p, L.st, call);
   ++*L.launches;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -412,6 +542,7 @@ cudaError_t im_launch_mem_update(const ImLaunch& L, const ImCall& call, int ne_m
 
 cudaError_t im_memory_prepare_decode() {
   cudaError_t e = im_prefer_max_smem(k_mem_fold);
+  if (e == cudaSuccess) e = im_prefer_max_smem(k_mem_fold_tc);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_mem_fold_commit);
   if (e == cudaSuccess) e = im_prefer_max_smem(k_mem_small);
   return e;

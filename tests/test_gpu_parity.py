@@ -168,7 +168,7 @@ def test_decay_and_write_strength():
 
 
 def test_long_pending_list_folds_in_several_passes():
-    """A pending list of 40 entries (the fold kernel takes 16 listed entries per pass over a stripe of M) with decay and a
+    """A pending list of 40 entries (the fold kernels take 32 listed entries per pass over a stripe of M) with decay and a
     write strength, at the Llama head shape with a memory matrix of several stripes and column tiles: M, b and the
     outputs against the oracle through two folds."""
     wl = synth.CONFIGS["llama8b_b1"].replace(name="pend40", n_seq=2, ctx=400, chunk=200, B=128, steps=90, n_needles=0)
@@ -178,6 +178,36 @@ def test_long_pending_list_folds_in_several_passes():
     for s in range(wl.steps):
         p.decode(s, check=(s % 9 == 8 or s == wl.steps - 1))
     assert p.stats["max_M_err"] <= 2e-3 and p.stats["max_out_err"] <= 2e-3
+
+
+def test_fold_on_the_tensor_cores_differs_from_the_ffma_fold_by_rounding_only(im):
+    """The pending list of the default length (32 entries, one pass over M) folded by the tensor-core kernel and, on a
+    second context fed the same inputs, by the float32 multiply-add kernel (IM_OPT_FOLD_TENSOR 0), with decay and a write
+    strength, at the Llama and the Qwen head shape (d_M = 512 and 448, D_kv = 1024 and 512): M of both after every fold
+    agrees to a few float32 roundings relative to its largest entry, both follow the oracle, and the caches are
+    identical (no selection depends on M)."""
+    for shape in ("llama8b_b1", "qwen7b_b8"):
+        wl = synth.CONFIGS[shape].replace(name="foldtc_" + shape, n_seq=2, ctx=400, chunk=200, B=128, steps=70, n_needles=0)
+        pt = _pair(wl, lambda_=0.97, eta=0.7)
+        pf = _pair(wl, lambda_=0.97, eta=0.7)
+        im.im_set_option(pf.g.ctx, im.IM_OPT_FOLD_TENSOR, 0)
+        for p in (pt, pf):
+            p.prefill(0)
+            p.prefill(1)
+        worst = 0.0
+        for s in range(wl.steps):
+            chk = s % 8 == 7 or s == wl.steps - 1
+            pt.decode(s, check=chk)
+            pf.decode(s, check=chk)
+            if chk:
+                for q in range(wl.n_seq):
+                    Mt = pt.g.export(0, q, im.IM_S_M).astype(np.float64)
+                    Mf = pf.g.export(0, q, im.IM_S_M).astype(np.float64)
+                    worst = max(worst, float(np.abs(Mt - Mf).max() / np.abs(Mf).max()))
+                    assert np.array_equal(pt.g.export(0, q, im.IM_S_K), pf.g.export(0, q, im.IM_S_K))
+        assert pt.g.counts(0, 0)["n_pending"] < 32 and wl.steps > 64, "the list has been folded at least twice"
+        assert worst <= 2e-6, (shape, worst)
+        assert pt.stats["max_M_err"] <= 2e-3 and pf.stats["max_M_err"] <= 2e-3
 
 
 def test_interval_pooling_tau():
