@@ -167,11 +167,11 @@ def pick_workload(args):
 
 
 def measure_decode(wl, device, steps, warmup, graph=True, rank=0, world=1, log=lambda *a: None, opts=None,
-                   profile=True, e2e_args=None, score_share=0, steps_per_graph=1, stack_call=False):
+                   profile=True, e2e_args=None, score_share=0, steps_per_graph=1, stack_call=False, pending_slots=0):
     """Ingests the workload's context, then times `steps` decode steps (all layers, all sequences per step) replayed
     from CUDA graphs, inputs resident.  Returns the raw measurements; the context is closed before returning."""
     from paper_2605_25475_b200 import binding as im
-    g, ids = build_context(wl, device, log=log, score_share=score_share)
+    g, ids = build_context(wl, device, log=log, score_share=score_share, pending_slots=pending_slots)
     for opt, val in (opts or {}).items():
         im.im_set_option(g.ctx, opt, val)
     L = wl.n_layers
@@ -306,7 +306,8 @@ def run_ours(args, rank, world, device):
     if args.stack_reserved >= 0:
         opts[im.IM_OPT_STACK_RESERVED] = args.stack_reserved
     m = measure_decode(wl, device, args.steps, args.warmup, graph=bool(args.graph), rank=rank, world=world, log=log,
-                       opts=opts, e2e_args=args, score_share=args.score_share, stack_call=bool(args.stack_call))
+                       opts=opts, e2e_args=args, score_share=args.score_share, stack_call=bool(args.stack_call),
+                       pending_slots=args.pending_slots)
     ms = m["ms"]
     tokens = wl.n_seq * args.steps * world
     ab = algorithmic_bytes(wl)
@@ -335,6 +336,7 @@ def run_ours(args, rank, world, device):
                    "layers": wl.n_layers, "batch_per_gpu": wl.n_seq, "q_heads": wl.H,
                    "kv_heads": wl.Hkv, "head_dim": wl.d, "context": wl.ctx, "budget": wl.B, "tau": wl.tau,
                    "cuda_graph": m["cuda_graph"], "score_share": args.score_share,
+                   "pending_slots": args.pending_slots or 32,
                    "call": ("one im_decode_stack call per step: the inputs of all layers are resident when the step starts "
                             "(a stack driven from synthetic activations), so the call overlaps the layers"
                             if stack else "one im_decode_step call per layer"),
@@ -560,6 +562,9 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device, stack_call=False):
 
     # groups of consecutive layers, one stack call each: a short first group (its copy is the only one nothing hides)
     bounds = ([0, 2, 8] + list(range(16, L + 1, 8))) if (stack_call and L % 8 == 0 and L >= 16) else []
+    if stack_call and getattr(args, "e2e_groups", ""):
+        bounds = [int(b) for b in args.e2e_groups.split(",")]
+        assert bounds[0] == 0 and bounds[-1] == L and all(b > a for a, b in zip(bounds, bounds[1:]))
     n_groups = max(len(bounds) - 1, 0)
 
     def enqueue_groups(k):
@@ -758,6 +763,10 @@ def main():
                     help="0: readout on plain loads; k >= 1: on a ring of k 32 KB bulk copies per CTA (default: the library's choice)")
     ap.add_argument("--stack-call", type=int, default=1,
                     help="1: a step is one im_decode_stack call over all layers (the layers overlap); 0: one im_decode_step call per layer")
+    ap.add_argument("--pending-slots", type=int, default=0,
+                    help="length F of the list of rank-one writes folded lazily into M (0: the library's default, 32)")
+    ap.add_argument("--e2e-groups", default="",
+                    help="end-to-end step: layer boundaries of its im_decode_stack calls, e.g. 0,2,8,16,24,32 (the default for 32 layers)")
     ap.add_argument("--stack-reserved", type=int, default=-1,
                     help="SMs a pipelined stack call keeps free of streaming blocks (default: the library's choice)")
     ap.add_argument("--traffic", type=float, default=ATTN_TRAFFIC_NCU,
