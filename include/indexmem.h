@@ -213,6 +213,28 @@ int im_decode_stack(im_ctx* ctx, int n_layers, const int32_t* layers, int n_seq,
                     const void* const* x, const void* const* q_pre, const void* const* q, const void* const* k_new,
                     const void* const* v_new, void* const* out, void* cuda_stream);
 
+/*
+ * im_decode_stack for a caller whose per-layer inputs arrive, and whose per-layer outputs leave, while the call runs
+ * (copies from and to host memory on streams of the caller's, say): the same computation (Sec. 4 schedule, decode side;
+ * Eq. 4-7) with one event per layer on either side.
+ *   ready_events     host array of n_layers CUDA events (cudaEvent_t), or NULL; entries may be NULL.  The inputs of
+ *                    layers[j] (x[j], q_pre[j], q[j], k_new[j], v_new[j]) need only be complete once ready_events[j] has
+ *                    occurred: no kernel of the call reads them before.  The caller has recorded the event before
+ *                    the call (with a NULL entry, or a NULL array, the inputs are complete in `cuda_stream` order when
+ *                    the call is made, as for im_decode_stack).
+ *   done_events      host array of n_layers CUDA events, or NULL; entries may be NULL.  The call records
+ *                    done_events[j] on an internal stream once out[j] is complete; a stream of the caller's that waits
+ *                    for it may read out[j] while later layers of the call still run.
+ * The events are the caller's (created, and destroyed after the work has ended, by the caller).  Under stream
+ * capture the ready events must have been recorded on streams of the same capture, and the streams that wait for the
+ * done events must be joined back into the capturing stream by the caller.  Everything else as for im_decode_stack,
+ * which is this call with both arrays NULL.
+ */
+int im_decode_stack_events(im_ctx* ctx, int n_layers, const int32_t* layers, int n_seq, const int32_t* seq_ids,
+                           const void* const* x, const void* const* q_pre, const void* const* q, const void* const* k_new,
+                           const void* const* v_new, void* const* out, void* const* ready_events,
+                           void* const* done_events, void* cuda_stream);
+
 /* Copies one weight tensor of a layer from / to host memory (bytes must equal the tensor size). Synchronous. */
 int im_set_weights(im_ctx* ctx, int layer, int which, const void* host_buf, size_t bytes);
 int im_get_weights(im_ctx* ctx, int layer, int which, void* host_buf, size_t bytes);

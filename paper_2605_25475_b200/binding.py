@@ -55,6 +55,7 @@ _lib.im_prefill_chunk.argtypes = [_vp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp
 _lib.im_prefill_chunk_attend.argtypes = [_vp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.im_decode_step.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.im_decode_stack.argtypes = [_vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.im_decode_stack_events.argtypes = [_vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.im_set_weights.argtypes = [_vp, _i32, _i32, _vp, _sz]
 _lib.im_get_weights.argtypes = [_vp, _i32, _i32, _vp, _sz]
 _lib.im_state_export.argtypes = [_vp, _i32, _i32, _i32, _vp, _sz]
@@ -77,7 +78,8 @@ _lib.im_last_error.restype = C.c_char_p
 EXPORTED = ("im_workspace_bytes", "im_create", "im_destroy", "im_reset", "im_prefill_chunk", "im_decode_step",
             "im_set_weights", "im_get_weights", "im_state_export", "im_state_import", "im_topb_select",
             "im_status", "im_launch_count", "im_get_config", "im_last_error", "im_profile_begin", "im_profile_end", "im_set_option", "im_attention_noalloc", "im_event_count", "im_prefill_chunk_attend",
-            "im_set_scores", "im_state_export_head", "im_state_import_head", "im_decode_stack")
+            "im_set_scores", "im_state_export_head", "im_state_import_head", "im_decode_stack",
+            "im_decode_stack_events")
 
 
 def _check(rc: int):
@@ -150,6 +152,31 @@ def im_decode_stack(ctx, layers, seq_ids, x, q_pre, q, k_new, v_new, out):
     assert all(a.size == lay.size for a in lists)
     _check(_lib.im_decode_stack(ctx, lay.size, lay.ctypes.data, ids.size, ids.ctypes.data, *[a.ctypes.data for a in lists],
                                 _stream()))
+
+
+def _event_handles(events, n):
+    """torch.cuda.Event objects (already recorded once, so that they exist), raw handles or None -> uint64 array."""
+    if events is None:
+        return None
+    assert len(events) == n
+    h = []
+    for e in events:
+        v = 0 if e is None else (e.cuda_event if hasattr(e, "cuda_event") else int(e))
+        if e is not None and not v:
+            raise ValueError("a CUDA event that has never been recorded has no handle yet: record it once first")
+        h.append(v)
+    return np.asarray(h, dtype=np.uint64)
+
+
+def im_decode_stack_events(ctx, layers, seq_ids, x, q_pre, q, k_new, v_new, out, ready_events=None, done_events=None):
+    """im_decode_stack with one event per layer for inputs that arrive and outputs that leave while the call runs."""
+    ids, lay = _ids(seq_ids), _ids(layers)
+    lists = [np.asarray([t.data_ptr() for t in ts], dtype=np.uint64) for ts in (x, q_pre, q, k_new, v_new, out)]
+    assert all(a.size == lay.size for a in lists)
+    rdy, don = _event_handles(ready_events, lay.size), _event_handles(done_events, lay.size)
+    _check(_lib.im_decode_stack_events(ctx, lay.size, lay.ctypes.data, ids.size, ids.ctypes.data,
+                                       *[a.ctypes.data for a in lists], None if rdy is None else rdy.ctypes.data,
+                                       None if don is None else don.ctypes.data, _stream()))
 
 
 def im_set_weights(ctx, layer, which, host: np.ndarray):
@@ -374,8 +401,10 @@ class IndexMem:
         im_decode_step(self.ctx, layer, seq_ids, x, q_pre, q, k_new, v_new, out)
         return out
 
-    def decode_stack(self, layers, seq_ids, x, q_pre, q, k_new, v_new, out=None):
-        """One decode token for every layer of `layers` in one call; x .. v_new (and out) hold one tensor per layer."""
+    def decode_stack(self, layers, seq_ids, x, q_pre, q, k_new, v_new, out=None, ready_events=None, done_events=None):
+        """One decode token for every layer of `layers` in one call; x .. v_new (and out) hold one tensor per layer.
+        ready_events / done_events: one torch.cuda.Event per layer (or None) for inputs that arrive and outputs that are
+        fetched while the call runs (im_decode_stack_events)."""
         n, nl = len(seq_ids), len(layers)
         bf = torch.bfloat16
         for j in range(nl):
@@ -385,7 +414,10 @@ class IndexMem:
             out = torch.empty((nl, n, self.H, self.d), dtype=self.out_dtype, device=self.device)
         for j in range(nl):
             _dev(out[j], self.out_dtype, n * self.D, "out")
-        im_decode_stack(self.ctx, layers, seq_ids, x, q_pre, q, k_new, v_new, out)
+        if ready_events is None and done_events is None:
+            im_decode_stack(self.ctx, layers, seq_ids, x, q_pre, q, k_new, v_new, out)
+        else:
+            im_decode_stack_events(self.ctx, layers, seq_ids, x, q_pre, q, k_new, v_new, out, ready_events, done_events)
         return out
 
     def reset(self, layer=-1, seq=-1):

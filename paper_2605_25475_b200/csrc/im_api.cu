@@ -1396,7 +1396,8 @@ bool stack_bulk_readout(const im_ctx* ctx) {
 // One layer of a pipelined stack call (see im_decode_stack): the kernels of im_decode_step's concurrent schedule with
 // deferred compaction, enqueued on the lane's streams, the call's attention stream and its readout stream.
 int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids, int n_res, const unsigned long long* sm_stream,
-                const void* x, const void* q_pre, const void* q, const void* k_new, const void* v_new, void* out) {
+                const void* x, const void* q_pre, const void* q, const void* k_new, const void* v_new, void* out,
+                cudaEvent_t ready, cudaEvent_t done) {
   const ImDims& p = ctx->p;
   ImCall call;
   int rc = check_call(ctx, layer, n_seq, seq_ids, &call);
@@ -1446,6 +1447,13 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
     CK(cudaStreamWaitEvent(LA.stream, ln.done, 0));
     CK(cudaStreamWaitEvent(LR.stream, ln.done, 0));
   }
+  // The caller's event for this layer's inputs: every stream of the lane that reads them waits for it.  The attention
+  // kernel (launched as a programmatic dependent, and reading q before it waits for anything) is held behind the
+  // lane's first projection instead, an ordinary launch that has waited for the event in full.
+  if (ready) {
+    for (int w = 0; w < 4; ++w) CK(cudaStreamWaitEvent(ln.side[w], ready, 0));
+    CK(cudaStreamWaitEvent(ln.main, ready, 0));
+  }
   // a0: projections.  s1: indexer part (heads the chain that decides the eviction)
   ImRows r = im_rows(p);
   ImGemmArgs g;
@@ -1482,6 +1490,10 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
   // (no shared-memory floors here: in im_decode_step they keep the small kernels' blocks off the SMs of the attention
   // blocks, in a stack call they would keep an attention block off an SM it finds free between two layers)
   CKL(im_launch_gemm(L1, g));
+  if (ready) {
+    CK(cudaEventRecord(ln.ev[10], L1.stream));
+    CK(cudaStreamWaitEvent(LA.stream, ln.ev[10], 0));
+  }
   g.key_W = nullptr;
   // s3: key projection; s4: fold of the pending list
   if (!key_ride) CKL(im_launch_proj_key_split(L3, x, n_seq, call.ksplit_key));
@@ -1547,6 +1559,7 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
   CK(cudaStreamWaitEvent(ln.main, ln.ev[12], 0));
   CK(cudaStreamWaitEvent(ln.main, ln.ev[4], 0));
   CKL(im_launch_attention_merge(L, call, out, call.att_chunks, IM_ATTN_STREAM_TILE, ro_workers, q, k_new, v_new, 0));
+  if (done) CK(cudaEventRecord(done, ln.main));  // the layer's output is complete
   CK(cudaStreamWaitEvent(ln.main, ln.ev[5], 0));
   CK(cudaStreamWaitEvent(ln.main, ln.ev[2], 0));
   CK(cudaEventRecord(ln.done, ln.main));
@@ -1559,6 +1572,13 @@ int stack_layer(im_ctx* ctx, int j, int layer, int n_seq, const int32_t* seq_ids
 extern "C" int im_decode_stack(im_ctx* ctx, int n_layers, const int32_t* layers, int n_seq, const int32_t* seq_ids,
                                const void* const* x, const void* const* q_pre, const void* const* q, const void* const* k_new,
                                const void* const* v_new, void* const* out, void* cuda_stream) {
+  return im_decode_stack_events(ctx, n_layers, layers, n_seq, seq_ids, x, q_pre, q, k_new, v_new, out, nullptr, nullptr, cuda_stream);
+}
+
+extern "C" int im_decode_stack_events(im_ctx* ctx, int n_layers, const int32_t* layers, int n_seq, const int32_t* seq_ids,
+                                      const void* const* x, const void* const* q_pre, const void* const* q,
+                                      const void* const* k_new, const void* const* v_new, void* const* out,
+                                      void* const* ready_events, void* const* done_events, void* cuda_stream) {
   if (!ctx) return fail(IM_ERR_ARG, "null context");
   const ImDims& p = ctx->p;
   if (n_layers < 1 || n_layers > p.L) return fail(IM_ERR_ARG, "n_layers %d out of range [1,%d]", n_layers, p.L);
@@ -1597,9 +1617,11 @@ extern "C" int im_decode_stack(im_ctx* ctx, int n_layers, const int32_t* layers,
   }
   if (!pipe) {
     for (int j = 0; j < n_layers; ++j) {
+      if (ready_events && ready_events[j]) CK(cudaStreamWaitEvent((cudaStream_t)cuda_stream, (cudaEvent_t)ready_events[j], 0));
       const int rc = im_decode_step(ctx, layers[j], n_seq, seq_ids, x ? x[j] : nullptr, q_pre ? q_pre[j] : nullptr, q[j], k_new[j],
                                     v_new[j], out[j], cuda_stream);
       if (rc) return rc;
+      if (done_events && done_events[j]) CK(cudaEventRecord((cudaEvent_t)done_events[j], (cudaStream_t)cuda_stream));
     }
     return IM_OK;
   }
@@ -1630,7 +1652,8 @@ extern "C" int im_decode_stack(im_ctx* ctx, int n_layers, const int32_t* layers,
   CK(cudaStreamWaitEvent(ctx->st_ro, ctx->st_fork, 0));
   for (int k = 0; k < IM_STACK_LANES; ++k) ctx->lane[k].used = false;
   for (int j = 0; j < n_layers; ++j) {
-    const int rc = stack_layer(ctx, j, layers[j], n_seq, seq_ids, n_res, sm_stream, x[j], q_pre[j], q[j], k_new[j], v_new[j], out[j]);
+    const int rc = stack_layer(ctx, j, layers[j], n_seq, seq_ids, n_res, sm_stream, x[j], q_pre[j], q[j], k_new[j], v_new[j], out[j],
+                               ready_events ? (cudaEvent_t)ready_events[j] : nullptr, done_events ? (cudaEvent_t)done_events[j] : nullptr);
     if (rc) return rc;  // (streams forked so far are rejoined by the caller's next synchronisation only: the call has failed)
   }
   CK(cudaEventRecord(ctx->st_attn_done, ctx->st_attn));

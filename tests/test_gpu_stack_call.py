@@ -98,6 +98,75 @@ def test_stack_call_equals_layer_calls_bit_for_bit(tau):
     ga.close(); gb.close()
 
 
+def test_stack_call_with_events_takes_inputs_and_hands_out_outputs_layer_by_layer():
+    """im_decode_stack_events: every layer's inputs are copied from pinned host memory on a copy stream of the test's
+    while the call is being made and runs, one event per layer telling the call when they are complete, and every
+    layer's output is copied back on a third stream behind the call's event for that layer.  Outputs on the host and
+    the state of every unit equal those of im_decode_step calls on resident inputs, bit for bit, through evict steps
+    (the device buffers are overwritten with a poison value before every step: a kernel that read its inputs before
+    their event would see it)."""
+    wl = _stack(n_layers=7, n_seq=6, steps=10)
+    im, (ga, gb), ids, dev = _twin(wl, pending_slots=4)
+    layers = list(range(wl.n_layers))
+    L = wl.n_layers
+    cur = torch.cuda.current_stream(dev)
+    cs, ds = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ready = [torch.cuda.Event() for _ in range(L)]
+    done = [torch.cuda.Event() for _ in range(L)]
+    for e in ready + done:
+        e.record(cur)              # (an event has a handle once it has been recorded)
+    fork, join = torch.cuda.Event(), torch.cuda.Event()
+    x0 = _step_inputs(wl, 0, dev)
+    dbuf = [torch.empty_like(t) for t in x0]
+    hbuf = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in x0]
+    dout = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16, device=dev)
+    hout = torch.empty((L, wl.n_seq, wl.H, wl.d), dtype=torch.bfloat16).pin_memory()
+    for st in range(wl.steps):
+        inp = _step_inputs(wl, st, dev)
+        for h, t in zip(hbuf, inp):
+            h.copy_(t.cpu())
+        for d in dbuf:
+            d.fill_(float("nan"))
+        dout.fill_(float("nan"))
+        hout.fill_(float("nan"))
+        torch.cuda.synchronize(dev)
+        fork.record(cur)
+        cs.wait_event(fork)
+        ds.wait_event(fork)
+        with torch.cuda.stream(cs):
+            for layer in range(L):
+                for d, h in zip(dbuf, hbuf):
+                    d[layer].copy_(h[layer], non_blocking=True)
+                ready[layer].record(cs)
+        oa = gb.decode_stack(layers, ids, *dbuf, out=dout, ready_events=ready, done_events=done)
+        assert oa.data_ptr() == dout.data_ptr()
+        with torch.cuda.stream(ds):
+            for layer in range(L):
+                ds.wait_event(done[layer])
+                hout[layer].copy_(dout[layer], non_blocking=True)
+            join.record(ds)
+        cur.wait_event(join)
+        x, qp, q, k, v = inp
+        ob = torch.stack([ga.decode_step(layer, ids, x[layer], qp[layer], q[layer], k[layer], v[layer]) for layer in layers])
+        torch.cuda.synchronize(dev)
+        assert ga.status() == 0 and gb.status() == 0
+        assert torch.equal(hout.view(torch.int16), ob.cpu().view(torch.int16)), f"step {st}: outputs on the host differ"
+        if st % 3 == 2 or st == wl.steps - 1:
+            _same_state(im, ga, gb, wl, f"step {st}")
+    # without the pipeline the same call runs layer by layer and honours the events in stream order
+    im.im_set_option(gb.ctx, im.IM_OPT_STACK_PIPELINE, 0)
+    inp = _step_inputs(wl, wl.steps, dev)
+    for r in ready:
+        r.record(cur)
+    oa = gb.decode_stack(layers, ids, *inp, ready_events=ready, done_events=done)
+    x, qp, q, k, v = inp
+    ob = torch.stack([ga.decode_step(layer, ids, x[layer], qp[layer], q[layer], k[layer], v[layer]) for layer in layers])
+    done[-1].synchronize()
+    torch.cuda.synchronize(dev)
+    assert torch.equal(oa.view(torch.int16), ob.view(torch.int16))
+    ga.close(); gb.close()
+
+
 def test_stack_call_with_the_bulk_copy_readout_equals_layer_calls():
     """One sequence per call: the bulk-copy readout kernel then cuts a sequence's rows into the same runs in a stack
     call and in a layer call (fewer chunks than blocks in both), so the two agree bit for bit with that kernel too."""
