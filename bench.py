@@ -567,6 +567,37 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device, stack_call=False):
         assert bounds[0] == 0 and bounds[-1] == L and all(b > a for a, b in zip(bounds, bounds[1:]))
     n_groups = max(len(bounds) - 1, 0)
 
+    use_events = bool(stack_call and not getattr(args, "e2e_groups", "") and L >= 2)
+    ev_done = [torch.cuda.Event() for _ in range(L)]
+    if use_events:
+        for e in ev_in + ev_done:
+            e.record(stream)                             # (an event has a handle once it has been recorded)
+        stream.synchronize()
+
+    def enqueue_events(k):
+        """One step made of ONE im_decode_stack_events call: every layer's inputs are copied in on the copy stream with
+        an event behind them that the call makes the layer's kernels wait for, and every layer's output is copied out
+        behind the event the call records for it, while the later layers run."""
+        hb = host[k]
+        ev_fork.record(stream)
+        cs.wait_event(ev_fork)
+        ds.wait_event(ev_fork)
+        with torch.cuda.stream(cs):
+            for layer in range(L):
+                dbuf[layer].copy_(hb[layer], non_blocking=True)
+                tick[layer:layer + 1].fill_(1.0)         # (see below: the calls depend on a kernel, not on the copy node)
+                ev_in[layer].record(cs)
+        g.decode_stack(list(range(L)), ids, dx, dqp, dq, dk, dv, dout, ready_events=ev_in, done_events=ev_done)
+        with torch.cuda.stream(ds):
+            for layer in range(L):
+                ds.wait_event(ev_done[layer])
+                hout[layer].copy_(dout[layer], non_blocking=True)
+            ev_join.record(ds)
+        ev_cs = ev_out[0]
+        ev_cs.record(cs)
+        stream.wait_event(ev_cs)
+        stream.wait_event(ev_join)
+
     def enqueue_groups(k):
         """One step made of stack calls over groups of consecutive layers: the inputs of group g + 1 are copied in and
         the outputs of group g - 1 copied out while the stack call of group g runs."""
@@ -592,6 +623,8 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device, stack_call=False):
     def enqueue(k):
         """One step: the copies of layer l + 1's inputs and of layer l - 1's outputs run next to layer l's
         kernels (three streams, forked from and joined back into `stream`, so that it can be captured)."""
+        if use_events:
+            return enqueue_events(k)
         if n_groups:
             return enqueue_groups(k)
         hb = host[k]
@@ -655,7 +688,9 @@ def run_e2e(args, wl, g, ids, inputs, stream, world, device, stack_call=False):
     ms = max_over_ranks(ev0.elapsed_time(ev1), world, device)
     return {"value": wl.n_seq * args.steps * world / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms / args.steps, "cuda_graph": graphs is not None,
-            "calls_per_step": ("%d im_decode_stack calls over %s layers" % (n_groups, ", ".join(str(bounds[i + 1] - bounds[i]) for i in range(n_groups))))
+            "calls_per_step": ("one im_decode_stack_events call: a ready event per layer behind its input copy, a done event per layer "
+                               "ahead of its output copy") if use_events else
+                              ("%d im_decode_stack calls over %s layers" % (n_groups, ", ".join(str(bounds[i + 1] - bounds[i]) for i in range(n_groups))))
                               if n_groups else "%d im_decode_step calls" % L}
 
 
