@@ -6,6 +6,7 @@ attention, a brute-force sort, closed forms of Eq. 5-7, invariants of the update
 number the paper prints that depends on the layer widths (19.92M indexer parameters).
 """
 import math
+import os
 
 import numpy as np
 import pytest
@@ -75,6 +76,10 @@ def test_indexer_parameter_count_llama31_8b():
     shp = synth.weight_shapes(wl)
     per_layer = math.prod(shp["U_q"]) + math.prod(shp["U_k"]) + math.prod(shp["G"])
     assert 32 * per_layer == 19_922_944          # "19.92M"
+    # the figure as the paper prints it (tests/golden, with its citation)
+    golden = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "indexer_parameters_llama31_8b.txt")
+    printed = [ln.split()[1] for ln in open(golden) if ln.startswith("printed_millions")]
+    assert printed == ["%.2f" % (32 * per_layer / 1e6)]
     L = orc.OracleLayer(orc.OracleConfig(H=32, Hkv=8, d=128, B=8))
     assert L.weight_shapes()["U_q"] == shp["U_q"] == (8 * 16, 4096)
     assert L.weight_shapes()["U_k"] == shp["U_k"] == (16, 4096)
