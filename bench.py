@@ -452,6 +452,8 @@ def run_prefill(args, device):
     if args.context:
         wl = wl.replace(ctx=args.context)
     g, ids = build_context(wl, device, ingest=False, chunk_outputs=1)
+    if getattr(args, "prefill_pipeline", -1) >= 0:
+        im.im_set_option(g.ctx, im.IM_OPT_PREFILL_PIPELINE, args.prefill_pipeline)
     n_chunks = wl.ctx // wl.chunk
     chunks = [synth.prefill_inputs(wl, 0, c, device) for c in range(min(n_chunks, 4))]
     stream = torch.cuda.Stream(device)
@@ -478,6 +480,7 @@ def run_prefill(args, device):
             ev0.record(stream)
             for _ in range(args.steps):
                 one_pass()
+            assert g.status() == 0       # (also joins what the last call left running on the library's own streams)
             ev1.record(stream)
             stream.synchronize()
             ms = ev0.elapsed_time(ev1) / args.steps
@@ -798,6 +801,9 @@ def main():
                     help="0: readout on plain loads; k >= 1: on a ring of k 32 KB bulk copies per CTA (default: the library's choice)")
     ap.add_argument("--stack-call", type=int, default=1,
                     help="1: a step is one im_decode_stack call over all layers (the layers overlap); 0: one im_decode_step call per layer")
+    ap.add_argument("--prefill-pipeline", type=int, default=-1,
+                    help="--mode prefill: 0 = a chunk call leaves only its state update running when it returns; 1 (the library's "
+                         "default) = everything behind its append kernel, so that the next chunk's projections run next to it")
     ap.add_argument("--pending-slots", type=int, default=0,
                     help="length F of the list of rank-one writes folded lazily into M (0: the library's default, 32)")
     ap.add_argument("--e2e-groups", default="",

@@ -336,6 +336,13 @@ int im_profile_end(im_ctx* ctx, double* total_ms, int64_t* n_records);
  *                        the tensor cores (w_p phi_p as three bf16 terms, v_p as stored: exact products, float32 sums); 0:
  *                        by float32 multiply-adds in list order, as for every other shape.  The two differ by rounding
  *                        order only.
+ *   IM_OPT_PREFILL_PIPELINE 1 (default): an im_prefill_chunk call whose every sequence evicts more than pending_slots entries
+ *                        (tensor-core scoring, not under stream capture) returns with everything behind its append kernel
+ *                        still running on a stream of the library's own, so that the next chunk's projections run next to
+ *                        this chunk's scoring, selection and memory write; the next call of the context, whatever it is,
+ *                        orders itself behind that work (a stream of the caller's that reads the state by other means has
+ *                        to make a library call first, im_status for instance).  0: only the state update of the memory
+ *                        write is left running.  Results are the same.
  *   IM_OPT_WAIT_LIMIT    (test aid) attempts of the bounded device-side waits in which a consumer waits for its copies to
  *                        arrive (TMA / bulk-copy rings of the decode attention kernels, the bulk-copy readout kernel and
  *                        the tcgen05 chunk attention kernel): 0 restores the default (2^22), k >= 1 allows k - 1 attempts,
@@ -356,7 +363,8 @@ typedef enum im_option {
   IM_OPT_STACK_PIPELINE = 8,
   IM_OPT_STACK_RESERVED = 9,
   IM_OPT_STACK_CHUNKS = 10,
-  IM_OPT_FOLD_TENSOR = 11
+  IM_OPT_FOLD_TENSOR = 11,
+  IM_OPT_PREFILL_PIPELINE = 12
 } im_option;
 int im_set_option(im_ctx* ctx, int option, int value);
 

@@ -244,7 +244,7 @@ def im_profile_end(ctx):
 
 
 IM_OPT_CONCURRENCY, IM_OPT_PREFETCH_NEXT, IM_OPT_PREFILL_TENSOR, IM_OPT_PROFILE_TARGET, IM_OPT_DECODE_TENSOR, IM_OPT_READOUT_STAGES, IM_OPT_WAIT_LIMIT, IM_OPT_LAYER_OVERLAP = 0, 1, 2, 3, 4, 5, 6, 7
-IM_OPT_STACK_PIPELINE, IM_OPT_STACK_RESERVED, IM_OPT_STACK_CHUNKS, IM_OPT_FOLD_TENSOR = 8, 9, 10, 11
+IM_OPT_STACK_PIPELINE, IM_OPT_STACK_RESERVED, IM_OPT_STACK_CHUNKS, IM_OPT_FOLD_TENSOR, IM_OPT_PREFILL_PIPELINE = 8, 9, 10, 11, 12
 
 
 def im_set_option(ctx, option: int, value: int):

@@ -287,6 +287,15 @@ struct im_ctx {
   cudaStream_t late = nullptr;
   cudaEvent_t ev_late = nullptr, ev_phi = nullptr;
   bool late_pending = false;
+  // Such a call also leaves everything behind its append kernel (scoring, commit, selection, gather, hole filling, phi
+  // of the evicted keys) running on `pf_tail` when it returns, so that the NEXT chunk's projections, which read the
+  // caller's inputs and write scratch that only the append kernel reads, run next to it.  The next prefill call waits
+  // for `ev_cache` (cache and counters final) before its fold and append kernels and for `ev_late` before its commit
+  // kernel; every other call waits for `ev_late`, which is recorded behind all of it.  (IM_OPT_PREFILL_PIPELINE.)
+  cudaStream_t pf_tail = nullptr;
+  cudaEvent_t ev_cache = nullptr, ev_app = nullptr;
+  bool cache_pending = false;
+  bool prefill_pipeline = true;
   // Pipelined stack calls (im_decode_stack): the attention kernels of the call's layers follow one another on
   // `st_attn`, the readout kernels on `st_ro`; everything else of layer j runs on the streams of lane j %
   // IM_STACK_LANES (main: merge; side: the four chains of a decode call), with the lane's events and scratch set.
@@ -328,6 +337,7 @@ ImLaunch make_launch(im_ctx* ctx, int layer, cudaStream_t s) {
 
 // makes `s` wait for a state update that an earlier prefill call left running (see im_ctx::late)
 cudaError_t join_late(im_ctx* ctx, cudaStream_t s) {
+  ctx->cache_pending = false;  // (ev_late is recorded behind everything ev_cache covers)
   if (!ctx->late_pending) return cudaSuccess;
   ctx->late_pending = false;
   return cudaStreamWaitEvent(s, ctx->ev_late, 0);
@@ -407,7 +417,7 @@ cudaError_t launch_mem_update(im_ctx* ctx, const ImLaunch& L, const ImCall& call
 // With `update` = false only the GEMM is launched (the caller launches im_launch_mem_update later).
 // `before_update`: an event that the kernels changing the memory state wait for (a reader of the state of before)
 int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, bool update = true, int smem_floor = 0,
-                     cudaEvent_t before_update = nullptr, int programmatic = 0) {
+                     cudaEvent_t before_update = nullptr, int programmatic = 0, bool own_partials = true) {
   const ImDims& p = ctx->p;
   ImGemmArgs g;
   memset(&g, 0, sizeof(g));
@@ -431,7 +441,8 @@ int run_memory_write(im_ctx* ctx, const ImLaunch& L, ImCall& call, int ne_max, b
     g.ks_stride = 0;
     // a prefill chunk's few output tiles: two CTAs per tile over the K range, where the partial buffers have room
     const long long extent = (long long)call.n_seq * p.tail * p.dM;
-    if (call.prefill && (p.Dkv / 64) % 2 == 0 && 2 * extent <= (long long)IM_TC_KSPLIT * L.sc.gpart_vecs * p.R3) {
+    // (not while the next chunk's projections may be writing those buffers)
+    if (own_partials && call.prefill && (p.Dkv / 64) % 2 == 0 && 2 * extent <= (long long)IM_TC_KSPLIT * L.sc.gpart_vecs * p.R3) {
       g.tc_ksplit = 2;
       g.part = L.sc.gpart;
       g.part_stride = extent;
@@ -705,6 +716,9 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
   }
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_late, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_phi, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->pf_tail, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_cache, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_app, cudaEventDisableTiming);
   ctx->concurrent = ctx->fast_attn;
   if (e == cudaSuccess && ctx->fast_attn && !p.scorer) {
     // streams, events and the SM ids of pipelined stack calls
@@ -741,6 +755,9 @@ int im_create(const im_config* cfg, void* dev_workspace, size_t workspace_bytes,
     if (ctx->late) cudaStreamDestroy(ctx->late);
     if (ctx->ev_late) cudaEventDestroy(ctx->ev_late);
     if (ctx->ev_phi) cudaEventDestroy(ctx->ev_phi);
+    if (ctx->pf_tail) cudaStreamDestroy(ctx->pf_tail);
+    if (ctx->ev_cache) cudaEventDestroy(ctx->ev_cache);
+    if (ctx->ev_app) cudaEventDestroy(ctx->ev_app);
     delete ctx;
     return fail(IM_ERR_CUDA, "im_create: %s", cudaGetErrorString(e));
   }
@@ -757,6 +774,9 @@ int im_destroy(im_ctx* ctx) {
   if (ctx->late) cudaStreamDestroy(ctx->late);
   if (ctx->ev_late) cudaEventDestroy(ctx->ev_late);
   if (ctx->ev_phi) cudaEventDestroy(ctx->ev_phi);
+  if (ctx->pf_tail) cudaStreamDestroy(ctx->pf_tail);
+  if (ctx->ev_cache) cudaEventDestroy(ctx->ev_cache);
+  if (ctx->ev_app) cudaEventDestroy(ctx->ev_app);
   delete ctx;
   if (e != cudaSuccess) return fail(IM_ERR_CUDA, "im_destroy: %s", cudaGetErrorString(e));
   return IM_OK;
@@ -853,8 +873,20 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   // its commit kernel.  A call with outputs reads the memory early: it waits at once.
   if (attend || !ctx->concurrent) CK(join_late(ctx, L.stream));
   const int NV = n_seq * chunk_len;
-  // pending rank-one terms are folded into M before a compression that cannot append to the list
-  if (p.mem && (ne_max > 0 || attend)) CKL(im_launch_mem_fold(L, call));
+  // Is everything behind the append kernel left running when the call returns (im_ctx::pf_tail)?  Calls whose every
+  // sequence evicts more than the pending list holds (their state update is left running anyway), with the scoring on
+  // the tensor cores (the other scoring kernel reads the projections' scratch), not under stream capture.
+  bool pipe_tail = ctx->prefill_pipeline && ctx->concurrent && !attend && !follow && p.mem && call.pack && ne_max > p.F;
+  for (int i = 0; i < n_seq && pipe_tail; ++i)
+    pipe_tail = ctx->hu[(size_t)layer * p.S + call.seq[i]].n + chunk_len - p.B > p.F;
+  if (pipe_tail) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(L.stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) pipe_tail = false;
+  }
+  // pending rank-one terms are folded into M before a compression that cannot append to the list (behind the previous
+  // call's tail where that is still running: the fold kernels read the counters it leaves)
+  const bool fold_behind = ctx->cache_pending;
+  if (!fold_behind && p.mem && (ne_max > 0 || attend)) CKL(im_launch_mem_fold(L, call));
   // a0: indexer projections of every chunk token (Sec. 3.1)
   ImRows r = im_rows(p);
   ImGemmArgs g;
@@ -929,7 +961,19 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
     CK(cudaStreamWaitEvent(L.stream, ctx->ev[1], 0));
     CK(cudaStreamWaitEvent(L.stream, ctx->ev[2], 0));
   }
+  if (ctx->cache_pending) {  // the previous call's tail: cache compacted, counters final
+    CK(cudaStreamWaitEvent(L.stream, ctx->ev_cache, 0));
+    ctx->cache_pending = false;
+  }
+  if (fold_behind && p.mem && (ne_max > 0 || attend)) CKL(im_launch_mem_fold(L, call));
   CKL(im_launch_prefill_append(L, call, k, v));
+  // the rest of the call: on the caller's stream, or on a stream of the library's own that the call leaves running
+  ImLaunch T = L;
+  if (pipe_tail) {
+    CK(cudaEventRecord(ctx->ev_app, L.stream));
+    T.stream = ctx->pf_tail;
+    CK(cudaStreamWaitEvent(T.stream, ctx->ev_app, 0));
+  }
   if (attend) {
     // Layer outputs of the chunk's own queries, before the chunk is compressed: Eq. 5 over the memory of before
     // this chunk, then attention over (cached entries + causal chunk) with the readout added (Eq. 4).  They read the
@@ -959,31 +1003,35 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
   // a1: pooled importance under the causal mask
   {
     const bool prof = ctx->prof_target == 1 && ctx->prof_used + 2 <= ctx->prof_ev.size();
-    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], L.stream));
+    if (prof) CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used], T.stream));
     if (follow) {}  // the scores come from the leading layer, after the commit below
-    else if (call.pack) CKL(im_launch_prefill_score_tc(L, call, n_max, ctx->n_sm));
-    else CKL(im_launch_prefill_score(L, call, n_max));
+    else if (call.pack) CKL(im_launch_prefill_score_tc(T, call, n_max, ctx->n_sm));
+    else CKL(im_launch_prefill_score(T, call, n_max));
     if (prof) {
-      CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], L.stream));
+      CK(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], T.stream));
       ctx->prof_used += 2;
     }
   }
-  CK(join_late(ctx, L.stream));
-  CKL(im_launch_prefill_commit(L, call));
-  if (follow) CKL(im_launch_follow_scores(L, call));
+  CK(join_late(ctx, T.stream));
+  CKL(im_launch_prefill_commit(T, call));
+  if (follow) CKL(im_launch_follow_scores(T, call));
   // a2: selection (also restarts the pooling); a4: gather the evicted pairs, fill the holes
-  CKL(im_launch_select(L, call));
+  CKL(im_launch_select(T, call));
   if (ne_max > 0) {
     if (fork && p.mem) {
       // the holes are filled next to the memory write, which works from the gathered copies
-      ImLaunch Lm = L;
-      Lm.stream = ctx->side[0];
-      CKL(im_launch_gather(L, call, ne_max));
-      CK(cudaEventRecord(ctx->ev[5], L.stream));
+      ImLaunch Lm = T;
+      Lm.stream = pipe_tail ? ctx->side[2] : ctx->side[0];  // (side[0] may already run the next call's projections)
+      CKL(im_launch_gather(T, call, ne_max));
+      CK(cudaEventRecord(ctx->ev[5], T.stream));
       CK(cudaStreamWaitEvent(Lm.stream, ctx->ev[5], 0));
       if (attend) CK(cudaStreamWaitEvent(Lm.stream, ctx->ev[9], 0));  // the chunk attention reads the slots that are filled
       CKL(im_launch_move(Lm, call, ne_max));
       CK(cudaEventRecord(ctx->ev[6], Lm.stream));
+      if (pipe_tail) {
+        CK(cudaEventRecord(ctx->ev_cache, Lm.stream));
+        ctx->cache_pending = true;
+      }
       // a3.  When every sequence of the call evicts more than the pending list holds, the state update runs on a
       // stream of its own behind phi of the evicted keys and is left running (im_ctx::late); not under stream capture,
       // which every stream that was forked has to rejoin
@@ -995,23 +1043,24 @@ static int prefill_impl(im_ctx* ctx, int layer, int n_seq, const int32_t* seq_id
         if (cudaStreamIsCapturing(L.stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) late = false;
       }
       if (late) {
-        if ((rc = run_memory_write(ctx, L, call, ne_max, false))) return rc;  // phi of the evicted keys
-        CK(cudaEventRecord(ctx->ev_phi, L.stream));
-        ImLaunch Ll = L;
+        if ((rc = run_memory_write(ctx, T, call, ne_max, false, 0, nullptr, 0, !pipe_tail))) return rc;  // phi of the evicted keys
+        CK(cudaEventRecord(ctx->ev_phi, T.stream));
+        ImLaunch Ll = T;
         Ll.stream = ctx->late;
         CK(cudaStreamWaitEvent(Ll.stream, ctx->ev_phi, 0));
+        if (pipe_tail) CK(cudaStreamWaitEvent(Ll.stream, ctx->ev[6], 0));  // ev_late stands for all the call has left running
         CKL(launch_mem_update(ctx, Ll, call, ne_max));
         CK(cudaEventRecord(ctx->ev_late, Ll.stream));
         ctx->late_pending = true;
-      } else if ((rc = run_memory_write(ctx, L, call, ne_max, true, 0, memside ? ctx->ev[8] : nullptr))) {
+      } else if ((rc = run_memory_write(ctx, T, call, ne_max, true, 0, memside ? ctx->ev[8] : nullptr))) {
         return rc;
       }
-      CK(cudaStreamWaitEvent(L.stream, ctx->ev[6], 0));
+      CK(cudaStreamWaitEvent(T.stream, ctx->ev[6], 0));
     } else {
-      if (attend && fork) CK(cudaStreamWaitEvent(L.stream, ctx->ev[9], 0));  // the chunk attention reads the cache
-      CKL(im_launch_gather_move(L, call, ne_max));
+      if (attend && fork) CK(cudaStreamWaitEvent(T.stream, ctx->ev[9], 0));  // the chunk attention reads the cache
+      CKL(im_launch_gather_move(T, call, ne_max));
       // a3: memory write
-      if (p.mem && (rc = run_memory_write(ctx, L, call, ne_max))) return rc;
+      if (p.mem && (rc = run_memory_write(ctx, T, call, ne_max))) return rc;
     }
   }
   if (attend && fork) CK(cudaStreamWaitEvent(L.stream, ctx->ev[9], 0));  // join (also when nothing was evicted)
@@ -1698,6 +1747,7 @@ int im_set_option(im_ctx* ctx, int option, int value) {
     case IM_OPT_LAYER_OVERLAP: ctx->layer_overlap = value != 0; return IM_OK;
     case IM_OPT_STACK_PIPELINE: ctx->stack_pipeline = value != 0; return IM_OK;
     case IM_OPT_FOLD_TENSOR: ctx->fold_tensor = value != 0; return IM_OK;
+    case IM_OPT_PREFILL_PIPELINE: ctx->prefill_pipeline = value != 0; return IM_OK;
     case IM_OPT_STACK_CHUNKS:
       if (value < 1 || value > 16) return fail(IM_ERR_ARG, "runs per warp %d out of range [1,16]", value);
       ctx->stack_chunks = value;

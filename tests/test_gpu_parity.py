@@ -210,6 +210,53 @@ def test_fold_on_the_tensor_cores_differs_from_the_ffma_fold_by_rounding_only(im
         assert pt.stats["max_M_err"] <= 2e-3 and pf.stats["max_M_err"] <= 2e-3
 
 
+def test_prefill_calls_that_leave_their_tail_running_equal_calls_that_do_not(im):
+    """IM_OPT_PREFILL_PIPELINE: chunk calls that return with scoring, selection, gather and memory write still running
+    on the library's own streams (the next chunk's projections run next to them) leave every piece of the state, bit
+    for bit, as calls that leave only the state update running, chunk after chunk (each export joins the streams), for
+    two layers called in turn, and the decode steps that follow give the same outputs; both follow the oracle."""
+    wl = synth.CONFIGS["llama8b_b1"].replace(name="pftail", n_seq=2, ctx=6 * 256, chunk=256, B=128, steps=3, n_needles=0)
+    dev = torch.device("cuda:0")
+    cfg = dict(n_layers=2, max_seqs=wl.n_seq, n_q_heads=wl.H, n_kv_heads=wl.Hkv, head_dim=wl.d, budget=wl.B,
+               compress_interval=1, max_chunk=wl.chunk, n_sink=wl.n_sink, lambda_=0.98, eta=0.8)
+    gs = [im.IndexMem(im.Config(**cfg), dev) for _ in range(2)]
+    im.im_set_option(gs[1].ctx, im.IM_OPT_PREFILL_PIPELINE, 0)
+    ids = list(range(wl.n_seq))
+    for layer in range(2):
+        w = synth.make_weights(wl, layer)
+        for g in gs:
+            g.set_weights(layer, w)
+    pieces = (im.IM_S_POS, im.IM_S_IMP, im.IM_S_KIDX, im.IM_S_K, im.IM_S_V, im.IM_S_M, im.IM_S_B)
+    for c in range(wl.ctx // wl.chunk):
+        ins = [synth.prefill_inputs(wl, layer, c, dev) for layer in range(2)]
+        for g in gs:
+            for layer in range(2):
+                X, Qp, _, K, V = ins[layer]
+                g.prefill_chunk(layer, ids, X, Qp, K, V)
+        if c % 2 == 1 or c == wl.ctx // wl.chunk - 1:
+            for layer in range(2):
+                for q in ids:
+                    assert gs[0].counts(layer, q) == gs[1].counts(layer, q)
+                    for piece in pieces:
+                        assert np.array_equal(gs[0].export(layer, q, piece), gs[1].export(layer, q, piece)), (c, layer, q, piece)
+    for st in range(wl.steps):
+        for layer in range(2):
+            x, qp, q, k, v = synth.decode_inputs(wl, layer, st, dev)
+            oa = gs[0].decode_step(layer, ids, x, qp, q, k, v)
+            ob = gs[1].decode_step(layer, ids, x, qp, q, k, v)
+            assert torch.equal(oa, ob)
+    assert gs[0].status() == 0 and gs[1].status() == 0
+    for g in gs:
+        g.close()
+    # and against the oracle, through the usual pair (pipelined by default)
+    p = _pair(wl, lambda_=0.98, eta=0.8)
+    for c in range(wl.ctx // wl.chunk):
+        p.prefill(c)
+    for s_ in range(wl.steps):
+        p.decode(s_)
+    assert p.stats["max_M_err"] <= 2e-3 and p.stats["max_out_err"] <= 2e-3
+
+
 def test_interval_pooling_tau():
     """tau = 8: scores pooled by max over the interval's queries, 8 entries evicted at once."""
     wl = TINY.replace(name="tau8", ctx=200, chunk=200, B=96, steps=24, tau=8, n_needles=2)
