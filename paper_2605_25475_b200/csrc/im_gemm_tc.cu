@@ -430,13 +430,30 @@ bool encode_rows_map(CUtensorMap* m, const void* base, long long rows, long long
     enc = (EncodeTiledFn)fn;
   }
   if (((uintptr_t)base & 15) || (stride * 2) % 16 || rows < 1) return false;
+  // A map is a function of (base, rows, K, stride) alone, and a chunked prefill asks for the same dozen again in every
+  // call (weights; the caller's input buffers where it reuses them): the last few are kept per host thread.
+  struct Memo { const void* base; long long rows, K, stride; CUtensorMap map; };
+  constexpr int N_MEMO = 32;
+  thread_local Memo memo[N_MEMO];
+  thread_local int n_memo = 0, next_memo = 0;
+  for (int k = 0; k < n_memo; ++k)
+    if (memo[k].base == base && memo[k].rows == rows && memo[k].K == K && memo[k].stride == stride) {
+      *m = memo[k].map;
+      return true;
+    }
   const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)stride * 2};
   const cuuint32_t box[2] = {(cuuint32_t)GK, (cuuint32_t)GM};
   const cuuint32_t estr[2] = {1, 1};
-  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  Memo& e = memo[next_memo];
+  e.base = base; e.rows = rows; e.K = K; e.stride = stride; e.map = *m;
+  next_memo = (next_memo + 1) % N_MEMO;
+  if (n_memo < N_MEMO) ++n_memo;
+  return true;
 }
 
 }  // namespace
