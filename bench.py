@@ -391,7 +391,7 @@ def secondary_block(args, device, log):
         log(f"secondary {name}: {sec * 1e6:.1f} us/step")
     # configuration 4: chunked prefill
     pre_args = argparse.Namespace(**vars(args))
-    pre_args.steps, pre_args.warmup, pre_args.context = 2, 3, 0
+    pre_args.steps, pre_args.warmup, pre_args.context = 8, 3, 0
     pf = run_prefill(pre_args, device)
     wl4 = synth.CONFIGS["mistral7b_prefill"]
     out["mistral7b_prefill"] = {
