@@ -14,7 +14,8 @@
  *   - The two hot calls only enqueue kernels on `cuda_stream` (a cudaStream_t passed as void*, NULL =
  *     the legacy default stream) and return without synchronising; they allocate nothing.  All calls
  *     on one context must be issued in stream order on one stream at a time.  A prefill call may leave the last
- *     part of its work (the state update of its memory write) running on a stream of the context's own when it
+ *     part of its work (everything behind the kernel that appends the chunk, or the state update of its memory
+ *     write alone: IM_OPT_PREFILL_PIPELINE) running on streams of the context's own when it
  *     returns; every later call on the context orders itself behind that work, and im_destroy synchronises the
  *     device, so the caller sees no difference as long as the workspace is touched through this interface only
  *     (under stream capture nothing is left running: a capture has to end with every stream rejoined).
